@@ -1,0 +1,188 @@
+/*
+ * kvm.h -- C ABI of the Key-Value Means (KVM) attention layer for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the sequence-mixing hot path of the paper
+ * "Key-Value Means: Transformers with Expandable Block-Recurrent Compressed
+ * Memory" (Section 3 "Method", Appendix B "Pseudocode"): for every block (chunk)
+ * of the sequence one softmax attention over [compressed state ; exact block
+ * sliding window], then the fold of the block that leaves the window into the
+ * state (append / merge / value-radius preservation under a state budget), and
+ * the matching single-token decode step.
+ *
+ * Conventions
+ *   - All tensors named "device" are CUDA device pointers owned by the caller;
+ *     the library never frees or keeps them beyond the call.  Element type of
+ *     q/k/v/out is bfloat16.  Layout is [batch, heads, tokens, head_dim] with
+ *     optional element strides (head_dim stride must be 1).
+ *   - The state object and every scratch buffer are owned by the library and are
+ *     allocated once in kvm_state_create(); no call on the hot path allocates.
+ *   - Work is enqueued on the given CUDA stream (a cudaStream_t passed as
+ *     void*; NULL = default stream).  No entry point synchronises the host with
+ *     the device except kvm_state_export / kvm_debug_assignments (which copy to
+ *     host memory) and the *_host convenience variants.
+ *   - Host-side validation happens before any launch; a failed call leaves the
+ *     state untouched.  There is no CPU fallback: without a CUDA device
+ *     kvm_state_create() returns KVM_ERR_CUDA.
+ *   - Results are deterministic (bitwise identical from run to run).
+ *
+ * Notation (Section 3.2): C = block (chunk_len), w = n_bswa_chunks, L = w*C,
+ * r = rope_dims, S = sink_len, m = current number of state rows, d = head_dim.
+ */
+#ifndef KVM_H_
+#define KVM_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct kvm_state kvm_state_t; /* opaque, library-owned */
+
+typedef enum {
+  KVM_OK = 0,
+  KVM_ERR_INVALID_ARG = 1,    /* null pointer, bad shape, bad stride ...                 */
+  KVM_ERR_UNSUPPORTED = 2,    /* legal in the paper, not built (e.g. head_dim 96)         */
+  KVM_ERR_OOM = 3,            /* device allocation failed in kvm_state_create             */
+  KVM_ERR_CUDA = 4,           /* a CUDA runtime call failed / no device                   */
+  KVM_ERR_STATE_MISMATCH = 5, /* block / growth / rope_dims differ from the first call    */
+  KVM_ERR_CAPACITY = 6,       /* the call would exceed max_state_slots / max_call_tokens  */
+  KVM_ERR_TIMEOUT = 7         /* a bounded device-side wait expired (status word)         */
+} kvm_status_t;
+
+/* State budget B(e) of Section 3.2 ("We choose n_append as follows"):
+ *   FIXED      B(e) = fixed_slots                        ("KVM 256")
+ *   SQRT       B(e) = floor(sqrt_coeff * sqrt(e))        ("KVM sqrt", coeff 16), exact integer
+ *   UNBOUNDED  B(e) = infinity (every overflow token is appended; test limit in
+ *              which the layer never compresses)                                 */
+typedef enum { KVM_GROWTH_FIXED = 0, KVM_GROWTH_SQRT = 1, KVM_GROWTH_UNBOUNDED = 2 } kvm_growth_kind_t;
+
+typedef struct {
+  int32_t kind;        /* kvm_growth_kind_t */
+  int32_t sqrt_coeff;  /* SQRT only; the paper uses 16 */
+  int64_t fixed_slots; /* FIXED only; values below the block are clamped up by the rule itself */
+} kvm_growth_t;
+
+/* Element strides for dims (batch, head, token, channel); channel stride must be 1. */
+typedef struct { int64_t q[4], k[4], v[4], out[4]; } kvm_strides_t;
+
+enum {
+  KVM_FLAG_NO_RADIUS = 1u << 0,      /* ablation "no v-len normalization": read s^V out unnormalised */
+  KVM_FLAG_RECORD_ASSIGN = 1u << 1,  /* keep per-token slot ids / append flags for kvm_debug_assignments */
+  KVM_FLAG_SIMT_ATTENTION = 1u << 2, /* use the scalar-core attention kernel (cross-check path) */
+  KVM_FLAG_SIMT_ROUTING = 1u << 3    /* use the scalar-core routing filter (cross-check path)   */
+};
+
+typedef struct {
+  int32_t batch, n_q_heads, n_kv_heads, head_dim; /* head_dim in {64,128}; n_q_heads % n_kv_heads == 0 */
+  int32_t n_bswa_chunks;                           /* w, the paper uses 2 (Section 4)                    */
+  int32_t sink_len;                                /* S, the paper uses 1 (Section 3.2 "Merge")           */
+  float rope_base;                                 /* 10000 (Appendix D)                                  */
+  float ln_eps;                                    /* LayerNorm epsilon of LN_s, 1e-5                     */
+  float norm_eps;                                  /* epsilon_norm of the value readout, 1e-12            */
+  const float* ln_weight;                          /* host [n_kv_heads, head_dim] or NULL = 1 (copied)    */
+  const float* ln_bias;                            /* host [n_kv_heads, head_dim] or NULL = 0 (copied)    */
+  const float* tau_state;                          /* host [n_q_heads] or NULL = 1 (copied)               */
+  const float* tau_bswa;                           /* host [n_q_heads] or NULL = 1 (copied)               */
+  int32_t max_block;                               /* largest block C that will be used (<= 256)          */
+  int64_t max_state_slots;                         /* capacity in state rows (see kvm_plan_capacity)      */
+  int64_t max_call_tokens;                         /* largest n_tokens of one kvm_prefill call            */
+  int64_t max_seq_len;                             /* only used with KVM_FLAG_RECORD_ASSIGN               */
+  int32_t device;                                  /* CUDA device ordinal                                 */
+  uint32_t flags;
+} kvm_config_t;
+
+/* Rows a state needs after `seq_len` tokens under (block, growth): the closed form of
+ * the budget rule M* = max(m, min(B(e), m + C)) iterated over the folds.  Pure host
+ * arithmetic; returns -1 on invalid arguments. */
+int64_t kvm_plan_capacity(int32_t block, int32_t n_bswa_chunks, kvm_growth_t growth, int64_t seq_len);
+
+/* Creates an empty state (position 0, m = 0) and allocates every buffer on
+ * cfg->device.  Section 3.2 "Terminology": the state holds, per (batch, kv head), the
+ * rows (s^K_i, s^V_i, rho_i) plus the uncompressed BSWA window.
+ * Errors: INVALID_ARG, UNSUPPORTED, OOM, CUDA.  *out is set only on KVM_OK. */
+kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out);
+
+/* Chunk-wise prefill of n_tokens further tokens (Section 3.2 "Chunks and attention
+ * regions", "Readout", "Append", "Merge"; budget rule; Appendix B).
+ *   q      device bf16 [B, Hq,  n_tokens, d]   raw (un-rotated) queries
+ *   k, v   device bf16 [B, Hkv, n_tokens, d]   raw keys, values
+ *   block  C; growth B(e); rope_dims r (even, <= d; first r channels get RoPE with
+ *          half-split pairs (i, i + r/2), angle t * base^(-2i/r), position t absolute)
+ *   gate   device fp32 [B, Hkv, n_tokens] merge gate g_t (Eq. 2) or NULL = 1
+ *   out    device bf16 [B, Hq, n_tokens, d]    per-head attention outputs y_t
+ *   strides NULL = contiguous; otherwise element strides per tensor
+ * Resumable: tokens continue at the state's position; block, growth and rope_dims are
+ * fixed by the first call (later mismatch -> STATE_MISMATCH).  Any n_tokens in
+ * [1, max_call_tokens] is legal; a partial last block waits in the window and is
+ * folded once later tokens (prefill or decode) complete it.  A fold happens right
+ * after the block ending at e was attended, for every complete block.
+ * Errors: INVALID_ARG, UNSUPPORTED, STATE_MISMATCH, CAPACITY, CUDA. */
+kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kvm_state_t* state,
+                         int32_t block, kvm_growth_t growth, int32_t rope_dims,
+                         int64_t n_tokens, const float* gate, void* out,
+                         const kvm_strides_t* strides, void* cuda_stream);
+
+/* One decode token per sequence (Table 1 "Decode time per token"): rotates q,k at the
+ * state's position, pushes k,v into the window, attends over [state ; window], and
+ * folds the overflow block when the token completes a block.
+ *   q device bf16 [B, Hq, d]; k, v device bf16 [B, Hkv, d]; gate device fp32 [B, Hkv] or NULL
+ *   out device bf16 [B, Hq, d]
+ * Requires a state whose block/growth/rope_dims were fixed by a prefill call.
+ * Errors: INVALID_ARG, STATE_MISMATCH, CAPACITY, CUDA. */
+kvm_status_t kvm_decode_step(const void* q, const void* k, const void* v, kvm_state_t* state,
+                             const float* gate, void* out, void* cuda_stream);
+
+/* Same operations with HOST buffers (contiguous layouts as above): the call copies the
+ * inputs to library-owned device staging, runs the path, copies `out` back and
+ * synchronises the stream before returning.  n_tokens <= max_call_tokens. */
+kvm_status_t kvm_prefill_host(const void* q_host, const void* k_host, const void* v_host,
+                              kvm_state_t* state, int32_t block, kvm_growth_t growth,
+                              int32_t rope_dims, int64_t n_tokens, const float* gate_host,
+                              void* out_host, void* cuda_stream);
+kvm_status_t kvm_decode_step_host(const void* q_host, const void* k_host, const void* v_host,
+                                  kvm_state_t* state, const float* gate_host, void* out_host,
+                                  void* cuda_stream);
+
+/* Frees the state and all device memory it owns.  NULL is accepted. */
+kvm_status_t kvm_state_free(kvm_state_t* state);
+
+/* Host-side bookkeeping (no device access): rows m, tokens consumed, folds done.
+ * Any output pointer may be NULL.  m depends only on (position, block, growth), never
+ * on data (budget rule), so it is the same for every (batch, head). */
+kvm_status_t kvm_state_info(const kvm_state_t* state, int64_t* n_slots, int64_t* position,
+                            int64_t* n_folds);
+
+/* Reads the device status word (set by bounded device-side waits or debug index checks)
+ * after synchronising the stream: KVM_OK, KVM_ERR_TIMEOUT or KVM_ERR_CUDA. */
+kvm_status_t kvm_state_check(kvm_state_t* state, void* cuda_stream);
+
+/* Copies the state rows to HOST arrays (synchronises the stream).  Shapes, with
+ * U = batch * n_kv_heads and m = n_slots:
+ *   sum_k   double [U, m, d]  running key sums   s^K   (Section 3.2 "Merge")
+ *   sum_v   float  [U, m, d]  running value sums s^V
+ *   radius  float  [U, m]     rho_i, set when the row was created
+ *   weight  double [U, m]     1 + sum of merge gates of the row (means = sum / weight)
+ *   count   int32  [U, m]     number of tokens in the row
+ *   k_read  bf16   [U, m, d]  readout cache LN_s(s^K)   (may be NULL)
+ *   v_read  bf16   [U, m, d]  readout cache rho * s^V / max(||s^V||, eps) (may be NULL)
+ * Any pointer may be NULL to skip that array. */
+kvm_status_t kvm_state_export(kvm_state_t* state, double* sum_k, float* sum_v, float* radius,
+                              double* weight, int32_t* count, void* k_read, void* v_read,
+                              void* cuda_stream);
+
+/* With KVM_FLAG_RECORD_ASSIGN: copies, for tokens [0, n) (n <= position, n <= max_seq_len),
+ * slot_of_token int32 [U, n] (row merged into / appended as; -1 = not folded yet) and
+ * was_appended uint8 [U, n] to HOST arrays (synchronises the stream). */
+kvm_status_t kvm_debug_assignments(kvm_state_t* state, int64_t n, int32_t* slot_of_token,
+                                   uint8_t* was_appended, void* cuda_stream);
+
+/* Number of kernels the library has launched for this state so far (host counter). */
+int64_t kvm_launch_count(const kvm_state_t* state);
+
+const char* kvm_status_string(kvm_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVM_H_ */
