@@ -23,6 +23,9 @@
  *   - Host-side validation happens before any launch; a failed call leaves the
  *     state untouched.  There is no CPU fallback: without a CUDA device
  *     kvm_state_create() returns KVM_ERR_CUDA.
+ *   - Inside the library bf16 inputs are carried as fp16 (tensor-core operands, readout
+ *     cache, softmax weights): every bf16 value with 2^-14 <= |x| <= 65504 converts exactly,
+ *     larger magnitudes saturate at +-65504.  Accumulation is fp32; routing decisions fp64.
  *   - Results are deterministic (bitwise identical from run to run).
  *
  * Notation (Section 3.2): C = block (chunk_len), w = n_bswa_chunks, L = w*C,
@@ -164,8 +167,8 @@ kvm_status_t kvm_state_check(kvm_state_t* state, void* cuda_stream);
  *   radius  float  [U, m]     rho_i, set when the row was created
  *   weight  double [U, m]     1 + sum of merge gates of the row (means = sum / weight)
  *   count   int32  [U, m]     number of tokens in the row
- *   k_read  bf16   [U, m, d]  readout cache LN_s(s^K)   (may be NULL)
- *   v_read  bf16   [U, m, d]  readout cache rho * s^V / max(||s^V||, eps) (may be NULL)
+ *   k_read  fp16   [U, m, d]  readout cache LN_s(s^K)   (may be NULL)
+ *   v_read  fp16   [U, m, d]  readout cache rho * s^V / max(||s^V||, eps) (may be NULL)
  * Any pointer may be NULL to skip that array. */
 kvm_status_t kvm_state_export(kvm_state_t* state, double* sum_k, float* sum_v, float* radius,
                               double* weight, int32_t* count, void* k_read, void* v_read,

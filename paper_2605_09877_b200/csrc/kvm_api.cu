@@ -1,0 +1,496 @@
+// extern "C" entry points of libkvm (declared in include/kvm.h) and the host-side chunk loop.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "kvm_internal.h"
+
+using namespace kvm;
+
+struct kvm_state {
+  State s;
+  std::vector<void*> allocs;
+  bool host_staging = false;
+};
+
+namespace {
+
+uint64_t isqrt_u64(uint64_t x) {
+  uint64_t r = (uint64_t)sqrt((double)x);
+  while (r * r > x) --r;
+  while ((r + 1) * (r + 1) <= x) ++r;
+  return r;
+}
+
+// State budget B(e) (Section 3.2, budget rule; "16 sqrt(N)" and "KVM 256" of Section 4).
+int64_t budget(const kvm_growth_t& g, int64_t e) {
+  if (g.kind == KVM_GROWTH_FIXED) return g.fixed_slots;
+  if (g.kind == KVM_GROWTH_SQRT) return (int64_t)isqrt_u64((uint64_t)g.sqrt_coeff * (uint64_t)g.sqrt_coeff * (uint64_t)e);
+  return INT64_MAX / 4;
+}
+
+// n_append = min(M* - m, |Omega|), M* = max(m, min(B(e), m + C)).
+int64_t n_append_of(const kvm_growth_t& g, int64_t e, int64_t m, int C) {
+  const int64_t bud = budget(g, e);
+  const int64_t lim = bud < m + C ? bud : m + C;
+  const int64_t mstar = m > lim ? m : lim;
+  const int64_t na = mstar - m;
+  return na < C ? na : C;
+}
+
+bool growth_valid(const kvm_growth_t& g) {
+  if (g.kind == KVM_GROWTH_FIXED) return g.fixed_slots >= 1;
+  if (g.kind == KVM_GROWTH_SQRT) return g.sqrt_coeff >= 1 && g.sqrt_coeff <= 65535;
+  return g.kind == KVM_GROWTH_UNBOUNDED;
+}
+
+bool growth_equal(const kvm_growth_t& a, const kvm_growth_t& b) {
+  if (a.kind != b.kind) return false;
+  if (a.kind == KVM_GROWTH_FIXED) return a.fixed_slots == b.fixed_slots;
+  if (a.kind == KVM_GROWTH_SQRT) return a.sqrt_coeff == b.sqrt_coeff;
+  return true;
+}
+
+template <typename T>
+kvm_status_t dev_alloc(kvm_state* ks, T** p, size_t count, bool zero = true) {
+  void* ptr = nullptr;
+  size_t bytes = count * sizeof(T);
+  if (bytes == 0) bytes = sizeof(T);
+  cudaError_t e = cudaMalloc(&ptr, bytes);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return e == cudaErrorMemoryAllocation ? KVM_ERR_OOM : KVM_ERR_CUDA;
+  }
+  ks->allocs.push_back(ptr);
+  if (zero && cudaMemset(ptr, 0, bytes) != cudaSuccess) return KVM_ERR_CUDA;
+  *p = reinterpret_cast<T*>(ptr);
+  return KVM_OK;
+}
+
+void free_all(kvm_state* ks) {
+  for (void* p : ks->allocs) cudaFree(p);
+  ks->allocs.clear();
+}
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; cudaGetLastError(); return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) { ok = false; cudaGetLastError(); }
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+kvm_status_t bind_first_call(kvm_state* ks, int32_t block, const kvm_growth_t& growth, int32_t r, cudaStream_t stream) {
+  State& s = ks->s;
+  if (block < 8 || block > s.Cmax || (block % 8) != 0 || s.S >= block) return KVM_ERR_INVALID_ARG;
+  if (r < 0 || r > s.d || (r & 1)) return KVM_ERR_INVALID_ARG;
+  if (!growth_valid(growth)) return KVM_ERR_INVALID_ARG;
+  s.C = block; s.r = r; s.growth = growth; s.ringLen = (int64_t)s.w * block;
+  if (r > 0) {
+    std::vector<double> f(r / 2);
+    for (int i = 0; i < r / 2; ++i) f[i] = pow((double)s.rope_base, -2.0 * (double)i / (double)r);
+    if (cudaMemcpyAsync(s.inv_freq, f.data(), sizeof(double) * f.size(), cudaMemcpyHostToDevice, stream) != cudaSuccess)
+      return KVM_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return KVM_ERR_CUDA;
+  }
+  s.bound = true;
+  return KVM_OK;
+}
+
+kvm_status_t ensure_host_staging(kvm_state* ks) {
+  if (ks->host_staging) return KVM_OK;
+  State& s = ks->s;
+  const size_t nq = (size_t)s.B * s.Hq * s.Tcall * s.d, nk = (size_t)s.U * s.Tcall * s.d;
+  __nv_bfloat16 *a, *b, *c, *o;
+  kvm_status_t rc;
+  if ((rc = dev_alloc(ks, &a, nq, false)) != KVM_OK) return rc;
+  if ((rc = dev_alloc(ks, &b, nk, false)) != KVM_OK) return rc;
+  if ((rc = dev_alloc(ks, &c, nk, false)) != KVM_OK) return rc;
+  if ((rc = dev_alloc(ks, &o, nq, false)) != KVM_OK) return rc;
+  if ((rc = dev_alloc(ks, &s.hG, (size_t)s.U * s.Tcall, false)) != KVM_OK) return rc;
+  s.hQ = a; s.hK = b; s.hV = c; s.hOut = o;
+  ks->host_staging = true;
+  return KVM_OK;
+}
+
+bool launch_ok() { return cudaGetLastError() == cudaSuccess; }
+
+}  // namespace
+
+#define KVM_API __attribute__((visibility("default")))
+
+extern "C" {
+
+KVM_API const char* kvm_status_string(kvm_status_t s) {
+  switch (s) {
+    case KVM_OK: return "ok";
+    case KVM_ERR_INVALID_ARG: return "invalid argument";
+    case KVM_ERR_UNSUPPORTED: return "unsupported configuration";
+    case KVM_ERR_OOM: return "out of device memory";
+    case KVM_ERR_CUDA: return "CUDA error";
+    case KVM_ERR_STATE_MISMATCH: return "block/growth/rope_dims differ from the state's";
+    case KVM_ERR_CAPACITY: return "state or call capacity exceeded";
+    case KVM_ERR_TIMEOUT: return "device-side wait expired";
+  }
+  return "unknown status";
+}
+
+KVM_API int64_t kvm_plan_capacity(int32_t block, int32_t n_bswa_chunks, kvm_growth_t growth, int64_t seq_len) {
+  if (block < 1 || n_bswa_chunks < 1 || seq_len < 0 || !growth_valid(growth)) return -1;
+  int64_t m = 0;
+  for (int64_t c = n_bswa_chunks - 1; (c + 1) * block <= seq_len; ++c) {
+    const int64_t e = (c + 1) * block;
+    m += (m == 0) ? block : n_append_of(growth, e, m, block);
+  }
+  return m;
+}
+
+KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out) {
+  if (!cfg || !out) return KVM_ERR_INVALID_ARG;
+  if (cfg->batch < 1 || cfg->n_q_heads < 1 || cfg->n_kv_heads < 1 || cfg->n_q_heads % cfg->n_kv_heads) return KVM_ERR_INVALID_ARG;
+  if (cfg->n_bswa_chunks < 1 || cfg->sink_len < 0) return KVM_ERR_INVALID_ARG;
+  if (cfg->max_block < 8 || (cfg->max_block % 8) || cfg->sink_len >= cfg->max_block) return KVM_ERR_INVALID_ARG;
+  if (cfg->max_state_slots < cfg->max_block || cfg->max_call_tokens < 1) return KVM_ERR_INVALID_ARG;
+  if (!(cfg->rope_base > 0.f) || !(cfg->ln_eps >= 0.f) || !(cfg->norm_eps >= 0.f)) return KVM_ERR_INVALID_ARG;
+  if ((cfg->flags & KVM_FLAG_RECORD_ASSIGN) && cfg->max_seq_len < 1) return KVM_ERR_INVALID_ARG;
+  if (cfg->head_dim != 64 && cfg->head_dim != 128) return KVM_ERR_UNSUPPORTED;
+  if (cfg->max_block > kMaxBlock) return KVM_ERR_UNSUPPORTED;
+
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1 || cfg->device < 0 || cfg->device >= ndev) {
+    cudaGetLastError();
+    return KVM_ERR_CUDA;
+  }
+  DeviceGuard guard(cfg->device);
+  if (!guard.ok) return KVM_ERR_CUDA;
+
+  kvm_state* ks = new (std::nothrow) kvm_state();
+  if (!ks) return KVM_ERR_OOM;
+  State& s = ks->s;
+  memset(&s, 0, sizeof(State));
+  s.B = cfg->batch; s.Hq = cfg->n_q_heads; s.Hkv = cfg->n_kv_heads; s.d = cfg->head_dim;
+  s.G = s.Hq / s.Hkv; s.U = s.B * s.Hkv; s.w = cfg->n_bswa_chunks; s.S = cfg->sink_len;
+  s.Cmax = cfg->max_block;
+  s.Mcap = (cfg->max_state_slots + kRowAlign - 1) / kRowAlign * kRowAlign;
+  s.Tcall = cfg->max_call_tokens;
+  s.Tassign = (cfg->flags & KVM_FLAG_RECORD_ASSIGN) ? cfg->max_seq_len : 0;
+  s.rope_base = cfg->rope_base; s.ln_eps = cfg->ln_eps; s.norm_eps = cfg->norm_eps;
+  s.flags = cfg->flags; s.device = cfg->device;
+  s.stRows = (int64_t)s.w * s.Cmax + s.Tcall;
+
+  const int d = s.d;
+  std::vector<float> lw((size_t)s.Hkv * d, 1.f), lb((size_t)s.Hkv * d, 0.f), ts(s.Hq, 1.f), tb(s.Hq, 1.f);
+  if (cfg->ln_weight) memcpy(lw.data(), cfg->ln_weight, sizeof(float) * lw.size());
+  if (cfg->ln_bias) memcpy(lb.data(), cfg->ln_bias, sizeof(float) * lb.size());
+  if (cfg->tau_state) memcpy(ts.data(), cfg->tau_state, sizeof(float) * ts.size());
+  if (cfg->tau_bswa) memcpy(tb.data(), cfg->tau_bswa, sizeof(float) * tb.size());
+  double bound = 0.0;
+  for (int h = 0; h < s.Hkv; ++h) {
+    double gmax = 0.0, b2 = 0.0;
+    for (int x = 0; x < d; ++x) {
+      gmax = fmax(gmax, fabs((double)lw[(size_t)h * d + x]));
+      b2 += (double)lb[(size_t)h * d + x] * lb[(size_t)h * d + x];
+    }
+    bound = fmax(bound, sqrt((double)d) * gmax + sqrt(b2));
+  }
+  if (!(bound < 3.0e4)) { delete ks; return KVM_ERR_UNSUPPORTED; }   // fp16 routing copies must not overflow
+  s.sim_norm_bound = (float)(bound * 1.0001);
+
+  const size_t U = s.U, M = s.Mcap, ringCap = (size_t)s.w * s.Cmax, Cm = s.Cmax;
+  s.nsplitRoute = (int)((2 * 148 + U - 1) / U);
+  if (s.nsplitRoute > kMaxSplits) s.nsplitRoute = kMaxSplits;
+  if (s.nsplitRoute < 1) s.nsplitRoute = 1;
+  s.nsplitDec = (int)((4 * 148 + (size_t)s.B * s.Hq - 1) / ((size_t)s.B * s.Hq));
+  if (s.nsplitDec > kMaxSplits) s.nsplitDec = kMaxSplits;
+  if (s.nsplitDec < 1) s.nsplitDec = 1;
+
+  kvm_status_t rc = KVM_OK;
+#define A(ptr, count) if (rc == KVM_OK) rc = dev_alloc(ks, &(ptr), (count))
+  A(s.ln_w, (size_t)s.Hkv * d); A(s.ln_b, (size_t)s.Hkv * d); A(s.tau_s, (size_t)s.Hq); A(s.tau_b, (size_t)s.Hq);
+  A(s.inv_freq, (size_t)d / 2);
+  A(s.sumK, U * M * d); A(s.sumV, U * M * d); A(s.rho, U * M); A(s.wsum, U * M); A(s.cnt, U * M);
+  A(s.kmu, U * M); A(s.krstd, U * M);
+  A(s.Khat, U * M * d); A(s.Vhat, U * M * d);
+  A(s.ringK, U * ringCap * d); A(s.ringV, U * ringCap * d); A(s.ringG, U * ringCap);
+  A(s.stQ, (size_t)s.B * s.Hq * s.Tcall * d);
+  A(s.stK, U * (size_t)s.stRows * d); A(s.stV, U * (size_t)s.stRows * d); A(s.stG, U * (size_t)s.stRows);
+  A(s.ropeCS, (size_t)s.Tcall * (d / 2));
+  A(s.kbar64, U * Cm * d); A(s.kbarH, U * Cm * d); A(s.kbarNorm, U * Cm); A(s.newhat64, U * Cm * d);
+  A(s.candV, U * (size_t)s.nsplitRoute * Cm * kTopK); A(s.candI, U * (size_t)s.nsplitRoute * Cm * kTopK);
+  A(s.decPart, (size_t)s.B * s.Hq * s.nsplitDec * (d + 2)); A(s.decQ, (size_t)s.B * s.Hq * d);
+  A(s.status, (size_t)1);
+  if (s.Tassign > 0) { A(s.slotTok, U * (size_t)s.Tassign); A(s.appTok, U * (size_t)s.Tassign); }
+#undef A
+  if (rc == KVM_OK && s.Tassign > 0 && cudaMemset(s.slotTok, 0xff, U * (size_t)s.Tassign * sizeof(int32_t)) != cudaSuccess) rc = KVM_ERR_CUDA;
+  if (rc == KVM_OK) {
+    bool ok = cudaMemcpy(s.ln_w, lw.data(), sizeof(float) * lw.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(s.ln_b, lb.data(), sizeof(float) * lb.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(s.tau_s, ts.data(), sizeof(float) * ts.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaMemcpy(s.tau_b, tb.data(), sizeof(float) * tb.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+    if (!ok) rc = KVM_ERR_CUDA;
+  }
+  if (rc != KVM_OK) {
+    cudaGetLastError();
+    free_all(ks);
+    delete ks;
+    return rc;
+  }
+  *out = ks;
+  return KVM_OK;
+}
+
+KVM_API kvm_status_t kvm_state_free(kvm_state_t* ks) {
+  if (!ks) return KVM_OK;
+  DeviceGuard guard(ks->s.device);
+  cudaDeviceSynchronize();
+  free_all(ks);
+  delete ks;
+  return KVM_OK;
+}
+
+KVM_API kvm_status_t kvm_state_info(const kvm_state_t* ks, int64_t* n_slots, int64_t* position, int64_t* n_folds) {
+  if (!ks) return KVM_ERR_INVALID_ARG;
+  if (n_slots) *n_slots = ks->s.m;
+  if (position) *position = ks->s.pos;
+  if (n_folds) *n_folds = ks->s.nfolds;
+  return KVM_OK;
+}
+
+KVM_API int64_t kvm_launch_count(const kvm_state_t* ks) { return ks ? ks->s.launches : -1; }
+
+KVM_API kvm_status_t kvm_state_check(kvm_state_t* ks, void* cuda_stream) {
+  if (!ks) return KVM_ERR_INVALID_ARG;
+  DeviceGuard guard(ks->s.device);
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  int32_t w = 0;
+  if (cudaMemcpyAsync(&w, ks->s.status, sizeof(w), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return KVM_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return KVM_ERR_CUDA;
+  if (w == 0) return KVM_OK;
+  return w == KVM_ERR_TIMEOUT ? KVM_ERR_TIMEOUT : KVM_ERR_CUDA;
+}
+
+KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kvm_state_t* ks, int32_t block,
+                         kvm_growth_t growth, int32_t rope_dims, int64_t n_tokens, const float* gate, void* out,
+                         const kvm_strides_t* strides, void* cuda_stream) {
+  if (!q || !k || !v || !ks || !out) return KVM_ERR_INVALID_ARG;
+  State& s = ks->s;
+  if (n_tokens < 1) return KVM_ERR_INVALID_ARG;
+  if (n_tokens > s.Tcall) return KVM_ERR_CAPACITY;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  DeviceGuard guard(s.device);
+  if (!guard.ok) return KVM_ERR_CUDA;
+
+  const int d = s.d;
+  const int64_t n = n_tokens;
+  IngestArgs ia;
+  AttnArgs aa;
+  if (strides) {
+    for (int i = 0; i < 4; ++i) { ia.sq[i] = strides->q[i]; ia.sk[i] = strides->k[i]; ia.sv[i] = strides->v[i]; aa.so[i] = strides->out[i]; }
+    if (ia.sq[3] != 1 || ia.sk[3] != 1 || ia.sv[3] != 1 || aa.so[3] != 1) return KVM_ERR_INVALID_ARG;
+    // rows are read and written as pairs of bf16
+    for (int i = 0; i < 3; ++i)
+      if ((ia.sq[i] & 1) || (ia.sk[i] & 1) || (ia.sv[i] & 1) || (aa.so[i] & 1)) return KVM_ERR_INVALID_ARG;
+  } else {
+    ia.sq[0] = (int64_t)s.Hq * n * d; ia.sq[1] = n * d; ia.sq[2] = d; ia.sq[3] = 1;
+    ia.sk[0] = (int64_t)s.Hkv * n * d; ia.sk[1] = n * d; ia.sk[2] = d; ia.sk[3] = 1;
+    for (int i = 0; i < 4; ++i) { ia.sv[i] = ia.sk[i]; aa.so[i] = ia.sq[i]; }
+  }
+  if (((uintptr_t)q & 3) || ((uintptr_t)k & 3) || ((uintptr_t)v & 3) || ((uintptr_t)out & 3)) return KVM_ERR_INVALID_ARG;
+  ia.sg[0] = (int64_t)s.Hkv * n; ia.sg[1] = n; ia.sg[2] = 1;
+
+  if (!s.bound) {
+    kvm_status_t rc = bind_first_call(ks, block, growth, rope_dims, stream);
+    if (rc != KVM_OK) return rc;
+  } else if (block != s.C || rope_dims != s.r || !growth_equal(growth, s.growth)) {
+    return KVM_ERR_STATE_MISMATCH;
+  }
+  const int C = s.C;
+  const int64_t L = (int64_t)s.w * C;
+  const int64_t pos0 = s.pos, pos1 = pos0 + n;
+  const int64_t c0 = pos0 / C, c_last = (pos1 - 1) / C;
+
+  // capacity: the row count after this call follows from the budget rule alone
+  {
+    int64_t m_sim = s.m;
+    for (int64_t c = c0; c <= c_last; ++c) {
+      const int64_t e = (c + 1) * C;
+      if (e <= pos1 && c >= s.w - 1) m_sim += (m_sim == 0) ? C : n_append_of(s.growth, e, m_sim, C);
+    }
+    if (m_sim > s.Mcap) return KVM_ERR_CAPACITY;
+  }
+
+  ia.q = (const __nv_bfloat16*)q; ia.k = (const __nv_bfloat16*)k; ia.v = (const __nv_bfloat16*)v; ia.gate = gate;
+  ia.pos0 = pos0; ia.n = n;
+  ia.hist_start = (c0 + 1) * C - L; if (ia.hist_start < 0) ia.hist_start = 0;
+  ia.nhist = pos0 - ia.hist_start;
+  {
+    const int64_t c_next = pos1 / C;
+    ia.tail_start = (c_next + 1) * C - L; if (ia.tail_start < 0) ia.tail_start = 0;
+  }
+  s.launches += launch_ingest(&s, ia, stream);
+
+  const bool simt_attn = true;  // replaced by the tcgen05 kernel selection below once available
+  (void)simt_attn;
+  for (int64_t c = c0; c <= c_last; ++c) {
+    const int64_t e = (c + 1) * C;
+    const int64_t qs = c * C > pos0 ? c * C : pos0;
+    const int64_t qe = e < pos1 ? e : pos1;
+    int64_t b = e - L; if (b < 0) b = 0;
+    aa.q_row0 = qs - pos0; aa.nq = (int)(qe - qs); aa.t0 = qs; aa.m = s.m;
+    aa.win_row0 = b - ia.hist_start; aa.b = b; aa.out = (__nv_bfloat16*)out; aa.out_t0 = qs - pos0;
+    if (s.flags & KVM_FLAG_SIMT_ATTENTION) s.launches += launch_attn_simt(&s, aa, stream);
+    else s.launches += launch_attn_tc(&s, aa, stream);
+    if (qe == e && c >= s.w - 1) {
+      FoldArgs fa;
+      fa.ok = s.stK + (b - ia.hist_start) * d; fa.ov = s.stV + (b - ia.hist_start) * d; fa.og = s.stG + (b - ia.hist_start);
+      fa.unit_stride = s.stRows * d; fa.gate_stride = s.stRows;
+      fa.b = b; fa.m = s.m; fa.first = (s.m == 0);
+      fa.n_append = fa.first ? C : (int)n_append_of(s.growth, e, s.m, C);
+      s.launches += launch_fold(&s, fa, stream);
+      s.m += fa.n_append;
+      s.nfolds += 1;
+    }
+  }
+  s.pos = pos1;
+  return launch_ok() ? KVM_OK : KVM_ERR_CUDA;
+}
+
+KVM_API kvm_status_t kvm_decode_step(const void* q, const void* k, const void* v, kvm_state_t* ks, const float* gate,
+                             void* out, void* cuda_stream) {
+  if (!q || !k || !v || !ks || !out) return KVM_ERR_INVALID_ARG;
+  State& s = ks->s;
+  if (!s.bound) return KVM_ERR_STATE_MISMATCH;
+  if (((uintptr_t)q & 1) || ((uintptr_t)k & 1) || ((uintptr_t)v & 1) || ((uintptr_t)out & 1)) return KVM_ERR_INVALID_ARG;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  DeviceGuard guard(s.device);
+  if (!guard.ok) return KVM_ERR_CUDA;
+  const int C = s.C, d = s.d;
+  const int64_t L = (int64_t)s.w * C;
+  const int64_t t = s.pos, c = t / C, e = (c + 1) * C;
+  int64_t b = e - L; if (b < 0) b = 0;
+  const bool fold = ((t + 1) % C == 0) && c >= s.w - 1;
+  int n_a = 0;
+  if (fold) {
+    n_a = (s.m == 0) ? C : (int)n_append_of(s.growth, e, s.m, C);
+    if (s.m + n_a > s.Mcap) return KVM_ERR_CAPACITY;
+  }
+  DecodeArgs da;
+  da.q = (const __nv_bfloat16*)q; da.k = (const __nv_bfloat16*)k; da.v = (const __nv_bfloat16*)v; da.gate = gate;
+  da.out = (__nv_bfloat16*)out; da.t = t; da.b = b; da.m = s.m;
+  s.launches += launch_decode(&s, da, stream);
+  if (fold) {
+    const int64_t ringCap = (int64_t)s.w * s.Cmax;
+    const int64_t slot = b % s.ringLen;
+    FoldArgs fa;
+    fa.ok = s.ringK + slot * d; fa.ov = s.ringV + slot * d; fa.og = s.ringG + slot;
+    fa.unit_stride = ringCap * d; fa.gate_stride = ringCap;
+    fa.b = b; fa.m = s.m; fa.first = (s.m == 0); fa.n_append = n_a;
+    s.launches += launch_fold(&s, fa, stream);
+    s.m += n_a;
+    s.nfolds += 1;
+  }
+  s.pos = t + 1;
+  return launch_ok() ? KVM_OK : KVM_ERR_CUDA;
+}
+
+KVM_API kvm_status_t kvm_prefill_host(const void* q_host, const void* k_host, const void* v_host, kvm_state_t* ks,
+                              int32_t block, kvm_growth_t growth, int32_t rope_dims, int64_t n_tokens,
+                              const float* gate_host, void* out_host, void* cuda_stream) {
+  if (!q_host || !k_host || !v_host || !ks || !out_host) return KVM_ERR_INVALID_ARG;
+  State& s = ks->s;
+  if (n_tokens < 1) return KVM_ERR_INVALID_ARG;
+  if (n_tokens > s.Tcall) return KVM_ERR_CAPACITY;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  DeviceGuard guard(s.device);
+  if (!guard.ok) return KVM_ERR_CUDA;
+  kvm_status_t rc = ensure_host_staging(ks);
+  if (rc != KVM_OK) return rc;
+  const size_t bq = (size_t)s.B * s.Hq * n_tokens * s.d * 2, bk = (size_t)s.U * n_tokens * s.d * 2;
+  bool ok = cudaMemcpyAsync(s.hQ, q_host, bq, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(s.hK, k_host, bk, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(s.hV, v_host, bk, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  if (gate_host) ok = ok && cudaMemcpyAsync(s.hG, gate_host, (size_t)s.U * n_tokens * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); return KVM_ERR_CUDA; }
+  rc = kvm_prefill(s.hQ, s.hK, s.hV, ks, block, growth, rope_dims, n_tokens, gate_host ? s.hG : nullptr, s.hOut, nullptr, cuda_stream);
+  if (rc != KVM_OK) return rc;
+  if (cudaMemcpyAsync(out_host, s.hOut, bq, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return KVM_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return KVM_ERR_CUDA;
+  return KVM_OK;
+}
+
+KVM_API kvm_status_t kvm_decode_step_host(const void* q_host, const void* k_host, const void* v_host, kvm_state_t* ks,
+                                  const float* gate_host, void* out_host, void* cuda_stream) {
+  if (!q_host || !k_host || !v_host || !ks || !out_host) return KVM_ERR_INVALID_ARG;
+  State& s = ks->s;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  DeviceGuard guard(s.device);
+  if (!guard.ok) return KVM_ERR_CUDA;
+  kvm_status_t rc = ensure_host_staging(ks);
+  if (rc != KVM_OK) return rc;
+  const size_t bq = (size_t)s.B * s.Hq * s.d * 2, bk = (size_t)s.U * s.d * 2;
+  bool ok = cudaMemcpyAsync(s.hQ, q_host, bq, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(s.hK, k_host, bk, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(s.hV, v_host, bk, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  if (gate_host) ok = ok && cudaMemcpyAsync(s.hG, gate_host, (size_t)s.U * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); return KVM_ERR_CUDA; }
+  rc = kvm_decode_step(s.hQ, s.hK, s.hV, ks, gate_host ? s.hG : nullptr, s.hOut, cuda_stream);
+  if (rc != KVM_OK) return rc;
+  if (cudaMemcpyAsync(out_host, s.hOut, bq, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return KVM_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return KVM_ERR_CUDA;
+  return KVM_OK;
+}
+
+KVM_API kvm_status_t kvm_state_export(kvm_state_t* ks, double* sum_k, float* sum_v, float* radius, double* weight,
+                              int32_t* count, void* k_read, void* v_read, void* cuda_stream) {
+  if (!ks) return KVM_ERR_INVALID_ARG;
+  State& s = ks->s;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  DeviceGuard guard(s.device);
+  if (!guard.ok) return KVM_ERR_CUDA;
+  const size_t m = (size_t)s.m, M = (size_t)s.Mcap, d = (size_t)s.d, U = (size_t)s.U;
+  bool ok = true;
+  if (m > 0) {
+#define CP(dst, src, elt, width) \
+  if (dst) ok = ok && cudaMemcpy2DAsync(dst, m * (width) * (elt), src, M * (width) * (elt), m * (width) * (elt), U, cudaMemcpyDeviceToHost, stream) == cudaSuccess
+    CP(sum_k, s.sumK, sizeof(double), d);
+    CP(sum_v, s.sumV, sizeof(float), d);
+    CP(radius, s.rho, sizeof(float), (size_t)1);
+    CP(weight, s.wsum, sizeof(double), (size_t)1);
+    CP(count, s.cnt, sizeof(int32_t), (size_t)1);
+    CP(k_read, s.Khat, (size_t)2, d);
+    CP(v_read, s.Vhat, (size_t)2, d);
+#undef CP
+  }
+  ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); return KVM_ERR_CUDA; }
+  return KVM_OK;
+}
+
+KVM_API kvm_status_t kvm_debug_assignments(kvm_state_t* ks, int64_t n, int32_t* slot_of_token, uint8_t* was_appended,
+                                   void* cuda_stream) {
+  if (!ks || n < 0) return KVM_ERR_INVALID_ARG;
+  State& s = ks->s;
+  if (s.Tassign == 0) return KVM_ERR_STATE_MISMATCH;
+  if (n > s.pos || n > s.Tassign) return KVM_ERR_INVALID_ARG;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  DeviceGuard guard(s.device);
+  if (!guard.ok) return KVM_ERR_CUDA;
+  bool ok = true;
+  if (n > 0) {
+    if (slot_of_token)
+      ok = ok && cudaMemcpy2DAsync(slot_of_token, n * 4, s.slotTok, s.Tassign * 4, n * 4, s.U, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (was_appended)
+      ok = ok && cudaMemcpy2DAsync(was_appended, n, s.appTok, s.Tassign, n, s.U, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+  }
+  ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); return KVM_ERR_CUDA; }
+  return KVM_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,159 @@
+// Ingest: partial RoPE of q and k (Section 3.1 "Positional Encoding"; Appendix C "RoPE query/key")
+// and staging of the call's tokens behind the not-yet-folded history taken from the window ring.
+//
+// Staging layout per unit u (rows of d bf16):  [ history tokens hist_start .. pos0-1 | new tokens ]
+// so that the attention kernels address every window key of the call by (t - hist_start).
+#include "kvm_internal.h"
+
+namespace kvm {
+
+// cos/sin of t * base^(-2p/r) for the call's tokens; the angle is formed in fp64 because at
+// t ~ 1e5 an fp32 product already loses ~1e-2 rad.
+__global__ void rope_table_kernel(float2* __restrict__ cs, const double* __restrict__ inv_freq,
+                                  int64_t pos0, int64_t n, int half) {
+  int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= n * half) return;
+  int64_t i = idx / half;
+  int p = (int)(idx % half);
+  double ang = (double)(pos0 + i) * inv_freq[p];
+  double s, c;
+  sincos(ang, &s, &c);
+  cs[idx] = make_float2((float)c, (float)s);
+}
+
+// Copies history tokens [hist_start, pos0) from the ring into staging rows [0, nhist).
+__global__ void ingest_hist_kernel(__half* __restrict__ stK, __half* __restrict__ stV,
+                                   float* __restrict__ stG, const __half* __restrict__ ringK,
+                                   const __half* __restrict__ ringV, const float* __restrict__ ringG,
+                                   int64_t stRows, int64_t ringCap, int64_t ringLen, int64_t hist_start,
+                                   int64_t nhist, int d) {
+  const int u = blockIdx.y;
+  const int hw = d / 2;
+  int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= nhist * hw) return;
+  int64_t i = idx / hw;
+  int c2 = (int)(idx % hw);
+  int64_t slot = (hist_start + i) % ringLen;
+  const uint32_t* sk = reinterpret_cast<const uint32_t*>(ringK + ((int64_t)u * ringCap + slot) * d);
+  const uint32_t* sv = reinterpret_cast<const uint32_t*>(ringV + ((int64_t)u * ringCap + slot) * d);
+  uint32_t* dk = reinterpret_cast<uint32_t*>(stK + ((int64_t)u * stRows + i) * d);
+  uint32_t* dv = reinterpret_cast<uint32_t*>(stV + ((int64_t)u * stRows + i) * d);
+  dk[c2] = sk[c2];
+  dv[c2] = sv[c2];
+  if (c2 == 0) stG[(int64_t)u * stRows + i] = ringG[(int64_t)u * ringCap + slot];
+}
+
+// bf16 inputs are carried as fp16 inside the library (same tensor-core rate, 3 more mantissa
+// bits for the rotated values, the readout cache and the softmax weights).  Every bf16 value
+// with 2^-14 <= |x| <= 65504 converts exactly; larger magnitudes saturate, smaller ones round
+// with an absolute error below 2^-25.
+__device__ __forceinline__ __half2 to_half2_sat(float a, float b) {
+  a = fminf(fmaxf(a, -65504.f), 65504.f);
+  b = fminf(fmaxf(b, -65504.f), 65504.f);
+  return __floats2half2_rn(a, b);
+}
+
+__device__ __forceinline__ float rope_channel(const __nv_bfloat16* row, int ch, int r, const float2* cs) {
+  float val = __bfloat162float(row[ch]);
+  if (ch >= r) return val;
+  const int half = r >> 1;
+  if (ch < half) {
+    float other = __bfloat162float(row[ch + half]);
+    float2 c = cs[ch];
+    return val * c.x - other * c.y;
+  }
+  float other = __bfloat162float(row[ch - half]);
+  float2 c = cs[ch - half];
+  return other * c.y + val * c.x;
+}
+
+// New keys / values / gates of the call: rotate k, copy v, stage both, and write the tokens that
+// stay in the window after this call (t >= tail_start) into the ring.
+__global__ void ingest_kv_kernel(__half* __restrict__ stK, __half* __restrict__ stV,
+                                 float* __restrict__ stG, __half* __restrict__ ringK,
+                                 __half* __restrict__ ringV, float* __restrict__ ringG,
+                                 const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v,
+                                 const float* __restrict__ gate, const float2* __restrict__ ropeCS,
+                                 int64_t sk0, int64_t sk1, int64_t sk2, int64_t sv0, int64_t sv1, int64_t sv2,
+                                 int64_t sg0, int64_t sg1, int64_t sg2, int Hkv, int d, int r,
+                                 int64_t stRows, int64_t ringCap, int64_t ringLen, int64_t pos0, int64_t n,
+                                 int64_t nhist, int64_t tail_start) {
+  const int u = blockIdx.y;
+  const int b = u / Hkv, hk = u % Hkv;
+  const int hw = d / 2;
+  int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= n * hw) return;
+  int64_t j = idx / hw;
+  int c2 = (int)(idx % hw);
+  const __nv_bfloat16* krow = k + b * sk0 + hk * sk1 + j * sk2;
+  const __nv_bfloat16* vrow = v + b * sv0 + hk * sv1 + j * sv2;
+  const float2* cs = ropeCS + j * (r >> 1);
+  const __half2 kk = to_half2_sat(rope_channel(krow, 2 * c2, r, cs), rope_channel(krow, 2 * c2 + 1, r, cs));
+  const __half2 vv = to_half2_sat(__bfloat162float(vrow[2 * c2]), __bfloat162float(vrow[2 * c2 + 1]));
+  float g = gate ? gate[b * sg0 + hk * sg1 + j * sg2] : 1.0f;
+  const int64_t row = (int64_t)u * stRows + nhist + j;
+  reinterpret_cast<__half2*>(stK + row * d)[c2] = kk;
+  reinterpret_cast<__half2*>(stV + row * d)[c2] = vv;
+  if (c2 == 0) stG[row] = g;
+  const int64_t t = pos0 + j;
+  if (t >= tail_start) {
+    const int64_t slot = t % ringLen;
+    const int64_t rrow = (int64_t)u * ringCap + slot;
+    reinterpret_cast<__half2*>(ringK + rrow * d)[c2] = kk;
+    reinterpret_cast<__half2*>(ringV + rrow * d)[c2] = vv;
+    if (c2 == 0) ringG[rrow] = g;
+  }
+}
+
+__global__ void ingest_q_kernel(__half* __restrict__ stQ, const __nv_bfloat16* __restrict__ q,
+                                const float2* __restrict__ ropeCS, int64_t sq0, int64_t sq1, int64_t sq2,
+                                int Hq, int d, int r, int64_t Tcall, int64_t n) {
+  const int bh = blockIdx.y;
+  const int b = bh / Hq, h = bh % Hq;
+  const int hw = d / 2;
+  int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= n * hw) return;
+  int64_t j = idx / hw;
+  int c2 = (int)(idx % hw);
+  const __nv_bfloat16* qrow = q + b * sq0 + h * sq1 + j * sq2;
+  const float2* cs = ropeCS + j * (r >> 1);
+  reinterpret_cast<__half2*>(stQ + ((int64_t)bh * Tcall + j) * d)[c2] =
+      to_half2_sat(rope_channel(qrow, 2 * c2, r, cs), rope_channel(qrow, 2 * c2 + 1, r, cs));
+}
+
+int launch_ingest(State* st, const IngestArgs& a, cudaStream_t s) {
+  int launches = 0;
+  const int d = st->d, hw = d / 2;
+  const int threads = 256;
+  if (st->r > 0) {
+    int64_t tot = a.n * (st->r / 2);
+    rope_table_kernel<<<(unsigned)((tot + threads - 1) / threads), threads, 0, s>>>(st->ropeCS, st->inv_freq,
+                                                                                  a.pos0, a.n, st->r / 2);
+    ++launches;
+  }
+  if (a.nhist > 0) {
+    dim3 grid((unsigned)((a.nhist * hw + threads - 1) / threads), st->U);
+    ingest_hist_kernel<<<grid, threads, 0, s>>>(st->stK, st->stV, st->stG, st->ringK, st->ringV, st->ringG,
+                                                st->stRows, (int64_t)st->w * st->Cmax, st->ringLen,
+                                                a.hist_start, a.nhist, d);
+    ++launches;
+  }
+  {
+    dim3 grid((unsigned)((a.n * hw + threads - 1) / threads), st->U);
+    ingest_kv_kernel<<<grid, threads, 0, s>>>(st->stK, st->stV, st->stG, st->ringK, st->ringV, st->ringG, a.k,
+                                              a.v, a.gate, st->ropeCS, a.sk[0], a.sk[1], a.sk[2], a.sv[0],
+                                              a.sv[1], a.sv[2], a.sg[0], a.sg[1], a.sg[2], st->Hkv, d, st->r,
+                                              st->stRows, (int64_t)st->w * st->Cmax, st->ringLen, a.pos0, a.n,
+                                              a.nhist, a.tail_start);
+    ++launches;
+  }
+  {
+    dim3 grid((unsigned)((a.n * hw + threads - 1) / threads), st->B * st->Hq);
+    ingest_q_kernel<<<grid, threads, 0, s>>>(st->stQ, a.q, st->ropeCS, a.sq[0], a.sq[1], a.sq[2], st->Hq, d,
+                                             st->r, st->Tcall, a.n);
+    ++launches;
+  }
+  return launches;
+}
+
+}  // namespace kvm

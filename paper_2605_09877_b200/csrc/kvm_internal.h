@@ -1,0 +1,128 @@
+// Internal declarations shared by the translation units of libkvm (not installed).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kvm.h"
+
+namespace kvm {
+
+constexpr int kMaxBlock = 256;      // largest block C (one thread per overflow token in the fold)
+constexpr int kTopK = 8;            // routing filter keeps the K best approximate similarities per split
+constexpr int kMaxSplits = 32;      // routing filter / decode split count upper bound
+constexpr int kRowAlign = 128;      // state capacity is rounded up to the attention key tile
+
+// State of one layer: host bookkeeping + device buffers.  U = batch * n_kv_heads "units";
+// unit u = b * Hkv + hk owns rows [u*Mcap, (u+1)*Mcap) of every per-row array.
+struct State {
+  // ---- configuration (host) ----
+  int B, Hq, Hkv, d, G, U, w, S;
+  int Cmax;            // max block
+  int64_t Mcap;        // state rows capacity (multiple of kRowAlign)
+  int64_t Tcall;       // max tokens per prefill call
+  int64_t Tassign;     // max_seq_len for assignment recording (0 = off)
+  float rope_base, ln_eps, norm_eps;
+  uint32_t flags;
+  int device;
+  float sim_norm_bound;  // upper bound of ||LN_s(x)||_2 for any x (per layer)
+  // ---- bound by the first prefill ----
+  bool bound;
+  int C, r;
+  kvm_growth_t growth;
+  int64_t ringLen;     // w * C
+  // ---- progress (host) ----
+  int64_t pos, m, nfolds, launches;
+  // ---- parameters (device) ----
+  float *ln_w, *ln_b;     // [Hkv, d]
+  float *tau_s, *tau_b;   // [Hq]
+  double* inv_freq;       // [r/2]
+  // ---- state rows (device) ----
+  double* sumK;           // [U, Mcap, d]  running key sums (fp64: routing decisions are taken on them)
+  float* sumV;            // [U, Mcap, d]
+  float* rho;             // [U, Mcap]
+  double* wsum;           // [U, Mcap]
+  int32_t* cnt;           // [U, Mcap]
+  double *kmu, *krstd;    // [U, Mcap]   mean / rstd of LN_s(s^K_i)
+  __half *Khat, *Vhat;    // [U, Mcap, d]  readout cache (fp16): LN_s(s^K) and the value readout;
+                          //               operand of attention, decode and the routing filter
+  // ---- window ring (device): slot = t mod ringLen ----
+  __half *ringK, *ringV;         // [U, w*Cmax, d]  rotated keys / values (fp16)
+  float* ringG;                  // [U, w*Cmax]
+  // ---- per-call staging (device) ----
+  int64_t stRows;                // w*Cmax + Tcall
+  __half* stQ;                   // [B*Hq, Tcall, d] rotated queries (fp16)
+  __half *stK, *stV;             // [U, stRows, d]   history + new tokens (rotated keys, fp16)
+  float* stG;                    // [U, stRows]
+  float2* ropeCS;                // [Tcall, r/2] (cos, sin)
+  // ---- fold scratch (device) ----
+  double* kbar64;                // [U, Cmax, d]
+  __half* kbarH;                 // [U, Cmax, d]
+  float* kbarNorm;               // [U, Cmax]
+  double* newhat64;              // [U, Cmax, d]  LN_s of rows appended in this fold
+  int nsplitRoute;               // splits the routing filter may use
+  float* candV;                  // [U, nsplitRoute, Cmax, kTopK]
+  int32_t* candI;
+  // ---- decode scratch (device) ----
+  int nsplitDec;
+  float* decPart;                // [B*Hq, nsplitDec, d + 2]
+  __half* decQ;                  // [B*Hq, d] rotated query
+  // ---- recording / status ----
+  int32_t* slotTok;              // [U, Tassign]
+  uint8_t* appTok;               // [U, Tassign]
+  int32_t* status;               // device status word
+  // ---- device staging for the *_host entry points ----
+  void *hQ, *hK, *hV, *hOut;
+  float* hG;
+};
+
+inline int64_t budget_of(const kvm_growth_t& g, int64_t e);
+
+// ---------------- launchers (each returns the number of kernels it launched) ----------------
+
+struct IngestArgs {
+  const __nv_bfloat16 *q, *k, *v;
+  const float* gate;
+  int64_t sq[4], sk[4], sv[4];  // element strides (B, H, T, 1)
+  int64_t sg[3];
+  int64_t pos0, n, hist_start, nhist, tail_start;
+};
+int launch_ingest(State* st, const IngestArgs& a, cudaStream_t s);
+
+struct AttnArgs {
+  int64_t q_row0;      // first query row in stQ (local token index)
+  int nq;              // queries in this launch (<= C)
+  int64_t t0;          // absolute position of the first query
+  int64_t m;           // visible state rows
+  int64_t win_row0;    // row in stK/stV of window begin b
+  int64_t b;           // absolute position of window begin
+  __nv_bfloat16* out;  // user tensor
+  int64_t so[4];       // out strides
+  int64_t out_t0;      // token index inside `out` of the first query
+};
+int launch_attn_simt(State* st, const AttnArgs& a, cudaStream_t s);
+int launch_attn_tc(State* st, const AttnArgs& a, cudaStream_t s);
+
+struct FoldArgs {
+  const __half *ok, *ov;         // overflow block rows: unit u at ok + u*unit_stride (elements), C rows
+  const float* og;               // gates, unit u at og + u*gate_stride
+  int64_t unit_stride, gate_stride;
+  int64_t b;        // absolute position of the first overflow token
+  int64_t m;        // rows before the fold
+  int n_append;     // rows to append (== C on the first fold)
+  bool first;       // first state-creation step
+};
+int launch_fold(State* st, const FoldArgs& a, cudaStream_t s);
+
+struct DecodeArgs {
+  const __nv_bfloat16 *q, *k, *v;
+  const float* gate;
+  __nv_bfloat16* out;
+  int64_t t;   // absolute position of the token
+  int64_t b;   // window begin
+  int64_t m;
+};
+int launch_decode(State* st, const DecodeArgs& a, cudaStream_t s);
+
+}  // namespace kvm
