@@ -1,0 +1,406 @@
+#!/usr/bin/env python
+"""Benchmark of the KVM layer hot path on B200 (one JSON line on stdout).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+
+A "step" is one pass of the whole hot path over one batch of synthetic input:
+  prefill workloads (cfg1..cfg4, paper-speed): kvm_prefill of the full sequence on an empty
+      state (ingest/RoPE, per-chunk attention over [state ; window], every fold);
+      metric = prefill tokens/s (batch * sequence tokens per second).
+  decode workload (cfg5-decode): one kvm_decode_step for the whole batch on a state of
+      m = 4096 rows plus a 256..511-token window; metric = decode us per step.
+`value` is measured with inputs resident in HBM; `e2e` goes through the *_host entry points
+with pinned host buffers (H2D and D2H inside the timed region).  With N > 1 every rank runs
+the same per-GPU workload on its own units (weak scaling, no data-path collective).
+"""
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2605_09877_b200 import synth  # noqa: E402
+
+
+# ------------------------------------------------------------------------------------------
+# workload table and algorithmic work
+
+def workload(name):
+    c = synth.CONFIGS
+    if name in c and name != "cfg5":
+        return c[name], "prefill"
+    if name == "paper-speed":   # the paper's speed-benchmark shape: B8 H32 d128 C256, KVM-sqrt, T=32768
+        return synth.Workload("paper-speed", 8, 32, 32, 128, 32768, 256, "sqrt", r=0, seed=7), "prefill"
+    if name == "cfg5-decode":
+        return c["cfg5"], "decode"
+    raise SystemExit(f"unknown workload {name}")
+
+
+def fold_schedule(wl, T):
+    """(e, m_before, n_append) per fold from the budget rule M* = max(m, min(B(e), m + C))."""
+    out, m = [], 0
+    for c in range(T // wl.C):
+        e = (c + 1) * wl.C
+        if c < wl.w - 1:
+            continue
+        if m == 0:
+            out.append((e, 0, wl.C)); m = wl.C
+            continue
+        bud = wl.fixed_slots if wl.growth == "fixed" else (math.isqrt(wl.sqrt_coeff ** 2 * e) if wl.growth == "sqrt" else 1 << 60)
+        na = min(max(m, min(bud, m + wl.C)) - m, wl.C)
+        out.append((e, m, na)); m += na
+    return out
+
+
+def prefill_flops(wl, T):
+    """Algorithmic flops of one prefill: attention 4*d per (query, visible key) with the causal
+    triangle counted as a triangle, routing 2*d per (overflow token, state row) similarity."""
+    folds = {e: (m0, na) for e, m0, na in fold_schedule(wl, T)}
+    m, att_pairs, route_pairs = 0, 0, 0
+    for c in range(T // wl.C):
+        e = (c + 1) * wl.C
+        win_prev = min(c, wl.w - 1) * wl.C
+        att_pairs += wl.C * (m + win_prev) + wl.C * (wl.C + 1) // 2
+        if e in folds:
+            m0, na = folds[e]
+            if m0 > 0:
+                route_pairs += wl.C * m0 + (wl.C - na) * na
+            m = m0 + na
+    units_q, units_kv = wl.B * wl.Hq, wl.B * wl.Hkv
+    return 4 * wl.d * att_pairs * units_q, 2 * wl.d * route_pairs * units_kv
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=d["hbm_gbs"], tf_burst=d["bf16_tflops"], tf_sust=d["bf16_tflops_sustained"], src="measured")
+    return dict(hbm=6650.0, tf_burst=1590.0, tf_sust=1400.0, src="fallback")
+
+
+# ------------------------------------------------------------------------------------------
+# clocks
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.path = tempfile.mktemp(prefix="kvm_clocks_", suffix=".csv")
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        self.proc.wait()
+        sm, mx, reasons = [], [], set()
+        for line in open(self.path):
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples"])
+        sm.sort()
+        return dict(sm_mhz=sm[len(sm) // 2], sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle leg (reported baseline; the only place bench.py touches oracle/)
+
+def oracle_sample(wl, mode, budget_s=20.0):
+    """Times the fp64 oracle, as it stands, on a bounded sample of the workload."""
+    from oracle import kvm_oracle as ko
+    from tests.parity_util import oracle_config
+    cores = ko.threads()
+    if mode == "prefill":
+        # sample: `n_units` (batch, head) units over a prefix of T_s tokens sized for ~budget_s
+        n_units = min(cores, wl.B * wl.Hkv)
+        T_s = wl.T
+        att, rt = prefill_flops(wl.scaled(B=1, Hq=n_units * (wl.Hq // wl.Hkv), Hkv=n_units), T_s)
+        rate = 0.6e9 * cores   # rough fp64 flop/s of the plain loops; only used to size the sample
+        while (att + rt) / rate > budget_s and T_s > 4 * wl.C:
+            T_s //= 2
+            att, rt = prefill_flops(wl.scaled(B=1, Hq=n_units * (wl.Hq // wl.Hkv), Hkv=n_units), T_s)
+        small = wl.scaled(B=1, Hq=n_units * (wl.Hq // wl.Hkv), Hkv=n_units, T=T_s)
+        t = synth.make_inputs(small)
+        o = ko.KVMOracle(oracle_config(small))
+        q, k, v = (t[n].double().numpy() for n in "qkv")
+        t0 = time.perf_counter()
+        o.forward(q, k, v)
+        dt = time.perf_counter() - t0
+        # tokens/s of the whole layer (all B*Hkv units) at the oracle's measured unit rate
+        layer_tokens = wl.B * T_s * (n_units / (wl.B * wl.Hkv))
+        return dict(value=layer_tokens / dt, unit="tokens/s", cores=cores, kind="oracle",
+                    sample=f"{n_units} of {wl.B * wl.Hkv} (batch,head) units x first {T_s} of {wl.T} tokens, "
+                           f"{dt:.1f} s wall; value = layer tokens/s at that unit rate"), dt
+    # decode: oracle state built by a short unbounded-growth prefill to m rows, then timed steps
+    n_units = min(cores, wl.B * wl.Hkv)
+    small = synth.Workload("dec-sample", 1, n_units, n_units, wl.d, 4096 + 256 + 128, 256, "unbounded", seed=wl.seed)
+    t = synth.make_inputs(small)
+    o = ko.KVMOracle(oracle_config(small))
+    q, k, v = (t[n].double().numpy() for n in "qkv")
+    o.forward(q, k, v)
+    steps = 8
+    dq = synth.make_inputs(small.scaled(T=steps, seed=wl.seed + 1))
+    q, k, v = (dq[n].double().numpy() for n in "qkv")
+    t0 = time.perf_counter()
+    for s in range(steps):
+        o.forward(q[:, :, s:s + 1], k[:, :, s:s + 1], v[:, :, s:s + 1])
+    dt = (time.perf_counter() - t0) / steps
+    us_full = dt * 1e6 * (wl.B * wl.Hkv / n_units)
+    return dict(value=us_full, unit="us/step", cores=cores, kind="oracle",
+                sample=f"{n_units} of {wl.B * wl.Hkv} units, state of {o.rows} rows + window, {steps} steps; "
+                       f"value = measured step time x {wl.B * wl.Hkv // n_units} (units are independent)"), dt * steps
+
+
+# ------------------------------------------------------------------------------------------
+
+def dist_setup(n):
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    return rank, world, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+def max_over_ranks(x, world):
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device="cuda")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl, mode = workload(args.workload)
+    vals, last = [], None
+    for i in range(args.warmup + args.steps):
+        res, _ = oracle_sample(wl, mode, budget_s=8.0)
+        if i >= args.warmup:
+            vals.append(res["value"])
+        last = res
+    v = sum(vals) / len(vals)
+    unit = last["unit"]
+    ms = (wl.B * wl.T / v * 1e3) if mode == "prefill" else v / 1e3
+    line = dict(metric="kvm_prefill_tokens_per_s" if mode == "prefill" else "kvm_decode_us_per_step", value=v, unit=unit,
+                n_gpus=args.gpus, steps=args.steps, warmup=args.warmup, ms_per_step=ms,
+                higher_is_better=(mode == "prefill"), scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=wl.name, mode=mode), impl="reference",
+                cpu_baseline=dict(value=v, unit=unit, cores=last["cores"], kind="oracle", sample=last["sample"]),
+                e2e=dict(value=v, unit=unit, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--impl", default="kvm")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--simt", action="store_true", help="time the scalar-core cross-check kernels")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    from paper_2605_09877_b200 import kvm
+    rank, world, local = dist_setup(args.gpus)
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    wl, mode = workload(args.workload)
+    pk = peaks()
+    W, K = max(args.warmup, 3), args.steps
+    g = kvm.growth(wl.growth, wl.fixed_slots, wl.sqrt_coeff)
+    flags = (kvm.FLAG_SIMT_ATTENTION | kvm.FLAG_SIMT_ROUTING) if args.simt else 0
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    if mode == "prefill":
+        T = wl.T
+        cap = kvm.kvm_plan_capacity(wl.C, wl.w, g, T)
+        st = kvm.KVMState(kvm.LayerConfig(wl.B, wl.Hq, wl.Hkv, wl.d, wl.C, max(cap, wl.C), T, n_bswa_chunks=wl.w,
+                                          sink_len=wl.S, device=local, flags=flags))
+        cpu = synth.make_inputs(wl.scaled(seed=wl.seed + 1000 * rank))
+        q, k, v = (cpu[n].to(dev) for n in "qkv")
+        out = torch.empty_like(q)
+
+        def step():
+            st.reset()
+            st.prefill(q, k, v, wl.C, g, wl.r, out=out)
+
+        units_per_step = wl.B * T   # tokens
+    else:
+        # state of m = 4096 rows (fixed budget 4096 reached by appends) and a one-block window
+        m_rows, Tp = 4096, 4096 + 2 * 256 + 256
+        seg = 1024
+        st = kvm.KVMState(kvm.LayerConfig(wl.B, wl.Hq, wl.Hkv, wl.d, wl.C, m_rows + 256, seg, n_bswa_chunks=wl.w,
+                                          sink_len=wl.S, device=local, flags=flags))
+        gfix = kvm.growth("fixed", fixed_slots=m_rows)
+        for s in range(Tp // seg):
+            t = synth.make_segment(wl, s, seg, device=dev)
+            st.prefill(t["q"], t["k"], t["v"], wl.C, gfix, wl.r)
+        torch.cuda.synchronize()
+        assert st.info()["n_slots"] == m_rows
+        dq = [synth.make_decode_inputs(wl, i % 8, device=dev) for i in range(8)]
+        out = torch.empty_like(dq[0]["q"])
+        cnt = [0]
+
+        def step():
+            d = dq[cnt[0] % 8]
+            cnt[0] += 1
+            st.decode_step(d["q"], d["k"], d["v"], out=out)
+
+        units_per_step = wl.B       # sequence-tokens per step
+
+    for _ in range(W):
+        step()
+    barrier(world)
+    sampler = ClockSampler(local)
+    sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    l0 = st.launch_count()
+    for i in range(K):
+        flush.fill_(i & 0xff)             # L2 flush between timed iterations (untimed)
+        ev[i][0].record(stream)
+        step()
+        ev[i][1].record(stream)
+    barrier(world)
+    launches = st.launch_count() - l0
+    clocks = sampler.stop()
+    times = [a.elapsed_time(b) for a, b in ev]
+    ms_step = max_over_ranks(sum(times) / K, world)
+
+    # per-phase device time (separate pass with event brackets) -> roofline of the dominant phase
+    st.profile_enable(True)
+    st.profile_read()
+    for i in range(min(K, 3)):
+        flush.fill_(i)
+        step()
+    prof = st.profile_read()
+    st.profile_enable(False)
+    nprof = min(K, 3)
+
+    if mode == "prefill":
+        att_f, rt_f = prefill_flops(wl, wl.T)
+        value = world * units_per_step / (ms_step * 1e-3)
+        att_ms = prof["attention"][0] / nprof
+        fold_ms = prof["fold"][0] / nprof
+        n_att = prof["attention"][1] / nprof
+        dom = "attention" if att_ms >= fold_ms else "fold"
+        ach = (att_f / 1e12) / (att_ms * 1e-3) if dom == "attention" else (rt_f / 1e12) / (fold_ms * 1e-3)
+        peak = pk["tf_sust"]
+        roof = dict(bound="tensor", kernel=dom, achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak, traffic=None,
+                    peak_source=f"{pk['src']} bf16 sustained (fp16 operands run at the bf16 rate)",
+                    launches_per_step=n_att, avg_launch_us=1e3 * att_ms / max(n_att, 1),
+                    whole_step_tflops=(att_f + rt_f) / 1e12 / (ms_step * 1e-3),
+                    whole_step_frac_of_burst=(att_f + rt_f) / 1e12 / (ms_step * 1e-3) / pk["tf_burst"],
+                    phase_ms={k_: v_[0] / nprof for k_, v_ in prof.items()})
+        metric, unit, hib = "kvm_prefill_tokens_per_s", "tokens/s", True
+    else:
+        info = st.info()
+        nwin_avg = 256 + 128
+        bytes_step = wl.B * wl.Hkv * (info["n_slots"] + nwin_avg) * wl.d * 2 * 2
+        value = ms_step * 1e3     # us per step (whole batch); per-sequence = value / B
+        dec_ms = prof["decode"][0] / max(prof["decode"][1], 1)
+        ach = bytes_step / 1e9 / (dec_ms * 1e-3)
+        roof = dict(bound="hbm", kernel="decode", achieved=ach, peak=pk["hbm"], unit="GB/s", frac=ach / pk["hbm"],
+                    traffic=None, peak_source=f"{pk['src']} copy bandwidth", bytes_per_step=bytes_step,
+                    frac_of_nominal_8TBs=ach / 8000.0, phase_ms={k_: v_[0] / max(v_[1], 1) for k_, v_ in prof.items()})
+        metric, unit, hib = "kvm_decode_us_per_step", "us/step", False
+
+    # end to end through the host-buffer entry points (pinned memory)
+    e2e = None
+    if not args.no_e2e:
+        if mode == "prefill":
+            hq, hk, hv = (cpu[n].contiguous().pin_memory() for n in "qkv")
+            hout = torch.empty_like(hq).pin_memory()
+            def estep():
+                st.reset()
+                st.prefill_host(hq, hk, hv, wl.C, g, wl.r, hout)
+            bi = (hq.numel() + hk.numel() + hv.numel()) * 2
+            bo = hout.numel() * 2
+        else:
+            hd = {n: dq[0][n].cpu().pin_memory() for n in "qkv"}
+            hout = torch.empty_like(hd["q"]).pin_memory()
+            def estep():
+                st.decode_step_host(hd["q"], hd["k"], hd["v"], hout)
+            bi = sum(hd[n].numel() for n in "qkv") * 2
+            bo = hout.numel() * 2
+        ne = min(K, 5)
+        for _ in range(2):
+            estep()
+        barrier(world)
+        t0 = time.perf_counter()
+        for _ in range(ne):
+            estep()
+        torch.cuda.synchronize()
+        dt = max_over_ranks((time.perf_counter() - t0) / ne, world)
+        ev_ = world * units_per_step / dt if mode == "prefill" else dt * 1e6
+        e2e = dict(value=ev_, unit=unit, h2d_bytes_per_step=bi, d2h_bytes_per_step=bo)
+
+    cpu_base = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu_base, _ = oracle_sample(wl, mode)
+
+    if rank == 0:
+        line = dict(metric=metric, value=value, unit=unit, n_gpus=world, steps=K, warmup=W, ms_per_step=ms_step,
+                    higher_is_better=hib, scaling="weak", vs_baseline=None, dtype="f16 operands, f32 accumulate, f64 routing",
+                    data="synthetic",
+                    config=dict(workload=wl.name, mode=mode, B=wl.B, Hq=wl.Hq, Hkv=wl.Hkv, d=wl.d, T=wl.T, C=wl.C,
+                                growth=wl.growth, rope_dims=wl.r, l2="256 MiB flush between timed steps",
+                                kernels="simt" if args.simt else "default"),
+                    clocks=clocks, e2e=e2e, gpu_launches=launches, roofline=roof, cpu_baseline=cpu_base)
+        print(json.dumps(line))
+    st.free()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -180,6 +180,21 @@ kvm_status_t kvm_state_export(kvm_state_t* state, double* sum_k, float* sum_v, f
 kvm_status_t kvm_debug_assignments(kvm_state_t* state, int64_t n, int32_t* slot_of_token,
                                    uint8_t* was_appended, void* cuda_stream);
 
+/* Returns the state to "empty" (position 0, no rows, no folds, block/growth/rope_dims unbound)
+ * without freeing or clearing device memory, so that one allocation serves many sequences.
+ * Host bookkeeping only; pending work on the stream is not waited for (the next call is
+ * ordered behind it on the same stream). */
+kvm_status_t kvm_state_reset(kvm_state_t* state);
+
+/* Per-phase device timing for benchmarks.  kvm_profile_enable(state, 1) makes every later
+ * call bracket each phase's launches with CUDA events on the call's stream (phases:
+ * 0 ingest, 1 attention, 2 fold, 3 decode attention); kvm_profile_read synchronises the
+ * device, adds the elapsed milliseconds and launch-group counts of the recorded brackets into
+ * ms[4] / groups[4] and clears the record.  Off by default; at most 8192 brackets are kept
+ * between reads (later ones are dropped and not counted). */
+kvm_status_t kvm_profile_enable(kvm_state_t* state, int32_t on);
+kvm_status_t kvm_profile_read(kvm_state_t* state, double* ms, int64_t* groups);
+
 /* Number of kernels the library has launched for this state so far (host counter). */
 int64_t kvm_launch_count(const kvm_state_t* state);
 

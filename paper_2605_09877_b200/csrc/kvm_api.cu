@@ -10,11 +10,34 @@
 
 using namespace kvm;
 
+struct ProfBracket { cudaEvent_t a, b; int phase; };
+
 struct kvm_state {
   State s;
   std::vector<void*> allocs;
   bool host_staging = false;
+  bool prof_on = false;
+  std::vector<ProfBracket> prof_free, prof_used;
 };
+
+namespace {
+// Brackets the launches of one phase with two events when profiling is enabled.
+struct PhaseTimer {
+  kvm_state* ks; cudaStream_t stream; bool active = false; ProfBracket br{};
+  PhaseTimer(kvm_state* k, int phase, cudaStream_t s) : ks(k), stream(s) {
+    if (!ks->prof_on || ks->prof_used.size() >= 8192) return;
+    if (!ks->prof_free.empty()) { br = ks->prof_free.back(); ks->prof_free.pop_back(); }
+    else if (cudaEventCreate(&br.a) != cudaSuccess || cudaEventCreate(&br.b) != cudaSuccess) { cudaGetLastError(); return; }
+    br.phase = phase;
+    active = cudaEventRecord(br.a, stream) == cudaSuccess;
+  }
+  ~PhaseTimer() {
+    if (!active) return;
+    cudaEventRecord(br.b, stream);
+    ks->prof_used.push_back(br);
+  }
+};
+}  // namespace
 
 namespace {
 
@@ -235,6 +258,7 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) rc = KVM_ERR_CUDA;
   }
+  if (rc == KVM_OK && !setup_attn_tc(&s)) rc = KVM_ERR_CUDA;
   if (rc != KVM_OK) {
     cudaGetLastError();
     free_all(ks);
@@ -249,8 +273,41 @@ KVM_API kvm_status_t kvm_state_free(kvm_state_t* ks) {
   if (!ks) return KVM_OK;
   DeviceGuard guard(ks->s.device);
   cudaDeviceSynchronize();
+  for (auto& v : {&ks->prof_free, &ks->prof_used})
+    for (const ProfBracket& br : *v) { cudaEventDestroy(br.a); cudaEventDestroy(br.b); }
   free_all(ks);
   delete ks;
+  return KVM_OK;
+}
+
+KVM_API kvm_status_t kvm_state_reset(kvm_state_t* ks) {
+  if (!ks) return KVM_ERR_INVALID_ARG;
+  State& s = ks->s;
+  s.bound = false; s.pos = 0; s.m = 0; s.nfolds = 0;
+  if (s.slotTok) {  // debug recording only: forget the previous sequence's assignments
+    DeviceGuard guard(s.device);
+    if (cudaMemset(s.slotTok, 0xff, (size_t)s.U * s.Tassign * sizeof(int32_t)) != cudaSuccess) return KVM_ERR_CUDA;
+  }
+  return KVM_OK;
+}
+
+KVM_API kvm_status_t kvm_profile_enable(kvm_state_t* ks, int32_t on) {
+  if (!ks) return KVM_ERR_INVALID_ARG;
+  ks->prof_on = on != 0;
+  return KVM_OK;
+}
+
+KVM_API kvm_status_t kvm_profile_read(kvm_state_t* ks, double* ms, int64_t* groups) {
+  if (!ks || !ms || !groups) return KVM_ERR_INVALID_ARG;
+  DeviceGuard guard(ks->s.device);
+  if (cudaDeviceSynchronize() != cudaSuccess) return KVM_ERR_CUDA;
+  for (const ProfBracket& br : ks->prof_used) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, br.a, br.b) == cudaSuccess) { ms[br.phase] += t; groups[br.phase] += 1; }
+    else cudaGetLastError();
+    ks->prof_free.push_back(br);
+  }
+  ks->prof_used.clear();
   return KVM_OK;
 }
 
@@ -333,7 +390,7 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
     const int64_t c_next = pos1 / C;
     ia.tail_start = (c_next + 1) * C - L; if (ia.tail_start < 0) ia.tail_start = 0;
   }
-  s.launches += launch_ingest(&s, ia, stream);
+  { PhaseTimer pt(ks, 0, stream); s.launches += launch_ingest(&s, ia, stream); }
 
   const bool simt_attn = true;  // replaced by the tcgen05 kernel selection below once available
   (void)simt_attn;
@@ -344,15 +401,18 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
     int64_t b = e - L; if (b < 0) b = 0;
     aa.q_row0 = qs - pos0; aa.nq = (int)(qe - qs); aa.t0 = qs; aa.m = s.m;
     aa.win_row0 = b - ia.hist_start; aa.b = b; aa.out = (__nv_bfloat16*)out; aa.out_t0 = qs - pos0;
-    if (s.flags & KVM_FLAG_SIMT_ATTENTION) s.launches += launch_attn_simt(&s, aa, stream);
-    else s.launches += launch_attn_tc(&s, aa, stream);
+    {
+      PhaseTimer pt(ks, 1, stream);
+      if (s.flags & KVM_FLAG_SIMT_ATTENTION) s.launches += launch_attn_simt(&s, aa, stream);
+      else s.launches += launch_attn_tc(&s, aa, stream);
+    }
     if (qe == e && c >= s.w - 1) {
       FoldArgs fa;
       fa.ok = s.stK + (b - ia.hist_start) * d; fa.ov = s.stV + (b - ia.hist_start) * d; fa.og = s.stG + (b - ia.hist_start);
       fa.unit_stride = s.stRows * d; fa.gate_stride = s.stRows;
       fa.b = b; fa.m = s.m; fa.first = (s.m == 0);
       fa.n_append = fa.first ? C : (int)n_append_of(s.growth, e, s.m, C);
-      s.launches += launch_fold(&s, fa, stream);
+      { PhaseTimer pt(ks, 2, stream); s.launches += launch_fold(&s, fa, stream); }
       s.m += fa.n_append;
       s.nfolds += 1;
     }
@@ -383,7 +443,7 @@ KVM_API kvm_status_t kvm_decode_step(const void* q, const void* k, const void* v
   DecodeArgs da;
   da.q = (const __nv_bfloat16*)q; da.k = (const __nv_bfloat16*)k; da.v = (const __nv_bfloat16*)v; da.gate = gate;
   da.out = (__nv_bfloat16*)out; da.t = t; da.b = b; da.m = s.m;
-  s.launches += launch_decode(&s, da, stream);
+  { PhaseTimer pt(ks, 3, stream); s.launches += launch_decode(&s, da, stream); }
   if (fold) {
     const int64_t ringCap = (int64_t)s.w * s.Cmax;
     const int64_t slot = b % s.ringLen;
@@ -391,7 +451,7 @@ KVM_API kvm_status_t kvm_decode_step(const void* q, const void* k, const void* v
     fa.ok = s.ringK + slot * d; fa.ov = s.ringV + slot * d; fa.og = s.ringG + slot;
     fa.unit_stride = ringCap * d; fa.gate_stride = ringCap;
     fa.b = b; fa.m = s.m; fa.first = (s.m == 0); fa.n_append = n_a;
-    s.launches += launch_fold(&s, fa, stream);
+    { PhaseTimer pt(ks, 2, stream); s.launches += launch_fold(&s, fa, stream); }
     s.m += n_a;
     s.nfolds += 1;
   }

@@ -1,5 +1,358 @@
-// Placeholder while the tcgen05 kernel is brought up: routes to the scalar-core kernel.
+// Fused attention of one chunk over [state rows ; window] on the 5th-generation tensor cores
+// (Section 3.2 "Readout": one softmax over the concatenation, state fully visible, causal in
+// the window, per-region temperatures).
+//
+// One CTA owns a 128-query tile of one (batch, query head) and walks the key tiles (128 keys:
+// first the state's readout cache, then the window) with three warp roles:
+//   warp 0      TMA producer: Q once, then K/V tiles into a 2-stage shared-memory ring
+//               (cp.async.bulk.tensor, 128-byte swizzle, mbarrier complete_tx)
+//   warp 1      MMA issuer: S = Q K^T into a double-buffered TMEM accumulator and
+//               O += P V into a second TMEM accumulator (tcgen05.mma kind::f16, fp32 accumulate)
+//   warps 2-5   softmax: each thread owns one query row (tcgen05.ld 32x32b), applies the region
+//               temperature and masks, keeps the running max / sum in registers, rescales O in TMEM
+//               only when the max grew by more than 2^8 (the final 1/l normalisation makes the
+//               stale max exact), writes P as fp16 into swizzled shared memory for the PV MMA,
+//               and finally normalises O and stores bf16 rows.
+// Every mbarrier wait is bounded; on expiry the CTA records KVM_ERR_TIMEOUT and tears down.
 #include "kvm_internal.h"
+#include "tc_common.cuh"
+
 namespace kvm {
-int launch_attn_tc(State* st, const AttnArgs& a, cudaStream_t s) { return launch_attn_simt(st, a, s); }
+
+struct AttnTcParams {
+  int64_t q_row0, t0, m, win_row0, b, out_t0;
+  int64_t so0, so1, so2;
+  __nv_bfloat16* out;
+  const float *tau_s, *tau_b;
+  int32_t* status;
+  int nq, Hq, Hkv, G;
+};
+
+template <int D>
+struct AttnTcCfg {
+  static constexpr int BM = 128, BN = 128, NS = 2;
+  static constexpr int NKB = D / 64;                 // 64-channel boxes per tile row
+  static constexpr int BOX_BYTES = 128 * 128;        // 128 rows x 64 fp16
+  static constexpr int TILE_BYTES = NKB * BOX_BYTES; // Q, K or V tile
+  static constexpr int P_BYTES = 2 * BOX_BYTES;      // 128 rows x 128 keys fp16
+  static constexpr int OFF_Q = 0;
+  static constexpr int OFF_K = OFF_Q + TILE_BYTES;
+  static constexpr int OFF_V = OFF_K + NS * TILE_BYTES;
+  static constexpr int OFF_P = OFF_V + NS * TILE_BYTES;
+  static constexpr int OFF_BAR = OFF_P + P_BYTES;
+  // + alignment slack; never less than half an SM so that one CTA (and one 512-column TMEM
+  // allocation) is resident per SM
+  static constexpr int SMEM_BYTES = (OFF_BAR + 256 + 1024) > 120 * 1024 ? (OFF_BAR + 256 + 1024) : 120 * 1024;
+  static constexpr uint32_t TMEM_COLS = 512;
+  static constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_O = 256;
+};
+
+enum { BAR_QFULL = 0, BAR_KFULL = 1, BAR_VFULL = 3, BAR_FREE = 5, BAR_SFULL = 7, BAR_PFULL = 9, BAR_PVDONE = 10, BAR_COUNT = 11 };
+
+template <int D>
+__global__ void __launch_bounds__(192, 1)
+attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapKs,
+               const __grid_constant__ CUtensorMap mapVs, const __grid_constant__ CUtensorMap mapKw,
+               const __grid_constant__ CUtensorMap mapVw, const AttnTcParams p) {
+  using Cfg = AttnTcCfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sQ = base + Cfg::OFF_Q;
+  uint8_t* sK = base + Cfg::OFF_K;
+  uint8_t* sV = base + Cfg::OFF_V;
+  uint8_t* sP = base + Cfg::OFF_P;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(base + Cfg::OFF_BAR);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + BAR_COUNT);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int qt = blockIdx.x, bh = blockIdx.y;
+  const int bb = bh / p.Hq, hq = bh % p.Hq, hk = hq / p.G;
+  const int u = bb * p.Hkv + hk;
+  const int rows_valid = min(128, p.nq - qt * 128);
+  const int64_t t_first = p.t0 + (int64_t)qt * 128;
+  const int64_t t_last = t_first + rows_valid - 1;
+  const int nst = (int)((p.m + 127) / 128);
+  const int nwt = (int)((t_last - p.b + 1 + 127) / 128);
+  const int ntiles = nst + nwt;
+
+  if (tid == 0) {
+    tc::mbar_init(&bars[BAR_QFULL], 1);
+    for (int s = 0; s < Cfg::NS; ++s) {
+      tc::mbar_init(&bars[BAR_KFULL + s], 1);
+      tc::mbar_init(&bars[BAR_VFULL + s], 1);
+      tc::mbar_init(&bars[BAR_FREE + s], 1);
+    }
+    tc::mbar_init(&bars[BAR_SFULL + 0], 1);
+    tc::mbar_init(&bars[BAR_SFULL + 1], 1);
+    tc::mbar_init(&bars[BAR_PFULL], 4);
+    tc::mbar_init(&bars[BAR_PVDONE], 1);
+    *abort_flag = 0;
+    tc::fence_barrier_init();
+  }
+  if (warp == 1) {
+    tc::tmem_alloc(tmem_slot, Cfg::TMEM_COLS);
+    tc::tmem_relinquish();
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+#define KVM_WAIT(bar, par)                                   \
+  if (!tc::mbar_wait((bar), (par))) {                        \
+    atomicExch(p.status, (int)KVM_ERR_TIMEOUT);              \
+    *abort_flag = 1;                                         \
+    break;                                                   \
+  }
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------
+    if (lane == 0) {
+      tc::prefetch_tmap(&mapQ); tc::prefetch_tmap(&mapKs); tc::prefetch_tmap(&mapVs);
+      tc::prefetch_tmap(&mapKw); tc::prefetch_tmap(&mapVw);
+      tc::mbar_expect_tx(&bars[BAR_QFULL], Cfg::TILE_BYTES);
+      for (int kb = 0; kb < Cfg::NKB; ++kb)
+        tc::tma_load_3d(sQ + kb * Cfg::BOX_BYTES, &mapQ, &bars[BAR_QFULL], kb * 64, (int)(p.q_row0 + qt * 128), bh);
+      for (int j = 0; j < ntiles; ++j) {
+        const int s = j % Cfg::NS;
+        if (*abort_flag) break;
+        if (j >= Cfg::NS) { KVM_WAIT(&bars[BAR_FREE + s], ((j / Cfg::NS) - 1) & 1); }
+        const bool st = j < nst;
+        const CUtensorMap* mk = st ? &mapKs : &mapKw;
+        const CUtensorMap* mv = st ? &mapVs : &mapVw;
+        const int row = st ? j * 128 : (int)(p.win_row0 + (int64_t)(j - nst) * 128);
+        tc::mbar_expect_tx(&bars[BAR_KFULL + s], Cfg::TILE_BYTES);
+        for (int kb = 0; kb < Cfg::NKB; ++kb)
+          tc::tma_load_3d(sK + s * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, mk, &bars[BAR_KFULL + s], kb * 64, row, u);
+        tc::mbar_expect_tx(&bars[BAR_VFULL + s], Cfg::TILE_BYTES);
+        for (int kb = 0; kb < Cfg::NKB; ++kb)
+          tc::tma_load_3d(sV + s * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, mv, &bars[BAR_VFULL + s], kb * 64, row, u);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer ------------------------------
+    if (lane == 0) {
+      constexpr uint32_t IDESC_QK = tc::idesc_f16(128, 128, false);
+      constexpr uint32_t IDESC_PV = tc::idesc_f16(128, D, true);
+      const uint32_t aQ = tc::smem_u32(sQ), aK = tc::smem_u32(sK), aV = tc::smem_u32(sV), aP = tc::smem_u32(sP);
+      bool dead = false;
+      auto issue_qk = [&](int j) -> bool {
+        const int s = j % Cfg::NS;
+        if (!tc::mbar_wait(&bars[BAR_KFULL + s], (j / Cfg::NS) & 1)) return false;
+        tc::tc_fence_after();
+        const uint32_t dS = tmem + ((j & 1) ? Cfg::COL_S1 : Cfg::COL_S0);
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint32_t off = (ks / 4) * Cfg::BOX_BYTES + (ks % 4) * 32;
+          tc::mma_f16_ss(dS, tc::smem_desc_sw128(aQ + off, 16, 1024),
+                         tc::smem_desc_sw128(aK + s * Cfg::TILE_BYTES + off, 16, 1024), IDESC_QK, ks > 0);
+        }
+        tc::mma_commit(&bars[BAR_SFULL + (j & 1)]);
+        return true;
+      };
+      do {
+        if (!tc::mbar_wait(&bars[BAR_QFULL], 0)) { dead = true; break; }
+        if (ntiles > 0 && !issue_qk(0)) { dead = true; break; }
+        for (int j = 0; j < ntiles; ++j) {
+          const int s = j % Cfg::NS;
+          if (*abort_flag) { dead = true; break; }
+          if (j + 1 < ntiles && !issue_qk(j + 1)) { dead = true; break; }
+          if (!tc::mbar_wait(&bars[BAR_PFULL], j & 1)) { dead = true; break; }
+          if (!tc::mbar_wait(&bars[BAR_VFULL + s], (j / Cfg::NS) & 1)) { dead = true; break; }
+          tc::tc_fence_after();
+          const uint32_t dO = tmem + Cfg::COL_O;
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint32_t offP = (kk / 4) * Cfg::BOX_BYTES + (kk % 4) * 32;
+            const uint32_t offV = kk * 2048;   // 16 key rows x 128 B
+            tc::mma_f16_ss(dO, tc::smem_desc_sw128(aP + offP, 16, 1024),
+                           tc::smem_desc_sw128(aV + s * Cfg::TILE_BYTES + offV, Cfg::BOX_BYTES, 1024), IDESC_PV,
+                           (j > 0 || kk > 0) ? 1u : 0u);
+          }
+          tc::mma_commit(&bars[BAR_FREE + s]);
+          tc::mma_commit(&bars[BAR_PVDONE]);
+        }
+      } while (false);
+      if (dead) { atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; }
+    }
+  } else {
+    // ------------------------------ softmax / epilogue ------------------------------
+    const int quarter = warp & 3;                     // TMEM lane quarter this warp may access
+    const int row = quarter * 32 + lane;              // query row inside the tile
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    const int64_t t_row = t_first + row;
+    const float kLog2e = 1.4426950408889634f;
+    const float sc_s = p.tau_s[hq] * rsqrtf((float)D) * kLog2e;
+    const float sc_b = p.tau_b[hq] * rsqrtf((float)D) * kLog2e;
+    float m_run = -INFINITY, l_run = 0.f;
+    bool ok = true;
+    for (int j = 0; j < ntiles && ok; ++j) {
+      do {
+        ok = false;
+        KVM_WAIT(&bars[BAR_SFULL + (j & 1)], (j >> 1) & 1);
+        tc::tc_fence_after();
+        float x[128];
+        {
+          const uint32_t ts = tmem + lane_base + ((j & 1) ? Cfg::COL_S1 : Cfg::COL_S0);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t r[32];
+            tc::tmem_ld32(ts + c * 32, r);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) x[c * 32 + i] = __uint_as_float(r[i]);
+          }
+          tc::tmem_wait_ld();
+        }
+        // region scale + mask
+        const bool st = j < nst;
+        const float sc = st ? sc_s : sc_b;
+        // number of visible columns of this tile for this row
+        int64_t nvis;
+        if (st) nvis = p.m - (int64_t)j * 128;
+        else nvis = t_row - (p.b + (int64_t)(j - nst) * 128) + 1;
+        const int vis = (int)max((int64_t)0, min((int64_t)128, nvis));
+        float mx = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 128; ++c) {
+          x[c] = (c < vis) ? x[c] * sc : -INFINITY;
+          mx = fmaxf(mx, x[c]);
+        }
+        float mnew = fmaxf(m_run, mx);
+        if (j > 0) {
+          KVM_WAIT(&bars[BAR_PVDONE], (j - 1) & 1);   // P buffer free, O quiescent
+          tc::tc_fence_after();
+          const bool need = mnew > m_run + 8.0f;
+          if (__any_sync(0xffffffffu, need)) {
+            const float corr = (m_run == -INFINITY) ? 0.f : tc::ex2_approx(m_run - mnew);
+            l_run *= corr;
+            m_run = mnew;
+            const uint32_t to = tmem + lane_base + Cfg::COL_O;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t r[32];
+              tc::tmem_ld32(to + c * 32, r);
+              tc::tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
+              tc::tmem_st32(to + c * 32, r);
+            }
+            tc::tmem_wait_st();
+          }
+        } else {
+          m_run = mnew;
+        }
+        const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
+        float lsum = 0.f;
+        // P row -> shared memory, K-major, 128-byte swizzle: 16-byte chunk ch of row r lives at
+        // r*128 + ((ch ^ (r & 7)) * 16) inside its 64-key box.
+        uint8_t* prow = sP + row * 128;
+#pragma unroll
+        for (int ch = 0; ch < 16; ++ch) {
+          uint32_t w[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float p0 = tc::ex2_approx(x[ch * 8 + 2 * i] - m_use);
+            const float p1 = tc::ex2_approx(x[ch * 8 + 2 * i + 1] - m_use);
+            lsum += p0 + p1;
+            const __half2 h = __floats2half2_rn(p0, p1);
+            w[i] = *reinterpret_cast<const uint32_t*>(&h);
+          }
+          uint8_t* dst = prow + (ch >> 3) * Cfg::BOX_BYTES + (((ch & 7) ^ (row & 7)) << 4);
+          *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        l_run += lsum;
+        tc::fence_proxy_async();
+        tc::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(&bars[BAR_PFULL]);
+        ok = true;
+      } while (false);
+    }
+    // epilogue
+    do {
+      if (!ok || ntiles == 0) break;
+      KVM_WAIT(&bars[BAR_PVDONE], (ntiles - 1) & 1);
+      tc::tc_fence_after();
+      const float inv = 1.f / l_run;
+      const uint32_t to = tmem + lane_base + Cfg::COL_O;
+      __nv_bfloat16* orow = p.out + bb * p.so0 + hq * p.so1 + (p.out_t0 + (int64_t)qt * 128 + row) * p.so2;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t r[32];
+        tc::tmem_ld32(to + c * 32, r);
+        tc::tmem_wait_ld();
+        if (row < rows_valid) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const __nv_bfloat162 o2 = __floats2bfloat162_rn(__uint_as_float(r[2 * i]) * inv, __uint_as_float(r[2 * i + 1]) * inv);
+            reinterpret_cast<__nv_bfloat162*>(orow + c * 32)[i] = o2;
+          }
+        }
+      }
+    } while (false);
+  }
+#undef KVM_WAIT
+  tc::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc::tmem_dealloc(tmem, Cfg::TMEM_COLS);
+  }
 }
+
+// ------------------------------------------------------------------------------------------
+
+bool encode_tmap_rows(CUtensorMap* map, const void* base, int d, int64_t rows, int64_t units, int box_rows) {
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                               const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                               CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static EncodeFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess || !ptr) {
+      cudaGetLastError();
+      return false;
+    }
+    fn = reinterpret_cast<EncodeFn>(ptr);
+  }
+  cuuint64_t gdim[3] = {(cuuint64_t)d, (cuuint64_t)rows, (cuuint64_t)units};
+  cuuint64_t gstr[2] = {(cuuint64_t)d * 2, (cuuint64_t)rows * d * 2};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(base), gdim, gstr, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int launch_attn_tc(State* st, const AttnArgs& a, cudaStream_t s) {
+  AttnTcParams p;
+  p.q_row0 = a.q_row0; p.t0 = a.t0; p.m = a.m; p.win_row0 = a.win_row0; p.b = a.b; p.out_t0 = a.out_t0;
+  p.so0 = a.so[0]; p.so1 = a.so[1]; p.so2 = a.so[2];
+  p.out = a.out; p.tau_s = st->tau_s; p.tau_b = st->tau_b; p.status = st->status;
+  p.nq = a.nq; p.Hq = st->Hq; p.Hkv = st->Hkv; p.G = st->G;
+  dim3 grid((a.nq + 127) / 128, st->B * st->Hq);
+  const CUtensorMap* tm = reinterpret_cast<const CUtensorMap*>(st->tmaps);
+  if (st->d == 128) {
+    attn_tc_kernel<128><<<grid, 192, AttnTcCfg<128>::SMEM_BYTES, s>>>(tm[0], tm[1], tm[2], tm[3], tm[4], p);
+  } else {
+    attn_tc_kernel<64><<<grid, 192, AttnTcCfg<64>::SMEM_BYTES, s>>>(tm[0], tm[1], tm[2], tm[3], tm[4], p);
+  }
+  return 1;
+}
+
+bool setup_attn_tc(State* st) {
+  CUtensorMap* tm = reinterpret_cast<CUtensorMap*>(st->tmaps);
+  bool ok = encode_tmap_rows(&tm[0], st->stQ, st->d, st->Tcall, (int64_t)st->B * st->Hq, 128);
+  ok = ok && encode_tmap_rows(&tm[1], st->Khat, st->d, st->Mcap, st->U, 128);
+  ok = ok && encode_tmap_rows(&tm[2], st->Vhat, st->d, st->Mcap, st->U, 128);
+  ok = ok && encode_tmap_rows(&tm[3], st->stK, st->d, st->stRows, st->U, 128);
+  ok = ok && encode_tmap_rows(&tm[4], st->stV, st->d, st->stRows, st->U, 128);
+  if (!ok) return false;
+  if (cudaFuncSetAttribute(attn_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<128>::SMEM_BYTES) != cudaSuccess) return false;
+  if (cudaFuncSetAttribute(attn_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnTcCfg<64>::SMEM_BYTES) != cudaSuccess) return false;
+  return true;
+}
+
+}  // namespace kvm

@@ -72,6 +72,8 @@ struct State {
   int32_t* slotTok;              // [U, Tassign]
   uint8_t* appTok;               // [U, Tassign]
   int32_t* status;               // device status word
+  // ---- TMA tensor maps (host copies, passed to kernels by value): stQ, Khat, Vhat, stK, stV, kbarH ----
+  alignas(64) unsigned char tmaps[8 * 128];
   // ---- device staging for the *_host entry points ----
   void *hQ, *hK, *hV, *hOut;
   float* hG;
@@ -103,6 +105,7 @@ struct AttnArgs {
 };
 int launch_attn_simt(State* st, const AttnArgs& a, cudaStream_t s);
 int launch_attn_tc(State* st, const AttnArgs& a, cudaStream_t s);
+bool setup_attn_tc(State* st);   // encodes the tensor maps, raises the shared-memory limits
 
 struct FoldArgs {
   const __half *ok, *ov;         // overflow block rows: unit u at ok + u*unit_stride (elements), C rows

@@ -24,7 +24,8 @@ FLAG_NO_RADIUS, FLAG_RECORD_ASSIGN, FLAG_SIMT_ATTENTION, FLAG_SIMT_ROUTING = 1, 
 
 EXPORTS = ["kvm_plan_capacity", "kvm_state_create", "kvm_prefill", "kvm_decode_step", "kvm_prefill_host",
            "kvm_decode_step_host", "kvm_state_free", "kvm_state_info", "kvm_state_check", "kvm_state_export",
-           "kvm_debug_assignments", "kvm_launch_count", "kvm_status_string"]
+           "kvm_debug_assignments", "kvm_launch_count", "kvm_status_string", "kvm_state_reset",
+           "kvm_profile_enable", "kvm_profile_read"]
 
 
 class KVMError(RuntimeError):
@@ -81,6 +82,12 @@ def _load():
     L.kvm_state_export.argtypes = [vp] * 9
     L.kvm_debug_assignments.restype = C.c_int
     L.kvm_debug_assignments.argtypes = [vp, C.c_int64, vp, vp, vp]
+    L.kvm_state_reset.restype = C.c_int
+    L.kvm_state_reset.argtypes = [vp]
+    L.kvm_profile_enable.restype = C.c_int
+    L.kvm_profile_enable.argtypes = [vp, C.c_int32]
+    L.kvm_profile_read.restype = C.c_int
+    L.kvm_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     L.kvm_launch_count.restype = C.c_int64
     L.kvm_launch_count.argtypes = [vp]
     L.kvm_status_string.restype = C.c_char_p
@@ -227,6 +234,23 @@ class KVMState:
 
     def check(self, stream=None):
         return lib.kvm_state_check(self._h, _stream_ptr(stream))
+
+    def reset(self):
+        rc = lib.kvm_state_reset(self._h)
+        if rc != KVM_OK:
+            raise KVMError(rc, "kvm_state_reset")
+
+    def profile_enable(self, on=True):
+        lib.kvm_profile_enable(self._h, 1 if on else 0)
+
+    def profile_read(self):
+        """Returns {phase: (milliseconds, bracket count)} accumulated since the last read."""
+        ms = (C.c_double * 4)(); n = (C.c_int64 * 4)()
+        rc = lib.kvm_profile_read(self._h, ms, n)
+        if rc != KVM_OK:
+            raise KVMError(rc, "kvm_profile_read")
+        names = ("ingest", "attention", "fold", "decode")
+        return {names[i]: (ms[i], n[i]) for i in range(4)}
 
     def launch_count(self):
         return lib.kvm_launch_count(self._h)
