@@ -276,7 +276,7 @@ def main():
         units_per_step = wl.B * T   # tokens
     else:
         # state of m = 4096 rows (fixed budget 4096 reached by appends) and a one-block window
-        m_rows, Tp = 4096, 4096 + 2 * 256 + 256
+        m_rows, Tp = 4096, 5120   # 16 appending folds (e = 512 .. 4352), then 3 merging folds
         seg = 1024
         st = kvm.KVMState(kvm.LayerConfig(wl.B, wl.Hq, wl.Hkv, wl.d, wl.C, m_rows + 256, seg, n_bswa_chunks=wl.w,
                                           sink_len=wl.S, device=local, flags=flags))

@@ -243,7 +243,10 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   A(s.stQ, (size_t)s.B * s.Hq * s.Tcall * d);
   A(s.stK, U * (size_t)s.stRows * d); A(s.stV, U * (size_t)s.stRows * d); A(s.stG, U * (size_t)s.stRows);
   A(s.ropeCS, (size_t)s.Tcall * (d / 2));
-  A(s.kbar64, U * Cm * d); A(s.kbarH, U * Cm * d); A(s.kbarNorm, U * Cm); A(s.newhat64, U * Cm * d);
+  s.CbarRows = (s.Cmax + 127) / 128 * 128;
+  A(s.kbar64, U * Cm * d); A(s.kbarH, U * (size_t)s.CbarRows * d); A(s.kbarNorm, U * Cm);
+  A(s.kbarMu, U * Cm); A(s.kbarRstd, U * Cm);
+  A(s.foldPi, U * Cm); A(s.foldSorted, U * Cm); A(s.foldCreator, U * Cm); A(s.foldSegNew, U * Cm); A(s.foldNMerge, U);
   A(s.candV, U * (size_t)s.nsplitRoute * Cm * kTopK); A(s.candI, U * (size_t)s.nsplitRoute * Cm * kTopK);
   A(s.decPart, (size_t)s.B * s.Hq * s.nsplitDec * (d + 2)); A(s.decQ, (size_t)s.B * s.Hq * d);
   A(s.status, (size_t)1);
@@ -258,7 +261,7 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) rc = KVM_ERR_CUDA;
   }
-  if (rc == KVM_OK && !setup_attn_tc(&s)) rc = KVM_ERR_CUDA;
+  if (rc == KVM_OK && !(setup_attn_tc(&s) && setup_route_tc(&s))) rc = KVM_ERR_CUDA;
   if (rc != KVM_OK) {
     cudaGetLastError();
     free_all(ks);

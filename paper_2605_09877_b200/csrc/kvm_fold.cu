@@ -1,11 +1,14 @@
 // The fold of one overflow block into the state (Section 3.2 "Append", "Merge", budget rule,
 // value-radius preservation) for every unit:
 //   1. kbar_kernel          memory keys kbar_j = LN_s(zero_r(k_j))            (Eq. 1) in fp64
-//   2. route filter         approximate similarities kbar_j . LN_s(s^K_i) in fp16 x fp16 -> fp32,
-//                           K best per token and per row split (candidates only)
-//   3. fold_update_kernel   exact fp64 similarities for the candidates, append selection,
-//                           merge routing against s_+, deterministic per-row accumulation,
-//                           refresh of the readout caches of the touched rows
+//   2. routing filter       approximate similarities kbar_j . LN_s(s^K_i) in fp16 x fp16 -> fp32
+//                           (tcgen05 kernel in kvm_route_tc.cu, scalar-core cross-check here),
+//                           K best rows per token and per row split: candidates only
+//   3. fold_decide_kernel   exact fp64 similarities of the candidates, append selection, merge
+//                           routing against s_+, grouping of the merged tokens by target row
+//   4. fold_apply_kernel    one warp per touched row: creates appended rows, accumulates the
+//                           members in ascending token order (deterministic), refreshes the
+//                           readout cache (LN_s of the key sum, value-radius readout)
 //
 // Integer decisions (which tokens are appended, which row each token merges into) are taken on
 // fp64 similarities computed from fp64 key sums, so they agree with an fp64 reference unless two
@@ -22,15 +25,29 @@ __device__ __forceinline__ double warp_sum_d(double v) {
   return v;
 }
 
+// LN_s statistics of one row held as D/32 strided channels per lane.
+template <int CH>
+__device__ __forceinline__ void row_stats(const double (&x)[CH], int D, double eps, double& mean, double& rstd) {
+  double s = 0.0;
+#pragma unroll
+  for (int i = 0; i < CH; ++i) s += x[i];
+  mean = warp_sum_d(s) / D;
+  double q = 0.0;
+#pragma unroll
+  for (int i = 0; i < CH; ++i) q += (x[i] - mean) * (x[i] - mean);
+  rstd = 1.0 / sqrt(warp_sum_d(q) / D + eps);
+}
+
 // ------------------------------------------------------------------------------------------
-// 1. memory keys
+// 1. memory keys (one warp per overflow token)
 
 template <int D>
 __global__ void __launch_bounds__(256) kbar_kernel(const __half* __restrict__ ok, int64_t unit_stride,
                                                    const float* __restrict__ ln_w, const float* __restrict__ ln_b,
                                                    double* __restrict__ kbar64, __half* __restrict__ kbarH,
-                                                   float* __restrict__ kbarNorm, int C, int Cmax, int Hkv, int r,
-                                                   double ln_eps) {
+                                                   float* __restrict__ kbarNorm, double* __restrict__ kbarMu,
+                                                   double* __restrict__ kbarRstd, int C, int Cmax, int CbarRows,
+                                                   int Hkv, int r, double ln_eps) {
   constexpr int CH = D / 32;
   const int u = blockIdx.y, hk = u % Hkv;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -38,31 +55,34 @@ __global__ void __launch_bounds__(256) kbar_kernel(const __half* __restrict__ ok
   if (j >= C) return;
   const __half* row = ok + (int64_t)u * unit_stride + (int64_t)j * D;
   double val[CH];
-  double sum = 0.0;
 #pragma unroll
   for (int i = 0; i < CH; ++i) {
     const int x = lane + 32 * i;
     val[i] = (x < r) ? 0.0 : (double)__half2float(row[x]);
-    sum += val[i];
   }
-  const double mean = warp_sum_d(sum) / D;
-  double sq = 0.0;
-#pragma unroll
-  for (int i = 0; i < CH; ++i) sq += (val[i] - mean) * (val[i] - mean);
-  const double var = warp_sum_d(sq) / D;
-  const double rstd = 1.0 / sqrt(var + ln_eps);
+  double mean, rstd;
+  row_stats<CH>(val, D, ln_eps, mean, rstd);
+  double kb[CH];
   double n2 = 0.0;
   const int64_t o = ((int64_t)u * Cmax + j) * D;
+  const int64_t oh = ((int64_t)u * CbarRows + j) * D;
 #pragma unroll
   for (int i = 0; i < CH; ++i) {
     const int x = lane + 32 * i;
-    const double kb = (double)ln_w[hk * D + x] * ((val[i] - mean) * rstd) + (double)ln_b[hk * D + x];
-    kbar64[o + x] = kb;
-    kbarH[o + x] = __float2half_rn((float)kb);
-    n2 += kb * kb;
+    kb[i] = (double)ln_w[hk * D + x] * ((val[i] - mean) * rstd) + (double)ln_b[hk * D + x];
+    kbar64[o + x] = kb[i];
+    kbarH[oh + x] = __float2half_rn((float)kb[i]);
+    n2 += kb[i] * kb[i];
   }
   n2 = warp_sum_d(n2);
-  if (lane == 0) kbarNorm[(int64_t)u * Cmax + j] = (float)sqrt(n2) * 1.000001f;
+  // statistics of LN_s applied to kbar itself: the key of a row that this token would create
+  double mu2, rs2;
+  row_stats<CH>(kb, D, ln_eps, mu2, rs2);
+  if (lane == 0) {
+    kbarNorm[(int64_t)u * Cmax + j] = (float)sqrt(n2) * 1.000001f;
+    kbarMu[(int64_t)u * Cmax + j] = mu2;
+    kbarRstd[(int64_t)u * Cmax + j] = rs2;
+  }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -70,22 +90,22 @@ __global__ void __launch_bounds__(256) kbar_kernel(const __half* __restrict__ ok
 
 template <int D>
 __global__ void __launch_bounds__(256) route_filter_simt_kernel(const __half* __restrict__ kbarH,
-                                                                const __half* __restrict__ KhatH,
+                                                                const __half* __restrict__ Khat,
                                                                 float* __restrict__ candV,
                                                                 int32_t* __restrict__ candI, int C, int Cmax,
-                                                                int64_t Mcap, int64_t m, int nsplit) {
+                                                                int CbarRows, int64_t Mcap, int64_t m, int nsplit) {
   __shared__ __half2 sH[32 * (D / 2)];
   const int split = blockIdx.x, u = blockIdx.y;
   const int j = threadIdx.x;
   const bool active = j < C;
   int64_t per = (m + nsplit - 1) / nsplit;
-  per = (per + 31) / 32 * 32;
+  per = (per + 127) / 128 * 128;
   const int64_t i0 = (int64_t)split * per;
   const int64_t i1 = min(m, i0 + per);
 
   __half2 kb[D / 2];
   if (active) {
-    const __half2* src = reinterpret_cast<const __half2*>(kbarH + ((int64_t)u * Cmax + j) * D);
+    const __half2* src = reinterpret_cast<const __half2*>(kbarH + ((int64_t)u * CbarRows + j) * D);
 #pragma unroll
     for (int c = 0; c < D / 2; ++c) kb[c] = src[c];
   }
@@ -99,7 +119,7 @@ __global__ void __launch_bounds__(256) route_filter_simt_kernel(const __half* __
     for (int wd = threadIdx.x; wd < 32 * (D / 2); wd += 256) {
       const int row = wd / (D / 2), cw = wd % (D / 2);
       const int64_t i = tile + row;
-      sH[wd] = (i < i1) ? reinterpret_cast<const __half2*>(KhatH + ((int64_t)u * Mcap + i) * D)[cw]
+      sH[wd] = (i < i1) ? reinterpret_cast<const __half2*>(Khat + ((int64_t)u * Mcap + i) * D)[cw]
                         : __floats2half2_rn(0.f, 0.f);
     }
     __syncthreads();
@@ -136,49 +156,31 @@ __global__ void __launch_bounds__(256) route_filter_simt_kernel(const __half* __
 }
 
 // ------------------------------------------------------------------------------------------
-// 3. exact refine, append selection, routing, accumulation, readout refresh
+// 3. decisions
 
-struct FoldUpdateParams {
-  const __half* ov;          // overflow values
-  const float* og;           // overflow gates
-  int64_t unit_stride, gate_stride;
+struct FoldDecideParams {
   const double* kbar64;
   const float* kbarNorm;
-  double* newhat64;
+  const double *kbarMu, *kbarRstd;
   const float* candV;
   const int32_t* candI;
   const float *ln_w, *ln_b;
-  double* sumK; float* sumV; float* rho; double* wsum; int32_t* cnt; double *kmu, *krstd;
-  __half *Khat, *Vhat;
-  int32_t* slotTok; uint8_t* appTok;
-  int64_t Mcap, Tassign, m, b;
-  int C, Cmax, Hkv, S, n_append, nsplit, first, radius_on;
-  double ln_eps, norm_eps;
-  float thr_coeff;   // 2 * (fp16 error coefficient) * bound of ||LN_s(.)||
+  const double* sumK;
+  const double *kmu, *krstd;
+  int32_t *pi, *sorted, *creator, *segnew, *nmerge;   // outputs, [U, Cmax] (nmerge [U])
+  int64_t Mcap, m;
+  int C, Cmax, Hkv, S, n_append, nsplit;
+  float thr_coeff;
 };
 
 constexpr int kPairCap = 1536;
 constexpr int kPairPerTok = 24;
 
-// LN_s statistics of one row held as D/32 strided channels per lane.
-template <int CH>
-__device__ __forceinline__ void row_stats(const double (&x)[CH], int D, double eps, double& mean, double& rstd) {
-  double s = 0.0;
-#pragma unroll
-  for (int i = 0; i < CH; ++i) s += x[i];
-  mean = warp_sum_d(s) / D;
-  double q = 0.0;
-#pragma unroll
-  for (int i = 0; i < CH; ++i) q += (x[i] - mean) * (x[i] - mean);
-  rstd = 1.0 / sqrt(warp_sum_d(q) / D + eps);
-}
-
 template <int D>
-__global__ void __launch_bounds__(256) fold_update_kernel(FoldUpdateParams p) {
-  constexpr int CH = D / 32;
+__global__ void __launch_bounds__(256) fold_decide_kernel(FoldDecideParams p) {
   __shared__ double s_gamma[D], s_beta[D];
   __shared__ double s_score[kMaxBlock], s_best[kMaxBlock];
-  __shared__ int s_barg[kMaxBlock], s_pi[kMaxBlock], s_newrow[kMaxBlock], s_sorted[kMaxBlock];
+  __shared__ int s_barg[kMaxBlock], s_pi[kMaxBlock], s_creator[kMaxBlock];
   __shared__ int s_pstart[kMaxBlock], s_pcnt[kMaxBlock];
   __shared__ unsigned char s_app[kMaxBlock], s_exh[kMaxBlock];
   __shared__ int s_prow[kPairCap];
@@ -191,11 +193,9 @@ __global__ void __launch_bounds__(256) fold_update_kernel(FoldUpdateParams p) {
   const int C = p.C;
   const int64_t m = p.m;
   const int n_a = p.n_append;
-  const bool all_append = p.first || n_a >= C;
   const double* kbarU = p.kbar64 + (int64_t)u * p.Cmax * D;
-  const __half* ovU = p.ov + (int64_t)u * p.unit_stride;
-  const float* ogU = p.og + (int64_t)u * p.gate_stride;
   const int64_t rowBase = (int64_t)u * p.Mcap;
+  const int64_t tokBase = (int64_t)u * p.Cmax;
 
   for (int x = tid; x < D; x += 256) {
     s_gamma[x] = (double)p.ln_w[hk * D + x];
@@ -203,260 +203,283 @@ __global__ void __launch_bounds__(256) fold_update_kernel(FoldUpdateParams p) {
   }
   if (tid == 0) { s_np = 0; s_nmerge = 0; }
   if (tid < kMaxBlock) {
-    s_app[tid] = (all_append && tid < C) ? 1 : 0;
-    s_exh[tid] = 0;
-    s_pcnt[tid] = 0;
-    s_pstart[tid] = 0;
-    s_pi[tid] = -1;
-    s_best[tid] = -INFINITY;
-    s_barg[tid] = -1;
-    s_score[tid] = -INFINITY;
-    s_newrow[tid] = all_append ? (int)m + tid : -1;   // first fold: m == 0
+    s_app[tid] = 0; s_exh[tid] = 0; s_pcnt[tid] = 0; s_pstart[tid] = 0; s_pi[tid] = -1;
+    s_best[tid] = -INFINITY; s_barg[tid] = -1; s_score[tid] = -INFINITY; s_creator[tid] = -1;
+    if (tid < p.Cmax) p.segnew[tokBase + tid] = -1;
   }
   __syncthreads();
 
-  if (!all_append) {
-    // ---- A1/A2: candidate pairs from the filter lists ----
-    if (tid < C) {
-      const int j = tid;
-      const float thr = p.thr_coeff * p.kbarNorm[(int64_t)u * p.Cmax + j] + 1e-5f;
-      float vmax_all = -INFINITY, vmax_ns = -INFINITY;
+  // ---- A1/A2: candidate pairs from the filter lists ----
+  if (tid < C) {
+    const int j = tid;
+    const float thr = p.thr_coeff * p.kbarNorm[tokBase + j] + 1e-5f;
+    float vmax_all = -INFINITY, vmax_ns = -INFINITY;
+    for (int sp = 0; sp < p.nsplit; ++sp) {
+      const int64_t o = (((int64_t)u * p.nsplit + sp) * p.Cmax + j) * kTopK;
+      for (int k = 0; k < kTopK; ++k) {
+        const int i = p.candI[o + k];
+        if (i < 0) break;
+        const float v = p.candV[o + k];
+        vmax_all = fmaxf(vmax_all, v);
+        if (i >= p.S) vmax_ns = fmaxf(vmax_ns, v);
+      }
+    }
+    const float cut_ns = vmax_ns - thr;     // merge candidates (rows >= S)
+    const float cut_all = vmax_all - thr;   // append-score candidates (all rows)
+    bool exh = !(vmax_ns > -INFINITY);
+    int cntc = 0;
+    for (int sp = 0; sp < p.nsplit && !exh; ++sp) {
+      const int64_t o = (((int64_t)u * p.nsplit + sp) * p.Cmax + j) * kTopK;
+      // a full list whose last entry is still above the cut may have dropped a candidate
+      if (p.candI[o + kTopK - 1] >= 0 && p.candV[o + kTopK - 1] >= cut_ns) exh = true;
+      for (int k = 0; k < kTopK; ++k) {
+        const int i = p.candI[o + k];
+        if (i < 0) break;
+        const float v = p.candV[o + k];
+        if ((i >= p.S && v >= cut_ns) || (n_a > 0 && v >= cut_all)) ++cntc;
+      }
+    }
+    if (cntc > kPairPerTok) exh = true;
+    int start = 0;
+    if (!exh) {
+      start = atomicAdd(&s_np, cntc);
+      if (start + cntc > kPairCap) exh = true;
+    }
+    if (!exh) {
+      int w = start;
       for (int sp = 0; sp < p.nsplit; ++sp) {
         const int64_t o = (((int64_t)u * p.nsplit + sp) * p.Cmax + j) * kTopK;
         for (int k = 0; k < kTopK; ++k) {
           const int i = p.candI[o + k];
           if (i < 0) break;
           const float v = p.candV[o + k];
-          vmax_all = fmaxf(vmax_all, v);
-          if (i >= p.S) vmax_ns = fmaxf(vmax_ns, v);
-        }
-      }
-      const float cut_ns = vmax_ns - thr;     // merge candidates (rows >= S)
-      const float cut_all = vmax_all - thr;   // append-score candidates (all rows)
-      bool exh = !(vmax_ns > -INFINITY);
-      int cntc = 0;
-      for (int sp = 0; sp < p.nsplit && !exh; ++sp) {
-        const int64_t o = (((int64_t)u * p.nsplit + sp) * p.Cmax + j) * kTopK;
-        if (p.candI[o + kTopK - 1] >= 0 && p.candV[o + kTopK - 1] >= fminf(cut_ns, cut_all)) exh = true;
-        for (int k = 0; k < kTopK; ++k) {
-          const int i = p.candI[o + k];
-          if (i < 0) break;
-          const float v = p.candV[o + k];
-          if ((i >= p.S && v >= cut_ns) || (n_a > 0 && v >= cut_all)) ++cntc;
-        }
-      }
-      if (cntc > kPairPerTok) exh = true;
-      int start = 0;
-      if (!exh) {
-        start = atomicAdd(&s_np, cntc);
-        if (start + cntc > kPairCap) exh = true;
-      }
-      if (!exh) {
-        int w = start;
-        for (int sp = 0; sp < p.nsplit; ++sp) {
-          const int64_t o = (((int64_t)u * p.nsplit + sp) * p.Cmax + j) * kTopK;
-          for (int k = 0; k < kTopK; ++k) {
-            const int i = p.candI[o + k];
-            if (i < 0) break;
-            const float v = p.candV[o + k];
-            if ((i >= p.S && v >= cut_ns) || (n_a > 0 && v >= cut_all)) {
-              s_prow[w] = i;
-              s_ptok[w] = (unsigned short)j;
-              ++w;
-            }
+          if ((i >= p.S && v >= cut_ns) || (n_a > 0 && v >= cut_all)) {
+            s_prow[w] = i;
+            s_ptok[w] = (unsigned short)j;
+            ++w;
           }
         }
-        s_pstart[j] = start;
-        s_pcnt[j] = cntc;
       }
-      s_exh[j] = exh ? 1 : 0;
+      s_pstart[j] = start;
+      s_pcnt[j] = cntc;
     }
-    __syncthreads();
-    // ---- A3: exact fp64 similarity of every candidate pair ----
-    const int np = min(s_np, kPairCap);
-    for (int q = tid; q < np; q += 256) {
-      const int j = s_ptok[q];
+    s_exh[j] = exh ? 1 : 0;
+  }
+  __syncthreads();
+  // ---- A3: exact fp64 similarity of every candidate pair ----
+  const int np = min(s_np, kPairCap);
+  for (int q = tid; q < np; q += 256) {
+    const int j = s_ptok[q];
+    const int i = s_prow[q];
+    if (s_exh[j]) continue;   // slots of tokens that fell back to the exhaustive path are unused
+    const double* kb = kbarU + (int64_t)j * D;
+    const double* sk = p.sumK + (rowBase + i) * D;
+    const double mu = p.kmu[rowBase + i], rs = p.krstd[rowBase + i];
+    double acc = 0.0;
+#pragma unroll 8
+    for (int x = 0; x < D; ++x) acc += kb[x] * (s_gamma[x] * ((sk[x] - mu) * rs) + s_beta[x]);
+    s_pval[q] = acc;
+  }
+  __syncthreads();
+  // ---- A4: per-token reduction (ties: lowest row) ----
+  if (tid < C && !s_exh[tid]) {
+    double score = -INFINITY, best = -INFINITY;
+    int barg = -1;
+    const int st0 = s_pstart[tid];
+    for (int q = st0; q < st0 + s_pcnt[tid]; ++q) {
+      const double v = s_pval[q];
       const int i = s_prow[q];
-      // pairs of tokens that fell back to the exhaustive path are skipped (their slots are unused)
-      if (s_exh[j]) continue;
-      const double* kb = kbarU + (int64_t)j * D;
+      if (v > score) score = v;
+      if (i >= p.S && (v > best || (v == best && i < barg))) { best = v; barg = i; }
+    }
+    s_score[tid] = score;
+    s_best[tid] = best;
+    s_barg[tid] = barg;
+  }
+  // ---- A5: exhaustive path: one warp per flagged token, one lane per row ----
+  for (int j = warp; j < C; j += 8) {
+    if (!s_exh[j]) continue;
+    const double* kb = kbarU + (int64_t)j * D;
+    double score = -INFINITY, best = -INFINITY;
+    int barg = 0x7fffffff;
+    for (int64_t i = lane; i < m; i += 32) {
       const double* sk = p.sumK + (rowBase + i) * D;
       const double mu = p.kmu[rowBase + i], rs = p.krstd[rowBase + i];
       double acc = 0.0;
-#pragma unroll 8
       for (int x = 0; x < D; ++x) acc += kb[x] * (s_gamma[x] * ((sk[x] - mu) * rs) + s_beta[x]);
-      s_pval[q] = acc;
+      if (acc > score) score = acc;
+      if (i >= p.S && acc > best) { best = acc; barg = (int)i; }
     }
-    __syncthreads();
-    // ---- A4: per-token reduction (ties: lowest row) ----
-    if (tid < C && !s_exh[tid]) {
-      double score = -INFINITY, best = -INFINITY;
-      int barg = -1;
-      const int st0 = s_pstart[tid];
-      for (int q = st0; q < st0 + s_pcnt[tid]; ++q) {
-        const double v = s_pval[q];
-        const int i = s_prow[q];
-        if (v > score) score = v;
-        if (i >= p.S && (v > best || (v == best && i < barg))) { best = v; barg = i; }
-      }
-      s_score[tid] = score;
-      s_best[tid] = best;
-      s_barg[tid] = barg;
-    }
-    // ---- A5: exhaustive path: one warp per flagged token, one lane per row ----
-    for (int j = warp; j < C; j += 8) {
-      if (!s_exh[j]) continue;
-      const double* kb = kbarU + (int64_t)j * D;
-      double score = -INFINITY, best = -INFINITY;
-      int barg = 0x7fffffff;
-      for (int64_t i = lane; i < m; i += 32) {
-        const double* sk = p.sumK + (rowBase + i) * D;
-        const double mu = p.kmu[rowBase + i], rs = p.krstd[rowBase + i];
-        double acc = 0.0;
-        for (int x = 0; x < D; ++x) acc += kb[x] * (s_gamma[x] * ((sk[x] - mu) * rs) + s_beta[x]);
-        if (acc > score) score = acc;
-        if (i >= p.S && acc > best) { best = acc; barg = (int)i; }
-      }
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const double os = __shfl_xor_sync(0xffffffffu, score, o);
-        const double ob = __shfl_xor_sync(0xffffffffu, best, o);
-        const int oa = __shfl_xor_sync(0xffffffffu, barg, o);
-        if (os > score) score = os;
-        if (ob > best || (ob == best && oa < barg)) { best = ob; barg = oa; }
-      }
-      if (lane == 0) { s_score[j] = score; s_best[j] = best; s_barg[j] = barg; }
+    for (int o = 16; o > 0; o >>= 1) {
+      const double os = __shfl_xor_sync(0xffffffffu, score, o);
+      const double ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oa = __shfl_xor_sync(0xffffffffu, barg, o);
+      if (os > score) score = os;
+      if (ob > best || (ob == best && oa < barg)) { best = ob; barg = oa; }
     }
-    __syncthreads();
-    // ---- B: append selection: the n_a smallest scores, ties to the smaller token index ----
-    if (n_a > 0) {
-      int rank = 0;
-      if (tid < C) {
-        const double sj = s_score[tid];
-        for (int jj = 0; jj < C; ++jj) {
-          const double so = s_score[jj];
-          rank += (so < sj || (so == sj && jj < tid)) ? 1 : 0;
-        }
-      }
-      __syncthreads();
-      if (tid < C) s_app[tid] = rank < n_a ? 1 : 0;
-      __syncthreads();
-      if (tid < C && s_app[tid]) {
-        int before = 0;
-        for (int jj = 0; jj < tid; ++jj) before += s_app[jj];
-        s_newrow[tid] = (int)m + before;
-      }
-      __syncthreads();
-    }
+    if (lane == 0) { s_score[j] = score; s_best[j] = best; s_barg[j] = barg; }
   }
-
-  // ---- C: create the appended rows ----
-  for (int j = warp; j < C; j += 8) {
-    if (!s_app[j]) continue;
-    const int64_t row = rowBase + s_newrow[j];
-    const double* kb = kbarU + (int64_t)j * D;
-    const __half* vr = ovU + (int64_t)j * D;
-    double kx[CH];
-    float vx[CH];
-    double v2 = 0.0;
-#pragma unroll
-    for (int i = 0; i < CH; ++i) {
-      const int x = lane + 32 * i;
-      kx[i] = kb[x];
-      vx[i] = __half2float(vr[x]);
-      v2 += (double)vx[i] * (double)vx[i];
-    }
-    double mu, rs;
-    row_stats<CH>(kx, D, p.ln_eps, mu, rs);
-    const double vnorm = sqrt(warp_sum_d(v2));
-    const double den = vnorm > p.norm_eps ? vnorm : p.norm_eps;
-#pragma unroll
-    for (int i = 0; i < CH; ++i) {
-      const int x = lane + 32 * i;
-      const double hat = s_gamma[x] * ((kx[i] - mu) * rs) + s_beta[x];
-      p.sumK[row * D + x] = kx[i];
-      p.sumV[row * D + x] = vx[i];
-      p.newhat64[((int64_t)u * p.Cmax + (s_newrow[j] - (int)m)) * D + x] = hat;
-      p.Khat[row * D + x] = __float2half_rn((float)hat);
-      const double vo = p.radius_on ? (vnorm * (double)vx[i] / den) : (double)vx[i];
-      p.Vhat[row * D + x] = __float2half_rn((float)vo);
-    }
-    if (lane == 0) {
-      p.rho[row] = (float)vnorm;
-      p.wsum[row] = 1.0;
-      p.cnt[row] = 1;
-      p.kmu[row] = mu;
-      p.krstd[row] = rs;
-      if (p.slotTok && p.b + j < p.Tassign) {
-        p.slotTok[(int64_t)u * p.Tassign + p.b + j] = s_newrow[j];
-        p.appTok[(int64_t)u * p.Tassign + p.b + j] = 1;
-      }
-    }
-  }
-  if (all_append) return;
   __syncthreads();
-
+  // ---- B: append selection: the n_a smallest scores, ties to the smaller token index ----
+  if (n_a > 0) {
+    int rank = 0;
+    if (tid < C) {
+      const double sj = s_score[tid];
+      for (int jj = 0; jj < C; ++jj) {
+        const double so = s_score[jj];
+        rank += (so < sj || (so == sj && jj < tid)) ? 1 : 0;
+      }
+      s_app[tid] = rank < n_a ? 1 : 0;
+    }
+    __syncthreads();
+    if (tid < C && s_app[tid]) {
+      int before = 0;
+      for (int jj = 0; jj < tid; ++jj) before += s_app[jj];
+      s_creator[before] = tid;          // rows are laid down in ascending token order
+    }
+    __syncthreads();
+  }
   // ---- D: merge target against s_+ (old rows: refined candidates; new rows: exact) ----
   if (tid < C && !s_app[tid]) {
     const double* kb = kbarU + (int64_t)tid * D;
     double best = s_best[tid];
     int arg = s_barg[tid];
     for (int a = 0; a < n_a; ++a) {
-      const double* nh = p.newhat64 + ((int64_t)u * p.Cmax + a) * D;
+      const int jc = s_creator[a];
+      const double* ka = kbarU + (int64_t)jc * D;
+      const double mu = p.kbarMu[tokBase + jc], rs = p.kbarRstd[tokBase + jc];
       double acc = 0.0;
 #pragma unroll 8
-      for (int x = 0; x < D; ++x) acc += kb[x] * nh[x];
+      for (int x = 0; x < D; ++x) acc += kb[x] * (s_gamma[x] * ((ka[x] - mu) * rs) + s_beta[x]);
       if (acc > best) { best = acc; arg = (int)m + a; }
     }
     s_pi[tid] = arg;
     atomicAdd(&s_nmerge, 1);
   }
   __syncthreads();
-  // ---- E: order merged tokens by (row, token) ----
-  if (tid < C && s_pi[tid] >= 0) {
+  // ---- E: order merged tokens by (row, token); publish ----
+  if (tid < C) {
     const int pj = s_pi[tid];
-    int ord = 0;
-    for (int jj = 0; jj < C; ++jj) {
-      const int po = s_pi[jj];
-      ord += (po >= 0 && (po < pj || (po == pj && jj < tid))) ? 1 : 0;
+    p.pi[tokBase + tid] = pj;
+    p.creator[tokBase + tid] = s_creator[tid];
+    if (pj >= 0) {
+      int ord = 0;
+      bool head = true;
+      for (int jj = 0; jj < C; ++jj) {
+        const int po = s_pi[jj];
+        ord += (po >= 0 && (po < pj || (po == pj && jj < tid))) ? 1 : 0;
+        if (po == pj && jj < tid) head = false;
+      }
+      p.sorted[tokBase + ord] = tid;
+      if (head && pj >= m) p.segnew[tokBase + (pj - (int)m)] = ord;
     }
-    s_sorted[ord] = tid;
   }
-  __syncthreads();
-  // ---- F: per-row accumulation in ascending token order, then readout refresh ----
-  const int nmerge = s_nmerge;
-  for (int q = warp; q < nmerge; q += 8) {
-    const int j0 = s_sorted[q];
-    const int rowi = s_pi[j0];
-    if (q > 0 && s_pi[s_sorted[q - 1]] == rowi) continue;   // not the head of its segment
+  if (tid == 0) p.nmerge[u] = s_nmerge;
+}
+
+// ------------------------------------------------------------------------------------------
+// 4. application: one warp per touched row
+
+struct FoldApplyParams {
+  const __half* ov;
+  const float* og;
+  int64_t unit_stride, gate_stride;
+  const double* kbar64;
+  const float *ln_w, *ln_b;
+  const int32_t *pi, *sorted, *creator, *segnew, *nmerge;
+  double* sumK; float* sumV; float* rho; double* wsum; int32_t* cnt; double *kmu, *krstd;
+  __half *Khat, *Vhat;
+  int32_t* slotTok; uint8_t* appTok;
+  int64_t Mcap, Tassign, m, b;
+  int C, Cmax, Hkv, n_append, all_append, radius_on;
+  double ln_eps, norm_eps;
+};
+
+template <int D>
+__global__ void __launch_bounds__(256) fold_apply_kernel(FoldApplyParams p) {
+  constexpr int CH = D / 32;
+  const int u = blockIdx.y, hk = u % p.Hkv;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int q = blockIdx.x * 8 + warp;
+  if (q >= p.C) return;
+  const int64_t tokBase = (int64_t)u * p.Cmax;
+  const int64_t rowBase = (int64_t)u * p.Mcap;
+  const double* kbarU = p.kbar64 + tokBase * D;
+  const __half* ovU = p.ov + (int64_t)u * p.unit_stride;
+  const float* ogU = p.og + (int64_t)u * p.gate_stride;
+  const int nmerge = p.all_append ? 0 : p.nmerge[u];
+  const int m = (int)p.m;
+
+  // task 0: the q-th appended row; task 1: the segment of an old row whose head sits at sorted[q]
+  for (int task = 0; task < 2; ++task) {
+    int rowi, seg, jc = -1;
+    if (task == 0) {
+      if (q >= p.n_append) continue;
+      rowi = m + q;
+      jc = p.all_append ? q : p.creator[tokBase + q];
+      seg = p.all_append ? -1 : p.segnew[tokBase + q];
+    } else {
+      if (q >= nmerge) continue;
+      const int j0 = p.sorted[tokBase + q];
+      rowi = p.pi[tokBase + j0];
+      if (rowi >= m) continue;                                              // new rows are task 0
+      if (q > 0 && p.pi[tokBase + p.sorted[tokBase + q - 1]] == rowi) continue;   // not a head
+      seg = q;
+    }
     const int64_t row = rowBase + rowi;
     double kx[CH];
     float vx[CH];
-#pragma unroll
-    for (int i = 0; i < CH; ++i) {
-      const int x = lane + 32 * i;
-      kx[i] = p.sumK[row * D + x];
-      vx[i] = p.sumV[row * D + x];
-    }
-    double wacc = p.wsum[row];
-    int nacc = p.cnt[row];
-    for (int qq = q; qq < nmerge; ++qq) {
-      const int j = s_sorted[qq];
-      if (s_pi[j] != rowi) break;
-      const float g = ogU[j];
-      const double* kb = kbarU + (int64_t)j * D;
-      const __half* vr = ovU + (int64_t)j * D;
+    double wacc, rad;
+    int nacc;
+    if (task == 0) {
+      const double* kb = kbarU + (int64_t)jc * D;
+      const __half* vr = ovU + (int64_t)jc * D;
+      double v2 = 0.0;
 #pragma unroll
       for (int i = 0; i < CH; ++i) {
         const int x = lane + 32 * i;
-        kx[i] += (double)g * kb[x];
-        vx[i] = fmaf(g, __half2float(vr[x]), vx[i]);
+        kx[i] = kb[x];
+        vx[i] = __half2float(vr[x]);
+        v2 += (double)vx[i] * (double)vx[i];
       }
-      wacc += (double)g;
-      nacc += 1;
-      if (lane == 0 && p.slotTok && p.b + j < p.Tassign) {
-        p.slotTok[(int64_t)u * p.Tassign + p.b + j] = rowi;
-        p.appTok[(int64_t)u * p.Tassign + p.b + j] = 0;
+      rad = (double)(float)sqrt(warp_sum_d(v2));   // the radius is kept in fp32
+      wacc = 1.0;
+      nacc = 1;
+      if (lane == 0 && p.slotTok && p.b + jc < p.Tassign) {
+        p.slotTok[(int64_t)u * p.Tassign + p.b + jc] = rowi;
+        p.appTok[(int64_t)u * p.Tassign + p.b + jc] = 1;
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < CH; ++i) {
+        const int x = lane + 32 * i;
+        kx[i] = p.sumK[row * D + x];
+        vx[i] = p.sumV[row * D + x];
+      }
+      wacc = p.wsum[row];
+      nacc = p.cnt[row];
+      rad = (double)p.rho[row];
+    }
+    if (seg >= 0) {
+      for (int qq = seg; qq < nmerge; ++qq) {
+        const int j = p.sorted[tokBase + qq];
+        if (p.pi[tokBase + j] != rowi) break;
+        const float g = ogU[j];
+        const double* kb = kbarU + (int64_t)j * D;
+        const __half* vr = ovU + (int64_t)j * D;
+#pragma unroll
+        for (int i = 0; i < CH; ++i) {
+          const int x = lane + 32 * i;
+          kx[i] += (double)g * kb[x];
+          vx[i] = fmaf(g, __half2float(vr[x]), vx[i]);
+        }
+        wacc += (double)g;
+        nacc += 1;
+        if (lane == 0 && p.slotTok && p.b + j < p.Tassign) {
+          p.slotTok[(int64_t)u * p.Tassign + p.b + j] = rowi;
+          p.appTok[(int64_t)u * p.Tassign + p.b + j] = 0;
+        }
       }
     }
     double mu, rs;
@@ -466,11 +489,10 @@ __global__ void __launch_bounds__(256) fold_update_kernel(FoldUpdateParams p) {
     for (int i = 0; i < CH; ++i) v2 += (double)vx[i] * (double)vx[i];
     const double vnorm = sqrt(warp_sum_d(v2));
     const double den = vnorm > p.norm_eps ? vnorm : p.norm_eps;
-    const double rad = (double)p.rho[row];
 #pragma unroll
     for (int i = 0; i < CH; ++i) {
       const int x = lane + 32 * i;
-      const double hat = s_gamma[x] * ((kx[i] - mu) * rs) + s_beta[x];
+      const double hat = (double)p.ln_w[hk * D + x] * ((kx[i] - mu) * rs) + (double)p.ln_b[hk * D + x];
       p.sumK[row * D + x] = kx[i];
       p.sumV[row * D + x] = vx[i];
       p.Khat[row * D + x] = __float2half_rn((float)hat);
@@ -478,6 +500,7 @@ __global__ void __launch_bounds__(256) fold_update_kernel(FoldUpdateParams p) {
       p.Vhat[row * D + x] = __float2half_rn((float)vo);
     }
     if (lane == 0) {
+      p.rho[row] = (float)rad;
       p.wsum[row] = wacc;
       p.cnt[row] = nacc;
       p.kmu[row] = mu;
@@ -486,7 +509,7 @@ __global__ void __launch_bounds__(256) fold_update_kernel(FoldUpdateParams p) {
   }
 }
 
-int launch_route_filter_tc(State* st, const FoldArgs& a, int nsplit, cudaStream_t s);
+int launch_route_filter_tc(State* st, int64_t m, int nsplit, cudaStream_t s);
 
 int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
   int launches = 0;
@@ -495,46 +518,65 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
     dim3 grid((C + 7) / 8, st->U);
     if (D == 128)
       kbar_kernel<128><<<grid, 256, 0, s>>>(a.ok, a.unit_stride, st->ln_w, st->ln_b, st->kbar64, st->kbarH,
-                                            st->kbarNorm, C, st->Cmax, st->Hkv, st->r, (double)st->ln_eps);
+                                            st->kbarNorm, st->kbarMu, st->kbarRstd, C, st->Cmax, st->CbarRows,
+                                            st->Hkv, st->r, (double)st->ln_eps);
     else
       kbar_kernel<64><<<grid, 256, 0, s>>>(a.ok, a.unit_stride, st->ln_w, st->ln_b, st->kbar64, st->kbarH,
-                                           st->kbarNorm, C, st->Cmax, st->Hkv, st->r, (double)st->ln_eps);
+                                           st->kbarNorm, st->kbarMu, st->kbarRstd, C, st->Cmax, st->CbarRows,
+                                           st->Hkv, st->r, (double)st->ln_eps);
     ++launches;
   }
   const bool all_append = a.first || a.n_append >= C;
-  int nsplit = 1;
   if (!all_append) {
-    // enough CTAs to fill the GPU, at least 128 rows per split
-    int64_t want = (2 * 148 + st->U - 1) / st->U;
-    int64_t maxs = (a.m + 127) / 128;
-    nsplit = (int)(want < maxs ? want : maxs);
+    // enough CTAs to fill the GPU, at least 256 rows per split
+    int64_t want = (148 + st->U - 1) / st->U;
+    int64_t maxs = (a.m + 255) / 256;
+    int nsplit = (int)(want < maxs ? want : maxs);
     if (nsplit < 1) nsplit = 1;
     if (nsplit > st->nsplitRoute) nsplit = st->nsplitRoute;
-    dim3 grid(nsplit, st->U);
-    if (D == 128)
-      route_filter_simt_kernel<128><<<grid, 256, 0, s>>>(st->kbarH, st->Khat, st->candV, st->candI, C, st->Cmax,
-                                                         st->Mcap, a.m, nsplit);
-    else
-      route_filter_simt_kernel<64><<<grid, 256, 0, s>>>(st->kbarH, st->Khat, st->candV, st->candI, C, st->Cmax,
-                                                        st->Mcap, a.m, nsplit);
+    if (st->flags & KVM_FLAG_SIMT_ROUTING) {
+      dim3 grid(nsplit, st->U);
+      if (D == 128)
+        route_filter_simt_kernel<128><<<grid, 256, 0, s>>>(st->kbarH, st->Khat, st->candV, st->candI, C, st->Cmax,
+                                                           st->CbarRows, st->Mcap, a.m, nsplit);
+      else
+        route_filter_simt_kernel<64><<<grid, 256, 0, s>>>(st->kbarH, st->Khat, st->candV, st->candI, C, st->Cmax,
+                                                          st->CbarRows, st->Mcap, a.m, nsplit);
+      ++launches;
+    } else {
+      launches += launch_route_filter_tc(st, a.m, nsplit, s);
+    }
+    FoldDecideParams p;
+    p.kbar64 = st->kbar64; p.kbarNorm = st->kbarNorm; p.kbarMu = st->kbarMu; p.kbarRstd = st->kbarRstd;
+    p.candV = st->candV; p.candI = st->candI; p.ln_w = st->ln_w; p.ln_b = st->ln_b;
+    p.sumK = st->sumK; p.kmu = st->kmu; p.krstd = st->krstd;
+    p.pi = st->foldPi; p.sorted = st->foldSorted; p.creator = st->foldCreator; p.segnew = st->foldSegNew;
+    p.nmerge = st->foldNMerge;
+    p.Mcap = st->Mcap; p.m = a.m;
+    p.C = C; p.Cmax = st->Cmax; p.Hkv = st->Hkv; p.S = st->S; p.n_append = a.n_append; p.nsplit = nsplit;
+    // fp16 rounding of both operands: |err| <= (2u + u^2) |a|.|b| with u = 2^-11, plus slack for
+    // fp16 subnormals and for the fp32 accumulation (2^-13 |a|.|b| covers 128 truncating adds);
+    // candidates lie within twice that of the approximate maximum.
+    p.thr_coeff = 2.0f * (1.0f / 1024.0f + 1.0f / 8192.0f) * st->sim_norm_bound;
+    if (D == 128) fold_decide_kernel<128><<<st->U, 256, 0, s>>>(p);
+    else fold_decide_kernel<64><<<st->U, 256, 0, s>>>(p);
     ++launches;
   }
-  FoldUpdateParams p;
-  p.ov = a.ov; p.og = a.og; p.unit_stride = a.unit_stride; p.gate_stride = a.gate_stride;
-  p.kbar64 = st->kbar64; p.kbarNorm = st->kbarNorm; p.newhat64 = st->newhat64;
-  p.candV = st->candV; p.candI = st->candI; p.ln_w = st->ln_w; p.ln_b = st->ln_b;
-  p.sumK = st->sumK; p.sumV = st->sumV; p.rho = st->rho; p.wsum = st->wsum; p.cnt = st->cnt;
-  p.kmu = st->kmu; p.krstd = st->krstd; p.Khat = st->Khat; p.Vhat = st->Vhat;
-  p.slotTok = st->slotTok; p.appTok = st->appTok;
-  p.Mcap = st->Mcap; p.Tassign = st->Tassign; p.m = a.m; p.b = a.b;
-  p.C = C; p.Cmax = st->Cmax; p.Hkv = st->Hkv; p.S = st->S; p.n_append = a.n_append; p.nsplit = nsplit;
-  p.first = a.first ? 1 : 0; p.radius_on = (st->flags & KVM_FLAG_NO_RADIUS) ? 0 : 1;
-  p.ln_eps = (double)st->ln_eps; p.norm_eps = (double)st->norm_eps;
-  // fp16 rounding of both operands: |err| <= (2u + u^2) |a|.|b| with u = 2^-11, plus subnormal
-  // and fp32 accumulation slack; candidates lie within twice that of the approximate maximum.
-  p.thr_coeff = 2.0f * (1.0f / 1024.0f + 1.0f / 65536.0f) * st->sim_norm_bound;
-  if (D == 128) fold_update_kernel<128><<<st->U, 256, 0, s>>>(p);
-  else fold_update_kernel<64><<<st->U, 256, 0, s>>>(p);
+  FoldApplyParams q;
+  q.ov = a.ov; q.og = a.og; q.unit_stride = a.unit_stride; q.gate_stride = a.gate_stride;
+  q.kbar64 = st->kbar64; q.ln_w = st->ln_w; q.ln_b = st->ln_b;
+  q.pi = st->foldPi; q.sorted = st->foldSorted; q.creator = st->foldCreator; q.segnew = st->foldSegNew;
+  q.nmerge = st->foldNMerge;
+  q.sumK = st->sumK; q.sumV = st->sumV; q.rho = st->rho; q.wsum = st->wsum; q.cnt = st->cnt;
+  q.kmu = st->kmu; q.krstd = st->krstd; q.Khat = st->Khat; q.Vhat = st->Vhat;
+  q.slotTok = st->slotTok; q.appTok = st->appTok;
+  q.Mcap = st->Mcap; q.Tassign = st->Tassign; q.m = a.m; q.b = a.b;
+  q.C = C; q.Cmax = st->Cmax; q.Hkv = st->Hkv; q.n_append = a.n_append; q.all_append = all_append ? 1 : 0;
+  q.radius_on = (st->flags & KVM_FLAG_NO_RADIUS) ? 0 : 1;
+  q.ln_eps = (double)st->ln_eps; q.norm_eps = (double)st->norm_eps;
+  dim3 grid((C + 7) / 8, st->U);
+  if (D == 128) fold_apply_kernel<128><<<grid, 256, 0, s>>>(q);
+  else fold_apply_kernel<64><<<grid, 256, 0, s>>>(q);
   ++launches;
   return launches;
 }

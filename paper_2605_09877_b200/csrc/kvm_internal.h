@@ -58,9 +58,11 @@ struct State {
   float2* ropeCS;                // [Tcall, r/2] (cos, sin)
   // ---- fold scratch (device) ----
   double* kbar64;                // [U, Cmax, d]
-  __half* kbarH;                 // [U, Cmax, d]
+  __half* kbarH;                 // [U, CbarRows, d]
   float* kbarNorm;               // [U, Cmax]
-  double* newhat64;              // [U, Cmax, d]  LN_s of rows appended in this fold
+  int CbarRows;                  // rows per unit of kbarH (Cmax rounded up to the 128-row MMA tile)
+  double *kbarMu, *kbarRstd;     // [U, Cmax]  statistics of LN_s(kbar_j): the key of a row created by j
+  int32_t *foldPi, *foldSorted, *foldCreator, *foldSegNew, *foldNMerge;  // decisions of the current fold
   int nsplitRoute;               // splits the routing filter may use
   float* candV;                  // [U, nsplitRoute, Cmax, kTopK]
   int32_t* candI;
@@ -106,6 +108,7 @@ struct AttnArgs {
 int launch_attn_simt(State* st, const AttnArgs& a, cudaStream_t s);
 int launch_attn_tc(State* st, const AttnArgs& a, cudaStream_t s);
 bool setup_attn_tc(State* st);   // encodes the tensor maps, raises the shared-memory limits
+bool setup_route_tc(State* st);
 
 struct FoldArgs {
   const __half *ok, *ov;         // overflow block rows: unit u at ok + u*unit_stride (elements), C rows

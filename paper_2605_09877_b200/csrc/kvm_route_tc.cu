@@ -1,0 +1,211 @@
+// Routing filter on the tensor cores: approximate similarities S = Kbar . LN_s(S^K)^T between
+// the overflow block's memory keys (fp16, up to 256 tokens = two 128-row M tiles) and a split of
+// the state's readout keys, reduced on the fly to the K best rows per token (Section 3.2
+// "Append" score and "Merge" arg max; the exact decision is taken later in fp64 on these
+// candidates only).
+//
+//   warp 0      TMA producer: the Kbar tiles once, then 128-row tiles of K_hat in a 3-stage ring
+//   warp 1      MMA issuer: per key tile one 128x128x(d) product per M tile into a
+//               double-buffered TMEM accumulator (tcgen05.mma kind::f16)
+//   warps 2-9   epilogue: one thread per token row; tcgen05.ld of its 128 similarities and an
+//               insertion-sorted top-K list in registers
+// All waits are bounded (error word + normal teardown on expiry).
+#include "kvm_internal.h"
+#include "tc_common.cuh"
+
+namespace kvm {
+
+struct RouteTcParams {
+  float* candV;
+  int32_t* candI;
+  int32_t* status;
+  int64_t m;
+  int C, Cmax, nsplit;
+};
+
+template <int D>
+struct RouteTcCfg {
+  static constexpr int NS = 3, MT = 2;
+  static constexpr int NKB = D / 64;
+  static constexpr int BOX_BYTES = 128 * 128;
+  static constexpr int TILE_BYTES = NKB * BOX_BYTES;
+  static constexpr int OFF_A = 0;
+  static constexpr int OFF_B = OFF_A + MT * TILE_BYTES;
+  static constexpr int OFF_BAR = OFF_B + NS * TILE_BYTES;
+  static constexpr int SMEM_BYTES = (OFF_BAR + 256 + 1024) > 120 * 1024 ? (OFF_BAR + 256 + 1024) : 120 * 1024;
+  static constexpr uint32_t TMEM_COLS = 512;   // [buffer][M tile] x 128 columns
+};
+
+enum { RB_AFULL = 0, RB_BFULL = 1, RB_BFREE = 4, RB_SFULL = 7, RB_ACCFREE = 9, RB_COUNT = 11 };
+
+template <int D>
+__global__ void __launch_bounds__(320, 1)
+route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                       const RouteTcParams p) {
+  using Cfg = RouteTcCfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sA = base + Cfg::OFF_A;
+  uint8_t* sB = base + Cfg::OFF_B;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(base + Cfg::OFF_BAR);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + RB_COUNT);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int split = blockIdx.x, u = blockIdx.y;
+  const int mt_used = (p.C + 127) / 128;
+  int64_t per = (p.m + p.nsplit - 1) / p.nsplit;
+  per = (per + 127) / 128 * 128;
+  const int64_t i0 = (int64_t)split * per;
+  const int64_t i1 = min(p.m, i0 + per);
+  const int ntiles = i1 > i0 ? (int)((i1 - i0 + 127) / 128) : 0;
+
+  if (tid == 0) {
+    tc::mbar_init(&bars[RB_AFULL], 1);
+    for (int s = 0; s < Cfg::NS; ++s) {
+      tc::mbar_init(&bars[RB_BFULL + s], 1);
+      tc::mbar_init(&bars[RB_BFREE + s], 1);
+    }
+    tc::mbar_init(&bars[RB_SFULL + 0], 1);
+    tc::mbar_init(&bars[RB_SFULL + 1], 1);
+    tc::mbar_init(&bars[RB_ACCFREE + 0], 4 * mt_used);
+    tc::mbar_init(&bars[RB_ACCFREE + 1], 4 * mt_used);
+    *abort_flag = 0;
+    tc::fence_barrier_init();
+  }
+  if (warp == 1) {
+    tc::tmem_alloc(tmem_slot, Cfg::TMEM_COLS);
+    tc::tmem_relinquish();
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      tc::prefetch_tmap(&mapA); tc::prefetch_tmap(&mapB);
+      tc::mbar_expect_tx(&bars[RB_AFULL], mt_used * Cfg::TILE_BYTES);
+      for (int mt = 0; mt < mt_used; ++mt)
+        for (int kb = 0; kb < Cfg::NKB; ++kb)
+          tc::tma_load_3d(sA + mt * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, &mapA, &bars[RB_AFULL], kb * 64, mt * 128, u);
+      for (int j = 0; j < ntiles; ++j) {
+        const int s = j % Cfg::NS;
+        if (*abort_flag) break;
+        if (j >= Cfg::NS && !tc::mbar_wait(&bars[RB_BFREE + s], ((j / Cfg::NS) - 1) & 1)) {
+          atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; break;
+        }
+        tc::mbar_expect_tx(&bars[RB_BFULL + s], Cfg::TILE_BYTES);
+        for (int kb = 0; kb < Cfg::NKB; ++kb)
+          tc::tma_load_3d(sB + s * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, &mapB, &bars[RB_BFULL + s], kb * 64,
+                          (int)(i0 + (int64_t)j * 128), u);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t IDESC = tc::idesc_f16(128, 128, false);
+      const uint32_t aA = tc::smem_u32(sA), aB = tc::smem_u32(sB);
+      bool dead = !tc::mbar_wait(&bars[RB_AFULL], 0);
+      for (int j = 0; j < ntiles && !dead; ++j) {
+        const int s = j % Cfg::NS, buf = j & 1;
+        if (*abort_flag) { dead = true; break; }
+        if (!tc::mbar_wait(&bars[RB_BFULL + s], (j / Cfg::NS) & 1)) { dead = true; break; }
+        if (j >= 2 && !tc::mbar_wait(&bars[RB_ACCFREE + buf], ((j >> 1) - 1) & 1)) { dead = true; break; }
+        tc::tc_fence_after();
+        for (int mt = 0; mt < mt_used; ++mt) {
+          const uint32_t dS = tmem + buf * 256 + mt * 128;
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks) {
+            const uint32_t off = (ks / 4) * Cfg::BOX_BYTES + (ks % 4) * 32;
+            tc::mma_f16_ss(dS, tc::smem_desc_sw128(aA + mt * Cfg::TILE_BYTES + off, 16, 1024),
+                           tc::smem_desc_sw128(aB + s * Cfg::TILE_BYTES + off, 16, 1024), IDESC, ks > 0);
+          }
+        }
+        tc::mma_commit(&bars[RB_SFULL + buf]);
+        tc::mma_commit(&bars[RB_BFREE + s]);
+      }
+      if (dead) { atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; }
+    }
+  } else {
+    const int e = warp - 2;
+    const int mt = e >> 2;
+    if (mt < mt_used) {
+      const int quarter = warp & 3;
+      const int tok = mt * 128 + quarter * 32 + lane;
+      const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+      float tv[kTopK];
+      int ti[kTopK];
+#pragma unroll
+      for (int k = 0; k < kTopK; ++k) { tv[k] = -INFINITY; ti[k] = -1; }
+      for (int j = 0; j < ntiles; ++j) {
+        const int buf = j & 1;
+        if (!tc::mbar_wait(&bars[RB_SFULL + buf], (j >> 1) & 1)) {
+          atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; break;
+        }
+        tc::tc_fence_after();
+        const uint32_t ts = tmem + lane_base + buf * 256 + mt * 128;
+        const int64_t row0 = i0 + (int64_t)j * 128;
+        const int nvalid = (int)min((int64_t)128, i1 - row0);
+#pragma unroll 1
+        for (int c4 = 0; c4 < 4; ++c4) {
+          uint32_t r[32];
+          tc::tmem_ld32(ts + c4 * 32, r);
+          tc::tmem_wait_ld();
+          if (c4 == 3) {   // all 128 columns are in registers: the accumulator may be overwritten
+            tc::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(&bars[RB_ACCFREE + buf]);
+          }
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float v = __uint_as_float(r[i]);
+            const int c = c4 * 32 + i;
+            if (c < nvalid && v > tv[kTopK - 1]) {
+              tv[kTopK - 1] = v;
+              ti[kTopK - 1] = (int)row0 + c;
+#pragma unroll
+              for (int k = kTopK - 1; k > 0; --k) {
+                if (tv[k] > tv[k - 1]) {
+                  const float fv = tv[k]; tv[k] = tv[k - 1]; tv[k - 1] = fv;
+                  const int iv = ti[k]; ti[k] = ti[k - 1]; ti[k - 1] = iv;
+                }
+              }
+            }
+          }
+        }
+      }
+      if (tok < p.C) {
+        const int64_t o = (((int64_t)u * p.nsplit + split) * p.Cmax + tok) * kTopK;
+#pragma unroll
+        for (int k = 0; k < kTopK; ++k) { p.candV[o + k] = tv[k]; p.candI[o + k] = ti[k]; }
+      }
+    }
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc::tmem_dealloc(tmem, Cfg::TMEM_COLS);
+  }
+}
+
+int launch_route_filter_tc(State* st, int64_t m, int nsplit, cudaStream_t s) {
+  RouteTcParams p;
+  p.candV = st->candV; p.candI = st->candI; p.status = st->status; p.m = m;
+  p.C = st->C; p.Cmax = st->Cmax; p.nsplit = nsplit;
+  const CUtensorMap* tm = reinterpret_cast<const CUtensorMap*>(st->tmaps);
+  dim3 grid(nsplit, st->U);
+  if (st->d == 128) route_filter_tc_kernel<128><<<grid, 320, RouteTcCfg<128>::SMEM_BYTES, s>>>(tm[5], tm[1], p);
+  else route_filter_tc_kernel<64><<<grid, 320, RouteTcCfg<64>::SMEM_BYTES, s>>>(tm[5], tm[1], p);
+  return 1;
+}
+
+bool setup_route_tc(State* st) {
+  CUtensorMap* tm = reinterpret_cast<CUtensorMap*>(st->tmaps);
+  if (!encode_tmap_rows(&tm[5], st->kbarH, st->d, st->CbarRows, st->U, 128)) return false;
+  if (cudaFuncSetAttribute(route_filter_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, RouteTcCfg<128>::SMEM_BYTES) != cudaSuccess) return false;
+  if (cudaFuncSetAttribute(route_filter_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, RouteTcCfg<64>::SMEM_BYTES) != cudaSuccess) return false;
+  return true;
+}
+
+}  // namespace kvm
