@@ -195,6 +195,11 @@ kvm_status_t kvm_state_reset(kvm_state_t* state);
 kvm_status_t kvm_profile_enable(kvm_state_t* state, int32_t on);
 kvm_status_t kvm_profile_read(kvm_state_t* state, double* ms, int64_t* groups);
 
+/* Debug counters of the fold since the state was created (synchronises the stream):
+ * out[0] overflow tokens whose routing fell back to the exhaustive fp64 scan, out[1] candidate
+ * (token, row) pairs refined in fp64, out[2] overflow tokens routed.  32-bit device counters. */
+kvm_status_t kvm_debug_counters(kvm_state_t* state, int64_t* out, void* cuda_stream);
+
 /* Number of kernels the library has launched for this state so far (host counter). */
 int64_t kvm_launch_count(const kvm_state_t* state);
 

@@ -249,7 +249,7 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   A(s.foldPi, U * Cm); A(s.foldSorted, U * Cm); A(s.foldCreator, U * Cm); A(s.foldSegNew, U * Cm); A(s.foldNMerge, U);
   A(s.candV, U * (size_t)s.nsplitRoute * Cm * kTopK); A(s.candI, U * (size_t)s.nsplitRoute * Cm * kTopK);
   A(s.decPart, (size_t)s.B * s.Hq * s.nsplitDec * (d + 2)); A(s.decQ, (size_t)s.B * s.Hq * d);
-  A(s.status, (size_t)1);
+  A(s.status, (size_t)16);   // [0] status word, [1..3] fold debug counters
   if (s.Tassign > 0) { A(s.slotTok, U * (size_t)s.Tassign); A(s.appTok, U * (size_t)s.Tassign); }
 #undef A
   if (rc == KVM_OK && s.Tassign > 0 && cudaMemset(s.slotTok, 0xff, U * (size_t)s.Tassign * sizeof(int32_t)) != cudaSuccess) rc = KVM_ERR_CUDA;
@@ -280,6 +280,17 @@ KVM_API kvm_status_t kvm_state_free(kvm_state_t* ks) {
     for (const ProfBracket& br : *v) { cudaEventDestroy(br.a); cudaEventDestroy(br.b); }
   free_all(ks);
   delete ks;
+  return KVM_OK;
+}
+
+KVM_API kvm_status_t kvm_debug_counters(kvm_state_t* ks, int64_t* out, void* cuda_stream) {
+  if (!ks || !out) return KVM_ERR_INVALID_ARG;
+  DeviceGuard guard(ks->s.device);
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  int32_t w[16];
+  if (cudaMemcpyAsync(w, ks->s.status, sizeof(w), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return KVM_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return KVM_ERR_CUDA;
+  for (int i = 0; i < 3; ++i) out[i] = w[1 + i];
   return KVM_OK;
 }
 

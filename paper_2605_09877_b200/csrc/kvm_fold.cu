@@ -168,6 +168,7 @@ struct FoldDecideParams {
   const double* sumK;
   const double *kmu, *krstd;
   int32_t *pi, *sorted, *creator, *segnew, *nmerge;   // outputs, [U, Cmax] (nmerge [U])
+  int32_t* counters;   // debug: [0] tokens on the exhaustive path, [1] candidate pairs, [2] tokens decided
   int64_t Mcap, m;
   int C, Cmax, Hkv, S, n_append, nsplit;
   float thr_coeff;
@@ -176,10 +177,33 @@ struct FoldDecideParams {
 constexpr int kPairCap = 1536;
 constexpr int kPairPerTok = 24;
 
+constexpr int kDecideThreads = 512;
+constexpr int kDecideWarps = kDecideThreads / 32;
+
+// One filter list (kTopK entries) of token j in split sp: two 16-byte loads each for values / rows.
+__device__ __forceinline__ void load_cand_list(const float* candV, const int32_t* candI, int64_t o, float (&v)[kTopK],
+                                               int (&i)[kTopK]) {
+  static_assert(kTopK == 8, "list loads are written for 8 entries");
+  const float4 v0 = *reinterpret_cast<const float4*>(candV + o), v1 = *reinterpret_cast<const float4*>(candV + o + 4);
+  const int4 i0 = *reinterpret_cast<const int4*>(candI + o), i1 = *reinterpret_cast<const int4*>(candI + o + 4);
+  v[0] = v0.x; v[1] = v0.y; v[2] = v0.z; v[3] = v0.w; v[4] = v1.x; v[5] = v1.y; v[6] = v1.z; v[7] = v1.w;
+  i[0] = i0.x; i[1] = i0.y; i[2] = i0.z; i[3] = i0.w; i[4] = i1.x; i[5] = i1.y; i[6] = i1.z; i[7] = i1.w;
+}
+
+// kb . LN_s(row) with the row's statistics given; channels are strided over the lanes of a warp.
+template <int CH>
+__device__ __forceinline__ double warp_sim(const double (&kb)[CH], const double* __restrict__ row, double mu, double rs,
+                                           const double (&g)[CH], const double (&b)[CH], int lane) {
+  double acc = 0.0;
+#pragma unroll
+  for (int i = 0; i < CH; ++i) acc += kb[i] * (g[i] * ((row[lane + 32 * i] - mu) * rs) + b[i]);
+  return warp_sum_d(acc);
+}
+
 template <int D>
-__global__ void __launch_bounds__(256) fold_decide_kernel(FoldDecideParams p) {
-  __shared__ double s_gamma[D], s_beta[D];
-  __shared__ double s_score[kMaxBlock], s_best[kMaxBlock];
+__global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideParams p) {
+  constexpr int CH = D / 32;
+  __shared__ double s_score[kMaxBlock], s_best[kMaxBlock], s_cmu[kMaxBlock], s_crs[kMaxBlock];
   __shared__ int s_barg[kMaxBlock], s_pi[kMaxBlock], s_creator[kMaxBlock];
   __shared__ int s_pstart[kMaxBlock], s_pcnt[kMaxBlock];
   __shared__ unsigned char s_app[kMaxBlock], s_exh[kMaxBlock];
@@ -197,9 +221,11 @@ __global__ void __launch_bounds__(256) fold_decide_kernel(FoldDecideParams p) {
   const int64_t rowBase = (int64_t)u * p.Mcap;
   const int64_t tokBase = (int64_t)u * p.Cmax;
 
-  for (int x = tid; x < D; x += 256) {
-    s_gamma[x] = (double)p.ln_w[hk * D + x];
-    s_beta[x] = (double)p.ln_b[hk * D + x];
+  double gam[CH], bet[CH];
+#pragma unroll
+  for (int i = 0; i < CH; ++i) {
+    gam[i] = (double)p.ln_w[hk * D + lane + 32 * i];
+    bet[i] = (double)p.ln_b[hk * D + lane + 32 * i];
   }
   if (tid == 0) { s_np = 0; s_nmerge = 0; }
   if (tid < kMaxBlock) {
@@ -213,31 +239,32 @@ __global__ void __launch_bounds__(256) fold_decide_kernel(FoldDecideParams p) {
   if (tid < C) {
     const int j = tid;
     const float thr = p.thr_coeff * p.kbarNorm[tokBase + j] + 1e-5f;
+    const int64_t o0 = ((int64_t)u * p.nsplit * p.Cmax + j) * kTopK;
+    const int64_t ostep = (int64_t)p.Cmax * kTopK;
     float vmax_all = -INFINITY, vmax_ns = -INFINITY;
+#pragma unroll 4
     for (int sp = 0; sp < p.nsplit; ++sp) {
-      const int64_t o = (((int64_t)u * p.nsplit + sp) * p.Cmax + j) * kTopK;
+      float v[kTopK]; int i[kTopK];
+      load_cand_list(p.candV, p.candI, o0 + sp * ostep, v, i);
+#pragma unroll
       for (int k = 0; k < kTopK; ++k) {
-        const int i = p.candI[o + k];
-        if (i < 0) break;
-        const float v = p.candV[o + k];
-        vmax_all = fmaxf(vmax_all, v);
-        if (i >= p.S) vmax_ns = fmaxf(vmax_ns, v);
+        if (i[k] >= 0) vmax_all = fmaxf(vmax_all, v[k]);
+        if (i[k] >= p.S) vmax_ns = fmaxf(vmax_ns, v[k]);
       }
     }
     const float cut_ns = vmax_ns - thr;     // merge candidates (rows >= S)
     const float cut_all = vmax_all - thr;   // append-score candidates (all rows)
     bool exh = !(vmax_ns > -INFINITY);
     int cntc = 0;
-    for (int sp = 0; sp < p.nsplit && !exh; ++sp) {
-      const int64_t o = (((int64_t)u * p.nsplit + sp) * p.Cmax + j) * kTopK;
+#pragma unroll 4
+    for (int sp = 0; sp < p.nsplit; ++sp) {
+      float v[kTopK]; int i[kTopK];
+      load_cand_list(p.candV, p.candI, o0 + sp * ostep, v, i);
       // a full list whose last entry is still above the cut may have dropped a candidate
-      if (p.candI[o + kTopK - 1] >= 0 && p.candV[o + kTopK - 1] >= cut_ns) exh = true;
-      for (int k = 0; k < kTopK; ++k) {
-        const int i = p.candI[o + k];
-        if (i < 0) break;
-        const float v = p.candV[o + k];
-        if ((i >= p.S && v >= cut_ns) || (n_a > 0 && v >= cut_all)) ++cntc;
-      }
+      if (i[kTopK - 1] >= 0 && v[kTopK - 1] >= cut_ns) exh = true;
+#pragma unroll
+      for (int k = 0; k < kTopK; ++k)
+        if (i[k] >= 0 && ((i[k] >= p.S && v[k] >= cut_ns) || (n_a > 0 && v[k] >= cut_all))) ++cntc;
     }
     if (cntc > kPairPerTok) exh = true;
     int start = 0;
@@ -248,13 +275,12 @@ __global__ void __launch_bounds__(256) fold_decide_kernel(FoldDecideParams p) {
     if (!exh) {
       int w = start;
       for (int sp = 0; sp < p.nsplit; ++sp) {
-        const int64_t o = (((int64_t)u * p.nsplit + sp) * p.Cmax + j) * kTopK;
+        float v[kTopK]; int i[kTopK];
+        load_cand_list(p.candV, p.candI, o0 + sp * ostep, v, i);
+#pragma unroll
         for (int k = 0; k < kTopK; ++k) {
-          const int i = p.candI[o + k];
-          if (i < 0) break;
-          const float v = p.candV[o + k];
-          if ((i >= p.S && v >= cut_ns) || (n_a > 0 && v >= cut_all)) {
-            s_prow[w] = i;
+          if (i[k] >= 0 && ((i[k] >= p.S && v[k] >= cut_ns) || (n_a > 0 && v[k] >= cut_all))) {
+            s_prow[w] = i[k];
             s_ptok[w] = (unsigned short)j;
             ++w;
           }
@@ -266,19 +292,27 @@ __global__ void __launch_bounds__(256) fold_decide_kernel(FoldDecideParams p) {
     s_exh[j] = exh ? 1 : 0;
   }
   __syncthreads();
-  // ---- A3: exact fp64 similarity of every candidate pair ----
+  // ---- A3: exact fp64 similarity of every candidate pair, one warp per pair, two in flight ----
   const int np = min(s_np, kPairCap);
-  for (int q = tid; q < np; q += 256) {
-    const int j = s_ptok[q];
-    const int i = s_prow[q];
-    if (s_exh[j]) continue;   // slots of tokens that fell back to the exhaustive path are unused
-    const double* kb = kbarU + (int64_t)j * D;
-    const double* sk = p.sumK + (rowBase + i) * D;
-    const double mu = p.kmu[rowBase + i], rs = p.krstd[rowBase + i];
-    double acc = 0.0;
-#pragma unroll 8
-    for (int x = 0; x < D; ++x) acc += kb[x] * (s_gamma[x] * ((sk[x] - mu) * rs) + s_beta[x]);
-    s_pval[q] = acc;
+  for (int q = warp; q < np; q += 2 * kDecideWarps) {
+    const int q2 = q + kDecideWarps;
+    const bool two = q2 < np;
+    const int j0 = s_ptok[q], i0 = s_prow[q];
+    const int j1 = two ? s_ptok[q2] : j0, i1 = two ? s_prow[q2] : i0;
+    double kb0[CH], kb1[CH];
+#pragma unroll
+    for (int i = 0; i < CH; ++i) {
+      kb0[i] = kbarU[(int64_t)j0 * D + lane + 32 * i];
+      kb1[i] = kbarU[(int64_t)j1 * D + lane + 32 * i];
+    }
+    const double mu0 = p.kmu[rowBase + i0], rs0 = p.krstd[rowBase + i0];
+    const double mu1 = p.kmu[rowBase + i1], rs1 = p.krstd[rowBase + i1];
+    const double a0 = warp_sim<CH>(kb0, p.sumK + (rowBase + i0) * D, mu0, rs0, gam, bet, lane);
+    const double a1 = warp_sim<CH>(kb1, p.sumK + (rowBase + i1) * D, mu1, rs1, gam, bet, lane);
+    if (lane == 0) {
+      s_pval[q] = a0;
+      if (two) s_pval[q2] = a1;
+    }
   }
   __syncthreads();
   // ---- A4: per-token reduction (ties: lowest row) ----
@@ -296,36 +330,28 @@ __global__ void __launch_bounds__(256) fold_decide_kernel(FoldDecideParams p) {
     s_best[tid] = best;
     s_barg[tid] = barg;
   }
-  // ---- A5: exhaustive path: one warp per flagged token, one lane per row ----
-  for (int j = warp; j < C; j += 8) {
+  // ---- A5: exhaustive path for flagged tokens: one warp per token, rows in sequence ----
+  for (int j = warp; j < C; j += kDecideWarps) {
     if (!s_exh[j]) continue;
-    const double* kb = kbarU + (int64_t)j * D;
+    double kb[CH];
+#pragma unroll
+    for (int i = 0; i < CH; ++i) kb[i] = kbarU[(int64_t)j * D + lane + 32 * i];
     double score = -INFINITY, best = -INFINITY;
-    int barg = 0x7fffffff;
-    for (int64_t i = lane; i < m; i += 32) {
-      const double* sk = p.sumK + (rowBase + i) * D;
-      const double mu = p.kmu[rowBase + i], rs = p.krstd[rowBase + i];
-      double acc = 0.0;
-      for (int x = 0; x < D; ++x) acc += kb[x] * (s_gamma[x] * ((sk[x] - mu) * rs) + s_beta[x]);
+    int barg = -1;
+    for (int64_t i = 0; i < m; ++i) {
+      const double acc = warp_sim<CH>(kb, p.sumK + (rowBase + i) * D, p.kmu[rowBase + i], p.krstd[rowBase + i], gam, bet, lane);
       if (acc > score) score = acc;
       if (i >= p.S && acc > best) { best = acc; barg = (int)i; }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const double os = __shfl_xor_sync(0xffffffffu, score, o);
-      const double ob = __shfl_xor_sync(0xffffffffu, best, o);
-      const int oa = __shfl_xor_sync(0xffffffffu, barg, o);
-      if (os > score) score = os;
-      if (ob > best || (ob == best && oa < barg)) { best = ob; barg = oa; }
     }
     if (lane == 0) { s_score[j] = score; s_best[j] = best; s_barg[j] = barg; }
   }
   __syncthreads();
   // ---- B: append selection: the n_a smallest scores, ties to the smaller token index ----
   if (n_a > 0) {
-    int rank = 0;
     if (tid < C) {
+      int rank = 0;
       const double sj = s_score[tid];
+#pragma unroll 8
       for (int jj = 0; jj < C; ++jj) {
         const double so = s_score[jj];
         rank += (so < sj || (so == sj && jj < tid)) ? 1 : 0;
@@ -335,27 +361,33 @@ __global__ void __launch_bounds__(256) fold_decide_kernel(FoldDecideParams p) {
     __syncthreads();
     if (tid < C && s_app[tid]) {
       int before = 0;
+#pragma unroll 8
       for (int jj = 0; jj < tid; ++jj) before += s_app[jj];
       s_creator[before] = tid;          // rows are laid down in ascending token order
+      s_cmu[before] = p.kbarMu[tokBase + tid];
+      s_crs[before] = p.kbarRstd[tokBase + tid];
     }
     __syncthreads();
   }
-  // ---- D: merge target against s_+ (old rows: refined candidates; new rows: exact) ----
-  if (tid < C && !s_app[tid]) {
-    const double* kb = kbarU + (int64_t)tid * D;
-    double best = s_best[tid];
-    int arg = s_barg[tid];
-    for (int a = 0; a < n_a; ++a) {
-      const int jc = s_creator[a];
-      const double* ka = kbarU + (int64_t)jc * D;
-      const double mu = p.kbarMu[tokBase + jc], rs = p.kbarRstd[tokBase + jc];
-      double acc = 0.0;
-#pragma unroll 8
-      for (int x = 0; x < D; ++x) acc += kb[x] * (s_gamma[x] * ((ka[x] - mu) * rs) + s_beta[x]);
-      if (acc > best) { best = acc; arg = (int)m + a; }
+  // ---- D: merge target against s_+ (old rows: refined candidates; new rows: exact), warp per token ----
+  for (int j = warp; j < C; j += kDecideWarps) {
+    if (s_app[j]) continue;
+    double best = s_best[j];
+    int arg = s_barg[j];
+    if (n_a > 0) {
+      double kb[CH];
+#pragma unroll
+      for (int i = 0; i < CH; ++i) kb[i] = kbarU[(int64_t)j * D + lane + 32 * i];
+#pragma unroll 2
+      for (int a = 0; a < n_a; ++a) {
+        const double acc = warp_sim<CH>(kb, kbarU + (int64_t)s_creator[a] * D, s_cmu[a], s_crs[a], gam, bet, lane);
+        if (acc > best) { best = acc; arg = (int)m + a; }
+      }
     }
-    s_pi[tid] = arg;
-    atomicAdd(&s_nmerge, 1);
+    if (lane == 0) {
+      s_pi[j] = arg;
+      atomicAdd(&s_nmerge, 1);
+    }
   }
   __syncthreads();
   // ---- E: order merged tokens by (row, token); publish ----
@@ -366,6 +398,7 @@ __global__ void __launch_bounds__(256) fold_decide_kernel(FoldDecideParams p) {
     if (pj >= 0) {
       int ord = 0;
       bool head = true;
+#pragma unroll 8
       for (int jj = 0; jj < C; ++jj) {
         const int po = s_pi[jj];
         ord += (po >= 0 && (po < pj || (po == pj && jj < tid))) ? 1 : 0;
@@ -375,7 +408,14 @@ __global__ void __launch_bounds__(256) fold_decide_kernel(FoldDecideParams p) {
       if (head && pj >= m) p.segnew[tokBase + (pj - (int)m)] = ord;
     }
   }
-  if (tid == 0) p.nmerge[u] = s_nmerge;
+  if (tid == 0) {
+    p.nmerge[u] = s_nmerge;
+    int nexh = 0;
+    for (int j = 0; j < C; ++j) nexh += s_exh[j];
+    atomicAdd(&p.counters[0], nexh);
+    atomicAdd(&p.counters[1], min(s_np, kPairCap));
+    atomicAdd(&p.counters[2], C);
+  }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -552,14 +592,15 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
     p.sumK = st->sumK; p.kmu = st->kmu; p.krstd = st->krstd;
     p.pi = st->foldPi; p.sorted = st->foldSorted; p.creator = st->foldCreator; p.segnew = st->foldSegNew;
     p.nmerge = st->foldNMerge;
+    p.counters = st->status + 1;
     p.Mcap = st->Mcap; p.m = a.m;
     p.C = C; p.Cmax = st->Cmax; p.Hkv = st->Hkv; p.S = st->S; p.n_append = a.n_append; p.nsplit = nsplit;
     // fp16 rounding of both operands: |err| <= (2u + u^2) |a|.|b| with u = 2^-11, plus slack for
     // fp16 subnormals and for the fp32 accumulation (2^-13 |a|.|b| covers 128 truncating adds);
     // candidates lie within twice that of the approximate maximum.
     p.thr_coeff = 2.0f * (1.0f / 1024.0f + 1.0f / 8192.0f) * st->sim_norm_bound;
-    if (D == 128) fold_decide_kernel<128><<<st->U, 256, 0, s>>>(p);
-    else fold_decide_kernel<64><<<st->U, 256, 0, s>>>(p);
+    if (D == 128) fold_decide_kernel<128><<<st->U, kDecideThreads, 0, s>>>(p);
+    else fold_decide_kernel<64><<<st->U, kDecideThreads, 0, s>>>(p);
     ++launches;
   }
   FoldApplyParams q;

@@ -25,7 +25,7 @@ FLAG_NO_RADIUS, FLAG_RECORD_ASSIGN, FLAG_SIMT_ATTENTION, FLAG_SIMT_ROUTING = 1, 
 EXPORTS = ["kvm_plan_capacity", "kvm_state_create", "kvm_prefill", "kvm_decode_step", "kvm_prefill_host",
            "kvm_decode_step_host", "kvm_state_free", "kvm_state_info", "kvm_state_check", "kvm_state_export",
            "kvm_debug_assignments", "kvm_launch_count", "kvm_status_string", "kvm_state_reset",
-           "kvm_profile_enable", "kvm_profile_read"]
+           "kvm_profile_enable", "kvm_profile_read", "kvm_debug_counters"]
 
 
 class KVMError(RuntimeError):
@@ -88,6 +88,8 @@ def _load():
     L.kvm_profile_enable.argtypes = [vp, C.c_int32]
     L.kvm_profile_read.restype = C.c_int
     L.kvm_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    L.kvm_debug_counters.restype = C.c_int
+    L.kvm_debug_counters.argtypes = [vp, C.POINTER(C.c_int64), vp]
     L.kvm_launch_count.restype = C.c_int64
     L.kvm_launch_count.argtypes = [vp]
     L.kvm_status_string.restype = C.c_char_p
@@ -251,6 +253,13 @@ class KVMState:
             raise KVMError(rc, "kvm_profile_read")
         names = ("ingest", "attention", "fold", "decode")
         return {names[i]: (ms[i], n[i]) for i in range(4)}
+
+    def debug_counters(self, stream=None):
+        out = (C.c_int64 * 3)()
+        rc = lib.kvm_debug_counters(self._h, out, _stream_ptr(stream))
+        if rc != KVM_OK:
+            raise KVMError(rc, "kvm_debug_counters")
+        return dict(exhaustive_tokens=out[0], candidate_pairs=out[1], tokens=out[2])
 
     def launch_count(self):
         return lib.kvm_launch_count(self._h)
