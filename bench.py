@@ -244,6 +244,8 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--simt", action="store_true", help="time the scalar-core cross-check kernels")
+    ap.add_argument("--tokens", type=int, default=0,
+                    help="prefill workloads: shorten the sequence to this many tokens (small cases for ncu captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -253,6 +255,8 @@ def main():
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     wl, mode = workload(args.workload)
+    if args.tokens and mode == "prefill":
+        wl = wl.scaled(T=args.tokens, name=f"{wl.name}-T{args.tokens}")
     pk = peaks()
     W, K = max(args.warmup, 3), args.steps
     g = kvm.growth(wl.growth, wl.fixed_slots, wl.sqrt_coeff)

@@ -595,10 +595,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
     p.counters = st->status + 1;
     p.Mcap = st->Mcap; p.m = a.m;
     p.C = C; p.Cmax = st->Cmax; p.Hkv = st->Hkv; p.S = st->S; p.n_append = a.n_append; p.nsplit = nsplit;
-    // fp16 rounding of both operands: |err| <= (2u + u^2) |a|.|b| with u = 2^-11, plus slack for
-    // fp16 subnormals and for the fp32 accumulation (2^-13 |a|.|b| covers 128 truncating adds);
-    // candidates lie within twice that of the approximate maximum.
-    p.thr_coeff = 2.0f * (1.0f / 1024.0f + 1.0f / 8192.0f) * st->sim_norm_bound;
+    p.thr_coeff = route_thr_coeff(st);
     if (D == 128) fold_decide_kernel<128><<<st->U, kDecideThreads, 0, s>>>(p);
     else fold_decide_kernel<64><<<st->U, kDecideThreads, 0, s>>>(p);
     ++launches;

@@ -109,6 +109,11 @@ int launch_attn_simt(State* st, const AttnArgs& a, cudaStream_t s);
 int launch_attn_tc(State* st, const AttnArgs& a, cudaStream_t s);
 bool setup_attn_tc(State* st);   // encodes the tensor maps, raises the shared-memory limits
 bool setup_route_tc(State* st);
+// Width of the candidate window of the routing filter per unit of ||kbar_j||: twice the bound on the
+// error of an fp16 x fp16 -> fp32 dot product against LN_s rows.  fp16 rounding of both operands
+// gives |err| <= (2u + u^2) |a|.|b| with u = 2^-11; 2^-13 |a|.|b| more covers fp16 subnormals and
+// 128 truncating fp32 additions.
+inline float route_thr_coeff(const State* st) { return 2.0f * (1.0f / 1024.0f + 1.0f / 8192.0f) * st->sim_norm_bound; }
 
 struct FoldArgs {
   const __half *ok, *ov;         // overflow block rows: unit u at ok + u*unit_stride (elements), C rows

@@ -1,14 +1,18 @@
 // Routing filter on the tensor cores: approximate similarities S = Kbar . LN_s(S^K)^T between
 // the overflow block's memory keys (fp16, up to 256 tokens = two 128-row M tiles) and a split of
-// the state's readout keys, reduced on the fly to the K best rows per token (Section 3.2
-// "Append" score and "Merge" arg max; the exact decision is taken later in fp64 on these
-// candidates only).
+// the state's readout keys, reduced on the fly to the rows whose similarity lies within the
+// rounding bound of the row maximum (Section 3.2 "Append" score and "Merge" arg max; the exact
+// decision is taken later in fp64 on these candidates only).  The split is streamed twice:
+// pass 1 keeps the running maximum per token (one FMNMX per element), pass 2 repeats the
+// products and collects the few elements above (maximum - bound).  The tensor work doubles but
+// the epilogue, which is the bottleneck of a 128 x 128 x d tile, stays at ~2 instructions per
+// element instead of a sorted insertion.
 //
 //   warp 0      TMA producer: the Kbar tiles once, then 128-row tiles of K_hat in a 3-stage ring
 //   warp 1      MMA issuer: per key tile one 128x128x(d) product per M tile into a
 //               double-buffered TMEM accumulator (tcgen05.mma kind::f16)
-//   warps 2-9   epilogue: one thread per token row; tcgen05.ld of its 128 similarities and an
-//               insertion-sorted top-K list in registers
+//   warps 2-9   epilogue: one thread per token row; tcgen05.ld of its 128 similarities, running
+//               maximum (pass 1) / candidate list of at most kTopK rows (pass 2) in registers
 // All waits are bounded (error word + normal teardown on expiry).
 #include "kvm_internal.h"
 #include "tc_common.cuh"
@@ -19,8 +23,10 @@ struct RouteTcParams {
   float* candV;
   int32_t* candI;
   int32_t* status;
+  const float* kbarNorm;   // [U, Cmax] upper bound of ||kbar_j||
+  float thr_coeff;         // candidate window = thr_coeff * ||kbar_j|| + 1e-5
   int64_t m;
-  int C, Cmax, nsplit;
+  int C, Cmax, nsplit, S;
 };
 
 template <int D>
@@ -59,6 +65,7 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
   const int64_t i0 = (int64_t)split * per;
   const int64_t i1 = min(p.m, i0 + per);
   const int ntiles = i1 > i0 ? (int)((i1 - i0 + 127) / 128) : 0;
+  const int nsteps = 2 * ntiles;   // every tile is visited in pass 1 and again in pass 2
 
   if (tid == 0) {
     tc::mbar_init(&bars[RB_AFULL], 1);
@@ -89,8 +96,9 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
       for (int mt = 0; mt < mt_used; ++mt)
         for (int kb = 0; kb < Cfg::NKB; ++kb)
           tc::tma_load_3d(sA + mt * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, &mapA, &bars[RB_AFULL], kb * 64, mt * 128, u);
-      for (int j = 0; j < ntiles; ++j) {
+      for (int j = 0; j < nsteps; ++j) {
         const int s = j % Cfg::NS;
+        const int jt = j >= ntiles ? j - ntiles : j;
         if (*abort_flag) break;
         if (j >= Cfg::NS && !tc::mbar_wait(&bars[RB_BFREE + s], ((j / Cfg::NS) - 1) & 1)) {
           atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; break;
@@ -98,7 +106,7 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
         tc::mbar_expect_tx(&bars[RB_BFULL + s], Cfg::TILE_BYTES);
         for (int kb = 0; kb < Cfg::NKB; ++kb)
           tc::tma_load_3d(sB + s * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, &mapB, &bars[RB_BFULL + s], kb * 64,
-                          (int)(i0 + (int64_t)j * 128), u);
+                          (int)(i0 + (int64_t)jt * 128), u);
       }
     }
   } else if (warp == 1) {
@@ -106,7 +114,7 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
       constexpr uint32_t IDESC = tc::idesc_f16(128, 128, false);
       const uint32_t aA = tc::smem_u32(sA), aB = tc::smem_u32(sB);
       bool dead = !tc::mbar_wait(&bars[RB_AFULL], 0);
-      for (int j = 0; j < ntiles && !dead; ++j) {
+      for (int j = 0; j < nsteps && !dead; ++j) {
         const int s = j % Cfg::NS, buf = j & 1;
         if (*abort_flag) { dead = true; break; }
         if (!tc::mbar_wait(&bars[RB_BFULL + s], (j / Cfg::NS) & 1)) { dead = true; break; }
@@ -133,51 +141,77 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
       const int quarter = warp & 3;
       const int tok = mt * 128 + quarter * 32 + lane;
       const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-      float tv[kTopK];
-      int ti[kTopK];
+      float cv[kTopK];
+      int ci[kTopK];
 #pragma unroll
-      for (int k = 0; k < kTopK; ++k) { tv[k] = -INFINITY; ti[k] = -1; }
-      for (int j = 0; j < ntiles; ++j) {
+      for (int k = 0; k < kTopK; ++k) { cv[k] = -INFINITY; ci[k] = -1; }
+      int ncand = 0;
+      float mx = -INFINITY;        // pass 1: running maximum over rows >= S of this split
+      float cut = INFINITY;        // pass 2: collect elements >= cut
+      const float thr = (tok < p.C) ? p.thr_coeff * p.kbarNorm[(int64_t)u * p.Cmax + tok] + 1e-5f : 0.f;
+      for (int j = 0; j < nsteps; ++j) {
         const int buf = j & 1;
+        const bool pass2 = j >= ntiles;
+        const int jt = pass2 ? j - ntiles : j;
+        if (j == ntiles) cut = mx - thr;
         if (!tc::mbar_wait(&bars[RB_SFULL + buf], (j >> 1) & 1)) {
           atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; break;
         }
         tc::tc_fence_after();
         const uint32_t ts = tmem + lane_base + buf * 256 + mt * 128;
-        const int64_t row0 = i0 + (int64_t)j * 128;
+        const int64_t row0 = i0 + (int64_t)jt * 128;
         const int nvalid = (int)min((int64_t)128, i1 - row0);
+        const bool plain = nvalid == 128 && row0 >= p.S;   // no masking needed in this tile
 #pragma unroll 1
-        for (int c4 = 0; c4 < 4; ++c4) {
-          uint32_t r[32];
-          tc::tmem_ld32(ts + c4 * 32, r);
+        for (int h = 0; h < 2; ++h) {
+          uint32_t r[64];
+          tc::tmem_ld32(ts + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
+          tc::tmem_ld32(ts + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
           tc::tmem_wait_ld();
-          if (c4 == 3) {   // all 128 columns are in registers: the accumulator may be overwritten
+          if (h == 1) {   // all 128 columns are in registers: the accumulator may be overwritten
             tc::tc_fence_before();
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(&bars[RB_ACCFREE + buf]);
           }
+          if (!pass2) {
+            if (plain) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float v = __uint_as_float(r[i]);
-            const int c = c4 * 32 + i;
-            if (c < nvalid && v > tv[kTopK - 1]) {
-              tv[kTopK - 1] = v;
-              ti[kTopK - 1] = (int)row0 + c;
+              for (int i = 0; i < 64; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
+            } else {
 #pragma unroll
-              for (int k = kTopK - 1; k > 0; --k) {
-                if (tv[k] > tv[k - 1]) {
-                  const float fv = tv[k]; tv[k] = tv[k - 1]; tv[k - 1] = fv;
-                  const int iv = ti[k]; ti[k] = ti[k - 1]; ti[k - 1] = iv;
+              for (int i = 0; i < 64; ++i) {
+                const int c = h * 64 + i;
+                if (c < nvalid && row0 + c >= p.S) mx = fmaxf(mx, __uint_as_float(r[i]));
+              }
+            }
+          } else {
+            float hm = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 64; ++i) hm = fmaxf(hm, __uint_as_float(r[i]));
+            if (hm >= cut) {   // rare: at least one candidate (or a masked element) in this half tile
+#pragma unroll
+              for (int i = 0; i < 64; ++i) {
+                const int c = h * 64 + i;
+                const float v = __uint_as_float(r[i]);
+                if (v >= cut && c < nvalid) {
+                  if (ncand < kTopK) {
+#pragma unroll
+                    for (int k = 0; k < kTopK; ++k)
+                      if (k == ncand) { cv[k] = v; ci[k] = (int)row0 + c; }
+                  }
+                  ++ncand;
                 }
               }
             }
           }
         }
       }
+      // more candidates than the list holds: mark the list so that the decision kernel scans all rows
+      if (ncand > kTopK) cv[kTopK - 1] = INFINITY;
       if (tok < p.C) {
         const int64_t o = (((int64_t)u * p.nsplit + split) * p.Cmax + tok) * kTopK;
 #pragma unroll
-        for (int k = 0; k < kTopK; ++k) { p.candV[o + k] = tv[k]; p.candI[o + k] = ti[k]; }
+        for (int k = 0; k < kTopK; ++k) { p.candV[o + k] = cv[k]; p.candI[o + k] = ci[k]; }
       }
     }
   }
@@ -192,7 +226,8 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
 int launch_route_filter_tc(State* st, int64_t m, int nsplit, cudaStream_t s) {
   RouteTcParams p;
   p.candV = st->candV; p.candI = st->candI; p.status = st->status; p.m = m;
-  p.C = st->C; p.Cmax = st->Cmax; p.nsplit = nsplit;
+  p.C = st->C; p.Cmax = st->Cmax; p.nsplit = nsplit; p.S = st->S;
+  p.kbarNorm = st->kbarNorm; p.thr_coeff = route_thr_coeff(st);
   const CUtensorMap* tm = reinterpret_cast<const CUtensorMap*>(st->tmaps);
   dim3 grid(nsplit, st->U);
   if (st->d == 128) route_filter_tc_kernel<128><<<grid, 320, RouteTcCfg<128>::SMEM_BYTES, s>>>(tm[5], tm[1], p);
