@@ -93,7 +93,9 @@ __global__ void __launch_bounds__(256) route_filter_simt_kernel(const __half* __
                                                                 const __half* __restrict__ Khat,
                                                                 float* __restrict__ candV,
                                                                 int32_t* __restrict__ candI, int C, int Cmax,
-                                                                int CbarRows, int64_t Mcap, int64_t m, int nsplit) {
+                                                                int CbarRows, int64_t Mcap, int64_t m, int nsplit,
+                                                                const float* __restrict__ kbarNorm, float thr_coeff,
+                                                                int S) {
   __shared__ __half2 sH[32 * (D / 2)];
   const int split = blockIdx.x, u = blockIdx.y;
   const int j = threadIdx.x;
@@ -149,9 +151,22 @@ __global__ void __launch_bounds__(256) route_filter_simt_kernel(const __half* __
     }
   }
   if (active) {
+    // same output format as the tensor-core filter: candidate rows within the window of the split's
+    // maximum over rows >= S, that maximum, and the candidate count (kTopK + 1 = overflow)
     const int64_t o = (((int64_t)u * nsplit + split) * Cmax + j) * kTopK;
+    float mx = -INFINITY;
 #pragma unroll
-    for (int k = 0; k < kTopK; ++k) { candV[o + k] = tv[k]; candI[o + k] = ti[k]; }
+    for (int k = 0; k < kTopK; ++k) if (ti[k] >= S) mx = fmaxf(mx, tv[k]);
+    const float cut = mx - (thr_coeff * kbarNorm[(int64_t)u * Cmax + j] + 1e-5f);
+    int n = 0;
+#pragma unroll
+    for (int k = 0; k < kTopK; ++k) {
+      const bool in = ti[k] >= 0 && tv[k] >= cut;
+      candI[o + k] = in ? ti[k] : -1;
+      n += in ? 1 : 0;
+    }
+    candV[o] = mx;
+    candV[o + 1] = (float)(n == kTopK ? kTopK + 1 : n);
   }
 }
 
@@ -180,13 +195,10 @@ constexpr int kPairPerTok = 24;
 constexpr int kDecideThreads = 512;
 constexpr int kDecideWarps = kDecideThreads / 32;
 
-// One filter list (kTopK entries) of token j in split sp: two 16-byte loads each for values / rows.
-__device__ __forceinline__ void load_cand_list(const float* candV, const int32_t* candI, int64_t o, float (&v)[kTopK],
-                                               int (&i)[kTopK]) {
+// The candidate rows (kTopK entries, -1 = none) of one token in one split: two 16-byte loads.
+__device__ __forceinline__ void load_cand_rows(const int32_t* candI, int64_t o, int (&i)[kTopK]) {
   static_assert(kTopK == 8, "list loads are written for 8 entries");
-  const float4 v0 = *reinterpret_cast<const float4*>(candV + o), v1 = *reinterpret_cast<const float4*>(candV + o + 4);
   const int4 i0 = *reinterpret_cast<const int4*>(candI + o), i1 = *reinterpret_cast<const int4*>(candI + o + 4);
-  v[0] = v0.x; v[1] = v0.y; v[2] = v0.z; v[3] = v0.w; v[4] = v1.x; v[5] = v1.y; v[6] = v1.z; v[7] = v1.w;
   i[0] = i0.x; i[1] = i0.y; i[2] = i0.z; i[3] = i0.w; i[4] = i1.x; i[5] = i1.y; i[6] = i1.z; i[7] = i1.w;
 }
 
@@ -241,30 +253,24 @@ __global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideP
     const float thr = p.thr_coeff * p.kbarNorm[tokBase + j] + 1e-5f;
     const int64_t o0 = ((int64_t)u * p.nsplit * p.Cmax + j) * kTopK;
     const int64_t ostep = (int64_t)p.Cmax * kTopK;
-    float vmax_all = -INFINITY, vmax_ns = -INFINITY;
+    // a split keeps its candidates when its own maximum is within the window of the global one;
+    // sink rows (< S) only matter for the append score and are kept whenever rows are appended
+    float gmax = -INFINITY;
 #pragma unroll 4
-    for (int sp = 0; sp < p.nsplit; ++sp) {
-      float v[kTopK]; int i[kTopK];
-      load_cand_list(p.candV, p.candI, o0 + sp * ostep, v, i);
-#pragma unroll
-      for (int k = 0; k < kTopK; ++k) {
-        if (i[k] >= 0) vmax_all = fmaxf(vmax_all, v[k]);
-        if (i[k] >= p.S) vmax_ns = fmaxf(vmax_ns, v[k]);
-      }
-    }
-    const float cut_ns = vmax_ns - thr;     // merge candidates (rows >= S)
-    const float cut_all = vmax_all - thr;   // append-score candidates (all rows)
-    bool exh = !(vmax_ns > -INFINITY);
+    for (int sp = 0; sp < p.nsplit; ++sp) gmax = fmaxf(gmax, p.candV[o0 + sp * ostep]);
+    const float gcut = gmax - thr;
+    bool exh = !(gmax > -INFINITY);
     int cntc = 0;
 #pragma unroll 4
     for (int sp = 0; sp < p.nsplit; ++sp) {
-      float v[kTopK]; int i[kTopK];
-      load_cand_list(p.candV, p.candI, o0 + sp * ostep, v, i);
-      // a full list whose last entry is still above the cut may have dropped a candidate
-      if (i[kTopK - 1] >= 0 && v[kTopK - 1] >= cut_ns) exh = true;
+      const float2 hd = *reinterpret_cast<const float2*>(p.candV + o0 + sp * ostep);
+      int i[kTopK];
+      load_cand_rows(p.candI, o0 + sp * ostep, i);
+      const bool keep = hd.x >= gcut;
+      if (hd.y > (float)kTopK && (keep || (n_a > 0 && sp == 0))) exh = true;   // list overflowed
 #pragma unroll
       for (int k = 0; k < kTopK; ++k)
-        if (i[k] >= 0 && ((i[k] >= p.S && v[k] >= cut_ns) || (n_a > 0 && v[k] >= cut_all))) ++cntc;
+        if (i[k] >= 0 && (i[k] < p.S ? n_a > 0 : keep)) ++cntc;
     }
     if (cntc > kPairPerTok) exh = true;
     int start = 0;
@@ -275,11 +281,12 @@ __global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideP
     if (!exh) {
       int w = start;
       for (int sp = 0; sp < p.nsplit; ++sp) {
-        float v[kTopK]; int i[kTopK];
-        load_cand_list(p.candV, p.candI, o0 + sp * ostep, v, i);
+        const bool keep = p.candV[o0 + sp * ostep] >= gcut;
+        int i[kTopK];
+        load_cand_rows(p.candI, o0 + sp * ostep, i);
 #pragma unroll
         for (int k = 0; k < kTopK; ++k) {
-          if (i[k] >= 0 && ((i[k] >= p.S && v[k] >= cut_ns) || (n_a > 0 && v[k] >= cut_all))) {
+          if (i[k] >= 0 && (i[k] < p.S ? n_a > 0 : keep)) {
             s_prow[w] = i[k];
             s_ptok[w] = (unsigned short)j;
             ++w;
@@ -578,10 +585,12 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
       dim3 grid(nsplit, st->U);
       if (D == 128)
         route_filter_simt_kernel<128><<<grid, 256, 0, s>>>(st->kbarH, st->Khat, st->candV, st->candI, C, st->Cmax,
-                                                           st->CbarRows, st->Mcap, a.m, nsplit);
+                                                           st->CbarRows, st->Mcap, a.m, nsplit, st->kbarNorm,
+                                                           route_thr_coeff(st), st->S);
       else
         route_filter_simt_kernel<64><<<grid, 256, 0, s>>>(st->kbarH, st->Khat, st->candV, st->candI, C, st->Cmax,
-                                                          st->CbarRows, st->Mcap, a.m, nsplit);
+                                                          st->CbarRows, st->Mcap, a.m, nsplit, st->kbarNorm,
+                                                          route_thr_coeff(st), st->S);
       ++launches;
     } else {
       launches += launch_route_filter_tc(st, a.m, nsplit, s);

@@ -12,7 +12,10 @@
 //   warp 1      MMA issuer: per key tile one 128x128x(d) product per M tile into a
 //               double-buffered TMEM accumulator (tcgen05.mma kind::f16)
 //   warps 2-9   epilogue: one thread per token row; tcgen05.ld of its 128 similarities, running
-//               maximum (pass 1) / candidate list of at most kTopK rows (pass 2) in registers
+//               maximum (pass 1) / list of at most kTopK candidate rows (pass 2) in registers.
+// Output per (unit, split, token): candI[0..kTopK) candidate rows in ascending order (-1 = none),
+// candV[0] = the split's maximum over rows >= S, candV[1] = number of candidates found (more than
+// kTopK = the list overflowed and the decision kernel scans all rows for that token).
 // All waits are bounded (error word + normal teardown on expiry).
 #include "kvm_internal.h"
 #include "tc_common.cuh"
@@ -141,13 +144,12 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
       const int quarter = warp & 3;
       const int tok = mt * 128 + quarter * 32 + lane;
       const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-      float cv[kTopK];
       int ci[kTopK];
 #pragma unroll
-      for (int k = 0; k < kTopK; ++k) { cv[k] = -INFINITY; ci[k] = -1; }
+      for (int k = 0; k < kTopK; ++k) ci[k] = -1;
       int ncand = 0;
       float mx = -INFINITY;        // pass 1: running maximum over rows >= S of this split
-      float cut = INFINITY;        // pass 2: collect elements >= cut
+      float cut = INFINITY;        // pass 2: collect rows whose similarity is >= cut
       const float thr = (tok < p.C) ? p.thr_coeff * p.kbarNorm[(int64_t)u * p.Cmax + tok] + 1e-5f : 0.f;
       for (int j = 0; j < nsteps; ++j) {
         const int buf = j & 1;
@@ -159,59 +161,62 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
         }
         tc::tc_fence_after();
         const uint32_t ts = tmem + lane_base + buf * 256 + mt * 128;
-        const int64_t row0 = i0 + (int64_t)jt * 128;
+        const int row0 = (int)(i0 + (int64_t)jt * 128);
         const int nvalid = (int)min((int64_t)128, i1 - row0);
-        const bool plain = nvalid == 128 && row0 >= p.S;   // no masking needed in this tile
+        // pass 1 ignores the sink rows (< S) and the rows past the end of the split; pass 2 only the latter
+        const int lo = pass2 ? 0 : max(0, p.S - row0);
+        const bool plain = nvalid == 128 && lo == 0;
 #pragma unroll 1
-        for (int h = 0; h < 2; ++h) {
-          uint32_t r[64];
-          tc::tmem_ld32(ts + h * 64, *reinterpret_cast<uint32_t(*)[32]>(&r[0]));
-          tc::tmem_ld32(ts + h * 64 + 32, *reinterpret_cast<uint32_t(*)[32]>(&r[32]));
+        for (int c4 = 0; c4 < 4; ++c4) {
+          uint32_t r[32];
+          tc::tmem_ld32(ts + c4 * 32, r);
           tc::tmem_wait_ld();
-          if (h == 1) {   // all 128 columns are in registers: the accumulator may be overwritten
+          if (c4 == 3) {   // all 128 columns are in registers: the accumulator may be overwritten
             tc::tc_fence_before();
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(&bars[RB_ACCFREE + buf]);
           }
+          uint32_t vm = 0xffffffffu;   // columns of this chunk that count
+          if (!plain) {
+            const int a = min(32, max(0, lo - c4 * 32)), b = min(32, max(0, nvalid - c4 * 32));
+            vm = (b <= a) ? 0u : ((b == 32 ? 0xffffffffu : ((1u << b) - 1u)) & ~((1u << a) - 1u));
+          }
           if (!pass2) {
+            float cm = -INFINITY;
             if (plain) {
 #pragma unroll
-              for (int i = 0; i < 64; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
+              for (int i = 0; i < 32; ++i) cm = fmaxf(cm, __uint_as_float(r[i]));
             } else {
 #pragma unroll
-              for (int i = 0; i < 64; ++i) {
-                const int c = h * 64 + i;
-                if (c < nvalid && row0 + c >= p.S) mx = fmaxf(mx, __uint_as_float(r[i]));
-              }
+              for (int i = 0; i < 32; ++i) cm = fmaxf(cm, ((vm >> i) & 1u) ? __uint_as_float(r[i]) : -INFINITY);
             }
+            mx = fmaxf(mx, cm);
           } else {
-            float hm = -INFINITY;
+            uint32_t hit = 0u;
 #pragma unroll
-            for (int i = 0; i < 64; ++i) hm = fmaxf(hm, __uint_as_float(r[i]));
-            if (hm >= cut) {   // rare: at least one candidate (or a masked element) in this half tile
+            for (int i = 0; i < 32; ++i) hit |= (__uint_as_float(r[i]) >= cut) ? (1u << i) : 0u;
+            hit &= vm;
+            while (hit) {   // rare per lane: about one candidate per token and split
+              const int bit = __ffs(hit) - 1;
+              hit &= hit - 1;
+              const int idx = row0 + c4 * 32 + bit;
+              if (ncand < kTopK) {
 #pragma unroll
-              for (int i = 0; i < 64; ++i) {
-                const int c = h * 64 + i;
-                const float v = __uint_as_float(r[i]);
-                if (v >= cut && c < nvalid) {
-                  if (ncand < kTopK) {
-#pragma unroll
-                    for (int k = 0; k < kTopK; ++k)
-                      if (k == ncand) { cv[k] = v; ci[k] = (int)row0 + c; }
-                  }
-                  ++ncand;
-                }
+                for (int k = 0; k < kTopK; ++k)
+                  if (k == ncand) ci[k] = idx;
               }
+              ++ncand;
             }
           }
         }
       }
-      // more candidates than the list holds: mark the list so that the decision kernel scans all rows
-      if (ncand > kTopK) cv[kTopK - 1] = INFINITY;
       if (tok < p.C) {
         const int64_t o = (((int64_t)u * p.nsplit + split) * p.Cmax + tok) * kTopK;
 #pragma unroll
-        for (int k = 0; k < kTopK; ++k) { p.candV[o + k] = cv[k]; p.candI[o + k] = ci[k]; }
+        for (int k = 0; k < kTopK; ++k) p.candI[o + k] = ci[k];
+        // values are not kept: the decision kernel needs the split's maximum and the candidate count
+        p.candV[o] = mx;
+        p.candV[o + 1] = (float)ncand;
       }
     }
   }
