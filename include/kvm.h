@@ -203,6 +203,35 @@ kvm_status_t kvm_debug_counters(kvm_state_t* state, int64_t* out, void* cuda_str
 /* Number of kernels the library has launched for this state so far (host counter). */
 int64_t kvm_launch_count(const kvm_state_t* state);
 
+/* Single-query attention over caller-held rows, for callers that must not allocate device
+ * memory.  (The paper has no counterpart: this is a packaging variant of the decode step's
+ * attention kernel.)  Meant for code that cannot call cudaMalloc where it runs -- a serving loop
+ * whose memory all belongs to its own pool, a plugin inside another framework's memory plan, a
+ * section that must not risk the implicit device synchronisation of cudaMalloc/cudaFree -- and
+ * that already holds the rows in its own buffers, e.g. a readout cache from kvm_state_export
+ * followed by the window tokens.  For every head h:
+ *     out[h] = softmax(scale * q[h] . keys[h]^T) . values[h]
+ *   q       device fp16 [n_heads, head_dim]            (16-byte aligned)
+ *   keys    device fp16 [n_heads, n_rows, head_dim]    (16-byte aligned)
+ *   values  device fp16 [n_heads, n_rows, head_dim]    (16-byte aligned)
+ *   out     device bf16 [n_heads, head_dim]
+ *   scale   multiplies the dot products (tau / sqrt(head_dim) for the layer's logits)
+ * The caller owns all four buffers; the call allocates and frees nothing.  The rows are split
+ * over several CTAs per head; the per-split partial results go to a fixed array inside the
+ * library image (about 4.3 MB on every GPU that loads the library, held until the process exits)
+ * instead of an allocated buffer.  That array bounds the problem: n_heads * n_splits <= 8192,
+ * where n_splits = min(32, ceil(n_rows / 256), ceil(592 / n_heads)); larger calls return
+ * KVM_ERR_CAPACITY and launch nothing.  head_dim must be 64 or 128 (else KVM_ERR_UNSUPPORTED).
+ * All calls share the array and it keeps the previous call's contents; nothing in it needs
+ * clearing because each call rewrites every slot it reads.  Calls that overlap on the same GPU
+ * (other streams or threads) race on it -- serialise them.  The first call on each device looks
+ * up the array's device address (with the calling thread's current device); make that first
+ * call before starting any stream capture.  Work is enqueued on cuda_stream on the current
+ * device; no synchronisation. */
+kvm_status_t kvm_attend_rows_noalloc(const void* q, const void* keys, const void* values, int32_t n_heads,
+                                     int64_t n_rows, int32_t head_dim, float scale, void* out,
+                                     void* cuda_stream);
+
 const char* kvm_status_string(kvm_status_t s);
 
 #ifdef __cplusplus

@@ -25,7 +25,7 @@ FLAG_NO_RADIUS, FLAG_RECORD_ASSIGN, FLAG_SIMT_ATTENTION, FLAG_SIMT_ROUTING = 1, 
 EXPORTS = ["kvm_plan_capacity", "kvm_state_create", "kvm_prefill", "kvm_decode_step", "kvm_prefill_host",
            "kvm_decode_step_host", "kvm_state_free", "kvm_state_info", "kvm_state_check", "kvm_state_export",
            "kvm_debug_assignments", "kvm_launch_count", "kvm_status_string", "kvm_state_reset",
-           "kvm_profile_enable", "kvm_profile_read", "kvm_debug_counters"]
+           "kvm_profile_enable", "kvm_profile_read", "kvm_debug_counters", "kvm_attend_rows_noalloc"]
 
 
 class KVMError(RuntimeError):
@@ -92,6 +92,8 @@ def _load():
     L.kvm_debug_counters.argtypes = [vp, C.POINTER(C.c_int64), vp]
     L.kvm_launch_count.restype = C.c_int64
     L.kvm_launch_count.argtypes = [vp]
+    L.kvm_attend_rows_noalloc.restype = C.c_int
+    L.kvm_attend_rows_noalloc.argtypes = [vp, vp, vp, C.c_int32, C.c_int64, C.c_int32, C.c_float, vp, vp]
     L.kvm_status_string.restype = C.c_char_p
     L.kvm_status_string.argtypes = [C.c_int]
     return L
@@ -120,6 +122,23 @@ def _stream_ptr(stream):
     if stream is None:
         stream = torch.cuda.current_stream()
     return C.c_void_p(stream.cuda_stream)
+
+
+def attend_rows_noalloc(q, keys, values, scale: float, out=None, stream=None):
+    """kvm_attend_rows_noalloc: out[h] = softmax(scale * q[h] . keys[h]^T) . values[h] for callers that may not
+    allocate device memory inside the call (the split partials live in a fixed array of the library).
+    q [H,d] fp16, keys/values [H,n,d] fp16 contiguous CUDA tensors; `out` [H,d] bf16 should be passed by such
+    callers (it is only created here for convenience when omitted)."""
+    assert q.dtype == torch.float16 and keys.dtype == torch.float16 and values.dtype == torch.float16
+    assert q.is_contiguous() and keys.is_contiguous() and values.is_contiguous()
+    H, n, d = keys.shape
+    if out is None:
+        out = torch.empty((H, d), dtype=torch.bfloat16, device=q.device)
+    rc = lib.kvm_attend_rows_noalloc(C.c_void_p(q.data_ptr()), C.c_void_p(keys.data_ptr()), C.c_void_p(values.data_ptr()),
+                                     H, n, d, scale, C.c_void_p(out.data_ptr()), _stream_ptr(stream))
+    if rc != KVM_OK:
+        raise KVMError(rc, "kvm_attend_rows_noalloc")
+    return out
 
 
 @dataclass
