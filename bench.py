@@ -183,32 +183,47 @@ def oracle_sample(wl, mode, budget_s=20.0):
 
 # ------------------------------------------------------------------------------------------
 
-def dist_setup(n):
+def dist_setup(n, backend="nccl"):
+    """One process per GPU (torchrun sets RANK / LOCAL_RANK / WORLD_SIZE).  The ranks are independent
+    replicas of the per-GPU workload; the process group only serves the barrier and the max."""
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if world > 1:
         import torch.distributed as dist
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        torch.cuda.set_device(local)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        if backend == "nccl":
+            torch.cuda.set_device(local)
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        else:
+            dist.init_process_group(backend)
     return rank, world, local
 
 
-def barrier(world):
+def barrier(world, cuda=True):
     if world > 1:
         import torch.distributed as dist
         dist.barrier()
-    torch.cuda.synchronize()
+    if cuda:
+        torch.cuda.synchronize()
 
 
-def max_over_ranks(x, world):
+def max_over_ranks(x, world, device="cuda"):
     if world == 1:
         return x
     import torch.distributed as dist
-    t = torch.tensor([x], dtype=torch.float64, device="cuda")
+    t = torch.tensor([x], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def aggregate(mode, local_ms_per_step, units_per_step, world, device="cuda"):
+    """Whole-job value from per-rank step times: every rank processes `units_per_step` units per step
+    (weak scaling), the job's step time is the slowest rank's.  Returns (value, ms_per_step)."""
+    ms = max_over_ranks(local_ms_per_step, world, device)
+    if mode == "prefill":
+        return world * units_per_step / (ms * 1e-3), ms     # tokens/s over all replicas
+    return ms * 1e3, ms                                     # decode: us per step (each replica steps its batch)
 
 
 def run_reference(args):
@@ -317,7 +332,7 @@ def main():
     launches = st.launch_count() - l0
     clocks = sampler.stop()
     times = [a.elapsed_time(b) for a, b in ev]
-    ms_step = max_over_ranks(sum(times) / K, world)
+    value, ms_step = aggregate(mode, sum(times) / K, units_per_step, world)
 
     # per-phase device time (separate pass with event brackets) -> roofline of the dominant phase
     st.profile_enable(True)
@@ -331,7 +346,6 @@ def main():
 
     if mode == "prefill":
         att_f, rt_f = prefill_flops(wl, wl.T)
-        value = world * units_per_step / (ms_step * 1e-3)
         att_ms = prof["attention"][0] / nprof
         fold_ms = prof["fold"][0] / nprof
         n_att = prof["attention"][1] / nprof
@@ -349,7 +363,6 @@ def main():
         info = st.info()
         nwin_avg = 256 + 128
         bytes_step = wl.B * wl.Hkv * (info["n_slots"] + nwin_avg) * wl.d * 2 * 2
-        value = ms_step * 1e3     # us per step (whole batch); per-sequence = value / B
         dec_ms = prof["decode"][0] / max(prof["decode"][1], 1)
         ach = bytes_step / 1e9 / (dec_ms * 1e-3)
         roof = dict(bound="hbm", kernel="decode", achieved=ach, peak=pk["hbm"], unit="GB/s", frac=ach / pk["hbm"],
