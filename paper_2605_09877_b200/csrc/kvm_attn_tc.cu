@@ -11,7 +11,8 @@
 //   warps 2-5   softmax: each thread owns one query row (tcgen05.ld 32x32b), applies the region
 //               temperature and masks, keeps the running max / sum in registers, rescales O in TMEM
 //               only when the max grew by more than 2^8 (the final 1/l normalisation makes the
-//               stale max exact), writes P as fp16 into swizzled shared memory for the PV MMA,
+//               stale max exact), writes P as fp16 into double-buffered swizzled shared memory for
+//               the PV MMA (so the exponentials of tile j+1 overlap the PV product of tile j),
 //               and finally normalises O and stores bf16 rows.
 // Every mbarrier wait is bounded; on expiry the CTA records KVM_ERR_TIMEOUT and tears down.
 #include "kvm_internal.h"
@@ -39,7 +40,7 @@ struct AttnTcCfg {
   static constexpr int OFF_K = OFF_Q + TILE_BYTES;
   static constexpr int OFF_V = OFF_K + NS * TILE_BYTES;
   static constexpr int OFF_P = OFF_V + NS * TILE_BYTES;
-  static constexpr int OFF_BAR = OFF_P + P_BYTES;
+  static constexpr int OFF_BAR = OFF_P + 2 * P_BYTES;  // P is double-buffered: softmax of tile j+1 overlaps PV of tile j
   // + alignment slack; never less than half an SM so that one CTA (and one 512-column TMEM
   // allocation) is resident per SM
   static constexpr int SMEM_BYTES = (OFF_BAR + 256 + 1024) > 120 * 1024 ? (OFF_BAR + 256 + 1024) : 120 * 1024;
@@ -47,7 +48,7 @@ struct AttnTcCfg {
   static constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_O = 256;
 };
 
-enum { BAR_QFULL = 0, BAR_KFULL = 1, BAR_VFULL = 3, BAR_FREE = 5, BAR_SFULL = 7, BAR_PFULL = 9, BAR_PVDONE = 10, BAR_COUNT = 11 };
+enum { BAR_QFULL = 0, BAR_KFULL = 1, BAR_VFULL = 3, BAR_FREE = 5, BAR_SFULL = 7, BAR_PFULL = 9, BAR_PVDONE = 11, BAR_COUNT = 13 };
 
 template <int D>
 __global__ void __launch_bounds__(192, 1)
@@ -85,8 +86,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     }
     tc::mbar_init(&bars[BAR_SFULL + 0], 1);
     tc::mbar_init(&bars[BAR_SFULL + 1], 1);
-    tc::mbar_init(&bars[BAR_PFULL], 4);
-    tc::mbar_init(&bars[BAR_PVDONE], 1);
+    tc::mbar_init(&bars[BAR_PFULL + 0], 4);
+    tc::mbar_init(&bars[BAR_PFULL + 1], 4);
+    tc::mbar_init(&bars[BAR_PVDONE + 0], 1);
+    tc::mbar_init(&bars[BAR_PVDONE + 1], 1);
     *abort_flag = 0;
     tc::fence_barrier_init();
   }
@@ -158,20 +161,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           const int s = j % Cfg::NS;
           if (*abort_flag) { dead = true; break; }
           if (j + 1 < ntiles && !issue_qk(j + 1)) { dead = true; break; }
-          if (!tc::mbar_wait(&bars[BAR_PFULL], j & 1)) { dead = true; break; }
+          if (!tc::mbar_wait(&bars[BAR_PFULL + (j & 1)], (j >> 1) & 1)) { dead = true; break; }
           if (!tc::mbar_wait(&bars[BAR_VFULL + s], (j / Cfg::NS) & 1)) { dead = true; break; }
           tc::tc_fence_after();
           const uint32_t dO = tmem + Cfg::COL_O;
 #pragma unroll
           for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t offP = (kk / 4) * Cfg::BOX_BYTES + (kk % 4) * 32;
+            const uint32_t offP = (j & 1) * Cfg::P_BYTES + (kk / 4) * Cfg::BOX_BYTES + (kk % 4) * 32;
             const uint32_t offV = kk * 2048;   // 16 key rows x 128 B
             tc::mma_f16_ss(dO, tc::smem_desc_sw128(aP + offP, 16, 1024),
                            tc::smem_desc_sw128(aV + s * Cfg::TILE_BYTES + offV, Cfg::BOX_BYTES, 1024), IDESC_PV,
                            (j > 0 || kk > 0) ? 1u : 0u);
           }
           tc::mma_commit(&bars[BAR_FREE + s]);
-          tc::mma_commit(&bars[BAR_PVDONE]);
+          tc::mma_commit(&bars[BAR_PVDONE + (j & 1)]);
         }
       } while (false);
       if (dead) { atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; }
@@ -204,26 +207,34 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           }
           tc::tmem_wait_ld();
         }
-        // region scale + mask
+        // region scale (folded into the exponent) and masks; the scale is positive, so the row
+        // maximum can be taken on the raw products
         const bool st = j < nst;
         const float sc = st ? sc_s : sc_b;
-        // number of visible columns of this tile for this row
-        int64_t nvis;
+        int64_t nvis;   // number of visible columns of this tile for this row
         if (st) nvis = p.m - (int64_t)j * 128;
         else nvis = t_row - (p.b + (int64_t)(j - nst) * 128) + 1;
         const int vis = (int)max((int64_t)0, min((int64_t)128, nvis));
         float mx = -INFINITY;
+        if (vis == 128) {
 #pragma unroll
-        for (int c = 0; c < 128; ++c) {
-          x[c] = (c < vis) ? x[c] * sc : -INFINITY;
-          mx = fmaxf(mx, x[c]);
+          for (int c = 0; c < 128; ++c) mx = fmaxf(mx, x[c]);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 128; ++c) {
+            x[c] = (c < vis) ? x[c] : -INFINITY;
+            mx = fmaxf(mx, x[c]);
+          }
         }
-        float mnew = fmaxf(m_run, mx);
-        if (j > 0) {
-          KVM_WAIT(&bars[BAR_PVDONE], (j - 1) & 1);   // P buffer free, O quiescent
-          tc::tc_fence_after();
+        const float mnew = fmaxf(m_run, mx * sc);
+        if (j == 0) {
+          m_run = mnew;
+        } else {
           const bool need = mnew > m_run + 8.0f;
           if (__any_sync(0xffffffffu, need)) {
+            // all earlier PV products must have landed before O is touched (commits complete in order)
+            KVM_WAIT(&bars[BAR_PVDONE + ((j - 1) & 1)], ((j - 1) >> 1) & 1);
+            tc::tc_fence_after();
             const float corr = (m_run == -INFINITY) ? 0.f : tc::ex2_approx(m_run - mnew);
             l_run *= corr;
             m_run = mnew;
@@ -239,21 +250,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
             }
             tc::tmem_wait_st();
           }
-        } else {
-          m_run = mnew;
         }
-        const float m_use = (m_run == -INFINITY) ? 0.f : m_run;
+        if (j >= 2) {   // the PV product that read this P buffer two tiles ago has finished
+          KVM_WAIT(&bars[BAR_PVDONE + (j & 1)], ((j >> 1) - 1) & 1);
+        }
+        const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
         float lsum = 0.f;
         // P row -> shared memory, K-major, 128-byte swizzle: 16-byte chunk ch of row r lives at
         // r*128 + ((ch ^ (r & 7)) * 16) inside its 64-key box.
-        uint8_t* prow = sP + row * 128;
+        uint8_t* prow = sP + (j & 1) * Cfg::P_BYTES + row * 128;
 #pragma unroll
         for (int ch = 0; ch < 16; ++ch) {
           uint32_t w[4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
-            const float p0 = tc::ex2_approx(x[ch * 8 + 2 * i] - m_use);
-            const float p1 = tc::ex2_approx(x[ch * 8 + 2 * i + 1] - m_use);
+            const float p0 = tc::ex2_approx(fmaf(x[ch * 8 + 2 * i], sc, neg_m));
+            const float p1 = tc::ex2_approx(fmaf(x[ch * 8 + 2 * i + 1], sc, neg_m));
             lsum += p0 + p1;
             const __half2 h = __floats2half2_rn(p0, p1);
             w[i] = *reinterpret_cast<const uint32_t*>(&h);
@@ -265,14 +277,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         tc::fence_proxy_async();
         tc::tc_fence_before();
         __syncwarp();
-        if (lane == 0) tc::mbar_arrive(&bars[BAR_PFULL]);
+        if (lane == 0) tc::mbar_arrive(&bars[BAR_PFULL + (j & 1)]);
         ok = true;
       } while (false);
     }
     // epilogue
     do {
       if (!ok || ntiles == 0) break;
-      KVM_WAIT(&bars[BAR_PVDONE], (ntiles - 1) & 1);
+      KVM_WAIT(&bars[BAR_PVDONE + ((ntiles - 1) & 1)], ((ntiles - 1) >> 1) & 1);
       tc::tc_fence_after();
       const float inv = 1.f / l_run;
       const uint32_t to = tmem + lane_base + Cfg::COL_O;
