@@ -48,7 +48,7 @@ struct AttnTcCfg {
   static constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_O = 256;
 };
 
-enum { BAR_QFULL = 0, BAR_KFULL = 1, BAR_VFULL = 3, BAR_FREE = 5, BAR_SFULL = 7, BAR_PFULL = 9, BAR_PVDONE = 11, BAR_COUNT = 13 };
+enum { BAR_QFULL = 0, BAR_KFULL = 1, BAR_VFULL = 3, BAR_FREE = 5, BAR_SFULL = 7, BAR_PFULL = 9, BAR_PVDONE = 11, BAR_KFREE = 13, BAR_COUNT = 15 };
 
 template <int D>
 __global__ void __launch_bounds__(192, 1)
@@ -83,6 +83,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       tc::mbar_init(&bars[BAR_KFULL + s], 1);
       tc::mbar_init(&bars[BAR_VFULL + s], 1);
       tc::mbar_init(&bars[BAR_FREE + s], 1);
+      tc::mbar_init(&bars[BAR_KFREE + s], 1);
     }
     tc::mbar_init(&bars[BAR_SFULL + 0], 1);
     tc::mbar_init(&bars[BAR_SFULL + 1], 1);
@@ -117,21 +118,32 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       tc::mbar_expect_tx(&bars[BAR_QFULL], Cfg::TILE_BYTES);
       for (int kb = 0; kb < Cfg::NKB; ++kb)
         tc::tma_load_3d(sQ + kb * Cfg::BOX_BYTES, &mapQ, &bars[BAR_QFULL], kb * 64, (int)(p.q_row0 + qt * 128), bh);
-      for (int j = 0; j < ntiles; ++j) {
+      // A K stage is released as soon as its QK^T product has completed, a V stage only after its
+      // PV product, so K of tile j+1 is requested before V of tile j: the keys of the next tile are
+      // in flight while the softmax of the current one runs.
+      auto load_k = [&](int j) -> bool {
         const int s = j % Cfg::NS;
-        if (*abort_flag) break;
-        if (j >= Cfg::NS) { KVM_WAIT(&bars[BAR_FREE + s], ((j / Cfg::NS) - 1) & 1); }
+        if (j >= Cfg::NS && !tc::mbar_wait(&bars[BAR_KFREE + s], ((j / Cfg::NS) - 1) & 1)) return false;
         const bool st = j < nst;
-        const CUtensorMap* mk = st ? &mapKs : &mapKw;
-        const CUtensorMap* mv = st ? &mapVs : &mapVw;
         const int row = st ? j * 128 : (int)(p.win_row0 + (int64_t)(j - nst) * 128);
         tc::mbar_expect_tx(&bars[BAR_KFULL + s], Cfg::TILE_BYTES);
         for (int kb = 0; kb < Cfg::NKB; ++kb)
-          tc::tma_load_3d(sK + s * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, mk, &bars[BAR_KFULL + s], kb * 64, row, u);
+          tc::tma_load_3d(sK + s * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, st ? &mapKs : &mapKw, &bars[BAR_KFULL + s], kb * 64, row, u);
+        return true;
+      };
+      bool okp = ntiles == 0 || load_k(0);
+      for (int j = 0; j < ntiles && okp; ++j) {
+        const int s = j % Cfg::NS;
+        if (*abort_flag) break;
+        if (j + 1 < ntiles && !load_k(j + 1)) { okp = false; break; }
+        if (j >= Cfg::NS && !tc::mbar_wait(&bars[BAR_FREE + s], ((j / Cfg::NS) - 1) & 1)) { okp = false; break; }
+        const bool st = j < nst;
+        const int row = st ? j * 128 : (int)(p.win_row0 + (int64_t)(j - nst) * 128);
         tc::mbar_expect_tx(&bars[BAR_VFULL + s], Cfg::TILE_BYTES);
         for (int kb = 0; kb < Cfg::NKB; ++kb)
-          tc::tma_load_3d(sV + s * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, mv, &bars[BAR_VFULL + s], kb * 64, row, u);
+          tc::tma_load_3d(sV + s * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, st ? &mapVs : &mapVw, &bars[BAR_VFULL + s], kb * 64, row, u);
       }
+      if (!okp) { atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; }
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer ------------------------------
@@ -152,6 +164,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
                          tc::smem_desc_sw128(aK + s * Cfg::TILE_BYTES + off, 16, 1024), IDESC_QK, ks > 0);
         }
         tc::mma_commit(&bars[BAR_SFULL + (j & 1)]);
+        tc::mma_commit(&bars[BAR_KFREE + s]);
         return true;
       };
       do {
