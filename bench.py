@@ -79,6 +79,11 @@ def prefill_flops(wl, T):
     return 4 * wl.d * att_pairs * units_q, 2 * wl.d * route_pairs * units_kv
 
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the kernels that carry a
+# roofline, from the ncu captures summarised under profiles/ (null until captured for the workload).
+NCU_TRAFFIC = {}
+
+
 def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -346,15 +351,20 @@ def main():
 
     if mode == "prefill":
         att_f, rt_f = prefill_flops(wl, wl.T)
-        att_ms = prof["attention"][0] / nprof
-        fold_ms = prof["fold"][0] / nprof
-        n_att = prof["attention"][1] / nprof
-        dom = "attention" if att_ms >= fold_ms else "fold"
-        ach = (att_f / 1e12) / (att_ms * 1e-3) if dom == "attention" else (rt_f / 1e12) / (fold_ms * 1e-3)
+        per_kernel = {k_: v_[0] / nprof for k_, v_ in prof.items()}
+        # the dominant kernel by device time; the two tensor-core kernels have an algorithmic flop count
+        dom = max(per_kernel, key=per_kernel.get)
+        if dom not in ("attention", "route_filter"):
+            dom = "attention"   # decide / apply / kbar are latency-bound helpers without a flop model
+        dom_ms = per_kernel[dom]
+        n_dom = prof[dom][1] / nprof
+        ach = ((att_f if dom == "attention" else rt_f) / 1e12) / (dom_ms * 1e-3)
         peak = pk["tf_sust"]
-        roof = dict(bound="tensor", kernel=dom, achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak, traffic=None,
+        roof = dict(bound="tensor", kernel=dom, achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak,
+                    traffic=NCU_TRAFFIC.get(dom),
                     peak_source=f"{pk['src']} bf16 sustained (fp16 operands run at the bf16 rate)",
-                    launches_per_step=n_att, avg_launch_us=1e3 * att_ms / max(n_att, 1),
+                    launches_per_step=n_dom, avg_launch_us=1e3 * dom_ms / max(n_dom, 1),
+                    share_of_device_time=dom_ms / max(sum(per_kernel.values()), 1e-9),
                     whole_step_tflops=(att_f + rt_f) / 1e12 / (ms_step * 1e-3),
                     whole_step_frac_of_burst=(att_f + rt_f) / 1e12 / (ms_step * 1e-3) / pk["tf_burst"],
                     phase_ms={k_: v_[0] / nprof for k_, v_ in prof.items()})

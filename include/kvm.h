@@ -186,12 +186,13 @@ kvm_status_t kvm_debug_assignments(kvm_state_t* state, int64_t n, int32_t* slot_
  * ordered behind it on the same stream). */
 kvm_status_t kvm_state_reset(kvm_state_t* state);
 
-/* Per-phase device timing for benchmarks.  kvm_profile_enable(state, 1) makes every later
- * call bracket each phase's launches with CUDA events on the call's stream (phases:
- * 0 ingest, 1 attention, 2 fold, 3 decode attention); kvm_profile_read synchronises the
- * device, adds the elapsed milliseconds and launch-group counts of the recorded brackets into
- * ms[4] / groups[4] and clears the record.  Off by default; at most 8192 brackets are kept
- * between reads (later ones are dropped and not counted). */
+/* Per-kernel device timing for benchmarks.  kvm_profile_enable(state, 1) makes every later
+ * call bracket the launches of each phase with CUDA events on the call's stream (phases:
+ * 0 ingest, 1 attention, 2 memory keys, 3 routing filter, 4 fold decision, 5 fold application,
+ * 6 decode step attention incl. its ingest/combine, 7 unused); kvm_profile_read synchronises
+ * the device, adds the elapsed milliseconds and bracket counts into ms[8] / groups[8] and
+ * clears the record.  Off by default; at most 16384 brackets are kept between reads (later
+ * ones are dropped and not counted). */
 kvm_status_t kvm_profile_enable(kvm_state_t* state, int32_t on);
 kvm_status_t kvm_profile_read(kvm_state_t* state, double* ms, int64_t* groups);
 

@@ -17,26 +17,32 @@ struct kvm_state {
   std::vector<void*> allocs;
   bool host_staging = false;
   bool prof_on = false;
+  bool prof_open = false;
+  ProfBracket prof_cur{};
   std::vector<ProfBracket> prof_free, prof_used;
 };
 
 namespace {
-// Brackets the launches of one phase with two events when profiling is enabled.
-struct PhaseTimer {
-  kvm_state* ks; cudaStream_t stream; bool active = false; ProfBracket br{};
-  PhaseTimer(kvm_state* k, int phase, cudaStream_t s) : ks(k), stream(s) {
-    if (!ks->prof_on || ks->prof_used.size() >= 8192) return;
+constexpr size_t kProfMaxBrackets = 16384;
+// Timing hook installed in State::prof_hook: brackets the launches of one phase with two events.
+void prof_hook_fn(void* ctx, int phase, int begin, cudaStream_t stream) {
+  kvm_state* ks = static_cast<kvm_state*>(ctx);
+  if (begin) {
+    if (ks->prof_open || ks->prof_used.size() >= kProfMaxBrackets) return;
+    ProfBracket br{};
     if (!ks->prof_free.empty()) { br = ks->prof_free.back(); ks->prof_free.pop_back(); }
     else if (cudaEventCreate(&br.a) != cudaSuccess || cudaEventCreate(&br.b) != cudaSuccess) { cudaGetLastError(); return; }
     br.phase = phase;
-    active = cudaEventRecord(br.a, stream) == cudaSuccess;
+    if (cudaEventRecord(br.a, stream) != cudaSuccess) { cudaGetLastError(); ks->prof_free.push_back(br); return; }
+    ks->prof_cur = br;
+    ks->prof_open = true;
+  } else {
+    if (!ks->prof_open || ks->prof_cur.phase != phase) return;
+    cudaEventRecord(ks->prof_cur.b, stream);
+    ks->prof_used.push_back(ks->prof_cur);
+    ks->prof_open = false;
   }
-  ~PhaseTimer() {
-    if (!active) return;
-    cudaEventRecord(br.b, stream);
-    ks->prof_used.push_back(br);
-  }
-};
+}
 }  // namespace
 
 namespace {
@@ -308,6 +314,8 @@ KVM_API kvm_status_t kvm_state_reset(kvm_state_t* ks) {
 KVM_API kvm_status_t kvm_profile_enable(kvm_state_t* ks, int32_t on) {
   if (!ks) return KVM_ERR_INVALID_ARG;
   ks->prof_on = on != 0;
+  ks->s.prof_hook = ks->prof_on ? prof_hook_fn : nullptr;
+  ks->s.prof_ctx = ks;
   return KVM_OK;
 }
 
@@ -404,7 +412,7 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
     const int64_t c_next = pos1 / C;
     ia.tail_start = (c_next + 1) * C - L; if (ia.tail_start < 0) ia.tail_start = 0;
   }
-  { PhaseTimer pt(ks, 0, stream); s.launches += launch_ingest(&s, ia, stream); }
+  { KernelTimer pt(&s, 0, stream); s.launches += launch_ingest(&s, ia, stream); }
 
   const bool simt_attn = true;  // replaced by the tcgen05 kernel selection below once available
   (void)simt_attn;
@@ -416,7 +424,7 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
     aa.q_row0 = qs - pos0; aa.nq = (int)(qe - qs); aa.t0 = qs; aa.m = s.m;
     aa.win_row0 = b - ia.hist_start; aa.b = b; aa.out = (__nv_bfloat16*)out; aa.out_t0 = qs - pos0;
     {
-      PhaseTimer pt(ks, 1, stream);
+      KernelTimer pt(&s, 1, stream);
       if (s.flags & KVM_FLAG_SIMT_ATTENTION) s.launches += launch_attn_simt(&s, aa, stream);
       else s.launches += launch_attn_tc(&s, aa, stream);
     }
@@ -426,7 +434,7 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
       fa.unit_stride = s.stRows * d; fa.gate_stride = s.stRows;
       fa.b = b; fa.m = s.m; fa.first = (s.m == 0);
       fa.n_append = fa.first ? C : (int)n_append_of(s.growth, e, s.m, C);
-      { PhaseTimer pt(ks, 2, stream); s.launches += launch_fold(&s, fa, stream); }
+      s.launches += launch_fold(&s, fa, stream);
       s.m += fa.n_append;
       s.nfolds += 1;
     }
@@ -457,7 +465,7 @@ KVM_API kvm_status_t kvm_decode_step(const void* q, const void* k, const void* v
   DecodeArgs da;
   da.q = (const __nv_bfloat16*)q; da.k = (const __nv_bfloat16*)k; da.v = (const __nv_bfloat16*)v; da.gate = gate;
   da.out = (__nv_bfloat16*)out; da.t = t; da.b = b; da.m = s.m;
-  { PhaseTimer pt(ks, 3, stream); s.launches += launch_decode(&s, da, stream); }
+  { KernelTimer pt(&s, 6, stream); s.launches += launch_decode(&s, da, stream); }
   if (fold) {
     const int64_t ringCap = (int64_t)s.w * s.Cmax;
     const int64_t slot = b % s.ringLen;
@@ -465,7 +473,7 @@ KVM_API kvm_status_t kvm_decode_step(const void* q, const void* k, const void* v
     fa.ok = s.ringK + slot * d; fa.ov = s.ringV + slot * d; fa.og = s.ringG + slot;
     fa.unit_stride = ringCap * d; fa.gate_stride = ringCap;
     fa.b = b; fa.m = s.m; fa.first = (s.m == 0); fa.n_append = n_a;
-    { PhaseTimer pt(ks, 2, stream); s.launches += launch_fold(&s, fa, stream); }
+    s.launches += launch_fold(&s, fa, stream);
     s.m += n_a;
     s.nfolds += 1;
   }

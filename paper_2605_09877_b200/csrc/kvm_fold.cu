@@ -299,26 +299,31 @@ __global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideP
     s_exh[j] = exh ? 1 : 0;
   }
   __syncthreads();
-  // ---- A3: exact fp64 similarity of every candidate pair, one warp per pair, two in flight ----
+  // ---- A3: exact fp64 similarity of every candidate pair, one warp per pair, four in flight ----
   const int np = min(s_np, kPairCap);
-  for (int q = warp; q < np; q += 2 * kDecideWarps) {
-    const int q2 = q + kDecideWarps;
-    const bool two = q2 < np;
-    const int j0 = s_ptok[q], i0 = s_prow[q];
-    const int j1 = two ? s_ptok[q2] : j0, i1 = two ? s_prow[q2] : i0;
-    double kb0[CH], kb1[CH];
+  for (int q0 = warp; q0 < np; q0 += 4 * kDecideWarps) {
+    double part[4];
 #pragma unroll
-    for (int i = 0; i < CH; ++i) {
-      kb0[i] = kbarU[(int64_t)j0 * D + lane + 32 * i];
-      kb1[i] = kbarU[(int64_t)j1 * D + lane + 32 * i];
+    for (int k = 0; k < 4; ++k) {
+      const int q = min(q0 + k * kDecideWarps, np - 1);   // clamped duplicates are computed and dropped
+      const int j = s_ptok[q], i = s_prow[q];
+      const double* kb = kbarU + (int64_t)j * D;
+      const double* sk = p.sumK + (rowBase + i) * D;
+      const double mu = p.kmu[rowBase + i], rs = p.krstd[rowBase + i];
+      double acc = 0.0;
+#pragma unroll
+      for (int c = 0; c < CH; ++c) acc += kb[lane + 32 * c] * (gam[c] * ((sk[lane + 32 * c] - mu) * rs) + bet[c]);
+      part[k] = acc;
     }
-    const double mu0 = p.kmu[rowBase + i0], rs0 = p.krstd[rowBase + i0];
-    const double mu1 = p.kmu[rowBase + i1], rs1 = p.krstd[rowBase + i1];
-    const double a0 = warp_sim<CH>(kb0, p.sumK + (rowBase + i0) * D, mu0, rs0, gam, bet, lane);
-    const double a1 = warp_sim<CH>(kb1, p.sumK + (rowBase + i1) * D, mu1, rs1, gam, bet, lane);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) part[k] += __shfl_xor_sync(0xffffffffu, part[k], o);
+    }
     if (lane == 0) {
-      s_pval[q] = a0;
-      if (two) s_pval[q2] = a1;
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (q0 + k * kDecideWarps < np) s_pval[q0 + k * kDecideWarps] = part[k];
     }
   }
   __syncthreads();
@@ -385,10 +390,26 @@ __global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideP
       double kb[CH];
 #pragma unroll
       for (int i = 0; i < CH; ++i) kb[i] = kbarU[(int64_t)j * D + lane + 32 * i];
-#pragma unroll 2
-      for (int a = 0; a < n_a; ++a) {
-        const double acc = warp_sim<CH>(kb, kbarU + (int64_t)s_creator[a] * D, s_cmu[a], s_crs[a], gam, bet, lane);
-        if (acc > best) { best = acc; arg = (int)m + a; }
+      for (int a0 = 0; a0 < n_a; a0 += 4) {
+        double part[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int a = min(a0 + k, n_a - 1);
+          const double* ka = kbarU + (int64_t)s_creator[a] * D;
+          const double mu = s_cmu[a], rs = s_crs[a];
+          double acc = 0.0;
+#pragma unroll
+          for (int c = 0; c < CH; ++c) acc += kb[c] * (gam[c] * ((ka[lane + 32 * c] - mu) * rs) + bet[c]);
+          part[k] = acc;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) part[k] += __shfl_xor_sync(0xffffffffu, part[k], o);
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (a0 + k < n_a && part[k] > best) { best = part[k]; arg = (int)m + a0 + k; }
       }
     }
     if (lane == 0) {
@@ -446,11 +467,21 @@ struct FoldApplyParams {
 template <int D>
 __global__ void __launch_bounds__(256) fold_apply_kernel(FoldApplyParams p) {
   constexpr int CH = D / 32;
+  __shared__ int s_pi[kMaxBlock], s_sorted[kMaxBlock], s_creator[kMaxBlock], s_segnew[kMaxBlock];
   const int u = blockIdx.y, hk = u % p.Hkv;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q = blockIdx.x * 8 + warp;
-  if (q >= p.C) return;
   const int64_t tokBase = (int64_t)u * p.Cmax;
+  if (!p.all_append) {   // the decisions of this unit, read once per CTA instead of chased per warp
+    for (int i = threadIdx.x; i < p.C; i += 256) {
+      s_pi[i] = p.pi[tokBase + i];
+      s_sorted[i] = p.sorted[tokBase + i];
+      s_creator[i] = p.creator[tokBase + i];
+      s_segnew[i] = p.segnew[tokBase + i];
+    }
+    __syncthreads();
+  }
+  if (q >= p.C) return;
   const int64_t rowBase = (int64_t)u * p.Mcap;
   const double* kbarU = p.kbar64 + tokBase * D;
   const __half* ovU = p.ov + (int64_t)u * p.unit_stride;
@@ -464,14 +495,14 @@ __global__ void __launch_bounds__(256) fold_apply_kernel(FoldApplyParams p) {
     if (task == 0) {
       if (q >= p.n_append) continue;
       rowi = m + q;
-      jc = p.all_append ? q : p.creator[tokBase + q];
-      seg = p.all_append ? -1 : p.segnew[tokBase + q];
+      jc = p.all_append ? q : s_creator[q];
+      seg = p.all_append ? -1 : s_segnew[q];
     } else {
       if (q >= nmerge) continue;
-      const int j0 = p.sorted[tokBase + q];
-      rowi = p.pi[tokBase + j0];
-      if (rowi >= m) continue;                                              // new rows are task 0
-      if (q > 0 && p.pi[tokBase + p.sorted[tokBase + q - 1]] == rowi) continue;   // not a head
+      const int j0 = s_sorted[q];
+      rowi = s_pi[j0];
+      if (rowi >= m) continue;                                 // new rows are task 0
+      if (q > 0 && s_pi[s_sorted[q - 1]] == rowi) continue;    // not a head
       seg = q;
     }
     const int64_t row = rowBase + rowi;
@@ -510,8 +541,8 @@ __global__ void __launch_bounds__(256) fold_apply_kernel(FoldApplyParams p) {
     }
     if (seg >= 0) {
       for (int qq = seg; qq < nmerge; ++qq) {
-        const int j = p.sorted[tokBase + qq];
-        if (p.pi[tokBase + j] != rowi) break;
+        const int j = s_sorted[qq];
+        if (s_pi[j] != rowi) break;
         const float g = ogU[j];
         const double* kb = kbarU + (int64_t)j * D;
         const __half* vr = ovU + (int64_t)j * D;
@@ -562,6 +593,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
   int launches = 0;
   const int C = st->C, D = st->d;
   {
+    KernelTimer kt(st, 2, s);
     dim3 grid((C + 7) / 8, st->U);
     if (D == 128)
       kbar_kernel<128><<<grid, 256, 0, s>>>(a.ok, a.unit_stride, st->ln_w, st->ln_b, st->kbar64, st->kbarH,
@@ -582,6 +614,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
     if (nsplit < 1) nsplit = 1;
     if (nsplit > st->nsplitRoute) nsplit = st->nsplitRoute;
     if (st->flags & KVM_FLAG_SIMT_ROUTING) {
+      KernelTimer kt(st, 3, s);
       dim3 grid(nsplit, st->U);
       if (D == 128)
         route_filter_simt_kernel<128><<<grid, 256, 0, s>>>(st->kbarH, st->Khat, st->candV, st->candI, C, st->Cmax,
@@ -593,6 +626,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
                                                           route_thr_coeff(st), st->S);
       ++launches;
     } else {
+      KernelTimer kt(st, 3, s);
       launches += launch_route_filter_tc(st, a.m, nsplit, s);
     }
     FoldDecideParams p;
@@ -605,6 +639,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
     p.Mcap = st->Mcap; p.m = a.m;
     p.C = C; p.Cmax = st->Cmax; p.Hkv = st->Hkv; p.S = st->S; p.n_append = a.n_append; p.nsplit = nsplit;
     p.thr_coeff = route_thr_coeff(st);
+    KernelTimer kt(st, 4, s);
     if (D == 128) fold_decide_kernel<128><<<st->U, kDecideThreads, 0, s>>>(p);
     else fold_decide_kernel<64><<<st->U, kDecideThreads, 0, s>>>(p);
     ++launches;
@@ -621,6 +656,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
   q.C = C; q.Cmax = st->Cmax; q.Hkv = st->Hkv; q.n_append = a.n_append; q.all_append = all_append ? 1 : 0;
   q.radius_on = (st->flags & KVM_FLAG_NO_RADIUS) ? 0 : 1;
   q.ln_eps = (double)st->ln_eps; q.norm_eps = (double)st->norm_eps;
+  KernelTimer kt(st, 5, s);
   dim3 grid((C + 7) / 8, st->U);
   if (D == 128) fold_apply_kernel<128><<<grid, 256, 0, s>>>(q);
   else fold_apply_kernel<64><<<grid, 256, 0, s>>>(q);

@@ -70,6 +70,10 @@ struct State {
   int nsplitDec;
   float* decPart;                // [B*Hq, nsplitDec, d + 2]
   __half* decQ;                  // [B*Hq, d] rotated query
+  // ---- optional per-kernel timing hook (set by kvm_profile_enable): phase ids
+  //      0 ingest, 1 attention, 2 memory keys, 3 routing filter, 4 decide, 5 apply, 6 decode ----
+  void (*prof_hook)(void* ctx, int phase, int begin, cudaStream_t s);
+  void* prof_ctx;
   // ---- recording / status ----
   int32_t* slotTok;              // [U, Tassign]
   uint8_t* appTok;               // [U, Tassign]
@@ -135,5 +139,14 @@ struct DecodeArgs {
   int64_t m;
 };
 int launch_decode(State* st, const DecodeArgs& a, cudaStream_t s);
+
+// Brackets the launches issued during its lifetime with the state's timing hook (no-op when off).
+struct KernelTimer {
+  State* st; int phase; cudaStream_t s;
+  KernelTimer(State* st_, int phase_, cudaStream_t s_) : st(st_), phase(phase_), s(s_) {
+    if (st->prof_hook) st->prof_hook(st->prof_ctx, phase, 1, s);
+  }
+  ~KernelTimer() { if (st->prof_hook) st->prof_hook(st->prof_ctx, phase, 0, s); }
+};
 
 }  // namespace kvm

@@ -266,12 +266,12 @@ class KVMState:
 
     def profile_read(self):
         """Returns {phase: (milliseconds, bracket count)} accumulated since the last read."""
-        ms = (C.c_double * 4)(); n = (C.c_int64 * 4)()
+        ms = (C.c_double * 8)(); n = (C.c_int64 * 8)()
         rc = lib.kvm_profile_read(self._h, ms, n)
         if rc != KVM_OK:
             raise KVMError(rc, "kvm_profile_read")
-        names = ("ingest", "attention", "fold", "decode")
-        return {names[i]: (ms[i], n[i]) for i in range(4)}
+        names = ("ingest", "attention", "kbar", "route_filter", "fold_decide", "fold_apply", "decode")
+        return {names[i]: (ms[i], n[i]) for i in range(7)}
 
     def debug_counters(self, stream=None):
         out = (C.c_int64 * 3)()
