@@ -251,7 +251,7 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   A(s.ropeCS, (size_t)s.Tcall * (d / 2));
   s.CbarRows = (s.Cmax + 127) / 128 * 128;
   A(s.kbar64, U * Cm * d); A(s.kbarH, U * (size_t)s.CbarRows * d); A(s.kbarNorm, U * Cm);
-  A(s.kbarMu, U * Cm); A(s.kbarRstd, U * Cm);
+  A(s.kbarHat64, U * Cm * d);
   A(s.foldPi, U * Cm); A(s.foldSorted, U * Cm); A(s.foldCreator, U * Cm); A(s.foldSegNew, U * Cm); A(s.foldNMerge, U);
   A(s.candV, U * (size_t)s.nsplitRoute * Cm * kTopK); A(s.candI, U * (size_t)s.nsplitRoute * Cm * kTopK);
   A(s.decPart, (size_t)s.B * s.Hq * s.nsplitDec * (d + 2)); A(s.decQ, (size_t)s.B * s.Hq * d);

@@ -45,8 +45,8 @@ template <int D>
 __global__ void __launch_bounds__(256) kbar_kernel(const __half* __restrict__ ok, int64_t unit_stride,
                                                    const float* __restrict__ ln_w, const float* __restrict__ ln_b,
                                                    double* __restrict__ kbar64, __half* __restrict__ kbarH,
-                                                   float* __restrict__ kbarNorm, double* __restrict__ kbarMu,
-                                                   double* __restrict__ kbarRstd, int C, int Cmax, int CbarRows,
+                                                   float* __restrict__ kbarNorm, double* __restrict__ kbarHat64,
+                                                   int write_hat, int C, int Cmax, int CbarRows,
                                                    int Hkv, int r, double ln_eps) {
   constexpr int CH = D / 32;
   const int u = blockIdx.y, hk = u % Hkv;
@@ -75,14 +75,17 @@ __global__ void __launch_bounds__(256) kbar_kernel(const __half* __restrict__ ok
     n2 += kb[i] * kb[i];
   }
   n2 = warp_sum_d(n2);
-  // statistics of LN_s applied to kbar itself: the key of a row that this token would create
+  // LN_s applied to kbar itself: the readout key of the row that this token would create
   double mu2, rs2;
   row_stats<CH>(kb, D, ln_eps, mu2, rs2);
-  if (lane == 0) {
-    kbarNorm[(int64_t)u * Cmax + j] = (float)sqrt(n2) * 1.000001f;
-    kbarMu[(int64_t)u * Cmax + j] = mu2;
-    kbarRstd[(int64_t)u * Cmax + j] = rs2;
+  if (write_hat) {   // only folds that append rows need the would-be row keys
+#pragma unroll
+    for (int i = 0; i < CH; ++i) {
+      const int x = lane + 32 * i;
+      kbarHat64[o + x] = (double)ln_w[hk * D + x] * ((kb[i] - mu2) * rs2) + (double)ln_b[hk * D + x];
+    }
   }
+  if (lane == 0) kbarNorm[(int64_t)u * Cmax + j] = (float)sqrt(n2) * 1.000001f;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -176,7 +179,7 @@ __global__ void __launch_bounds__(256) route_filter_simt_kernel(const __half* __
 struct FoldDecideParams {
   const double* kbar64;
   const float* kbarNorm;
-  const double *kbarMu, *kbarRstd;
+  const double* kbarHat64;   // LN_s(kbar_j): keys of the rows the block's tokens would create
   const float* candV;
   const int32_t* candI;
   const float *ln_w, *ln_b;
@@ -202,6 +205,22 @@ __device__ __forceinline__ void load_cand_rows(const int32_t* candI, int64_t o, 
   i[0] = i0.x; i[1] = i0.y; i[2] = i0.z; i[3] = i0.w; i[4] = i1.x; i[5] = i1.y; i[6] = i1.z; i[7] = i1.w;
 }
 
+// Sums four per-lane partials over the warp with six exchanges instead of twenty: after the call a
+// lane holds the full sum of partial number t = 2*bit4(lane) + bit3(lane) (all 8 lanes of that
+// group agree).  Fixed exchange order, so results are reproducible.
+__device__ __forceinline__ double warp_reduce4(double v0, double v1, double v2, double v3, int lane) {
+  const bool hi16 = lane & 16, hi8 = lane & 8;
+  const double r0 = __shfl_xor_sync(0xffffffffu, hi16 ? v0 : v2, 16);
+  const double r1 = __shfl_xor_sync(0xffffffffu, hi16 ? v1 : v3, 16);
+  const double w0 = (hi16 ? v2 : v0) + r0;
+  const double w1 = (hi16 ? v3 : v1) + r1;
+  double z = (hi8 ? w1 : w0) + __shfl_xor_sync(0xffffffffu, hi8 ? w0 : w1, 8);
+  z += __shfl_xor_sync(0xffffffffu, z, 4);
+  z += __shfl_xor_sync(0xffffffffu, z, 2);
+  z += __shfl_xor_sync(0xffffffffu, z, 1);
+  return z;
+}
+
 // kb . LN_s(row) with the row's statistics given; channels are strided over the lanes of a warp.
 template <int CH>
 __device__ __forceinline__ double warp_sim(const double (&kb)[CH], const double* __restrict__ row, double mu, double rs,
@@ -215,7 +234,7 @@ __device__ __forceinline__ double warp_sim(const double (&kb)[CH], const double*
 template <int D>
 __global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideParams p) {
   constexpr int CH = D / 32;
-  __shared__ double s_score[kMaxBlock], s_best[kMaxBlock], s_cmu[kMaxBlock], s_crs[kMaxBlock];
+  __shared__ double s_score[kMaxBlock], s_best[kMaxBlock];
   __shared__ int s_barg[kMaxBlock], s_pi[kMaxBlock], s_creator[kMaxBlock];
   __shared__ int s_pstart[kMaxBlock], s_pcnt[kMaxBlock];
   __shared__ unsigned char s_app[kMaxBlock], s_exh[kMaxBlock];
@@ -315,15 +334,10 @@ __global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideP
       for (int c = 0; c < CH; ++c) acc += kb[lane + 32 * c] * (gam[c] * ((sk[lane + 32 * c] - mu) * rs) + bet[c]);
       part[k] = acc;
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-      for (int k = 0; k < 4; ++k) part[k] += __shfl_xor_sync(0xffffffffu, part[k], o);
-    }
-    if (lane == 0) {
-#pragma unroll
-      for (int k = 0; k < 4; ++k)
-        if (q0 + k * kDecideWarps < np) s_pval[q0 + k * kDecideWarps] = part[k];
+    const double z = warp_reduce4(part[0], part[1], part[2], part[3], lane);
+    if ((lane & 7) == 0) {   // lanes 0, 8, 16, 24 hold pairs 0, 1, 2, 3
+      const int q = q0 + (lane >> 3) * kDecideWarps;
+      if (q < np) s_pval[q] = z;
     }
   }
   __syncthreads();
@@ -376,44 +390,44 @@ __global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideP
 #pragma unroll 8
       for (int jj = 0; jj < tid; ++jj) before += s_app[jj];
       s_creator[before] = tid;          // rows are laid down in ascending token order
-      s_cmu[before] = p.kbarMu[tokBase + tid];
-      s_crs[before] = p.kbarRstd[tokBase + tid];
     }
     __syncthreads();
   }
-  // ---- D: merge target against s_+ (old rows: refined candidates; new rows: exact), warp per token ----
-  for (int j = warp; j < C; j += kDecideWarps) {
-    if (s_app[j]) continue;
-    double best = s_best[j];
-    int arg = s_barg[j];
+  // ---- D: merge target against s_+ (old rows: refined candidates; new rows: exact).  A warp takes
+  //      four tokens at a time, so every row key it loads is used four times, and reduces the four
+  //      partial sums together; lane group t (8 lanes) ends up owning token t of the quad. ----
+  for (int j0 = 4 * warp; j0 < C; j0 += 4 * kDecideWarps) {
+    const int t = ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1);
+    const int jt = j0 + t;                        // the token this lane group decides
+    const bool live = jt < C && !s_app[jt];
+    double best = live ? s_best[jt] : -INFINITY;
+    int arg = live ? s_barg[jt] : -1;
     if (n_a > 0) {
-      double kb[CH];
+      double kb[4][CH];
 #pragma unroll
-      for (int i = 0; i < CH; ++i) kb[i] = kbarU[(int64_t)j * D + lane + 32 * i];
-      for (int a0 = 0; a0 < n_a; a0 += 4) {
-        double part[4];
+      for (int q = 0; q < 4; ++q) {
+        const int j = min(j0 + q, C - 1);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const int a = min(a0 + k, n_a - 1);
-          const double* ka = kbarU + (int64_t)s_creator[a] * D;
-          const double mu = s_cmu[a], rs = s_crs[a];
-          double acc = 0.0;
+        for (int c = 0; c < CH; ++c) kb[q][c] = kbarU[(int64_t)j * D + lane + 32 * c];
+      }
+#pragma unroll 2
+      for (int a = 0; a < n_a; ++a) {
+        const double* kh = p.kbarHat64 + (tokBase + s_creator[a]) * D;
+        double h[CH];
 #pragma unroll
-          for (int c = 0; c < CH; ++c) acc += kb[c] * (gam[c] * ((ka[lane + 32 * c] - mu) * rs) + bet[c]);
-          part[k] = acc;
+        for (int c = 0; c < CH; ++c) h[c] = kh[lane + 32 * c];
+        double part[4] = {0.0, 0.0, 0.0, 0.0};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+#pragma unroll
+          for (int c = 0; c < CH; ++c) part[q] += kb[q][c] * h[c];
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-          for (int k = 0; k < 4; ++k) part[k] += __shfl_xor_sync(0xffffffffu, part[k], o);
-        }
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-          if (a0 + k < n_a && part[k] > best) { best = part[k]; arg = (int)m + a0 + k; }
+        const double z = warp_reduce4(part[0], part[1], part[2], part[3], lane);
+        if (z > best) { best = z; arg = (int)m + a; }
       }
     }
-    if (lane == 0) {
-      s_pi[j] = arg;
+    if (live && (lane & 7) == 0) {
+      s_pi[jt] = arg;
       atomicAdd(&s_nmerge, 1);
     }
   }
@@ -594,14 +608,15 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
   const int C = st->C, D = st->d;
   {
     KernelTimer kt(st, 2, s);
+    const int write_hat = (!a.first && a.n_append > 0 && a.n_append < C) ? 1 : 0;
     dim3 grid((C + 7) / 8, st->U);
     if (D == 128)
       kbar_kernel<128><<<grid, 256, 0, s>>>(a.ok, a.unit_stride, st->ln_w, st->ln_b, st->kbar64, st->kbarH,
-                                            st->kbarNorm, st->kbarMu, st->kbarRstd, C, st->Cmax, st->CbarRows,
+                                            st->kbarNorm, st->kbarHat64, write_hat, C, st->Cmax, st->CbarRows,
                                             st->Hkv, st->r, (double)st->ln_eps);
     else
       kbar_kernel<64><<<grid, 256, 0, s>>>(a.ok, a.unit_stride, st->ln_w, st->ln_b, st->kbar64, st->kbarH,
-                                           st->kbarNorm, st->kbarMu, st->kbarRstd, C, st->Cmax, st->CbarRows,
+                                           st->kbarNorm, st->kbarHat64, write_hat, C, st->Cmax, st->CbarRows,
                                            st->Hkv, st->r, (double)st->ln_eps);
     ++launches;
   }
@@ -630,7 +645,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
       launches += launch_route_filter_tc(st, a.m, nsplit, s);
     }
     FoldDecideParams p;
-    p.kbar64 = st->kbar64; p.kbarNorm = st->kbarNorm; p.kbarMu = st->kbarMu; p.kbarRstd = st->kbarRstd;
+    p.kbar64 = st->kbar64; p.kbarNorm = st->kbarNorm; p.kbarHat64 = st->kbarHat64;
     p.candV = st->candV; p.candI = st->candI; p.ln_w = st->ln_w; p.ln_b = st->ln_b;
     p.sumK = st->sumK; p.kmu = st->kmu; p.krstd = st->krstd;
     p.pi = st->foldPi; p.sorted = st->foldSorted; p.creator = st->foldCreator; p.segnew = st->foldSegNew;

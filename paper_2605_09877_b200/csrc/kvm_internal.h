@@ -61,7 +61,7 @@ struct State {
   __half* kbarH;                 // [U, CbarRows, d]
   float* kbarNorm;               // [U, Cmax]
   int CbarRows;                  // rows per unit of kbarH (Cmax rounded up to the 128-row MMA tile)
-  double *kbarMu, *kbarRstd;     // [U, Cmax]  statistics of LN_s(kbar_j): the key of a row created by j
+  double* kbarHat64;             // [U, Cmax, d]  LN_s(kbar_j): the readout key of a row created by token j
   int32_t *foldPi, *foldSorted, *foldCreator, *foldSegNew, *foldNMerge;  // decisions of the current fold
   int nsplitRoute;               // splits the routing filter may use
   float* candV;                  // [U, nsplitRoute, Cmax, kTopK]
