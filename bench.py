@@ -81,7 +81,9 @@ def prefill_flops(wl, T):
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the kernels that carry a
 # roofline, from the ncu captures summarised under profiles/ (null until captured for the workload).
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    ("cfg5", "decode"): 4.574e9,    # profiles/ncu_full_attn_route_decide_decode_small_cases.md (4.570 GB read + 4 MB written)
+}
 
 
 def peaks():
@@ -361,7 +363,7 @@ def main():
         ach = ((att_f if dom == "attention" else rt_f) / 1e12) / (dom_ms * 1e-3)
         peak = pk["tf_sust"]
         roof = dict(bound="tensor", kernel=dom, achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak,
-                    traffic=NCU_TRAFFIC.get(dom),
+                    traffic=NCU_TRAFFIC.get((wl.name, dom)),
                     peak_source=f"{pk['src']} bf16 sustained (fp16 operands run at the bf16 rate)",
                     launches_per_step=n_dom, avg_launch_us=1e3 * dom_ms / max(n_dom, 1),
                     share_of_device_time=dom_ms / max(sum(per_kernel.values()), 1e-9),
@@ -371,12 +373,16 @@ def main():
         metric, unit, hib = "kvm_prefill_tokens_per_s", "tokens/s", True
     else:
         info = st.info()
-        nwin_avg = 256 + 128
+        # window tokens seen by the profiled steps (the last `nprof` ones): positions t attend [b, t]
+        pos_end = info["position"]
+        steps_t = range(pos_end - nprof, pos_end)
+        nwin_avg = sum(t - max(0, (t // wl.C + 1) * wl.C - wl.w * wl.C) + 1 for t in steps_t) / nprof
         bytes_step = wl.B * wl.Hkv * (info["n_slots"] + nwin_avg) * wl.d * 2 * 2
         dec_ms = prof["decode"][0] / max(prof["decode"][1], 1)
         ach = bytes_step / 1e9 / (dec_ms * 1e-3)
         roof = dict(bound="hbm", kernel="decode", achieved=ach, peak=pk["hbm"], unit="GB/s", frac=ach / pk["hbm"],
-                    traffic=None, peak_source=f"{pk['src']} copy bandwidth", bytes_per_step=bytes_step,
+                    traffic=NCU_TRAFFIC.get((wl.name, "decode")), peak_source=f"{pk['src']} copy bandwidth",
+                    bytes_per_step=bytes_step,
                     frac_of_nominal_8TBs=ach / 8000.0, phase_ms={k_: v_[0] / max(v_[1], 1) for k_, v_ in prof.items()})
         metric, unit, hib = "kvm_decode_us_per_step", "us/step", False
 
