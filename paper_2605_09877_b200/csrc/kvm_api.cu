@@ -102,6 +102,10 @@ kvm_status_t dev_alloc(kvm_state* ks, T** p, size_t count, bool zero = true) {
 void free_all(kvm_state* ks) {
   for (void* p : ks->allocs) cudaFree(p);
   ks->allocs.clear();
+  State& s = ks->s;
+  if (s.foldStream) { cudaStreamDestroy(s.foldStream); s.foldStream = nullptr; }
+  for (cudaEvent_t* e : {&s.evJoin, &s.evAttn[0], &s.evAttn[1], &s.evFold[0], &s.evFold[1]})
+    if (*e) { cudaEventDestroy(*e); *e = nullptr; }
 }
 
 struct DeviceGuard {
@@ -244,7 +248,7 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   A(s.inv_freq, (size_t)d / 2);
   A(s.sumK, U * M * d); A(s.sumV, U * M * d); A(s.rho, U * M); A(s.wsum, U * M); A(s.cnt, U * M);
   A(s.kmu, U * M); A(s.krstd, U * M);
-  A(s.Khat, U * M * d); A(s.Vhat, U * M * d);
+  for (int i = 0; i < 2; ++i) { A(s.KhatBuf[i], U * M * d); A(s.VhatBuf[i], U * M * d); }
   A(s.ringK, U * ringCap * d); A(s.ringV, U * ringCap * d); A(s.ringG, U * ringCap);
   A(s.stQ, (size_t)s.B * s.Hq * s.Tcall * d);
   A(s.stK, U * (size_t)s.stRows * d); A(s.stV, U * (size_t)s.stRows * d); A(s.stG, U * (size_t)s.stRows);
@@ -252,7 +256,10 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   s.CbarRows = (s.Cmax + 127) / 128 * 128;
   A(s.kbar64, U * Cm * d); A(s.kbarH, U * (size_t)s.CbarRows * d); A(s.kbarNorm, U * Cm);
   A(s.kbarHat64, U * Cm * d);
-  A(s.foldPi, U * Cm); A(s.foldSorted, U * Cm); A(s.foldCreator, U * Cm); A(s.foldSegNew, U * Cm); A(s.foldNMerge, U);
+  for (int i = 0; i < 2; ++i) {
+    A(s.foldPi[i], U * Cm); A(s.foldSorted[i], U * Cm); A(s.foldCreator[i], U * Cm); A(s.foldSegNew[i], U * Cm);
+    A(s.foldNMerge[i], U);
+  }
   A(s.candV, U * (size_t)s.nsplitRoute * Cm * kTopK); A(s.candI, U * (size_t)s.nsplitRoute * Cm * kTopK);
   A(s.decPart, (size_t)s.B * s.Hq * s.nsplitDec * (d + 2)); A(s.decQ, (size_t)s.B * s.Hq * d);
   A(s.status, (size_t)16);   // [0] status word, [1..3] fold debug counters
@@ -268,6 +275,12 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
     if (!ok) rc = KVM_ERR_CUDA;
   }
   if (rc == KVM_OK && !(setup_attn_tc(&s) && setup_route_tc(&s))) rc = KVM_ERR_CUDA;
+  if (rc == KVM_OK) {
+    bool ok = cudaStreamCreateWithFlags(&s.foldStream, cudaStreamNonBlocking) == cudaSuccess;
+    for (cudaEvent_t* e : {&s.evJoin, &s.evAttn[0], &s.evAttn[1], &s.evFold[0], &s.evFold[1]})
+      ok = ok && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) rc = KVM_ERR_CUDA;
+  }
   if (rc != KVM_OK) {
     cudaGetLastError();
     free_all(ks);
@@ -303,7 +316,7 @@ KVM_API kvm_status_t kvm_debug_counters(kvm_state_t* ks, int64_t* out, void* cud
 KVM_API kvm_status_t kvm_state_reset(kvm_state_t* ks) {
   if (!ks) return KVM_ERR_INVALID_ARG;
   State& s = ks->s;
-  s.bound = false; s.pos = 0; s.m = 0; s.nfolds = 0;
+  s.bound = false; s.pos = 0; s.m = 0; s.nfolds = 0; s.prevValid = false;
   if (s.slotTok) {  // debug recording only: forget the previous sequence's assignments
     DeviceGuard guard(s.device);
     if (cudaMemset(s.slotTok, 0xff, (size_t)s.U * s.Tassign * sizeof(int32_t)) != cudaSuccess) return KVM_ERR_CUDA;
@@ -414,8 +427,24 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
   }
   { KernelTimer pt(&s, 0, stream); s.launches += launch_ingest(&s, ia, stream); }
 
-  const bool simt_attn = true;  // replaced by the tcgen05 kernel selection below once available
-  (void)simt_attn;
+  // Two streams: attention runs on the caller's stream, folds on the state's own stream.  The fold
+  // that ends block c needs the state after the fold before it and block c-w+1's keys, not block c's
+  // attention, so the two overlap.  Orderings kept by events:
+  //   fold stream waits for the ingest (and with it for everything earlier on the caller's stream);
+  //   attention(c+1) waits for the fold that ends block c (it reads the readout copy that fold wrote);
+  //   the fold that ends block c waits for attention(c-1), which read the copy it overwrites;
+  //   the caller's stream waits for the last fold before the call returns.
+  // With the per-kernel timing hook on, everything stays on the caller's stream so that the
+  // measured durations are those of kernels running alone.
+  const bool overlap = s.prof_hook == nullptr;
+  cudaStream_t fstream = overlap ? s.foldStream : stream;
+  bool ev_ok = true;
+  if (overlap) {
+    ev_ok = ev_ok && cudaEventRecord(s.evJoin, stream) == cudaSuccess;
+    ev_ok = ev_ok && cudaStreamWaitEvent(fstream, s.evJoin, 0) == cudaSuccess;
+  }
+  bool attn_rec[2] = {false, false};   // evAttn[i] recorded in this call
+  int fold_pending = -1;               // evFold index the next attention must wait for
   for (int64_t c = c0; c <= c_last; ++c) {
     const int64_t e = (c + 1) * C;
     const int64_t qs = c * C > pos0 ? c * C : pos0;
@@ -423,10 +452,18 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
     int64_t b = e - L; if (b < 0) b = 0;
     aa.q_row0 = qs - pos0; aa.nq = (int)(qe - qs); aa.t0 = qs; aa.m = s.m;
     aa.win_row0 = b - ia.hist_start; aa.b = b; aa.out = (__nv_bfloat16*)out; aa.out_t0 = qs - pos0;
+    if (overlap && fold_pending >= 0) {
+      ev_ok = ev_ok && cudaStreamWaitEvent(stream, s.evFold[fold_pending], 0) == cudaSuccess;
+      fold_pending = -1;
+    }
     {
       KernelTimer pt(&s, 1, stream);
       if (s.flags & KVM_FLAG_SIMT_ATTENTION) s.launches += launch_attn_simt(&s, aa, stream);
       else s.launches += launch_attn_tc(&s, aa, stream);
+    }
+    if (overlap) {
+      ev_ok = ev_ok && cudaEventRecord(s.evAttn[c & 1], stream) == cudaSuccess;
+      attn_rec[c & 1] = true;
     }
     if (qe == e && c >= s.w - 1) {
       FoldArgs fa;
@@ -434,12 +471,20 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
       fa.unit_stride = s.stRows * d; fa.gate_stride = s.stRows;
       fa.b = b; fa.m = s.m; fa.first = (s.m == 0);
       fa.n_append = fa.first ? C : (int)n_append_of(s.growth, e, s.m, C);
-      s.launches += launch_fold(&s, fa, stream);
+      if (overlap && attn_rec[(c - 1) & 1])
+        ev_ok = ev_ok && cudaStreamWaitEvent(fstream, s.evAttn[(c - 1) & 1], 0) == cudaSuccess;
+      s.launches += launch_fold(&s, fa, fstream);
       s.m += fa.n_append;
       s.nfolds += 1;
+      if (overlap) {
+        fold_pending = (int)(s.nfolds & 1);
+        ev_ok = ev_ok && cudaEventRecord(s.evFold[fold_pending], fstream) == cudaSuccess;
+      }
     }
   }
+  if (overlap && fold_pending >= 0) ev_ok = ev_ok && cudaStreamWaitEvent(stream, s.evFold[fold_pending], 0) == cudaSuccess;
   s.pos = pos1;
+  if (!ev_ok) { cudaGetLastError(); return KVM_ERR_CUDA; }
   return launch_ok() ? KVM_OK : KVM_ERR_CUDA;
 }
 
@@ -545,8 +590,8 @@ KVM_API kvm_status_t kvm_state_export(kvm_state_t* ks, double* sum_k, float* sum
     CP(radius, s.rho, sizeof(float), (size_t)1);
     CP(weight, s.wsum, sizeof(double), (size_t)1);
     CP(count, s.cnt, sizeof(int32_t), (size_t)1);
-    CP(k_read, s.Khat, (size_t)2, d);
-    CP(v_read, s.Vhat, (size_t)2, d);
+    CP(k_read, s.KhatBuf[s.nfolds & 1], (size_t)2, d);
+    CP(v_read, s.VhatBuf[s.nfolds & 1], (size_t)2, d);
 #undef CP
   }
   ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;

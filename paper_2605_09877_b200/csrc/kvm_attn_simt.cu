@@ -132,7 +132,7 @@ __global__ void __launch_bounds__(256) attn_simt_kernel(AttnSimtParams p) {
 
 int launch_attn_simt(State* st, const AttnArgs& a, cudaStream_t s) {
   AttnSimtParams p;
-  p.stQ = st->stQ; p.stK = st->stK; p.stV = st->stV; p.Khat = st->Khat; p.Vhat = st->Vhat;
+  p.stQ = st->stQ; p.stK = st->stK; p.stV = st->stV; p.Khat = st->KhatBuf[st->nfolds & 1]; p.Vhat = st->VhatBuf[st->nfolds & 1];
   p.tau_s = st->tau_s; p.tau_b = st->tau_b;
   p.out = a.out;
   p.Tcall = st->Tcall; p.stRows = st->stRows; p.Mcap = st->Mcap;

@@ -359,10 +359,11 @@ int launch_attn_tc(State* st, const AttnArgs& a, cudaStream_t s) {
   p.nq = a.nq; p.Hq = st->Hq; p.Hkv = st->Hkv; p.G = st->G;
   dim3 grid((a.nq + 127) / 128, st->B * st->Hq);
   const CUtensorMap* tm = reinterpret_cast<const CUtensorMap*>(st->tmaps);
+  const int ks = (st->nfolds & 1) ? 6 : 1, vs = (st->nfolds & 1) ? 7 : 2;   // readout copy of the current version
   if (st->d == 128) {
-    attn_tc_kernel<128><<<grid, 192, AttnTcCfg<128>::SMEM_BYTES, s>>>(tm[0], tm[1], tm[2], tm[3], tm[4], p);
+    attn_tc_kernel<128><<<grid, 192, AttnTcCfg<128>::SMEM_BYTES, s>>>(tm[0], tm[ks], tm[vs], tm[3], tm[4], p);
   } else {
-    attn_tc_kernel<64><<<grid, 192, AttnTcCfg<64>::SMEM_BYTES, s>>>(tm[0], tm[1], tm[2], tm[3], tm[4], p);
+    attn_tc_kernel<64><<<grid, 192, AttnTcCfg<64>::SMEM_BYTES, s>>>(tm[0], tm[ks], tm[vs], tm[3], tm[4], p);
   }
   return 1;
 }
@@ -370,8 +371,10 @@ int launch_attn_tc(State* st, const AttnArgs& a, cudaStream_t s) {
 bool setup_attn_tc(State* st) {
   CUtensorMap* tm = reinterpret_cast<CUtensorMap*>(st->tmaps);
   bool ok = encode_tmap_rows(&tm[0], st->stQ, st->d, st->Tcall, (int64_t)st->B * st->Hq, 128);
-  ok = ok && encode_tmap_rows(&tm[1], st->Khat, st->d, st->Mcap, st->U, 128);
-  ok = ok && encode_tmap_rows(&tm[2], st->Vhat, st->d, st->Mcap, st->U, 128);
+  ok = ok && encode_tmap_rows(&tm[1], st->KhatBuf[0], st->d, st->Mcap, st->U, 128);
+  ok = ok && encode_tmap_rows(&tm[2], st->VhatBuf[0], st->d, st->Mcap, st->U, 128);
+  ok = ok && encode_tmap_rows(&tm[6], st->KhatBuf[1], st->d, st->Mcap, st->U, 128);
+  ok = ok && encode_tmap_rows(&tm[7], st->VhatBuf[1], st->d, st->Mcap, st->U, 128);
   ok = ok && encode_tmap_rows(&tm[3], st->stK, st->d, st->stRows, st->U, 128);
   ok = ok && encode_tmap_rows(&tm[4], st->stV, st->d, st->stRows, st->U, 128);
   if (!ok) return false;

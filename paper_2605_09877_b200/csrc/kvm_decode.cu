@@ -235,7 +235,7 @@ int launch_decode(State* st, const DecodeArgs& a, cudaStream_t s) {
                                               st->ringLen);
   ++launches;
   DecodeParams p;
-  p.decQ = st->decQ; p.Khat = st->Khat; p.Vhat = st->Vhat; p.ringK = st->ringK; p.ringV = st->ringV;
+  p.decQ = st->decQ; p.Khat = st->KhatBuf[st->nfolds & 1]; p.Vhat = st->VhatBuf[st->nfolds & 1]; p.ringK = st->ringK; p.ringV = st->ringV;
   p.tau_s = st->tau_s; p.tau_b = st->tau_b; p.out = a.out; p.part = st->decPart;
   p.Mcap = st->Mcap; p.ringCap = (int64_t)st->w * st->Cmax; p.ringLen = st->ringLen;
   p.m = a.m; p.b = a.b; p.t = a.t;

@@ -41,18 +41,50 @@ __device__ __forceinline__ void row_stats(const double (&x)[CH], int D, double e
 // ------------------------------------------------------------------------------------------
 // 1. memory keys (one warp per overflow token)
 
+struct PrevFoldCopy {
+  int valid, all_append, n_append;
+  int64_t m, Mcap;                       // rows before the previous fold; row capacity per unit
+  const int32_t *pi, *sorted, *nmerge;   // the previous fold's decisions
+  const __half *Ksrc, *Vsrc;             // readout copy of the current version
+  __half *Kdst, *Vdst;                   // readout copy this fold writes
+};
+
 template <int D>
 __global__ void __launch_bounds__(256) kbar_kernel(const __half* __restrict__ ok, int64_t unit_stride,
                                                    const float* __restrict__ ln_w, const float* __restrict__ ln_b,
                                                    double* __restrict__ kbar64, __half* __restrict__ kbarH,
                                                    float* __restrict__ kbarNorm, double* __restrict__ kbarHat64,
                                                    int write_hat, int C, int Cmax, int CbarRows,
-                                                   int Hkv, int r, double ln_eps) {
+                                                   int Hkv, int r, double ln_eps, PrevFoldCopy pc) {
   constexpr int CH = D / 32;
   const int u = blockIdx.y, hk = u % Hkv;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int j = blockIdx.x * 8 + warp;
   if (j >= C) return;
+  // Rows that the previous fold touched are current in the source readout copy only: bring them
+  // over to the copy this fold writes (warp j takes the j-th appended row and the j-th merge target,
+  // as the apply kernel did).  The index loads are independent of one another and the rows are held
+  // in registers across the normalisation below, so their latency overlaps it.
+  uint2 cpK[2], cpV[2];
+  int64_t cpo[2] = {-1, -1};
+  if (pc.valid) {
+    const int64_t tb = (int64_t)u * Cmax;
+    if (j < pc.n_append) cpo[0] = ((int64_t)u * pc.Mcap + pc.m + j) * D;
+    if (!pc.all_append) {
+      const int nm = pc.nmerge[u];
+      int s0 = pc.sorted[tb + j], s1 = pc.sorted[tb + (j > 0 ? j - 1 : 0)];
+      s0 = (unsigned)s0 < (unsigned)Cmax ? s0 : 0;   // entries past nmerge are not defined
+      s1 = (unsigned)s1 < (unsigned)Cmax ? s1 : 0;
+      const int r1 = pc.pi[tb + s0], r0 = pc.pi[tb + s1];
+      if (j < nm && r1 >= 0 && r1 < pc.m && (j == 0 || r0 != r1)) cpo[1] = ((int64_t)u * pc.Mcap + r1) * D;
+    }
+#pragma unroll
+    for (int t = 0; t < 2; ++t)
+      if (cpo[t] >= 0 && lane < D / 4) {   // 8 bytes per lane
+        cpK[t] = reinterpret_cast<const uint2*>(pc.Ksrc + cpo[t])[lane];
+        cpV[t] = reinterpret_cast<const uint2*>(pc.Vsrc + cpo[t])[lane];
+      }
+  }
   const __half* row = ok + (int64_t)u * unit_stride + (int64_t)j * D;
   double val[CH];
 #pragma unroll
@@ -86,6 +118,12 @@ __global__ void __launch_bounds__(256) kbar_kernel(const __half* __restrict__ ok
     }
   }
   if (lane == 0) kbarNorm[(int64_t)u * Cmax + j] = (float)sqrt(n2) * 1.000001f;
+#pragma unroll
+  for (int t = 0; t < 2; ++t)
+    if (cpo[t] >= 0 && lane < D / 4) {
+      reinterpret_cast<uint2*>(pc.Kdst + cpo[t])[lane] = cpK[t];
+      reinterpret_cast<uint2*>(pc.Vdst + cpo[t])[lane] = cpV[t];
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -606,18 +644,25 @@ int launch_route_filter_tc(State* st, int64_t m, int nsplit, cudaStream_t s);
 int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
   int launches = 0;
   const int C = st->C, D = st->d;
+  // the state after nfolds folds is read from readout copy `src`; this fold writes copy `dst`
+  const int src = (int)(st->nfolds & 1), dst = src ^ 1;
   {
     KernelTimer kt(st, 2, s);
     const int write_hat = (!a.first && a.n_append > 0 && a.n_append < C) ? 1 : 0;
+    PrevFoldCopy pc;
+    pc.valid = st->prevValid ? 1 : 0; pc.all_append = st->prevAllAppend ? 1 : 0; pc.n_append = st->prevNAppend;
+    pc.m = st->prevM; pc.Mcap = st->Mcap;
+    pc.pi = st->foldPi[src]; pc.sorted = st->foldSorted[src]; pc.nmerge = st->foldNMerge[src];
+    pc.Ksrc = st->KhatBuf[src]; pc.Vsrc = st->VhatBuf[src]; pc.Kdst = st->KhatBuf[dst]; pc.Vdst = st->VhatBuf[dst];
     dim3 grid((C + 7) / 8, st->U);
     if (D == 128)
       kbar_kernel<128><<<grid, 256, 0, s>>>(a.ok, a.unit_stride, st->ln_w, st->ln_b, st->kbar64, st->kbarH,
                                             st->kbarNorm, st->kbarHat64, write_hat, C, st->Cmax, st->CbarRows,
-                                            st->Hkv, st->r, (double)st->ln_eps);
+                                            st->Hkv, st->r, (double)st->ln_eps, pc);
     else
       kbar_kernel<64><<<grid, 256, 0, s>>>(a.ok, a.unit_stride, st->ln_w, st->ln_b, st->kbar64, st->kbarH,
                                            st->kbarNorm, st->kbarHat64, write_hat, C, st->Cmax, st->CbarRows,
-                                           st->Hkv, st->r, (double)st->ln_eps);
+                                           st->Hkv, st->r, (double)st->ln_eps, pc);
     ++launches;
   }
   const bool all_append = a.first || a.n_append >= C;
@@ -632,11 +677,11 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
       KernelTimer kt(st, 3, s);
       dim3 grid(nsplit, st->U);
       if (D == 128)
-        route_filter_simt_kernel<128><<<grid, 256, 0, s>>>(st->kbarH, st->Khat, st->candV, st->candI, C, st->Cmax,
+        route_filter_simt_kernel<128><<<grid, 256, 0, s>>>(st->kbarH, st->KhatBuf[src], st->candV, st->candI, C, st->Cmax,
                                                            st->CbarRows, st->Mcap, a.m, nsplit, st->kbarNorm,
                                                            route_thr_coeff(st), st->S);
       else
-        route_filter_simt_kernel<64><<<grid, 256, 0, s>>>(st->kbarH, st->Khat, st->candV, st->candI, C, st->Cmax,
+        route_filter_simt_kernel<64><<<grid, 256, 0, s>>>(st->kbarH, st->KhatBuf[src], st->candV, st->candI, C, st->Cmax,
                                                           st->CbarRows, st->Mcap, a.m, nsplit, st->kbarNorm,
                                                           route_thr_coeff(st), st->S);
       ++launches;
@@ -648,8 +693,8 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
     p.kbar64 = st->kbar64; p.kbarNorm = st->kbarNorm; p.kbarHat64 = st->kbarHat64;
     p.candV = st->candV; p.candI = st->candI; p.ln_w = st->ln_w; p.ln_b = st->ln_b;
     p.sumK = st->sumK; p.kmu = st->kmu; p.krstd = st->krstd;
-    p.pi = st->foldPi; p.sorted = st->foldSorted; p.creator = st->foldCreator; p.segnew = st->foldSegNew;
-    p.nmerge = st->foldNMerge;
+    p.pi = st->foldPi[dst]; p.sorted = st->foldSorted[dst]; p.creator = st->foldCreator[dst];
+    p.segnew = st->foldSegNew[dst]; p.nmerge = st->foldNMerge[dst];
     p.counters = st->status + 1;
     p.Mcap = st->Mcap; p.m = a.m;
     p.C = C; p.Cmax = st->Cmax; p.Hkv = st->Hkv; p.S = st->S; p.n_append = a.n_append; p.nsplit = nsplit;
@@ -662,10 +707,10 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
   FoldApplyParams q;
   q.ov = a.ov; q.og = a.og; q.unit_stride = a.unit_stride; q.gate_stride = a.gate_stride;
   q.kbar64 = st->kbar64; q.ln_w = st->ln_w; q.ln_b = st->ln_b;
-  q.pi = st->foldPi; q.sorted = st->foldSorted; q.creator = st->foldCreator; q.segnew = st->foldSegNew;
-  q.nmerge = st->foldNMerge;
+  q.pi = st->foldPi[dst]; q.sorted = st->foldSorted[dst]; q.creator = st->foldCreator[dst];
+  q.segnew = st->foldSegNew[dst]; q.nmerge = st->foldNMerge[dst];
   q.sumK = st->sumK; q.sumV = st->sumV; q.rho = st->rho; q.wsum = st->wsum; q.cnt = st->cnt;
-  q.kmu = st->kmu; q.krstd = st->krstd; q.Khat = st->Khat; q.Vhat = st->Vhat;
+  q.kmu = st->kmu; q.krstd = st->krstd; q.Khat = st->KhatBuf[dst]; q.Vhat = st->VhatBuf[dst];
   q.slotTok = st->slotTok; q.appTok = st->appTok;
   q.Mcap = st->Mcap; q.Tassign = st->Tassign; q.m = a.m; q.b = a.b;
   q.C = C; q.Cmax = st->Cmax; q.Hkv = st->Hkv; q.n_append = a.n_append; q.all_append = all_append ? 1 : 0;
@@ -676,6 +721,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
   if (D == 128) fold_apply_kernel<128><<<grid, 256, 0, s>>>(q);
   else fold_apply_kernel<64><<<grid, 256, 0, s>>>(q);
   ++launches;
+  st->prevValid = true; st->prevAllAppend = all_append; st->prevM = a.m; st->prevNAppend = a.n_append;
   return launches;
 }
 

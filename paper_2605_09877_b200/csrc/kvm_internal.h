@@ -45,8 +45,17 @@ struct State {
   double* wsum;           // [U, Mcap]
   int32_t* cnt;           // [U, Mcap]
   double *kmu, *krstd;    // [U, Mcap]   mean / rstd of LN_s(s^K_i)
-  __half *Khat, *Vhat;    // [U, Mcap, d]  readout cache (fp16): LN_s(s^K) and the value readout;
-                          //               operand of attention, decode and the routing filter
+  // Readout cache (fp16): LN_s(s^K) and the value readout, each [U, Mcap, d]; operand of attention,
+  // decode and the routing filter.  Two copies: the state after f folds is read from copy f & 1, so
+  // fold f+1 can write copy (f+1) & 1 while the attention of the current block still reads copy f & 1.
+  __half *KhatBuf[2], *VhatBuf[2];
+  // what the previous fold touched (host): its rows are copied into the other copy by the next fold
+  bool prevValid, prevAllAppend;
+  int64_t prevM;
+  int prevNAppend;
+  // second stream and events that let a block's attention and the fold of the block before it overlap
+  cudaStream_t foldStream;
+  cudaEvent_t evJoin, evAttn[2], evFold[2];
   // ---- window ring (device): slot = t mod ringLen ----
   __half *ringK, *ringV;         // [U, w*Cmax, d]  rotated keys / values (fp16)
   float* ringG;                  // [U, w*Cmax]
@@ -62,7 +71,8 @@ struct State {
   float* kbarNorm;               // [U, Cmax]
   int CbarRows;                  // rows per unit of kbarH (Cmax rounded up to the 128-row MMA tile)
   double* kbarHat64;             // [U, Cmax, d]  LN_s(kbar_j): the readout key of a row created by token j
-  int32_t *foldPi, *foldSorted, *foldCreator, *foldSegNew, *foldNMerge;  // decisions of the current fold
+  // decisions of the fold being computed ([(nfolds+1) & 1]) and of the one before ([nfolds & 1])
+  int32_t *foldPi[2], *foldSorted[2], *foldCreator[2], *foldSegNew[2], *foldNMerge[2];
   int nsplitRoute;               // splits the routing filter may use
   float* candV;                  // [U, nsplitRoute, Cmax, kTopK]
   int32_t* candI;
@@ -78,7 +88,8 @@ struct State {
   int32_t* slotTok;              // [U, Tassign]
   uint8_t* appTok;               // [U, Tassign]
   int32_t* status;               // device status word
-  // ---- TMA tensor maps (host copies, passed to kernels by value): stQ, Khat, Vhat, stK, stV, kbarH ----
+  // ---- TMA tensor maps (host copies, passed to kernels by value):
+  //      0 stQ, 1 Khat copy 0, 2 Vhat copy 0, 3 stK, 4 stV, 5 kbarH, 6 Khat copy 1, 7 Vhat copy 1 ----
   alignas(64) unsigned char tmaps[8 * 128];
   // ---- device staging for the *_host entry points ----
   void *hQ, *hK, *hV, *hOut;

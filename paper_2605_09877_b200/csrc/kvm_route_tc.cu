@@ -235,8 +235,9 @@ int launch_route_filter_tc(State* st, int64_t m, int nsplit, cudaStream_t s) {
   p.kbarNorm = st->kbarNorm; p.thr_coeff = route_thr_coeff(st);
   const CUtensorMap* tm = reinterpret_cast<const CUtensorMap*>(st->tmaps);
   dim3 grid(nsplit, st->U);
-  if (st->d == 128) route_filter_tc_kernel<128><<<grid, 320, RouteTcCfg<128>::SMEM_BYTES, s>>>(tm[5], tm[1], p);
-  else route_filter_tc_kernel<64><<<grid, 320, RouteTcCfg<64>::SMEM_BYTES, s>>>(tm[5], tm[1], p);
+  const int ks = (st->nfolds & 1) ? 6 : 1;   // the fold reads the readout copy of the current version
+  if (st->d == 128) route_filter_tc_kernel<128><<<grid, 320, RouteTcCfg<128>::SMEM_BYTES, s>>>(tm[5], tm[ks], p);
+  else route_filter_tc_kernel<64><<<grid, 320, RouteTcCfg<64>::SMEM_BYTES, s>>>(tm[5], tm[ks], p);
   return 1;
 }
 
