@@ -3,17 +3,22 @@
 // the window, per-region temperatures).
 //
 // One CTA owns a 128-query tile of one (batch, query head) and walks the key tiles (128 keys:
-// first the state's readout cache, then the window) with three warp roles:
+// first the state's readout cache, then the window) with these warp roles:
 //   warp 0      TMA producer: Q once, then K/V tiles into a 2-stage shared-memory ring
 //               (cp.async.bulk.tensor, 128-byte swizzle, mbarrier complete_tx)
-//   warp 1      MMA issuer: S = Q K^T into a double-buffered TMEM accumulator and
-//               O += P V into a second TMEM accumulator (tcgen05.mma kind::f16, fp32 accumulate)
-//   warps 2-5   softmax: each thread owns one query row (tcgen05.ld 32x32b), applies the region
-//               temperature and masks, keeps the running max / sum in registers, rescales O in TMEM
-//               only when the max grew by more than 2^8 (the final 1/l normalisation makes the
-//               stale max exact), writes P as fp16 into double-buffered swizzled shared memory for
-//               the PV MMA (so the exponentials of tile j+1 overlap the PV product of tile j),
-//               and finally normalises O and stores bf16 rows.
+//   warp 1      QK^T issuer: S = Q K^T into a double-buffered TMEM accumulator
+//   warp 2      PV issuer: O_h += P_h V_h into two more TMEM accumulators
+//               (tcgen05.mma kind::f16, fp32 accumulate; one elected thread each - issuing an MMA
+//               takes about as long as executing it, so one thread cannot keep the pipe full and
+//               also wait on barriers)
+//   warps 4-11  softmax, two warpgroups: warpgroup h owns keys [64h, 64h+64) of every tile and each of
+//               its threads one query row (tcgen05.ld 32x32b); it applies the region temperature and
+//               masks, keeps a running max / sum of its own in registers, and its half of P (fp16,
+//               double-buffered swizzled shared memory) feeds PV products that accumulate into an O
+//               accumulator of its own, rescaled in TMEM only when its max grew by more than 2^8.
+//               The two partial results (O_h, m_h, l_h) are merged in the epilogue like split-K
+//               partials, normalised and stored as bf16 rows.  Splitting by columns halves the
+//               exponentials and conversions per thread, which is what bounds a tile's turnaround.
 // Every mbarrier wait is bounded; on expiry the CTA records KVM_ERR_TIMEOUT and tears down.
 #include "kvm_internal.h"
 #include "tc_common.cuh"
@@ -45,13 +50,15 @@ struct AttnTcCfg {
   // allocation) is resident per SM
   static constexpr int SMEM_BYTES = (OFF_BAR + 256 + 1024) > 120 * 1024 ? (OFF_BAR + 256 + 1024) : 120 * 1024;
   static constexpr uint32_t TMEM_COLS = 512;
-  static constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_O = 256;
+  static constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_O0 = 256, COL_O1 = 384;
 };
 
-enum { BAR_QFULL = 0, BAR_KFULL = 1, BAR_VFULL = 3, BAR_FREE = 5, BAR_SFULL = 7, BAR_PFULL = 9, BAR_PVDONE = 11, BAR_KFREE = 13, BAR_COUNT = 15 };
+// SFULL[i] (QK^T of a tile done) also tells the producer that K stage i is free again, PVDONE[i]
+// (PV of a tile done) that V stage i is: stage and accumulator parity coincide because NS == 2.
+enum { BAR_QFULL = 0, BAR_KFULL = 1, BAR_VFULL = 3, BAR_SFULL = 5, BAR_PFULL = 7, BAR_PVDONE = 9, BAR_COUNT = 11 };
 
 template <int D>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(384, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapKs,
                const __grid_constant__ CUtensorMap mapVs, const __grid_constant__ CUtensorMap mapKw,
                const __grid_constant__ CUtensorMap mapVw, const AttnTcParams p) {
@@ -82,13 +89,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     for (int s = 0; s < Cfg::NS; ++s) {
       tc::mbar_init(&bars[BAR_KFULL + s], 1);
       tc::mbar_init(&bars[BAR_VFULL + s], 1);
-      tc::mbar_init(&bars[BAR_FREE + s], 1);
-      tc::mbar_init(&bars[BAR_KFREE + s], 1);
     }
     tc::mbar_init(&bars[BAR_SFULL + 0], 1);
     tc::mbar_init(&bars[BAR_SFULL + 1], 1);
-    tc::mbar_init(&bars[BAR_PFULL + 0], 4);
-    tc::mbar_init(&bars[BAR_PFULL + 1], 4);
+    tc::mbar_init(&bars[BAR_PFULL + 0], 8);
+    tc::mbar_init(&bars[BAR_PFULL + 1], 8);
     tc::mbar_init(&bars[BAR_PVDONE + 0], 1);
     tc::mbar_init(&bars[BAR_PVDONE + 1], 1);
     *abort_flag = 0;
@@ -123,7 +128,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       // in flight while the softmax of the current one runs.
       auto load_k = [&](int j) -> bool {
         const int s = j % Cfg::NS;
-        if (j >= Cfg::NS && !tc::mbar_wait(&bars[BAR_KFREE + s], ((j / Cfg::NS) - 1) & 1)) return false;
+        if (j >= Cfg::NS && !tc::mbar_wait(&bars[BAR_SFULL + s], ((j / Cfg::NS) - 1) & 1)) return false;
         const bool st = j < nst;
         const int row = st ? j * 128 : (int)(p.win_row0 + (int64_t)(j - nst) * 128);
         tc::mbar_expect_tx(&bars[BAR_KFULL + s], Cfg::TILE_BYTES);
@@ -136,7 +141,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         const int s = j % Cfg::NS;
         if (*abort_flag) break;
         if (j + 1 < ntiles && !load_k(j + 1)) { okp = false; break; }
-        if (j >= Cfg::NS && !tc::mbar_wait(&bars[BAR_FREE + s], ((j / Cfg::NS) - 1) & 1)) { okp = false; break; }
+        if (j >= Cfg::NS && !tc::mbar_wait(&bars[BAR_PVDONE + s], ((j / Cfg::NS) - 1) & 1)) { okp = false; break; }
         const bool st = j < nst;
         const int row = st ? j * 128 : (int)(p.win_row0 + (int64_t)(j - nst) * 128);
         tc::mbar_expect_tx(&bars[BAR_VFULL + s], Cfg::TILE_BYTES);
@@ -146,57 +151,73 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       if (!okp) { atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; }
     }
   } else if (warp == 1) {
-    // ------------------------------ MMA issuer ------------------------------
+    // ------------------------------ QK^T issuer ------------------------------
+    // Issuing a tcgen05.mma takes about as long as executing it, so the two products of a tile are
+    // issued by two threads: the waits, fences and commits of one overlap the issue of the other.
     if (lane == 0) {
       constexpr uint32_t IDESC_QK = tc::idesc_f16(128, 128, false);
-      constexpr uint32_t IDESC_PV = tc::idesc_f16(128, D, true);
-      const uint32_t aQ = tc::smem_u32(sQ), aK = tc::smem_u32(sK), aV = tc::smem_u32(sV), aP = tc::smem_u32(sP);
+      const uint32_t aQ = tc::smem_u32(sQ), aK = tc::smem_u32(sK);
       bool dead = false;
-      auto issue_qk = [&](int j) -> bool {
-        const int s = j % Cfg::NS;
-        if (!tc::mbar_wait(&bars[BAR_KFULL + s], (j / Cfg::NS) & 1)) return false;
-        tc::tc_fence_after();
-        const uint32_t dS = tmem + ((j & 1) ? Cfg::COL_S1 : Cfg::COL_S0);
-#pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-          const uint32_t off = (ks / 4) * Cfg::BOX_BYTES + (ks % 4) * 32;
-          tc::mma_f16_ss(dS, tc::smem_desc_sw128(aQ + off, 16, 1024),
-                         tc::smem_desc_sw128(aK + s * Cfg::TILE_BYTES + off, 16, 1024), IDESC_QK, ks > 0);
-        }
-        tc::mma_commit(&bars[BAR_SFULL + (j & 1)]);
-        tc::mma_commit(&bars[BAR_KFREE + s]);
-        return true;
-      };
       do {
         if (!tc::mbar_wait(&bars[BAR_QFULL], 0)) { dead = true; break; }
-        if (ntiles > 0 && !issue_qk(0)) { dead = true; break; }
         for (int j = 0; j < ntiles; ++j) {
           const int s = j % Cfg::NS;
           if (*abort_flag) { dead = true; break; }
-          if (j + 1 < ntiles && !issue_qk(j + 1)) { dead = true; break; }
-          if (!tc::mbar_wait(&bars[BAR_PFULL + (j & 1)], (j >> 1) & 1)) { dead = true; break; }
-          if (!tc::mbar_wait(&bars[BAR_VFULL + s], (j / Cfg::NS) & 1)) { dead = true; break; }
+          // accumulator S[j & 1] is free once both softmax halves have read tile j-2 out of it
+          if (j >= 2 && !tc::mbar_wait(&bars[BAR_PFULL + (j & 1)], ((j >> 1) - 1) & 1)) { dead = true; break; }
+          if (!tc::mbar_wait(&bars[BAR_KFULL + s], (j / Cfg::NS) & 1)) { dead = true; break; }
           tc::tc_fence_after();
-          const uint32_t dO = tmem + Cfg::COL_O;
+          const uint32_t dS = tmem + ((j & 1) ? Cfg::COL_S1 : Cfg::COL_S0);
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint32_t offP = (j & 1) * Cfg::P_BYTES + (kk / 4) * Cfg::BOX_BYTES + (kk % 4) * 32;
-            const uint32_t offV = kk * 2048;   // 16 key rows x 128 B
-            tc::mma_f16_ss(dO, tc::smem_desc_sw128(aP + offP, 16, 1024),
-                           tc::smem_desc_sw128(aV + s * Cfg::TILE_BYTES + offV, Cfg::BOX_BYTES, 1024), IDESC_PV,
-                           (j > 0 || kk > 0) ? 1u : 0u);
+          for (int ks = 0; ks < D / 16; ++ks) {
+            const uint32_t off = (ks / 4) * Cfg::BOX_BYTES + (ks % 4) * 32;
+            tc::mma_f16_ss(dS, tc::smem_desc_sw128(aQ + off, 16, 1024),
+                           tc::smem_desc_sw128(aK + s * Cfg::TILE_BYTES + off, 16, 1024), IDESC_QK, ks > 0);
           }
-          tc::mma_commit(&bars[BAR_FREE + s]);
-          tc::mma_commit(&bars[BAR_PVDONE + (j & 1)]);
+          tc::mma_commit(&bars[BAR_SFULL + (j & 1)]);
         }
       } while (false);
       if (dead) { atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; }
     }
+  } else if (warp == 2) {
+    // ------------------------------ PV issuer ------------------------------
+    if (lane == 0) {
+      constexpr uint32_t IDESC_PV = tc::idesc_f16(128, D, true);
+      const uint32_t aV = tc::smem_u32(sV), aP = tc::smem_u32(sP);
+      bool dead = false;
+      for (int j = 0; j < ntiles; ++j) {
+        const int s = j % Cfg::NS;
+        if (*abort_flag) { dead = true; break; }
+        if (!tc::mbar_wait(&bars[BAR_VFULL + s], (j / Cfg::NS) & 1)) { dead = true; break; }
+        if (!tc::mbar_wait(&bars[BAR_PFULL + (j & 1)], (j >> 1) & 1)) { dead = true; break; }
+        tc::tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          // keys 0..63 of the tile accumulate into O0, keys 64..127 into O1
+          const uint32_t dO = tmem + (kk < 4 ? Cfg::COL_O0 : Cfg::COL_O1);
+          const uint32_t offP = (j & 1) * Cfg::P_BYTES + (kk / 4) * Cfg::BOX_BYTES + (kk % 4) * 32;
+          const uint32_t offV = kk * 2048;   // 16 key rows x 128 B
+          tc::mma_f16_ss(dO, tc::smem_desc_sw128(aP + offP, 16, 1024),
+                         tc::smem_desc_sw128(aV + s * Cfg::TILE_BYTES + offV, Cfg::BOX_BYTES, 1024), IDESC_PV,
+                         (j > 0 || (kk & 3) > 0) ? 1u : 0u);
+        }
+        tc::mma_commit(&bars[BAR_PVDONE + (j & 1)]);
+      }
+      if (dead) { atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; }
+    }
+  } else if (warp == 3) {
+    // spare warp: keeps the softmax warps aligned to the TMEM lane quarters
   } else {
     // ------------------------------ softmax / epilogue ------------------------------
+    // Two warpgroups split every key tile by columns: half 0 owns keys 0..63 of the tile, half 1
+    // keys 64..127.  Each thread keeps its own running max / sum for (row, half) and its half's
+    // products accumulate into an O accumulator of their own, so the two halves never exchange
+    // anything inside the tile loop; they are merged like two split-K partial results at the end.
+    const int half = (warp - 4) >> 2;                 // which 64 columns of every tile
     const int quarter = warp & 3;                     // TMEM lane quarter this warp may access
     const int row = quarter * 32 + lane;              // query row inside the tile
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    const uint32_t col_o = half ? Cfg::COL_O1 : Cfg::COL_O0;
     const int64_t t_row = t_first + row;
     const float kLog2e = 1.4426950408889634f;
     const float sc_s = p.tau_s[hq] * rsqrtf((float)D) * kLog2e;
@@ -208,11 +229,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         ok = false;
         KVM_WAIT(&bars[BAR_SFULL + (j & 1)], (j >> 1) & 1);
         tc::tc_fence_after();
-        float x[128];
+        float x[64];
         {
-          const uint32_t ts = tmem + lane_base + ((j & 1) ? Cfg::COL_S1 : Cfg::COL_S0);
+          const uint32_t ts = tmem + lane_base + ((j & 1) ? Cfg::COL_S1 : Cfg::COL_S0) + half * 64;
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
+          for (int c = 0; c < 2; ++c) {
             uint32_t r[32];
             tc::tmem_ld32(ts + c * 32, r);
 #pragma unroll
@@ -227,14 +248,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         int64_t nvis;   // number of visible columns of this tile for this row
         if (st) nvis = p.m - (int64_t)j * 128;
         else nvis = t_row - (p.b + (int64_t)(j - nst) * 128) + 1;
-        const int vis = (int)max((int64_t)0, min((int64_t)128, nvis));
+        const int vis = (int)max((int64_t)0, min((int64_t)64, nvis - half * 64));
         float mx = -INFINITY;
-        if (vis == 128) {
+        if (vis == 64) {
 #pragma unroll
-          for (int c = 0; c < 128; ++c) mx = fmaxf(mx, x[c]);
+          for (int c = 0; c < 64; ++c) mx = fmaxf(mx, x[c]);
         } else {
 #pragma unroll
-          for (int c = 0; c < 128; ++c) {
+          for (int c = 0; c < 64; ++c) {
             x[c] = (c < vis) ? x[c] : -INFINITY;
             mx = fmaxf(mx, x[c]);
           }
@@ -251,7 +272,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
             const float corr = (m_run == -INFINITY) ? 0.f : tc::ex2_approx(m_run - mnew);
             l_run *= corr;
             m_run = mnew;
-            const uint32_t to = tmem + lane_base + Cfg::COL_O;
+            const uint32_t to = tmem + lane_base + col_o;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
               uint32_t r[32];
@@ -270,10 +291,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
         float lsum = 0.f;
         // P row -> shared memory, K-major, 128-byte swizzle: 16-byte chunk ch of row r lives at
-        // r*128 + ((ch ^ (r & 7)) * 16) inside its 64-key box.
-        uint8_t* prow = sP + (j & 1) * Cfg::P_BYTES + row * 128;
+        // r*128 + ((ch ^ (r & 7)) * 16) inside its 64-key box; box `half` is this thread's.
+        uint8_t* prow = sP + (j & 1) * Cfg::P_BYTES + half * Cfg::BOX_BYTES + row * 128;
 #pragma unroll
-        for (int ch = 0; ch < 16; ++ch) {
+        for (int ch = 0; ch < 8; ++ch) {
           uint32_t w[4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
@@ -283,8 +304,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
             const __half2 h = __floats2half2_rn(p0, p1);
             w[i] = *reinterpret_cast<const uint32_t*>(&h);
           }
-          uint8_t* dst = prow + (ch >> 3) * Cfg::BOX_BYTES + (((ch & 7) ^ (row & 7)) << 4);
-          *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(prow + ((ch ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
         l_run += lsum;
         tc::fence_proxy_async();
@@ -294,28 +314,60 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         ok = true;
       } while (false);
     }
-    // epilogue
+    // Epilogue: merge the two halves.  out = (O0 w0 + O1 w1) / (l0 w0 + l1 w1), w_h = 2^(m_h - max(m0, m1)).
+    // Half h stores channels [h D/2, (h+1) D/2): it hands the other half its accumulator's columns
+    // of the other channel range through shared memory (column-major, one row per thread: no bank
+    // conflicts), laid over the K stages, which nothing reads any more once the last PV product is done.
+    constexpr int HD = D / 2;
+    float* xch = reinterpret_cast<float*>(sK);          // [2][HD][128]
+    float* xml = reinterpret_cast<float*>(sV);          // [2][2][128]: m and l of each half
     do {
-      if (!ok || ntiles == 0) break;
+      if (!ok) break;
+      ok = false;
       KVM_WAIT(&bars[BAR_PVDONE + ((ntiles - 1) & 1)], ((ntiles - 1) >> 1) & 1);
       tc::tc_fence_after();
-      const float inv = 1.f / l_run;
-      const uint32_t to = tmem + lane_base + Cfg::COL_O;
-      __nv_bfloat16* orow = p.out + bb * p.so0 + hq * p.so1 + (p.out_t0 + (int64_t)qt * 128 + row) * p.so2;
+      const uint32_t to = tmem + lane_base + col_o + (1 - half) * HD;
+      float* dstx = xch + half * HD * 128 + row;
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
+      for (int c = 0; c < HD / 32; ++c) {
+        uint32_t r[32];
+        tc::tmem_ld32(to + c * 32, r);
+        tc::tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) dstx[(c * 32 + i) * 128] = __uint_as_float(r[i]);
+      }
+      xml[(half * 2 + 0) * 128 + row] = m_run;
+      xml[(half * 2 + 1) * 128 + row] = l_run;
+      ok = true;
+    } while (false);
+    // every softmax thread reaches this barrier, whether or not its waits succeeded
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (ok && !*abort_flag) {
+      const float m_o = xml[((1 - half) * 2 + 0) * 128 + row];
+      const float l_o = xml[((1 - half) * 2 + 1) * 128 + row];
+      const float mm = fmaxf(m_run, m_o);
+      const float w_me = (m_run == -INFINITY) ? 0.f : tc::ex2_approx(m_run - mm);
+      const float w_ot = (m_o == -INFINITY) ? 0.f : tc::ex2_approx(m_o - mm);
+      const float inv = 1.f / (l_run * w_me + l_o * w_ot);
+      const float a_me = w_me * inv, a_ot = w_ot * inv;
+      const uint32_t to = tmem + lane_base + col_o + half * HD;
+      const float* srcx = xch + (1 - half) * HD * 128 + row;
+      __nv_bfloat16* orow = p.out + bb * p.so0 + hq * p.so1 + (p.out_t0 + (int64_t)qt * 128 + row) * p.so2 + half * HD;
+#pragma unroll
+      for (int c = 0; c < HD / 32; ++c) {
         uint32_t r[32];
         tc::tmem_ld32(to + c * 32, r);
         tc::tmem_wait_ld();
         if (row < rows_valid) {
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const __nv_bfloat162 o2 = __floats2bfloat162_rn(__uint_as_float(r[2 * i]) * inv, __uint_as_float(r[2 * i + 1]) * inv);
-            reinterpret_cast<__nv_bfloat162*>(orow + c * 32)[i] = o2;
+            const float o0 = __uint_as_float(r[2 * i]) * a_me + srcx[(c * 32 + 2 * i) * 128] * a_ot;
+            const float o1 = __uint_as_float(r[2 * i + 1]) * a_me + srcx[(c * 32 + 2 * i + 1) * 128] * a_ot;
+            reinterpret_cast<__nv_bfloat162*>(orow + c * 32)[i] = __floats2bfloat162_rn(o0, o1);
           }
         }
       }
-    } while (false);
+    }
   }
 #undef KVM_WAIT
   tc::tc_fence_before();
@@ -361,9 +413,9 @@ int launch_attn_tc(State* st, const AttnArgs& a, cudaStream_t s) {
   const CUtensorMap* tm = reinterpret_cast<const CUtensorMap*>(st->tmaps);
   const int ks = (st->nfolds & 1) ? 6 : 1, vs = (st->nfolds & 1) ? 7 : 2;   // readout copy of the current version
   if (st->d == 128) {
-    attn_tc_kernel<128><<<grid, 192, AttnTcCfg<128>::SMEM_BYTES, s>>>(tm[0], tm[ks], tm[vs], tm[3], tm[4], p);
+    attn_tc_kernel<128><<<grid, 384, AttnTcCfg<128>::SMEM_BYTES, s>>>(tm[0], tm[ks], tm[vs], tm[3], tm[4], p);
   } else {
-    attn_tc_kernel<64><<<grid, 192, AttnTcCfg<64>::SMEM_BYTES, s>>>(tm[0], tm[ks], tm[vs], tm[3], tm[4], p);
+    attn_tc_kernel<64><<<grid, 384, AttnTcCfg<64>::SMEM_BYTES, s>>>(tm[0], tm[ks], tm[vs], tm[3], tm[4], p);
   }
   return 1;
 }
