@@ -104,7 +104,7 @@ void free_all(kvm_state* ks) {
   ks->allocs.clear();
   State& s = ks->s;
   if (s.foldStream) { cudaStreamDestroy(s.foldStream); s.foldStream = nullptr; }
-  for (cudaEvent_t* e : {&s.evJoin, &s.evAttn[0], &s.evAttn[1], &s.evFold[0], &s.evFold[1]})
+  for (cudaEvent_t* e : {&s.evJoin, &s.evPre[0], &s.evPre[1], &s.evFold[0], &s.evFold[1]})
     if (*e) { cudaEventDestroy(*e); *e = nullptr; }
 }
 
@@ -254,8 +254,22 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   A(s.stK, U * (size_t)s.stRows * d); A(s.stV, U * (size_t)s.stRows * d); A(s.stG, U * (size_t)s.stRows);
   A(s.ropeCS, (size_t)s.Tcall * (d / 2));
   s.CbarRows = (s.Cmax + 127) / 128 * 128;
-  A(s.kbar64, U * Cm * d); A(s.kbarH, U * (size_t)s.CbarRows * d); A(s.kbarNorm, U * Cm);
-  A(s.kbarHat64, U * Cm * d);
+  {
+    // memory-key slots: as many blocks per batched launch as fit in 1 GiB (at least 1, at most 64,
+    // never more than a call can hold)
+    const size_t per_slot = U * Cm * d * 16 + U * (size_t)s.CbarRows * d * 2 + U * Cm * 4;
+    size_t slots = ((size_t)1 << 30) / per_slot;
+    const size_t call_blocks = (size_t)(s.Tcall / s.Cmax) + 2;
+    if (slots > call_blocks) slots = call_blocks;
+    if (slots > 64) slots = 64;
+    if (slots < 1) slots = 1;
+    s.kbSlots = (int)slots;
+  }
+  {
+    const size_t G = (size_t)s.kbSlots;
+    A(s.kbar64, G * U * Cm * d); A(s.kbarH, G * U * (size_t)s.CbarRows * d); A(s.kbarNorm, G * U * Cm);
+    A(s.kbarHat64, G * U * Cm * d);
+  }
   for (int i = 0; i < 2; ++i) {
     A(s.foldPi[i], U * Cm); A(s.foldSorted[i], U * Cm); A(s.foldCreator[i], U * Cm); A(s.foldSegNew[i], U * Cm);
     A(s.foldNMerge[i], U);
@@ -277,7 +291,7 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   if (rc == KVM_OK && !(setup_attn_tc(&s) && setup_route_tc(&s))) rc = KVM_ERR_CUDA;
   if (rc == KVM_OK) {
     bool ok = cudaStreamCreateWithFlags(&s.foldStream, cudaStreamNonBlocking) == cudaSuccess;
-    for (cudaEvent_t* e : {&s.evJoin, &s.evAttn[0], &s.evAttn[1], &s.evFold[0], &s.evFold[1]})
+    for (cudaEvent_t* e : {&s.evJoin, &s.evPre[0], &s.evPre[1], &s.evFold[0], &s.evFold[1]})
       ok = ok && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) rc = KVM_ERR_CUDA;
   }
@@ -430,9 +444,11 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
   // Two streams: attention runs on the caller's stream, folds on the state's own stream.  The fold
   // that ends block c needs the state after the fold before it and block c-w+1's keys, not block c's
   // attention, so the two overlap.  Orderings kept by events:
-  //   fold stream waits for the ingest (and with it for everything earlier on the caller's stream);
+  //   the fold stream waits for the ingest (and with it for everything earlier on the caller's stream);
   //   attention(c+1) waits for the fold that ends block c (it reads the readout copy that fold wrote);
-  //   the fold that ends block c waits for attention(c-1), which read the copy it overwrites;
+  //   before attention(c) the caller's stream brings the rows the last fold touched over to the other
+  //   readout copy (attention(c-1), the last reader of that copy, is earlier on the same stream) and
+  //   records evPre; the last kernel of the fold that ends block c, which writes that copy, waits for evPre;
   //   the caller's stream waits for the last fold before the call returns.
   // With the per-kernel timing hook on, everything stays on the caller's stream so that the
   // measured durations are those of kernels running alone.
@@ -443,8 +459,8 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
     ev_ok = ev_ok && cudaEventRecord(s.evJoin, stream) == cudaSuccess;
     ev_ok = ev_ok && cudaStreamWaitEvent(fstream, s.evJoin, 0) == cudaSuccess;
   }
-  bool attn_rec[2] = {false, false};   // evAttn[i] recorded in this call
   int fold_pending = -1;               // evFold index the next attention must wait for
+  int kb_left = 0, kb_slot = 0;        // memory-key slots computed ahead and not yet used
   for (int64_t c = c0; c <= c_last; ++c) {
     const int64_t e = (c + 1) * C;
     const int64_t qs = c * C > pos0 ? c * C : pos0;
@@ -456,24 +472,36 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
       ev_ok = ev_ok && cudaStreamWaitEvent(stream, s.evFold[fold_pending], 0) == cudaSuccess;
       fold_pending = -1;
     }
+    s.launches += launch_prev_copy(&s, stream);
+    if (overlap) ev_ok = ev_ok && cudaEventRecord(s.evPre[c & 1], stream) == cudaSuccess;
     {
       KernelTimer pt(&s, 1, stream);
       if (s.flags & KVM_FLAG_SIMT_ATTENTION) s.launches += launch_attn_simt(&s, aa, stream);
       else s.launches += launch_attn_tc(&s, aa, stream);
     }
-    if (overlap) {
-      ev_ok = ev_ok && cudaEventRecord(s.evAttn[c & 1], stream) == cudaSuccess;
-      attn_rec[c & 1] = true;
-    }
     if (qe == e && c >= s.w - 1) {
+      if (kb_left == 0) {
+        // memory keys of this and the following overflow blocks of the call, one launch
+        int64_t nf = c_last - c + 1;                   // blocks c .. c_last may end inside the call
+        if ((c_last + 1) * C > pos1) nf -= 1;          // the last one does not
+        if (nf > s.kbSlots) nf = s.kbSlots;
+        s.launches += launch_kbar(&s, s.stK + (b - ia.hist_start) * d, s.stRows * d, (int)nf, 0, fstream);
+        kb_left = (int)nf; kb_slot = 0;
+      }
       FoldArgs fa;
       fa.ok = s.stK + (b - ia.hist_start) * d; fa.ov = s.stV + (b - ia.hist_start) * d; fa.og = s.stG + (b - ia.hist_start);
       fa.unit_stride = s.stRows * d; fa.gate_stride = s.stRows;
       fa.b = b; fa.m = s.m; fa.first = (s.m == 0);
       fa.n_append = fa.first ? C : (int)n_append_of(s.growth, e, s.m, C);
-      if (overlap && attn_rec[(c - 1) & 1])
-        ev_ok = ev_ok && cudaStreamWaitEvent(fstream, s.evAttn[(c - 1) & 1], 0) == cudaSuccess;
-      s.launches += launch_fold(&s, fa, fstream);
+      fa.slot = kb_slot;
+      kb_slot += 1; kb_left -= 1;
+      // only the last kernel of the fold writes the readout copy: the routing filter and the
+      // decisions run while the caller's stream still copies the previous fold's rows
+      fa.before_apply = overlap ? s.evPre[c & 1] : nullptr;
+      {
+        const int nl = launch_fold(&s, fa, fstream);
+        if (nl < 0) ev_ok = false; else s.launches += nl;
+      }
       s.m += fa.n_append;
       s.nfolds += 1;
       if (overlap) {
@@ -517,7 +545,9 @@ KVM_API kvm_status_t kvm_decode_step(const void* q, const void* k, const void* v
     FoldArgs fa;
     fa.ok = s.ringK + slot * d; fa.ov = s.ringV + slot * d; fa.og = s.ringG + slot;
     fa.unit_stride = ringCap * d; fa.gate_stride = ringCap;
-    fa.b = b; fa.m = s.m; fa.first = (s.m == 0); fa.n_append = n_a;
+    fa.b = b; fa.m = s.m; fa.first = (s.m == 0); fa.n_append = n_a; fa.slot = 0; fa.before_apply = nullptr;
+    s.launches += launch_prev_copy(&s, stream);
+    s.launches += launch_kbar(&s, fa.ok, fa.unit_stride, 1, 0, stream);
     s.launches += launch_fold(&s, fa, stream);
     s.m += n_a;
     s.nfolds += 1;

@@ -41,51 +41,20 @@ __device__ __forceinline__ void row_stats(const double (&x)[CH], int D, double e
 // ------------------------------------------------------------------------------------------
 // 1. memory keys (one warp per overflow token)
 
-struct PrevFoldCopy {
-  int valid, all_append, n_append;
-  int64_t m, Mcap;                       // rows before the previous fold; row capacity per unit
-  const int32_t *pi, *sorted, *nmerge;   // the previous fold's decisions
-  const __half *Ksrc, *Vsrc;             // readout copy of the current version
-  __half *Kdst, *Vdst;                   // readout copy this fold writes
-};
-
 template <int D>
 __global__ void __launch_bounds__(256) kbar_kernel(const __half* __restrict__ ok, int64_t unit_stride,
                                                    const float* __restrict__ ln_w, const float* __restrict__ ln_b,
                                                    double* __restrict__ kbar64, __half* __restrict__ kbarH,
                                                    float* __restrict__ kbarNorm, double* __restrict__ kbarHat64,
-                                                   int write_hat, int C, int Cmax, int CbarRows,
-                                                   int Hkv, int r, double ln_eps, PrevFoldCopy pc) {
+                                                   int C, int Cmax, int CbarRows, int U, int Hkv, int r,
+                                                   double ln_eps) {
   constexpr int CH = D / 32;
   const int u = blockIdx.y, hk = u % Hkv;
+  const int g = blockIdx.z;   // block of the batch = slot
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int j = blockIdx.x * 8 + warp;
   if (j >= C) return;
-  // Rows that the previous fold touched are current in the source readout copy only: bring them
-  // over to the copy this fold writes (warp j takes the j-th appended row and the j-th merge target,
-  // as the apply kernel did).  The index loads are independent of one another and the rows are held
-  // in registers across the normalisation below, so their latency overlaps it.
-  uint2 cpK[2], cpV[2];
-  int64_t cpo[2] = {-1, -1};
-  if (pc.valid) {
-    const int64_t tb = (int64_t)u * Cmax;
-    if (j < pc.n_append) cpo[0] = ((int64_t)u * pc.Mcap + pc.m + j) * D;
-    if (!pc.all_append) {
-      const int nm = pc.nmerge[u];
-      int s0 = pc.sorted[tb + j], s1 = pc.sorted[tb + (j > 0 ? j - 1 : 0)];
-      s0 = (unsigned)s0 < (unsigned)Cmax ? s0 : 0;   // entries past nmerge are not defined
-      s1 = (unsigned)s1 < (unsigned)Cmax ? s1 : 0;
-      const int r1 = pc.pi[tb + s0], r0 = pc.pi[tb + s1];
-      if (j < nm && r1 >= 0 && r1 < pc.m && (j == 0 || r0 != r1)) cpo[1] = ((int64_t)u * pc.Mcap + r1) * D;
-    }
-#pragma unroll
-    for (int t = 0; t < 2; ++t)
-      if (cpo[t] >= 0 && lane < D / 4) {   // 8 bytes per lane
-        cpK[t] = reinterpret_cast<const uint2*>(pc.Ksrc + cpo[t])[lane];
-        cpV[t] = reinterpret_cast<const uint2*>(pc.Vsrc + cpo[t])[lane];
-      }
-  }
-  const __half* row = ok + (int64_t)u * unit_stride + (int64_t)j * D;
+  const __half* row = ok + (int64_t)u * unit_stride + ((int64_t)g * C + j) * D;
   double val[CH];
 #pragma unroll
   for (int i = 0; i < CH; ++i) {
@@ -96,8 +65,8 @@ __global__ void __launch_bounds__(256) kbar_kernel(const __half* __restrict__ ok
   row_stats<CH>(val, D, ln_eps, mean, rstd);
   double kb[CH];
   double n2 = 0.0;
-  const int64_t o = ((int64_t)u * Cmax + j) * D;
-  const int64_t oh = ((int64_t)u * CbarRows + j) * D;
+  const int64_t o = (((int64_t)g * U + u) * Cmax + j) * D;
+  const int64_t oh = (((int64_t)g * U + u) * CbarRows + j) * D;
 #pragma unroll
   for (int i = 0; i < CH; ++i) {
     const int x = lane + 32 * i;
@@ -110,14 +79,48 @@ __global__ void __launch_bounds__(256) kbar_kernel(const __half* __restrict__ ok
   // LN_s applied to kbar itself: the readout key of the row that this token would create
   double mu2, rs2;
   row_stats<CH>(kb, D, ln_eps, mu2, rs2);
-  if (write_hat) {   // only folds that append rows need the would-be row keys
 #pragma unroll
-    for (int i = 0; i < CH; ++i) {
-      const int x = lane + 32 * i;
-      kbarHat64[o + x] = (double)ln_w[hk * D + x] * ((kb[i] - mu2) * rs2) + (double)ln_b[hk * D + x];
-    }
+  for (int i = 0; i < CH; ++i) {
+    const int x = lane + 32 * i;
+    kbarHat64[o + x] = (double)ln_w[hk * D + x] * ((kb[i] - mu2) * rs2) + (double)ln_b[hk * D + x];
   }
-  if (lane == 0) kbarNorm[(int64_t)u * Cmax + j] = (float)sqrt(n2) * 1.000001f;
+  if (lane == 0) kbarNorm[((int64_t)g * U + u) * Cmax + j] = (float)sqrt(n2) * 1.000001f;
+}
+
+// Rows that the last fold touched are current in one readout copy only: bring them over to the
+// other one (warp j takes the j-th appended row and the j-th merge target, as the apply kernel did).
+struct PrevFoldCopy {
+  int all_append, n_append, C, Cmax;
+  int64_t m, Mcap;                       // rows before that fold; row capacity per unit
+  const int32_t *pi, *sorted, *nmerge;   // that fold's decisions
+  const __half *Ksrc, *Vsrc;
+  __half *Kdst, *Vdst;
+};
+
+template <int D>
+__global__ void __launch_bounds__(256) prev_copy_kernel(PrevFoldCopy pc) {
+  const int u = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int j = blockIdx.x * 8 + warp;
+  if (j >= pc.C) return;
+  const int64_t tb = (int64_t)u * pc.Cmax;
+  int64_t cpo[2] = {-1, -1};
+  if (j < pc.n_append) cpo[0] = ((int64_t)u * pc.Mcap + pc.m + j) * D;
+  if (!pc.all_append) {
+    const int nm = pc.nmerge[u];
+    int s0 = pc.sorted[tb + j], s1 = pc.sorted[tb + (j > 0 ? j - 1 : 0)];
+    s0 = (unsigned)s0 < (unsigned)pc.Cmax ? s0 : 0;   // entries past nmerge are not defined
+    s1 = (unsigned)s1 < (unsigned)pc.Cmax ? s1 : 0;
+    const int r1 = pc.pi[tb + s0], r0 = pc.pi[tb + s1];
+    if (j < nm && r1 >= 0 && r1 < pc.m && (j == 0 || r0 != r1)) cpo[1] = ((int64_t)u * pc.Mcap + r1) * D;
+  }
+  uint2 cpK[2], cpV[2];
+#pragma unroll
+  for (int t = 0; t < 2; ++t)
+    if (cpo[t] >= 0 && lane < D / 4) {   // 8 bytes per lane
+      cpK[t] = reinterpret_cast<const uint2*>(pc.Ksrc + cpo[t])[lane];
+      cpV[t] = reinterpret_cast<const uint2*>(pc.Vsrc + cpo[t])[lane];
+    }
 #pragma unroll
   for (int t = 0; t < 2; ++t)
     if (cpo[t] >= 0 && lane < D / 4) {
@@ -639,32 +642,53 @@ __global__ void __launch_bounds__(256) fold_apply_kernel(FoldApplyParams p) {
   }
 }
 
-int launch_route_filter_tc(State* st, int64_t m, int nsplit, cudaStream_t s);
+int launch_route_filter_tc(State* st, int64_t m, int nsplit, int slot, cudaStream_t s);
+
+int launch_kbar(State* st, const __half* ok, int64_t unit_stride, int nblk, int slot0, cudaStream_t s) {
+  KernelTimer kt(st, 2, s);
+  const int C = st->C, D = st->d;
+  const int64_t U = st->U;
+  dim3 grid((C + 7) / 8, st->U, nblk);
+  double* k64 = st->kbar64 + (int64_t)slot0 * U * st->Cmax * D;
+  __half* kh = st->kbarH + (int64_t)slot0 * U * st->CbarRows * D;
+  float* kn = st->kbarNorm + (int64_t)slot0 * U * st->Cmax;
+  double* khat = st->kbarHat64 + (int64_t)slot0 * U * st->Cmax * D;
+  if (D == 128)
+    kbar_kernel<128><<<grid, 256, 0, s>>>(ok, unit_stride, st->ln_w, st->ln_b, k64, kh, kn, khat, C, st->Cmax,
+                                          st->CbarRows, st->U, st->Hkv, st->r, (double)st->ln_eps);
+  else
+    kbar_kernel<64><<<grid, 256, 0, s>>>(ok, unit_stride, st->ln_w, st->ln_b, k64, kh, kn, khat, C, st->Cmax,
+                                         st->CbarRows, st->U, st->Hkv, st->r, (double)st->ln_eps);
+  return 1;
+}
+
+int launch_prev_copy(State* st, cudaStream_t s) {
+  if (!st->prevValid) return 0;
+  st->prevValid = false;
+  // the last fold (number nfolds) wrote copy nfolds & 1; the other copy lacks the rows it touched
+  const int src = (int)(st->nfolds & 1), dst = src ^ 1;
+  PrevFoldCopy pc;
+  pc.all_append = st->prevAllAppend ? 1 : 0; pc.n_append = st->prevNAppend; pc.C = st->C; pc.Cmax = st->Cmax;
+  pc.m = st->prevM; pc.Mcap = st->Mcap;
+  pc.pi = st->foldPi[src]; pc.sorted = st->foldSorted[src]; pc.nmerge = st->foldNMerge[src];
+  pc.Ksrc = st->KhatBuf[src]; pc.Vsrc = st->VhatBuf[src]; pc.Kdst = st->KhatBuf[dst]; pc.Vdst = st->VhatBuf[dst];
+  KernelTimer kt(st, 2, s);
+  dim3 grid((st->C + 7) / 8, st->U);
+  if (st->d == 128) prev_copy_kernel<128><<<grid, 256, 0, s>>>(pc);
+  else prev_copy_kernel<64><<<grid, 256, 0, s>>>(pc);
+  return 1;
+}
 
 int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
   int launches = 0;
   const int C = st->C, D = st->d;
   // the state after nfolds folds is read from readout copy `src`; this fold writes copy `dst`
   const int src = (int)(st->nfolds & 1), dst = src ^ 1;
-  {
-    KernelTimer kt(st, 2, s);
-    const int write_hat = (!a.first && a.n_append > 0 && a.n_append < C) ? 1 : 0;
-    PrevFoldCopy pc;
-    pc.valid = st->prevValid ? 1 : 0; pc.all_append = st->prevAllAppend ? 1 : 0; pc.n_append = st->prevNAppend;
-    pc.m = st->prevM; pc.Mcap = st->Mcap;
-    pc.pi = st->foldPi[src]; pc.sorted = st->foldSorted[src]; pc.nmerge = st->foldNMerge[src];
-    pc.Ksrc = st->KhatBuf[src]; pc.Vsrc = st->VhatBuf[src]; pc.Kdst = st->KhatBuf[dst]; pc.Vdst = st->VhatBuf[dst];
-    dim3 grid((C + 7) / 8, st->U);
-    if (D == 128)
-      kbar_kernel<128><<<grid, 256, 0, s>>>(a.ok, a.unit_stride, st->ln_w, st->ln_b, st->kbar64, st->kbarH,
-                                            st->kbarNorm, st->kbarHat64, write_hat, C, st->Cmax, st->CbarRows,
-                                            st->Hkv, st->r, (double)st->ln_eps, pc);
-    else
-      kbar_kernel<64><<<grid, 256, 0, s>>>(a.ok, a.unit_stride, st->ln_w, st->ln_b, st->kbar64, st->kbarH,
-                                           st->kbarNorm, st->kbarHat64, write_hat, C, st->Cmax, st->CbarRows,
-                                           st->Hkv, st->r, (double)st->ln_eps, pc);
-    ++launches;
-  }
+  const int64_t U = st->U;
+  const double* kbar64 = st->kbar64 + (int64_t)a.slot * U * st->Cmax * D;
+  const __half* kbarH = st->kbarH + (int64_t)a.slot * U * st->CbarRows * D;
+  const float* kbarNorm = st->kbarNorm + (int64_t)a.slot * U * st->Cmax;
+  const double* kbarHat64 = st->kbarHat64 + (int64_t)a.slot * U * st->Cmax * D;
   const bool all_append = a.first || a.n_append >= C;
   if (!all_append) {
     // enough CTAs to fill the GPU, at least 256 rows per split
@@ -677,20 +701,20 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
       KernelTimer kt(st, 3, s);
       dim3 grid(nsplit, st->U);
       if (D == 128)
-        route_filter_simt_kernel<128><<<grid, 256, 0, s>>>(st->kbarH, st->KhatBuf[src], st->candV, st->candI, C, st->Cmax,
-                                                           st->CbarRows, st->Mcap, a.m, nsplit, st->kbarNorm,
+        route_filter_simt_kernel<128><<<grid, 256, 0, s>>>(kbarH, st->KhatBuf[src], st->candV, st->candI, C, st->Cmax,
+                                                           st->CbarRows, st->Mcap, a.m, nsplit, kbarNorm,
                                                            route_thr_coeff(st), st->S);
       else
-        route_filter_simt_kernel<64><<<grid, 256, 0, s>>>(st->kbarH, st->KhatBuf[src], st->candV, st->candI, C, st->Cmax,
-                                                          st->CbarRows, st->Mcap, a.m, nsplit, st->kbarNorm,
+        route_filter_simt_kernel<64><<<grid, 256, 0, s>>>(kbarH, st->KhatBuf[src], st->candV, st->candI, C, st->Cmax,
+                                                          st->CbarRows, st->Mcap, a.m, nsplit, kbarNorm,
                                                           route_thr_coeff(st), st->S);
       ++launches;
     } else {
       KernelTimer kt(st, 3, s);
-      launches += launch_route_filter_tc(st, a.m, nsplit, s);
+      launches += launch_route_filter_tc(st, a.m, nsplit, a.slot, s);
     }
     FoldDecideParams p;
-    p.kbar64 = st->kbar64; p.kbarNorm = st->kbarNorm; p.kbarHat64 = st->kbarHat64;
+    p.kbar64 = kbar64; p.kbarNorm = kbarNorm; p.kbarHat64 = kbarHat64;
     p.candV = st->candV; p.candI = st->candI; p.ln_w = st->ln_w; p.ln_b = st->ln_b;
     p.sumK = st->sumK; p.kmu = st->kmu; p.krstd = st->krstd;
     p.pi = st->foldPi[dst]; p.sorted = st->foldSorted[dst]; p.creator = st->foldCreator[dst];
@@ -706,7 +730,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
   }
   FoldApplyParams q;
   q.ov = a.ov; q.og = a.og; q.unit_stride = a.unit_stride; q.gate_stride = a.gate_stride;
-  q.kbar64 = st->kbar64; q.ln_w = st->ln_w; q.ln_b = st->ln_b;
+  q.kbar64 = kbar64; q.ln_w = st->ln_w; q.ln_b = st->ln_b;
   q.pi = st->foldPi[dst]; q.sorted = st->foldSorted[dst]; q.creator = st->foldCreator[dst];
   q.segnew = st->foldSegNew[dst]; q.nmerge = st->foldNMerge[dst];
   q.sumK = st->sumK; q.sumV = st->sumV; q.rho = st->rho; q.wsum = st->wsum; q.cnt = st->cnt;
@@ -716,6 +740,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
   q.C = C; q.Cmax = st->Cmax; q.Hkv = st->Hkv; q.n_append = a.n_append; q.all_append = all_append ? 1 : 0;
   q.radius_on = (st->flags & KVM_FLAG_NO_RADIUS) ? 0 : 1;
   q.ln_eps = (double)st->ln_eps; q.norm_eps = (double)st->norm_eps;
+  if (a.before_apply && cudaStreamWaitEvent(s, a.before_apply, 0) != cudaSuccess) return -1000000;
   KernelTimer kt(st, 5, s);
   dim3 grid((C + 7) / 8, st->U);
   if (D == 128) fold_apply_kernel<128><<<grid, 256, 0, s>>>(q);

@@ -49,13 +49,14 @@ struct State {
   // decode and the routing filter.  Two copies: the state after f folds is read from copy f & 1, so
   // fold f+1 can write copy (f+1) & 1 while the attention of the current block still reads copy f & 1.
   __half *KhatBuf[2], *VhatBuf[2];
-  // what the previous fold touched (host): its rows are copied into the other copy by the next fold
+  // what the previous fold touched (host): its rows are copied into the other copy (launch_prev_copy)
+  // before the next fold writes there; prevValid = such a copy is still owed
   bool prevValid, prevAllAppend;
   int64_t prevM;
   int prevNAppend;
   // second stream and events that let a block's attention and the fold of the block before it overlap
   cudaStream_t foldStream;
-  cudaEvent_t evJoin, evAttn[2], evFold[2];
+  cudaEvent_t evJoin, evPre[2], evFold[2];
   // ---- window ring (device): slot = t mod ringLen ----
   __half *ringK, *ringV;         // [U, w*Cmax, d]  rotated keys / values (fp16)
   float* ringG;                  // [U, w*Cmax]
@@ -65,12 +66,15 @@ struct State {
   __half *stK, *stV;             // [U, stRows, d]   history + new tokens (rotated keys, fp16)
   float* stG;                    // [U, stRows]
   float2* ropeCS;                // [Tcall, r/2] (cos, sin)
-  // ---- fold scratch (device) ----
-  double* kbar64;                // [U, Cmax, d]
-  __half* kbarH;                 // [U, CbarRows, d]
-  float* kbarNorm;               // [U, Cmax]
+  // ---- fold scratch (device).  The memory keys depend on the block's own keys only, so a prefill
+  //      call computes them for up to kbSlots consecutive overflow blocks in one launch; slot g holds
+  //      one block's arrays in the layouts below ----
+  int kbSlots;
+  double* kbar64;                // [kbSlots][U, Cmax, d]
+  __half* kbarH;                 // [kbSlots][U, CbarRows, d]
+  float* kbarNorm;               // [kbSlots][U, Cmax]
   int CbarRows;                  // rows per unit of kbarH (Cmax rounded up to the 128-row MMA tile)
-  double* kbarHat64;             // [U, Cmax, d]  LN_s(kbar_j): the readout key of a row created by token j
+  double* kbarHat64;             // [kbSlots][U, Cmax, d]  LN_s(kbar_j): the readout key of a row created by token j
   // decisions of the fold being computed ([(nfolds+1) & 1]) and of the one before ([nfolds & 1])
   int32_t *foldPi[2], *foldSorted[2], *foldCreator[2], *foldSegNew[2], *foldNMerge[2];
   int nsplitRoute;               // splits the routing filter may use
@@ -138,8 +142,17 @@ struct FoldArgs {
   int64_t m;        // rows before the fold
   int n_append;     // rows to append (== C on the first fold)
   bool first;       // first state-creation step
+  int slot;         // memory-key slot that holds this block's keys (launch_kbar)
+  cudaEvent_t before_apply;   // if set, the stream waits for it before the kernel that writes the readout copy
 };
 int launch_fold(State* st, const FoldArgs& a, cudaStream_t s);
+// Memory keys of nblk consecutive blocks (C rows each, starting at ok within every unit) into slots
+// slot0 .. slot0 + nblk - 1.
+int launch_kbar(State* st, const __half* ok, int64_t unit_stride, int nblk, int slot0, cudaStream_t s);
+// Copies the readout rows that the last fold touched from the current readout copy into the other
+// one (no-op when nothing is owed).  Must run after every reader of the other copy has finished and
+// before the next fold writes it.
+int launch_prev_copy(State* st, cudaStream_t s);
 
 struct DecodeArgs {
   const __nv_bfloat16 *q, *k, *v;

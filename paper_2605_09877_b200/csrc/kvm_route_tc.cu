@@ -27,6 +27,7 @@ struct RouteTcParams {
   int32_t* candI;
   int32_t* status;
   const float* kbarNorm;   // [U, Cmax] upper bound of ||kbar_j||
+  int a_unit0;             // first unit of this block's slot in the memory-key tensor map
   float thr_coeff;         // candidate window = thr_coeff * ||kbar_j|| + 1e-5
   int64_t m;
   int C, Cmax, nsplit, S;
@@ -98,7 +99,7 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
       tc::mbar_expect_tx(&bars[RB_AFULL], mt_used * Cfg::TILE_BYTES);
       for (int mt = 0; mt < mt_used; ++mt)
         for (int kb = 0; kb < Cfg::NKB; ++kb)
-          tc::tma_load_3d(sA + mt * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, &mapA, &bars[RB_AFULL], kb * 64, mt * 128, u);
+          tc::tma_load_3d(sA + mt * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, &mapA, &bars[RB_AFULL], kb * 64, mt * 128, p.a_unit0 + u);
       for (int j = 0; j < nsteps; ++j) {
         const int s = j % Cfg::NS;
         const int jt = j >= ntiles ? j - ntiles : j;
@@ -228,11 +229,12 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
   }
 }
 
-int launch_route_filter_tc(State* st, int64_t m, int nsplit, cudaStream_t s) {
+int launch_route_filter_tc(State* st, int64_t m, int nsplit, int slot, cudaStream_t s) {
   RouteTcParams p;
   p.candV = st->candV; p.candI = st->candI; p.status = st->status; p.m = m;
   p.C = st->C; p.Cmax = st->Cmax; p.nsplit = nsplit; p.S = st->S;
-  p.kbarNorm = st->kbarNorm; p.thr_coeff = route_thr_coeff(st);
+  p.kbarNorm = st->kbarNorm + (int64_t)slot * st->U * st->Cmax; p.thr_coeff = route_thr_coeff(st);
+  p.a_unit0 = slot * st->U;
   const CUtensorMap* tm = reinterpret_cast<const CUtensorMap*>(st->tmaps);
   dim3 grid(nsplit, st->U);
   const int ks = (st->nfolds & 1) ? 6 : 1;   // the fold reads the readout copy of the current version
@@ -243,7 +245,7 @@ int launch_route_filter_tc(State* st, int64_t m, int nsplit, cudaStream_t s) {
 
 bool setup_route_tc(State* st) {
   CUtensorMap* tm = reinterpret_cast<CUtensorMap*>(st->tmaps);
-  if (!encode_tmap_rows(&tm[5], st->kbarH, st->d, st->CbarRows, st->U, 128)) return false;
+  if (!encode_tmap_rows(&tm[5], st->kbarH, st->d, st->CbarRows, (int64_t)st->kbSlots * st->U, 128)) return false;
   if (cudaFuncSetAttribute(route_filter_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, RouteTcCfg<128>::SMEM_BYTES) != cudaSuccess) return false;
   if (cudaFuncSetAttribute(route_filter_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, RouteTcCfg<64>::SMEM_BYTES) != cudaSuccess) return false;
   return true;
