@@ -104,7 +104,8 @@ void free_all(kvm_state* ks) {
   ks->allocs.clear();
   State& s = ks->s;
   if (s.foldStream) { cudaStreamDestroy(s.foldStream); s.foldStream = nullptr; }
-  for (cudaEvent_t* e : {&s.evJoin, &s.evPre[0], &s.evPre[1], &s.evFold[0], &s.evFold[1]})
+  if (s.kbStream) { cudaStreamDestroy(s.kbStream); s.kbStream = nullptr; }
+  for (cudaEvent_t* e : {&s.evJoin, &s.evPre[0], &s.evPre[1], &s.evFold[0], &s.evFold[1], &s.evKb[0], &s.evKb[1], &s.evBatchDone[0], &s.evBatchDone[1]})
     if (*e) { cudaEventDestroy(*e); *e = nullptr; }
 }
 
@@ -255,10 +256,10 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   A(s.ropeCS, (size_t)s.Tcall * (d / 2));
   s.CbarRows = (s.Cmax + 127) / 128 * 128;
   {
-    // memory-key slots: as many blocks per batched launch as fit in 1 GiB (at least 1, at most 64,
+    // memory-key slots: as many blocks per batched launch as fit in 2 GiB (at least 1, at most 64,
     // never more than a call can hold)
-    const size_t per_slot = U * Cm * d * 16 + U * (size_t)s.CbarRows * d * 2 + U * Cm * 4;
-    size_t slots = ((size_t)1 << 30) / per_slot;
+    const size_t per_slot = U * Cm * d * 16 + U * (size_t)s.CbarRows * d * 4 + U * Cm * 4 + U * Cm * Cm * 4;
+    size_t slots = ((size_t)2 << 30) / per_slot;
     const size_t call_blocks = (size_t)(s.Tcall / s.Cmax) + 2;
     if (slots > call_blocks) slots = call_blocks;
     if (slots > 64) slots = 64;
@@ -268,7 +269,8 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   {
     const size_t G = (size_t)s.kbSlots;
     A(s.kbar64, G * U * Cm * d); A(s.kbarH, G * U * (size_t)s.CbarRows * d); A(s.kbarNorm, G * U * Cm);
-    A(s.kbarHat64, G * U * Cm * d);
+    A(s.kbarHat64, G * U * Cm * d); A(s.kbarHatH, G * U * (size_t)s.CbarRows * d);
+    A(s.gramT, G * U * Cm * Cm);
   }
   for (int i = 0; i < 2; ++i) {
     A(s.foldPi[i], U * Cm); A(s.foldSorted[i], U * Cm); A(s.foldCreator[i], U * Cm); A(s.foldSegNew[i], U * Cm);
@@ -291,7 +293,8 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   if (rc == KVM_OK && !(setup_attn_tc(&s) && setup_route_tc(&s))) rc = KVM_ERR_CUDA;
   if (rc == KVM_OK) {
     bool ok = cudaStreamCreateWithFlags(&s.foldStream, cudaStreamNonBlocking) == cudaSuccess;
-    for (cudaEvent_t* e : {&s.evJoin, &s.evPre[0], &s.evPre[1], &s.evFold[0], &s.evFold[1]})
+    ok = ok && cudaStreamCreateWithFlags(&s.kbStream, cudaStreamNonBlocking) == cudaSuccess;
+    for (cudaEvent_t* e : {&s.evJoin, &s.evPre[0], &s.evPre[1], &s.evFold[0], &s.evFold[1], &s.evKb[0], &s.evKb[1], &s.evBatchDone[0], &s.evBatchDone[1]})
       ok = ok && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
     if (!ok) rc = KVM_ERR_CUDA;
   }
@@ -460,7 +463,46 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
     ev_ok = ev_ok && cudaStreamWaitEvent(fstream, s.evJoin, 0) == cudaSuccess;
   }
   int fold_pending = -1;               // evFold index the next attention must wait for
-  int kb_left = 0, kb_slot = 0;        // memory-key slots computed ahead and not yet used
+  // The folds of this call, planned ahead from the budget rule: fold i ends block cf0 + i, folds the
+  // block that starts at bf0 + i*C and appends fold_na[i] rows.  Their memory keys (and new-row
+  // filters) need the ingested keys only, so they are computed in batches on a third stream, one
+  // batch ahead of the folds; a batch fills one half of the slots.
+  std::vector<int> fold_na;
+  int64_t cf0 = -1;
+  int n_done_folds = 0;                // folds of this call launched so far
+  {
+    int64_t m_sim = s.m;
+    for (int64_t c = c0; c <= c_last; ++c) {
+      const int64_t e = (c + 1) * C;
+      if (e > pos1 || c < s.w - 1) continue;
+      if (cf0 < 0) cf0 = c;
+      const int64_t na = m_sim == 0 ? C : n_append_of(s.growth, e, m_sim, C);
+      fold_na.push_back((int)na);
+      m_sim += na;
+    }
+  }
+  const int n_call_folds = (int)fold_na.size();
+  const int halves = s.kbSlots >= 2 ? 2 : 1;
+  const int per_batch = s.kbSlots >= 2 ? s.kbSlots / 2 : 1;
+  cudaStream_t kstream = overlap ? s.kbStream : stream;
+  if (overlap && n_call_folds > 0) ev_ok = ev_ok && cudaStreamWaitEvent(kstream, s.evJoin, 0) == cudaSuccess;
+  bool batch_done_rec[2] = {false, false};
+  auto launch_batch = [&](int k) {      // batch k = folds [k*per_batch, ...) into slot half k % halves
+    const int f0 = k * per_batch;
+    if (f0 >= n_call_folds) return;
+    const int nf = n_call_folds - f0 < per_batch ? n_call_folds - f0 : per_batch;
+    const int h = k % halves;
+    bool want_gram = false;              // does a fold of the batch append some, not all, of its tokens?
+    int64_t m_sim = s.m;
+    for (int i = 0; i < f0 + nf; ++i) {
+      // (m_sim restarts from the current rows: folds before f0 that are already launched moved s.m)
+      if (i >= n_done_folds) { if (i >= f0 && fold_na[i] > 0 && fold_na[i] < C && m_sim > 0) want_gram = true; m_sim += fold_na[i]; }
+    }
+    if (overlap && batch_done_rec[h]) ev_ok = ev_ok && cudaStreamWaitEvent(kstream, s.evBatchDone[h], 0) == cudaSuccess;
+    const int64_t bf = (cf0 + f0 + 1) * C - L;   // first token of the first block of the batch
+    s.launches += launch_kbar(&s, s.stK + (bf - ia.hist_start) * d, s.stRows * d, nf, h * per_batch, want_gram, kstream);
+    if (overlap) ev_ok = ev_ok && cudaEventRecord(s.evKb[h], kstream) == cudaSuccess;
+  };
   for (int64_t c = c0; c <= c_last; ++c) {
     const int64_t e = (c + 1) * C;
     const int64_t qs = c * C > pos0 ? c * C : pos0;
@@ -480,21 +522,20 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
       else s.launches += launch_attn_tc(&s, aa, stream);
     }
     if (qe == e && c >= s.w - 1) {
-      if (kb_left == 0) {
-        // memory keys of this and the following overflow blocks of the call, one launch
-        int64_t nf = c_last - c + 1;                   // blocks c .. c_last may end inside the call
-        if ((c_last + 1) * C > pos1) nf -= 1;          // the last one does not
-        if (nf > s.kbSlots) nf = s.kbSlots;
-        s.launches += launch_kbar(&s, s.stK + (b - ia.hist_start) * d, s.stRows * d, (int)nf, 0, fstream);
-        kb_left = (int)nf; kb_slot = 0;
+      const int fi = n_done_folds, bk = fi / per_batch;
+      if (fi % per_batch == 0) {
+        if (!overlap || fi == 0) launch_batch(bk);        // (with one stream: just in time)
+        if (overlap) {
+          launch_batch(bk + 1);                            // one batch ahead
+          ev_ok = ev_ok && cudaStreamWaitEvent(fstream, s.evKb[bk % halves], 0) == cudaSuccess;
+        }
       }
       FoldArgs fa;
       fa.ok = s.stK + (b - ia.hist_start) * d; fa.ov = s.stV + (b - ia.hist_start) * d; fa.og = s.stG + (b - ia.hist_start);
       fa.unit_stride = s.stRows * d; fa.gate_stride = s.stRows;
       fa.b = b; fa.m = s.m; fa.first = (s.m == 0);
       fa.n_append = fa.first ? C : (int)n_append_of(s.growth, e, s.m, C);
-      fa.slot = kb_slot;
-      kb_slot += 1; kb_left -= 1;
+      fa.slot = (bk % halves) * per_batch + fi % per_batch;
       // only the last kernel of the fold writes the readout copy: the routing filter and the
       // decisions run while the caller's stream still copies the previous fold's rows
       fa.before_apply = overlap ? s.evPre[c & 1] : nullptr;
@@ -504,6 +545,11 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
       }
       s.m += fa.n_append;
       s.nfolds += 1;
+      n_done_folds += 1;
+      if (overlap && (n_done_folds % per_batch == 0 || n_done_folds == n_call_folds)) {
+        ev_ok = ev_ok && cudaEventRecord(s.evBatchDone[bk % halves], fstream) == cudaSuccess;
+        batch_done_rec[bk % halves] = true;
+      }
       if (overlap) {
         fold_pending = (int)(s.nfolds & 1);
         ev_ok = ev_ok && cudaEventRecord(s.evFold[fold_pending], fstream) == cudaSuccess;
@@ -547,7 +593,7 @@ KVM_API kvm_status_t kvm_decode_step(const void* q, const void* k, const void* v
     fa.unit_stride = ringCap * d; fa.gate_stride = ringCap;
     fa.b = b; fa.m = s.m; fa.first = (s.m == 0); fa.n_append = n_a; fa.slot = 0; fa.before_apply = nullptr;
     s.launches += launch_prev_copy(&s, stream);
-    s.launches += launch_kbar(&s, fa.ok, fa.unit_stride, 1, 0, stream);
+    s.launches += launch_kbar(&s, fa.ok, fa.unit_stride, 1, 0, n_a > 0 && n_a < C && s.m > 0, stream);
     s.launches += launch_fold(&s, fa, stream);
     s.m += n_a;
     s.nfolds += 1;

@@ -46,7 +46,7 @@ __global__ void __launch_bounds__(256) kbar_kernel(const __half* __restrict__ ok
                                                    const float* __restrict__ ln_w, const float* __restrict__ ln_b,
                                                    double* __restrict__ kbar64, __half* __restrict__ kbarH,
                                                    float* __restrict__ kbarNorm, double* __restrict__ kbarHat64,
-                                                   int C, int Cmax, int CbarRows, int U, int Hkv, int r,
+                                                   __half* __restrict__ kbarHatH, int C, int Cmax, int CbarRows, int U, int Hkv, int r,
                                                    double ln_eps) {
   constexpr int CH = D / 32;
   const int u = blockIdx.y, hk = u % Hkv;
@@ -82,7 +82,9 @@ __global__ void __launch_bounds__(256) kbar_kernel(const __half* __restrict__ ok
 #pragma unroll
   for (int i = 0; i < CH; ++i) {
     const int x = lane + 32 * i;
-    kbarHat64[o + x] = (double)ln_w[hk * D + x] * ((kb[i] - mu2) * rs2) + (double)ln_b[hk * D + x];
+    const double hat = (double)ln_w[hk * D + x] * ((kb[i] - mu2) * rs2) + (double)ln_b[hk * D + x];
+    kbarHat64[o + x] = hat;
+    kbarHatH[oh + x] = __float2half_rn((float)hat);
   }
   if (lane == 0) kbarNorm[((int64_t)g * U + u) * Cmax + j] = (float)sqrt(n2) * 1.000001f;
 }
@@ -221,6 +223,7 @@ struct FoldDecideParams {
   const double* kbar64;
   const float* kbarNorm;
   const double* kbarHat64;   // LN_s(kbar_j): keys of the rows the block's tokens would create
+  const float* gramT;        // [U, Cmax, Cmax] approximate kbarHat_a . kbar_j at [a][j] (fp16 operands)
   const float* candV;
   const int32_t* candI;
   const float *ln_w, *ln_b;
@@ -238,6 +241,7 @@ constexpr int kPairPerTok = 24;
 
 constexpr int kDecideThreads = 512;
 constexpr int kDecideWarps = kDecideThreads / 32;
+static_assert(kDecideThreads >= 2 * kMaxBlock, "the ranking loops give every token at least two threads");
 
 // The candidate rows (kTopK entries, -1 = none) of one token in one split: two 16-byte loads.
 __device__ __forceinline__ void load_cand_rows(const int32_t* candI, int64_t o, int (&i)[kTopK]) {
@@ -282,13 +286,14 @@ __global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideP
   __shared__ int s_prow[kPairCap];
   __shared__ unsigned short s_ptok[kPairCap];
   __shared__ double s_pval[kPairCap];
-  __shared__ int s_np, s_nmerge;
+  __shared__ int s_np, s_nmerge, s_nexh;
 
   const int u = blockIdx.x, hk = u % p.Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int C = p.C;
   const int64_t m = p.m;
   const int n_a = p.n_append;
+  const int parts = C <= 64 ? 8 : (C <= 128 ? 4 : 2);   // adjacent threads that share a token in the ranking loops
   const double* kbarU = p.kbar64 + (int64_t)u * p.Cmax * D;
   const int64_t rowBase = (int64_t)u * p.Mcap;
   const int64_t tokBase = (int64_t)u * p.Cmax;
@@ -299,7 +304,7 @@ __global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideP
     gam[i] = (double)p.ln_w[hk * D + lane + 32 * i];
     bet[i] = (double)p.ln_b[hk * D + lane + 32 * i];
   }
-  if (tid == 0) { s_np = 0; s_nmerge = 0; }
+  if (tid == 0) { s_np = 0; s_nmerge = 0; s_nexh = 0; }
   if (tid < kMaxBlock) {
     s_app[tid] = 0; s_exh[tid] = 0; s_pcnt[tid] = 0; s_pstart[tid] = 0; s_pi[tid] = -1;
     s_best[tid] = -INFINITY; s_barg[tid] = -1; s_score[tid] = -INFINITY; s_creator[tid] = -1;
@@ -357,14 +362,16 @@ __global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideP
       s_pcnt[j] = cntc;
     }
     s_exh[j] = exh ? 1 : 0;
+    if (exh) atomicAdd(&s_nexh, 1);
   }
   __syncthreads();
-  // ---- A3: exact fp64 similarity of every candidate pair, one warp per pair, four in flight ----
+  // ---- A3: exact fp64 similarity of every candidate pair, one warp per pair, eight in flight
+  //      (the loads of a pair hang on one another: pair list -> rows -> statistics) ----
   const int np = min(s_np, kPairCap);
-  for (int q0 = warp; q0 < np; q0 += 4 * kDecideWarps) {
-    double part[4];
+  for (int q0 = warp; q0 < np; q0 += 8 * kDecideWarps) {
+    double part[8];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
+    for (int k = 0; k < 8; ++k) {
       const int q = min(q0 + k * kDecideWarps, np - 1);   // clamped duplicates are computed and dropped
       const int j = s_ptok[q], i = s_prow[q];
       const double* kb = kbarU + (int64_t)j * D;
@@ -375,10 +382,12 @@ __global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideP
       for (int c = 0; c < CH; ++c) acc += kb[lane + 32 * c] * (gam[c] * ((sk[lane + 32 * c] - mu) * rs) + bet[c]);
       part[k] = acc;
     }
-    const double z = warp_reduce4(part[0], part[1], part[2], part[3], lane);
-    if ((lane & 7) == 0) {   // lanes 0, 8, 16, 24 hold pairs 0, 1, 2, 3
-      const int q = q0 + (lane >> 3) * kDecideWarps;
-      if (q < np) s_pval[q] = z;
+    const double z0 = warp_reduce4(part[0], part[1], part[2], part[3], lane);
+    const double z1 = warp_reduce4(part[4], part[5], part[6], part[7], lane);
+    if ((lane & 7) == 0) {   // lanes 0, 8, 16, 24 hold pairs 0..3 of z0 and 4..7 of z1
+      const int qa = q0 + (lane >> 3) * kDecideWarps, qb = qa + 4 * kDecideWarps;
+      if (qa < np) s_pval[qa] = z0;
+      if (qb < np) s_pval[qb] = z1;
     }
   }
   __syncthreads();
@@ -415,87 +424,172 @@ __global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideP
   __syncthreads();
   // ---- B: append selection: the n_a smallest scores, ties to the smaller token index ----
   if (n_a > 0) {
-    if (tid < C) {
+    // `parts` threads share a token: each counts over a quarter (or half) of the block, the counts
+    // are added inside the group of adjacent lanes
+    {
+      const int j = tid / parts, part = tid % parts;
       int rank = 0;
-      const double sj = s_score[tid];
-#pragma unroll 8
-      for (int jj = 0; jj < C; ++jj) {
-        const double so = s_score[jj];
-        rank += (so < sj || (so == sj && jj < tid)) ? 1 : 0;
+      if (j < C) {
+        const double sj = s_score[j];
+        const int per = (C + parts - 1) / parts;
+        const int j1 = min(C, (part + 1) * per);
+#pragma unroll 4
+        for (int jj = part * per; jj < j1; ++jj) {
+          const double so = s_score[jj];
+          rank += (so < sj || (so == sj && jj < j)) ? 1 : 0;
+        }
       }
-      s_app[tid] = rank < n_a ? 1 : 0;
+#pragma unroll
+      for (int o = parts / 2; o > 0; o >>= 1) rank += __shfl_xor_sync(0xffffffffu, rank, o);
+      if (j < C && part == 0) s_app[j] = rank < n_a ? 1 : 0;
     }
     __syncthreads();
-    if (tid < C && s_app[tid]) {
+    {
+      const int j = tid / parts, part = tid % parts;
       int before = 0;
-#pragma unroll 8
-      for (int jj = 0; jj < tid; ++jj) before += s_app[jj];
-      s_creator[before] = tid;          // rows are laid down in ascending token order
+      if (j < C && s_app[j]) {
+        const int per = (C + parts - 1) / parts;
+        const int j1 = min(j, (part + 1) * per);
+        for (int jj = part * per; jj < j1; ++jj) before += s_app[jj];
+      }
+#pragma unroll
+      for (int o = parts / 2; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
+      if (j < C && part == 0 && s_app[j]) s_creator[before] = j;   // rows are laid down in ascending token order
     }
     __syncthreads();
   }
-  // ---- D: merge target against s_+ (old rows: refined candidates; new rows: exact).  A warp takes
-  //      four tokens at a time, so every row key it loads is used four times, and reduces the four
-  //      partial sums together; lane group t (8 lanes) ends up owning token t of the quad. ----
-  for (int j0 = 4 * warp; j0 < C; j0 += 4 * kDecideWarps) {
-    const int t = ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1);
-    const int jt = j0 + t;                        // the token this lane group decides
-    const bool live = jt < C && !s_app[jt];
-    double best = live ? s_best[jt] : -INFINITY;
-    int arg = live ? s_barg[jt] : -1;
-    if (n_a > 0) {
-      double kb[4][CH];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const int j = min(j0 + q, C - 1);
-#pragma unroll
-        for (int c = 0; c < CH; ++c) kb[q][c] = kbarU[(int64_t)j * D + lane + 32 * c];
+  // ---- D: merge target against s_+ = old rows (best exact similarity known from A) and the rows
+  //      appended by this fold.  The tensor-core products gramT[a][j] ~ kbarHat_a . kbar_j are within
+  //      eps_j = thr_j / 2 of the exact values, so a new row can only win when its approximate value
+  //      plus eps_j reaches both the exact best old value and (best approximate new value - eps_j).
+  //      Those few pairs are recomputed in fp64; everything else is decided by the bound. ----
+  if (tid == 0) s_np = 0;
+  __syncthreads();
+  if (n_a > 0 && tid < C) {
+    const int j = tid;
+    s_pcnt[j] = 0;
+    s_exh[j] = 0;
+    if (!s_app[j]) {
+      const double eps = 0.5 * (double)(p.thr_coeff * p.kbarNorm[tokBase + j] + 1e-5f);
+      const float* gcol = p.gramT + (int64_t)u * p.Cmax * p.Cmax + j;
+      float gm = -INFINITY;
+#pragma unroll 8
+      for (int a = 0; a < n_a; ++a) gm = fmaxf(gm, gcol[(int64_t)s_creator[a] * p.Cmax]);
+      const double bar = fmax(s_best[j], (double)gm - eps) - eps;
+      int cntc = 0;
+#pragma unroll 8
+      for (int a = 0; a < n_a; ++a) cntc += ((double)gcol[(int64_t)s_creator[a] * p.Cmax] >= bar) ? 1 : 0;
+      bool exh = cntc > kPairPerTok;
+      int start = 0;
+      if (!exh && cntc > 0) {
+        start = atomicAdd(&s_np, cntc);
+        if (start + cntc > kPairCap) exh = true;
       }
-#pragma unroll 2
-      for (int a = 0; a < n_a; ++a) {
-        const double* kh = p.kbarHat64 + (tokBase + s_creator[a]) * D;
-        double h[CH];
-#pragma unroll
-        for (int c = 0; c < CH; ++c) h[c] = kh[lane + 32 * c];
-        double part[4] = {0.0, 0.0, 0.0, 0.0};
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-#pragma unroll
-          for (int c = 0; c < CH; ++c) part[q] += kb[q][c] * h[c];
+      if (!exh && cntc > 0) {
+        int w = start;
+        for (int a = 0; a < n_a; ++a) {
+          if ((double)gcol[(int64_t)s_creator[a] * p.Cmax] >= bar) {
+            s_prow[w] = a;                      // index of the new row, ascending within a token
+            s_ptok[w] = (unsigned short)j;
+            ++w;
+          }
         }
-        const double z = warp_reduce4(part[0], part[1], part[2], part[3], lane);
-        if (z > best) { best = z; arg = (int)m + a; }
+        s_pstart[j] = start;
+        s_pcnt[j] = cntc;
       }
-    }
-    if (live && (lane & 7) == 0) {
-      s_pi[jt] = arg;
-      atomicAdd(&s_nmerge, 1);
+      s_exh[j] = exh ? 1 : 0;
+      if (exh) atomicAdd(&s_nexh, 1);
     }
   }
   __syncthreads();
-  // ---- E: order merged tokens by (row, token); publish ----
-  if (tid < C) {
-    const int pj = s_pi[tid];
-    p.pi[tokBase + tid] = pj;
-    p.creator[tokBase + tid] = s_creator[tid];
-    if (pj >= 0) {
-      int ord = 0;
-      bool head = true;
-#pragma unroll 8
-      for (int jj = 0; jj < C; ++jj) {
-        const int po = s_pi[jj];
-        ord += (po >= 0 && (po < pj || (po == pj && jj < tid))) ? 1 : 0;
-        if (po == pj && jj < tid) head = false;
+  if (n_a > 0) {
+    const int np2 = min(s_np, kPairCap);
+    for (int q0 = warp; q0 < np2; q0 += 8 * kDecideWarps) {
+      double part[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int q = min(q0 + k * kDecideWarps, np2 - 1);
+        const double* kb = kbarU + (int64_t)s_ptok[q] * D;
+        const double* kh = p.kbarHat64 + (tokBase + s_creator[s_prow[q]]) * D;
+        double acc = 0.0;
+#pragma unroll
+        for (int c = 0; c < CH; ++c) acc += kb[lane + 32 * c] * kh[lane + 32 * c];
+        part[k] = acc;
       }
-      p.sorted[tokBase + ord] = tid;
-      if (head && pj >= m) p.segnew[tokBase + (pj - (int)m)] = ord;
+      const double z0 = warp_reduce4(part[0], part[1], part[2], part[3], lane);
+      const double z1 = warp_reduce4(part[4], part[5], part[6], part[7], lane);
+      if ((lane & 7) == 0) {
+        const int qa = q0 + (lane >> 3) * kDecideWarps, qb = qa + 4 * kDecideWarps;
+        if (qa < np2) s_pval[qa] = z0;
+        if (qb < np2) s_pval[qb] = z1;
+      }
+    }
+    // tokens whose candidate list did not fit: every new row exactly, one warp per token
+    for (int j = warp; j < C; j += kDecideWarps) {
+      if (!s_exh[j]) continue;
+      double kb[CH];
+#pragma unroll
+      for (int c = 0; c < CH; ++c) kb[c] = kbarU[(int64_t)j * D + lane + 32 * c];
+      double best = s_best[j];
+      int arg = s_barg[j];
+      for (int a = 0; a < n_a; ++a) {
+        const double* kh = p.kbarHat64 + (tokBase + s_creator[a]) * D;
+        double acc = 0.0;
+#pragma unroll
+        for (int c = 0; c < CH; ++c) acc += kb[c] * kh[lane + 32 * c];
+        acc = warp_sum_d(acc);
+        if (acc > best) { best = acc; arg = (int)m + a; }
+      }
+      if (lane == 0) { s_best[j] = best; s_barg[j] = arg; }
+    }
+  }
+  __syncthreads();
+  if (tid < C && !s_app[tid]) {
+    double best = s_best[tid];
+    int arg = s_barg[tid];
+    if (n_a > 0 && !s_exh[tid]) {
+      const int st0 = s_pstart[tid];
+      for (int q = st0; q < st0 + s_pcnt[tid]; ++q) {   // ascending new-row index: the first maximum wins
+        const double v = s_pval[q];
+        if (v > best) { best = v; arg = (int)m + s_prow[q]; }
+      }
+    }
+    s_pi[tid] = arg;
+    atomicAdd(&s_nmerge, 1);
+  }
+  __syncthreads();
+  // ---- E: order merged tokens by (row, token); publish ----
+  {
+    const int j = tid / parts, part = tid % parts;
+    const int pj = j < C ? s_pi[j] : -1;
+    if (j < C && part == 0) {
+      p.pi[tokBase + j] = pj;
+      p.creator[tokBase + j] = s_creator[j];
+    }
+    int ord = 0, nothead = 0;
+    if (pj >= 0) {
+      const int per = (C + parts - 1) / parts;
+      const int j1 = min(C, (part + 1) * per);
+#pragma unroll 4
+      for (int jj = part * per; jj < j1; ++jj) {
+        const int po = s_pi[jj];
+        ord += (po >= 0 && (po < pj || (po == pj && jj < j))) ? 1 : 0;
+        nothead |= (po == pj && jj < j) ? 1 : 0;
+      }
+    }
+#pragma unroll
+    for (int o = parts / 2; o > 0; o >>= 1) {
+      ord += __shfl_xor_sync(0xffffffffu, ord, o);
+      nothead |= __shfl_xor_sync(0xffffffffu, nothead, o);
+    }
+    if (pj >= 0 && part == 0) {
+      p.sorted[tokBase + ord] = j;
+      if (!nothead && pj >= m) p.segnew[tokBase + (pj - (int)m)] = ord;
     }
   }
   if (tid == 0) {
     p.nmerge[u] = s_nmerge;
-    int nexh = 0;
-    for (int j = 0; j < C; ++j) nexh += s_exh[j];
-    atomicAdd(&p.counters[0], nexh);
+    atomicAdd(&p.counters[0], s_nexh);
     atomicAdd(&p.counters[1], min(s_np, kPairCap));
     atomicAdd(&p.counters[2], C);
   }
@@ -643,8 +737,9 @@ __global__ void __launch_bounds__(256) fold_apply_kernel(FoldApplyParams p) {
 }
 
 int launch_route_filter_tc(State* st, int64_t m, int nsplit, int slot, cudaStream_t s);
+int launch_gram_tc(State* st, int slot0, int nblk, cudaStream_t s);
 
-int launch_kbar(State* st, const __half* ok, int64_t unit_stride, int nblk, int slot0, cudaStream_t s) {
+int launch_kbar(State* st, const __half* ok, int64_t unit_stride, int nblk, int slot0, bool want_gram, cudaStream_t s) {
   KernelTimer kt(st, 2, s);
   const int C = st->C, D = st->d;
   const int64_t U = st->U;
@@ -653,13 +748,17 @@ int launch_kbar(State* st, const __half* ok, int64_t unit_stride, int nblk, int 
   __half* kh = st->kbarH + (int64_t)slot0 * U * st->CbarRows * D;
   float* kn = st->kbarNorm + (int64_t)slot0 * U * st->Cmax;
   double* khat = st->kbarHat64 + (int64_t)slot0 * U * st->Cmax * D;
+  __half* khh = st->kbarHatH + (int64_t)slot0 * U * st->CbarRows * D;
   if (D == 128)
-    kbar_kernel<128><<<grid, 256, 0, s>>>(ok, unit_stride, st->ln_w, st->ln_b, k64, kh, kn, khat, C, st->Cmax,
+    kbar_kernel<128><<<grid, 256, 0, s>>>(ok, unit_stride, st->ln_w, st->ln_b, k64, kh, kn, khat, khh, C, st->Cmax,
                                           st->CbarRows, st->U, st->Hkv, st->r, (double)st->ln_eps);
   else
-    kbar_kernel<64><<<grid, 256, 0, s>>>(ok, unit_stride, st->ln_w, st->ln_b, k64, kh, kn, khat, C, st->Cmax,
+    kbar_kernel<64><<<grid, 256, 0, s>>>(ok, unit_stride, st->ln_w, st->ln_b, k64, kh, kn, khat, khh, C, st->Cmax,
                                          st->CbarRows, st->U, st->Hkv, st->r, (double)st->ln_eps);
-  return 1;
+  int launches = 1;
+  // the new-row filter is only read by folds that append some but not all of their tokens
+  if (want_gram) launches += launch_gram_tc(st, slot0, nblk, s);
+  return launches;
 }
 
 int launch_prev_copy(State* st, cudaStream_t s) {
@@ -715,6 +814,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
     }
     FoldDecideParams p;
     p.kbar64 = kbar64; p.kbarNorm = kbarNorm; p.kbarHat64 = kbarHat64;
+    p.gramT = st->gramT + (int64_t)a.slot * U * st->Cmax * st->Cmax;
     p.candV = st->candV; p.candI = st->candI; p.ln_w = st->ln_w; p.ln_b = st->ln_b;
     p.sumK = st->sumK; p.kmu = st->kmu; p.krstd = st->krstd;
     p.pi = st->foldPi[dst]; p.sorted = st->foldSorted[dst]; p.creator = st->foldCreator[dst];

@@ -55,8 +55,8 @@ struct State {
   int64_t prevM;
   int prevNAppend;
   // second stream and events that let a block's attention and the fold of the block before it overlap
-  cudaStream_t foldStream;
-  cudaEvent_t evJoin, evPre[2], evFold[2];
+  cudaStream_t foldStream, kbStream;   // folds; memory keys computed ahead of the folds
+  cudaEvent_t evJoin, evPre[2], evFold[2], evKb[2], evBatchDone[2];
   // ---- window ring (device): slot = t mod ringLen ----
   __half *ringK, *ringV;         // [U, w*Cmax, d]  rotated keys / values (fp16)
   float* ringG;                  // [U, w*Cmax]
@@ -75,6 +75,8 @@ struct State {
   float* kbarNorm;               // [kbSlots][U, Cmax]
   int CbarRows;                  // rows per unit of kbarH (Cmax rounded up to the 128-row MMA tile)
   double* kbarHat64;             // [kbSlots][U, Cmax, d]  LN_s(kbar_j): the readout key of a row created by token j
+  __half* kbarHatH;              // [kbSlots][U, CbarRows, d]  the same in fp16 (operand of the new-row filter)
+  float* gramT;                  // [kbSlots][U, Cmax, Cmax]  approximate kbarHat_a . kbar_j at [a][j] (new-row filter)
   // decisions of the fold being computed ([(nfolds+1) & 1]) and of the one before ([nfolds & 1])
   int32_t *foldPi[2], *foldSorted[2], *foldCreator[2], *foldSegNew[2], *foldNMerge[2];
   int nsplitRoute;               // splits the routing filter may use
@@ -93,8 +95,9 @@ struct State {
   uint8_t* appTok;               // [U, Tassign]
   int32_t* status;               // device status word
   // ---- TMA tensor maps (host copies, passed to kernels by value):
-  //      0 stQ, 1 Khat copy 0, 2 Vhat copy 0, 3 stK, 4 stV, 5 kbarH, 6 Khat copy 1, 7 Vhat copy 1 ----
-  alignas(64) unsigned char tmaps[8 * 128];
+  //      0 stQ, 1 Khat copy 0, 2 Vhat copy 0, 3 stK, 4 stV, 5 kbarH, 6 Khat copy 1, 7 Vhat copy 1,
+  //      8 kbarHatH ----
+  alignas(64) unsigned char tmaps[9 * 128];
   // ---- device staging for the *_host entry points ----
   void *hQ, *hK, *hV, *hOut;
   float* hG;
@@ -148,7 +151,7 @@ struct FoldArgs {
 int launch_fold(State* st, const FoldArgs& a, cudaStream_t s);
 // Memory keys of nblk consecutive blocks (C rows each, starting at ok within every unit) into slots
 // slot0 .. slot0 + nblk - 1.
-int launch_kbar(State* st, const __half* ok, int64_t unit_stride, int nblk, int slot0, cudaStream_t s);
+int launch_kbar(State* st, const __half* ok, int64_t unit_stride, int nblk, int slot0, bool want_gram, cudaStream_t s);
 // Copies the readout rows that the last fold touched from the current readout copy into the other
 // one (no-op when nothing is owed).  Must run after every reader of the other copy has finished and
 // before the next fold writes it.

@@ -28,6 +28,8 @@ struct RouteTcParams {
   int32_t* status;
   const float* kbarNorm;   // [U, Cmax] upper bound of ||kbar_j||
   int a_unit0;             // first unit of this block's slot in the memory-key tensor map
+  float* gramT;            // [slots][U, Cmax, Cmax]: output of the new-row filter launch (gram_mode), see below
+  int gram_mode, U;        // gram_mode: grid (1, U, blocks), block z uses slot a_unit0 / U + z
   float thr_coeff;         // candidate window = thr_coeff * ||kbar_j|| + 1e-5
   int64_t m;
   int C, Cmax, nsplit, S;
@@ -51,7 +53,7 @@ enum { RB_AFULL = 0, RB_BFULL = 1, RB_BFREE = 4, RB_SFULL = 7, RB_ACCFREE = 9, R
 template <int D>
 __global__ void __launch_bounds__(320, 1)
 route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
-                       const RouteTcParams p) {
+                       const __grid_constant__ CUtensorMap mapH, const RouteTcParams p) {
   using Cfg = RouteTcCfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -64,12 +66,17 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int split = blockIdx.x, u = blockIdx.y;
   const int mt_used = (p.C + 127) / 128;
+  // New-row filter mode (a launch of its own, ahead of the folds: it needs the block's keys only):
+  // the would-be row keys LN_s(kbar_a) are the M operand, the memory keys kbar_j the N operand, one
+  // pass, and the products themselves are stored, gramT[a][j]; which rows a exist is known later.
+  const bool gram = p.gram_mode != 0;
+  const int a_unit = p.a_unit0 + (gram ? (int)blockIdx.z * p.U : 0) + u;
   int64_t per = (p.m + p.nsplit - 1) / p.nsplit;
   per = (per + 127) / 128 * 128;
-  const int64_t i0 = (int64_t)split * per;
-  const int64_t i1 = min(p.m, i0 + per);
+  const int64_t i0 = gram ? 0 : (int64_t)split * per;
+  const int64_t i1 = gram ? (int64_t)p.C : min(p.m, i0 + per);
   const int ntiles = i1 > i0 ? (int)((i1 - i0 + 127) / 128) : 0;
-  const int nsteps = 2 * ntiles;   // every tile is visited in pass 1 and again in pass 2
+  const int nsteps = gram ? ntiles : 2 * ntiles;   // a split's tiles are visited in pass 1 and again in pass 2
 
   if (tid == 0) {
     tc::mbar_init(&bars[RB_AFULL], 1);
@@ -95,11 +102,11 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
 
   if (warp == 0) {
     if (lane == 0) {
-      tc::prefetch_tmap(&mapA); tc::prefetch_tmap(&mapB);
+      tc::prefetch_tmap(&mapA); tc::prefetch_tmap(&mapB); tc::prefetch_tmap(&mapH);
       tc::mbar_expect_tx(&bars[RB_AFULL], mt_used * Cfg::TILE_BYTES);
       for (int mt = 0; mt < mt_used; ++mt)
         for (int kb = 0; kb < Cfg::NKB; ++kb)
-          tc::tma_load_3d(sA + mt * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, &mapA, &bars[RB_AFULL], kb * 64, mt * 128, p.a_unit0 + u);
+          tc::tma_load_3d(sA + mt * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, gram ? &mapH : &mapA, &bars[RB_AFULL], kb * 64, mt * 128, a_unit);
       for (int j = 0; j < nsteps; ++j) {
         const int s = j % Cfg::NS;
         const int jt = j >= ntiles ? j - ntiles : j;
@@ -109,8 +116,8 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
         }
         tc::mbar_expect_tx(&bars[RB_BFULL + s], Cfg::TILE_BYTES);
         for (int kb = 0; kb < Cfg::NKB; ++kb)
-          tc::tma_load_3d(sB + s * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, &mapB, &bars[RB_BFULL + s], kb * 64,
-                          (int)(i0 + (int64_t)jt * 128), u);
+          tc::tma_load_3d(sB + s * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, gram ? &mapA : &mapB, &bars[RB_BFULL + s], kb * 64,
+                          (int)(i0 + (int64_t)jt * 128), gram ? a_unit : u);
       }
     }
   } else if (warp == 1) {
@@ -177,6 +184,20 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(&bars[RB_ACCFREE + buf]);
           }
+          if (gram) {   // row `tok` of gramT: 32 consecutive tokens j = row0 + c4*32 .. (rows past C are never read)
+            if (tok < p.C) {
+              float* dst = p.gramT + ((int64_t)a_unit * p.Cmax + tok) * p.Cmax + row0 + c4 * 32;
+              if (row0 + c4 * 32 + 32 <= p.Cmax) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                  reinterpret_cast<uint4*>(dst)[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+              } else {
+                for (int i = 0; i < 32; ++i)
+                  if (row0 + c4 * 32 + i < p.Cmax) dst[i] = __uint_as_float(r[i]);
+              }
+            }
+            continue;
+          }
           uint32_t vm = 0xffffffffu;   // columns of this chunk that count
           if (!plain) {
             const int a = min(32, max(0, lo - c4 * 32)), b = min(32, max(0, nvalid - c4 * 32));
@@ -211,7 +232,7 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
           }
         }
       }
-      if (tok < p.C) {
+      if (tok < p.C && !gram) {
         const int64_t o = (((int64_t)u * p.nsplit + split) * p.Cmax + tok) * kTopK;
 #pragma unroll
         for (int k = 0; k < kTopK; ++k) p.candI[o + k] = ci[k];
@@ -234,18 +255,33 @@ int launch_route_filter_tc(State* st, int64_t m, int nsplit, int slot, cudaStrea
   p.candV = st->candV; p.candI = st->candI; p.status = st->status; p.m = m;
   p.C = st->C; p.Cmax = st->Cmax; p.nsplit = nsplit; p.S = st->S;
   p.kbarNorm = st->kbarNorm + (int64_t)slot * st->U * st->Cmax; p.thr_coeff = route_thr_coeff(st);
-  p.a_unit0 = slot * st->U;
+  p.a_unit0 = slot * st->U; p.gramT = st->gramT; p.gram_mode = 0; p.U = st->U;
   const CUtensorMap* tm = reinterpret_cast<const CUtensorMap*>(st->tmaps);
   dim3 grid(nsplit, st->U);
   const int ks = (st->nfolds & 1) ? 6 : 1;   // the fold reads the readout copy of the current version
-  if (st->d == 128) route_filter_tc_kernel<128><<<grid, 320, RouteTcCfg<128>::SMEM_BYTES, s>>>(tm[5], tm[ks], p);
-  else route_filter_tc_kernel<64><<<grid, 320, RouteTcCfg<64>::SMEM_BYTES, s>>>(tm[5], tm[ks], p);
+  if (st->d == 128) route_filter_tc_kernel<128><<<grid, 320, RouteTcCfg<128>::SMEM_BYTES, s>>>(tm[5], tm[ks], tm[8], p);
+  else route_filter_tc_kernel<64><<<grid, 320, RouteTcCfg<64>::SMEM_BYTES, s>>>(tm[5], tm[ks], tm[8], p);
+  return 1;
+}
+
+// New-row filter of nblk blocks whose memory keys sit in slots slot0 .. slot0 + nblk - 1.
+int launch_gram_tc(State* st, int slot0, int nblk, cudaStream_t s) {
+  RouteTcParams p;
+  p.candV = st->candV; p.candI = st->candI; p.status = st->status; p.m = 0;
+  p.C = st->C; p.Cmax = st->Cmax; p.nsplit = 1; p.S = st->S;
+  p.kbarNorm = st->kbarNorm; p.thr_coeff = 0.f;
+  p.a_unit0 = slot0 * st->U; p.gramT = st->gramT; p.gram_mode = 1; p.U = st->U;
+  const CUtensorMap* tm = reinterpret_cast<const CUtensorMap*>(st->tmaps);
+  dim3 grid(1, st->U, nblk);
+  if (st->d == 128) route_filter_tc_kernel<128><<<grid, 320, RouteTcCfg<128>::SMEM_BYTES, s>>>(tm[5], tm[1], tm[8], p);
+  else route_filter_tc_kernel<64><<<grid, 320, RouteTcCfg<64>::SMEM_BYTES, s>>>(tm[5], tm[1], tm[8], p);
   return 1;
 }
 
 bool setup_route_tc(State* st) {
   CUtensorMap* tm = reinterpret_cast<CUtensorMap*>(st->tmaps);
   if (!encode_tmap_rows(&tm[5], st->kbarH, st->d, st->CbarRows, (int64_t)st->kbSlots * st->U, 128)) return false;
+  if (!encode_tmap_rows(&tm[8], st->kbarHatH, st->d, st->CbarRows, (int64_t)st->kbSlots * st->U, 128)) return false;
   if (cudaFuncSetAttribute(route_filter_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, RouteTcCfg<128>::SMEM_BYTES) != cudaSuccess) return false;
   if (cudaFuncSetAttribute(route_filter_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, RouteTcCfg<64>::SMEM_BYTES) != cudaSuccess) return false;
   return true;
