@@ -276,7 +276,9 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
     A(s.foldPi[i], U * Cm); A(s.foldSorted[i], U * Cm); A(s.foldCreator[i], U * Cm); A(s.foldSegNew[i], U * Cm);
     A(s.foldNMerge[i], U);
   }
-  A(s.candV, U * (size_t)s.nsplitRoute * Cm * kTopK); A(s.candI, U * (size_t)s.nsplitRoute * Cm * kTopK);
+  A(s.xScore, U * Cm); A(s.xBest, U * Cm); A(s.xArg, U * Cm); A(s.xCount, U);
+  if (rc == KVM_OK && cudaMemset(s.xCount, 0, U * sizeof(int32_t)) != cudaSuccess) rc = KVM_ERR_CUDA;
+  A(s.candV, U * (size_t)(2 * s.nsplitRoute) * Cm * kTopK); A(s.candI, U * (size_t)(2 * s.nsplitRoute) * Cm * kTopK);
   A(s.decPart, (size_t)s.B * s.Hq * s.nsplitDec * (d + 2)); A(s.decQ, (size_t)s.B * s.Hq * d);
   A(s.status, (size_t)16);   // [0] status word, [1..3] fold debug counters
   if (s.Tassign > 0) { A(s.slotTok, U * (size_t)s.Tassign); A(s.appTok, U * (size_t)s.Tassign); }

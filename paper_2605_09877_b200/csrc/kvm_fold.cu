@@ -230,6 +230,8 @@ struct FoldDecideParams {
   const double* sumK;
   const double *kmu, *krstd;
   int32_t *pi, *sorted, *creator, *segnew, *nmerge;   // outputs, [U, Cmax] (nmerge [U])
+  double *xScore, *xBest;   // [U, Cmax] per-token results handed from the slice CTAs to the last one
+  int32_t *xArg, *xCount;   // [U, Cmax]; [U] ticket counter (zero between launches)
   int32_t* counters;   // debug: [0] tokens on the exhaustive path, [1] candidate pairs, [2] tokens decided
   int64_t Mcap, m;
   int C, Cmax, Hkv, S, n_append, nsplit;
@@ -277,7 +279,7 @@ __device__ __forceinline__ double warp_sim(const double (&kb)[CH], const double*
 }
 
 template <int D>
-__global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideParams p) {
+__global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDecideParams p) {
   constexpr int CH = D / 32;
   __shared__ double s_score[kMaxBlock], s_best[kMaxBlock];
   __shared__ int s_barg[kMaxBlock], s_pi[kMaxBlock], s_creator[kMaxBlock];
@@ -286,11 +288,15 @@ __global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideP
   __shared__ int s_prow[kPairCap];
   __shared__ unsigned short s_ptok[kPairCap];
   __shared__ double s_pval[kPairCap];
-  __shared__ int s_np, s_nmerge, s_nexh;
+  __shared__ int s_np, s_nmerge, s_nexh, s_last;
 
-  const int u = blockIdx.x, hk = u % p.Hkv;
+  // grid (R, U): CTA r of a unit refines the candidates of tokens [jlo, jhi); the CTA of the unit
+  // that finishes last (a ticket, nobody waits) takes the decisions that need every token
+  const int u = blockIdx.y, hk = u % p.Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int C = p.C;
+  const int R = gridDim.x;
+  const int jlo = (int)blockIdx.x * ((C + R - 1) / R), jhi = min(C, jlo + (C + R - 1) / R);
   const int64_t m = p.m;
   const int n_a = p.n_append;
   const int parts = C <= 64 ? 8 : (C <= 128 ? 4 : 2);   // adjacent threads that share a token in the ranking loops
@@ -313,8 +319,8 @@ __global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideP
   __syncthreads();
 
   // ---- A1/A2: candidate pairs from the filter lists ----
-  if (tid < C) {
-    const int j = tid;
+  if (jlo + tid < jhi) {
+    const int j = jlo + tid;
     const float thr = p.thr_coeff * p.kbarNorm[tokBase + j] + 1e-5f;
     const int64_t o0 = ((int64_t)u * p.nsplit * p.Cmax + j) * kTopK;
     const int64_t ostep = (int64_t)p.Cmax * kTopK;
@@ -392,22 +398,23 @@ __global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideP
   }
   __syncthreads();
   // ---- A4: per-token reduction (ties: lowest row) ----
-  if (tid < C && !s_exh[tid]) {
+  if (jlo + tid < jhi && !s_exh[jlo + tid]) {
+    const int j = jlo + tid;
     double score = -INFINITY, best = -INFINITY;
     int barg = -1;
-    const int st0 = s_pstart[tid];
-    for (int q = st0; q < st0 + s_pcnt[tid]; ++q) {
+    const int st0 = s_pstart[j];
+    for (int q = st0; q < st0 + s_pcnt[j]; ++q) {
       const double v = s_pval[q];
       const int i = s_prow[q];
       if (v > score) score = v;
       if (i >= p.S && (v > best || (v == best && i < barg))) { best = v; barg = i; }
     }
-    s_score[tid] = score;
-    s_best[tid] = best;
-    s_barg[tid] = barg;
+    s_score[j] = score;
+    s_best[j] = best;
+    s_barg[j] = barg;
   }
   // ---- A5: exhaustive path for flagged tokens: one warp per token, rows in sequence ----
-  for (int j = warp; j < C; j += kDecideWarps) {
+  for (int j = jlo + warp; j < jhi; j += kDecideWarps) {
     if (!s_exh[j]) continue;
     double kb[CH];
 #pragma unroll
@@ -422,6 +429,32 @@ __global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideP
     if (lane == 0) { s_score[j] = score; s_best[j] = best; s_barg[j] = barg; }
   }
   __syncthreads();
+  if (R > 1) {
+    // hand the slice's results over; the last CTA of the unit to get here carries on with all of them
+    if (jlo + tid < jhi) {
+      const int j = jlo + tid;
+      p.xScore[tokBase + j] = s_score[j];
+      p.xBest[tokBase + j] = s_best[j];
+      p.xArg[tokBase + j] = s_barg[j];
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+      atomicAdd(&p.counters[0], s_nexh);
+      atomicAdd(&p.counters[1], min(s_np, kPairCap));
+      s_last = atomicAdd(&p.xCount[u], 1) == R - 1 ? 1 : 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (tid == 0) { p.xCount[u] = 0; s_nexh = 0; s_np = 0; }
+    if (tid < C) {   // read past the L1, which may hold stale lines of these arrays
+      s_score[tid] = __ldcg(p.xScore + tokBase + tid);
+      s_best[tid] = __ldcg(p.xBest + tokBase + tid);
+      s_barg[tid] = __ldcg(p.xArg + tokBase + tid);
+    }
+    __syncthreads();
+  }
   // ---- B: append selection: the n_a smallest scores, ties to the smaller token index ----
   if (n_a > 0) {
     // `parts` threads share a token: each counts over a quarter (or half) of the block, the counts
@@ -463,7 +496,7 @@ __global__ void __launch_bounds__(kDecideThreads) fold_decide_kernel(FoldDecideP
   //      eps_j = thr_j / 2 of the exact values, so a new row can only win when its approximate value
   //      plus eps_j reaches both the exact best old value and (best approximate new value - eps_j).
   //      Those few pairs are recomputed in fp64; everything else is decided by the bound. ----
-  if (tid == 0) s_np = 0;
+  if (tid == 0) { atomicAdd(&p.counters[1], min(s_np, kPairCap)); s_np = 0; }
   __syncthreads();
   if (n_a > 0 && tid < C) {
     const int j = tid;
@@ -820,12 +853,17 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
     p.pi = st->foldPi[dst]; p.sorted = st->foldSorted[dst]; p.creator = st->foldCreator[dst];
     p.segnew = st->foldSegNew[dst]; p.nmerge = st->foldNMerge[dst];
     p.counters = st->status + 1;
+    p.xScore = st->xScore; p.xBest = st->xBest; p.xArg = st->xArg; p.xCount = st->xCount;
     p.Mcap = st->Mcap; p.m = a.m;
     p.C = C; p.Cmax = st->Cmax; p.Hkv = st->Hkv; p.S = st->S; p.n_append = a.n_append; p.nsplit = nsplit;
     p.thr_coeff = route_thr_coeff(st);
     KernelTimer kt(st, 4, s);
-    if (D == 128) fold_decide_kernel<128><<<st->U, kDecideThreads, 0, s>>>(p);
-    else fold_decide_kernel<64><<<st->U, kDecideThreads, 0, s>>>(p);
+    // two CTAs per unit while that still fits the GPU in one wave (measured: the hand-over costs
+    // more than it saves beyond two), one otherwise
+    int R = (2 * st->U <= 2 * 148 && C >= 32) ? 2 : 1;
+    dim3 dgrid(R, st->U);
+    if (D == 128) fold_decide_kernel<128><<<dgrid, kDecideThreads, 0, s>>>(p);
+    else fold_decide_kernel<64><<<dgrid, kDecideThreads, 0, s>>>(p);
     ++launches;
   }
   FoldApplyParams q;

@@ -79,6 +79,8 @@ struct State {
   float* gramT;                  // [kbSlots][U, Cmax, Cmax]  approximate kbarHat_a . kbar_j at [a][j] (new-row filter)
   // decisions of the fold being computed ([(nfolds+1) & 1]) and of the one before ([nfolds & 1])
   int32_t *foldPi[2], *foldSorted[2], *foldCreator[2], *foldSegNew[2], *foldNMerge[2];
+  double *xScore, *xBest;        // [U, Cmax] hand-over between the CTAs of the decide kernel
+  int32_t *xArg, *xCount;        // [U, Cmax]; [U]
   int nsplitRoute;               // splits the routing filter may use
   float* candV;                  // [U, nsplitRoute, Cmax, kTopK]
   int32_t* candI;
