@@ -311,6 +311,8 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
     bet[i] = (double)p.ln_b[hk * D + lane + 32 * i];
   }
   if (tid == 0) { s_np = 0; s_nmerge = 0; s_nexh = 0; }
+  // everything above reads parameters only; the routing filter's lists are read from here on
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (tid < kMaxBlock) {
     s_app[tid] = 0; s_exh[tid] = 0; s_pcnt[tid] = 0; s_pstart[tid] = 0; s_pi[tid] = -1;
     s_best[tid] = -INFINITY; s_barg[tid] = -1; s_score[tid] = -INFINITY; s_creator[tid] = -1;
@@ -824,7 +826,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
   const bool all_append = a.first || a.n_append >= C;
   if (!all_append) {
     // enough CTAs to fill the GPU, at least 256 rows per split
-    int64_t want = (148 + st->U - 1) / st->U;
+    int64_t want = 148 / st->U;   // rounded down: a few CTAs in a second wave would double the kernel's time
     int64_t maxs = (a.m + 255) / 256;
     int nsplit = (int)(want < maxs ? want : maxs);
     if (nsplit < 1) nsplit = 1;
@@ -862,8 +864,22 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
     // more than it saves beyond two), one otherwise
     int R = (2 * st->U <= 2 * 148 && C >= 32) ? 2 : 1;
     dim3 dgrid(R, st->U);
-    if (D == 128) fold_decide_kernel<128><<<dgrid, kDecideThreads, 0, s>>>(p);
-    else fold_decide_kernel<64><<<dgrid, kDecideThreads, 0, s>>>(p);
+    // programmatic dependent launch: the CTAs may start (and set up their shared memory) while the
+    // routing filter is still running; they wait for it before the first read of its output
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dgrid; lc.blockDim = dim3(kDecideThreads); lc.dynamicSmemBytes = 0; lc.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    // Measured: the early start pays when the filter, these CTAs and the attention CTAs of a block
+    // all find room on the GPU at once (or when every kernel fills it anyway); in between, CTAs
+    // that sit waiting keep the attention kernel, which needs whole SMs, off them.
+    const int sms_wanted = nsplit * st->U + (R * st->U + 1) / 2 + st->B * st->Hq * ((C + 127) / 128);
+    const bool pdl = st->prof_hook == nullptr && !(st->flags & KVM_FLAG_SIMT_ROUTING) &&
+                     (sms_wanted <= 148 || st->U >= 148);
+    lc.attrs = at; lc.numAttrs = pdl ? 1 : 0;
+    if (D == 128) cudaLaunchKernelEx(&lc, fold_decide_kernel<128>, p);
+    else cudaLaunchKernelEx(&lc, fold_decide_kernel<64>, p);
     ++launches;
   }
   FoldApplyParams q;

@@ -99,6 +99,9 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
   __syncthreads();
   tc::tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  // the kernel launched behind this one may begin its set-up now (it waits for this grid to finish
+  // before it reads anything written here)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (warp == 0) {
     if (lane == 0) {
