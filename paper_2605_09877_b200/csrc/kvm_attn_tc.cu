@@ -31,6 +31,8 @@ struct AttnTcParams {
   __nv_bfloat16* out;
   const float *tau_s, *tau_b;
   int32_t* status;
+  float* part;       // split-KV partial results, [tile][split][D + 2][128] (see the epilogue)
+  int32_t* part_cnt; // [tile] tickets, zero between launches
   int nq, Hq, Hkv, G;
 };
 
@@ -82,7 +84,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   const int64_t t_last = t_first + rows_valid - 1;
   const int nst = (int)((p.m + 127) / 128);
   const int nwt = (int)((t_last - p.b + 1 + 127) / 128);
-  const int ntiles = nst + nwt;
+  // Split-KV: with few (batch, head, query tile) triples a launch is cut along the keys as well;
+  // CTA z of gridDim.z walks tiles [jbase, jbase + ntiles) of the nst + nwt tiles of its query tile,
+  // and the partial results are merged by whichever CTA of the tile finishes last.
+  const int nsp = (int)gridDim.z, sp = (int)blockIdx.z;
+  const int ntot = nst + nwt;
+  const int per_split = (ntot + nsp - 1) / nsp;
+  const int jbase = min(ntot, sp * per_split);
+  const int ntiles = min(ntot, jbase + per_split) - jbase;   // tiles of this CTA (0 is possible)
 
   if (tid == 0) {
     tc::mbar_init(&bars[BAR_QFULL], 1);
@@ -129,8 +138,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       auto load_k = [&](int j) -> bool {
         const int s = j % Cfg::NS;
         if (j >= Cfg::NS && !tc::mbar_wait(&bars[BAR_SFULL + s], ((j / Cfg::NS) - 1) & 1)) return false;
-        const bool st = j < nst;
-        const int row = st ? j * 128 : (int)(p.win_row0 + (int64_t)(j - nst) * 128);
+        const int gj = jbase + j;
+        const bool st = gj < nst;
+        const int row = st ? gj * 128 : (int)(p.win_row0 + (int64_t)(gj - nst) * 128);
         tc::mbar_expect_tx(&bars[BAR_KFULL + s], Cfg::TILE_BYTES);
         for (int kb = 0; kb < Cfg::NKB; ++kb)
           tc::tma_load_3d(sK + s * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, st ? &mapKs : &mapKw, &bars[BAR_KFULL + s], kb * 64, row, u);
@@ -142,8 +152,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         if (*abort_flag) break;
         if (j + 1 < ntiles && !load_k(j + 1)) { okp = false; break; }
         if (j >= Cfg::NS && !tc::mbar_wait(&bars[BAR_PVDONE + s], ((j / Cfg::NS) - 1) & 1)) { okp = false; break; }
-        const bool st = j < nst;
-        const int row = st ? j * 128 : (int)(p.win_row0 + (int64_t)(j - nst) * 128);
+        const int gj = jbase + j;
+        const bool st = gj < nst;
+        const int row = st ? gj * 128 : (int)(p.win_row0 + (int64_t)(gj - nst) * 128);
         tc::mbar_expect_tx(&bars[BAR_VFULL + s], Cfg::TILE_BYTES);
         for (int kb = 0; kb < Cfg::NKB; ++kb)
           tc::tma_load_3d(sV + s * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, st ? &mapVs : &mapVw, &bars[BAR_VFULL + s], kb * 64, row, u);
@@ -243,11 +254,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         }
         // region scale (folded into the exponent) and masks; the scale is positive, so the row
         // maximum can be taken on the raw products
-        const bool st = j < nst;
+        const int gj = jbase + j;
+        const bool st = gj < nst;
         const float sc = st ? sc_s : sc_b;
         int64_t nvis;   // number of visible columns of this tile for this row
-        if (st) nvis = p.m - (int64_t)j * 128;
-        else nvis = t_row - (p.b + (int64_t)(j - nst) * 128) + 1;
+        if (st) nvis = p.m - (int64_t)gj * 128;
+        else nvis = t_row - (p.b + (int64_t)(gj - nst) * 128) + 1;
         const int vis = (int)max((int64_t)0, min((int64_t)64, nvis - half * 64));
         float mx = -INFINITY;
         if (vis == 64) {
@@ -321,8 +333,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     constexpr int HD = D / 2;
     float* xch = reinterpret_cast<float*>(sK);          // [2][HD][128]
     float* xml = reinterpret_cast<float*>(sV);          // [2][2][128]: m and l of each half
+    int* last_flag = reinterpret_cast<int*>(tmem_slot + 2);
     do {
       if (!ok) break;
+      if (ntiles == 0) {   // a split without tiles: nothing accumulated, nothing to read back
+        xml[(half * 2 + 0) * 128 + row] = -INFINITY;
+        xml[(half * 2 + 1) * 128 + row] = 0.f;
+        break;
+      }
       ok = false;
       KVM_WAIT(&bars[BAR_PVDONE + ((ntiles - 1) & 1)], ((ntiles - 1) >> 1) & 1);
       tc::tc_fence_after();
@@ -342,29 +360,85 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     } while (false);
     // every softmax thread reaches this barrier, whether or not its waits succeeded
     asm volatile("bar.sync 1, 256;" ::: "memory");
-    if (ok && !*abort_flag) {
-      const float m_o = xml[((1 - half) * 2 + 0) * 128 + row];
-      const float l_o = xml[((1 - half) * 2 + 1) * 128 + row];
-      const float mm = fmaxf(m_run, m_o);
-      const float w_me = (m_run == -INFINITY) ? 0.f : tc::ex2_approx(m_run - mm);
-      const float w_ot = (m_o == -INFINITY) ? 0.f : tc::ex2_approx(m_o - mm);
-      const float inv = 1.f / (l_run * w_me + l_o * w_ot);
-      const float a_me = w_me * inv, a_ot = w_ot * inv;
-      const uint32_t to = tmem + lane_base + col_o + half * HD;
-      const float* srcx = xch + (1 - half) * HD * 128 + row;
-      __nv_bfloat16* orow = p.out + bb * p.so0 + hq * p.so1 + (p.out_t0 + (int64_t)qt * 128 + row) * p.so2 + half * HD;
+    const bool good = ok && !*abort_flag;
+    const float m_o = xml[((1 - half) * 2 + 0) * 128 + row];
+    const float l_o = xml[((1 - half) * 2 + 1) * 128 + row];
+    const float mm = fmaxf(m_run, m_o);
+    const float w_me = (m_run == -INFINITY) ? 0.f : tc::ex2_approx(m_run - mm);
+    const float w_ot = (m_o == -INFINITY) ? 0.f : tc::ex2_approx(m_o - mm);
+    const float lsum2 = l_run * w_me + l_o * w_ot;
+    __nv_bfloat16* orow = p.out + bb * p.so0 + hq * p.so1 + (p.out_t0 + (int64_t)qt * 128 + row) * p.so2 + half * HD;
+    if (nsp == 1) {
+      if (good) {
+        const float inv = 1.f / lsum2;
+        const float a_me = w_me * inv, a_ot = w_ot * inv;
+        const uint32_t to = tmem + lane_base + col_o + half * HD;
+        const float* srcx = xch + (1 - half) * HD * 128 + row;
 #pragma unroll
-      for (int c = 0; c < HD / 32; ++c) {
-        uint32_t r[32];
-        tc::tmem_ld32(to + c * 32, r);
-        tc::tmem_wait_ld();
-        if (row < rows_valid) {
+        for (int c = 0; c < HD / 32; ++c) {
+          uint32_t r[32];
+          tc::tmem_ld32(to + c * 32, r);
+          tc::tmem_wait_ld();
+          if (row < rows_valid) {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float o0 = __uint_as_float(r[2 * i]) * a_me + srcx[(c * 32 + 2 * i) * 128] * a_ot;
-            const float o1 = __uint_as_float(r[2 * i + 1]) * a_me + srcx[(c * 32 + 2 * i + 1) * 128] * a_ot;
-            reinterpret_cast<__nv_bfloat162*>(orow + c * 32)[i] = __floats2bfloat162_rn(o0, o1);
+            for (int i = 0; i < 16; ++i) {
+              const float o0 = __uint_as_float(r[2 * i]) * a_me + srcx[(c * 32 + 2 * i) * 128] * a_ot;
+              const float o1 = __uint_as_float(r[2 * i + 1]) * a_me + srcx[(c * 32 + 2 * i + 1) * 128] * a_ot;
+              reinterpret_cast<__nv_bfloat162*>(orow + c * 32)[i] = __floats2bfloat162_rn(o0, o1);
+            }
           }
+        }
+      }
+    } else {
+      // Partial result of this split: unnormalised O (relative to mm), mm and the sum, column-major
+      // ([channel][row]) so that the rows of a warp are contiguous.
+      const int tile_id = bh * (int)gridDim.x + qt;
+      float* mine = p.part + ((int64_t)tile_id * nsp + sp) * (D + 2) * 128;
+      if (good && ntiles > 0) {
+        const uint32_t to = tmem + lane_base + col_o + half * HD;
+        const float* srcx = xch + (1 - half) * HD * 128 + row;
+#pragma unroll
+        for (int c = 0; c < HD / 32; ++c) {
+          uint32_t r[32];
+          tc::tmem_ld32(to + c * 32, r);
+          tc::tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            mine[(half * HD + c * 32 + i) * 128 + row] = __uint_as_float(r[i]) * w_me + srcx[(c * 32 + i) * 128] * w_ot;
+        }
+      }
+      if (half == 0) {
+        mine[(D + 0) * 128 + row] = (good && ntiles > 0) ? mm : -INFINITY;
+        mine[(D + 1) * 128 + row] = (good && ntiles > 0) ? lsum2 : 0.f;
+      }
+      __threadfence();
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (warp == 4 && lane == 0) *last_flag = atomicAdd(&p.part_cnt[tile_id], 1) == nsp - 1 ? 1 : 0;
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (*last_flag) {   // the last split of the tile to arrive merges all of them (nobody waits)
+        __threadfence();
+        if (warp == 4 && lane == 0) p.part_cnt[tile_id] = 0;
+        const float* allp = p.part + (int64_t)tile_id * nsp * (D + 2) * 128;
+        float mstar = -INFINITY;
+        for (int z = 0; z < nsp; ++z) mstar = fmaxf(mstar, __ldcg(allp + ((int64_t)z * (D + 2) + D) * 128 + row));
+        float acc[HD];
+#pragma unroll
+        for (int c = 0; c < HD; ++c) acc[c] = 0.f;
+        float den = 0.f;
+        for (int z = 0; z < nsp; ++z) {
+          const float* pz = allp + (int64_t)z * (D + 2) * 128;
+          const float mz = __ldcg(pz + D * 128 + row);
+          if (mz == -INFINITY) continue;
+          const float wz = tc::ex2_approx(mz - mstar);
+          den += __ldcg(pz + (D + 1) * 128 + row) * wz;
+#pragma unroll
+          for (int c = 0; c < HD; ++c) acc[c] += __ldcg(pz + (half * HD + c) * 128 + row) * wz;
+        }
+        if (row < rows_valid) {
+          const float inv = 1.f / den;
+#pragma unroll
+          for (int c = 0; c < HD / 2; ++c)
+            reinterpret_cast<__nv_bfloat162*>(orow)[c] = __floats2bfloat162_rn(acc[2 * c] * inv, acc[2 * c + 1] * inv);
         }
       }
     }
@@ -409,7 +483,20 @@ int launch_attn_tc(State* st, const AttnArgs& a, cudaStream_t s) {
   p.so0 = a.so[0]; p.so1 = a.so[1]; p.so2 = a.so[2];
   p.out = a.out; p.tau_s = st->tau_s; p.tau_b = st->tau_b; p.status = st->status;
   p.nq = a.nq; p.Hq = st->Hq; p.Hkv = st->Hkv; p.G = st->G;
-  dim3 grid((a.nq + 127) / 128, st->B * st->Hq);
+  p.part = st->attnPart; p.part_cnt = st->attnCnt;
+  // key splits when there are few query tiles: up to half of the GPU (the folds of the block before
+  // run beside this kernel and are usually the longer chain), at least two key tiles per split
+  const int qtiles = (a.nq + 127) / 128;
+  const int ctas = qtiles * st->B * st->Hq;
+  int nsp = 1;
+  if (ctas <= kAttnSplitTiles) {
+    nsp = kAttnSplitTiles / ctas;
+    const int ntot_min = (int)((a.m + 127) / 128) + 1;
+    if (nsp > ntot_min / 2) nsp = ntot_min / 2;
+    if (nsp > kAttnMaxSplits) nsp = kAttnMaxSplits;
+    if (nsp < 1) nsp = 1;
+  }
+  dim3 grid(qtiles, st->B * st->Hq, nsp);
   const CUtensorMap* tm = reinterpret_cast<const CUtensorMap*>(st->tmaps);
   const int ks = (st->nfolds & 1) ? 6 : 1, vs = (st->nfolds & 1) ? 7 : 2;   // readout copy of the current version
   if (st->d == 128) {

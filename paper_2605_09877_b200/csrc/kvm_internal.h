@@ -12,6 +12,8 @@ namespace kvm {
 constexpr int kMaxBlock = 256;      // largest block C (one thread per overflow token in the fold)
 constexpr int kTopK = 8;            // routing filter keeps the K best approximate similarities per split
 constexpr int kMaxSplits = 32;      // routing filter / decode split count upper bound
+constexpr int kAttnSplitTiles = 74; // launches with at most this many (batch, head, query tile) CTAs are split along the keys
+constexpr int kAttnMaxSplits = 8;
 constexpr int kRowAlign = 128;      // state capacity is rounded up to the attention key tile
 
 // State of one layer: host bookkeeping + device buffers.  U = batch * n_kv_heads "units";
@@ -84,6 +86,9 @@ struct State {
   int nsplitRoute;               // splits the routing filter may use
   float* candV;                  // [U, nsplitRoute, Cmax, kTopK]
   int32_t* candI;
+  // ---- split-KV attention scratch (device) ----
+  float* attnPart;               // [kAttnSplitTiles][kAttnMaxSplits][d + 2][128]
+  int32_t* attnCnt;              // [kAttnSplitTiles] tickets
   // ---- decode scratch (device) ----
   int nsplitDec;
   float* decPart;                // [B*Hq, nsplitDec, d + 2]
