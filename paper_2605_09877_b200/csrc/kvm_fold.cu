@@ -289,6 +289,8 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
   __shared__ unsigned short s_ptok[kPairCap];
   __shared__ double s_pval[kPairCap];
   __shared__ int s_np, s_nmerge, s_nexh, s_last;
+  __shared__ int s_gmaxi[kMaxBlock], s_fill[kMaxBlock];
+  __shared__ float s_thr[kMaxBlock];
 
   // grid (R, U): CTA r of a unit refines the candidates of tokens [jlo, jhi); the CTA of the unit
   // that finishes last (a ticket, nobody waits) takes the decisions that need every token
@@ -316,63 +318,111 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
   if (tid < kMaxBlock) {
     s_app[tid] = 0; s_exh[tid] = 0; s_pcnt[tid] = 0; s_pstart[tid] = 0; s_pi[tid] = -1;
     s_best[tid] = -INFINITY; s_barg[tid] = -1; s_score[tid] = -INFINITY; s_creator[tid] = -1;
+    s_gmaxi[tid] = (int)0x80000000; s_fill[tid] = 0; s_thr[tid] = 0.f;
     if (tid < p.Cmax) p.segnew[tokBase + tid] = -1;
   }
   __syncthreads();
 
-  // ---- A1/A2: candidate pairs from the filter lists ----
-  if (jlo + tid < jhi) {
-    const int j = jlo + tid;
-    const float thr = p.thr_coeff * p.kbarNorm[tokBase + j] + 1e-5f;
-    const int64_t o0 = ((int64_t)u * p.nsplit * p.Cmax + j) * kTopK;
-    const int64_t ostep = (int64_t)p.Cmax * kTopK;
-    // a split keeps its candidates when its own maximum is within the window of the global one;
-    // sink rows (< S) only matter for the append score and are kept whenever rows are appended
-    float gmax = -INFINITY;
-#pragma unroll 4
-    for (int sp = 0; sp < p.nsplit; ++sp) gmax = fmaxf(gmax, p.candV[o0 + sp * ostep]);
-    const float gcut = gmax - thr;
-    bool exh = !(gmax > -INFINITY);
-    int cntc = 0;
-#pragma unroll 4
-    for (int sp = 0; sp < p.nsplit; ++sp) {
-      const float2 hd = *reinterpret_cast<const float2*>(p.candV + o0 + sp * ostep);
-      int i[kTopK];
-      load_cand_rows(p.candI, o0 + sp * ostep, i);
-      const bool keep = hd.x >= gcut;
-      if (hd.y > (float)kTopK && (keep || (n_a > 0 && sp == 0))) exh = true;   // list overflowed
-#pragma unroll
-      for (int k = 0; k < kTopK; ++k)
-        if (i[k] >= 0 && (i[k] < p.S ? n_a > 0 : keep)) ++cntc;
-    }
-    if (cntc > kPairPerTok) exh = true;
-    int start = 0;
-    if (!exh) {
-      start = atomicAdd(&s_np, cntc);
-      if (start + cntc > kPairCap) exh = true;
-    }
-    if (!exh) {
-      int w = start;
-      for (int sp = 0; sp < p.nsplit; ++sp) {
-        const bool keep = p.candV[o0 + sp * ostep] >= gcut;
-        int i[kTopK];
-        load_cand_rows(p.candI, o0 + sp * ostep, i);
-#pragma unroll
-        for (int k = 0; k < kTopK; ++k) {
-          if (i[k] >= 0 && (i[k] < p.S ? n_a > 0 : keep)) {
-            s_prow[w] = i[k];
-            s_ptok[w] = (unsigned short)j;
-            ++w;
-          }
-        }
-      }
-      s_pstart[j] = start;
-      s_pcnt[j] = cntc;
-    }
-    s_exh[j] = exh ? 1 : 0;
-    if (exh) atomicAdd(&s_nexh, 1);
+  // ---- A1/A2: candidate pairs from the filter lists.  The work items are (token of the slice, split),
+  //      consecutive threads taking consecutive tokens of one split, in three rounds: the maximum over
+  //      the splits per token; the number of pairs per token; the pairs themselves, into the token's
+  //      segment of the pair list (order inside a segment does not matter to what follows).
+  //      A split keeps its candidates when its own maximum is within the window of the global one;
+  //      sink rows (< S) only matter for the append score and are kept whenever rows are appended. ----
+  const int nslice = jhi - jlo;
+  const int nitems = nslice > 0 ? nslice * p.nsplit : 0;
+  const int64_t ostep = (int64_t)p.Cmax * kTopK;
+  const int64_t obase = (int64_t)u * p.nsplit * p.Cmax * kTopK;
+  for (int it = tid; it < nitems; it += kDecideThreads) {
+    const int sp = it / nslice, j = jlo + it % nslice;
+    const int vi = __float_as_int(p.candV[obase + sp * ostep + (int64_t)j * kTopK]);
+    atomicMax(&s_gmaxi[j], vi >= 0 ? vi : vi ^ 0x7fffffff);   // order-preserving integer image of the float
+    if (sp == 0) s_thr[j] = p.thr_coeff * p.kbarNorm[tokBase + j] + 1e-5f;
   }
   __syncthreads();
+  for (int it = tid; it < nitems; it += kDecideThreads) {
+    const int sp = it / nslice, j = jlo + it % nslice;
+    const int gi = s_gmaxi[j];
+    const float gmax = __int_as_float(gi >= 0 ? gi : gi ^ 0x7fffffff);
+    if (!(gmax > -INFINITY)) { s_exh[j] = 1; continue; }
+    const int64_t o = obase + sp * ostep + (int64_t)j * kTopK;
+    const float2 hd = *reinterpret_cast<const float2*>(p.candV + o);
+    int i[kTopK];
+    load_cand_rows(p.candI, o, i);
+    const bool keep = hd.x >= gmax - s_thr[j];
+    if (hd.y > (float)kTopK && (keep || (n_a > 0 && sp == 0))) s_exh[j] = 1;   // list overflowed
+    int c = 0;
+#pragma unroll
+    for (int k = 0; k < kTopK; ++k)
+      if (i[k] >= 0 && (i[k] < p.S ? n_a > 0 : keep)) ++c;
+    if (c > 0) atomicAdd(&s_pcnt[j], c);
+  }
+  __syncthreads();
+  if (warp == 0) {   // segment starts: exclusive prefix sum over the slice's tokens, eight per lane
+    int cnt[8], tot = 0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const int j = jlo + lane * 8 + k;
+      int c = 0;
+      if (j < jhi) {
+        c = s_pcnt[j];
+        if (c > kPairPerTok) { s_exh[j] = 1; }
+        if (s_exh[j]) c = 0;
+      }
+      cnt[k] = c;
+      tot += c;
+    }
+    int incl = tot;
+#pragma unroll
+    for (int o2 = 1; o2 < 32; o2 <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o2);
+      if (lane >= o2) incl += v;
+    }
+    int start = incl - tot;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const int j = jlo + lane * 8 + k;
+      if (j < jhi) {
+        if (start + cnt[k] > kPairCap) { s_exh[j] = 1; cnt[k] = 0; }   // the list is full: exact scan instead
+        s_pstart[j] = start;
+        s_pcnt[j] = cnt[k];
+        s_fill[j] = 0;
+      }
+      start += cnt[k];
+    }
+    if (lane == 31) s_np = min(start, kPairCap);
+  }
+  __syncthreads();
+  for (int it = tid; it < nitems; it += kDecideThreads) {
+    const int sp = it / nslice, j = jlo + it % nslice;
+    if (s_exh[j]) continue;
+    const int gi = s_gmaxi[j];
+    const float gmax = __int_as_float(gi >= 0 ? gi : gi ^ 0x7fffffff);
+    const int64_t o = obase + sp * ostep + (int64_t)j * kTopK;
+    const bool keep = p.candV[o] >= gmax - s_thr[j];
+    int i[kTopK];
+    load_cand_rows(p.candI, o, i);
+    int c = 0;
+#pragma unroll
+    for (int k = 0; k < kTopK; ++k)
+      if (i[k] >= 0 && (i[k] < p.S ? n_a > 0 : keep)) ++c;
+    if (c == 0) continue;
+    int w = s_pstart[j] + atomicAdd(&s_fill[j], c);
+#pragma unroll
+    for (int k = 0; k < kTopK; ++k) {
+      if (i[k] >= 0 && (i[k] < p.S ? n_a > 0 : keep)) {
+        s_prow[w] = i[k];
+        s_ptok[w] = (unsigned short)j;
+        ++w;
+      }
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int ne = 0;
+    for (int j = jlo; j < jhi; ++j) ne += s_exh[j];
+    s_nexh += ne;
+  }
   // ---- A3: exact fp64 similarity of every candidate pair, one warp per pair, eight in flight
   //      (the loads of a pair hang on one another: pair list -> rows -> statistics) ----
   const int np = min(s_np, kPairCap);
