@@ -4,21 +4,24 @@
 //
 // One CTA owns a 128-query tile of one (batch, query head) and walks the key tiles (128 keys:
 // first the state's readout cache, then the window) with these warp roles:
-//   warp 0      TMA producer: Q once, then K/V tiles into a 2-stage shared-memory ring
-//               (cp.async.bulk.tensor, 128-byte swizzle, mbarrier complete_tx)
-//   warp 1      QK^T issuer: S = Q K^T into a double-buffered TMEM accumulator
-//   warp 2      PV issuer: O_h += P_h V_h into two more TMEM accumulators
-//               (tcgen05.mma kind::f16, fp32 accumulate; one elected thread each - issuing an MMA
-//               takes about as long as executing it, so one thread cannot keep the pipe full and
-//               also wait on barriers)
+//   warp 0      TMA producer: Q once, then K and V tiles into 3-stage shared-memory rings
+//               (cp.async.bulk.tensor, 128-byte swizzle, mbarrier complete_tx), keys two tiles ahead
+//   warp 1      QK^T issuer: S = Q K^T (both operands from shared memory) into a double-buffered
+//               TMEM accumulator
+//   warp 2      PV issuer: O_h += P_h V_h into two more TMEM accumulators; P is read from TMEM
+//               (tcgen05.mma with the A operand in tensor memory), V from shared memory
+//               (kind::f16, fp32 accumulate; one elected thread each - issuing an MMA takes about as
+//               long as executing it, so one thread cannot keep the pipe full and also wait on barriers)
 //   warps 4-11  softmax, two warpgroups: warpgroup h owns keys [64h, 64h+64) of every tile and each of
 //               its threads one query row (tcgen05.ld 32x32b); it applies the region temperature and
-//               masks, keeps a running max / sum of its own in registers, and its half of P (fp16,
-//               double-buffered swizzled shared memory) feeds PV products that accumulate into an O
-//               accumulator of its own, rescaled in TMEM only when its max grew by more than 2^8.
-//               The two partial results (O_h, m_h, l_h) are merged in the epilogue like split-K
-//               partials, normalised and stored as bf16 rows.  Splitting by columns halves the
-//               exponentials and conversions per thread, which is what bounds a tile's turnaround.
+//               masks, keeps a running max / sum of its own in registers, and writes its half of P as
+//               packed fp16 back into tensor memory, over the columns of S it has just read
+//               (tcgen05.st) - P never passes through shared memory.  Each half feeds PV products that
+//               accumulate into an O accumulator of its own, rescaled in TMEM only when its max grew
+//               by more than 2^8.  The two partial results (O_h, m_h, l_h) are merged in the epilogue
+//               like split-K partials, normalised and stored as bf16 rows.
+// With few query tiles per launch the key tiles are also split over gridDim.z CTAs whose partial
+// results are merged by the CTA that finishes last.
 // Every mbarrier wait is bounded; on expiry the CTA records KVM_ERR_TIMEOUT and tears down.
 #include "kvm_internal.h"
 #include "tc_common.cuh"
@@ -38,16 +41,14 @@ struct AttnTcParams {
 
 template <int D>
 struct AttnTcCfg {
-  static constexpr int BM = 128, BN = 128, NS = 2;
+  static constexpr int BM = 128, BN = 128, NS = 3;
   static constexpr int NKB = D / 64;                 // 64-channel boxes per tile row
   static constexpr int BOX_BYTES = 128 * 128;        // 128 rows x 64 fp16
   static constexpr int TILE_BYTES = NKB * BOX_BYTES; // Q, K or V tile
-  static constexpr int P_BYTES = 2 * BOX_BYTES;      // 128 rows x 128 keys fp16
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_K = OFF_Q + TILE_BYTES;
   static constexpr int OFF_V = OFF_K + NS * TILE_BYTES;
-  static constexpr int OFF_P = OFF_V + NS * TILE_BYTES;
-  static constexpr int OFF_BAR = OFF_P + 2 * P_BYTES;  // P is double-buffered: softmax of tile j+1 overlaps PV of tile j
+  static constexpr int OFF_BAR = OFF_V + NS * TILE_BYTES;
   // + alignment slack; never less than half an SM so that one CTA (and one 512-column TMEM
   // allocation) is resident per SM
   static constexpr int SMEM_BYTES = (OFF_BAR + 256 + 1024) > 120 * 1024 ? (OFF_BAR + 256 + 1024) : 120 * 1024;
@@ -55,9 +56,9 @@ struct AttnTcCfg {
   static constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_O0 = 256, COL_O1 = 384;
 };
 
-// SFULL[i] (QK^T of a tile done) also tells the producer that K stage i is free again, PVDONE[i]
-// (PV of a tile done) that V stage i is: stage and accumulator parity coincide because NS == 2.
-enum { BAR_QFULL = 0, BAR_KFULL = 1, BAR_VFULL = 3, BAR_SFULL = 5, BAR_PFULL = 7, BAR_PVDONE = 9, BAR_COUNT = 11 };
+// K / V stages cycle with period NS = 3, the S / P accumulators with period 2.
+enum { BAR_QFULL = 0, BAR_KFULL = 1, BAR_VFULL = 4, BAR_KFREE = 7, BAR_VFREE = 10, BAR_SFULL = 13, BAR_PFULL = 15,
+       BAR_PVDONE = 17, BAR_COUNT = 19 };
 
 template <int D>
 __global__ void __launch_bounds__(384, 1)
@@ -70,7 +71,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   uint8_t* sQ = base + Cfg::OFF_Q;
   uint8_t* sK = base + Cfg::OFF_K;
   uint8_t* sV = base + Cfg::OFF_V;
-  uint8_t* sP = base + Cfg::OFF_P;
   uint64_t* bars = reinterpret_cast<uint64_t*>(base + Cfg::OFF_BAR);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + BAR_COUNT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -98,6 +98,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     for (int s = 0; s < Cfg::NS; ++s) {
       tc::mbar_init(&bars[BAR_KFULL + s], 1);
       tc::mbar_init(&bars[BAR_VFULL + s], 1);
+      tc::mbar_init(&bars[BAR_KFREE + s], 1);
+      tc::mbar_init(&bars[BAR_VFREE + s], 1);
     }
     tc::mbar_init(&bars[BAR_SFULL + 0], 1);
     tc::mbar_init(&bars[BAR_SFULL + 1], 1);
@@ -132,32 +134,30 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       tc::mbar_expect_tx(&bars[BAR_QFULL], Cfg::TILE_BYTES);
       for (int kb = 0; kb < Cfg::NKB; ++kb)
         tc::tma_load_3d(sQ + kb * Cfg::BOX_BYTES, &mapQ, &bars[BAR_QFULL], kb * 64, (int)(p.q_row0 + qt * 128), bh);
-      // A K stage is released as soon as its QK^T product has completed, a V stage only after its
-      // PV product, so K of tile j+1 is requested before V of tile j: the keys of the next tile are
-      // in flight while the softmax of the current one runs.
-      auto load_k = [&](int j) -> bool {
+      // Three stages each: keys run two tiles ahead of the product that needs them, values one.
+      // A K stage is released as soon as its QK^T product has completed, a V stage after its PV product.
+      auto load_kv = [&](int j, bool keys) -> bool {
         const int s = j % Cfg::NS;
-        if (j >= Cfg::NS && !tc::mbar_wait(&bars[BAR_SFULL + s], ((j / Cfg::NS) - 1) & 1)) return false;
+        if (j >= Cfg::NS && !tc::mbar_wait(&bars[(keys ? BAR_KFREE : BAR_VFREE) + s], ((j / Cfg::NS) - 1) & 1)) return false;
         const int gj = jbase + j;
         const bool st = gj < nst;
         const int row = st ? gj * 128 : (int)(p.win_row0 + (int64_t)(gj - nst) * 128);
-        tc::mbar_expect_tx(&bars[BAR_KFULL + s], Cfg::TILE_BYTES);
+        uint64_t* full = &bars[(keys ? BAR_KFULL : BAR_VFULL) + s];
+        uint8_t* dst = (keys ? sK : sV) + s * Cfg::TILE_BYTES;
+        const CUtensorMap* map = keys ? (st ? &mapKs : &mapKw) : (st ? &mapVs : &mapVw);
+        tc::mbar_expect_tx(full, Cfg::TILE_BYTES);
         for (int kb = 0; kb < Cfg::NKB; ++kb)
-          tc::tma_load_3d(sK + s * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, st ? &mapKs : &mapKw, &bars[BAR_KFULL + s], kb * 64, row, u);
+          tc::tma_load_3d(dst + kb * Cfg::BOX_BYTES, map, full, kb * 64, row, u);
         return true;
       };
-      bool okp = ntiles == 0 || load_k(0);
+      bool okp = true;
+      if (ntiles > 0) okp = load_kv(0, true);
+      if (okp && ntiles > 1) okp = load_kv(1, true);
+      if (okp && ntiles > 0) okp = load_kv(0, false);
       for (int j = 0; j < ntiles && okp; ++j) {
-        const int s = j % Cfg::NS;
         if (*abort_flag) break;
-        if (j + 1 < ntiles && !load_k(j + 1)) { okp = false; break; }
-        if (j >= Cfg::NS && !tc::mbar_wait(&bars[BAR_PVDONE + s], ((j / Cfg::NS) - 1) & 1)) { okp = false; break; }
-        const int gj = jbase + j;
-        const bool st = gj < nst;
-        const int row = st ? gj * 128 : (int)(p.win_row0 + (int64_t)(gj - nst) * 128);
-        tc::mbar_expect_tx(&bars[BAR_VFULL + s], Cfg::TILE_BYTES);
-        for (int kb = 0; kb < Cfg::NKB; ++kb)
-          tc::tma_load_3d(sV + s * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, st ? &mapVs : &mapVw, &bars[BAR_VFULL + s], kb * 64, row, u);
+        if (j + 2 < ntiles && !load_kv(j + 2, true)) { okp = false; break; }
+        if (j + 1 < ntiles && !load_kv(j + 1, false)) { okp = false; break; }
       }
       if (!okp) { atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; }
     }
@@ -174,8 +174,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         for (int j = 0; j < ntiles; ++j) {
           const int s = j % Cfg::NS;
           if (*abort_flag) { dead = true; break; }
-          // accumulator S[j & 1] is free once both softmax halves have read tile j-2 out of it
-          if (j >= 2 && !tc::mbar_wait(&bars[BAR_PFULL + (j & 1)], ((j >> 1) - 1) & 1)) { dead = true; break; }
+          // accumulator S[j & 1] also holds P of tile j-2 (fp16, written over the columns the softmax
+          // has read): it is free once the PV product of tile j-2 has consumed it
+          if (j >= 2 && !tc::mbar_wait(&bars[BAR_PVDONE + (j & 1)], ((j >> 1) - 1) & 1)) { dead = true; break; }
           if (!tc::mbar_wait(&bars[BAR_KFULL + s], (j / Cfg::NS) & 1)) { dead = true; break; }
           tc::tc_fence_after();
           const uint32_t dS = tmem + ((j & 1) ? Cfg::COL_S1 : Cfg::COL_S0);
@@ -186,6 +187,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
                            tc::smem_desc_sw128(aK + s * Cfg::TILE_BYTES + off, 16, 1024), IDESC_QK, ks > 0);
           }
           tc::mma_commit(&bars[BAR_SFULL + (j & 1)]);
+          tc::mma_commit(&bars[BAR_KFREE + s]);
         }
       } while (false);
       if (dead) { atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; }
@@ -194,7 +196,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     // ------------------------------ PV issuer ------------------------------
     if (lane == 0) {
       constexpr uint32_t IDESC_PV = tc::idesc_f16(128, D, true);
-      const uint32_t aV = tc::smem_u32(sV), aP = tc::smem_u32(sP);
+      const uint32_t aV = tc::smem_u32(sV);
       bool dead = false;
       for (int j = 0; j < ntiles; ++j) {
         const int s = j % Cfg::NS;
@@ -204,15 +206,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         tc::tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
-          // keys 0..63 of the tile accumulate into O0, keys 64..127 into O1
-          const uint32_t dO = tmem + (kk < 4 ? Cfg::COL_O0 : Cfg::COL_O1);
-          const uint32_t offP = (j & 1) * Cfg::P_BYTES + (kk / 4) * Cfg::BOX_BYTES + (kk % 4) * 32;
+          // keys 0..63 of the tile accumulate into O0, keys 64..127 into O1.  P comes from TMEM (A
+          // operand, one row per lane, two fp16 per column): half h of tile j sits in the first 32
+          // columns of that half's share of S[j & 1]; a k-step of 16 keys is 8 columns.
+          const int h = kk >> 2;
+          const uint32_t dO = tmem + (h ? Cfg::COL_O1 : Cfg::COL_O0);
+          const uint32_t aP = tmem + ((j & 1) ? Cfg::COL_S1 : Cfg::COL_S0) + 64 * h + 8 * (kk & 3);
           const uint32_t offV = kk * 2048;   // 16 key rows x 128 B
-          tc::mma_f16_ss(dO, tc::smem_desc_sw128(aP + offP, 16, 1024),
-                         tc::smem_desc_sw128(aV + s * Cfg::TILE_BYTES + offV, Cfg::BOX_BYTES, 1024), IDESC_PV,
+          tc::mma_f16_ts(dO, aP, tc::smem_desc_sw128(aV + s * Cfg::TILE_BYTES + offV, Cfg::BOX_BYTES, 1024), IDESC_PV,
                          (j > 0 || (kk & 3) > 0) ? 1u : 0u);
         }
         tc::mma_commit(&bars[BAR_PVDONE + (j & 1)]);
+        tc::mma_commit(&bars[BAR_VFREE + s]);
       }
       if (dead) { atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; }
     }
@@ -261,16 +266,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         if (st) nvis = p.m - (int64_t)gj * 128;
         else nvis = t_row - (p.b + (int64_t)(gj - nst) * 128) + 1;
         const int vis = (int)max((int64_t)0, min((int64_t)64, nvis - half * 64));
-        float mx = -INFINITY;
-        if (vis == 64) {
+        if (vis != 64) {
 #pragma unroll
-          for (int c = 0; c < 64; ++c) mx = fmaxf(mx, x[c]);
-        } else {
+          for (int c = 0; c < 64; ++c) x[c] = (c < vis) ? x[c] : -INFINITY;
+        }
+        float mx;
+        {   // four chains: a single chain of 64 dependent maxima is latency bound
+          float m4[4] = {x[0], x[1], x[2], x[3]};
 #pragma unroll
-          for (int c = 0; c < 64; ++c) {
-            x[c] = (c < vis) ? x[c] : -INFINITY;
-            mx = fmaxf(mx, x[c]);
-          }
+          for (int c = 4; c < 64; ++c) m4[c & 3] = fmaxf(m4[c & 3], x[c]);
+          mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
         }
         const float mnew = fmaxf(m_run, mx * sc);
         if (j == 0) {
@@ -297,29 +302,24 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
             tc::tmem_wait_st();
           }
         }
-        if (j >= 2) {   // the PV product that read this P buffer two tiles ago has finished
-          KVM_WAIT(&bars[BAR_PVDONE + (j & 1)], ((j >> 1) - 1) & 1);
-        }
         const float neg_m = (m_run == -INFINITY) ? 0.f : -m_run;
-        float lsum = 0.f;
-        // P row -> shared memory, K-major, 128-byte swizzle: 16-byte chunk ch of row r lives at
-        // r*128 + ((ch ^ (r & 7)) * 16) inside its 64-key box; box `half` is this thread's.
-        uint8_t* prow = sP + (j & 1) * Cfg::P_BYTES + half * Cfg::BOX_BYTES + row * 128;
+        float lsum = 0.f, lsum2 = 0.f;
+        // P row -> tensor memory, as the A operand of the PV product: this thread's lane, two fp16
+        // per column, over the first 32 of the 64 columns of S that it has just read out (the QK^T
+        // issuer does not touch this accumulator again before the PV product has consumed it)
+        uint32_t w[32];
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-          uint32_t w[4];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const float p0 = tc::ex2_approx(fmaf(x[ch * 8 + 2 * i], sc, neg_m));
-            const float p1 = tc::ex2_approx(fmaf(x[ch * 8 + 2 * i + 1], sc, neg_m));
-            lsum += p0 + p1;
-            const __half2 h = __floats2half2_rn(p0, p1);
-            w[i] = *reinterpret_cast<const uint32_t*>(&h);
-          }
-          *reinterpret_cast<uint4*>(prow + ((ch ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        for (int i = 0; i < 32; ++i) {
+          const float p0 = tc::ex2_approx(fmaf(x[2 * i], sc, neg_m));
+          const float p1 = tc::ex2_approx(fmaf(x[2 * i + 1], sc, neg_m));
+          if (i & 1) lsum += p0 + p1; else lsum2 += p0 + p1;
+          const __half2 h = __floats2half2_rn(p0, p1);
+          w[i] = *reinterpret_cast<const uint32_t*>(&h);
         }
+        lsum += lsum2;
+        tc::tmem_st32(tmem + lane_base + ((j & 1) ? Cfg::COL_S1 : Cfg::COL_S0) + half * 64, w);
+        tc::tmem_wait_st();
         l_run += lsum;
-        tc::fence_proxy_async();
         tc::tc_fence_before();
         __syncwarp();
         if (lane == 0) tc::mbar_arrive(&bars[BAR_PFULL + (j & 1)]);
