@@ -4,22 +4,24 @@
 //
 // One CTA owns a 128-query tile of one (batch, query head) and walks the key tiles (128 keys:
 // first the state's readout cache, then the window) with these warp roles:
-//   warp 0      TMA producer: Q once, then K and V tiles into 3-stage shared-memory rings
-//               (cp.async.bulk.tensor, 128-byte swizzle, mbarrier complete_tx), keys two tiles ahead
-//   warp 1      QK^T issuer: S = Q K^T (both operands from shared memory) into a double-buffered
-//               TMEM accumulator
-//   warp 2      PV issuer: O_h += P_h V_h into two more TMEM accumulators; P is read from TMEM
-//               (tcgen05.mma with the A operand in tensor memory), V from shared memory
+//   warp 0      TMA producer: Q once, then K tiles into a 3-stage and V tiles into a 2-stage
+//               shared-memory ring (cp.async.bulk.tensor, 128-byte swizzle, mbarrier complete_tx),
+//               keys two tiles ahead, values one
+//   warp 1      QK^T issuer: S = Q K^T (both operands from shared memory) into one of three TMEM
+//               accumulators
+//   warp 2      PV issuer: O += P V into a fourth TMEM accumulator; P is read from TMEM (tcgen05.mma
+//               with the A operand in tensor memory), V from shared memory
 //               (kind::f16, fp32 accumulate; one elected thread each - issuing an MMA takes about as
 //               long as executing it, so one thread cannot keep the pipe full and also wait on barriers)
 //   warps 4-11  softmax, two warpgroups: warpgroup h owns keys [64h, 64h+64) of every tile and each of
 //               its threads one query row (tcgen05.ld 32x32b); it applies the region temperature and
-//               masks, keeps a running max / sum of its own in registers, and writes its half of P as
-//               packed fp16 back into tensor memory, over the columns of S it has just read
-//               (tcgen05.st) - P never passes through shared memory.  Each half feeds PV products that
-//               accumulate into an O accumulator of its own, rescaled in TMEM only when its max grew
-//               by more than 2^8.  The two partial results (O_h, m_h, l_h) are merged in the epilogue
-//               like split-K partials, normalised and stored as bf16 rows.
+//               masks, agrees with the thread that holds the other half of the row on the tile's row
+//               maximum (shared memory + mbarrier), keeps the running max and the sum of its own
+//               columns in registers, and writes its half of P as packed fp16 back into tensor memory,
+//               over the columns of S it has just read (tcgen05.st) - P never passes through shared
+//               memory, and the S accumulator is handed back to the QK^T issuer when the PV product
+//               has consumed it.  O is rescaled in TMEM only when the max grew by more than 2^8
+//               (each half rescales, and at the end normalises and stores, its share of the channels).
 // With few query tiles per launch the key tiles are also split over gridDim.z CTAs whose partial
 // results are merged by the CTA that finishes last.
 // Every mbarrier wait is bounded; on expiry the CTA records KVM_ERR_TIMEOUT and tears down.
@@ -41,24 +43,25 @@ struct AttnTcParams {
 
 template <int D>
 struct AttnTcCfg {
-  static constexpr int BM = 128, BN = 128, NS = 3;
+  static constexpr int BM = 128, BN = 128, NS = 3, NSV = 2, NACC = 3;   // K stages, V stages, S/P accumulators
   static constexpr int NKB = D / 64;                 // 64-channel boxes per tile row
   static constexpr int BOX_BYTES = 128 * 128;        // 128 rows x 64 fp16
   static constexpr int TILE_BYTES = NKB * BOX_BYTES; // Q, K or V tile
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_K = OFF_Q + TILE_BYTES;
   static constexpr int OFF_V = OFF_K + NS * TILE_BYTES;
-  static constexpr int OFF_BAR = OFF_V + NS * TILE_BYTES;
+  static constexpr int OFF_XM = OFF_V + NSV * TILE_BYTES;   // float [2][2][128]: row maxima exchanged between the column halves
+  static constexpr int OFF_BAR = OFF_XM + 2 * 2 * 128 * 4;
   // + alignment slack; never less than half an SM so that one CTA (and one 512-column TMEM
   // allocation) is resident per SM
   static constexpr int SMEM_BYTES = (OFF_BAR + 256 + 1024) > 120 * 1024 ? (OFF_BAR + 256 + 1024) : 120 * 1024;
   static constexpr uint32_t TMEM_COLS = 512;
-  static constexpr uint32_t COL_S0 = 0, COL_S1 = 128, COL_O0 = 256, COL_O1 = 384;
+  static constexpr uint32_t COL_S = 0, COL_O = 384;   // S/P accumulator i at COL_S + 128 i
 };
 
-// K / V stages cycle with period NS = 3, the S / P accumulators with period 2.
-enum { BAR_QFULL = 0, BAR_KFULL = 1, BAR_VFULL = 4, BAR_KFREE = 7, BAR_VFREE = 10, BAR_SFULL = 13, BAR_PFULL = 15,
-       BAR_PVDONE = 17, BAR_COUNT = 19 };
+// K stages and the S / P accumulators cycle with period 3, V stages with period 2.
+enum { BAR_QFULL = 0, BAR_KFULL = 1, BAR_KFREE = 4, BAR_VFULL = 7, BAR_VFREE = 9, BAR_SFULL = 11, BAR_PFULL = 14,
+       BAR_PVDONE = 17, BAR_XM = 20, BAR_COUNT = 22 };
 
 template <int D>
 __global__ void __launch_bounds__(384, 1)
@@ -95,18 +98,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 
   if (tid == 0) {
     tc::mbar_init(&bars[BAR_QFULL], 1);
-    for (int s = 0; s < Cfg::NS; ++s) {
+    for (int s = 0; s < 3; ++s) {
       tc::mbar_init(&bars[BAR_KFULL + s], 1);
-      tc::mbar_init(&bars[BAR_VFULL + s], 1);
       tc::mbar_init(&bars[BAR_KFREE + s], 1);
-      tc::mbar_init(&bars[BAR_VFREE + s], 1);
+      tc::mbar_init(&bars[BAR_SFULL + s], 1);
+      tc::mbar_init(&bars[BAR_PFULL + s], 8);
+      tc::mbar_init(&bars[BAR_PVDONE + s], 1);
     }
-    tc::mbar_init(&bars[BAR_SFULL + 0], 1);
-    tc::mbar_init(&bars[BAR_SFULL + 1], 1);
-    tc::mbar_init(&bars[BAR_PFULL + 0], 8);
-    tc::mbar_init(&bars[BAR_PFULL + 1], 8);
-    tc::mbar_init(&bars[BAR_PVDONE + 0], 1);
-    tc::mbar_init(&bars[BAR_PVDONE + 1], 1);
+    for (int s = 0; s < Cfg::NSV; ++s) {
+      tc::mbar_init(&bars[BAR_VFULL + s], 1);
+      tc::mbar_init(&bars[BAR_VFREE + s], 1);
+      tc::mbar_init(&bars[BAR_XM + s], 8);
+    }
     *abort_flag = 0;
     tc::fence_barrier_init();
   }
@@ -134,11 +137,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       tc::mbar_expect_tx(&bars[BAR_QFULL], Cfg::TILE_BYTES);
       for (int kb = 0; kb < Cfg::NKB; ++kb)
         tc::tma_load_3d(sQ + kb * Cfg::BOX_BYTES, &mapQ, &bars[BAR_QFULL], kb * 64, (int)(p.q_row0 + qt * 128), bh);
-      // Three stages each: keys run two tiles ahead of the product that needs them, values one.
-      // A K stage is released as soon as its QK^T product has completed, a V stage after its PV product.
+      // Three key stages, two value stages: keys run two tiles ahead of the product that needs them,
+      // values one.  A K stage is released as soon as its QK^T product has completed, a V stage after
+      // its PV product.
       auto load_kv = [&](int j, bool keys) -> bool {
-        const int s = j % Cfg::NS;
-        if (j >= Cfg::NS && !tc::mbar_wait(&bars[(keys ? BAR_KFREE : BAR_VFREE) + s], ((j / Cfg::NS) - 1) & 1)) return false;
+        const int ns = keys ? Cfg::NS : Cfg::NSV;
+        const int s = j % ns;
+        if (j >= ns && !tc::mbar_wait(&bars[(keys ? BAR_KFREE : BAR_VFREE) + s], ((j / ns) - 1) & 1)) return false;
         const int gj = jbase + j;
         const bool st = gj < nst;
         const int row = st ? gj * 128 : (int)(p.win_row0 + (int64_t)(gj - nst) * 128);
@@ -174,19 +179,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         for (int j = 0; j < ntiles; ++j) {
           const int s = j % Cfg::NS;
           if (*abort_flag) { dead = true; break; }
-          // accumulator S[j & 1] also holds P of tile j-2 (fp16, written over the columns the softmax
-          // has read): it is free once the PV product of tile j-2 has consumed it
-          if (j >= 2 && !tc::mbar_wait(&bars[BAR_PVDONE + (j & 1)], ((j >> 1) - 1) & 1)) { dead = true; break; }
+          // accumulator j % 3 also holds P of tile j-3 (fp16, written over the columns the softmax
+          // has read): it is free once the PV product of tile j-3 has consumed it
+          const int acc = j % Cfg::NACC;
+          if (j >= Cfg::NACC && !tc::mbar_wait(&bars[BAR_PVDONE + acc], ((j / Cfg::NACC) - 1) & 1)) { dead = true; break; }
           if (!tc::mbar_wait(&bars[BAR_KFULL + s], (j / Cfg::NS) & 1)) { dead = true; break; }
           tc::tc_fence_after();
-          const uint32_t dS = tmem + ((j & 1) ? Cfg::COL_S1 : Cfg::COL_S0);
+          const uint32_t dS = tmem + Cfg::COL_S + 128 * acc;
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks) {
             const uint32_t off = (ks / 4) * Cfg::BOX_BYTES + (ks % 4) * 32;
             tc::mma_f16_ss(dS, tc::smem_desc_sw128(aQ + off, 16, 1024),
                            tc::smem_desc_sw128(aK + s * Cfg::TILE_BYTES + off, 16, 1024), IDESC_QK, ks > 0);
           }
-          tc::mma_commit(&bars[BAR_SFULL + (j & 1)]);
+          tc::mma_commit(&bars[BAR_SFULL + acc]);
           tc::mma_commit(&bars[BAR_KFREE + s]);
         }
       } while (false);
@@ -199,24 +205,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
       const uint32_t aV = tc::smem_u32(sV);
       bool dead = false;
       for (int j = 0; j < ntiles; ++j) {
-        const int s = j % Cfg::NS;
+        const int s = j % Cfg::NSV, acc = j % Cfg::NACC;
         if (*abort_flag) { dead = true; break; }
-        if (!tc::mbar_wait(&bars[BAR_VFULL + s], (j / Cfg::NS) & 1)) { dead = true; break; }
-        if (!tc::mbar_wait(&bars[BAR_PFULL + (j & 1)], (j >> 1) & 1)) { dead = true; break; }
+        if (!tc::mbar_wait(&bars[BAR_VFULL + s], (j / Cfg::NSV) & 1)) { dead = true; break; }
+        if (!tc::mbar_wait(&bars[BAR_PFULL + acc], (j / Cfg::NACC) & 1)) { dead = true; break; }
         tc::tc_fence_after();
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
-          // keys 0..63 of the tile accumulate into O0, keys 64..127 into O1.  P comes from TMEM (A
-          // operand, one row per lane, two fp16 per column): half h of tile j sits in the first 32
-          // columns of that half's share of S[j & 1]; a k-step of 16 keys is 8 columns.
-          const int h = kk >> 2;
-          const uint32_t dO = tmem + (h ? Cfg::COL_O1 : Cfg::COL_O0);
-          const uint32_t aP = tmem + ((j & 1) ? Cfg::COL_S1 : Cfg::COL_S0) + 64 * h + 8 * (kk & 3);
+          // P comes from TMEM (A operand, one row per lane, two fp16 per column): the column half h
+          // of tile j sits in the first 32 columns of that half's share of its S accumulator; a
+          // k-step of 16 keys is 8 columns.
+          const uint32_t aP = tmem + Cfg::COL_S + 128 * acc + 64 * (kk >> 2) + 8 * (kk & 3);
           const uint32_t offV = kk * 2048;   // 16 key rows x 128 B
-          tc::mma_f16_ts(dO, aP, tc::smem_desc_sw128(aV + s * Cfg::TILE_BYTES + offV, Cfg::BOX_BYTES, 1024), IDESC_PV,
-                         (j > 0 || (kk & 3) > 0) ? 1u : 0u);
+          tc::mma_f16_ts(tmem + Cfg::COL_O, aP, tc::smem_desc_sw128(aV + s * Cfg::TILE_BYTES + offV, Cfg::BOX_BYTES, 1024),
+                         IDESC_PV, (j > 0 || kk > 0) ? 1u : 0u);
         }
-        tc::mma_commit(&bars[BAR_PVDONE + (j & 1)]);
+        tc::mma_commit(&bars[BAR_PVDONE + acc]);
         tc::mma_commit(&bars[BAR_VFREE + s]);
       }
       if (dead) { atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; }
@@ -226,14 +230,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   } else {
     // ------------------------------ softmax / epilogue ------------------------------
     // Two warpgroups split every key tile by columns: half 0 owns keys 0..63 of the tile, half 1
-    // keys 64..127.  Each thread keeps its own running max / sum for (row, half) and its half's
-    // products accumulate into an O accumulator of their own, so the two halves never exchange
-    // anything inside the tile loop; they are merged like two split-K partial results at the end.
+    // keys 64..127, one thread per (row, half).  The two threads of a row agree on the row maximum
+    // of each tile through shared memory (an mbarrier per tile parity, so the wait is bounded), keep
+    // the same running maximum, and each keeps the sum of its own columns; all PV products go into
+    // one O accumulator, of which each half rescales and finally stores its share of the channels.
     const int half = (warp - 4) >> 2;                 // which 64 columns of every tile
     const int quarter = warp & 3;                     // TMEM lane quarter this warp may access
     const int row = quarter * 32 + lane;              // query row inside the tile
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-    const uint32_t col_o = half ? Cfg::COL_O1 : Cfg::COL_O0;
+    constexpr int HD = D / 2;
+    const uint32_t to_mine = tmem + lane_base + Cfg::COL_O + half * HD;   // this thread's share of O
+    float* xm = reinterpret_cast<float*>(base + Cfg::OFF_XM);             // [parity][half][row]
     const int64_t t_row = t_first + row;
     const float kLog2e = 1.4426950408889634f;
     const float sc_s = p.tau_s[hq] * rsqrtf((float)D) * kLog2e;
@@ -243,11 +250,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     for (int j = 0; j < ntiles && ok; ++j) {
       do {
         ok = false;
-        KVM_WAIT(&bars[BAR_SFULL + (j & 1)], (j >> 1) & 1);
+        const int acc = j % Cfg::NACC;
+        KVM_WAIT(&bars[BAR_SFULL + acc], (j / Cfg::NACC) & 1);
         tc::tc_fence_after();
+        const uint32_t ts = tmem + lane_base + Cfg::COL_S + 128 * acc + half * 64;
         float x[64];
         {
-          const uint32_t ts = tmem + lane_base + ((j & 1) ? Cfg::COL_S1 : Cfg::COL_S0) + half * 64;
 #pragma unroll
           for (int c = 0; c < 2; ++c) {
             uint32_t r[32];
@@ -277,27 +285,32 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           for (int c = 4; c < 64; ++c) m4[c & 3] = fmaxf(m4[c & 3], x[c]);
           mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
         }
+        // the other half's maximum of this row
+        xm[((j & 1) * 2 + half) * 128 + row] = mx;
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(&bars[BAR_XM + (j & 1)]);
+        KVM_WAIT(&bars[BAR_XM + (j & 1)], (j >> 1) & 1);
+        mx = fmaxf(mx, xm[((j & 1) * 2 + (1 - half)) * 128 + row]);
         const float mnew = fmaxf(m_run, mx * sc);
         if (j == 0) {
           m_run = mnew;
         } else {
           const bool need = mnew > m_run + 8.0f;
-          if (__any_sync(0xffffffffu, need)) {
+          if (__any_sync(0xffffffffu, need)) {   // the same decision in both warps that share these rows
             // all earlier PV products must have landed before O is touched (commits complete in order)
-            KVM_WAIT(&bars[BAR_PVDONE + ((j - 1) & 1)], ((j - 1) >> 1) & 1);
+            KVM_WAIT(&bars[BAR_PVDONE + (j - 1) % Cfg::NACC], ((j - 1) / Cfg::NACC) & 1);
             tc::tc_fence_after();
             const float corr = (m_run == -INFINITY) ? 0.f : tc::ex2_approx(m_run - mnew);
             l_run *= corr;
             m_run = mnew;
-            const uint32_t to = tmem + lane_base + col_o;
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
+            for (int c = 0; c < HD / 32; ++c) {
               uint32_t r[32];
-              tc::tmem_ld32(to + c * 32, r);
+              tc::tmem_ld32(to_mine + c * 32, r);
               tc::tmem_wait_ld();
 #pragma unroll
               for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
-              tc::tmem_st32(to + c * 32, r);
+              tc::tmem_st32(to_mine + c * 32, r);
             }
             tc::tmem_wait_st();
           }
@@ -317,98 +330,68 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           w[i] = *reinterpret_cast<const uint32_t*>(&h);
         }
         lsum += lsum2;
-        tc::tmem_st32(tmem + lane_base + ((j & 1) ? Cfg::COL_S1 : Cfg::COL_S0) + half * 64, w);
+        tc::tmem_st32(ts, w);
         tc::tmem_wait_st();
         l_run += lsum;
         tc::tc_fence_before();
         __syncwarp();
-        if (lane == 0) tc::mbar_arrive(&bars[BAR_PFULL + (j & 1)]);
+        if (lane == 0) tc::mbar_arrive(&bars[BAR_PFULL + acc]);
         ok = true;
       } while (false);
     }
-    // Epilogue: merge the two halves.  out = (O0 w0 + O1 w1) / (l0 w0 + l1 w1), w_h = 2^(m_h - max(m0, m1)).
-    // Half h stores channels [h D/2, (h+1) D/2): it hands the other half its accumulator's columns
-    // of the other channel range through shared memory (column-major, one row per thread: no bank
-    // conflicts), laid over the K stages, which nothing reads any more once the last PV product is done.
-    constexpr int HD = D / 2;
-    float* xch = reinterpret_cast<float*>(sK);          // [2][HD][128]
-    float* xml = reinterpret_cast<float*>(sV);          // [2][2][128]: m and l of each half
+    // Epilogue: the row sum is the sum of the two halves' sums (exchanged through shared memory, laid
+    // over the value stages, which nothing reads any more once the last PV product is done); half h
+    // normalises and stores channels [h D/2, (h+1) D/2).
+    float* xl = reinterpret_cast<float*>(sV);           // [2][128]
     int* last_flag = reinterpret_cast<int*>(tmem_slot + 2);
     do {
       if (!ok) break;
-      if (ntiles == 0) {   // a split without tiles: nothing accumulated, nothing to read back
-        xml[(half * 2 + 0) * 128 + row] = -INFINITY;
-        xml[(half * 2 + 1) * 128 + row] = 0.f;
-        break;
+      if (ntiles > 0) {
+        ok = false;
+        KVM_WAIT(&bars[BAR_PVDONE + (ntiles - 1) % Cfg::NACC], ((ntiles - 1) / Cfg::NACC) & 1);
+        tc::tc_fence_after();
+        ok = true;
       }
-      ok = false;
-      KVM_WAIT(&bars[BAR_PVDONE + ((ntiles - 1) & 1)], ((ntiles - 1) >> 1) & 1);
-      tc::tc_fence_after();
-      const uint32_t to = tmem + lane_base + col_o + (1 - half) * HD;
-      float* dstx = xch + half * HD * 128 + row;
-#pragma unroll
-      for (int c = 0; c < HD / 32; ++c) {
-        uint32_t r[32];
-        tc::tmem_ld32(to + c * 32, r);
-        tc::tmem_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) dstx[(c * 32 + i) * 128] = __uint_as_float(r[i]);
-      }
-      xml[(half * 2 + 0) * 128 + row] = m_run;
-      xml[(half * 2 + 1) * 128 + row] = l_run;
-      ok = true;
+      xl[half * 128 + row] = l_run;
     } while (false);
     // every softmax thread reaches this barrier, whether or not its waits succeeded
     asm volatile("bar.sync 1, 256;" ::: "memory");
     const bool good = ok && !*abort_flag;
-    const float m_o = xml[((1 - half) * 2 + 0) * 128 + row];
-    const float l_o = xml[((1 - half) * 2 + 1) * 128 + row];
-    const float mm = fmaxf(m_run, m_o);
-    const float w_me = (m_run == -INFINITY) ? 0.f : tc::ex2_approx(m_run - mm);
-    const float w_ot = (m_o == -INFINITY) ? 0.f : tc::ex2_approx(m_o - mm);
-    const float lsum2 = l_run * w_me + l_o * w_ot;
+    const float lsum2 = l_run + xl[(1 - half) * 128 + row];
     __nv_bfloat16* orow = p.out + bb * p.so0 + hq * p.so1 + (p.out_t0 + (int64_t)qt * 128 + row) * p.so2 + half * HD;
     if (nsp == 1) {
       if (good) {
         const float inv = 1.f / lsum2;
-        const float a_me = w_me * inv, a_ot = w_ot * inv;
-        const uint32_t to = tmem + lane_base + col_o + half * HD;
-        const float* srcx = xch + (1 - half) * HD * 128 + row;
 #pragma unroll
         for (int c = 0; c < HD / 32; ++c) {
           uint32_t r[32];
-          tc::tmem_ld32(to + c * 32, r);
+          tc::tmem_ld32(to_mine + c * 32, r);
           tc::tmem_wait_ld();
           if (row < rows_valid) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float o0 = __uint_as_float(r[2 * i]) * a_me + srcx[(c * 32 + 2 * i) * 128] * a_ot;
-              const float o1 = __uint_as_float(r[2 * i + 1]) * a_me + srcx[(c * 32 + 2 * i + 1) * 128] * a_ot;
-              reinterpret_cast<__nv_bfloat162*>(orow + c * 32)[i] = __floats2bfloat162_rn(o0, o1);
-            }
+            for (int i = 0; i < 16; ++i)
+              reinterpret_cast<__nv_bfloat162*>(orow + c * 32)[i] =
+                  __floats2bfloat162_rn(__uint_as_float(r[2 * i]) * inv, __uint_as_float(r[2 * i + 1]) * inv);
           }
         }
       }
     } else {
-      // Partial result of this split: unnormalised O (relative to mm), mm and the sum, column-major
+      // Partial result of this split: unnormalised O (relative to m_run), m_run and the sum, column-major
       // ([channel][row]) so that the rows of a warp are contiguous.
       const int tile_id = bh * (int)gridDim.x + qt;
       float* mine = p.part + ((int64_t)tile_id * nsp + sp) * (D + 2) * 128;
       if (good && ntiles > 0) {
-        const uint32_t to = tmem + lane_base + col_o + half * HD;
-        const float* srcx = xch + (1 - half) * HD * 128 + row;
 #pragma unroll
         for (int c = 0; c < HD / 32; ++c) {
           uint32_t r[32];
-          tc::tmem_ld32(to + c * 32, r);
+          tc::tmem_ld32(to_mine + c * 32, r);
           tc::tmem_wait_ld();
 #pragma unroll
-          for (int i = 0; i < 32; ++i)
-            mine[(half * HD + c * 32 + i) * 128 + row] = __uint_as_float(r[i]) * w_me + srcx[(c * 32 + i) * 128] * w_ot;
+          for (int i = 0; i < 32; ++i) mine[(half * HD + c * 32 + i) * 128 + row] = __uint_as_float(r[i]);
         }
       }
       if (half == 0) {
-        mine[(D + 0) * 128 + row] = (good && ntiles > 0) ? mm : -INFINITY;
+        mine[(D + 0) * 128 + row] = (good && ntiles > 0) ? m_run : -INFINITY;
         mine[(D + 1) * 128 + row] = (good && ntiles > 0) ? lsum2 : 0.f;
       }
       __threadfence();
@@ -421,9 +404,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
         const float* allp = p.part + (int64_t)tile_id * nsp * (D + 2) * 128;
         float mstar = -INFINITY;
         for (int z = 0; z < nsp; ++z) mstar = fmaxf(mstar, __ldcg(allp + ((int64_t)z * (D + 2) + D) * 128 + row));
-        float acc[HD];
+        float accv[HD];
 #pragma unroll
-        for (int c = 0; c < HD; ++c) acc[c] = 0.f;
+        for (int c = 0; c < HD; ++c) accv[c] = 0.f;
         float den = 0.f;
         for (int z = 0; z < nsp; ++z) {
           const float* pz = allp + (int64_t)z * (D + 2) * 128;
@@ -432,13 +415,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
           const float wz = tc::ex2_approx(mz - mstar);
           den += __ldcg(pz + (D + 1) * 128 + row) * wz;
 #pragma unroll
-          for (int c = 0; c < HD; ++c) acc[c] += __ldcg(pz + (half * HD + c) * 128 + row) * wz;
+          for (int c = 0; c < HD; ++c) accv[c] += __ldcg(pz + (half * HD + c) * 128 + row) * wz;
         }
         if (row < rows_valid) {
           const float inv = 1.f / den;
 #pragma unroll
           for (int c = 0; c < HD / 2; ++c)
-            reinterpret_cast<__nv_bfloat162*>(orow)[c] = __floats2bfloat162_rn(acc[2 * c] * inv, acc[2 * c + 1] * inv);
+            reinterpret_cast<__nv_bfloat162*>(orow)[c] = __floats2bfloat162_rn(accv[2 * c] * inv, accv[2 * c + 1] * inv);
         }
       }
     }
