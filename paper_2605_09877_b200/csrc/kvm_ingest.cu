@@ -121,6 +121,102 @@ __global__ void ingest_q_kernel(__half* __restrict__ stQ, const __nv_bfloat16* _
       to_half2_sat(rope_channel(qrow, 2 * c2, r, cs), rope_channel(qrow, 2 * c2 + 1, r, cs));
 }
 
+// ---- 16-byte versions (rows 16-byte aligned, rotary half a multiple of 8 channels): a thread
+//      converts eight consecutive channels of one token; same arithmetic as the scalar kernels ----
+
+// Eight bf16 channels starting at channel c8*8 of `row`, rotated when they lie in the rotary range.
+__device__ __forceinline__ void rope8(const __nv_bfloat16* __restrict__ row, int c8, int r,
+                                      const float2* __restrict__ cs, float (&out)[8]) {
+  const uint4 raw = *reinterpret_cast<const uint4*>(row + c8 * 8);
+  const __nv_bfloat162* pv = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 f = __bfloat1622float2(pv[i]);
+    out[2 * i] = f.x; out[2 * i + 1] = f.y;
+  }
+  const int ch0 = c8 * 8;
+  if (ch0 >= r) return;
+  const int half = r >> 1;
+  const bool lower = ch0 < half;
+  const uint4 rawo = *reinterpret_cast<const uint4*>(row + (lower ? ch0 + half : ch0 - half));
+  const __nv_bfloat162* po = reinterpret_cast<const __nv_bfloat162*>(&rawo);
+  const float4* c4 = reinterpret_cast<const float4*>(cs + (lower ? ch0 : ch0 - half));   // (cos, sin) pairs
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 o = __bfloat1622float2(po[i]);
+    const float4 cc = c4[i];   // cos0 sin0 cos1 sin1
+    if (lower) {
+      out[2 * i] = out[2 * i] * cc.x - o.x * cc.y;
+      out[2 * i + 1] = out[2 * i + 1] * cc.z - o.y * cc.w;
+    } else {
+      out[2 * i] = o.x * cc.y + out[2 * i] * cc.x;
+      out[2 * i + 1] = o.y * cc.w + out[2 * i + 1] * cc.z;
+    }
+  }
+}
+
+__device__ __forceinline__ uint4 pack8_sat(const float (&x)[8]) {
+  uint4 o;
+  __half2 h0 = to_half2_sat(x[0], x[1]), h1 = to_half2_sat(x[2], x[3]), h2 = to_half2_sat(x[4], x[5]), h3 = to_half2_sat(x[6], x[7]);
+  o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
+  o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
+  return o;
+}
+
+__global__ void __launch_bounds__(256) ingest_kv_vec_kernel(
+    __half* __restrict__ stK, __half* __restrict__ stV, float* __restrict__ stG, __half* __restrict__ ringK,
+    __half* __restrict__ ringV, float* __restrict__ ringG, const __nv_bfloat16* __restrict__ k,
+    const __nv_bfloat16* __restrict__ v, const float* __restrict__ gate, const float2* __restrict__ ropeCS,
+    int64_t sk0, int64_t sk1, int64_t sk2, int64_t sv0, int64_t sv1, int64_t sv2, int64_t sg0, int64_t sg1,
+    int64_t sg2, int Hkv, int d, int r, int64_t stRows, int64_t ringCap, int64_t ringLen, int64_t pos0, int64_t n,
+    int64_t nhist, int64_t tail_start) {
+  const int u = blockIdx.y;
+  const int b = u / Hkv, hk = u % Hkv;
+  const int w8 = d / 8;                       // 16-byte chunks per row
+  const int tpb = 256 / w8;                   // tokens per block
+  const int64_t j = (int64_t)blockIdx.x * tpb + threadIdx.x / w8;
+  const int c8 = threadIdx.x % w8;
+  if (j >= n) return;
+  float kx[8], vx[8];
+  rope8(k + b * sk0 + hk * sk1 + j * sk2, c8, r, ropeCS + j * (r >> 1), kx);
+  {
+    const uint4 raw = *reinterpret_cast<const uint4*>(v + b * sv0 + hk * sv1 + j * sv2 + c8 * 8);
+    const __nv_bfloat162* pv = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __bfloat1622float2(pv[i]);
+      vx[2 * i] = f.x; vx[2 * i + 1] = f.y;
+    }
+  }
+  const uint4 kk = pack8_sat(kx), vv = pack8_sat(vx);
+  const float g = gate ? gate[b * sg0 + hk * sg1 + j * sg2] : 1.0f;
+  const int64_t row = (int64_t)u * stRows + nhist + j;
+  reinterpret_cast<uint4*>(stK + row * d)[c8] = kk;
+  reinterpret_cast<uint4*>(stV + row * d)[c8] = vv;
+  if (c8 == 0) stG[row] = g;
+  const int64_t t = pos0 + j;
+  if (t >= tail_start) {
+    const int64_t rrow = (int64_t)u * ringCap + t % ringLen;
+    reinterpret_cast<uint4*>(ringK + rrow * d)[c8] = kk;
+    reinterpret_cast<uint4*>(ringV + rrow * d)[c8] = vv;
+    if (c8 == 0) ringG[rrow] = g;
+  }
+}
+
+__global__ void __launch_bounds__(256) ingest_q_vec_kernel(__half* __restrict__ stQ, const __nv_bfloat16* __restrict__ q,
+                                                           const float2* __restrict__ ropeCS, int64_t sq0, int64_t sq1,
+                                                           int64_t sq2, int Hq, int d, int r, int64_t Tcall, int64_t n) {
+  const int bh = blockIdx.y;
+  const int b = bh / Hq, h = bh % Hq;
+  const int w8 = d / 8, tpb = 256 / w8;
+  const int64_t j = (int64_t)blockIdx.x * tpb + threadIdx.x / w8;
+  const int c8 = threadIdx.x % w8;
+  if (j >= n) return;
+  float qx[8];
+  rope8(q + b * sq0 + h * sq1 + j * sq2, c8, r, ropeCS + j * (r >> 1), qx);
+  reinterpret_cast<uint4*>(stQ + ((int64_t)bh * Tcall + j) * d)[c8] = pack8_sat(qx);
+}
+
 int launch_ingest(State* st, const IngestArgs& a, cudaStream_t s) {
   int launches = 0;
   const int d = st->d, hw = d / 2;
@@ -138,7 +234,21 @@ int launch_ingest(State* st, const IngestArgs& a, cudaStream_t s) {
                                                 a.hist_start, a.nhist, d);
     ++launches;
   }
-  {
+  // 16-byte path: every row of q, k, v starts on a 16-byte boundary and a rotary half is whole chunks
+  auto al16 = [](const void* ptr, const int64_t* st3) {
+    return ((uintptr_t)ptr & 15) == 0 && (st3[0] & 7) == 0 && (st3[1] & 7) == 0 && (st3[2] & 7) == 0;
+  };
+  const bool rope_ok = st->r == 0 || ((st->r / 2) % 8) == 0;
+  const int tpb = 256 / (d / 8);
+  if (rope_ok && al16(a.k, a.sk) && al16(a.v, a.sv)) {
+    dim3 grid((unsigned)((a.n + tpb - 1) / tpb), st->U);
+    ingest_kv_vec_kernel<<<grid, 256, 0, s>>>(st->stK, st->stV, st->stG, st->ringK, st->ringV, st->ringG, a.k,
+                                              a.v, a.gate, st->ropeCS, a.sk[0], a.sk[1], a.sk[2], a.sv[0],
+                                              a.sv[1], a.sv[2], a.sg[0], a.sg[1], a.sg[2], st->Hkv, d, st->r,
+                                              st->stRows, (int64_t)st->w * st->Cmax, st->ringLen, a.pos0, a.n,
+                                              a.nhist, a.tail_start);
+    ++launches;
+  } else {
     dim3 grid((unsigned)((a.n * hw + threads - 1) / threads), st->U);
     ingest_kv_kernel<<<grid, threads, 0, s>>>(st->stK, st->stV, st->stG, st->ringK, st->ringV, st->ringG, a.k,
                                               a.v, a.gate, st->ropeCS, a.sk[0], a.sk[1], a.sk[2], a.sv[0],
@@ -147,7 +257,12 @@ int launch_ingest(State* st, const IngestArgs& a, cudaStream_t s) {
                                               a.nhist, a.tail_start);
     ++launches;
   }
-  {
+  if (rope_ok && al16(a.q, a.sq)) {
+    dim3 grid((unsigned)((a.n + tpb - 1) / tpb), st->B * st->Hq);
+    ingest_q_vec_kernel<<<grid, 256, 0, s>>>(st->stQ, a.q, st->ropeCS, a.sq[0], a.sq[1], a.sq[2], st->Hq, d,
+                                             st->r, st->Tcall, a.n);
+    ++launches;
+  } else {
     dim3 grid((unsigned)((a.n * hw + threads - 1) / threads), st->B * st->Hq);
     ingest_q_kernel<<<grid, threads, 0, s>>>(st->stQ, a.q, st->ropeCS, a.sq[0], a.sq[1], a.sq[2], st->Hq, d,
                                              st->r, st->Tcall, a.n);
