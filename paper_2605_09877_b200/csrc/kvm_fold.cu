@@ -699,7 +699,7 @@ struct FoldApplyParams {
 };
 
 template <int D>
-__global__ void __launch_bounds__(256) fold_apply_kernel(FoldApplyParams p) {
+__global__ void __launch_bounds__(256, 4) fold_apply_kernel(FoldApplyParams p) {
   constexpr int CH = D / 32;
   __shared__ int s_pi[kMaxBlock], s_sorted[kMaxBlock], s_creator[kMaxBlock], s_segnew[kMaxBlock];
   const int u = blockIdx.y, hk = u % p.Hkv;
