@@ -910,9 +910,14 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
     p.C = C; p.Cmax = st->Cmax; p.Hkv = st->Hkv; p.S = st->S; p.n_append = a.n_append; p.nsplit = nsplit;
     p.thr_coeff = route_thr_coeff(st);
     KernelTimer kt(st, 4, s);
-    // two CTAs per unit while that still fits the GPU in one wave (measured: the hand-over costs
-    // more than it saves beyond two), one otherwise
-    int R = (2 * st->U <= 2 * 148 && C >= 32) ? 2 : 1;
+    // CTAs per unit (measured on U = 8, 32, 256): about 64 CTAs in all, at least two per unit while
+    // 2U CTAs fit the GPU in one wave, at most eight, at least 16 tokens each - beyond that the
+    // hand-over costs more than the shorter slices save
+    int R = 64 / st->U;
+    if (R < 2 && 2 * st->U <= 2 * 148) R = 2;
+    if (R > 8) R = 8;
+    if (R > C / 16) R = C / 16;
+    if (R < 1) R = 1;
     dim3 dgrid(R, st->U);
     // programmatic dependent launch: the CTAs may start (and set up their shared memory) while the
     // routing filter is still running; they wait for it before the first read of its output
