@@ -141,6 +141,20 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
+// 2^x on the FMA pipe: x = n + f with n = round(x) (taken from the mantissa of x + 1.5*2^23),
+// f in [-1/2, 1/2], 2^f by its degree-4 Taylor polynomial (relative error < 5e-5), n added to the
+// exponent field.  Inputs below -125 (masked entries are -inf) give 2^-125.
+__device__ __forceinline__ float ex2_poly(float x) {
+  x = fmaxf(x, -125.f);
+  const float r = x + 12582912.f;
+  const float f = x - (r - 12582912.f);
+  float p = fmaf(f, 0.0096181291f, 0.0555041087f);
+  p = fmaf(p, f, 0.2402265070f);
+  p = fmaf(p, f, 0.6931471806f);
+  p = fmaf(p, f, 1.0f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(r) << 23));
+}
+
 }  // namespace tc
 
 // Host: encodes a 3-D tiled tensor map over a [units, rows, d] fp16 array (d contiguous), box
