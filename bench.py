@@ -83,6 +83,7 @@ def prefill_flops(wl, T):
 # roofline, from the ncu captures summarised under profiles/ (null until captured for the workload).
 NCU_TRAFFIC = {
     ("cfg5", "decode"): 4.574e9,    # profiles/ncu_full_attn_route_decide_decode_small_cases.md (4.570 GB read + 4 MB written)
+    ("cfg2", "attention"): 13.72e6,  # same file: 13.72 MB read, 0 written per launch (algorithmic: 14.6 MB)
 }
 
 
