@@ -138,7 +138,11 @@ kvm_status_t kvm_decode_step(const void* q, const void* k, const void* v, kvm_st
 
 /* Same operations with HOST buffers (contiguous layouts as above): the call copies the
  * inputs to library-owned device staging, runs the path, copies `out` back and
- * synchronises the stream before returning.  n_tokens <= max_call_tokens. */
+ * synchronises the stream before returning.  n_tokens <= max_call_tokens.  A long prefill is cut
+ * into up to eight segments of whole blocks whose host-to-device and device-to-host copies run on
+ * the state's own streams beside the computation of the neighbouring segments (pinned host memory
+ * is needed for the copies to overlap; pageable memory works, serially).  The result is identical to
+ * one kvm_prefill call. */
 kvm_status_t kvm_prefill_host(const void* q_host, const void* k_host, const void* v_host,
                               kvm_state_t* state, int32_t block, kvm_growth_t growth,
                               int32_t rope_dims, int64_t n_tokens, const float* gate_host,

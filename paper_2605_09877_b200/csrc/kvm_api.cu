@@ -105,6 +105,13 @@ void free_all(kvm_state* ks) {
   State& s = ks->s;
   if (s.foldStream) { cudaStreamDestroy(s.foldStream); s.foldStream = nullptr; }
   if (s.kbStream) { cudaStreamDestroy(s.kbStream); s.kbStream = nullptr; }
+  if (s.hinStream) { cudaStreamDestroy(s.hinStream); s.hinStream = nullptr; }
+  if (s.houtStream) { cudaStreamDestroy(s.houtStream); s.houtStream = nullptr; }
+  for (cudaEvent_t* e : {&s.evHostStart, &s.evHostOut}) if (*e) { cudaEventDestroy(*e); *e = nullptr; }
+  for (int i = 0; i < 8; ++i) {
+    if (s.evIn[i]) { cudaEventDestroy(s.evIn[i]); s.evIn[i] = nullptr; }
+    if (s.evComp[i]) { cudaEventDestroy(s.evComp[i]); s.evComp[i] = nullptr; }
+  }
   for (cudaEvent_t* e : {&s.evJoin, &s.evPre[0], &s.evPre[1], &s.evFold[0], &s.evFold[1], &s.evKb[0], &s.evKb[1], &s.evBatchDone[0], &s.evBatchDone[1]})
     if (*e) { cudaEventDestroy(*e); *e = nullptr; }
 }
@@ -148,6 +155,15 @@ kvm_status_t ensure_host_staging(kvm_state* ks) {
   if ((rc = dev_alloc(ks, &o, nq, false)) != KVM_OK) return rc;
   if ((rc = dev_alloc(ks, &s.hG, (size_t)s.U * s.Tcall, false)) != KVM_OK) return rc;
   s.hQ = a; s.hK = b; s.hV = c; s.hOut = o;
+  bool ok = cudaStreamCreateWithFlags(&s.hinStream, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&s.houtStream, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&s.evHostStart, cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&s.evHostOut, cudaEventDisableTiming) == cudaSuccess;
+  for (int i = 0; i < 8; ++i) {
+    ok = ok && cudaEventCreateWithFlags(&s.evIn[i], cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&s.evComp[i], cudaEventDisableTiming) == cudaSuccess;
+  }
+  if (!ok) { cudaGetLastError(); return KVM_ERR_CUDA; }
   ks->host_staging = true;
   return KVM_OK;
 }
@@ -618,16 +634,57 @@ KVM_API kvm_status_t kvm_prefill_host(const void* q_host, const void* k_host, co
   if (!guard.ok) return KVM_ERR_CUDA;
   kvm_status_t rc = ensure_host_staging(ks);
   if (rc != KVM_OK) return rc;
-  const size_t bq = (size_t)s.B * s.Hq * n_tokens * s.d * 2, bk = (size_t)s.U * n_tokens * s.d * 2;
-  bool ok = cudaMemcpyAsync(s.hQ, q_host, bq, cudaMemcpyHostToDevice, stream) == cudaSuccess;
-  ok = ok && cudaMemcpyAsync(s.hK, k_host, bk, cudaMemcpyHostToDevice, stream) == cudaSuccess;
-  ok = ok && cudaMemcpyAsync(s.hV, v_host, bk, cudaMemcpyHostToDevice, stream) == cudaSuccess;
-  if (gate_host) ok = ok && cudaMemcpyAsync(s.hG, gate_host, (size_t)s.U * n_tokens * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  // The call is cut into up to eight segments of whole blocks; segment i+1 is copied in, and segment
+  // i-1 copied out, while segment i is computed (three streams, the copies as strided 2-D copies into /
+  // out of staging buffers that have the host layout [batch, head, token, channel]).
+  const int64_t n = n_tokens;
+  const int64_t d = s.d;
+  int nseg = (int)(n / (4 * (int64_t)block));
+  if (nseg > 8) nseg = 8;
+  if (nseg < 1) nseg = 1;
+  const int64_t seg_len = ((n + nseg - 1) / nseg + block - 1) / block * block;
+  bool ok = cudaEventRecord(s.evHostStart, stream) == cudaSuccess;
+  ok = ok && cudaStreamWaitEvent(s.hinStream, s.evHostStart, 0) == cudaSuccess;
+  ok = ok && cudaStreamWaitEvent(s.houtStream, s.evHostStart, 0) == cudaSuccess;
   if (!ok) { cudaGetLastError(); return KVM_ERR_CUDA; }
-  rc = kvm_prefill(s.hQ, s.hK, s.hV, ks, block, growth, rope_dims, n_tokens, gate_host ? s.hG : nullptr, s.hOut, nullptr, cuda_stream);
-  if (rc != KVM_OK) return rc;
-  if (cudaMemcpyAsync(out_host, s.hOut, bq, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return KVM_ERR_CUDA;
-  if (cudaStreamSynchronize(stream) != cudaSuccess) return KVM_ERR_CUDA;
+  kvm_strides_t st;
+  st.q[0] = (int64_t)s.Hq * n * d; st.q[1] = n * d; st.q[2] = d; st.q[3] = 1;
+  st.k[0] = (int64_t)s.Hkv * n * d; st.k[1] = n * d; st.k[2] = d; st.k[3] = 1;
+  for (int i = 0; i < 4; ++i) { st.v[i] = st.k[i]; st.out[i] = st.q[i]; }
+  const size_t pitch = (size_t)n * d * 2;
+  int iseg = 0;
+  for (int64_t t0 = 0; t0 < n; t0 += seg_len, ++iseg) {
+    const int64_t len = t0 + seg_len <= n ? seg_len : n - t0;
+    const size_t width = (size_t)len * d * 2;
+    const size_t off = (size_t)t0 * d;   // elements
+    ok = cudaMemcpy2DAsync((__nv_bfloat16*)s.hQ + off, pitch, (const __nv_bfloat16*)q_host + off, pitch, width,
+                           (size_t)s.B * s.Hq, cudaMemcpyHostToDevice, s.hinStream) == cudaSuccess;
+    ok = ok && cudaMemcpy2DAsync((__nv_bfloat16*)s.hK + off, pitch, (const __nv_bfloat16*)k_host + off, pitch, width,
+                                 (size_t)s.U, cudaMemcpyHostToDevice, s.hinStream) == cudaSuccess;
+    ok = ok && cudaMemcpy2DAsync((__nv_bfloat16*)s.hV + off, pitch, (const __nv_bfloat16*)v_host + off, pitch, width,
+                                 (size_t)s.U, cudaMemcpyHostToDevice, s.hinStream) == cudaSuccess;
+    float* gseg = nullptr;
+    if (gate_host) {   // gates of the segment, contiguous [unit, token] as kvm_prefill expects them
+      gseg = s.hG + (size_t)s.U * t0;
+      ok = ok && cudaMemcpy2DAsync(gseg, (size_t)len * 4, gate_host + t0, (size_t)n * 4, (size_t)len * 4, (size_t)s.U,
+                                   cudaMemcpyHostToDevice, s.hinStream) == cudaSuccess;
+    }
+    ok = ok && cudaEventRecord(s.evIn[iseg], s.hinStream) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(stream, s.evIn[iseg], 0) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return KVM_ERR_CUDA; }
+    rc = kvm_prefill((__nv_bfloat16*)s.hQ + off, (__nv_bfloat16*)s.hK + off, (__nv_bfloat16*)s.hV + off, ks, block, growth,
+                     rope_dims, len, gseg, (__nv_bfloat16*)s.hOut + off, &st, cuda_stream);
+    if (rc != KVM_OK) return rc;
+    ok = cudaEventRecord(s.evComp[iseg], stream) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(s.houtStream, s.evComp[iseg], 0) == cudaSuccess;
+    ok = ok && cudaMemcpy2DAsync((__nv_bfloat16*)out_host + off, pitch, (__nv_bfloat16*)s.hOut + off, pitch, width,
+                                 (size_t)s.B * s.Hq, cudaMemcpyDeviceToHost, s.houtStream) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return KVM_ERR_CUDA; }
+  }
+  ok = cudaEventRecord(s.evHostOut, s.houtStream) == cudaSuccess;
+  ok = ok && cudaStreamWaitEvent(stream, s.evHostOut, 0) == cudaSuccess;
+  ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); return KVM_ERR_CUDA; }
   return KVM_OK;
 }
 

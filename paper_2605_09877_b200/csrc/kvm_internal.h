@@ -58,6 +58,9 @@ struct State {
   int prevNAppend;
   // second stream and events that let a block's attention and the fold of the block before it overlap
   cudaStream_t foldStream, kbStream;   // folds; memory keys computed ahead of the folds
+  // host-buffer entry points: copy-in / copy-out streams and per-segment events (created on first use)
+  cudaStream_t hinStream, houtStream;
+  cudaEvent_t evHostStart, evHostOut, evIn[8], evComp[8];
   cudaEvent_t evJoin, evPre[2], evFold[2], evKb[2], evBatchDone[2];
   // ---- window ring (device): slot = t mod ringLen ----
   __half *ringK, *ringV;         // [U, w*Cmax, d]  rotated keys / values (fp16)

@@ -148,6 +148,26 @@ def test_host_buffer_entry_points_match_device_ones():
     st3.free()
 
 
+def test_host_prefill_pipelined_segments_match_device_prefill():
+    """A long call through kvm_prefill_host is cut into segments whose copies overlap the compute;
+    the result must equal the single device call bit for bit (gates included)."""
+    wl = CFG["cfg2"].scaled(B=1, Hq=2, Hkv=2, T=128 * 33 + 5)
+    tensors = synth.make_inputs(wl)
+    tensors["gate"] = synth.make_gate(wl)
+    params = synth.make_layer_params(wl)
+    y_dev, st = pu.run_gpu(wl, tensors, params)
+    ref = st.export()
+    st.free()
+    st2, g = pu.gpu_layer(wl, params)
+    out = torch.zeros_like(tensors["q"])
+    st2.prefill_host(tensors["q"].contiguous(), tensors["k"].contiguous(), tensors["v"].contiguous(), wl.C, g, wl.r, out,
+                     gate=tensors["gate"].contiguous())
+    assert torch.equal(out, y_dev)
+    got = st2.export()
+    assert np.array_equal(got["sum_k"], ref["sum_k"]) and np.array_equal(got["count"], ref["count"])
+    st2.free()
+
+
 def test_api_errors_leave_state_usable():
     from paper_2605_09877_b200 import kvm
     wl = CFG["cfg1"].scaled(T=128)
