@@ -274,7 +274,7 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   {
     // memory-key slots: as many blocks per batched launch as fit in 2 GiB (at least 1, at most 64,
     // never more than a call can hold)
-    const size_t per_slot = U * Cm * d * 16 + U * (size_t)s.CbarRows * d * 4 + U * Cm * 4 + U * Cm * Cm * 4;
+    const size_t per_slot = U * Cm * d * 8 + U * (size_t)s.CbarRows * d * 4 + U * Cm * 20 + U * Cm * Cm * 4;
     size_t slots = ((size_t)2 << 30) / per_slot;
     const size_t call_blocks = (size_t)(s.Tcall / s.Cmax) + 2;
     if (slots > call_blocks) slots = call_blocks;
@@ -285,7 +285,7 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   {
     const size_t G = (size_t)s.kbSlots;
     A(s.kbar64, G * U * Cm * d); A(s.kbarH, G * U * (size_t)s.CbarRows * d); A(s.kbarNorm, G * U * Cm);
-    A(s.kbarHat64, G * U * Cm * d); A(s.kbarHatH, G * U * (size_t)s.CbarRows * d);
+    A(s.kbarHatStat, G * U * Cm); A(s.kbarHatH, G * U * (size_t)s.CbarRows * d);
     A(s.gramT, G * U * Cm * Cm);
   }
   for (int i = 0; i < 2; ++i) {

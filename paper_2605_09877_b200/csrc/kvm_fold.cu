@@ -45,7 +45,7 @@ template <int D>
 __global__ void __launch_bounds__(256) kbar_kernel(const __half* __restrict__ ok, int64_t unit_stride,
                                                    const float* __restrict__ ln_w, const float* __restrict__ ln_b,
                                                    double* __restrict__ kbar64, __half* __restrict__ kbarH,
-                                                   float* __restrict__ kbarNorm, double* __restrict__ kbarHat64,
+                                                   float* __restrict__ kbarNorm, double2* __restrict__ kbarHatStat,
                                                    __half* __restrict__ kbarHatH, int C, int Cmax, int CbarRows, int U, int Hkv, int r,
                                                    double ln_eps) {
   constexpr int CH = D / 32;
@@ -83,10 +83,12 @@ __global__ void __launch_bounds__(256) kbar_kernel(const __half* __restrict__ ok
   for (int i = 0; i < CH; ++i) {
     const int x = lane + 32 * i;
     const double hat = (double)ln_w[hk * D + x] * ((kb[i] - mu2) * rs2) + (double)ln_b[hk * D + x];
-    kbarHat64[o + x] = hat;
     kbarHatH[oh + x] = __float2half_rn((float)hat);
   }
-  if (lane == 0) kbarNorm[((int64_t)g * U + u) * Cmax + j] = (float)sqrt(n2) * 1.000001f;
+  if (lane == 0) {
+    kbarNorm[((int64_t)g * U + u) * Cmax + j] = (float)sqrt(n2) * 1.000001f;
+    kbarHatStat[((int64_t)g * U + u) * Cmax + j] = make_double2(mu2, rs2);
+  }
 }
 
 // Rows that the last fold touched are current in one readout copy only: bring them over to the
@@ -222,7 +224,8 @@ __global__ void __launch_bounds__(256) route_filter_simt_kernel(const __half* __
 struct FoldDecideParams {
   const double* kbar64;
   const float* kbarNorm;
-  const double* kbarHat64;   // LN_s(kbar_j): keys of the rows the block's tokens would create
+  const double2* kbarHatStat;   // (mean, rstd) of kbar_j: LN_s(kbar_j), the key of the row token j would create,
+                                // is gam * ((kbar_j - mean) * rstd) + bet, the expression of the memory-key kernel
   const float* gramT;        // [U, Cmax, Cmax] approximate kbarHat_a . kbar_j at [a][j] (fp16 operands)
   const float* candV;
   const int32_t* candI;
@@ -595,10 +598,15 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
       for (int k = 0; k < 8; ++k) {
         const int q = min(q0 + k * kDecideWarps, np2 - 1);
         const double* kb = kbarU + (int64_t)s_ptok[q] * D;
-        const double* kh = p.kbarHat64 + (tokBase + s_creator[s_prow[q]]) * D;
+        const int jc = s_creator[s_prow[q]];
+        const double* ka = kbarU + (int64_t)jc * D;
+        const double2 hs = p.kbarHatStat[tokBase + jc];
         double acc = 0.0;
 #pragma unroll
-        for (int c = 0; c < CH; ++c) acc += kb[lane + 32 * c] * kh[lane + 32 * c];
+        for (int c = 0; c < CH; ++c) {
+          const double hat = gam[c] * ((ka[lane + 32 * c] - hs.x) * hs.y) + bet[c];
+          acc += kb[lane + 32 * c] * hat;
+        }
         part[k] = acc;
       }
       const double z0 = warp_reduce4(part[0], part[1], part[2], part[3], lane);
@@ -618,10 +626,14 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
       double best = s_best[j];
       int arg = s_barg[j];
       for (int a = 0; a < n_a; ++a) {
-        const double* kh = p.kbarHat64 + (tokBase + s_creator[a]) * D;
+        const double* ka = kbarU + (int64_t)s_creator[a] * D;
+        const double2 hs = p.kbarHatStat[tokBase + s_creator[a]];
         double acc = 0.0;
 #pragma unroll
-        for (int c = 0; c < CH; ++c) acc += kb[c] * kh[lane + 32 * c];
+        for (int c = 0; c < CH; ++c) {
+          const double hat = gam[c] * ((ka[lane + 32 * c] - hs.x) * hs.y) + bet[c];
+          acc += kb[c] * hat;
+        }
         acc = warp_sum_d(acc);
         if (acc > best) { best = acc; arg = (int)m + a; }
       }
@@ -832,7 +844,7 @@ int launch_kbar(State* st, const __half* ok, int64_t unit_stride, int nblk, int 
   double* k64 = st->kbar64 + (int64_t)slot0 * U * st->Cmax * D;
   __half* kh = st->kbarH + (int64_t)slot0 * U * st->CbarRows * D;
   float* kn = st->kbarNorm + (int64_t)slot0 * U * st->Cmax;
-  double* khat = st->kbarHat64 + (int64_t)slot0 * U * st->Cmax * D;
+  double2* khat = st->kbarHatStat + (int64_t)slot0 * U * st->Cmax;
   __half* khh = st->kbarHatH + (int64_t)slot0 * U * st->CbarRows * D;
   if (D == 128)
     kbar_kernel<128><<<grid, 256, 0, s>>>(ok, unit_stride, st->ln_w, st->ln_b, k64, kh, kn, khat, khh, C, st->Cmax,
@@ -872,7 +884,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
   const double* kbar64 = st->kbar64 + (int64_t)a.slot * U * st->Cmax * D;
   const __half* kbarH = st->kbarH + (int64_t)a.slot * U * st->CbarRows * D;
   const float* kbarNorm = st->kbarNorm + (int64_t)a.slot * U * st->Cmax;
-  const double* kbarHat64 = st->kbarHat64 + (int64_t)a.slot * U * st->Cmax * D;
+  const double2* kbarHatStat = st->kbarHatStat + (int64_t)a.slot * U * st->Cmax;
   const bool all_append = a.first || a.n_append >= C;
   if (!all_append) {
     // enough CTAs to fill the GPU, at least 256 rows per split
@@ -898,7 +910,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
       launches += launch_route_filter_tc(st, a.m, nsplit, a.slot, s);
     }
     FoldDecideParams p;
-    p.kbar64 = kbar64; p.kbarNorm = kbarNorm; p.kbarHat64 = kbarHat64;
+    p.kbar64 = kbar64; p.kbarNorm = kbarNorm; p.kbarHatStat = kbarHatStat;
     p.gramT = st->gramT + (int64_t)a.slot * U * st->Cmax * st->Cmax;
     p.candV = st->candV; p.candI = st->candI; p.ln_w = st->ln_w; p.ln_b = st->ln_b;
     p.sumK = st->sumK; p.kmu = st->kmu; p.krstd = st->krstd;

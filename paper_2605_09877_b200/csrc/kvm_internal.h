@@ -79,7 +79,8 @@ struct State {
   __half* kbarH;                 // [kbSlots][U, CbarRows, d]
   float* kbarNorm;               // [kbSlots][U, Cmax]
   int CbarRows;                  // rows per unit of kbarH (Cmax rounded up to the 128-row MMA tile)
-  double* kbarHat64;             // [kbSlots][U, Cmax, d]  LN_s(kbar_j): the readout key of a row created by token j
+  double2* kbarHatStat;          // [kbSlots][U, Cmax]  (mean, rstd) of kbar_j: LN_s(kbar_j), the readout key of a row
+                                 // created by token j, is recomputed from kbar64 and these where it is needed
   __half* kbarHatH;              // [kbSlots][U, CbarRows, d]  the same in fp16 (operand of the new-row filter)
   float* gramT;                  // [kbSlots][U, Cmax, Cmax]  approximate kbarHat_a . kbar_j at [a][j] (new-row filter)
   // decisions of the fold being computed ([(nfolds+1) & 1]) and of the one before ([nfolds & 1])
