@@ -714,6 +714,9 @@ template <int D>
 __global__ void __launch_bounds__(256, 4) fold_apply_kernel(FoldApplyParams p) {
   constexpr int CH = D / 32;
   __shared__ int s_pi[kMaxBlock], s_sorted[kMaxBlock], s_creator[kMaxBlock], s_segnew[kMaxBlock];
+  // the routing filter of the next fold may start its set-up now; it waits for this grid to finish
+  // before it reads the readout keys written here
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int u = blockIdx.y, hk = u % p.Hkv;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q = blockIdx.x * 8 + warp;

@@ -110,6 +110,9 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
       for (int mt = 0; mt < mt_used; ++mt)
         for (int kb = 0; kb < Cfg::NKB; ++kb)
           tc::tma_load_3d(sA + mt * Cfg::TILE_BYTES + kb * Cfg::BOX_BYTES, gram ? &mapH : &mapA, &bars[RB_AFULL], kb * 64, mt * 128, a_unit);
+      // the readout keys are written by the apply kernel of the fold before this one: wait for it here
+      // (the set-up above and the load of the block's own keys run beside its tail)
+      asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int j = 0; j < nsteps; ++j) {
         const int s = j % Cfg::NS;
         const int jt = j >= ntiles ? j - ntiles : j;
@@ -262,8 +265,16 @@ int launch_route_filter_tc(State* st, int64_t m, int nsplit, int slot, cudaStrea
   const CUtensorMap* tm = reinterpret_cast<const CUtensorMap*>(st->tmaps);
   dim3 grid(nsplit, st->U);
   const int ks = (st->nfolds & 1) ? 6 : 1;   // the fold reads the readout copy of the current version
-  if (st->d == 128) route_filter_tc_kernel<128><<<grid, 320, RouteTcCfg<128>::SMEM_BYTES, s>>>(tm[5], tm[ks], tm[8], p);
-  else route_filter_tc_kernel<64><<<grid, 320, RouteTcCfg<64>::SMEM_BYTES, s>>>(tm[5], tm[ks], tm[8], p);
+  // programmatic dependent launch behind the apply kernel of the previous fold: the CTAs set up and
+  // fetch the block's memory keys while it finishes
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = grid; lc.blockDim = dim3(320); lc.stream = s;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = at; lc.numAttrs = st->prof_hook == nullptr ? 1 : 0;
+  if (st->d == 128) { lc.dynamicSmemBytes = RouteTcCfg<128>::SMEM_BYTES; cudaLaunchKernelEx(&lc, route_filter_tc_kernel<128>, tm[5], tm[ks], tm[8], p); }
+  else { lc.dynamicSmemBytes = RouteTcCfg<64>::SMEM_BYTES; cudaLaunchKernelEx(&lc, route_filter_tc_kernel<64>, tm[5], tm[ks], tm[8], p); }
   return 1;
 }
 
