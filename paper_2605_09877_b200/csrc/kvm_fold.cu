@@ -363,6 +363,7 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
   __syncthreads();
   if (warp == 0) {   // segment starts: exclusive prefix sum over the slice's tokens, eight per lane
     int cnt[8], tot = 0;
+    unsigned single = 0u;
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
       const int j = jlo + lane * 8 + k;
@@ -371,6 +372,10 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
         c = s_pcnt[j];
         if (c > kPairPerTok) { s_exh[j] = 1; }
         if (s_exh[j]) c = 0;
+        // A fold that appends nothing needs no scores, and the true arg max is always among the
+        // candidates: a token with a single candidate is decided without the exact similarity
+        // (it takes no room in the pair list).
+        if (n_a == 0 && c == 1) { single |= 1u << k; c = 0; }
       }
       cnt[k] = c;
       tot += c;
@@ -389,7 +394,7 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
         if (start + cnt[k] > kPairCap) { s_exh[j] = 1; cnt[k] = 0; }   // the list is full: exact scan instead
         s_pstart[j] = start;
         s_pcnt[j] = cnt[k];
-        s_fill[j] = 0;
+        s_fill[j] = ((single >> k) & 1u) ? -1 : 0;
       }
       start += cnt[k];
     }
@@ -410,6 +415,12 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
     for (int k = 0; k < kTopK; ++k)
       if (i[k] >= 0 && (i[k] < p.S ? n_a > 0 : keep)) ++c;
     if (c == 0) continue;
+    if (s_fill[j] < 0) {   // the token's only candidate: its row is the merge target
+#pragma unroll
+      for (int k = 0; k < kTopK; ++k)
+        if (i[k] >= 0 && (i[k] < p.S ? n_a > 0 : keep)) s_barg[j] = i[k];
+      continue;
+    }
     int w = s_pstart[j] + atomicAdd(&s_fill[j], c);
 #pragma unroll
     for (int k = 0; k < kTopK; ++k) {
@@ -453,7 +464,7 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
   }
   __syncthreads();
   // ---- A4: per-token reduction (ties: lowest row) ----
-  if (jlo + tid < jhi && !s_exh[jlo + tid]) {
+  if (jlo + tid < jhi && !s_exh[jlo + tid] && s_fill[jlo + tid] >= 0) {
     const int j = jlo + tid;
     double score = -INFINITY, best = -INFINITY;
     int barg = -1;
