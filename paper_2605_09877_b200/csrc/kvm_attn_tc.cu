@@ -469,8 +469,9 @@ int launch_attn_tc(State* st, const AttnArgs& a, cudaStream_t s) {
   p.out = a.out; p.tau_s = st->tau_s; p.tau_b = st->tau_b; p.status = st->status;
   p.nq = a.nq; p.Hq = st->Hq; p.Hkv = st->Hkv; p.G = st->G;
   p.part = st->attnPart; p.part_cnt = st->attnCnt;
-  // key splits when there are few query tiles: up to half of the GPU (the folds of the block before
-  // run beside this kernel and are usually the longer chain), at least two key tiles per split
+  // key splits when there are few query tiles: up to a quarter of the GPU (the folds of the block
+  // before run beside this kernel and are usually the longer chain; measured: a wider attention
+  // kernel only takes SMs away from them), at least two key tiles per split
   const int qtiles = (a.nq + 127) / 128;
   const int ctas = qtiles * st->B * st->Hq;
   int nsp = 1;

@@ -12,7 +12,7 @@ namespace kvm {
 constexpr int kMaxBlock = 256;      // largest block C (one thread per overflow token in the fold)
 constexpr int kTopK = 8;            // routing filter keeps the K best approximate similarities per split
 constexpr int kMaxSplits = 32;      // routing filter / decode split count upper bound
-constexpr int kAttnSplitTiles = 74; // launches with at most this many (batch, head, query tile) CTAs are split along the keys
+constexpr int kAttnSplitTiles = 37; // launches with at most this many (batch, head, query tile) CTAs - a quarter of the GPU - are split along the keys
 constexpr int kAttnMaxSplits = 8;
 constexpr int kRowAlign = 128;      // state capacity is rounded up to the attention key tile
 
