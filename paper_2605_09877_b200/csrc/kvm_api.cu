@@ -210,6 +210,7 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   if ((cfg->flags & KVM_FLAG_RECORD_ASSIGN) && cfg->max_seq_len < 1) return KVM_ERR_INVALID_ARG;
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return KVM_ERR_UNSUPPORTED;
   if (cfg->max_block > kMaxBlock) return KVM_ERR_UNSUPPORTED;
+  if (cfg->max_state_slots >= (1 << 23)) return KVM_ERR_UNSUPPORTED;   // sort keys of the fold hold a row in 23 bits
 
   int ndev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1 || cfg->device < 0 || cfg->device >= ndev) {

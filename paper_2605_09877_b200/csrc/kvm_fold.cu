@@ -281,6 +281,29 @@ __device__ __forceinline__ double warp_sim(const double (&kb)[CH], const double*
   return warp_sum_d(acc);
 }
 
+// Bitonic sort of N (a power of two, <= 2 * blockDim.x) keys in shared memory, ascending; `val` (may
+// be null) is permuted along and breaks ties (smaller value first).  All threads of the CTA call it.
+template <typename K>
+__device__ __forceinline__ void cta_bitonic_sort(K* key, int* val, int N, int tid) {
+  for (int k = 2; k <= N; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      if (tid < (N >> 1)) {
+        const int i = 2 * tid - (tid & (j - 1));
+        const int l = i + j;
+        const bool up = (i & k) == 0;
+        const K a = key[i], b = key[l];
+        bool gt = a > b;
+        if (val != nullptr && a == b) gt = val[i] > val[l];
+        if (gt == up) {
+          key[i] = b; key[l] = a;
+          if (val != nullptr) { const int t = val[i]; val[i] = val[l]; val[l] = t; }
+        }
+      }
+      __syncthreads();
+    }
+  }
+}
+
 template <int D>
 __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDecideParams p) {
   constexpr int CH = D / 32;
@@ -304,7 +327,6 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
   const int jlo = (int)blockIdx.x * ((C + R - 1) / R), jhi = min(C, jlo + (C + R - 1) / R);
   const int64_t m = p.m;
   const int n_a = p.n_append;
-  const int parts = C <= 64 ? 8 : (C <= 128 ? 4 : 2);   // adjacent threads that share a token in the ranking loops
   const double* kbarU = p.kbar64 + (int64_t)u * p.Cmax * D;
   const int64_t rowBase = (int64_t)u * p.Mcap;
   const int64_t tokBase = (int64_t)u * p.Cmax;
@@ -523,37 +545,36 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
   }
   // ---- B: append selection: the n_a smallest scores, ties to the smaller token index ----
   if (n_a > 0) {
-    // `parts` threads share a token: each counts over a quarter (or half) of the block, the counts
-    // are added inside the group of adjacent lanes
-    {
-      const int j = tid / parts, part = tid % parts;
-      int rank = 0;
-      if (j < C) {
-        const double sj = s_score[j];
-        const int per = (C + parts - 1) / parts;
-        const int j1 = min(C, (part + 1) * per);
-#pragma unroll 4
-        for (int jj = part * per; jj < j1; ++jj) {
-          const double so = s_score[jj];
-          rank += (so < sj || (so == sj && jj < j)) ? 1 : 0;
-        }
+    // sort (score, token) ascending; the first n_a entries are appended
+    unsigned long long* skey = reinterpret_cast<unsigned long long*>(s_pval);   // (the pair list is idle here)
+    int* sidx = s_prow;
+    const int N = C <= 64 ? 64 : (C <= 128 ? 128 : 256);
+    if (tid < N) {
+      unsigned long long kbits = ~0ull;
+      if (tid < C) {   // order-preserving integer image of the double
+        const long long bits = __double_as_longlong(s_score[tid]);
+        kbits = (unsigned long long)bits ^ (bits < 0 ? ~0ull : 0x8000000000000000ull);
       }
-#pragma unroll
-      for (int o = parts / 2; o > 0; o >>= 1) rank += __shfl_xor_sync(0xffffffffu, rank, o);
-      if (j < C && part == 0) s_app[j] = rank < n_a ? 1 : 0;
+      skey[tid] = kbits;
+      sidx[tid] = tid;
     }
     __syncthreads();
-    {
-      const int j = tid / parts, part = tid % parts;
-      int before = 0;
-      if (j < C && s_app[j]) {
-        const int per = (C + parts - 1) / parts;
-        const int j1 = min(j, (part + 1) * per);
-        for (int jj = part * per; jj < j1; ++jj) before += s_app[jj];
-      }
-#pragma unroll
-      for (int o = parts / 2; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
-      if (j < C && part == 0 && s_app[j]) s_creator[before] = j;   // rows are laid down in ascending token order
+    cta_bitonic_sort<unsigned long long>(skey, sidx, N, tid);
+    if (tid < N && sidx[tid] < C) s_app[sidx[tid]] = tid < n_a ? 1 : 0;
+    __syncthreads();
+    // rows are laid down in ascending token order: position of an appended token = appended tokens before it
+    if (tid < kMaxBlock) {
+      const bool ap = tid < C && s_app[tid];
+      const unsigned bal = __ballot_sync(0xffffffffu, ap);
+      if (lane == 0) s_fill[warp] = __popc(bal);   // (s_fill is idle here)
+      __syncwarp();
+      s_pcnt[tid] = __popc(bal & ((1u << lane) - 1u));   // appended tokens before this one inside its warp
+    }
+    __syncthreads();
+    if (tid < C && s_app[tid]) {
+      int before = s_pcnt[tid];
+      for (int wq = 0; wq < warp; ++wq) before += s_fill[wq];
+      s_creator[before] = tid;
     }
     __syncthreads();
   }
@@ -668,31 +689,26 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
   __syncthreads();
   // ---- E: order merged tokens by (row, token); publish ----
   {
-    const int j = tid / parts, part = tid % parts;
-    const int pj = j < C ? s_pi[j] : -1;
-    if (j < C && part == 0) {
-      p.pi[tokBase + j] = pj;
-      p.creator[tokBase + j] = s_creator[j];
-    }
-    int ord = 0, nothead = 0;
-    if (pj >= 0) {
-      const int per = (C + parts - 1) / parts;
-      const int j1 = min(C, (part + 1) * per);
-#pragma unroll 4
-      for (int jj = part * per; jj < j1; ++jj) {
-        const int po = s_pi[jj];
-        ord += (po >= 0 && (po < pj || (po == pj && jj < j))) ? 1 : 0;
-        nothead |= (po == pj && jj < j) ? 1 : 0;
+    unsigned* ekey = reinterpret_cast<unsigned*>(s_prow);   // (the pair list is idle here)
+    const int N = C <= 64 ? 64 : (C <= 128 ? 128 : 256);
+    if (tid < N) {
+      const int pj = tid < C ? s_pi[tid] : -1;
+      ekey[tid] = pj >= 0 ? (((unsigned)pj << 9) | (unsigned)tid) : 0xffffffffu;   // rows < 2^23, tokens < 2^9
+      if (tid < C) {
+        p.pi[tokBase + tid] = pj;
+        p.creator[tokBase + tid] = s_creator[tid];
       }
     }
-#pragma unroll
-    for (int o = parts / 2; o > 0; o >>= 1) {
-      ord += __shfl_xor_sync(0xffffffffu, ord, o);
-      nothead |= __shfl_xor_sync(0xffffffffu, nothead, o);
-    }
-    if (pj >= 0 && part == 0) {
-      p.sorted[tokBase + ord] = j;
-      if (!nothead && pj >= m) p.segnew[tokBase + (pj - (int)m)] = ord;
+    __syncthreads();
+    cta_bitonic_sort<unsigned>(ekey, nullptr, N, tid);
+    if (tid < N) {
+      const unsigned kq = ekey[tid];
+      if (kq != 0xffffffffu) {
+        const int rowq = (int)(kq >> 9);
+        p.sorted[tokBase + tid] = (int)(kq & 511u);
+        const bool head = tid == 0 || (int)(ekey[tid - 1] >> 9) != rowq;
+        if (head && rowq >= m) p.segnew[tokBase + (rowq - (int)m)] = tid;
+      }
     }
   }
   if (tid == 0) {
