@@ -281,25 +281,28 @@ __device__ __forceinline__ double warp_sim(const double (&kb)[CH], const double*
   return warp_sum_d(acc);
 }
 
-// Bitonic sort of N (a power of two, <= 2 * blockDim.x) keys in shared memory, ascending; `val` (may
-// be null) is permuted along and breaks ties (smaller value first).  All threads of the CTA call it.
+// Bitonic sort of 256 (key, val) pairs, ascending by key and then val, held one per thread by the
+// first 256 threads of the CTA (the only callers; the others must not call): stages that stay inside a
+// warp exchange through shuffles, the six that cross warps through shared memory (sk / sv, 256 entries
+// each) and a named barrier of those 256 threads.  Afterwards thread t holds the pair of rank t.
 template <typename K>
-__device__ __forceinline__ void cta_bitonic_sort(K* key, int* val, int N, int tid) {
-  for (int k = 2; k <= N; k <<= 1) {
+__device__ __forceinline__ void sort256(K& key, int& val, K* sk, int* sv, int t) {
+  for (int k = 2; k <= 256; k <<= 1) {
     for (int j = k >> 1; j > 0; j >>= 1) {
-      if (tid < (N >> 1)) {
-        const int i = 2 * tid - (tid & (j - 1));
-        const int l = i + j;
-        const bool up = (i & k) == 0;
-        const K a = key[i], b = key[l];
-        bool gt = a > b;
-        if (val != nullptr && a == b) gt = val[i] > val[l];
-        if (gt == up) {
-          key[i] = b; key[l] = a;
-          if (val != nullptr) { const int t = val[i]; val[i] = val[l]; val[l] = t; }
-        }
+      K ok;
+      int ov;
+      if (j < 32) {
+        ok = __shfl_xor_sync(0xffffffffu, key, j);
+        ov = __shfl_xor_sync(0xffffffffu, val, j);
+      } else {
+        sk[t] = key; sv[t] = val;
+        asm volatile("bar.sync 2, 256;" ::: "memory");
+        ok = sk[t ^ j]; ov = sv[t ^ j];
+        asm volatile("bar.sync 2, 256;" ::: "memory");
       }
-      __syncthreads();
+      const bool take_min = ((t & j) == 0) == ((t & k) == 0);   // lower index of the pair in an ascending run
+      const bool other_less = ok < key || (ok == key && ov < val);
+      if (other_less == take_min) { key = ok; val = ov; }
     }
   }
 }
@@ -546,21 +549,16 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
   // ---- B: append selection: the n_a smallest scores, ties to the smaller token index ----
   if (n_a > 0) {
     // sort (score, token) ascending; the first n_a entries are appended
-    unsigned long long* skey = reinterpret_cast<unsigned long long*>(s_pval);   // (the pair list is idle here)
-    int* sidx = s_prow;
-    const int N = C <= 64 ? 64 : (C <= 128 ? 128 : 256);
-    if (tid < N) {
+    if (tid < 256) {
       unsigned long long kbits = ~0ull;
       if (tid < C) {   // order-preserving integer image of the double
         const long long bits = __double_as_longlong(s_score[tid]);
         kbits = (unsigned long long)bits ^ (bits < 0 ? ~0ull : 0x8000000000000000ull);
       }
-      skey[tid] = kbits;
-      sidx[tid] = tid;
+      int tok = tid;
+      sort256<unsigned long long>(kbits, tok, reinterpret_cast<unsigned long long*>(s_pval), s_prow, tid);   // (the pair list is idle here)
+      if (tok < C) s_app[tok] = tid < n_a ? 1 : 0;
     }
-    __syncthreads();
-    cta_bitonic_sort<unsigned long long>(skey, sidx, N, tid);
-    if (tid < N && sidx[tid] < C) s_app[sidx[tid]] = tid < n_a ? 1 : 0;
     __syncthreads();
     // rows are laid down in ascending token order: position of an appended token = appended tokens before it
     if (tid < kMaxBlock) {
@@ -690,19 +688,17 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
   // ---- E: order merged tokens by (row, token); publish ----
   {
     unsigned* ekey = reinterpret_cast<unsigned*>(s_prow);   // (the pair list is idle here)
-    const int N = C <= 64 ? 64 : (C <= 128 ? 128 : 256);
-    if (tid < N) {
+    if (tid < 256) {
       const int pj = tid < C ? s_pi[tid] : -1;
-      ekey[tid] = pj >= 0 ? (((unsigned)pj << 9) | (unsigned)tid) : 0xffffffffu;   // rows < 2^23, tokens < 2^9
+      unsigned kq = pj >= 0 ? (((unsigned)pj << 9) | (unsigned)tid) : 0xffffffffu;   // rows < 2^23, tokens < 2^9
       if (tid < C) {
         p.pi[tokBase + tid] = pj;
         p.creator[tokBase + tid] = s_creator[tid];
       }
-    }
-    __syncthreads();
-    cta_bitonic_sort<unsigned>(ekey, nullptr, N, tid);
-    if (tid < N) {
-      const unsigned kq = ekey[tid];
+      int zero = 0;
+      sort256<unsigned>(kq, zero, ekey + 256, reinterpret_cast<int*>(s_pval), tid);
+      ekey[tid] = kq;
+      asm volatile("bar.sync 2, 256;" ::: "memory");
       if (kq != 0xffffffffu) {
         const int rowq = (int)(kq >> 9);
         p.sorted[tokBase + tid] = (int)(kq & 511u);
