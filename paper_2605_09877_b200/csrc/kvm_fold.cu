@@ -594,22 +594,29 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
 #pragma unroll 8
       for (int a = 0; a < n_a; ++a) gm = fmaxf(gm, gcol[(int64_t)s_creator[a] * p.Cmax]);
       const double bar = fmax(s_best[j], (double)gm - eps) - eps;
-      int cntc = 0;
+      // second and last pass over the row of products: the (few) contenders, kept in registers
+      int cntc = 0, ca[4] = {0, 0, 0, 0};
 #pragma unroll 8
-      for (int a = 0; a < n_a; ++a) cntc += ((double)gcol[(int64_t)s_creator[a] * p.Cmax] >= bar) ? 1 : 0;
-      bool exh = cntc > kPairPerTok;
+      for (int a = 0; a < n_a; ++a) {
+        if ((double)gcol[(int64_t)s_creator[a] * p.Cmax] >= bar) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            if (k == cntc) ca[k] = a;
+          ++cntc;
+        }
+      }
+      bool exh = cntc > 4;   // more than four contenders: every new row exactly
       int start = 0;
       if (!exh && cntc > 0) {
         start = atomicAdd(&s_np, cntc);
         if (start + cntc > kPairCap) exh = true;
       }
       if (!exh && cntc > 0) {
-        int w = start;
-        for (int a = 0; a < n_a; ++a) {
-          if ((double)gcol[(int64_t)s_creator[a] * p.Cmax] >= bar) {
-            s_prow[w] = a;                      // index of the new row, ascending within a token
-            s_ptok[w] = (unsigned short)j;
-            ++w;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (k < cntc) {
+            s_prow[start + k] = ca[k];          // index of the new row, ascending within a token
+            s_ptok[start + k] = (unsigned short)j;
           }
         }
         s_pstart[j] = start;
