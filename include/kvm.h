@@ -88,7 +88,7 @@ typedef struct {
   const float* tau_state;                          /* host [n_q_heads] or NULL = 1 (copied)               */
   const float* tau_bswa;                           /* host [n_q_heads] or NULL = 1 (copied)               */
   int32_t max_block;                               /* largest block C that will be used (<= 256)          */
-  int64_t max_state_slots;                         /* capacity in state rows (see kvm_plan_capacity)      */
+  int64_t max_state_slots;                         /* capacity in state rows (see kvm_plan_capacity), < 2^23 */
   int64_t max_call_tokens;                         /* largest n_tokens of one kvm_prefill call            */
   int64_t max_seq_len;                             /* only used with KVM_FLAG_RECORD_ASSIGN               */
   int32_t device;                                  /* CUDA device ordinal                                 */

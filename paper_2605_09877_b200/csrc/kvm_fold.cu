@@ -1,14 +1,21 @@
 // The fold of one overflow block into the state (Section 3.2 "Append", "Merge", budget rule,
 // value-radius preservation) for every unit:
-//   1. kbar_kernel          memory keys kbar_j = LN_s(zero_r(k_j))            (Eq. 1) in fp64
+//   1. kbar_kernel          memory keys kbar_j = LN_s(zero_r(k_j))            (Eq. 1) in fp64 and
+//                           fp16, the keys LN_s(kbar_j) of the rows the tokens would create (fp16, and
+//                           their LayerNorm statistics); computed for a batch of blocks ahead of the folds,
+//                           together with the tensor-core products LN_s(kbar_a) . kbar_j (new-row filter)
 //   2. routing filter       approximate similarities kbar_j . LN_s(s^K_i) in fp16 x fp16 -> fp32
 //                           (tcgen05 kernel in kvm_route_tc.cu, scalar-core cross-check here),
-//                           K best rows per token and per row split: candidates only
+//                           the rows within the rounding window of the best one, per token and row split
 //   3. fold_decide_kernel   exact fp64 similarities of the candidates, append selection, merge
-//                           routing against s_+, grouping of the merged tokens by target row
+//                           routing against s_+ (new rows: filtered by the products of step 1, the few
+//                           contenders exactly), grouping of the merged tokens by target row; several CTAs
+//                           per unit share the refinement, the last one to finish takes the block-wide steps
 //   4. fold_apply_kernel    one warp per touched row: creates appended rows, accumulates the
 //                           members in ascending token order (deterministic), refreshes the
-//                           readout cache (LN_s of the key sum, value-radius readout)
+//                           readout cache (LN_s of the key sum, value-radius readout) in the readout
+//                           copy of the new state version
+//   (prev_copy_kernel brings the rows the previous fold touched over to that copy first.)
 //
 // Integer decisions (which tokens are appended, which row each token merges into) are taken on
 // fp64 similarities computed from fp64 key sums, so they agree with an fp64 reference unless two
