@@ -39,7 +39,45 @@ struct AttnTcParams {
   float* part;       // split-KV partial results, [tile][split][D + 2][128] (see the epilogue)
   int32_t* part_cnt; // [tile] tickets, zero between launches
   int nq, Hq, Hkv, G;
+  int out_vec;       // rows of `out` can be written with 16-byte stores (alignment of base and strides)
 };
+
+// Output staging: a 128 x D bf16 tile, row-major in shared memory, the 16-byte chunks of a row
+// permuted by the row index so that neither the row-per-thread writes nor the row-contiguous reads
+// conflict on the banks.
+template <int D>
+__device__ __forceinline__ uint4* stage_chunk(uint8_t* stage, int row, int k) {
+  constexpr int CPR = D / 8;   // chunks per row
+  return reinterpret_cast<uint4*>(stage + row * (D * 2) + ((k ^ (row & (CPR - 1))) << 4));
+}
+// 32 fp32 accumulator values of one row -> four chunks (channels [32 c, 32 c + 32)), scaled
+template <int D>
+__device__ __forceinline__ void stage_row32(uint8_t* stage, int row, int c, const uint32_t (&r)[32], float inv) {
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[8 * q + 2 * i]) * inv, __uint_as_float(r[8 * q + 2 * i + 1]) * inv);
+      w[i] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    *stage_chunk<D>(stage, row, 4 * c + q) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+// One warp writes rows [row0, row0 + nrows) of the staged tile to global memory, 32 / (D / 8) rows
+// per instruction, every row as one contiguous run of 16-byte stores.
+template <int D>
+__device__ __forceinline__ void store_staged_rows(uint8_t* stage, __nv_bfloat16* out_row0, int64_t row_stride, int row0, int nrows,
+                                                  int rows_valid, int lane) {
+  constexpr int CPR = D / 8, RPI = 32 / CPR;
+  const int k = lane % CPR;
+  for (int r = row0 + lane / CPR; r < row0 + nrows; r += RPI) {
+    if (r < rows_valid) {
+      const uint4 v = *stage_chunk<D>(stage, r, k);
+      *reinterpret_cast<uint4*>(out_row0 + (int64_t)r * row_stride + k * 8) = v;
+    }
+  }
+}
 
 template <int D>
 struct AttnTcCfg {
@@ -361,7 +399,24 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     const bool good = ok && !*abort_flag;
     const float lsum2 = l_run + xl[(1 - half) * 128 + row];
     __nv_bfloat16* orow = p.out + bb * p.so0 + hq * p.so1 + (p.out_t0 + (int64_t)qt * 128 + row) * p.so2 + half * HD;
-    if (nsp == 1) {
+    if (nsp == 1 && p.out_vec) {
+      // rows go through shared memory (the key stages, idle by now) so that the global stores are
+      // whole rows of 16-byte pieces instead of one 4-byte piece per row and instruction
+      if (good) {
+        const float inv = 1.f / lsum2;
+#pragma unroll
+        for (int c = 0; c < HD / 32; ++c) {
+          uint32_t r[32];
+          tc::tmem_ld32(to_mine + c * 32, r);
+          tc::tmem_wait_ld();
+          stage_row32<D>(sK, row, half * (HD / 32) + c, r, inv);
+        }
+      }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (good)
+        store_staged_rows<D>(sK, p.out + bb * p.so0 + hq * p.so1 + (p.out_t0 + (int64_t)qt * 128) * p.so2, p.so2,
+                             (warp - 4) * 16, 16, rows_valid, lane);
+    } else if (nsp == 1) {
       if (good) {
         const float inv = 1.f / lsum2;
 #pragma unroll
@@ -469,6 +524,7 @@ int launch_attn_tc(State* st, const AttnArgs& a, cudaStream_t s) {
   p.out = a.out; p.tau_s = st->tau_s; p.tau_b = st->tau_b; p.status = st->status;
   p.nq = a.nq; p.Hq = st->Hq; p.Hkv = st->Hkv; p.G = st->G;
   p.part = st->attnPart; p.part_cnt = st->attnCnt;
+  p.out_vec = (reinterpret_cast<uintptr_t>(a.out) % 16 == 0 && a.so[0] % 8 == 0 && a.so[1] % 8 == 0 && a.so[2] % 8 == 0) ? 1 : 0;
   // key splits when there are few query tiles: up to a quarter of the GPU (the folds of the block
   // before run beside this kernel and are usually the longer chain; measured: a wider attention
   // kernel only takes SMs away from them), at least two key tiles per split
