@@ -135,6 +135,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   const int ntiles = min(ntot, jbase + per_split) - jbase;   // tiles of this CTA (0 is possible)
 
   if (tid == 0) {
+    tc::prefetch_tmap(&mapQ); tc::prefetch_tmap(&mapKs); tc::prefetch_tmap(&mapVs);
+    tc::prefetch_tmap(&mapKw); tc::prefetch_tmap(&mapVw);
     tc::mbar_init(&bars[BAR_QFULL], 1);
     for (int s = 0; s < 3; ++s) {
       tc::mbar_init(&bars[BAR_KFULL + s], 1);
@@ -150,6 +152,35 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     }
     *abort_flag = 0;
     tc::fence_barrier_init();
+  }
+  // Three key stages, two value stages: keys run two tiles ahead of the product that needs them,
+  // values one.  A K stage is released as soon as its QK^T product has completed, a V stage after
+  // its PV product.  (Called by thread 0 only.)
+  auto load_kv = [&](int j, bool keys) -> bool {
+    const int ns = keys ? Cfg::NS : Cfg::NSV;
+    const int s = j % ns;
+    if (j >= ns && !tc::mbar_wait(&bars[(keys ? BAR_KFREE : BAR_VFREE) + s], ((j / ns) - 1) & 1)) return false;
+    const int gj = jbase + j;
+    const bool st = gj < nst;
+    const int row = st ? gj * 128 : (int)(p.win_row0 + (int64_t)(gj - nst) * 128);
+    uint64_t* full = &bars[(keys ? BAR_KFULL : BAR_VFULL) + s];
+    uint8_t* dst = (keys ? sK : sV) + s * Cfg::TILE_BYTES;
+    const CUtensorMap* map = keys ? (st ? &mapKs : &mapKw) : (st ? &mapVs : &mapVw);
+    tc::mbar_expect_tx(full, Cfg::TILE_BYTES);
+    for (int kb = 0; kb < Cfg::NKB; ++kb)
+      tc::tma_load_3d(dst + kb * Cfg::BOX_BYTES, map, full, kb * 64, row, u);
+    return true;
+  };
+  if (tid == 0) {
+    // the first loads start before the tensor memory is allocated and the roles split: they need
+    // nothing but their own barriers (no stage is waited for yet)
+    tc::fence_proxy_async();
+    tc::mbar_expect_tx(&bars[BAR_QFULL], Cfg::TILE_BYTES);
+    for (int kb = 0; kb < Cfg::NKB; ++kb)
+      tc::tma_load_3d(sQ + kb * Cfg::BOX_BYTES, &mapQ, &bars[BAR_QFULL], kb * 64, (int)(p.q_row0 + qt * 128), bh);
+    if (ntiles > 0) load_kv(0, true);
+    if (ntiles > 1) load_kv(1, true);
+    if (ntiles > 0) load_kv(0, false);
   }
   if (warp == 1) {
     tc::tmem_alloc(tmem_slot, Cfg::TMEM_COLS);
@@ -170,33 +201,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     if (lane == 0) {
-      tc::prefetch_tmap(&mapQ); tc::prefetch_tmap(&mapKs); tc::prefetch_tmap(&mapVs);
-      tc::prefetch_tmap(&mapKw); tc::prefetch_tmap(&mapVw);
-      tc::mbar_expect_tx(&bars[BAR_QFULL], Cfg::TILE_BYTES);
-      for (int kb = 0; kb < Cfg::NKB; ++kb)
-        tc::tma_load_3d(sQ + kb * Cfg::BOX_BYTES, &mapQ, &bars[BAR_QFULL], kb * 64, (int)(p.q_row0 + qt * 128), bh);
-      // Three key stages, two value stages: keys run two tiles ahead of the product that needs them,
-      // values one.  A K stage is released as soon as its QK^T product has completed, a V stage after
-      // its PV product.
-      auto load_kv = [&](int j, bool keys) -> bool {
-        const int ns = keys ? Cfg::NS : Cfg::NSV;
-        const int s = j % ns;
-        if (j >= ns && !tc::mbar_wait(&bars[(keys ? BAR_KFREE : BAR_VFREE) + s], ((j / ns) - 1) & 1)) return false;
-        const int gj = jbase + j;
-        const bool st = gj < nst;
-        const int row = st ? gj * 128 : (int)(p.win_row0 + (int64_t)(gj - nst) * 128);
-        uint64_t* full = &bars[(keys ? BAR_KFULL : BAR_VFULL) + s];
-        uint8_t* dst = (keys ? sK : sV) + s * Cfg::TILE_BYTES;
-        const CUtensorMap* map = keys ? (st ? &mapKs : &mapKw) : (st ? &mapVs : &mapVw);
-        tc::mbar_expect_tx(full, Cfg::TILE_BYTES);
-        for (int kb = 0; kb < Cfg::NKB; ++kb)
-          tc::tma_load_3d(dst + kb * Cfg::BOX_BYTES, map, full, kb * 64, row, u);
-        return true;
-      };
       bool okp = true;
-      if (ntiles > 0) okp = load_kv(0, true);
-      if (okp && ntiles > 1) okp = load_kv(1, true);
-      if (okp && ntiles > 0) okp = load_kv(0, false);
       for (int j = 0; j < ntiles && okp; ++j) {
         if (*abort_flag) break;
         if (j + 2 < ntiles && !load_kv(j + 2, true)) { okp = false; break; }
