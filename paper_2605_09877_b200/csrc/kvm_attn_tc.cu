@@ -479,8 +479,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
 #pragma unroll
           for (int c = 0; c < HD; ++c) accv[c] += __ldcg(pz + (half * HD + c) * 128 + row) * wz;
         }
-        if (row < rows_valid) {
-          const float inv = 1.f / den;
+        const float inv = 1.f / den;
+        if (p.out_vec) {   // (uniform over the CTA, as is last_flag: every softmax thread reaches the barrier)
+#pragma unroll
+          for (int c = 0; c < HD / 8; ++c) {
+            uint32_t w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const __nv_bfloat162 h = __floats2bfloat162_rn(accv[8 * c + 2 * i] * inv, accv[8 * c + 2 * i + 1] * inv);
+              w[i] = *reinterpret_cast<const uint32_t*>(&h);
+            }
+            *stage_chunk<D>(sK, row, half * (HD / 8) + c) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+          asm volatile("bar.sync 1, 256;" ::: "memory");
+          store_staged_rows<D>(sK, p.out + bb * p.so0 + hq * p.so1 + (p.out_t0 + (int64_t)qt * 128) * p.so2, p.so2,
+                               (warp - 4) * 16, 16, rows_valid, lane);
+        } else if (row < rows_valid) {
 #pragma unroll
           for (int c = 0; c < HD / 2; ++c)
             reinterpret_cast<__nv_bfloat162*>(orow)[c] = __floats2bfloat162_rn(accv[2 * c] * inv, accv[2 * c + 1] * inv);
