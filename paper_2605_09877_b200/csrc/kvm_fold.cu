@@ -348,14 +348,15 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
     bet[i] = (double)p.ln_b[hk * D + lane + 32 * i];
   }
   if (tid == 0) { s_np = 0; s_nmerge = 0; s_nexh = 0; }
-  // everything above reads parameters only; the routing filter's lists are read from here on
-  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (tid < kMaxBlock) {
     s_app[tid] = 0; s_exh[tid] = 0; s_pcnt[tid] = 0; s_pstart[tid] = 0; s_pi[tid] = -1;
     s_best[tid] = -INFINITY; s_barg[tid] = -1; s_score[tid] = -INFINITY; s_creator[tid] = -1;
     s_gmaxi[tid] = (int)0x80000000; s_fill[tid] = 0; s_thr[tid] = 0.f;
-    if (tid < p.Cmax) p.segnew[tokBase + tid] = -1;
   }
+  // everything above reads parameters and writes shared memory only; the routing filter's lists are
+  // read, and global memory is written, from here on
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (tid < p.Cmax && tid < kMaxBlock) p.segnew[tokBase + tid] = -1;
   __syncthreads();
 
   // ---- A1/A2: candidate pairs from the filter lists.  The work items are (token of the slice, split),
@@ -431,6 +432,15 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
       start += cnt[k];
     }
     if (lane == 31) s_np = min(start, kPairCap);
+    int ne = 0;   // tokens of the slice that take the exhaustive path
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const int j = jlo + lane * 8 + k;
+      if (j < jhi) ne += s_exh[j];
+    }
+#pragma unroll
+    for (int o2 = 16; o2 > 0; o2 >>= 1) ne += __shfl_xor_sync(0xffffffffu, ne, o2);
+    if (lane == 0) s_nexh += ne;
   }
   __syncthreads();
   for (int it = tid; it < nitems; it += kDecideThreads) {
@@ -464,11 +474,6 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
     }
   }
   __syncthreads();
-  if (tid == 0) {
-    int ne = 0;
-    for (int j = jlo; j < jhi; ++j) ne += s_exh[j];
-    s_nexh += ne;
-  }
   // ---- A3: exact fp64 similarity of every candidate pair, one warp per pair, eight in flight
   //      (the loads of a pair hang on one another: pair list -> rows -> statistics) ----
   const int np = min(s_np, kPairCap);
@@ -962,14 +967,15 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
     p.C = C; p.Cmax = st->Cmax; p.Hkv = st->Hkv; p.S = st->S; p.n_append = a.n_append; p.nsplit = nsplit;
     p.thr_coeff = route_thr_coeff(st);
     KernelTimer kt(st, 4, s);
-    // CTAs per unit (measured on U = 8, 32, 256): about 64 CTAs in all, at least two per unit while
+    // CTAs per unit (measured on U = 1, 8, 32, 256): about 64 CTAs in all, at least two per unit while
     // 2U CTAs fit the GPU in one wave, at most eight, at least 16 tokens each - beyond that the
-    // hand-over costs more than the shorter slices save
+    // hand-over costs more than the shorter slices save.  A fold that appends nothing has few pairs
+    // to refine (most tokens have one candidate and need no exact similarity): one CTA per unit.
     int R = 64 / st->U;
     if (R < 2 && 2 * st->U <= 2 * 148) R = 2;
     if (R > 8) R = 8;
     if (R > C / 16) R = C / 16;
-    if (R < 1) R = 1;
+    if (R < 1 || a.n_append == 0) R = 1;
     dim3 dgrid(R, st->U);
     // programmatic dependent launch: the CTAs may start (and set up their shared memory) while the
     // routing filter is still running; they wait for it before the first read of its output
