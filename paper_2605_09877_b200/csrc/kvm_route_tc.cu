@@ -51,7 +51,7 @@ struct RouteTcCfg {
 enum { RB_AFULL = 0, RB_BFULL = 1, RB_BFREE = 4, RB_SFULL = 7, RB_ACCFREE = 9, RB_COUNT = 11 };
 
 template <int D>
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(352, 1)
 route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
                        const __grid_constant__ CUtensorMap mapH, const RouteTcParams p) {
   using Cfg = RouteTcCfg<D>;
@@ -82,10 +82,10 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
     tc::mbar_init(&bars[RB_AFULL], 1);
     for (int s = 0; s < Cfg::NS; ++s) {
       tc::mbar_init(&bars[RB_BFULL + s], 1);
-      tc::mbar_init(&bars[RB_BFREE + s], 1);
+      tc::mbar_init(&bars[RB_BFREE + s], mt_used);      // one commit per issuer
     }
-    tc::mbar_init(&bars[RB_SFULL + 0], 1);
-    tc::mbar_init(&bars[RB_SFULL + 1], 1);
+    tc::mbar_init(&bars[RB_SFULL + 0], mt_used);
+    tc::mbar_init(&bars[RB_SFULL + 1], mt_used);
     tc::mbar_init(&bars[RB_ACCFREE + 0], 4 * mt_used);
     tc::mbar_init(&bars[RB_ACCFREE + 1], 4 * mt_used);
     *abort_flag = 0;
@@ -115,7 +115,7 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
       asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int j = 0; j < nsteps; ++j) {
         const int s = j % Cfg::NS;
-        const int jt = j >= ntiles ? j - ntiles : j;
+        const int jt = j >= ntiles ? 2 * ntiles - 1 - j : j;   // pass 2 walks back: its first tiles are the ones pass 1 read last (L2)
         if (*abort_flag) break;
         if (j >= Cfg::NS && !tc::mbar_wait(&bars[RB_BFREE + s], ((j / Cfg::NS) - 1) & 1)) {
           atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; break;
@@ -126,8 +126,11 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
                           (int)(i0 + (int64_t)jt * 128), gram ? a_unit : u);
       }
     }
-  } else if (warp == 1) {
-    if (lane == 0) {
+  } else if (warp == 1 || warp == 10) {
+    // one issuer thread per 128-token M tile: issuing an MMA takes longer than executing it, so one
+    // thread cannot keep the pipe busy
+    const int mt = warp == 1 ? 0 : 1;
+    if (lane == 0 && mt < mt_used) {
       constexpr uint32_t IDESC = tc::idesc_f16(128, 128, false);
       const uint32_t aA = tc::smem_u32(sA), aB = tc::smem_u32(sB);
       bool dead = !tc::mbar_wait(&bars[RB_AFULL], 0);
@@ -137,14 +140,12 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
         if (!tc::mbar_wait(&bars[RB_BFULL + s], (j / Cfg::NS) & 1)) { dead = true; break; }
         if (j >= 2 && !tc::mbar_wait(&bars[RB_ACCFREE + buf], ((j >> 1) - 1) & 1)) { dead = true; break; }
         tc::tc_fence_after();
-        for (int mt = 0; mt < mt_used; ++mt) {
-          const uint32_t dS = tmem + buf * 256 + mt * 128;
+        const uint32_t dS = tmem + buf * 256 + mt * 128;
 #pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks) {
-            const uint32_t off = (ks / 4) * Cfg::BOX_BYTES + (ks % 4) * 32;
-            tc::mma_f16_ss(dS, tc::smem_desc_sw128(aA + mt * Cfg::TILE_BYTES + off, 16, 1024),
-                           tc::smem_desc_sw128(aB + s * Cfg::TILE_BYTES + off, 16, 1024), IDESC, ks > 0);
-          }
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint32_t off = (ks / 4) * Cfg::BOX_BYTES + (ks % 4) * 32;
+          tc::mma_f16_ss(dS, tc::smem_desc_sw128(aA + mt * Cfg::TILE_BYTES + off, 16, 1024),
+                         tc::smem_desc_sw128(aB + s * Cfg::TILE_BYTES + off, 16, 1024), IDESC, ks > 0);
         }
         tc::mma_commit(&bars[RB_SFULL + buf]);
         tc::mma_commit(&bars[RB_BFREE + s]);
@@ -168,7 +169,7 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
       for (int j = 0; j < nsteps; ++j) {
         const int buf = j & 1;
         const bool pass2 = j >= ntiles;
-        const int jt = pass2 ? j - ntiles : j;
+        const int jt = pass2 ? 2 * ntiles - 1 - j : j;
         if (j == ntiles) cut = mx - thr;
         if (!tc::mbar_wait(&bars[RB_SFULL + buf], (j >> 1) & 1)) {
           atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; break;
@@ -180,16 +181,18 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
         // pass 1 ignores the sink rows (< S) and the rows past the end of the split; pass 2 only the latter
         const int lo = pass2 ? 0 : max(0, p.S - row0);
         const bool plain = nvalid == 128 && lo == 0;
-#pragma unroll 1
+        // all 128 columns of the row go to registers in one round trip; the accumulator is handed
+        // back before they are looked at
+        uint32_t rr[4][32];
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) tc::tmem_ld32(ts + c4 * 32, rr[c4]);
+        tc::tmem_wait_ld();
+        tc::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(&bars[RB_ACCFREE + buf]);
+#pragma unroll
         for (int c4 = 0; c4 < 4; ++c4) {
-          uint32_t r[32];
-          tc::tmem_ld32(ts + c4 * 32, r);
-          tc::tmem_wait_ld();
-          if (c4 == 3) {   // all 128 columns are in registers: the accumulator may be overwritten
-            tc::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) tc::mbar_arrive(&bars[RB_ACCFREE + buf]);
-          }
+          uint32_t (&r)[32] = rr[c4];
           if (gram) {   // row `tok` of gramT: 32 consecutive tokens j = row0 + c4*32 .. (rows past C are never read)
             if (tok < p.C) {
               float* dst = p.gramT + ((int64_t)a_unit * p.Cmax + tok) * p.Cmax + row0 + c4 * 32;
@@ -268,7 +271,7 @@ int launch_route_filter_tc(State* st, int64_t m, int nsplit, int slot, cudaStrea
   // programmatic dependent launch behind the apply kernel of the previous fold: the CTAs set up and
   // fetch the block's memory keys while it finishes
   cudaLaunchConfig_t lc = {};
-  lc.gridDim = grid; lc.blockDim = dim3(320); lc.stream = s;
+  lc.gridDim = grid; lc.blockDim = dim3(352); lc.stream = s;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
@@ -287,8 +290,8 @@ int launch_gram_tc(State* st, int slot0, int nblk, cudaStream_t s) {
   p.a_unit0 = slot0 * st->U; p.gramT = st->gramT; p.gram_mode = 1; p.U = st->U;
   const CUtensorMap* tm = reinterpret_cast<const CUtensorMap*>(st->tmaps);
   dim3 grid(1, st->U, nblk);
-  if (st->d == 128) route_filter_tc_kernel<128><<<grid, 320, RouteTcCfg<128>::SMEM_BYTES, s>>>(tm[5], tm[1], tm[8], p);
-  else route_filter_tc_kernel<64><<<grid, 320, RouteTcCfg<64>::SMEM_BYTES, s>>>(tm[5], tm[1], tm[8], p);
+  if (st->d == 128) route_filter_tc_kernel<128><<<grid, 352, RouteTcCfg<128>::SMEM_BYTES, s>>>(tm[5], tm[1], tm[8], p);
+  else route_filter_tc_kernel<64><<<grid, 352, RouteTcCfg<64>::SMEM_BYTES, s>>>(tm[5], tm[1], tm[8], p);
   return 1;
 }
 
