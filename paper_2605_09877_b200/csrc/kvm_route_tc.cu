@@ -213,19 +213,21 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
             vm = (b <= a) ? 0u : ((b == 32 ? 0xffffffffu : ((1u << b) - 1u)) & ~((1u << a) - 1u));
           }
           if (!pass2) {
-            float cm = -INFINITY;
+            // four independent chains: one chain of 32 dependent maxima is latency-bound
+            float cm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
             if (plain) {
 #pragma unroll
-              for (int i = 0; i < 32; ++i) cm = fmaxf(cm, __uint_as_float(r[i]));
+              for (int i = 0; i < 32; ++i) cm[i & 3] = fmaxf(cm[i & 3], __uint_as_float(r[i]));
             } else {
 #pragma unroll
-              for (int i = 0; i < 32; ++i) cm = fmaxf(cm, ((vm >> i) & 1u) ? __uint_as_float(r[i]) : -INFINITY);
+              for (int i = 0; i < 32; ++i) cm[i & 3] = fmaxf(cm[i & 3], ((vm >> i) & 1u) ? __uint_as_float(r[i]) : -INFINITY);
             }
-            mx = fmaxf(mx, cm);
+            mx = fmaxf(mx, fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3])));
           } else {
-            uint32_t hit = 0u;
+            uint32_t h4[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-            for (int i = 0; i < 32; ++i) hit |= (__uint_as_float(r[i]) >= cut) ? (1u << i) : 0u;
+            for (int i = 0; i < 32; ++i) h4[i & 3] |= (__uint_as_float(r[i]) >= cut) ? (1u << i) : 0u;
+            uint32_t hit = (h4[0] | h4[1]) | (h4[2] | h4[3]);
             hit &= vm;
             while (hit) {   // rare per lane: about one candidate per token and split
               const int bit = __ffs(hit) - 1;
