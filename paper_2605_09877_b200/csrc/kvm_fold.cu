@@ -48,51 +48,101 @@ __device__ __forceinline__ void row_stats(const double (&x)[CH], int D, double e
 // ------------------------------------------------------------------------------------------
 // 1. memory keys (one warp per overflow token)
 
+// Four token rows per warp, eight lanes per row: every fp64 reduction step, divide and square root
+// is an instruction of the whole warp whatever the number of rows it serves, and with one row per
+// warp those made up most of the ~375 instructions per row (the kernel was bound by the fp64 pipe,
+// not by memory).  Lane `sub` of a row's group holds channels 32 i + 4 sub .. + 3, so that the eight
+// lanes of a group read and write contiguous runs.
+constexpr int kKbarRowsPerWarp = 4;
+constexpr int kKbarRowsPerCta = 8 * kKbarRowsPerWarp;
+
+__device__ __forceinline__ double group8_sum_d(double v) {
+#pragma unroll
+  for (int o = 4; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
 template <int D>
-__global__ void __launch_bounds__(256) kbar_kernel(const __half* __restrict__ ok, int64_t unit_stride,
-                                                   const float* __restrict__ ln_w, const float* __restrict__ ln_b,
-                                                   double* __restrict__ kbar64, __half* __restrict__ kbarH,
-                                                   float* __restrict__ kbarNorm, double2* __restrict__ kbarHatStat,
-                                                   __half* __restrict__ kbarHatH, int C, int Cmax, int CbarRows, int U, int Hkv, int r,
-                                                   double ln_eps) {
-  constexpr int CH = D / 32;
+__global__ void __launch_bounds__(256, 2) kbar_kernel(const __half* __restrict__ ok, int64_t unit_stride,
+                                                      const float* __restrict__ ln_w, const float* __restrict__ ln_b,
+                                                      double* __restrict__ kbar64, __half* __restrict__ kbarH,
+                                                      float* __restrict__ kbarNorm, double2* __restrict__ kbarHatStat,
+                                                      __half* __restrict__ kbarHatH, int C, int Cmax, int CbarRows, int U, int Hkv, int r,
+                                                      double ln_eps) {
+  constexpr int NI = D / 32;          // runs of four channels per lane
+  constexpr int NC = 4 * NI;          // channels per lane
+  constexpr double inv_d = 1.0 / D;   // D is a power of two: the multiplication is the division, exactly
   const int u = blockIdx.y, hk = u % Hkv;
   const int g = blockIdx.z;   // block of the batch = slot
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int j = blockIdx.x * 8 + warp;
-  if (j >= C) return;
-  const __half* row = ok + (int64_t)u * unit_stride + ((int64_t)g * C + j) * D;
-  double val[CH];
+  const int sub = lane & 7;
+  const int j = (blockIdx.x * 8 + warp) * kKbarRowsPerWarp + (lane >> 3);
+  const bool live = j < C;            // (dead groups compute a copy of the last row and store nothing:
+  const int jj = live ? j : C - 1;    //  the shuffles below need every lane)
+  const __half* row = ok + (int64_t)u * unit_stride + ((int64_t)g * C + jj) * D;
+  double val[NC];
 #pragma unroll
-  for (int i = 0; i < CH; ++i) {
-    const int x = lane + 32 * i;
-    val[i] = (x < r) ? 0.0 : (double)__half2float(row[x]);
+  for (int i = 0; i < NI; ++i) {
+    alignas(8) __half hv[4];
+    *reinterpret_cast<uint2*>(hv) = *reinterpret_cast<const uint2*>(row + 32 * i + 4 * sub);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) val[4 * i + e] = (32 * i + 4 * sub + e < r) ? 0.0 : (double)__half2float(hv[e]);
   }
-  double mean, rstd;
-  row_stats<CH>(val, D, ln_eps, mean, rstd);
-  double kb[CH];
+  double sum = 0.0;
+#pragma unroll
+  for (int c = 0; c < NC; ++c) sum += val[c];
+  const double mean = group8_sum_d(sum) * inv_d;
+  double dev = 0.0;
+#pragma unroll
+  for (int c = 0; c < NC; ++c) dev += (val[c] - mean) * (val[c] - mean);
+  const double rstd = 1.0 / sqrt(group8_sum_d(dev) * inv_d + ln_eps);
+  const int64_t o = (((int64_t)g * U + u) * Cmax + jj) * D;
+  const int64_t oh = (((int64_t)g * U + u) * CbarRows + jj) * D;
+  double kb[NC];
   double n2 = 0.0;
-  const int64_t o = (((int64_t)g * U + u) * Cmax + j) * D;
-  const int64_t oh = (((int64_t)g * U + u) * CbarRows + j) * D;
 #pragma unroll
-  for (int i = 0; i < CH; ++i) {
-    const int x = lane + 32 * i;
-    kb[i] = (double)ln_w[hk * D + x] * ((val[i] - mean) * rstd) + (double)ln_b[hk * D + x];
-    kbar64[o + x] = kb[i];
-    kbarH[oh + x] = __float2half_rn((float)kb[i]);
-    n2 += kb[i] * kb[i];
+  for (int i = 0; i < NI; ++i) {
+    const int x = 32 * i + 4 * sub;
+    const float4 w4 = *reinterpret_cast<const float4*>(ln_w + hk * D + x), b4 = *reinterpret_cast<const float4*>(ln_b + hk * D + x);
+    const float wv[4] = {w4.x, w4.y, w4.z, w4.w}, bv[4] = {b4.x, b4.y, b4.z, b4.w};
+    alignas(8) __half kh[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const double t = (double)wv[e] * ((val[4 * i + e] - mean) * rstd) + (double)bv[e];
+      kb[4 * i + e] = t;
+      kh[e] = __float2half_rn((float)t);
+      n2 += t * t;
+    }
+    if (live) {
+      reinterpret_cast<double2*>(kbar64 + o + x)[0] = make_double2(kb[4 * i], kb[4 * i + 1]);
+      reinterpret_cast<double2*>(kbar64 + o + x)[1] = make_double2(kb[4 * i + 2], kb[4 * i + 3]);
+      *reinterpret_cast<uint2*>(kbarH + oh + x) = *reinterpret_cast<const uint2*>(kh);
+    }
   }
-  n2 = warp_sum_d(n2);
+  n2 = group8_sum_d(n2);
   // LN_s applied to kbar itself: the readout key of the row that this token would create
-  double mu2, rs2;
-  row_stats<CH>(kb, D, ln_eps, mu2, rs2);
+  sum = 0.0;
 #pragma unroll
-  for (int i = 0; i < CH; ++i) {
-    const int x = lane + 32 * i;
-    const double hat = (double)ln_w[hk * D + x] * ((kb[i] - mu2) * rs2) + (double)ln_b[hk * D + x];
-    kbarHatH[oh + x] = __float2half_rn((float)hat);
+  for (int c = 0; c < NC; ++c) sum += kb[c];
+  const double mu2 = group8_sum_d(sum) * inv_d;
+  dev = 0.0;
+#pragma unroll
+  for (int c = 0; c < NC; ++c) dev += (kb[c] - mu2) * (kb[c] - mu2);
+  const double rs2 = 1.0 / sqrt(group8_sum_d(dev) * inv_d + ln_eps);
+#pragma unroll
+  for (int i = 0; i < NI; ++i) {
+    const int x = 32 * i + 4 * sub;
+    const float4 w4 = *reinterpret_cast<const float4*>(ln_w + hk * D + x), b4 = *reinterpret_cast<const float4*>(ln_b + hk * D + x);
+    const float wv[4] = {w4.x, w4.y, w4.z, w4.w}, bv[4] = {b4.x, b4.y, b4.z, b4.w};
+    alignas(8) __half kh[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const double hat = (double)wv[e] * ((kb[4 * i + e] - mu2) * rs2) + (double)bv[e];
+      kh[e] = __float2half_rn((float)hat);
+    }
+    if (live) *reinterpret_cast<uint2*>(kbarHatH + oh + x) = *reinterpret_cast<const uint2*>(kh);
   }
-  if (lane == 0) {
+  if (live && sub == 0) {
     kbarNorm[((int64_t)g * U + u) * Cmax + j] = (float)sqrt(n2) * 1.000001f;
     kbarHatStat[((int64_t)g * U + u) * Cmax + j] = make_double2(mu2, rs2);
   }
@@ -885,7 +935,7 @@ int launch_kbar(State* st, const __half* ok, int64_t unit_stride, int nblk, int 
   KernelTimer kt(st, 2, s);
   const int C = st->C, D = st->d;
   const int64_t U = st->U;
-  dim3 grid((C + 7) / 8, st->U, nblk);
+  dim3 grid((C + kKbarRowsPerCta - 1) / kKbarRowsPerCta, st->U, nblk);
   double* k64 = st->kbar64 + (int64_t)slot0 * U * st->Cmax * D;
   __half* kh = st->kbarH + (int64_t)slot0 * U * st->CbarRows * D;
   float* kn = st->kbarNorm + (int64_t)slot0 * U * st->Cmax;
