@@ -218,6 +218,9 @@ def test_api_errors_leave_state_usable():
     with pytest.raises(kvm.KVMError) as e:
         st.decode_step(q[:, :, 0].contiguous(), k[:, :, 0].contiguous(), v[:, :, 0].contiguous())
     assert e.value.code == 5                   # decode before any prefill fixed the block
+    with pytest.raises(kvm.KVMError) as e:
+        st.prefill(q[:, :, :0], k[:, :, :0], v[:, :, :0], 64, g, 0)   # an empty call is rejected, not ignored
+    assert e.value.code == 1
     st.prefill(q[:, :, :64], k[:, :, :64], v[:, :, :64], 64, g, 0)
     with pytest.raises(kvm.KVMError) as e:
         st.prefill(q[:, :, 64:], k[:, :, 64:], v[:, :, 64:], 32, g, 0)
