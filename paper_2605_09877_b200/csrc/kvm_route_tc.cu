@@ -9,11 +9,12 @@
 // element instead of a sorted insertion.
 //
 //   warp 0      TMA producer: the Kbar tiles once, then 128-row tiles of K_hat in a 3-stage ring
-//   warp 1      MMA issuer: per key tile one 128x128x(d) product per M tile into a
+//   warps 1, 10 MMA issuers, one thread per M tile: per key tile one 128x128x(d) product into a
 //               double-buffered TMEM accumulator (tcgen05.mma kind::f16)
 //   warps 2-9   epilogue: one thread per token row; tcgen05.ld of its 128 similarities, running
 //               maximum (pass 1) / list of at most kTopK candidate rows (pass 2) in registers.
-// Output per (unit, split, token): candI[0..kTopK) candidate rows in ascending order (-1 = none),
+//               Pass 2 walks the tiles in the opposite direction.
+// Output per (unit, split, token): candI[0..kTopK) candidate rows in the order found (-1 = none),
 // candV[0] = the split's maximum over rows >= S, candV[1] = number of candidates found (more than
 // kTopK = the list overflowed and the decision kernel scans all rows for that token).
 // All waits are bounded (error word + normal teardown on expiry).
