@@ -375,6 +375,7 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
   __shared__ unsigned short s_ptok[kPairCap];
   __shared__ double s_pval[kPairCap];
   __shared__ int s_np, s_nmerge, s_nexh, s_last;
+  __shared__ int s_wsum[kDecideWarps];
   __shared__ int s_gmaxi[kMaxBlock], s_fill[kMaxBlock];
   __shared__ float s_thr[kMaxBlock];
 
@@ -444,53 +445,42 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
     if (c > 0) atomicAdd(&s_pcnt[j], c);
   }
   __syncthreads();
-  if (warp == 0) {   // segment starts: exclusive prefix sum over the slice's tokens, eight per lane
-    int cnt[8], tot = 0;
-    unsigned single = 0u;
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      const int j = jlo + lane * 8 + k;
-      int c = 0;
-      if (j < jhi) {
-        c = s_pcnt[j];
-        if (c > kPairPerTok) { s_exh[j] = 1; }
-        if (s_exh[j]) c = 0;
-        // A fold that appends nothing needs no scores, and the true arg max is always among the
-        // candidates: a token with a single candidate is decided without the exact similarity
-        // (it takes no room in the pair list).
-        if (n_a == 0 && c == 1) { single |= 1u << k; c = 0; }
-      }
-      cnt[k] = c;
-      tot += c;
+  {   // segment starts: exclusive prefix sum over the slice's tokens, one token per thread
+    const int j = jlo + tid;
+    const bool mine = tid < nslice;
+    int c = 0;
+    bool exh = false, single = false;
+    if (mine) {
+      c = s_pcnt[j];
+      exh = s_exh[j] != 0 || c > kPairPerTok;
+      if (exh) c = 0;
+      // A fold that appends nothing needs no scores, and the true arg max is always among the
+      // candidates: a token with a single candidate is decided without the exact similarity
+      // (it takes no room in the pair list).
+      if (n_a == 0 && c == 1) { single = true; c = 0; }
     }
-    int incl = tot;
+    int incl = c;
 #pragma unroll
     for (int o2 = 1; o2 < 32; o2 <<= 1) {
       const int v = __shfl_up_sync(0xffffffffu, incl, o2);
       if (lane >= o2) incl += v;
     }
-    int start = incl - tot;
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      const int j = jlo + lane * 8 + k;
-      if (j < jhi) {
-        if (start + cnt[k] > kPairCap) { s_exh[j] = 1; cnt[k] = 0; }   // the list is full: exact scan instead
-        s_pstart[j] = start;
-        s_pcnt[j] = cnt[k];
-        s_fill[j] = ((single >> k) & 1u) ? -1 : 0;
-      }
-      start += cnt[k];
+    if (lane == 31) s_wsum[warp] = incl;
+    __syncthreads();
+    int start = incl - c;
+    for (int w = 0; w < warp; ++w) start += s_wsum[w];
+    if (mine) {
+      // a list that would pass the end of the pair buffer is dropped (so are the lists behind it):
+      // those tokens are scanned exactly instead
+      if (start + c > kPairCap) { exh = true; c = 0; }
+      s_pstart[j] = start;
+      s_pcnt[j] = c;
+      s_fill[j] = (single && !exh) ? -1 : 0;
+      s_exh[j] = exh ? 1 : 0;
+      if (c > 0) atomicMax(&s_np, start + c);   // pairs of the lists that were kept form a prefix of the buffer
     }
-    if (lane == 31) s_np = min(start, kPairCap);
-    int ne = 0;   // tokens of the slice that take the exhaustive path
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      const int j = jlo + lane * 8 + k;
-      if (j < jhi) ne += s_exh[j];
-    }
-#pragma unroll
-    for (int o2 = 16; o2 > 0; o2 >>= 1) ne += __shfl_xor_sync(0xffffffffu, ne, o2);
-    if (lane == 0) s_nexh += ne;
+    const int ne = __syncthreads_count(mine && exh);   // tokens of the slice that take the exhaustive path
+    if (tid == 0) s_nexh += ne;
   }
   __syncthreads();
   for (int it = tid; it < nitems; it += kDecideThreads) {
