@@ -338,13 +338,14 @@ __device__ __forceinline__ double warp_sim(const double (&kb)[CH], const double*
   return warp_sum_d(acc);
 }
 
-// Bitonic sort of 256 (key, val) pairs, ascending by key and then val, held one per thread by the
-// first 256 threads of the CTA (the only callers; the others must not call): stages that stay inside a
-// warp exchange through shuffles, the six that cross warps through shared memory (sk / sv, 256 entries
-// each) and a named barrier of those 256 threads.  Afterwards thread t holds the pair of rank t.
-template <typename K>
-__device__ __forceinline__ void sort256(K& key, int& val, K* sk, int* sv, int t) {
-  for (int k = 2; k <= 256; k <<= 1) {
+// Bitonic sort of N = 128 or 256 (key, val) pairs, ascending by key and then val, held one per thread
+// by the first N threads of the CTA (the only callers; the others must not call): stages that stay
+// inside a warp exchange through shuffles, those that cross warps (three for 128, six for 256) through
+// shared memory (sk / sv, N entries each) and a named barrier of those N threads.  Afterwards thread t
+// holds the pair of rank t.
+template <typename K, int N>
+__device__ __forceinline__ void sort_n(K& key, int& val, K* sk, int* sv, int t) {
+  for (int k = 2; k <= N; k <<= 1) {
     for (int j = k >> 1; j > 0; j >>= 1) {
       K ok;
       int ov;
@@ -353,9 +354,9 @@ __device__ __forceinline__ void sort256(K& key, int& val, K* sk, int* sv, int t)
         ov = __shfl_xor_sync(0xffffffffu, val, j);
       } else {
         sk[t] = key; sv[t] = val;
-        asm volatile("bar.sync 2, 256;" ::: "memory");
+        asm volatile("bar.sync 2, %0;" ::"n"(N) : "memory");
         ok = sk[t ^ j]; ov = sv[t ^ j];
-        asm volatile("bar.sync 2, 256;" ::: "memory");
+        asm volatile("bar.sync 2, %0;" ::"n"(N) : "memory");
       }
       const bool take_min = ((t & j) == 0) == ((t & k) == 0);   // lower index of the pair in an ascending run
       const bool other_less = ok < key || (ok == key && ov < val);
@@ -384,6 +385,7 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
   const int u = blockIdx.y, hk = u % p.Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int C = p.C;
+  const int nsort = C <= 128 ? 128 : 256;   // threads that take part in the block-wide sorts
   const int R = gridDim.x;
   const int jlo = (int)blockIdx.x * ((C + R - 1) / R), jhi = min(C, jlo + (C + R - 1) / R);
   const int64_t m = p.m;
@@ -601,14 +603,16 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
   // ---- B: append selection: the n_a smallest scores, ties to the smaller token index ----
   if (n_a > 0) {
     // sort (score, token) ascending; the first n_a entries are appended
-    if (tid < 256) {
+    if (tid < nsort) {
       unsigned long long kbits = ~0ull;
       if (tid < C) {   // order-preserving integer image of the double
         const long long bits = __double_as_longlong(s_score[tid]);
         kbits = (unsigned long long)bits ^ (bits < 0 ? ~0ull : 0x8000000000000000ull);
       }
       int tok = tid;
-      sort256<unsigned long long>(kbits, tok, reinterpret_cast<unsigned long long*>(s_pval), s_prow, tid);   // (the pair list is idle here)
+      // (the pair list is idle here)
+      if (nsort == 128) sort_n<unsigned long long, 128>(kbits, tok, reinterpret_cast<unsigned long long*>(s_pval), s_prow, tid);
+      else sort_n<unsigned long long, 256>(kbits, tok, reinterpret_cast<unsigned long long*>(s_pval), s_prow, tid);
       if (tok < C) s_app[tok] = tid < n_a ? 1 : 0;
     }
     __syncthreads();
@@ -747,7 +751,7 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
   // ---- E: order merged tokens by (row, token); publish ----
   {
     unsigned* ekey = reinterpret_cast<unsigned*>(s_prow);   // (the pair list is idle here)
-    if (tid < 256) {
+    if (tid < nsort) {
       const int pj = tid < C ? s_pi[tid] : -1;
       unsigned kq = pj >= 0 ? (((unsigned)pj << 9) | (unsigned)tid) : 0xffffffffu;   // rows < 2^23, tokens < 2^9
       if (tid < C) {
@@ -755,9 +759,10 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
         p.creator[tokBase + tid] = s_creator[tid];
       }
       int zero = 0;
-      sort256<unsigned>(kq, zero, ekey + 256, reinterpret_cast<int*>(s_pval), tid);
+      if (nsort == 128) sort_n<unsigned, 128>(kq, zero, ekey + 256, reinterpret_cast<int*>(s_pval), tid);
+      else sort_n<unsigned, 256>(kq, zero, ekey + 256, reinterpret_cast<int*>(s_pval), tid);
       ekey[tid] = kq;
-      asm volatile("bar.sync 2, 256;" ::: "memory");
+      asm volatile("bar.sync 2, %0;" ::"r"(nsort) : "memory");
       if (kq != 0xffffffffu) {
         const int rowq = (int)(kq >> 9);
         p.sorted[tokBase + tid] = (int)(kq & 511u);
