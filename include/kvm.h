@@ -57,13 +57,24 @@ typedef enum {
  *   FIXED      B(e) = fixed_slots                        ("KVM 256")
  *   SQRT       B(e) = floor(sqrt_coeff * sqrt(e))        ("KVM sqrt", coeff 16), exact integer
  *   UNBOUNDED  B(e) = infinity (every overflow token is appended; test limit in
- *              which the layer never compresses)                                 */
-typedef enum { KVM_GROWTH_FIXED = 0, KVM_GROWTH_SQRT = 1, KVM_GROWTH_UNBOUNDED = 2 } kvm_growth_kind_t;
+ *              which the layer never compresses)
+ * and the two further shapes the paper names without a formula ("power-law", "saturating";
+ * the figure that shows them is all it gives), each with an exact integer definition:
+ *   POWER      B(e) = floor(sqrt_coeff * e^(pow_num/pow_den)) = the largest n with
+ *              n^pow_den <= sqrt_coeff^pow_den * e^pow_num (SQRT is pow 1/2);
+ *              1 <= pow_num <= pow_den <= 4, sqrt_coeff <= 1024, positions below 2^26
+ *   SATURATING B(e) = floor(fixed_slots * e / (e + sat_half)): half of fixed_slots at
+ *              e = sat_half, approaching fixed_slots from below; sat_half >= 1            */
+typedef enum { KVM_GROWTH_FIXED = 0, KVM_GROWTH_SQRT = 1, KVM_GROWTH_UNBOUNDED = 2,
+               KVM_GROWTH_POWER = 3, KVM_GROWTH_SATURATING = 4 } kvm_growth_kind_t;
 
 typedef struct {
   int32_t kind;        /* kvm_growth_kind_t */
-  int32_t sqrt_coeff;  /* SQRT only; the paper uses 16 */
-  int64_t fixed_slots; /* FIXED only; values below the block are clamped up by the rule itself */
+  int32_t sqrt_coeff;  /* SQRT, POWER: the coefficient; the paper uses 16 */
+  int64_t fixed_slots; /* FIXED: the budget (values below the block are clamped up by the rule itself);
+                          SATURATING: the limit */
+  int32_t pow_num, pow_den; /* POWER only */
+  int64_t sat_half;    /* SATURATING only */
 } kvm_growth_t;
 
 /* Element strides for dims (batch, head, token, channel); channel stride must be 1. */

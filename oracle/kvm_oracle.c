@@ -47,12 +47,14 @@ static int omp_in_parallel(void) { return 0; }
 typedef struct {
   int32_t B, Hq, Hkv, d;
   int32_t C, w, S, r;
-  int32_t growth_kind; /* 0 fixed, 1 sqrt, 2 unbounded */
+  int32_t growth_kind; /* 0 fixed, 1 sqrt, 2 unbounded, 3 power, 4 saturating */
   int32_t sqrt_coeff;
   int64_t fixed_slots;
   double rope_base, ln_eps, norm_eps;
   int32_t radius_on; /* 1: rho * s^V / max(||s^V||, eps) ; 0: s^V / weight (ablation) */
   int32_t reserved;
+  int32_t pow_num, pow_den; /* power:      B(e) = floor(sqrt_coeff * e^(pow_num/pow_den)) */
+  int64_t sat_half;         /* saturating: B(e) = floor(fixed_slots * e / (e + sat_half)) */
 } kvm_oracle_cfg;
 
 typedef struct {
@@ -137,6 +139,26 @@ static int64_t budget(const kvm_oracle_cfg* c, int64_t e) {
   if (c->growth_kind == 0) return c->fixed_slots;
   if (c->growth_kind == 1)
     return (int64_t)isqrt_u64((uint64_t)c->sqrt_coeff * (uint64_t)c->sqrt_coeff * (uint64_t)e);
+  if (c->growth_kind == 3) {
+    /* Power law (the paper names the shape, Section 3.2 and the schedule figure, without a formula;
+     * reading: floor(a e^(p/q)), the integer n with n^q <= a^q e^p < (n+1)^q).  A floating-point
+     * estimate, then corrected in exact 128-bit integer arithmetic. */
+    unsigned __int128 rhs = 1;
+    for (int i = 0; i < c->pow_den; ++i) rhs *= (unsigned __int128)c->sqrt_coeff;
+    for (int i = 0; i < c->pow_num; ++i) rhs *= (unsigned __int128)e;
+    int64_t n = (int64_t)((double)c->sqrt_coeff * pow((double)e, (double)c->pow_num / (double)c->pow_den));
+    if (n < 0) n = 0;
+    for (;;) {
+      unsigned __int128 lo = 1, hi = 1;
+      for (int i = 0; i < c->pow_den; ++i) { lo *= (unsigned __int128)n; hi *= (unsigned __int128)(n + 1); }
+      if (lo > rhs) --n;
+      else if (hi <= rhs) ++n;
+      else break;
+    }
+    return n;
+  }
+  if (c->growth_kind == 4) /* saturating: rational reading, exact */
+    return (int64_t)(((unsigned __int128)c->fixed_slots * (unsigned __int128)e) / (unsigned __int128)(e + c->sat_half));
   return INT64_MAX / 4;
 }
 

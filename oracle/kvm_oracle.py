@@ -12,7 +12,7 @@ import numpy as np
 
 from . import build as _build
 
-GROWTH = {"fixed": 0, "sqrt": 1, "unbounded": 2}
+GROWTH = {"fixed": 0, "sqrt": 1, "unbounded": 2, "power": 3, "saturating": 4}
 
 
 class _Cfg(C.Structure):
@@ -22,6 +22,7 @@ class _Cfg(C.Structure):
         ("growth_kind", C.c_int32), ("sqrt_coeff", C.c_int32), ("fixed_slots", C.c_int64),
         ("rope_base", C.c_double), ("ln_eps", C.c_double), ("norm_eps", C.c_double),
         ("radius_on", C.c_int32), ("reserved", C.c_int32),
+        ("pow_num", C.c_int32), ("pow_den", C.c_int32), ("sat_half", C.c_int64),
     ]
 
 
@@ -72,6 +73,9 @@ class OracleConfig:
     growth: str = "fixed"
     fixed_slots: int = 0
     sqrt_coeff: int = 16
+    pow_num: int = 1      # "power": floor(sqrt_coeff * e^(pow_num/pow_den))
+    pow_den: int = 2
+    sat_half: int = 0     # "saturating": floor(fixed_slots * e / (e + sat_half))
     rope_base: float = 10000.0
     ln_eps: float = 1e-5
     norm_eps: float = 1e-12
@@ -85,7 +89,7 @@ class KVMOracle:
         self.cfg = cfg
         c = _Cfg(cfg.B, cfg.Hq, cfg.Hkv, cfg.d, cfg.C, cfg.w, cfg.S, cfg.r, GROWTH[cfg.growth],
                  cfg.sqrt_coeff, cfg.fixed_slots, cfg.rope_base, cfg.ln_eps, cfg.norm_eps,
-                 1 if cfg.radius_on else 0, 0)
+                 1 if cfg.radius_on else 0, 0, cfg.pow_num, cfg.pow_den, cfg.sat_half)
         ln_w, ln_b, tau_s, tau_b = _f64(ln_w), _f64(ln_b), _f64(tau_s), _f64(tau_b)
         if ln_w is not None:
             assert ln_w.shape == (cfg.Hkv, cfg.d)

@@ -58,6 +58,24 @@ uint64_t isqrt_u64(uint64_t x) {
 int64_t budget(const kvm_growth_t& g, int64_t e) {
   if (g.kind == KVM_GROWTH_FIXED) return g.fixed_slots;
   if (g.kind == KVM_GROWTH_SQRT) return (int64_t)isqrt_u64((uint64_t)g.sqrt_coeff * (uint64_t)g.sqrt_coeff * (uint64_t)e);
+  if (g.kind == KVM_GROWTH_POWER) {
+    // floor(a * e^(p/q)) = the largest n with n^q <= a^q * e^p, by bisection in 128-bit integers
+    // (a <= 2^10, q <= 4, e < 2^26: the right-hand side stays below 2^118)
+    typedef unsigned __int128 u128;
+    u128 rhs = 1;
+    for (int i = 0; i < g.pow_den; ++i) rhs *= (u128)g.sqrt_coeff;
+    for (int i = 0; i < g.pow_num; ++i) rhs *= (u128)e;
+    int64_t lo = 0, hi = (int64_t)g.sqrt_coeff * e;   // p <= q: the budget is at most a * e
+    while (lo < hi) {
+      const int64_t mid = lo + (hi - lo + 1) / 2;
+      u128 pw = 1;
+      for (int i = 0; i < g.pow_den; ++i) pw *= (u128)mid;
+      if (pw <= rhs) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+  }
+  if (g.kind == KVM_GROWTH_SATURATING)
+    return (int64_t)(((unsigned __int128)g.fixed_slots * (unsigned __int128)e) / (unsigned __int128)(e + g.sat_half));
   return INT64_MAX / 4;
 }
 
@@ -73,13 +91,19 @@ int64_t n_append_of(const kvm_growth_t& g, int64_t e, int64_t m, int C) {
 bool growth_valid(const kvm_growth_t& g) {
   if (g.kind == KVM_GROWTH_FIXED) return g.fixed_slots >= 1;
   if (g.kind == KVM_GROWTH_SQRT) return g.sqrt_coeff >= 1 && g.sqrt_coeff <= 65535;
+  if (g.kind == KVM_GROWTH_POWER)
+    return g.sqrt_coeff >= 1 && g.sqrt_coeff <= 1024 && g.pow_num >= 1 && g.pow_num <= g.pow_den && g.pow_den <= 4;
+  if (g.kind == KVM_GROWTH_SATURATING) return g.fixed_slots >= 1 && g.sat_half >= 1;
   return g.kind == KVM_GROWTH_UNBOUNDED;
 }
+constexpr int64_t kPowerMaxPos = (int64_t)1 << 26;   // positions the POWER budget is defined for
 
 bool growth_equal(const kvm_growth_t& a, const kvm_growth_t& b) {
   if (a.kind != b.kind) return false;
   if (a.kind == KVM_GROWTH_FIXED) return a.fixed_slots == b.fixed_slots;
   if (a.kind == KVM_GROWTH_SQRT) return a.sqrt_coeff == b.sqrt_coeff;
+  if (a.kind == KVM_GROWTH_POWER) return a.sqrt_coeff == b.sqrt_coeff && a.pow_num == b.pow_num && a.pow_den == b.pow_den;
+  if (a.kind == KVM_GROWTH_SATURATING) return a.fixed_slots == b.fixed_slots && a.sat_half == b.sat_half;
   return true;
 }
 
@@ -192,6 +216,7 @@ KVM_API const char* kvm_status_string(kvm_status_t s) {
 
 KVM_API int64_t kvm_plan_capacity(int32_t block, int32_t n_bswa_chunks, kvm_growth_t growth, int64_t seq_len) {
   if (block < 1 || n_bswa_chunks < 1 || seq_len < 0 || !growth_valid(growth)) return -1;
+  if (growth.kind == KVM_GROWTH_POWER && seq_len >= kPowerMaxPos) return -1;
   int64_t m = 0;
   for (int64_t c = n_bswa_chunks - 1; (c + 1) * block <= seq_len; ++c) {
     const int64_t e = (c + 1) * block;
@@ -443,6 +468,7 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
   const int C = s.C;
   const int64_t L = (int64_t)s.w * C;
   const int64_t pos0 = s.pos, pos1 = pos0 + n;
+  if (s.growth.kind == KVM_GROWTH_POWER && pos1 >= kPowerMaxPos) return KVM_ERR_UNSUPPORTED;
   const int64_t c0 = pos0 / C, c_last = (pos1 - 1) / C;
 
   // capacity: the row count after this call follows from the budget rule alone
@@ -595,6 +621,7 @@ KVM_API kvm_status_t kvm_decode_step(const void* q, const void* k, const void* v
   const int C = s.C, d = s.d;
   const int64_t L = (int64_t)s.w * C;
   const int64_t t = s.pos, c = t / C, e = (c + 1) * C;
+  if (s.growth.kind == KVM_GROWTH_POWER && e >= kPowerMaxPos) return KVM_ERR_UNSUPPORTED;
   int64_t b = e - L; if (b < 0) b = 0;
   const bool fold = ((t + 1) % C == 0) && c >= s.w - 1;
   int n_a = 0;

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libkvm.so")
 KVM_OK = 0
 STATUS = {0: "KVM_OK", 1: "KVM_ERR_INVALID_ARG", 2: "KVM_ERR_UNSUPPORTED", 3: "KVM_ERR_OOM",
           4: "KVM_ERR_CUDA", 5: "KVM_ERR_STATE_MISMATCH", 6: "KVM_ERR_CAPACITY", 7: "KVM_ERR_TIMEOUT"}
-GROWTH_FIXED, GROWTH_SQRT, GROWTH_UNBOUNDED = 0, 1, 2
+GROWTH_FIXED, GROWTH_SQRT, GROWTH_UNBOUNDED, GROWTH_POWER, GROWTH_SATURATING = 0, 1, 2, 3, 4
 FLAG_NO_RADIUS, FLAG_RECORD_ASSIGN, FLAG_SIMT_ATTENTION, FLAG_SIMT_ROUTING = 1, 2, 4, 8
 
 EXPORTS = ["kvm_plan_capacity", "kvm_state_create", "kvm_prefill", "kvm_decode_step", "kvm_prefill_host",
@@ -35,7 +35,8 @@ class KVMError(RuntimeError):
 
 
 class Growth(C.Structure):
-    _fields_ = [("kind", C.c_int32), ("sqrt_coeff", C.c_int32), ("fixed_slots", C.c_int64)]
+    _fields_ = [("kind", C.c_int32), ("sqrt_coeff", C.c_int32), ("fixed_slots", C.c_int64),
+                ("pow_num", C.c_int32), ("pow_den", C.c_int32), ("sat_half", C.c_int64)]
 
 
 class Strides(C.Structure):
@@ -102,9 +103,13 @@ def _load():
 lib = _load()
 
 
-def growth(kind: str, fixed_slots: int = 0, sqrt_coeff: int = 16) -> Growth:
-    k = {"fixed": GROWTH_FIXED, "sqrt": GROWTH_SQRT, "unbounded": GROWTH_UNBOUNDED}[kind]
-    return Growth(k, sqrt_coeff, fixed_slots)
+def growth(kind: str, fixed_slots: int = 0, sqrt_coeff: int = 16, pow_num: int = 1, pow_den: int = 2,
+           sat_half: int = 0) -> Growth:
+    """fixed: B = fixed_slots; sqrt: floor(sqrt_coeff sqrt(e)); power: floor(sqrt_coeff e^(pow_num/pow_den));
+    saturating: floor(fixed_slots e / (e + sat_half)); unbounded: no budget."""
+    k = {"fixed": GROWTH_FIXED, "sqrt": GROWTH_SQRT, "unbounded": GROWTH_UNBOUNDED, "power": GROWTH_POWER,
+         "saturating": GROWTH_SATURATING}[kind]
+    return Growth(k, sqrt_coeff, fixed_slots, pow_num, pow_den, sat_half)
 
 
 def kvm_plan_capacity(block: int, n_bswa_chunks: int, g: Growth, seq_len: int) -> int:

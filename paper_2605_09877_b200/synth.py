@@ -24,9 +24,12 @@ class Workload:
     d: int
     T: int
     C: int
-    growth: str          # "fixed" | "sqrt" | "unbounded"
+    growth: str          # "fixed" | "sqrt" | "unbounded" | "power" | "saturating"
     fixed_slots: int = 0
     sqrt_coeff: int = 16
+    pow_num: int = 1     # "power": budget floor(sqrt_coeff * e^(pow_num/pow_den))
+    pow_den: int = 2
+    sat_half: int = 0    # "saturating": budget floor(fixed_slots * e / (e + sat_half))
     r: int = 0           # rope_dims
     w: int = 2           # n_bswa_chunks
     S: int = 1           # sink rows

@@ -21,7 +21,8 @@ def oracle_config(wl: synth.Workload, n_units=None, radius_on=True, ln_eps=1e-5)
         G = wl.Hq // wl.Hkv
         B, Hq, Hkv = 1, n_units * G, n_units
     return OracleConfig(B=B, Hq=Hq, Hkv=Hkv, d=wl.d, C=wl.C, w=wl.w, S=wl.S, r=wl.r, growth=wl.growth,
-                        fixed_slots=wl.fixed_slots, sqrt_coeff=wl.sqrt_coeff, radius_on=radius_on, ln_eps=ln_eps)
+                        fixed_slots=wl.fixed_slots, sqrt_coeff=wl.sqrt_coeff, pow_num=wl.pow_num, pow_den=wl.pow_den,
+                        sat_half=wl.sat_half, radius_on=radius_on, ln_eps=ln_eps)
 
 
 def to_f64(t):
@@ -49,7 +50,7 @@ def select_units(wl, tensors, units, params):
 def gpu_layer(wl, params, flags=0, max_call_tokens=None, max_seq_len=None, radius_on=True, ln_eps=1e-5,
               extra_tokens=0):
     from paper_2605_09877_b200 import kvm
-    g = kvm.growth(wl.growth, wl.fixed_slots, wl.sqrt_coeff)
+    g = kvm.growth(wl.growth, wl.fixed_slots, wl.sqrt_coeff, wl.pow_num, wl.pow_den, wl.sat_half)
     total = wl.T + extra_tokens
     cap = max(kvm.kvm_plan_capacity(wl.C, wl.w, g, total), wl.C)
     fl = flags | kvm.FLAG_RECORD_ASSIGN | (0 if radius_on else kvm.FLAG_NO_RADIUS)

@@ -51,6 +51,26 @@ def test_plan_capacity_matches_the_budget_rule_closed_forms(kvm):
     assert kvm.kvm_plan_capacity(0, 2, g, 100) == -1
 
 
+def test_plan_capacity_power_and_saturating_schedules(kvm):
+    # floor(16 e^(1/2)) is the sqrt schedule
+    gp = kvm.growth("power", sqrt_coeff=16, pow_num=1, pow_den=2)
+    for e, m in ((768, 443), (1024, 512), (32768, 2896), (131072, 5792)):
+        assert kvm.kvm_plan_capacity(256, 2, gp, e) == m
+    # exact integer floors: rows = the largest n with n^3 <= 8^3 e^2 once the budget has passed one block
+    g23 = kvm.growth("power", sqrt_coeff=8, pow_num=2, pow_den=3)
+    for e in (4096, 8192, 65536, 1 << 20):
+        n = kvm.kvm_plan_capacity(32, 2, g23, e)
+        assert n ** 3 <= 8 ** 3 * e ** 2 < (n + 1) ** 3, (e, n)
+    gs = kvm.growth("saturating", fixed_slots=1024, sat_half=4096)
+    assert kvm.kvm_plan_capacity(64, 2, gs, 4096) == 512
+    assert kvm.kvm_plan_capacity(64, 2, gs, 1 << 22) == (1024 * (1 << 22)) // ((1 << 22) + 4096) == 1023
+    # parameters outside the defined range
+    assert kvm.kvm_plan_capacity(64, 2, kvm.growth("power", sqrt_coeff=16, pow_num=3, pow_den=2), 1024) == -1
+    assert kvm.kvm_plan_capacity(64, 2, kvm.growth("power", sqrt_coeff=2000, pow_num=1, pow_den=2), 1024) == -1
+    assert kvm.kvm_plan_capacity(64, 2, gp, 1 << 26) == -1
+    assert kvm.kvm_plan_capacity(64, 2, kvm.growth("saturating", fixed_slots=100, sat_half=0), 1024) == -1
+
+
 def test_create_validates_arguments_before_touching_the_device(kvm):
     h = C.c_void_p()
     assert kvm.lib.kvm_state_create(None, C.byref(h)) == 1

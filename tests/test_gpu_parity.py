@@ -89,6 +89,15 @@ def test_unbounded_growth_never_merges():
     print(stats)
 
 
+@pytest.mark.parametrize("kw", [dict(growth="power", sqrt_coeff=8, pow_num=2, pow_den=3),
+                                dict(growth="power", sqrt_coeff=3, pow_num=3, pow_den=4),
+                                dict(growth="saturating", fixed_slots=300, sat_half=1024)])
+def test_power_law_and_saturating_budgets(kw):
+    """The two further schedule shapes of Section 3.2 (exact integer budgets on both sides)."""
+    wl = synth.Workload("t", 1, 2, 2, 64, 64 * 40 + 9, 64, r=16, seed=17, kind="mixture", **kw)
+    print(_run(wl))
+
+
 def test_radius_switch_off():
     wl = synth.Workload("t", 1, 2, 2, 64, 640, 32, "fixed", fixed_slots=48, seed=14)
     print(_run(wl, radius_on=False, gate=True))

@@ -47,9 +47,9 @@ def read_golden(name):
 # ---------------------------------------------------------------------------------------
 # state sizes (Table 1; budget rule of Section 3.2; "16 sqrt(N)", "KVM 256" of Section 4)
 
-def run_sizes(C, T, growth, fixed_slots=0, d=4):
+def run_sizes(C, T, growth, fixed_slots=0, d=4, **kw):
     r = rng(0)
-    cfg = OracleConfig(B=1, Hq=1, Hkv=1, d=d, C=C, growth=growth, fixed_slots=fixed_slots)
+    cfg = OracleConfig(B=1, Hq=1, Hkv=1, d=d, C=C, growth=growth, fixed_slots=fixed_slots, **kw)
     o = KVMOracle(cfg)
     step = 4096
     for t0 in range(0, T, step):
@@ -100,6 +100,49 @@ def test_unbounded_budget_appends_everything():
     e, m, a = o.fold_log()
     assert np.all(a == 16)
     assert np.all(m == e - 16)  # every token older than the (w-1)-block window is a row
+
+
+def test_power_schedule_with_exponent_one_half_is_the_sqrt_schedule():
+    """The power-law budget floor(a e^(p/q)) at a = 16, p/q = 1/2 is the paper's 16 sqrt(N)."""
+    a = run_sizes(64, 8192, "sqrt", d=2)
+    b = run_sizes(64, 8192, "power", d=2, sqrt_coeff=16, pow_num=1, pow_den=2)
+    assert a.fold_log()[1].tolist() == b.fold_log()[1].tolist() and a.rows == b.rows
+
+
+@pytest.mark.parametrize("a,p,q", [(8, 2, 3), (3, 3, 4), (40, 1, 3), (1, 1, 1), (5, 1, 4)])
+def test_power_schedule_sizes_are_the_exact_integer_floor(a, p, q):
+    """Whenever the budget lies between the rows held and rows + C, the state has exactly B(e) rows,
+    and B(e) = n is pinned by its definition in integers: n^q <= a^q e^p < (n+1)^q."""
+    C = 32
+    o = run_sizes(C, 4096, "power", d=2, sqrt_coeff=a, pow_num=p, pow_den=q)
+    e, m, na = o.fold_log()
+    assert m[0] == C and np.all(np.diff(m) >= 0)
+    seen = 0
+    prev = 0
+    for ee, mm, aa in zip(e.tolist(), m.tolist(), na.tolist()):
+        if prev and prev < mm < prev + C:      # neither clamp of the budget rule is active: rows = B(e)
+            assert mm ** q <= a ** q * ee ** p < (mm + 1) ** q, (ee, mm)
+            seen += 1
+        elif prev and mm == prev + C:           # capped by the overflow block: the budget is at least that
+            assert (prev + C) ** q <= a ** q * ee ** p
+        elif prev:                              # nothing appended: the budget is at most the rows held
+            assert a ** q * ee ** p < (mm + 1) ** q
+        prev = mm
+    assert seen >= 3 or (a, p, q) == (1, 1, 1)
+
+
+def test_saturating_schedule_sizes():
+    """B(e) = floor(M e / (e + h)): half of M at e = h, below M for ever, never shrinking."""
+    M, h, C = 300, 2048, 32
+    o = run_sizes(C, 16384, "saturating", fixed_slots=M, d=2, sat_half=h)
+    e, m, _ = o.fold_log()
+    got = dict(zip(e.tolist(), m.tolist()))
+    assert got[h] == M // 2                                  # 150 rows when e = h
+    assert np.all(np.diff(m) >= 0) and m[0] == C and m[-1] < M
+    for ee, mm in got.items():
+        if mm > C:                                           # past the first state the rows follow the budget
+            assert mm * (ee + h) <= M * ee < (mm + 1) * (ee + h), (ee, mm)
+    assert got[16384] == (M * 16384) // (16384 + h) == 266
 
 
 # ---------------------------------------------------------------------------------------
