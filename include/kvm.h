@@ -248,6 +248,21 @@ kvm_status_t kvm_attend_rows_noalloc(const void* q, const void* keys, const void
                                      int64_t n_rows, int32_t head_dim, float scale, void* out,
                                      void* cuda_stream);
 
+/* Front end, merge gate (Section 3.2 "KVM weight preparation", Eq. 2): g_t = 1 + ELU(x_t W_g) with
+ * ELU's alpha = 1, i.e. g = 1 + z for z > 0 and exp(z) otherwise, z = x_t . W_g[h]; one scalar per
+ * token and kv head (W_g is one d_model-vector per head).  The result is what kvm_prefill and
+ * kvm_decode_step take as `gate` (for a decode step: batch rows of one token, n_tokens = 1).
+ *   x       device bf16 [batch, n_tokens, d_model]   the layer's input rows; 16-byte aligned,
+ *                                                    d_model a multiple of 8
+ *   w_gate  device fp32 [n_kv_heads, d_model]
+ *   gate    device fp32 [batch, n_kv_heads, n_tokens]   (out)
+ * Products and sums in fp32 (inputs bf16 -> fp32 exactly).  n_kv_heads <= 64 and batch <= 65535,
+ * else KVM_ERR_UNSUPPORTED; bad pointers, alignment or sizes KVM_ERR_INVALID_ARG; nothing is
+ * launched on an error.  The caller owns all three buffers; no allocation, no synchronisation;
+ * the work is enqueued on cuda_stream on the current device. */
+kvm_status_t kvm_merge_gate(const void* x, const float* w_gate, int32_t batch, int64_t n_tokens, int32_t d_model,
+                            int32_t n_kv_heads, float* gate, void* cuda_stream);
+
 const char* kvm_status_string(kvm_status_t s);
 
 #ifdef __cplusplus

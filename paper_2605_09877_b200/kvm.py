@@ -25,7 +25,7 @@ FLAG_NO_RADIUS, FLAG_RECORD_ASSIGN, FLAG_SIMT_ATTENTION, FLAG_SIMT_ROUTING = 1, 
 EXPORTS = ["kvm_plan_capacity", "kvm_state_create", "kvm_prefill", "kvm_decode_step", "kvm_prefill_host",
            "kvm_decode_step_host", "kvm_state_free", "kvm_state_info", "kvm_state_check", "kvm_state_export",
            "kvm_debug_assignments", "kvm_launch_count", "kvm_status_string", "kvm_state_reset",
-           "kvm_profile_enable", "kvm_profile_read", "kvm_debug_counters", "kvm_attend_rows_noalloc"]
+           "kvm_profile_enable", "kvm_profile_read", "kvm_debug_counters", "kvm_attend_rows_noalloc", "kvm_merge_gate"]
 
 
 class KVMError(RuntimeError):
@@ -95,6 +95,8 @@ def _load():
     L.kvm_launch_count.argtypes = [vp]
     L.kvm_attend_rows_noalloc.restype = C.c_int
     L.kvm_attend_rows_noalloc.argtypes = [vp, vp, vp, C.c_int32, C.c_int64, C.c_int32, C.c_float, vp, vp]
+    L.kvm_merge_gate.restype = C.c_int
+    L.kvm_merge_gate.argtypes = [vp, vp, C.c_int32, C.c_int64, C.c_int32, C.c_int32, vp, vp]
     L.kvm_status_string.restype = C.c_char_p
     L.kvm_status_string.argtypes = [C.c_int]
     return L
@@ -110,6 +112,23 @@ def growth(kind: str, fixed_slots: int = 0, sqrt_coeff: int = 16, pow_num: int =
     k = {"fixed": GROWTH_FIXED, "sqrt": GROWTH_SQRT, "unbounded": GROWTH_UNBOUNDED, "power": GROWTH_POWER,
          "saturating": GROWTH_SATURATING}[kind]
     return Growth(k, sqrt_coeff, fixed_slots, pow_num, pow_den, sat_half)
+
+
+def merge_gate(x: "torch.Tensor", w_gate: "torch.Tensor", out=None, stream=None) -> "torch.Tensor":
+    """g = 1 + ELU(x W_g): x bf16 [B, T, d_model], w_gate fp32 [Hkv, d_model] -> fp32 [B, Hkv, T]
+    (argument marshalling only; the product runs in kvm_merge_gate)."""
+    assert x.is_cuda and w_gate.is_cuda and x.dtype == torch.bfloat16 and w_gate.dtype == torch.float32
+    assert x.is_contiguous() and w_gate.is_contiguous() and x.dim() == 3 and w_gate.dim() == 2
+    B, T, dm = x.shape
+    H = w_gate.shape[0]
+    assert w_gate.shape[1] == dm
+    if out is None:
+        out = torch.empty((B, H, T), dtype=torch.float32, device=x.device)
+    rc = lib.kvm_merge_gate(C.c_void_p(x.data_ptr()), C.c_void_p(w_gate.data_ptr()), B, T, dm, H,
+                            C.c_void_p(out.data_ptr()), _stream_ptr(stream))
+    if rc != 0:
+        raise KVMError(rc, "kvm_merge_gate")
+    return out
 
 
 def kvm_plan_capacity(block: int, n_bswa_chunks: int, g: Growth, seq_len: int) -> int:

@@ -1,0 +1,78 @@
+"""Merge gate g_t = 1 + ELU(x_t W_g) (Section 3.2 "KVM weight preparation", Eq. 2): pins of the fp64
+oracle (closed forms, special cases, a library routine), then the CUDA entry point against it."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle.frontend import elu, merge_gate
+
+
+def test_gate_closed_forms():
+    # z = 0 -> g = 1 (a token that the gate neither damps nor amplifies); z > 0 -> 1 + z; z < 0 -> exp(z)
+    x = np.array([[[0.0, 0.0], [2.0, 0.0], [-math.log(2.0), 0.0], [0.0, 5.0]]])   # [1, 4, 2]
+    w = np.array([[1.0, 0.0]])                                                     # picks channel 0
+    g = merge_gate(x, w)
+    assert g.shape == (1, 1, 4)
+    assert np.allclose(g[0, 0], [1.0, 3.0, 0.5, 1.0], rtol=0, atol=1e-15)
+    # zero weights: every gate is exactly 1, the ungated layer
+    assert np.all(merge_gate(np.random.default_rng(0).standard_normal((2, 7, 5)), np.zeros((3, 5))) == 1.0)
+
+
+def test_gate_is_positive_monotone_and_continuous_at_zero():
+    z = np.linspace(-30, 30, 2001)
+    g = 1.0 + elu(z)
+    assert np.all(g > 0) and np.all(np.diff(g) > 0)
+    eps = 1e-9
+    assert abs((1.0 + elu(np.array([eps]))[0]) - (1.0 + elu(np.array([-eps]))[0])) < 3e-9
+    # derivative 1 on both sides of zero (ELU with alpha = 1 is C^1)
+    assert abs((elu(np.array([1e-6]))[0] - elu(np.array([-1e-6]))[0]) / 2e-6 - 1.0) < 1e-6
+
+
+def test_gate_matches_the_library_elu_and_a_plain_matmul():
+    rng = np.random.default_rng(1)
+    x = rng.standard_normal((2, 33, 48))
+    w = rng.standard_normal((5, 48)) / math.sqrt(48)
+    ref = 1.0 + torch.nn.functional.elu(torch.from_numpy(x) @ torch.from_numpy(w).T).permute(0, 2, 1).numpy()
+    assert np.allclose(merge_gate(x, w), ref, rtol=1e-13, atol=1e-13)
+    # layout: head h of batch b, token t uses W_g[h] and x[b, t]
+    assert np.isclose(merge_gate(x, w)[1, 3, 17], 1.0 + elu(np.array([x[1, 17] @ w[3]]))[0])
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("B,T,dm,H", [(2, 777, 1000, 3), (1, 64, 2048, 16), (3, 130, 72, 40), (2, 1, 256, 8),
+                                      (1, 4096, 1024, 64)])
+def test_gate_kernel_against_the_oracle(B, T, dm, H):
+    """fp32 products and sums of exactly converted bf16 inputs against fp64: with |x| ~ 1,
+    |w| ~ 1/sqrt(d_model), the sum of d_model products carries an error of about
+    d_model * 2^-24 * E|x w| ~ sqrt(d_model) * 6e-8 in z, and g = 1 + ELU(z) has slope <= max(1, g):
+    5e-5 * max(1, g) bounds it with a wide margin for every d_model used here."""
+    from paper_2605_09877_b200 import kvm
+    gen = torch.Generator().manual_seed(B * 1000 + T)
+    x = torch.randn((B, T, dm), generator=gen).to(torch.bfloat16)
+    w = (torch.randn((H, dm), generator=gen) / math.sqrt(dm)).float()
+    g = kvm.merge_gate(x.cuda(), w.cuda())
+    torch.cuda.synchronize()
+    ref = merge_gate(x.double().numpy(), w.double().numpy())
+    got = g.cpu().double().numpy()
+    assert got.shape == ref.shape
+    err = np.abs(got - ref) / np.maximum(1.0, ref)
+    assert err.max() < 5e-5, err.max()
+
+
+@pytest.mark.gpu
+def test_gate_argument_checks():
+    from paper_2605_09877_b200 import kvm
+    x = torch.zeros((1, 8, 12), dtype=torch.bfloat16, device="cuda")   # d_model not a multiple of 8
+    w = torch.zeros((2, 12), dtype=torch.float32, device="cuda")
+    with pytest.raises(kvm.KVMError) as e:
+        kvm.merge_gate(x, w)
+    assert e.value.code == 1
+    x = torch.zeros((1, 8, 16), dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros((65, 16), dtype=torch.float32, device="cuda")      # more than 64 heads
+    with pytest.raises(kvm.KVMError) as e:
+        kvm.merge_gate(x, w)
+    assert e.value.code == 2
+    g = kvm.merge_gate(x, torch.zeros((4, 16), dtype=torch.float32, device="cuda"))
+    assert torch.all(g == 1.0)
