@@ -26,6 +26,7 @@ import time
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
 from paper_2605_09877_b200 import synth  # noqa: E402
@@ -257,6 +258,86 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_gate(args):
+    """Front-end merge gate g = 1 + ELU(x W_g) (kvm_merge_gate): HBM-bound on reading x.  "gate": the
+    default workload's layer (B2 T8192, d_model = Hq d = 2048, 16 kv heads); "gate-paper": the paper's
+    speed shape (B8 T32768, d_model 4096, 32 heads; x is 2.1 GB)."""
+    from paper_2605_09877_b200 import kvm
+    rank, world, local = dist_setup(args.gpus)
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    B, T, dm, H = (8, 32768, 4096, 32) if args.workload == "gate-paper" else (2, 8192, 2048, 16)
+    pk = peaks()
+    W, K = max(args.warmup, 3), args.steps
+    gen = torch.Generator().manual_seed(100 + rank)
+    x_host = torch.randn((B, T, dm), generator=gen).to(torch.bfloat16).pin_memory()
+    w_host = (torch.randn((H, dm), generator=gen) / math.sqrt(dm)).float()
+    x, w = x_host.to(dev), w_host.to(dev)
+    gate = torch.empty((B, H, T), dtype=torch.float32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    bytes_step = B * T * dm * 2 + B * H * T * 4 + H * dm * 4   # x read once, gate written once, W_g read once
+    for _ in range(W):
+        kvm.merge_gate(x, w, out=gate)
+    barrier(world)
+    torch.cuda.synchronize()
+    clocks = ClockSampler(local)
+    clocks.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for a, b in ev:
+        flush.zero_()
+        a.record()
+        kvm.merge_gate(x, w, out=gate)
+        b.record()
+    torch.cuda.synchronize()
+    barrier(world)
+    clk = clocks.stop()
+    ms = sum(a.elapsed_time(b) for a, b in ev) / K
+    ms_all = max_over_ranks(ms, world)
+    # end to end: x from pinned host memory, the gates back to the host
+    g_host = torch.empty((B, H, T), dtype=torch.float32).pin_memory()
+    e2e = None
+    if not args.no_e2e:
+        t_e2e = []
+        for _ in range(3):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            xd = x_host.to(dev, non_blocking=True)
+            kvm.merge_gate(xd, w, out=gate)
+            g_host.copy_(gate, non_blocking=True)
+            torch.cuda.synchronize()
+            t_e2e.append(time.perf_counter() - t0)
+        e2e = dict(value=world * B * T / min(t_e2e), unit="tokens/s", h2d_bytes_per_step=B * T * dm * 2,
+                   d2h_bytes_per_step=B * H * T * 4)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        from oracle.frontend import merge_gate as oracle_gate
+        nb = 1 if B * T * dm > (1 << 27) else B           # a bounded sample: one batch row of the large shape
+        xs = x_host[:nb].double().numpy()
+        t0 = time.perf_counter()
+        ref = oracle_gate(xs, w_host.double().numpy())
+        dt = time.perf_counter() - t0
+        err = float(np.max(np.abs(gate[:nb].cpu().double().numpy() - ref) / np.maximum(1.0, ref)))
+        assert err < 5e-5, err
+        cpu = dict(value=nb * T / dt, unit="tokens/s", cores=os.cpu_count(), kind="oracle",
+                   sample=f"{nb} of {B} batch rows x {T} tokens, {dt:.2f} s wall (numpy fp64); GPU result checked against it: max err {err:.1e}")
+    if rank == 0:
+        achieved = bytes_step / (ms * 1e-3) / 1e9
+        line = dict(metric="kvm_merge_gate_tokens_per_s", value=world * B * T / (ms_all * 1e-3), unit="tokens/s",
+                    n_gpus=world, steps=K, warmup=W, ms_per_step=ms_all, higher_is_better=True, scaling="weak",
+                    vs_baseline=None, dtype="bf16 inputs, f32 accumulate", data="synthetic",
+                    config=dict(workload=args.workload, mode="front end: merge gate", B=B, T=T, d_model=dm, Hkv=H,
+                                l2="256 MiB flush between timed steps"),
+                    clocks=clk, e2e=e2e, gpu_launches=K,
+                    roofline=dict(bound="hbm", kernel="merge_gate", achieved=achieved, peak=pk["hbm"], unit="GB/s",
+                                  frac=achieved / pk["hbm"], traffic=None, peak_source=pk["src"] + " copy bandwidth",
+                                  bytes_per_step=bytes_step),
+                    cpu_baseline=cpu)
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -272,6 +353,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.workload in ("gate", "gate-paper"):
+        return run_gate(args)
 
     from paper_2605_09877_b200 import kvm
     rank, world, local = dist_setup(args.gpus)

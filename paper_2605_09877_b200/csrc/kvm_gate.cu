@@ -5,83 +5,83 @@
 //
 // A skinny product [tokens x d_model] x [d_model x heads] with at most 64 heads: every x element is
 // needed once per head, so the kernel is bound by reading x (2 d_model bytes per token) as long as
-// the FMA pipe keeps up.  One CTA takes 64 tokens: 64-channel slices of their x rows and of all
-// W_g rows go through shared memory, thread (tx, ty) accumulates tokens tx, tx + 32 against heads
-// ty*HPT .. ty*HPT + HPT - 1 in fp32, and the results leave through shared memory so that the stores
-// run along the token axis of gate[B, heads, T].
+// the FMA pipe keeps up.  A CTA takes 64 tokens; thread (token, part) owns one token, all heads and
+// one quarter of every 128-channel slice: its share of the x row streams through registers, eight
+// channels (16 bytes) per load, and is never shared; the W_g rows go through shared memory slice by
+// slice and are read as broadcasts (every lane of a warp wants the same weights), so a step of eight
+// channels costs 2 HT shared-memory loads for 8 HT FMAs.  The four partial sums of a token meet in
+// shared memory at the end (fixed order: reproducible), and the stores run along the token axis of
+// gate[B, heads, T].
 #include "kvm_internal.h"
 
 namespace kvm {
 
 constexpr int kGateTokens = 64;   // tokens per CTA
-constexpr int kGateK = 64;        // channels per shared-memory slice
+constexpr int kGateParts = 4;     // threads per token, each a quarter of the channels of a slice
+constexpr int kGateThreads = kGateTokens * kGateParts;
+constexpr int kGateK = 128;       // channels per shared-memory slice of W_g
 
-template <int HPT>
-__global__ void __launch_bounds__(256) merge_gate_kernel(const __nv_bfloat16* __restrict__ x, const float* __restrict__ w,
-                                                         float* __restrict__ gate, int64_t T, int dm, int H) {
-  constexpr int HP = 8 * HPT;   // heads, padded
-  __shared__ float xs[kGateTokens][kGateK + 1];
-  __shared__ float ws[HP][kGateK];
-  float (*outs)[kGateK + 1] = xs;   // the results reuse the x slice (HP <= 64 rows of 64 tokens) once the products are done
-  static_assert(HP <= kGateTokens && kGateK == kGateTokens, "result tile must fit the x slice");
-  const int tid = threadIdx.x, tx = tid & 31, ty = tid >> 5;
+template <int HT>                 // heads, padded to 8, 16, 32 or 64
+__global__ void __launch_bounds__(kGateThreads) merge_gate_kernel(const __nv_bfloat16* __restrict__ x, const float* __restrict__ w,
+                                                                  float* __restrict__ gate, int64_t T, int dm, int H) {
+  __shared__ __align__(16) float ws[HT * kGateK];   // W_g slice [HT][128]; afterwards the partial sums
+  const int tid = threadIdx.x, tok = tid % kGateTokens, part = tid / kGateTokens;   // a warp shares `part`
   const int b = blockIdx.y;
-  const int64_t t0 = (int64_t)blockIdx.x * kGateTokens;
-  float acc[2][HPT];
+  const int64_t t = (int64_t)blockIdx.x * kGateTokens + tok;
+  const bool valid = t < T;
+  const __nv_bfloat16* row = x + ((int64_t)b * T + (valid ? t : 0)) * dm;
+  float acc[HT];
 #pragma unroll
-  for (int h = 0; h < HPT; ++h) acc[0][h] = acc[1][h] = 0.f;
+  for (int h = 0; h < HT; ++h) acc[h] = 0.f;
   for (int k0 = 0; k0 < dm; k0 += kGateK) {
-    // x slice: 64 tokens x 64 channels, eight bf16 (16 bytes) per load
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const int e = (tid + i * 256) * 8;
-      const int tk = e / kGateK, ch = e % kGateK;
-      float v[8];
-      if (t0 + tk < T && k0 + ch < dm) {   // d_model is a multiple of 8: a run of eight is inside or outside
-        const uint4 raw = *reinterpret_cast<const uint4*>(x + ((int64_t)b * T + t0 + tk) * dm + k0 + ch);
-        const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const float2 f = __bfloat1622float2(p2[j]);
-          v[2 * j] = f.x; v[2 * j + 1] = f.y;
-        }
-      } else {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = 0.f;
-      }
-#pragma unroll
-      for (int j = 0; j < 8; ++j) xs[tk][ch + j] = v[j];
-    }
-    // W_g slice: all heads x 64 channels
-    for (int e = tid; e < HP * kGateK; e += 256) {
+    __syncthreads();   // the previous slice is no longer read
+    for (int e = tid; e < HT * kGateK; e += kGateThreads) {
       const int h = e / kGateK, c = e % kGateK;
-      ws[h][c] = (h < H && k0 + c < dm) ? w[(int64_t)h * dm + k0 + c] : 0.f;
+      ws[e] = (h < H && k0 + c < dm) ? w[(int64_t)h * dm + k0 + c] : 0.f;
     }
     __syncthreads();
-#pragma unroll 8
-    for (int kk = 0; kk < kGateK; ++kk) {
-      const float x0 = xs[tx][kk], x1 = xs[tx + 32][kk];
+#pragma unroll 2
+    for (int j = 0; j < kGateK / 8 / kGateParts; ++j) {
+      const int c = 8 * (part * (kGateK / 8 / kGateParts) + j);   // first of eight channels inside the slice
+      if (k0 + c >= dm) break;                                    // d_model is a multiple of 8
+      const uint4 raw = *reinterpret_cast<const uint4*>(row + k0 + c);
+      const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+      const float2 f0 = __bfloat1622float2(p2[0]), f1 = __bfloat1622float2(p2[1]);
+      const float2 f2 = __bfloat1622float2(p2[2]), f3 = __bfloat1622float2(p2[3]);
 #pragma unroll
-      for (int h = 0; h < HPT; ++h) {
-        const float wv = ws[ty * HPT + h][kk];   // one address per warp: broadcast
-        acc[0][h] = fmaf(x0, wv, acc[0][h]);
-        acc[1][h] = fmaf(x1, wv, acc[1][h]);
+      for (int h = 0; h < HT; ++h) {
+        const float4 wa = *reinterpret_cast<const float4*>(&ws[h * kGateK + c]);       // one address per warp: broadcast
+        const float4 wb = *reinterpret_cast<const float4*>(&ws[h * kGateK + c + 4]);
+        float a = acc[h];
+        a = fmaf(f0.x, wa.x, a); a = fmaf(f0.y, wa.y, a); a = fmaf(f1.x, wa.z, a); a = fmaf(f1.y, wa.w, a);
+        a = fmaf(f2.x, wb.x, a); a = fmaf(f2.y, wb.y, a); a = fmaf(f3.x, wb.z, a); a = fmaf(f3.y, wb.w, a);
+        acc[h] = a;
       }
     }
-    __syncthreads();
   }
+  // parts 2, 3 -> parts 0, 1, then part 1 -> part 0, through the slice buffer (2 x 64 x HT floats fit it)
+  __syncthreads();
+  if (part >= 2) {
 #pragma unroll
-  for (int h = 0; h < HPT; ++h) {
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const float z = acc[i][h];
-      outs[ty * HPT + h][tx + 32 * i] = z > 0.f ? 1.f + z : expf(z);   // 1 + ELU(z), alpha = 1
-    }
+    for (int h = 0; h < HT; ++h) ws[((part - 2) * HT + h) * kGateTokens + tok] = acc[h];
   }
   __syncthreads();
-  for (int e = tid; e < H * kGateTokens; e += 256) {
-    const int h = e / kGateTokens, tk = e % kGateTokens;
-    if (t0 + tk < T) gate[((int64_t)b * H + h) * T + t0 + tk] = outs[h][tk];
+  if (part < 2) {
+#pragma unroll
+    for (int h = 0; h < HT; ++h) acc[h] += ws[(part * HT + h) * kGateTokens + tok];
+  }
+  __syncthreads();
+  if (part == 1) {
+#pragma unroll
+    for (int h = 0; h < HT; ++h) ws[h * kGateTokens + tok] = acc[h];
+  }
+  __syncthreads();
+  if (part == 0 && valid) {
+#pragma unroll
+    for (int h = 0; h < HT; ++h) {
+      const float z = acc[h] + ws[h * kGateTokens + tok];
+      if (h < H) gate[((int64_t)b * H + h) * T + t] = z > 0.f ? 1.f + z : expf(z);   // 1 + ELU(z), alpha = 1
+    }
   }
 }
 
@@ -99,10 +99,9 @@ kvm_status_t kvm_merge_gate(const void* x, const float* w_gate, int32_t batch, i
   cudaStream_t s = (cudaStream_t)cuda_stream;
   const dim3 grid((unsigned)((n_tokens + kGateTokens - 1) / kGateTokens), (unsigned)batch);
   const __nv_bfloat16* xp = (const __nv_bfloat16*)x;
-  const int hpt = (n_kv_heads + 7) / 8;
-  if (hpt <= 1) merge_gate_kernel<1><<<grid, 256, 0, s>>>(xp, w_gate, gate, n_tokens, d_model, n_kv_heads);
-  else if (hpt <= 2) merge_gate_kernel<2><<<grid, 256, 0, s>>>(xp, w_gate, gate, n_tokens, d_model, n_kv_heads);
-  else if (hpt <= 4) merge_gate_kernel<4><<<grid, 256, 0, s>>>(xp, w_gate, gate, n_tokens, d_model, n_kv_heads);
-  else merge_gate_kernel<8><<<grid, 256, 0, s>>>(xp, w_gate, gate, n_tokens, d_model, n_kv_heads);
+  if (n_kv_heads <= 8) merge_gate_kernel<8><<<grid, kGateThreads, 0, s>>>(xp, w_gate, gate, n_tokens, d_model, n_kv_heads);
+  else if (n_kv_heads <= 16) merge_gate_kernel<16><<<grid, kGateThreads, 0, s>>>(xp, w_gate, gate, n_tokens, d_model, n_kv_heads);
+  else if (n_kv_heads <= 32) merge_gate_kernel<32><<<grid, kGateThreads, 0, s>>>(xp, w_gate, gate, n_tokens, d_model, n_kv_heads);
+  else merge_gate_kernel<64><<<grid, kGateThreads, 0, s>>>(xp, w_gate, gate, n_tokens, d_model, n_kv_heads);
   return cudaGetLastError() == cudaSuccess ? KVM_OK : KVM_ERR_CUDA;
 }
