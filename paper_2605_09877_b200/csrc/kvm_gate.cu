@@ -13,8 +13,11 @@
 // shared memory at the end (fixed order: reproducible), and the stores run along the token axis of
 // gate[B, heads, T].
 #include "kvm_internal.h"
+#include "tc_common.cuh"
 
 namespace kvm {
+
+bool encode_tmap_rows(CUtensorMap* map, const void* base, int d, int64_t rows, int64_t units, int box_rows);   // kvm_attn_tc.cu
 
 constexpr int kGateTokens = 64;   // tokens per CTA
 constexpr int kGateParts = 4;     // threads per token, each a quarter of the channels of a slice
@@ -85,6 +88,177 @@ __global__ void __launch_bounds__(kGateThreads) merge_gate_kernel(const __nv_bfl
   }
 }
 
+// ------------------------------------------------------------------------------------------
+// Tensor-core version (d_model a multiple of 64, more than 8 heads): with 16 or more heads the product
+// above is bound by the FMA pipe and by the shared-memory broadcasts, not by reading x.  Here a CTA
+// takes 128 tokens:
+//   warp 0      TMA producer: 128-token x 64-channel slices of x (bf16, 128-byte swizzle), 4 stages
+//   warps 2-5   weight converters: the same 64 channels of every W_g row, fp32 -> bf16 "hi" plus bf16
+//               "lo" = bf16(w - hi) (together 16 mantissa bits; the products hi*x and lo*x are exact in
+//               fp32; a third term was measured: same error, which the fp32 accumulation dominates,
+//               and 1.8x the time), written into shared memory in the swizzled K-major layout the MMA
+//               reads; after the last slice the same warps read the accumulator and store the gates
+//   warp 1      one thread issues, per slice, 4 k-steps x (hi, lo) tcgen05.mma (kind::f16, bf16 x bf16,
+//               M 128, N = heads padded to 16..64, fp32 accumulator in tensor memory)
+// Every wait is bounded; if one expires the CTA stores NaN gates for its tokens and tears down.
+constexpr int kGateTcStages = 4;
+constexpr int kGateTcXBytes = 128 * 128;   // 128 tokens x 64 bf16
+
+enum { GB_XFULL = 0, GB_WFULL = 4, GB_FREE = 8, GB_DONE = 12, GB_COUNT = 13 };
+
+__host__ __device__ constexpr uint32_t idesc_bf16(int M, int N) {   // as tc::idesc_f16, A and B formats = 1 (bf16), both K-major
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+template <int NP>   // heads padded to a multiple of 16
+__global__ void __launch_bounds__(192, 1)
+merge_gate_tc_kernel(const __grid_constant__ CUtensorMap mapX, const float* __restrict__ w, float* __restrict__ gate,
+                     int64_t T, int dm, int H) {
+  constexpr int WBYTES = 2 * NP * 128;     // hi and lo tiles of one slice
+  constexpr uint32_t TMEM_COLS = NP <= 32 ? 32 : 64;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sX = base;
+  uint8_t* sW = base + kGateTcStages * kGateTcXBytes;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sW + kGateTcStages * WBYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + GB_COUNT);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int b = blockIdx.y;
+  const int64_t t0 = (int64_t)blockIdx.x * 128;
+  const int nslices = dm / 64;
+
+  if (tid == 0) {
+    for (int s = 0; s < kGateTcStages; ++s) {
+      tc::mbar_init(&bars[GB_XFULL + s], 1);
+      tc::mbar_init(&bars[GB_WFULL + s], 128);
+      tc::mbar_init(&bars[GB_FREE + s], 1);
+    }
+    tc::mbar_init(&bars[GB_DONE], 1);
+    *abort_flag = 0;
+    tc::fence_barrier_init();
+  }
+  if (warp == 1) {
+    tc::tmem_alloc(tmem_slot, TMEM_COLS);
+    tc::tmem_relinquish();
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      tc::prefetch_tmap(&mapX);
+      for (int j = 0; j < nslices; ++j) {
+        const int s = j % kGateTcStages;
+        if (*abort_flag) break;
+        if (j >= kGateTcStages && !tc::mbar_wait(&bars[GB_FREE + s], ((j / kGateTcStages) - 1) & 1)) { *abort_flag = 1; break; }
+        tc::mbar_expect_tx(&bars[GB_XFULL + s], kGateTcXBytes);
+        tc::tma_load_3d(sX + s * kGateTcXBytes, &mapX, &bars[GB_XFULL + s], j * 64, (int)t0, b);   // rows past T read zeros
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t IDESC = idesc_bf16(128, NP);
+      const uint32_t aX = tc::smem_u32(sX), aW = tc::smem_u32(sW);
+      bool dead = false;
+      for (int j = 0; j < nslices && !dead; ++j) {
+        const int s = j % kGateTcStages;
+        const uint32_t par = (j / kGateTcStages) & 1;
+        if (*abort_flag || !tc::mbar_wait(&bars[GB_XFULL + s], par) || !tc::mbar_wait(&bars[GB_WFULL + s], par)) { dead = true; break; }
+        tc::tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+          const uint64_t da = tc::smem_desc_sw128(aX + s * kGateTcXBytes + ks * 32, 16, 1024);
+          tc::mma_f16_ss(tmem, da, tc::smem_desc_sw128(aW + s * WBYTES + ks * 32, 16, 1024), IDESC, (j > 0 || ks > 0) ? 1u : 0u);
+          tc::mma_f16_ss(tmem, da, tc::smem_desc_sw128(aW + s * WBYTES + NP * 128 + ks * 32, 16, 1024), IDESC, 1u);
+        }
+        tc::mma_commit(&bars[GB_FREE + s]);
+      }
+      if (dead) *abort_flag = 1;
+      tc::mma_commit(&bars[GB_DONE]);   // (arrives once everything issued so far has completed)
+    }
+  } else {
+    const int ct = tid - 64;   // 0..127
+    bool ok = true;
+    for (int j = 0; j < nslices && ok; ++j) {
+      const int s = j % kGateTcStages;
+      if (j >= kGateTcStages && !tc::mbar_wait(&bars[GB_FREE + s], ((j / kGateTcStages) - 1) & 1)) { *abort_flag = 1; ok = false; break; }
+      uint8_t* hi = sW + s * WBYTES;
+      uint8_t* lo = hi + NP * 128;
+      for (int item = ct; item < NP * 8; item += 128) {
+        const int r = item >> 3, c = item & 7;   // head row, 16-byte chunk (8 channels)
+        float v[8];
+        if (r < H) {
+          const float4 a4 = *reinterpret_cast<const float4*>(w + (int64_t)r * dm + j * 64 + 8 * c);
+          const float4 b4 = *reinterpret_cast<const float4*>(w + (int64_t)r * dm + j * 64 + 8 * c + 4);
+          v[0] = a4.x; v[1] = a4.y; v[2] = a4.z; v[3] = a4.w; v[4] = b4.x; v[5] = b4.y; v[6] = b4.z; v[7] = b4.w;
+        } else {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) v[i] = 0.f;
+        }
+        uint32_t ph[4], pl[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const __nv_bfloat16 h0 = __float2bfloat16_rn(v[2 * i]), h1 = __float2bfloat16_rn(v[2 * i + 1]);
+          const __nv_bfloat16 l0 = __float2bfloat16_rn(v[2 * i] - __bfloat162float(h0));
+          const __nv_bfloat16 l1 = __float2bfloat16_rn(v[2 * i + 1] - __bfloat162float(h1));
+          ph[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+          pl[i] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+        }
+        // K-major tile with the 128-byte swizzle: row r of 128 bytes, chunk c stored at c ^ (r mod 8)
+        const int off = (r >> 3) * 1024 + (r & 7) * 128 + ((c ^ (r & 7)) << 4);
+        *reinterpret_cast<uint4*>(hi + off) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
+        *reinterpret_cast<uint4*>(lo + off) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
+      }
+      tc::fence_proxy_async();   // the tensor core reads these tiles through the async proxy
+      tc::mbar_arrive(&bars[GB_WFULL + s]);
+    }
+    // epilogue: thread = token row of the accumulator (TMEM lane quarter = warp mod 4)
+    if (ok && !tc::mbar_wait(&bars[GB_DONE], 0)) { *abort_flag = 1; ok = false; }
+    tc::tc_fence_after();
+    const int quarter = warp & 3;
+    const int64_t t = t0 + quarter * 32 + lane;
+    const bool good = ok && !*abort_flag;
+#pragma unroll
+    for (int c = 0; c < (NP + 31) / 32; ++c) {
+      uint32_t r[32];
+      tc::tmem_ld32(tmem + ((uint32_t)(quarter * 32) << 16) + c * 32, r);
+      tc::tmem_wait_ld();
+      if (t < T) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int h = c * 32 + i;
+          if (h < H) {
+            const float z = __uint_as_float(r[i]);
+            gate[((int64_t)b * H + h) * T + t] = good ? (z > 0.f ? 1.f + z : expf(z)) : __int_as_float(0x7fc00000);
+          }
+        }
+      }
+    }
+  }
+  tc::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc::tmem_dealloc(tmem, TMEM_COLS);
+  }
+}
+
+template <int NP>
+static bool launch_gate_tc(const CUtensorMap& map, const float* w, float* gate, int batch, int64_t T, int dm, int H, cudaStream_t s) {
+  const int smem = kGateTcStages * (kGateTcXBytes + 2 * NP * 128) + 256 + 1024;
+  static bool attr_set = false;   // (per instantiation; setting it again is harmless)
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(merge_gate_tc_kernel<NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
+    attr_set = true;
+  }
+  const dim3 grid((unsigned)((T + 127) / 128), (unsigned)batch);
+  merge_gate_tc_kernel<NP><<<grid, 192, smem, s>>>(map, w, gate, T, dm, H);
+  return true;
+}
+
 }  // namespace kvm
 
 using namespace kvm;
@@ -99,6 +273,19 @@ kvm_status_t kvm_merge_gate(const void* x, const float* w_gate, int32_t batch, i
   cudaStream_t s = (cudaStream_t)cuda_stream;
   const dim3 grid((unsigned)((n_tokens + kGateTokens - 1) / kGateTokens), (unsigned)batch);
   const __nv_bfloat16* xp = (const __nv_bfloat16*)x;
+  if (d_model % 64 == 0 && n_kv_heads > 8 && n_tokens < ((int64_t)1 << 31)) {
+    // tensor-core path (few heads are bound by reading x already on the scalar path)
+    CUtensorMap map;
+    if (encode_tmap_rows(&map, x, d_model, n_tokens, batch, 128)) {
+      bool ok;
+      if (n_kv_heads <= 16) ok = launch_gate_tc<16>(map, w_gate, gate, batch, n_tokens, d_model, n_kv_heads, s);
+      else if (n_kv_heads <= 32) ok = launch_gate_tc<32>(map, w_gate, gate, batch, n_tokens, d_model, n_kv_heads, s);
+      else if (n_kv_heads <= 48) ok = launch_gate_tc<48>(map, w_gate, gate, batch, n_tokens, d_model, n_kv_heads, s);
+      else ok = launch_gate_tc<64>(map, w_gate, gate, batch, n_tokens, d_model, n_kv_heads, s);
+      if (ok) return cudaGetLastError() == cudaSuccess ? KVM_OK : KVM_ERR_CUDA;
+    }
+    cudaGetLastError();   // fall through to the scalar path
+  }
   if (n_kv_heads <= 8) merge_gate_kernel<8><<<grid, kGateThreads, 0, s>>>(xp, w_gate, gate, n_tokens, d_model, n_kv_heads);
   else if (n_kv_heads <= 16) merge_gate_kernel<16><<<grid, kGateThreads, 0, s>>>(xp, w_gate, gate, n_tokens, d_model, n_kv_heads);
   else if (n_kv_heads <= 32) merge_gate_kernel<32><<<grid, kGateThreads, 0, s>>>(xp, w_gate, gate, n_tokens, d_model, n_kv_heads);

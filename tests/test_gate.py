@@ -42,12 +42,18 @@ def test_gate_matches_the_library_elu_and_a_plain_matmul():
 
 @pytest.mark.gpu
 @pytest.mark.parametrize("B,T,dm,H", [(2, 777, 1000, 3), (1, 64, 2048, 16), (3, 130, 72, 40), (2, 1, 256, 8),
-                                      (1, 4096, 1024, 64)])
+                                      (1, 4096, 1024, 64), (2, 300, 512, 24), (1, 200, 256, 40), (2, 129, 64, 9),
+                                      (1, 1, 4096, 32)])
 def test_gate_kernel_against_the_oracle(B, T, dm, H):
-    """fp32 products and sums of exactly converted bf16 inputs against fp64: with |x| ~ 1,
-    |w| ~ 1/sqrt(d_model), the sum of d_model products carries an error of about
-    d_model * 2^-24 * E|x w| ~ sqrt(d_model) * 6e-8 in z, and g = 1 + ELU(z) has slope <= max(1, g):
-    5e-5 * max(1, g) bounds it with a wide margin for every d_model used here."""
+    """Shapes cover both kernels (tensor cores when d_model is a multiple of 64 and there are more
+    than 8 heads, else scalar cores), every head padding, ragged token tiles and a single token.
+    Products of exactly converted bf16 inputs, sums in fp32, against fp64.  With |x| ~ 1 and
+    |w| ~ 1/sqrt(d_model) a sum of d_model products in round-to-nearest fp32 carries an error of
+    about sqrt(d_model) * 6e-8 in z; the tensor-core accumulator truncates instead of rounding, so
+    its error grows like d_model * 2^-24 * |z| ~ 2.4e-4 |z| at d_model = 4096 in the worst case
+    (measured: 3e-5).  On that path the weights enter as bf16 hi + bf16 lo (relative error 2^-17 per
+    weight, products exact in fp32), which adds ~ 8e-6.  g = 1 + ELU(z) has slope <= max(1, g), hence
+    the bound 2e-4 * max(1, g)."""
     from paper_2605_09877_b200 import kvm
     gen = torch.Generator().manual_seed(B * 1000 + T)
     x = torch.randn((B, T, dm), generator=gen).to(torch.bfloat16)
@@ -58,7 +64,7 @@ def test_gate_kernel_against_the_oracle(B, T, dm, H):
     got = g.cpu().double().numpy()
     assert got.shape == ref.shape
     err = np.abs(got - ref) / np.maximum(1.0, ref)
-    assert err.max() < 5e-5, err.max()
+    assert err.max() < 2e-4, err.max()
 
 
 @pytest.mark.gpu
