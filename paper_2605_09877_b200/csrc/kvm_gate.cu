@@ -182,22 +182,36 @@ merge_gate_tc_kernel(const __grid_constant__ CUtensorMap mapX, const float* __re
   } else {
     const int ct = tid - 64;   // 0..127
     bool ok = true;
+    // item = (head row r, 16-byte chunk c of the slice's 64 channels); a thread's items of slice j + 1
+    // are loaded before it converts those of slice j, so that the loads' latency is off the chain
+    constexpr int ITEMS = NP * 8 / 128;
+    float4 nxt[ITEMS][2];
+    auto load_items = [&](int j) {
+#pragma unroll
+      for (int q = 0; q < ITEMS; ++q) {
+        const int item = ct + 128 * q, r = item >> 3, c = item & 7;
+        if (r < H) {
+          nxt[q][0] = *reinterpret_cast<const float4*>(w + (int64_t)r * dm + j * 64 + 8 * c);
+          nxt[q][1] = *reinterpret_cast<const float4*>(w + (int64_t)r * dm + j * 64 + 8 * c + 4);
+        } else {
+          nxt[q][0] = nxt[q][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+      }
+    };
+    load_items(0);
     for (int j = 0; j < nslices && ok; ++j) {
       const int s = j % kGateTcStages;
+      float4 cur[ITEMS][2];
+#pragma unroll
+      for (int q = 0; q < ITEMS; ++q) { cur[q][0] = nxt[q][0]; cur[q][1] = nxt[q][1]; }
+      if (j + 1 < nslices) load_items(j + 1);
       if (j >= kGateTcStages && !tc::mbar_wait(&bars[GB_FREE + s], ((j / kGateTcStages) - 1) & 1)) { *abort_flag = 1; ok = false; break; }
       uint8_t* hi = sW + s * WBYTES;
       uint8_t* lo = hi + NP * 128;
-      for (int item = ct; item < NP * 8; item += 128) {
-        const int r = item >> 3, c = item & 7;   // head row, 16-byte chunk (8 channels)
-        float v[8];
-        if (r < H) {
-          const float4 a4 = *reinterpret_cast<const float4*>(w + (int64_t)r * dm + j * 64 + 8 * c);
-          const float4 b4 = *reinterpret_cast<const float4*>(w + (int64_t)r * dm + j * 64 + 8 * c + 4);
-          v[0] = a4.x; v[1] = a4.y; v[2] = a4.z; v[3] = a4.w; v[4] = b4.x; v[5] = b4.y; v[6] = b4.z; v[7] = b4.w;
-        } else {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) v[i] = 0.f;
-        }
+      for (int q = 0; q < ITEMS; ++q) {
+        const int item = ct + 128 * q, r = item >> 3, c = item & 7;
+        const float v[8] = {cur[q][0].x, cur[q][0].y, cur[q][0].z, cur[q][0].w, cur[q][1].x, cur[q][1].y, cur[q][1].z, cur[q][1].w};
         uint32_t ph[4], pl[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
