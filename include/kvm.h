@@ -263,6 +263,18 @@ kvm_status_t kvm_attend_rows_noalloc(const void* q, const void* keys, const void
 kvm_status_t kvm_merge_gate(const void* x, const float* w_gate, int32_t batch, int64_t n_tokens, int32_t d_model,
                             int32_t n_kv_heads, float* gate, void* cuda_stream);
 
+/* Front end, LN_q / LN_k (Appendix, time mixer of the backbone: q_t <- RoPE_r(LN_q(q_t)),
+ * k_t <- RoPE_r(LN_k(k_t))): LayerNorm over the head channels of every (batch, head, token) row, in
+ * place; call it on q and on k before kvm_prefill / kvm_decode_step, which apply the RoPE.
+ *   x       device bf16 [batch, n_heads, n_tokens, head_dim], contiguous, 16-byte aligned (in/out)
+ *   weight  device fp32 [n_heads, head_dim] or NULL (= 1); bias likewise or NULL (= 0); 16-byte aligned
+ *   eps     added to the biased variance
+ * Statistics and the affine map in fp32, result rounded to bf16.  head_dim 64 or 128 (else
+ * KVM_ERR_UNSUPPORTED).  The caller owns the buffers; no allocation, no synchronisation; enqueued on
+ * cuda_stream on the current device. */
+kvm_status_t kvm_head_layernorm(void* x, const float* weight, const float* bias, int32_t batch, int32_t n_heads,
+                                int64_t n_tokens, int32_t head_dim, float eps, void* cuda_stream);
+
 const char* kvm_status_string(kvm_status_t s);
 
 #ifdef __cplusplus

@@ -25,7 +25,7 @@ FLAG_NO_RADIUS, FLAG_RECORD_ASSIGN, FLAG_SIMT_ATTENTION, FLAG_SIMT_ROUTING = 1, 
 EXPORTS = ["kvm_plan_capacity", "kvm_state_create", "kvm_prefill", "kvm_decode_step", "kvm_prefill_host",
            "kvm_decode_step_host", "kvm_state_free", "kvm_state_info", "kvm_state_check", "kvm_state_export",
            "kvm_debug_assignments", "kvm_launch_count", "kvm_status_string", "kvm_state_reset",
-           "kvm_profile_enable", "kvm_profile_read", "kvm_debug_counters", "kvm_attend_rows_noalloc", "kvm_merge_gate"]
+           "kvm_profile_enable", "kvm_profile_read", "kvm_debug_counters", "kvm_attend_rows_noalloc", "kvm_merge_gate", "kvm_head_layernorm"]
 
 
 class KVMError(RuntimeError):
@@ -97,6 +97,8 @@ def _load():
     L.kvm_attend_rows_noalloc.argtypes = [vp, vp, vp, C.c_int32, C.c_int64, C.c_int32, C.c_float, vp, vp]
     L.kvm_merge_gate.restype = C.c_int
     L.kvm_merge_gate.argtypes = [vp, vp, C.c_int32, C.c_int64, C.c_int32, C.c_int32, vp, vp]
+    L.kvm_head_layernorm.restype = C.c_int
+    L.kvm_head_layernorm.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, C.c_int64, C.c_int32, C.c_float, vp]
     L.kvm_status_string.restype = C.c_char_p
     L.kvm_status_string.argtypes = [C.c_int]
     return L
@@ -129,6 +131,19 @@ def merge_gate(x: "torch.Tensor", w_gate: "torch.Tensor", out=None, stream=None)
     if rc != 0:
         raise KVMError(rc, "kvm_merge_gate")
     return out
+
+
+def head_layernorm(x: "torch.Tensor", weight=None, bias=None, eps: float = 1e-5, stream=None) -> "torch.Tensor":
+    """LN_q / LN_k in place: x bf16 [B, H, T, d] contiguous; weight, bias fp32 [H, d] on the device or None."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and x.dim() == 4
+    B, H, T, d = x.shape
+    for t in (weight, bias):
+        assert t is None or (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous() and tuple(t.shape) == (H, d))
+    rc = lib.kvm_head_layernorm(C.c_void_p(x.data_ptr()), C.c_void_p(weight.data_ptr() if weight is not None else 0),
+                                C.c_void_p(bias.data_ptr() if bias is not None else 0), B, H, T, d, eps, _stream_ptr(stream))
+    if rc != 0:
+        raise KVMError(rc, "kvm_head_layernorm")
+    return x
 
 
 def kvm_plan_capacity(block: int, n_bswa_chunks: int, g: Growth, seq_len: int) -> int:

@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 import torch
 
-from oracle.frontend import elu, merge_gate
+from oracle.frontend import elu, head_layernorm, merge_gate
 
 
 def test_gate_closed_forms():
@@ -82,3 +82,44 @@ def test_gate_argument_checks():
     assert e.value.code == 2
     g = kvm.merge_gate(x, torch.zeros((4, 16), dtype=torch.float32, device="cuda"))
     assert torch.all(g == 1.0)
+
+
+# ---------------------------------------------------------------------------------------
+# LN_q / LN_k
+
+def test_head_layernorm_oracle_pins():
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((2, 3, 5, 16)) * 3.0 + 1.5
+    y = head_layernorm(x, eps=0.0)
+    assert np.allclose(y.mean(-1), 0.0, atol=1e-14) and np.allclose((y ** 2).mean(-1), 1.0, atol=1e-13)
+    # a constant row has no direction: with eps > 0 it maps to the bias
+    b = rng.standard_normal((3, 16))
+    yc = head_layernorm(np.full((1, 3, 2, 16), 7.0), bias=b, eps=1e-5)
+    assert np.allclose(yc, b[None, :, None, :])
+    # the library routine, head by head (weights are per head)
+    w = rng.standard_normal((3, 16))
+    ref = np.stack([torch.nn.functional.layer_norm(torch.from_numpy(x[:, h]), (16,), torch.from_numpy(w[h]),
+                                                   torch.from_numpy(b[h]), 1e-5).numpy() for h in range(3)], axis=1)
+    assert np.allclose(head_layernorm(x, w, b, 1e-5), ref, rtol=1e-12, atol=1e-12)
+    # invariance to shift and positive scale of the input (eps = 0)
+    assert np.allclose(head_layernorm(4.0 * x - 2.0, eps=0.0), y, atol=1e-12)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("B,H,T,d,affine", [(2, 3, 777, 128, True), (1, 5, 33, 64, True), (2, 2, 1, 128, False),
+                                             (1, 16, 4096, 128, True)])
+def test_head_layernorm_kernel_against_the_oracle(B, H, T, d, affine):
+    """fp32 statistics of bf16 inputs, result rounded to bf16: within half a bf16 ulp of the fp64 value
+    plus the fp32 error, i.e. |err| <= 2^-8 |y| + 1e-5 (the result of a rounding that may fall on
+    either side of a tie)."""
+    from paper_2605_09877_b200 import kvm
+    gen = torch.Generator().manual_seed(7 * B + T)
+    x = (torch.randn((B, H, T, d), generator=gen) * 2.0 + 0.5).to(torch.bfloat16)
+    w = (1.0 + 0.3 * torch.randn((H, d), generator=gen)).float() if affine else None
+    b = (0.2 * torch.randn((H, d), generator=gen)).float() if affine else None
+    ref = head_layernorm(x.double().numpy(), None if w is None else w.double().numpy(),
+                         None if b is None else b.double().numpy(), 1e-5)
+    y = kvm.head_layernorm(x.cuda(), None if w is None else w.cuda(), None if b is None else b.cuda(), 1e-5)
+    torch.cuda.synchronize()
+    got = y.cpu().double().numpy()
+    assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-5)
