@@ -338,6 +338,88 @@ def run_gate(args):
     return 0
 
 
+def run_headln(args):
+    """Front-end LN_q / LN_k (kvm_head_layernorm, in place): HBM-bound, every element read and written
+    once.  "headln": the default workload's q (B2 H16 T8192 d128, 67 MB); "headln-paper": B8 H32 T32768
+    d128 (2.1 GB)."""
+    from paper_2605_09877_b200 import kvm
+    rank, world, local = dist_setup(args.gpus)
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    B, H, T, d = (8, 32, 32768, 128) if args.workload == "headln-paper" else (2, 16, 8192, 128)
+    pk = peaks()
+    W, K = max(args.warmup, 3), args.steps
+    gen = torch.Generator().manual_seed(200 + rank)
+    x_host = (torch.randn((B, H, T, d), generator=gen) * 2.0 + 0.5).to(torch.bfloat16).pin_memory()
+    w = (1.0 + 0.3 * torch.randn((H, d), generator=gen)).float().to(dev)
+    bia = (0.2 * torch.randn((H, d), generator=gen)).float().to(dev)
+    x = x_host.to(dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    bytes_step = 2 * B * H * T * d * 2
+    for _ in range(W):
+        x.copy_(x_host, non_blocking=True)
+        kvm.head_layernorm(x, w, bia)
+    barrier(world)
+    clocks = ClockSampler(local)
+    clocks.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for a, b in ev:
+        x.copy_(x_host, non_blocking=True)   # (the kernel works in place: fresh inputs every step, outside the bracket)
+        flush.zero_()
+        a.record()
+        kvm.head_layernorm(x, w, bia)
+        b.record()
+    torch.cuda.synchronize()
+    barrier(world)
+    clk = clocks.stop()
+    ms = sum(a.elapsed_time(b) for a, b in ev) / K
+    ms_all = max_over_ranks(ms, world)
+    y_host = torch.empty_like(x_host).pin_memory()
+    e2e = None
+    if not args.no_e2e:
+        t_e2e = []
+        for _ in range(3):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            x.copy_(x_host, non_blocking=True)
+            kvm.head_layernorm(x, w, bia)
+            y_host.copy_(x, non_blocking=True)
+            torch.cuda.synchronize()
+            t_e2e.append(time.perf_counter() - t0)
+        e2e = dict(value=world * B * T / min(t_e2e), unit="tokens/s", h2d_bytes_per_step=B * H * T * d * 2,
+                   d2h_bytes_per_step=B * H * T * d * 2)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        from oracle.frontend import head_layernorm as oracle_ln
+        nb = 1 if B * H * T * d > (1 << 27) else B
+        hs = H if nb == B else 4                       # a bounded sample of the large shape: 4 heads of one batch row
+        xs = x_host[:nb, :hs].double().numpy()
+        t0 = time.perf_counter()
+        ref = oracle_ln(xs, w[:hs].cpu().double().numpy(), bia[:hs].cpu().double().numpy(), 1e-5)
+        dt = time.perf_counter() - t0
+        got = y_host[:nb, :hs].double().numpy() if e2e else None
+        if got is not None:
+            assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-5)
+        cpu = dict(value=nb * T * hs / H / dt, unit="tokens/s", cores=os.cpu_count(), kind="oracle",
+                   sample=f"{hs} of {H} heads x {nb} of {B} batch rows x {T} tokens, {dt:.2f} s wall (numpy fp64; value = layer tokens/s at that rate)")
+    if rank == 0:
+        achieved = bytes_step / (ms * 1e-3) / 1e9
+        line = dict(metric="kvm_head_layernorm_tokens_per_s", value=world * B * T / (ms_all * 1e-3), unit="tokens/s",
+                    n_gpus=world, steps=K, warmup=W, ms_per_step=ms_all, higher_is_better=True, scaling="weak",
+                    vs_baseline=None, dtype="bf16 in/out, f32 statistics", data="synthetic",
+                    config=dict(workload=args.workload, mode="front end: LN_q / LN_k", B=B, H=H, T=T, d=d,
+                                l2="256 MiB flush between timed steps"),
+                    clocks=clk, e2e=e2e, gpu_launches=K,
+                    roofline=dict(bound="hbm", kernel="head_layernorm", achieved=achieved, peak=pk["hbm"], unit="GB/s",
+                                  frac=achieved / pk["hbm"], traffic=None, peak_source=pk["src"] + " copy bandwidth",
+                                  bytes_per_step=bytes_step),
+                    cpu_baseline=cpu)
+        print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -355,6 +437,8 @@ def main():
         return run_reference(args)
     if args.workload in ("gate", "gate-paper"):
         return run_gate(args)
+    if args.workload in ("headln", "headln-paper"):
+        return run_headln(args)
 
     from paper_2605_09877_b200 import kvm
     rank, world, local = dist_setup(args.gpus)
