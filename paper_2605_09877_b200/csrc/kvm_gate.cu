@@ -315,58 +315,69 @@ kvm_status_t kvm_merge_gate(const void* x, const float* w_gate, int32_t batch, i
 // statistics in fp32 through shuffles inside the lane group (biased variance, as LN_s).
 namespace kvm {
 
+constexpr int kLnRowsPerGroup = 4;   // rows per lane group, loaded up front: enough bytes in flight per SM for the HBM latency
+
 template <int D>
 __global__ void __launch_bounds__(256) head_layernorm_kernel(__nv_bfloat16* __restrict__ x, const float* __restrict__ weight,
                                                              const float* __restrict__ bias, int64_t rows, int64_t T, int H,
                                                              float eps) {
   constexpr int LPR = D / 8;                 // lanes per row: 8 (d = 64) or 16 (d = 128)
-  constexpr int RPW = 32 / LPR;              // rows per warp
+  constexpr int RPW = 32 / LPR;              // lane groups per warp
+  constexpr int NR = kLnRowsPerGroup;
   const int lane = threadIdx.x & 31, sub = lane % LPR;
   const int64_t warp_global = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const int64_t row = warp_global * RPW + lane / LPR;
-  const bool live = row < rows;               // (dead groups still take part in the shuffles)
-  const int64_t rr = live ? row : rows - 1;
-  const int h = (int)((rr / T) % H);          // rows are [B, H, T]
-  __nv_bfloat16* p = x + rr * D + sub * 8;
-  const uint4 raw = *reinterpret_cast<const uint4*>(p);
-  const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
-  float v[8];
+  const int64_t row0 = warp_global * (RPW * NR) + lane / LPR;   // this group's rows: row0 + k RPW
+  uint4 raw[NR];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const float2 f = __bfloat1622float2(p2[i]);
-    v[2 * i] = f.x; v[2 * i + 1] = f.y;
+  for (int k = 0; k < NR; ++k) {
+    const int64_t rr = min(row0 + k * RPW, rows - 1);   // (a clamped duplicate is computed and not stored: the shuffles need every lane)
+    raw[k] = *reinterpret_cast<const uint4*>(x + rr * D + sub * 8);
   }
-  float s = 0.f;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) s += v[i];
+  for (int k = 0; k < NR; ++k) {
+    const int64_t row = row0 + k * RPW;
+    const bool live = row < rows;
+    const int64_t rr = live ? row : rows - 1;
+    const int h = (int)((rr / T) % H);          // rows are [B, H, T]
+    const __nv_bfloat162* p2 = reinterpret_cast<const __nv_bfloat162*>(&raw[k]);
+    float v[8];
 #pragma unroll
-  for (int o = LPR / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-  const float mean = s * (1.f / D);
-  float q = 0.f;
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __bfloat1622float2(p2[i]);
+      v[2 * i] = f.x; v[2 * i + 1] = f.y;
+    }
+    float s = 0.f;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) q += (v[i] - mean) * (v[i] - mean);
+    for (int i = 0; i < 8; ++i) s += v[i];
 #pragma unroll
-  for (int o = LPR / 2; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
-  const float rstd = rsqrtf(q * (1.f / D) + eps);
-  float wv[8], bv[8];
+    for (int o = LPR / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    const float mean = s * (1.f / D);
+    float q = 0.f;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) { wv[i] = 1.f; bv[i] = 0.f; }
-  if (weight) {
-    const float4 a = *reinterpret_cast<const float4*>(weight + (int64_t)h * D + sub * 8), b = *reinterpret_cast<const float4*>(weight + (int64_t)h * D + sub * 8 + 4);
-    wv[0] = a.x; wv[1] = a.y; wv[2] = a.z; wv[3] = a.w; wv[4] = b.x; wv[5] = b.y; wv[6] = b.z; wv[7] = b.w;
+    for (int i = 0; i < 8; ++i) q += (v[i] - mean) * (v[i] - mean);
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
+    const float rstd = rsqrtf(q * (1.f / D) + eps);
+    float wv[8], bv[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { wv[i] = 1.f; bv[i] = 0.f; }
+    if (weight) {
+      const float4 a = *reinterpret_cast<const float4*>(weight + (int64_t)h * D + sub * 8), b = *reinterpret_cast<const float4*>(weight + (int64_t)h * D + sub * 8 + 4);
+      wv[0] = a.x; wv[1] = a.y; wv[2] = a.z; wv[3] = a.w; wv[4] = b.x; wv[5] = b.y; wv[6] = b.z; wv[7] = b.w;
+    }
+    if (bias) {
+      const float4 a = *reinterpret_cast<const float4*>(bias + (int64_t)h * D + sub * 8), b = *reinterpret_cast<const float4*>(bias + (int64_t)h * D + sub * 8 + 4);
+      bv[0] = a.x; bv[1] = a.y; bv[2] = a.z; bv[3] = a.w; bv[4] = b.x; bv[5] = b.y; bv[6] = b.z; bv[7] = b.w;
+    }
+    uint32_t out[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __nv_bfloat162 o2 = __floats2bfloat162_rn(fmaf((v[2 * i] - mean) * rstd, wv[2 * i], bv[2 * i]),
+                                                      fmaf((v[2 * i + 1] - mean) * rstd, wv[2 * i + 1], bv[2 * i + 1]));
+      out[i] = *reinterpret_cast<const uint32_t*>(&o2);
+    }
+    if (live) *reinterpret_cast<uint4*>(x + rr * D + sub * 8) = make_uint4(out[0], out[1], out[2], out[3]);
   }
-  if (bias) {
-    const float4 a = *reinterpret_cast<const float4*>(bias + (int64_t)h * D + sub * 8), b = *reinterpret_cast<const float4*>(bias + (int64_t)h * D + sub * 8 + 4);
-    bv[0] = a.x; bv[1] = a.y; bv[2] = a.z; bv[3] = a.w; bv[4] = b.x; bv[5] = b.y; bv[6] = b.z; bv[7] = b.w;
-  }
-  uint32_t out[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const __nv_bfloat162 o2 = __floats2bfloat162_rn(fmaf((v[2 * i] - mean) * rstd, wv[2 * i], bv[2 * i]),
-                                                    fmaf((v[2 * i + 1] - mean) * rstd, wv[2 * i + 1], bv[2 * i + 1]));
-    out[i] = *reinterpret_cast<const uint32_t*>(&o2);
-  }
-  if (live) *reinterpret_cast<uint4*>(p) = make_uint4(out[0], out[1], out[2], out[3]);
 }
 
 }  // namespace kvm
@@ -379,7 +390,7 @@ kvm_status_t kvm_head_layernorm(void* x, const float* weight, const float* bias,
   if (head_dim != 64 && head_dim != 128) return KVM_ERR_UNSUPPORTED;
   cudaStream_t s = (cudaStream_t)cuda_stream;
   const int64_t rows = (int64_t)batch * n_heads * n_tokens;
-  const int rows_per_cta = 8 * (32 / (head_dim / 8));
+  const int rows_per_cta = 8 * (32 / (head_dim / 8)) * kvm::kLnRowsPerGroup;
   const int64_t ctas = (rows + rows_per_cta - 1) / rows_per_cta;
   if (ctas > 0x7fffffff) return KVM_ERR_UNSUPPORTED;
   __nv_bfloat16* xp = (__nv_bfloat16*)x;
