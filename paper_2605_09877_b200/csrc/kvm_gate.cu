@@ -333,6 +333,10 @@ __global__ void __launch_bounds__(256) head_layernorm_kernel(__nv_bfloat16* __re
     const int64_t rr = min(row0 + k * RPW, rows - 1);   // (a clamped duplicate is computed and not stored: the shuffles need every lane)
     raw[k] = *reinterpret_cast<const uint4*>(x + rr * D + sub * 8);
   }
+  float wv[8], bv[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { wv[i] = 1.f; bv[i] = 0.f; }
+  int h_cur = -1;
 #pragma unroll
   for (int k = 0; k < NR; ++k) {
     const int64_t row = row0 + k * RPW;
@@ -358,16 +362,16 @@ __global__ void __launch_bounds__(256) head_layernorm_kernel(__nv_bfloat16* __re
 #pragma unroll
     for (int o = LPR / 2; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
     const float rstd = rsqrtf(q * (1.f / D) + eps);
-    float wv[8], bv[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) { wv[i] = 1.f; bv[i] = 0.f; }
-    if (weight) {
-      const float4 a = *reinterpret_cast<const float4*>(weight + (int64_t)h * D + sub * 8), b = *reinterpret_cast<const float4*>(weight + (int64_t)h * D + sub * 8 + 4);
-      wv[0] = a.x; wv[1] = a.y; wv[2] = a.z; wv[3] = a.w; wv[4] = b.x; wv[5] = b.y; wv[6] = b.z; wv[7] = b.w;
-    }
-    if (bias) {
-      const float4 a = *reinterpret_cast<const float4*>(bias + (int64_t)h * D + sub * 8), b = *reinterpret_cast<const float4*>(bias + (int64_t)h * D + sub * 8 + 4);
-      bv[0] = a.x; bv[1] = a.y; bv[2] = a.z; bv[3] = a.w; bv[4] = b.x; bv[5] = b.y; bv[6] = b.z; bv[7] = b.w;
+    if (h != h_cur) {   // consecutive rows nearly always belong to one head: its weights stay in registers
+      h_cur = h;
+      if (weight) {
+        const float4 a = *reinterpret_cast<const float4*>(weight + (int64_t)h * D + sub * 8), b = *reinterpret_cast<const float4*>(weight + (int64_t)h * D + sub * 8 + 4);
+        wv[0] = a.x; wv[1] = a.y; wv[2] = a.z; wv[3] = a.w; wv[4] = b.x; wv[5] = b.y; wv[6] = b.z; wv[7] = b.w;
+      }
+      if (bias) {
+        const float4 a = *reinterpret_cast<const float4*>(bias + (int64_t)h * D + sub * 8), b = *reinterpret_cast<const float4*>(bias + (int64_t)h * D + sub * 8 + 4);
+        bv[0] = a.x; bv[1] = a.y; bv[2] = a.z; bv[3] = a.w; bv[4] = b.x; bv[5] = b.y; bv[6] = b.z; bv[7] = b.w;
+      }
     }
     uint32_t out[4];
 #pragma unroll
