@@ -903,6 +903,8 @@ __global__ void __launch_bounds__(256, 4) fold_apply_kernel(FoldApplyParams p) {
     for (int i = 0; i < CH; ++i) v2 += (double)vx[i] * (double)vx[i];
     const double vnorm = sqrt(warp_sum_d(v2));
     const double den = vnorm > p.norm_eps ? vnorm : p.norm_eps;
+    // one fp64 divide per row instead of one per channel (the readout values are rounded to fp16)
+    const double vscale = p.radius_on ? rad / den : 1.0 / wacc;
 #pragma unroll
     for (int i = 0; i < CH; ++i) {
       const int x = lane + 32 * i;
@@ -910,7 +912,7 @@ __global__ void __launch_bounds__(256, 4) fold_apply_kernel(FoldApplyParams p) {
       p.sumK[row * D + x] = kx[i];
       p.sumV[row * D + x] = vx[i];
       p.Khat[row * D + x] = __float2half_rn((float)hat);
-      const double vo = p.radius_on ? (rad * (double)vx[i] / den) : ((double)vx[i] / wacc);
+      const double vo = (double)vx[i] * vscale;
       p.Vhat[row * D + x] = __float2half_rn((float)vo);
     }
     if (lane == 0) {
