@@ -797,6 +797,8 @@ struct FoldApplyParams {
   double ln_eps, norm_eps;
 };
 
+// One touched row per warp: the shorter chain per row; used when a launch has too few rows to fill the
+// GPU, where the latency of a row is what counts.
 template <int D>
 __global__ void __launch_bounds__(256, 4) fold_apply_kernel(FoldApplyParams p) {
   constexpr int CH = D / 32;
@@ -916,6 +918,185 @@ __global__ void __launch_bounds__(256, 4) fold_apply_kernel(FoldApplyParams p) {
       p.Vhat[row * D + x] = __float2half_rn((float)vo);
     }
     if (lane == 0) {
+      p.rho[row] = (float)rad;
+      p.wsum[row] = wacc;
+      p.cnt[row] = nacc;
+      p.kmu[row] = mu;
+      p.krstd[row] = rs;
+    }
+  }
+}
+
+// Four touched rows per warp, eight lanes per row (lane `sub` of a group holds channels
+// 32 i + 4 sub .. + 3, as in the memory-key kernel): the fp64 reductions, square roots and divides of
+// a row are instructions of the whole warp, so one row per warp spent most of its instructions on
+// them, and four rows per warp also put four times the loads in flight.  The member loop of a group
+// runs without exchanges between lanes (each lane sums its own channels, members in ascending token
+// order: reproducible); all lanes meet again for the reductions.
+constexpr int kApplyRowsPerWarp = 4;
+constexpr int kApplyRowsPerCta = 8 * kApplyRowsPerWarp;
+
+template <int D>
+__global__ void __launch_bounds__(256, 2) fold_apply_rows4_kernel(FoldApplyParams p) {
+  constexpr int NI = D / 32;          // runs of four channels per lane
+  constexpr int NC = 4 * NI;          // channels per lane
+  constexpr double inv_d = 1.0 / D;   // D is a power of two: multiplying is dividing, exactly
+  __shared__ int s_pi[kMaxBlock], s_sorted[kMaxBlock], s_creator[kMaxBlock], s_segnew[kMaxBlock];
+  // the routing filter of the next fold may start its set-up now; it waits for this grid to finish
+  // before it reads the readout keys written here
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int u = blockIdx.y, hk = u % p.Hkv;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, sub = lane & 7;
+  const int q = (blockIdx.x * 8 + warp) * kApplyRowsPerWarp + (lane >> 3);
+  const int64_t tokBase = (int64_t)u * p.Cmax;
+  if (!p.all_append) {   // the decisions of this unit, read once per CTA instead of chased per warp
+    for (int i = threadIdx.x; i < p.C; i += 256) {
+      s_pi[i] = p.pi[tokBase + i];
+      s_sorted[i] = p.sorted[tokBase + i];
+      s_creator[i] = p.creator[tokBase + i];
+      s_segnew[i] = p.segnew[tokBase + i];
+    }
+    __syncthreads();
+  }
+  if ((blockIdx.x * 8 + warp) * kApplyRowsPerWarp >= p.C) return;   // (whole warp)
+  const int64_t rowBase = (int64_t)u * p.Mcap;
+  const double* kbarU = p.kbar64 + tokBase * D;
+  const __half* ovU = p.ov + (int64_t)u * p.unit_stride;
+  const float* ogU = p.og + (int64_t)u * p.gate_stride;
+  const int nmerge = p.all_append ? 0 : p.nmerge[u];
+  const int m = (int)p.m;
+
+  // task 0: the q-th appended row; task 1: the segment of an old row whose head sits at sorted[q]
+  for (int task = 0; task < 2; ++task) {
+    bool act = q < p.C;
+    int rowi = 0, seg = -1, jc = -1;
+    if (act) {
+      if (task == 0) {
+        if (q >= p.n_append) act = false;
+        else {
+          rowi = m + q;
+          jc = p.all_append ? q : s_creator[q];
+          seg = p.all_append ? -1 : s_segnew[q];
+        }
+      } else {
+        if (q >= nmerge) act = false;
+        else {
+          const int j0 = s_sorted[q];
+          rowi = s_pi[j0];
+          if (rowi >= m) act = false;                                          // new rows are task 0
+          else if (q > 0 && s_pi[s_sorted[q - 1]] == rowi) act = false;        // not a head
+          seg = q;
+        }
+      }
+    }
+    if (!__any_sync(0xffffffffu, act)) continue;
+    const int64_t row = rowBase + rowi;
+    double kx[NC];
+    float vx[NC];
+    double wacc = 1.0, rad = 0.0, v2 = 0.0;
+    int nacc = 1;
+#pragma unroll
+    for (int c = 0; c < NC; ++c) { kx[c] = 0.0; vx[c] = 0.f; }
+    if (act) {
+      if (task == 0) {
+        const double* kb = kbarU + (int64_t)jc * D;
+        const __half* vr = ovU + (int64_t)jc * D;
+#pragma unroll
+        for (int i = 0; i < NI; ++i) {
+          const int x = 32 * i + 4 * sub;
+          const double2 k01 = *reinterpret_cast<const double2*>(kb + x), k23 = *reinterpret_cast<const double2*>(kb + x + 2);
+          kx[4 * i] = k01.x; kx[4 * i + 1] = k01.y; kx[4 * i + 2] = k23.x; kx[4 * i + 3] = k23.y;
+          alignas(8) __half hv[4];
+          *reinterpret_cast<uint2*>(hv) = *reinterpret_cast<const uint2*>(vr + x);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            vx[4 * i + e] = __half2float(hv[e]);
+            v2 += (double)vx[4 * i + e] * (double)vx[4 * i + e];
+          }
+        }
+        if (sub == 0 && p.slotTok && p.b + jc < p.Tassign) {
+          p.slotTok[(int64_t)u * p.Tassign + p.b + jc] = rowi;
+          p.appTok[(int64_t)u * p.Tassign + p.b + jc] = 1;
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < NI; ++i) {
+          const int x = 32 * i + 4 * sub;
+          const double2 k01 = *reinterpret_cast<const double2*>(p.sumK + row * D + x), k23 = *reinterpret_cast<const double2*>(p.sumK + row * D + x + 2);
+          kx[4 * i] = k01.x; kx[4 * i + 1] = k01.y; kx[4 * i + 2] = k23.x; kx[4 * i + 3] = k23.y;
+          const float4 v4 = *reinterpret_cast<const float4*>(p.sumV + row * D + x);
+          vx[4 * i] = v4.x; vx[4 * i + 1] = v4.y; vx[4 * i + 2] = v4.z; vx[4 * i + 3] = v4.w;
+        }
+        wacc = p.wsum[row];
+        nacc = p.cnt[row];
+        rad = (double)p.rho[row];
+      }
+    }
+    // radius of a new row = the norm of its creator's value, kept in fp32 (all lanes: group reduction)
+    v2 = group8_sum_d(v2);
+    if (task == 0) rad = (double)(float)sqrt(v2);
+    if (act && seg >= 0) {
+      for (int qq = seg; qq < nmerge; ++qq) {
+        const int j = s_sorted[qq];
+        if (s_pi[j] != rowi) break;
+        const float g = ogU[j];
+        const double* kb = kbarU + (int64_t)j * D;
+        const __half* vr = ovU + (int64_t)j * D;
+#pragma unroll
+        for (int i = 0; i < NI; ++i) {
+          const int x = 32 * i + 4 * sub;
+          const double2 k01 = *reinterpret_cast<const double2*>(kb + x), k23 = *reinterpret_cast<const double2*>(kb + x + 2);
+          kx[4 * i] += (double)g * k01.x; kx[4 * i + 1] += (double)g * k01.y;
+          kx[4 * i + 2] += (double)g * k23.x; kx[4 * i + 3] += (double)g * k23.y;
+          alignas(8) __half hv[4];
+          *reinterpret_cast<uint2*>(hv) = *reinterpret_cast<const uint2*>(vr + x);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) vx[4 * i + e] = fmaf(g, __half2float(hv[e]), vx[4 * i + e]);
+        }
+        wacc += (double)g;
+        nacc += 1;
+        if (sub == 0 && p.slotTok && p.b + j < p.Tassign) {
+          p.slotTok[(int64_t)u * p.Tassign + p.b + j] = rowi;
+          p.appTok[(int64_t)u * p.Tassign + p.b + j] = 0;
+        }
+      }
+    }
+    // all lanes again: LayerNorm statistics of the key sum, norm of the value sum
+    double sum = 0.0;
+#pragma unroll
+    for (int c = 0; c < NC; ++c) sum += kx[c];
+    const double mu = group8_sum_d(sum) * inv_d;
+    double dev = 0.0, vv = 0.0;
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+      dev += (kx[c] - mu) * (kx[c] - mu);
+      vv += (double)vx[c] * (double)vx[c];
+    }
+    const double rs = 1.0 / sqrt(group8_sum_d(dev) * inv_d + p.ln_eps);
+    const double vnorm = sqrt(group8_sum_d(vv));
+    const double den = vnorm > p.norm_eps ? vnorm : p.norm_eps;
+    // one fp64 divide per row instead of one per channel (the readout values are rounded to fp16)
+    const double vscale = p.radius_on ? rad / den : 1.0 / wacc;
+    if (!act) continue;
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+      const int x = 32 * i + 4 * sub;
+      const float4 w4 = *reinterpret_cast<const float4*>(p.ln_w + hk * D + x), b4 = *reinterpret_cast<const float4*>(p.ln_b + hk * D + x);
+      const float wv[4] = {w4.x, w4.y, w4.z, w4.w}, bv[4] = {b4.x, b4.y, b4.z, b4.w};
+      alignas(8) __half kh[4], vh[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const double hat = (double)wv[e] * ((kx[4 * i + e] - mu) * rs) + (double)bv[e];
+        kh[e] = __float2half_rn((float)hat);
+        vh[e] = __float2half_rn((float)((double)vx[4 * i + e] * vscale));
+      }
+      reinterpret_cast<double2*>(p.sumK + row * D + x)[0] = make_double2(kx[4 * i], kx[4 * i + 1]);
+      reinterpret_cast<double2*>(p.sumK + row * D + x)[1] = make_double2(kx[4 * i + 2], kx[4 * i + 3]);
+      *reinterpret_cast<float4*>(p.sumV + row * D + x) = make_float4(vx[4 * i], vx[4 * i + 1], vx[4 * i + 2], vx[4 * i + 3]);
+      *reinterpret_cast<uint2*>(p.Khat + row * D + x) = *reinterpret_cast<const uint2*>(kh);
+      *reinterpret_cast<uint2*>(p.Vhat + row * D + x) = *reinterpret_cast<const uint2*>(vh);
+    }
+    if (sub == 0) {
       p.rho[row] = (float)rad;
       p.wsum[row] = wacc;
       p.cnt[row] = nacc;
@@ -1056,9 +1237,17 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
   q.ln_eps = (double)st->ln_eps; q.norm_eps = (double)st->norm_eps;
   if (a.before_apply && cudaStreamWaitEvent(s, a.before_apply, 0) != cudaSuccess) return -1000000;
   KernelTimer kt(st, 5, s);
-  dim3 grid((C + 7) / 8, st->U);
-  if (D == 128) fold_apply_kernel<128><<<grid, 256, 0, s>>>(q);
-  else fold_apply_kernel<64><<<grid, 256, 0, s>>>(q);
+  // four rows per warp when the launch is bound by throughput (measured: better from 8192 rows on:
+  // U = 32, C = 256; worse at 4096 and 2048 rows, where the longer chain per row shows)
+  if ((int64_t)C * st->U >= 8192) {
+    dim3 grid((C + kApplyRowsPerCta - 1) / kApplyRowsPerCta, st->U);
+    if (D == 128) fold_apply_rows4_kernel<128><<<grid, 256, 0, s>>>(q);
+    else fold_apply_rows4_kernel<64><<<grid, 256, 0, s>>>(q);
+  } else {
+    dim3 grid((C + 7) / 8, st->U);
+    if (D == 128) fold_apply_kernel<128><<<grid, 256, 0, s>>>(q);
+    else fold_apply_kernel<64><<<grid, 256, 0, s>>>(q);
+  }
   ++launches;
   st->prevValid = true; st->prevAllAppend = all_append; st->prevM = a.m; st->prevNAppend = a.n_append;
   return launches;
