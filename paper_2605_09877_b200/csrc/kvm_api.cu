@@ -322,8 +322,9 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   if (rc == KVM_OK && cudaMemset(s.xCount, 0, U * sizeof(int32_t)) != cudaSuccess) rc = KVM_ERR_CUDA;
   A(s.candV, U * (size_t)(2 * s.nsplitRoute) * Cm * kTopK); A(s.candI, U * (size_t)(2 * s.nsplitRoute) * Cm * kTopK);
   A(s.decPart, (size_t)s.B * s.Hq * s.nsplitDec * (d + 2)); A(s.decQ, (size_t)s.B * s.Hq * d);
-  A(s.attnPart, (size_t)kAttnSplitTiles * kAttnMaxSplits * (d + 2) * 128); A(s.attnCnt, (size_t)kAttnSplitTiles);
-  if (rc == KVM_OK && cudaMemset(s.attnCnt, 0, kAttnSplitTiles * sizeof(int32_t)) != cudaSuccess) rc = KVM_ERR_CUDA;
+  // (tiles x splits: up to kAttnSplitTiles x kAttnMaxSplits, or 2 kAttnSplitTiles tiles of two splits)
+  A(s.attnPart, (size_t)kAttnSplitTiles * kAttnMaxSplits * (d + 2) * 128); A(s.attnCnt, (size_t)2 * kAttnSplitTiles);
+  if (rc == KVM_OK && cudaMemset(s.attnCnt, 0, 2 * kAttnSplitTiles * sizeof(int32_t)) != cudaSuccess) rc = KVM_ERR_CUDA;
   A(s.status, (size_t)16);   // [0] status word, [1..3] fold debug counters
   if (s.Tassign > 0) { A(s.slotTok, U * (size_t)s.Tassign); A(s.appTok, U * (size_t)s.Tassign); }
 #undef A

@@ -22,8 +22,9 @@
 //               memory, and the S accumulator is handed back to the QK^T issuer when the PV product
 //               has consumed it.  O is rescaled in TMEM only when the max grew by more than 2^8
 //               (each half rescales, and at the end normalises and stores, its share of the channels).
-// With few query tiles per launch the key tiles are also split over gridDim.z CTAs whose partial
-// results are merged by the CTA that finishes last.
+// With few query tiles per launch the key tiles are also split over several CTAs whose partial
+// results are merged by the CTA that finishes last; with many, the tiles that would make up a last,
+// less than half full wave of CTAs are each split in two, so that the wave is half as long.
 // Every mbarrier wait is bounded; on expiry the CTA records KVM_ERR_TIMEOUT and tears down.
 #include "kvm_internal.h"
 #include "tc_common.cuh"
@@ -39,6 +40,9 @@ struct AttnTcParams {
   float* part;       // split-KV partial results, [tile][split][D + 2][128] (see the epilogue)
   int32_t* part_cnt; // [tile] tickets, zero between launches
   int nq, Hq, Hkv, G;
+  int qtiles;        // query tiles per (batch, head)
+  int n_whole;       // the first n_whole (batch, head, query tile) tiles have one CTA each,
+  int nsp_rest;      // the others nsp_rest CTAs each (key splits)
   int out_vec;       // rows of `out` can be written with 16-byte stores (alignment of base and strides)
 };
 
@@ -117,7 +121,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int qt = blockIdx.x, bh = blockIdx.y;
+  // linear CTA index -> (tile, split): whole tiles first, then the split ones
+  int tile, sp, nsp;
+  if ((int)blockIdx.x < p.n_whole) { tile = blockIdx.x; sp = 0; nsp = 1; }
+  else { const int r = (int)blockIdx.x - p.n_whole; tile = p.n_whole + r / p.nsp_rest; sp = r % p.nsp_rest; nsp = p.nsp_rest; }
+  const int tile_slot = tile - p.n_whole;   // index among the split tiles (partial results, tickets)
+  const int qt = tile % p.qtiles, bh = tile / p.qtiles;
   const int bb = bh / p.Hq, hq = bh % p.Hq, hk = hq / p.G;
   const int u = bb * p.Hkv + hk;
   const int rows_valid = min(128, p.nq - qt * 128);
@@ -126,9 +135,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
   const int nst = (int)((p.m + 127) / 128);
   const int nwt = (int)((t_last - p.b + 1 + 127) / 128);
   // Split-KV: with few (batch, head, query tile) triples a launch is cut along the keys as well;
-  // CTA z of gridDim.z walks tiles [jbase, jbase + ntiles) of the nst + nwt tiles of its query tile,
+  // CTA sp of nsp walks tiles [jbase, jbase + ntiles) of the nst + nwt tiles of its query tile,
   // and the partial results are merged by whichever CTA of the tile finishes last.
-  const int nsp = (int)gridDim.z, sp = (int)blockIdx.z;
   const int ntot = nst + nwt;
   const int per_split = (ntot + nsp - 1) / nsp;
   const int jbase = min(ntot, sp * per_split);
@@ -440,7 +448,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__
     } else {
       // Partial result of this split: unnormalised O (relative to m_run), m_run and the sum, column-major
       // ([channel][row]) so that the rows of a warp are contiguous.
-      const int tile_id = bh * (int)gridDim.x + qt;
+      const int tile_id = tile_slot;
       float* mine = p.part + ((int64_t)tile_id * nsp + sp) * (D + 2) * 128;
       if (good && ntiles > 0) {
 #pragma unroll
@@ -557,7 +565,17 @@ int launch_attn_tc(State* st, const AttnArgs& a, cudaStream_t s) {
     if (nsp > kAttnMaxSplits) nsp = kAttnMaxSplits;
     if (nsp < 1) nsp = 1;
   }
-  dim3 grid(qtiles, st->B * st->Hq, nsp);
+  // Many tiles: when the last wave of one-CTA-per-SM would be less than half full, its tiles are split
+  // in two (the partial-result buffer holds 2 * kAttnSplitTiles tiles of two splits).
+  const int tiles = qtiles * st->B * st->Hq;
+  int n_whole = nsp > 1 ? 0 : tiles, nsp_rest = nsp;
+  if (nsp == 1 && tiles > 148) {
+    const int rem = tiles % 148;
+    const int ntot_min2 = (int)((a.m + 127) / 128) + 1;
+    if (rem > 0 && rem <= 2 * kAttnSplitTiles && ntot_min2 >= 4) { n_whole = tiles - rem; nsp_rest = 2; }
+  }
+  p.qtiles = qtiles; p.n_whole = n_whole; p.nsp_rest = nsp_rest;
+  dim3 grid(n_whole + (tiles - n_whole) * nsp_rest);
   const CUtensorMap* tm = reinterpret_cast<const CUtensorMap*>(st->tmaps);
   const int ks = (st->nfolds & 1) ? 6 : 1, vs = (st->nfolds & 1) ? 7 : 2;   // readout copy of the current version
   if (st->d == 128) {

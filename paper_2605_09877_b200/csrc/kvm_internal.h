@@ -92,7 +92,7 @@ struct State {
   int32_t* candI;
   // ---- split-KV attention scratch (device) ----
   float* attnPart;               // [kAttnSplitTiles][kAttnMaxSplits][d + 2][128]
-  int32_t* attnCnt;              // [kAttnSplitTiles] tickets
+  int32_t* attnCnt;              // [2 kAttnSplitTiles] tickets
   // ---- decode scratch (device) ----
   int nsplitDec;
   float* decPart;                // [B*Hq, nsplitDec, d + 2]

@@ -98,6 +98,13 @@ def test_power_law_and_saturating_budgets(kw):
     print(_run(wl))
 
 
+def test_attention_with_more_tiles_than_sms_splits_the_last_partial_wave():
+    """160 (head, query tile) pairs on 148 SMs: the 12 tiles of the last wave run as two key splits each
+    while the others keep one CTA; outputs must not show which tiles were split."""
+    wl = synth.Workload("t", 1, 80, 80, 64, 256 * 5 + 60, 256, "sqrt", sqrt_coeff=16, r=16, seed=21)
+    print(_run(wl))
+
+
 def test_radius_switch_off():
     wl = synth.Workload("t", 1, 2, 2, 64, 640, 32, "fixed", fixed_slots=48, seed=14)
     print(_run(wl, radius_on=False, gate=True))
