@@ -105,6 +105,14 @@ def test_attention_with_more_tiles_than_sms_splits_the_last_partial_wave():
     print(_run(wl))
 
 
+def test_many_rows_per_fold_use_the_four_rows_per_warp_apply_kernel():
+    """32 units x 256 tokens = 8192 rows per fold: the apply variant for large launches, head_dim 128,
+    gates and affine LayerNorm included."""
+    wl = synth.Workload("t", 2, 16, 16, 128, 256 * 4 + 70, 256, "sqrt", sqrt_coeff=12, r=32, seed=22, kind="mixture")
+    params = synth.make_layer_params(wl, trivial=False)
+    print(_run(wl, params=params, gate=True))
+
+
 def test_radius_switch_off():
     wl = synth.Workload("t", 1, 2, 2, 64, 640, 32, "fixed", fixed_slots=48, seed=14)
     print(_run(wl, radius_on=False, gate=True))
