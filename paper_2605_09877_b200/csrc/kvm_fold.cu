@@ -479,8 +479,11 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
       s_pcnt[j] = c;
       s_fill[j] = (single && !exh) ? -1 : 0;
       s_exh[j] = exh ? 1 : 0;
-      if (c > 0) atomicMax(&s_np, start + c);   // pairs of the lists that were kept form a prefix of the buffer
     }
+    // pairs of the lists that were kept form a prefix of the buffer: its end, one atomic per warp
+    // (256 atomics on one shared-memory word serialise)
+    const unsigned wend = __reduce_max_sync(0xffffffffu, (unsigned)((mine && c > 0) ? start + c : 0));
+    if (lane == 0 && wend > 0) atomicMax(&s_np, (int)wend);
     const int ne = __syncthreads_count(mine && exh);   // tokens of the slice that take the exhaustive path
     if (tid == 0) s_nexh += ne;
   }
@@ -734,7 +737,8 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
     }
   }
   __syncthreads();
-  if (tid < C && !s_app[tid]) {
+  const bool merged = tid < C && !s_app[tid];
+  if (merged) {
     double best = s_best[tid];
     int arg = s_barg[tid];
     if (n_a > 0 && !s_exh[tid]) {
@@ -745,9 +749,11 @@ __global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDeci
       }
     }
     s_pi[tid] = arg;
-    atomicAdd(&s_nmerge, 1);
   }
-  __syncthreads();
+  {   // number of merged tokens: a block-wide count (an atomic per token on one word would serialise)
+    const int nm = __syncthreads_count(merged);
+    if (tid == 0) s_nmerge = nm;
+  }
   // ---- E: order merged tokens by (row, token); publish ----
   {
     unsigned* ekey = reinterpret_cast<unsigned*>(s_prow);   // (the pair list is idle here)
