@@ -152,6 +152,22 @@ def test_run_to_run_determinism():
         assert torch.equal(y, outs[0][0]) and np.array_equal(sk, outs[0][1]) and np.array_equal(sv, outs[0][2])
 
 
+def test_run_to_run_determinism_with_split_tail_and_four_row_apply():
+    """The shape of the many-tiles test (key splits on the last wave, whose merge order is fixed by
+    construction, and the apply variant for large launches): three runs, identical bits."""
+    wl = synth.Workload("t", 1, 80, 80, 64, 256 * 4 + 30, 256, "sqrt", sqrt_coeff=16, r=16, seed=23)
+    tensors = synth.make_inputs(wl)
+    params = synth.make_layer_params(wl)
+    outs = []
+    for _ in range(3):
+        y, st = pu.run_gpu(wl, tensors, params)
+        e = st.export()
+        outs.append((y, e["sum_k"].copy(), e["sum_v"].copy()))
+        st.free()
+    for y, sk, sv in outs[1:]:
+        assert torch.equal(y, outs[0][0]) and np.array_equal(sk, outs[0][1]) and np.array_equal(sv, outs[0][2])
+
+
 def test_host_buffer_entry_points_match_device_ones():
     from paper_2605_09877_b200 import kvm
     wl = CFG["cfg1"].scaled(T=300)
