@@ -43,7 +43,7 @@ def test_gate_matches_the_library_elu_and_a_plain_matmul():
 @pytest.mark.gpu
 @pytest.mark.parametrize("B,T,dm,H", [(2, 777, 1000, 3), (1, 64, 2048, 16), (3, 130, 72, 40), (2, 1, 256, 8),
                                       (1, 4096, 1024, 64), (2, 300, 512, 24), (1, 200, 256, 40), (2, 129, 64, 9),
-                                      (1, 1, 4096, 32)])
+                                      (1, 1, 4096, 32), (4, 19000, 128, 24), (2, 40000, 64, 40)])
 def test_gate_kernel_against_the_oracle(B, T, dm, H):
     """Shapes cover both kernels (tensor cores when d_model is a multiple of 64 and there are more
     than 8 heads, else scalar cores), every head padding, ragged token tiles and a single token.
