@@ -365,8 +365,10 @@ __device__ __forceinline__ void sort_n(K& key, int& val, K* sk, int* sv, int t) 
   }
 }
 
-template <int D>
-__global__ void __launch_bounds__(kDecideThreads, 2) fold_decide_kernel(FoldDecideParams p) {
+// PER_SM = 2 for grids that fill the GPU twice over (64 registers, a few spills), 1 for the small grids
+// of chain-bound shapes, where a CTA has an SM to itself anyway and keeps everything in registers.
+template <int D, int PER_SM>
+__global__ void __launch_bounds__(kDecideThreads, PER_SM) fold_decide_kernel(FoldDecideParams p) {
   constexpr int CH = D / 32;
   __shared__ double s_score[kMaxBlock], s_best[kMaxBlock];
   __shared__ int s_barg[kMaxBlock], s_pi[kMaxBlock], s_creator[kMaxBlock];
@@ -1225,8 +1227,9 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
     const bool pdl = st->prof_hook == nullptr && !(st->flags & KVM_FLAG_SIMT_ROUTING) &&
                      (sms_wanted <= 148 || st->U >= 148);
     lc.attrs = at; lc.numAttrs = pdl ? 1 : 0;
-    if (D == 128) cudaLaunchKernelEx(&lc, fold_decide_kernel<128>, p);
-    else cudaLaunchKernelEx(&lc, fold_decide_kernel<64>, p);
+    const bool roomy = R * st->U <= 148;
+    if (D == 128) { if (roomy) cudaLaunchKernelEx(&lc, fold_decide_kernel<128, 1>, p); else cudaLaunchKernelEx(&lc, fold_decide_kernel<128, 2>, p); }
+    else { if (roomy) cudaLaunchKernelEx(&lc, fold_decide_kernel<64, 1>, p); else cudaLaunchKernelEx(&lc, fold_decide_kernel<64, 2>, p); }
     ++launches;
   }
   FoldApplyParams q;
