@@ -18,8 +18,9 @@
  *     allocated once in kvm_state_create(); no call on the hot path allocates.
  *   - Work is enqueued on the given CUDA stream (a cudaStream_t passed as
  *     void*; NULL = default stream).  No entry point synchronises the host with
- *     the device except kvm_state_export / kvm_debug_assignments (which copy to
- *     host memory) and the *_host convenience variants.
+ *     the device except those that move data to or from HOST memory: kvm_state_export,
+ *     kvm_state_export_window, kvm_state_import, kvm_debug_assignments, kvm_debug_counters,
+ *     kvm_state_check, kvm_profile_read and the *_host convenience variants.
  *   - Host-side validation happens before any launch; a failed call leaves the
  *     state untouched.  There is no CPU fallback: without a CUDA device
  *     kvm_state_create() returns KVM_ERR_CUDA.
@@ -53,7 +54,7 @@ typedef enum {
   KVM_ERR_TIMEOUT = 7         /* a bounded device-side wait expired (status word)         */
 } kvm_status_t;
 
-/* State budget B(e) of Section 3.2 ("We choose n_append as follows"):
+/* State budget B(e) of Section 3.2, budget rule (M*, n_append):
  *   FIXED      B(e) = fixed_slots                        ("KVM 256")
  *   SQRT       B(e) = floor(sqrt_coeff * sqrt(e))        ("KVM sqrt", coeff 16), exact integer
  *   UNBOUNDED  B(e) = infinity (every overflow token is appended; test limit in
@@ -84,7 +85,9 @@ enum {
   KVM_FLAG_NO_RADIUS = 1u << 0,      /* ablation "no v-len normalization": read s^V out unnormalised */
   KVM_FLAG_RECORD_ASSIGN = 1u << 1,  /* keep per-token slot ids / append flags for kvm_debug_assignments */
   KVM_FLAG_SIMT_ATTENTION = 1u << 2, /* use the scalar-core attention kernel (cross-check path) */
-  KVM_FLAG_SIMT_ROUTING = 1u << 3    /* use the scalar-core routing filter (cross-check path)   */
+  KVM_FLAG_SIMT_ROUTING = 1u << 3,   /* use the scalar-core routing filter (cross-check path)   */
+  KVM_FLAG_MIN_KEY_SLOTS = 1u << 4   /* debug: keep only the minimum of two memory-key slots (the look-ahead
+                                        of one block that very large batches run with), whatever the size */
 };
 
 typedef struct {
@@ -189,6 +192,46 @@ kvm_status_t kvm_state_export(kvm_state_t* state, double* sum_k, float* sum_v, f
                               double* weight, int32_t* count, void* k_read, void* v_read,
                               void* cuda_stream);
 
+/* Checkpoint / resume (Section 3.2 "Terminology": the state is what is carried from one chunk to the
+ * later ones).  A snapshot is kvm_state_snapshot_info + the arrays of kvm_state_export (sums, radii,
+ * weights, counts) + the uncompressed window of kvm_state_export_window; kvm_state_import loads it into
+ * a state of the same shape (batch, heads, head_dim, n_bswa_chunks, sink_len, LayerNorm parameters and
+ * temperatures are the state's own and are not part of a snapshot), after which kvm_prefill /
+ * kvm_decode_step continue exactly -- bit for bit -- where the exported state stood. */
+typedef struct {
+  int32_t block, rope_dims;      /* bound by the first kvm_prefill; 0 / 0 while unbound               */
+  kvm_growth_t growth;
+  int64_t n_slots, position, n_folds;
+  int64_t window_begin;          /* tokens [window_begin, position) are held uncompressed             */
+  int64_t window_len;            /* position - window_begin, < (n_bswa_chunks + 1) * block             */
+} kvm_snapshot_info_t;
+
+/* Host bookkeeping only.  INVALID_ARG on NULL; a state that no prefill has bound yet reports zeros. */
+kvm_status_t kvm_state_snapshot_info(const kvm_state_t* state, kvm_snapshot_info_t* out);
+
+/* Copies the window tokens [window_begin, position) to HOST arrays (synchronises the stream):
+ *   win_k  fp16  [U, window_len, d]  keys as the window holds them (rotated by the partial RoPE)
+ *   win_v  fp16  [U, window_len, d]  values
+ *   win_gate float [U, window_len]   merge gates of those tokens
+ * Any pointer may be NULL.  STATE_MISMATCH when no prefill has bound the state yet. */
+kvm_status_t kvm_state_export_window(kvm_state_t* state, void* win_k, void* win_v, float* win_gate,
+                                     void* cuda_stream);
+
+/* Loads a snapshot (all arrays HOST memory, shapes as exported: [U, n_slots, ...] and
+ * [U, window_len, ...]; win_gate may be NULL = 1; the other arrays may be NULL only when their extent
+ * is zero).  The state's previous contents are dropped (as by kvm_state_reset) and block / growth /
+ * rope_dims are bound from `info`.  Row statistics and both readout caches are recomputed from the
+ * sums by the code that a fold uses, so the continuation equals the uninterrupted run bit for bit.
+ * With KVM_FLAG_RECORD_ASSIGN the recorded assignments of tokens before `position` are lost (-1).
+ * Validation (before anything is copied): info->n_slots and n_folds must be what the budget rule gives
+ * for `position`, window_begin / window_len what the block structure gives, block <= max_block,
+ * n_slots <= max_state_slots.  Synchronises the stream before returning.
+ * Errors: INVALID_ARG, UNSUPPORTED, CAPACITY, CUDA; a failed validation leaves the state untouched. */
+kvm_status_t kvm_state_import(kvm_state_t* state, const kvm_snapshot_info_t* info, const double* sum_k,
+                              const float* sum_v, const float* radius, const double* weight,
+                              const int32_t* count, const void* win_k, const void* win_v,
+                              const float* win_gate, void* cuda_stream);
+
 /* With KVM_FLAG_RECORD_ASSIGN: copies, for tokens [0, n) (n <= position, n <= max_seq_len),
  * slot_of_token int32 [U, n] (row merged into / appended as; -1 = not folded yet) and
  * was_appended uint8 [U, n] to HOST arrays (synchronises the stream). */
@@ -197,8 +240,9 @@ kvm_status_t kvm_debug_assignments(kvm_state_t* state, int64_t n, int32_t* slot_
 
 /* Returns the state to "empty" (position 0, no rows, no folds, block/growth/rope_dims unbound)
  * without freeing or clearing device memory, so that one allocation serves many sequences.
- * Host bookkeeping only; pending work on the stream is not waited for (the next call is
- * ordered behind it on the same stream). */
+ * Host bookkeeping only: nothing is enqueued and pending work is not waited for (the next call is
+ * ordered behind it on its own stream; with KVM_FLAG_RECORD_ASSIGN that next kvm_prefill also
+ * clears the recorded assignments, on its stream). */
 kvm_status_t kvm_state_reset(kvm_state_t* state);
 
 /* Per-kernel device timing for benchmarks.  kvm_profile_enable(state, 1) makes every later

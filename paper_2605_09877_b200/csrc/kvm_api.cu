@@ -150,21 +150,38 @@ struct DeviceGuard {
   ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
 };
 
-kvm_status_t bind_first_call(kvm_state* ks, int32_t block, const kvm_growth_t& growth, int32_t r, cudaStream_t stream) {
-  State& s = ks->s;
-  if (block < 8 || block > s.Cmax || (block % 8) != 0 || s.S >= block) return KVM_ERR_INVALID_ARG;
-  if (r < 0 || r > s.d || (r & 1)) return KVM_ERR_INVALID_ARG;
-  if (!growth_valid(growth)) return KVM_ERR_INVALID_ARG;
-  s.C = block; s.r = r; s.growth = growth; s.ringLen = (int64_t)s.w * block;
-  if (r > 0) {
-    std::vector<double> f(r / 2);
-    for (int i = 0; i < r / 2; ++i) f[i] = pow((double)s.rope_base, -2.0 * (double)i / (double)r);
-    if (cudaMemcpyAsync(s.inv_freq, f.data(), sizeof(double) * f.size(), cudaMemcpyHostToDevice, stream) != cudaSuccess)
-      return KVM_ERR_CUDA;
-    if (cudaStreamSynchronize(stream) != cudaSuccess) return KVM_ERR_CUDA;
+// Everything a prefill of n further tokens can fail on, checked on the host without touching the
+// state: block / growth / rope_dims (against the state's when it is bound), the positions the POWER
+// budget is defined for, and the row capacity - the row count after the call follows from the budget
+// rule alone.  (n_tokens against max_call_tokens is the caller's check: the host-buffer entry point
+// cuts a long call into segments.)
+kvm_status_t validate_prefill(const State& s, int32_t block, const kvm_growth_t& growth, int32_t r, int64_t n) {
+  if (n < 1) return KVM_ERR_INVALID_ARG;
+  if (!s.bound) {
+    if (block < 8 || block > s.Cmax || (block % 8) != 0 || s.S >= block) return KVM_ERR_INVALID_ARG;
+    if (r < 0 || r > s.d || (r & 1)) return KVM_ERR_INVALID_ARG;
+    if (!growth_valid(growth)) return KVM_ERR_INVALID_ARG;
+  } else if (block != s.C || r != s.r || !growth_equal(growth, s.growth)) {
+    return KVM_ERR_STATE_MISMATCH;
   }
-  s.bound = true;
+  const int C = block;
+  const int64_t pos0 = s.bound ? s.pos : 0, pos1 = pos0 + n;
+  if (growth.kind == KVM_GROWTH_POWER && pos1 >= kPowerMaxPos) return KVM_ERR_UNSUPPORTED;
+  int64_t m_sim = s.bound ? s.m : 0;
+  for (int64_t c = pos0 / C; c <= (pos1 - 1) / C; ++c) {
+    const int64_t e = (c + 1) * C;
+    if (e <= pos1 && c >= s.w - 1) m_sim += (m_sim == 0) ? C : n_append_of(growth, e, m_sim, C);
+  }
+  if (m_sim > s.Mcap) return KVM_ERR_CAPACITY;
   return KVM_OK;
+}
+
+// Binds block / growth / rope_dims (host bookkeeping only; called once the call can no longer fail).
+void bind_state(State& s, int32_t block, const kvm_growth_t& growth, int32_t r) {
+  s.C = block; s.r = r; s.growth = growth; s.ringLen = (int64_t)s.w * block;
+  const int k = r / 2;
+  s.inv_freq = s.inv_freq_all + (int64_t)k * (k - 1) / 2;
+  s.bound = true;
 }
 
 kvm_status_t ensure_host_staging(kvm_state* ks) {
@@ -194,6 +211,23 @@ kvm_status_t ensure_host_staging(kvm_state* ks) {
 
 bool launch_ok() { return cudaGetLastError() == cudaSuccess; }
 
+}  // namespace
+
+namespace {
+// Window tokens [wb, wb + len) <-> host arrays [U, len, ...]: the ring holds token t in slot t mod ringLen,
+// so the range is one or two runs of consecutive slots.
+template <typename F>
+bool for_ring_runs(const State& s, int64_t wb, int64_t len, F&& f) {
+  int64_t done = 0;
+  while (done < len) {
+    const int64_t slot = (wb + done) % s.ringLen;
+    int64_t run = s.ringLen - slot;
+    if (run > len - done) run = len - done;
+    if (!f(done, slot, run)) return false;
+    done += run;
+  }
+  return true;
+}
 }  // namespace
 
 #define KVM_API __attribute__((visibility("default")))
@@ -288,7 +322,7 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   kvm_status_t rc = KVM_OK;
 #define A(ptr, count) if (rc == KVM_OK) rc = dev_alloc(ks, &(ptr), (count))
   A(s.ln_w, (size_t)s.Hkv * d); A(s.ln_b, (size_t)s.Hkv * d); A(s.tau_s, (size_t)s.Hq); A(s.tau_b, (size_t)s.Hq);
-  A(s.inv_freq, (size_t)d / 2);
+  A(s.inv_freq_all, (size_t)(d / 2) * (d / 2 + 1) / 2);
   A(s.sumK, U * M * d); A(s.sumV, U * M * d); A(s.rho, U * M); A(s.wsum, U * M); A(s.cnt, U * M);
   A(s.kmu, U * M); A(s.krstd, U * M);
   for (int i = 0; i < 2; ++i) { A(s.KhatBuf[i], U * M * d); A(s.VhatBuf[i], U * M * d); }
@@ -298,14 +332,15 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   A(s.ropeCS, (size_t)s.Tcall * (d / 2));
   s.CbarRows = (s.Cmax + 127) / 128 * 128;
   {
-    // memory-key slots: as many blocks per batched launch as fit in 2 GiB (at least 1, at most 64,
-    // never more than a call can hold)
+    // memory-key slots: as many blocks per batched launch as fit in 2 GiB (at most 64, never more than
+    // a call can hold) and at least two, one per half: a prefill computes the keys of one batch of
+    // blocks while the folds consume the batch before it, so the two must never share a slot
     const size_t per_slot = U * Cm * d * 8 + U * (size_t)s.CbarRows * d * 4 + U * Cm * 20 + U * Cm * Cm * 4;
     size_t slots = ((size_t)2 << 30) / per_slot;
     const size_t call_blocks = (size_t)(s.Tcall / s.Cmax) + 2;
     if (slots > call_blocks) slots = call_blocks;
     if (slots > 64) slots = 64;
-    if (slots < 1) slots = 1;
+    if (slots < 2 || (cfg->flags & KVM_FLAG_MIN_KEY_SLOTS)) slots = 2;
     s.kbSlots = (int)slots;
   }
   {
@@ -334,6 +369,11 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
     ok = ok && cudaMemcpy(s.ln_b, lb.data(), sizeof(float) * lb.size(), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(s.tau_s, ts.data(), sizeof(float) * ts.size(), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaMemcpy(s.tau_b, tb.data(), sizeof(float) * tb.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+    // RoPE frequencies base^(-2i/r) for every even r <= d, so that binding rope_dims later needs no copy
+    std::vector<double> fr;
+    for (int k = 1; k <= d / 2; ++k)
+      for (int i = 0; i < k; ++i) fr.push_back(pow((double)s.rope_base, -2.0 * (double)i / (double)(2 * k)));
+    ok = ok && cudaMemcpy(s.inv_freq_all, fr.data(), sizeof(double) * fr.size(), cudaMemcpyHostToDevice) == cudaSuccess;
     ok = ok && cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) rc = KVM_ERR_CUDA;
   }
@@ -381,10 +421,7 @@ KVM_API kvm_status_t kvm_state_reset(kvm_state_t* ks) {
   if (!ks) return KVM_ERR_INVALID_ARG;
   State& s = ks->s;
   s.bound = false; s.pos = 0; s.m = 0; s.nfolds = 0; s.prevValid = false;
-  if (s.slotTok) {  // debug recording only: forget the previous sequence's assignments
-    DeviceGuard guard(s.device);
-    if (cudaMemset(s.slotTok, 0xff, (size_t)s.U * s.Tassign * sizeof(int32_t)) != cudaSuccess) return KVM_ERR_CUDA;
-  }
+  if (s.slotTok) s.assignDirty = true;   // debug recording only: the next prefill forgets the old assignments, on its stream
   return KVM_OK;
 }
 
@@ -460,26 +497,18 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
   if (((uintptr_t)q & 3) || ((uintptr_t)k & 3) || ((uintptr_t)v & 3) || ((uintptr_t)out & 3)) return KVM_ERR_INVALID_ARG;
   ia.sg[0] = (int64_t)s.Hkv * n; ia.sg[1] = n; ia.sg[2] = 1;
 
-  if (!s.bound) {
-    kvm_status_t rc = bind_first_call(ks, block, growth, rope_dims, stream);
+  {
+    const kvm_status_t rc = validate_prefill(s, block, growth, rope_dims, n);
     if (rc != KVM_OK) return rc;
-  } else if (block != s.C || rope_dims != s.r || !growth_equal(growth, s.growth)) {
-    return KVM_ERR_STATE_MISMATCH;
   }
+  if (!s.bound) bind_state(s, block, growth, rope_dims);
   const int C = s.C;
   const int64_t L = (int64_t)s.w * C;
   const int64_t pos0 = s.pos, pos1 = pos0 + n;
-  if (s.growth.kind == KVM_GROWTH_POWER && pos1 >= kPowerMaxPos) return KVM_ERR_UNSUPPORTED;
   const int64_t c0 = pos0 / C, c_last = (pos1 - 1) / C;
-
-  // capacity: the row count after this call follows from the budget rule alone
-  {
-    int64_t m_sim = s.m;
-    for (int64_t c = c0; c <= c_last; ++c) {
-      const int64_t e = (c + 1) * C;
-      if (e <= pos1 && c >= s.w - 1) m_sim += (m_sim == 0) ? C : n_append_of(s.growth, e, m_sim, C);
-    }
-    if (m_sim > s.Mcap) return KVM_ERR_CAPACITY;
+  if (s.assignDirty) {
+    s.assignDirty = false;
+    if (cudaMemsetAsync(s.slotTok, 0xff, (size_t)s.U * s.Tassign * sizeof(int32_t), stream) != cudaSuccess) return KVM_ERR_CUDA;
   }
 
   ia.q = (const __nv_bfloat16*)q; ia.k = (const __nv_bfloat16*)k; ia.v = (const __nv_bfloat16*)v; ia.gate = gate;
@@ -530,8 +559,8 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
     }
   }
   const int n_call_folds = (int)fold_na.size();
-  const int halves = s.kbSlots >= 2 ? 2 : 1;
-  const int per_batch = s.kbSlots >= 2 ? s.kbSlots / 2 : 1;
+  const int halves = 2;
+  const int per_batch = s.kbSlots / 2;   // (kbSlots >= 2)
   cudaStream_t kstream = overlap ? s.kbStream : stream;
   if (overlap && n_call_folds > 0) ev_ok = ev_ok && cudaStreamWaitEvent(kstream, s.evJoin, 0) == cudaSuccess;
   bool batch_done_rec[2] = {false, false};
@@ -587,6 +616,7 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
       // only the last kernel of the fold writes the readout copy: the routing filter and the
       // decisions run while the caller's stream still copies the previous fold's rows
       fa.before_apply = overlap ? s.evPre[c & 1] : nullptr;
+      fa.early_start = true;
       {
         const int nl = launch_fold(&s, fa, fstream);
         if (nl < 0) ev_ok = false; else s.launches += nl;
@@ -641,6 +671,7 @@ KVM_API kvm_status_t kvm_decode_step(const void* q, const void* k, const void* v
     fa.ok = s.ringK + slot * d; fa.ov = s.ringV + slot * d; fa.og = s.ringG + slot;
     fa.unit_stride = ringCap * d; fa.gate_stride = ringCap;
     fa.b = b; fa.m = s.m; fa.first = (s.m == 0); fa.n_append = n_a; fa.slot = 0; fa.before_apply = nullptr;
+    fa.early_start = false;   // the memory-key kernel runs right before the filter on this stream
     s.launches += launch_prev_copy(&s, stream);
     s.launches += launch_kbar(&s, fa.ok, fa.unit_stride, 1, 0, n_a > 0 && n_a < C && s.m > 0, stream);
     s.launches += launch_fold(&s, fa, stream);
@@ -658,10 +689,14 @@ KVM_API kvm_status_t kvm_prefill_host(const void* q_host, const void* k_host, co
   State& s = ks->s;
   if (n_tokens < 1) return KVM_ERR_INVALID_ARG;
   if (n_tokens > s.Tcall) return KVM_ERR_CAPACITY;
+  // the whole call is validated before the first copy is enqueued: a call that fails leaves the
+  // state and the caller's buffers untouched
+  kvm_status_t rc = validate_prefill(s, block, growth, rope_dims, n_tokens);
+  if (rc != KVM_OK) return rc;
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   DeviceGuard guard(s.device);
   if (!guard.ok) return KVM_ERR_CUDA;
-  kvm_status_t rc = ensure_host_staging(ks);
+  rc = ensure_host_staging(ks);
   if (rc != KVM_OK) return rc;
   // The call is cut into up to eight segments of whole blocks; segment i+1 is copied in, and segment
   // i-1 copied out, while segment i is computed (three streams, the copies as strided 2-D copies into /
@@ -672,10 +707,18 @@ KVM_API kvm_status_t kvm_prefill_host(const void* q_host, const void* k_host, co
   if (nseg > 8) nseg = 8;
   if (nseg < 1) nseg = 1;
   const int64_t seg_len = ((n + nseg - 1) / nseg + block - 1) / block * block;
+  // a failure after the first copy was enqueued (a CUDA error; the arguments were checked above): the
+  // caller gets its buffers back only once nothing reads or writes them any more
+  auto fail = [&](kvm_status_t code) {
+    cudaGetLastError();
+    cudaStreamSynchronize(s.hinStream); cudaStreamSynchronize(s.houtStream); cudaStreamSynchronize(stream);
+    cudaGetLastError();
+    return code;
+  };
   bool ok = cudaEventRecord(s.evHostStart, stream) == cudaSuccess;
   ok = ok && cudaStreamWaitEvent(s.hinStream, s.evHostStart, 0) == cudaSuccess;
   ok = ok && cudaStreamWaitEvent(s.houtStream, s.evHostStart, 0) == cudaSuccess;
-  if (!ok) { cudaGetLastError(); return KVM_ERR_CUDA; }
+  if (!ok) return fail(KVM_ERR_CUDA);
   kvm_strides_t st;
   st.q[0] = (int64_t)s.Hq * n * d; st.q[1] = n * d; st.q[2] = d; st.q[3] = 1;
   st.k[0] = (int64_t)s.Hkv * n * d; st.k[1] = n * d; st.k[2] = d; st.k[3] = 1;
@@ -700,20 +743,20 @@ KVM_API kvm_status_t kvm_prefill_host(const void* q_host, const void* k_host, co
     }
     ok = ok && cudaEventRecord(s.evIn[iseg], s.hinStream) == cudaSuccess;
     ok = ok && cudaStreamWaitEvent(stream, s.evIn[iseg], 0) == cudaSuccess;
-    if (!ok) { cudaGetLastError(); return KVM_ERR_CUDA; }
+    if (!ok) return fail(KVM_ERR_CUDA);
     rc = kvm_prefill((__nv_bfloat16*)s.hQ + off, (__nv_bfloat16*)s.hK + off, (__nv_bfloat16*)s.hV + off, ks, block, growth,
                      rope_dims, len, gseg, (__nv_bfloat16*)s.hOut + off, &st, cuda_stream);
-    if (rc != KVM_OK) return rc;
+    if (rc != KVM_OK) return fail(rc);
     ok = cudaEventRecord(s.evComp[iseg], stream) == cudaSuccess;
     ok = ok && cudaStreamWaitEvent(s.houtStream, s.evComp[iseg], 0) == cudaSuccess;
     ok = ok && cudaMemcpy2DAsync((__nv_bfloat16*)out_host + off, pitch, (__nv_bfloat16*)s.hOut + off, pitch, width,
                                  (size_t)s.B * s.Hq, cudaMemcpyDeviceToHost, s.houtStream) == cudaSuccess;
-    if (!ok) { cudaGetLastError(); return KVM_ERR_CUDA; }
+    if (!ok) return fail(KVM_ERR_CUDA);
   }
   ok = cudaEventRecord(s.evHostOut, s.houtStream) == cudaSuccess;
   ok = ok && cudaStreamWaitEvent(stream, s.evHostOut, 0) == cudaSuccess;
   ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
-  if (!ok) { cudaGetLastError(); return KVM_ERR_CUDA; }
+  if (!ok) return fail(KVM_ERR_CUDA);
   return KVM_OK;
 }
 
@@ -762,6 +805,104 @@ KVM_API kvm_status_t kvm_state_export(kvm_state_t* ks, double* sum_k, float* sum
   }
   ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
   if (!ok) { cudaGetLastError(); return KVM_ERR_CUDA; }
+  return KVM_OK;
+}
+
+KVM_API kvm_status_t kvm_state_snapshot_info(const kvm_state_t* ks, kvm_snapshot_info_t* out) {
+  if (!ks || !out) return KVM_ERR_INVALID_ARG;
+  const State& s = ks->s;
+  memset(out, 0, sizeof(*out));
+  if (!s.bound) return KVM_OK;
+  out->block = s.C; out->rope_dims = s.r; out->growth = s.growth;
+  out->n_slots = s.m; out->position = s.pos; out->n_folds = s.nfolds;
+  int64_t wb = (s.pos / s.C + 1) * s.C - (int64_t)s.w * s.C;   // first token that the next block's window still holds
+  if (wb < 0) wb = 0;
+  out->window_begin = wb; out->window_len = s.pos - wb;
+  return KVM_OK;
+}
+
+KVM_API kvm_status_t kvm_state_export_window(kvm_state_t* ks, void* win_k, void* win_v, float* win_gate, void* cuda_stream) {
+  if (!ks) return KVM_ERR_INVALID_ARG;
+  State& s = ks->s;
+  if (!s.bound) return KVM_ERR_STATE_MISMATCH;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  DeviceGuard guard(s.device);
+  if (!guard.ok) return KVM_ERR_CUDA;
+  kvm_snapshot_info_t info;
+  kvm_state_snapshot_info(ks, &info);
+  const size_t d = (size_t)s.d, U = (size_t)s.U, ringCap = (size_t)s.w * s.Cmax, len = (size_t)info.window_len;
+  bool ok = for_ring_runs(s, info.window_begin, info.window_len, [&](int64_t at, int64_t slot, int64_t run) {
+    bool k = true;
+    if (win_k) k = k && cudaMemcpy2DAsync((__half*)win_k + at * d, len * d * 2, s.ringK + slot * d, ringCap * d * 2, run * d * 2, U, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (win_v) k = k && cudaMemcpy2DAsync((__half*)win_v + at * d, len * d * 2, s.ringV + slot * d, ringCap * d * 2, run * d * 2, U, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (win_gate) k = k && cudaMemcpy2DAsync(win_gate + at, len * 4, s.ringG + slot, ringCap * 4, run * 4, U, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    return k;
+  });
+  ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); return KVM_ERR_CUDA; }
+  return KVM_OK;
+}
+
+KVM_API kvm_status_t kvm_state_import(kvm_state_t* ks, const kvm_snapshot_info_t* info, const double* sum_k, const float* sum_v,
+                              const float* radius, const double* weight, const int32_t* count, const void* win_k,
+                              const void* win_v, const float* win_gate, void* cuda_stream) {
+  if (!ks || !info) return KVM_ERR_INVALID_ARG;
+  State& s = ks->s;
+  // ---- validation on the host; nothing is touched before it has passed ----
+  const int C = info->block, r = info->rope_dims;
+  if (C < 8 || (C % 8) != 0 || s.S >= C) return KVM_ERR_INVALID_ARG;
+  if (C > s.Cmax) return KVM_ERR_CAPACITY;
+  if (r < 0 || r > s.d || (r & 1) || !growth_valid(info->growth)) return KVM_ERR_INVALID_ARG;
+  if (info->position < 0 || info->n_slots < 0 || info->n_folds < 0) return KVM_ERR_INVALID_ARG;
+  if (info->growth.kind == KVM_GROWTH_POWER && info->position >= kPowerMaxPos) return KVM_ERR_UNSUPPORTED;
+  {
+    // rows and folds follow from the position by the budget rule; the window from the block structure
+    int64_t m = 0, nf = 0;
+    for (int64_t c = s.w - 1; (c + 1) * C <= info->position; ++c) {
+      m += (m == 0) ? C : n_append_of(info->growth, (c + 1) * C, m, C);
+      ++nf;
+    }
+    int64_t wb = (info->position / C + 1) * C - (int64_t)s.w * C;
+    if (wb < 0) wb = 0;
+    if (m != info->n_slots || nf != info->n_folds || wb != info->window_begin || info->window_len != info->position - wb)
+      return KVM_ERR_INVALID_ARG;
+    if (m > s.Mcap) return KVM_ERR_CAPACITY;
+  }
+  if (info->n_slots > 0 && (!sum_k || !sum_v || !radius || !weight || !count)) return KVM_ERR_INVALID_ARG;
+  if (info->window_len > 0 && (!win_k || !win_v)) return KVM_ERR_INVALID_ARG;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  DeviceGuard guard(s.device);
+  if (!guard.ok) return KVM_ERR_CUDA;
+
+  kvm_state_reset(ks);
+  bind_state(s, C, info->growth, r);
+  s.pos = info->position; s.m = info->n_slots; s.nfolds = info->n_folds;
+  const size_t m = (size_t)s.m, M = (size_t)s.Mcap, d = (size_t)s.d, U = (size_t)s.U;
+  bool ok = true;
+  if (m > 0) {
+#define CP(dst, src, elt, width) \
+  ok = ok && cudaMemcpy2DAsync(dst, M * (width) * (elt), src, m * (width) * (elt), m * (width) * (elt), U, cudaMemcpyHostToDevice, stream) == cudaSuccess
+    CP(s.sumK, sum_k, sizeof(double), d);
+    CP(s.sumV, sum_v, sizeof(float), d);
+    CP(s.rho, radius, sizeof(float), (size_t)1);
+    CP(s.wsum, weight, sizeof(double), (size_t)1);
+    CP(s.cnt, count, sizeof(int32_t), (size_t)1);
+#undef CP
+    if (ok) s.launches += launch_refresh_rows(&s, s.m, stream);
+  }
+  const size_t ringCap = (size_t)s.w * s.Cmax, len = (size_t)info->window_len;
+  std::vector<float> ones;
+  if (len > 0 && !win_gate) ones.assign(U * len, 1.0f);
+  const float* wg = win_gate ? win_gate : ones.data();
+  ok = ok && for_ring_runs(s, info->window_begin, info->window_len, [&](int64_t at, int64_t slot, int64_t run) {
+    bool k = cudaMemcpy2DAsync(s.ringK + slot * d, ringCap * d * 2, (const __half*)win_k + at * d, len * d * 2, run * d * 2, U, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    k = k && cudaMemcpy2DAsync(s.ringV + slot * d, ringCap * d * 2, (const __half*)win_v + at * d, len * d * 2, run * d * 2, U, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    k = k && cudaMemcpy2DAsync(s.ringG + slot, ringCap * 4, wg + at, len * 4, run * 4, U, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    return k;
+  });
+  ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+  ok = ok && launch_ok();
+  if (!ok) { cudaGetLastError(); kvm_state_reset(ks); return KVM_ERR_CUDA; }
   return KVM_OK;
 }
 

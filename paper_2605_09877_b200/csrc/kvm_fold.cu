@@ -1114,7 +1114,135 @@ __global__ void __launch_bounds__(256, 2) fold_apply_rows4_kernel(FoldApplyParam
   }
 }
 
-int launch_route_filter_tc(State* st, int64_t m, int nsplit, int slot, cudaStream_t s);
+// Row statistics and readout rows (both copies) of rows [0, m) recomputed from the stored sums, for a
+// state whose sums were loaded from a snapshot.  The arithmetic and the reduction order are those of
+// the apply kernel that this state's folds run (ROWS4: four rows per warp, eight lanes per row; else
+// one row per warp), so the refreshed values equal bit for bit what the folds had left.
+struct RefreshParams {
+  const double* sumK; const float* sumV; const float* rho; const double* wsum;
+  const float *ln_w, *ln_b;
+  double *kmu, *krstd;
+  __half *Khat0, *Vhat0, *Khat1, *Vhat1;
+  int64_t Mcap, m;
+  int Hkv, radius_on;
+  double ln_eps, norm_eps;
+};
+
+template <int D, bool ROWS4>
+__global__ void __launch_bounds__(256) refresh_rows_kernel(RefreshParams p) {
+  const int u = blockIdx.y, hk = u % p.Hkv;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (ROWS4) {
+    constexpr int NI = D / 32, NC = 4 * NI;
+    constexpr double inv_d = 1.0 / D;
+    const int sub = lane & 7;
+    const int64_t q = ((int64_t)blockIdx.x * 8 + warp) * kApplyRowsPerWarp + (lane >> 3);
+    const bool act = q < p.m;
+    const int64_t row = (int64_t)u * p.Mcap + (act ? q : 0);
+    double kx[NC];
+    float vx[NC];
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+      const int x = 32 * i + 4 * sub;
+      const double2 k01 = *reinterpret_cast<const double2*>(p.sumK + row * D + x), k23 = *reinterpret_cast<const double2*>(p.sumK + row * D + x + 2);
+      kx[4 * i] = k01.x; kx[4 * i + 1] = k01.y; kx[4 * i + 2] = k23.x; kx[4 * i + 3] = k23.y;
+      const float4 v4 = *reinterpret_cast<const float4*>(p.sumV + row * D + x);
+      vx[4 * i] = v4.x; vx[4 * i + 1] = v4.y; vx[4 * i + 2] = v4.z; vx[4 * i + 3] = v4.w;
+    }
+    const double wacc = p.wsum[row], rad = (double)p.rho[row];
+    double sum = 0.0;
+#pragma unroll
+    for (int c = 0; c < NC; ++c) sum += kx[c];
+    const double mu = group8_sum_d(sum) * inv_d;
+    double dev = 0.0, vv = 0.0;
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+      dev += (kx[c] - mu) * (kx[c] - mu);
+      vv += (double)vx[c] * (double)vx[c];
+    }
+    const double rs = 1.0 / sqrt(group8_sum_d(dev) * inv_d + p.ln_eps);
+    const double vnorm = sqrt(group8_sum_d(vv));
+    const double den = vnorm > p.norm_eps ? vnorm : p.norm_eps;
+    const double vscale = p.radius_on ? rad / den : 1.0 / wacc;
+    if (!act) return;
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+      const int x = 32 * i + 4 * sub;
+      const float4 w4 = *reinterpret_cast<const float4*>(p.ln_w + hk * D + x), b4 = *reinterpret_cast<const float4*>(p.ln_b + hk * D + x);
+      const float wv[4] = {w4.x, w4.y, w4.z, w4.w}, bv[4] = {b4.x, b4.y, b4.z, b4.w};
+      alignas(8) __half kh[4], vh[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const double hat = (double)wv[e] * ((kx[4 * i + e] - mu) * rs) + (double)bv[e];
+        kh[e] = __float2half_rn((float)hat);
+        vh[e] = __float2half_rn((float)((double)vx[4 * i + e] * vscale));
+      }
+      *reinterpret_cast<uint2*>(p.Khat0 + row * D + x) = *reinterpret_cast<const uint2*>(kh);
+      *reinterpret_cast<uint2*>(p.Vhat0 + row * D + x) = *reinterpret_cast<const uint2*>(vh);
+      *reinterpret_cast<uint2*>(p.Khat1 + row * D + x) = *reinterpret_cast<const uint2*>(kh);
+      *reinterpret_cast<uint2*>(p.Vhat1 + row * D + x) = *reinterpret_cast<const uint2*>(vh);
+    }
+    if (sub == 0) { p.kmu[row] = mu; p.krstd[row] = rs; }
+  } else {
+    constexpr int CH = D / 32;
+    const int64_t q = (int64_t)blockIdx.x * 8 + warp;
+    if (q >= p.m) return;
+    const int64_t row = (int64_t)u * p.Mcap + q;
+    double kx[CH];
+    float vx[CH];
+#pragma unroll
+    for (int i = 0; i < CH; ++i) {
+      kx[i] = p.sumK[row * D + lane + 32 * i];
+      vx[i] = p.sumV[row * D + lane + 32 * i];
+    }
+    const double wacc = p.wsum[row], rad = (double)p.rho[row];
+    double mu, rs;
+    row_stats<CH>(kx, D, p.ln_eps, mu, rs);
+    double v2 = 0.0;
+#pragma unroll
+    for (int i = 0; i < CH; ++i) v2 += (double)vx[i] * (double)vx[i];
+    const double vnorm = sqrt(warp_sum_d(v2));
+    const double den = vnorm > p.norm_eps ? vnorm : p.norm_eps;
+    const double vscale = p.radius_on ? rad / den : 1.0 / wacc;
+#pragma unroll
+    for (int i = 0; i < CH; ++i) {
+      const int x = lane + 32 * i;
+      const double hat = (double)p.ln_w[hk * D + x] * ((kx[i] - mu) * rs) + (double)p.ln_b[hk * D + x];
+      const __half kh = __float2half_rn((float)hat);
+      const __half vh = __float2half_rn((float)((double)vx[i] * vscale));
+      p.Khat0[row * D + x] = kh; p.Vhat0[row * D + x] = vh;
+      p.Khat1[row * D + x] = kh; p.Vhat1[row * D + x] = vh;
+    }
+    if (lane == 0) { p.kmu[row] = mu; p.krstd[row] = rs; }
+  }
+}
+
+// which apply kernel the folds of this state run (fixed per state and block): four rows per warp when
+// the launch is bound by throughput (measured: better from 8192 rows on: U = 32, C = 256; worse at
+// 4096 and 2048 rows, where the longer chain per row shows)
+static bool apply_uses_rows4(const State* st) { return (int64_t)st->C * st->U >= 8192; }
+
+int launch_refresh_rows(State* st, int64_t m, cudaStream_t s) {
+  if (m <= 0) return 0;
+  RefreshParams p;
+  p.sumK = st->sumK; p.sumV = st->sumV; p.rho = st->rho; p.wsum = st->wsum; p.ln_w = st->ln_w; p.ln_b = st->ln_b;
+  p.kmu = st->kmu; p.krstd = st->krstd;
+  p.Khat0 = st->KhatBuf[0]; p.Vhat0 = st->VhatBuf[0]; p.Khat1 = st->KhatBuf[1]; p.Vhat1 = st->VhatBuf[1];
+  p.Mcap = st->Mcap; p.m = m; p.Hkv = st->Hkv; p.radius_on = (st->flags & KVM_FLAG_NO_RADIUS) ? 0 : 1;
+  p.ln_eps = (double)st->ln_eps; p.norm_eps = (double)st->norm_eps;
+  if (apply_uses_rows4(st)) {
+    dim3 grid((unsigned)((m + kApplyRowsPerCta - 1) / kApplyRowsPerCta), st->U);
+    if (st->d == 128) refresh_rows_kernel<128, true><<<grid, 256, 0, s>>>(p);
+    else refresh_rows_kernel<64, true><<<grid, 256, 0, s>>>(p);
+  } else {
+    dim3 grid((unsigned)((m + 7) / 8), st->U);
+    if (st->d == 128) refresh_rows_kernel<128, false><<<grid, 256, 0, s>>>(p);
+    else refresh_rows_kernel<64, false><<<grid, 256, 0, s>>>(p);
+  }
+  return 1;
+}
+
+int launch_route_filter_tc(State* st, int64_t m, int nsplit, int slot, bool early_start, cudaStream_t s);
 int launch_gram_tc(State* st, int slot0, int nblk, cudaStream_t s);
 
 int launch_kbar(State* st, const __half* ok, int64_t unit_stride, int nblk, int slot0, bool want_gram, cudaStream_t s) {
@@ -1188,7 +1316,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
       ++launches;
     } else {
       KernelTimer kt(st, 3, s);
-      launches += launch_route_filter_tc(st, a.m, nsplit, a.slot, s);
+      launches += launch_route_filter_tc(st, a.m, nsplit, a.slot, a.early_start, s);
     }
     FoldDecideParams p;
     p.kbar64 = kbar64; p.kbarNorm = kbarNorm; p.kbarHatStat = kbarHatStat;
@@ -1246,9 +1374,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
   q.ln_eps = (double)st->ln_eps; q.norm_eps = (double)st->norm_eps;
   if (a.before_apply && cudaStreamWaitEvent(s, a.before_apply, 0) != cudaSuccess) return -1000000;
   KernelTimer kt(st, 5, s);
-  // four rows per warp when the launch is bound by throughput (measured: better from 8192 rows on:
-  // U = 32, C = 256; worse at 4096 and 2048 rows, where the longer chain per row shows)
-  if ((int64_t)C * st->U >= 8192) {
+  if (apply_uses_rows4(st)) {
     dim3 grid((C + kApplyRowsPerCta - 1) / kApplyRowsPerCta, st->U);
     if (D == 128) fold_apply_rows4_kernel<128><<<grid, 256, 0, s>>>(q);
     else fold_apply_rows4_kernel<64><<<grid, 256, 0, s>>>(q);

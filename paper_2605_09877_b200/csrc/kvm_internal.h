@@ -39,7 +39,9 @@ struct State {
   // ---- parameters (device) ----
   float *ln_w, *ln_b;     // [Hkv, d]
   float *tau_s, *tau_b;   // [Hq]
-  double* inv_freq;       // [r/2]
+  double* inv_freq;       // [r/2]: the bound rope_dims' slice of inv_freq_all
+  double* inv_freq_all;   // base^(-2i/r), i < r/2, for every even r <= d, r's slice at offset (r/2)(r/2 - 1)/2
+  bool assignDirty;       // recorded assignments of an earlier sequence are still in slotTok (cleared by the next prefill)
   // ---- state rows (device) ----
   double* sumK;           // [U, Mcap, d]  running key sums (fp64: routing decisions are taken on them)
   float* sumV;            // [U, Mcap, d]
@@ -158,6 +160,9 @@ struct FoldArgs {
   bool first;       // first state-creation step
   int slot;         // memory-key slot that holds this block's keys (launch_kbar)
   cudaEvent_t before_apply;   // if set, the stream waits for it before the kernel that writes the readout copy
+  bool early_start;           // the routing filter may start under the kernel before it on the stream (programmatic
+                              // dependent launch) and fetch the block's memory keys before it waits: only where that
+                              // kernel is not the one that writes those keys
 };
 int launch_fold(State* st, const FoldArgs& a, cudaStream_t s);
 // Memory keys of nblk consecutive blocks (C rows each, starting at ok within every unit) into slots
@@ -167,6 +172,8 @@ int launch_kbar(State* st, const __half* ok, int64_t unit_stride, int nblk, int 
 // one (no-op when nothing is owed).  Must run after every reader of the other copy has finished and
 // before the next fold writes it.
 int launch_prev_copy(State* st, cudaStream_t s);
+// Recomputes the row statistics and both readout copies of rows [0, m) from the stored sums (snapshot import).
+int launch_refresh_rows(State* st, int64_t m, cudaStream_t s);
 
 struct DecodeArgs {
   const __nv_bfloat16 *q, *k, *v;

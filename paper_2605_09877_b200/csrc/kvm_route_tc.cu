@@ -262,7 +262,7 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
   }
 }
 
-int launch_route_filter_tc(State* st, int64_t m, int nsplit, int slot, cudaStream_t s) {
+int launch_route_filter_tc(State* st, int64_t m, int nsplit, int slot, bool early_start, cudaStream_t s) {
   RouteTcParams p;
   p.candV = st->candV; p.candI = st->candI; p.status = st->status; p.m = m;
   p.C = st->C; p.Cmax = st->Cmax; p.nsplit = nsplit; p.S = st->S;
@@ -272,13 +272,14 @@ int launch_route_filter_tc(State* st, int64_t m, int nsplit, int slot, cudaStrea
   dim3 grid(nsplit, st->U);
   const int ks = (st->nfolds & 1) ? 6 : 1;   // the fold reads the readout copy of the current version
   // programmatic dependent launch behind the apply kernel of the previous fold: the CTAs set up and
-  // fetch the block's memory keys while it finishes
+  // fetch the block's memory keys while it finishes (not where the kernel before this one on the
+  // stream is the one that writes those keys: a decode step's fold)
   cudaLaunchConfig_t lc = {};
   lc.gridDim = grid; lc.blockDim = dim3(352); lc.stream = s;
   cudaLaunchAttribute at[1];
   at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   at[0].val.programmaticStreamSerializationAllowed = 1;
-  lc.attrs = at; lc.numAttrs = st->prof_hook == nullptr ? 1 : 0;
+  lc.attrs = at; lc.numAttrs = (early_start && st->prof_hook == nullptr) ? 1 : 0;
   if (st->d == 128) { lc.dynamicSmemBytes = RouteTcCfg<128>::SMEM_BYTES; cudaLaunchKernelEx(&lc, route_filter_tc_kernel<128>, tm[5], tm[ks], tm[8], p); }
   else { lc.dynamicSmemBytes = RouteTcCfg<64>::SMEM_BYTES; cudaLaunchKernelEx(&lc, route_filter_tc_kernel<64>, tm[5], tm[ks], tm[8], p); }
   return 1;

@@ -20,12 +20,13 @@ KVM_OK = 0
 STATUS = {0: "KVM_OK", 1: "KVM_ERR_INVALID_ARG", 2: "KVM_ERR_UNSUPPORTED", 3: "KVM_ERR_OOM",
           4: "KVM_ERR_CUDA", 5: "KVM_ERR_STATE_MISMATCH", 6: "KVM_ERR_CAPACITY", 7: "KVM_ERR_TIMEOUT"}
 GROWTH_FIXED, GROWTH_SQRT, GROWTH_UNBOUNDED, GROWTH_POWER, GROWTH_SATURATING = 0, 1, 2, 3, 4
-FLAG_NO_RADIUS, FLAG_RECORD_ASSIGN, FLAG_SIMT_ATTENTION, FLAG_SIMT_ROUTING = 1, 2, 4, 8
+FLAG_NO_RADIUS, FLAG_RECORD_ASSIGN, FLAG_SIMT_ATTENTION, FLAG_SIMT_ROUTING, FLAG_MIN_KEY_SLOTS = 1, 2, 4, 8, 16
 
 EXPORTS = ["kvm_plan_capacity", "kvm_state_create", "kvm_prefill", "kvm_decode_step", "kvm_prefill_host",
            "kvm_decode_step_host", "kvm_state_free", "kvm_state_info", "kvm_state_check", "kvm_state_export",
            "kvm_debug_assignments", "kvm_launch_count", "kvm_status_string", "kvm_state_reset",
-           "kvm_profile_enable", "kvm_profile_read", "kvm_debug_counters", "kvm_attend_rows_noalloc", "kvm_merge_gate", "kvm_head_layernorm"]
+           "kvm_profile_enable", "kvm_profile_read", "kvm_debug_counters", "kvm_attend_rows_noalloc", "kvm_merge_gate", "kvm_head_layernorm",
+           "kvm_state_snapshot_info", "kvm_state_export_window", "kvm_state_import"]
 
 
 class KVMError(RuntimeError):
@@ -41,6 +42,11 @@ class Growth(C.Structure):
 
 class Strides(C.Structure):
     _fields_ = [("q", C.c_int64 * 4), ("k", C.c_int64 * 4), ("v", C.c_int64 * 4), ("out", C.c_int64 * 4)]
+
+
+class SnapshotInfo(C.Structure):
+    _fields_ = [("block", C.c_int32), ("rope_dims", C.c_int32), ("growth", Growth), ("n_slots", C.c_int64),
+                ("position", C.c_int64), ("n_folds", C.c_int64), ("window_begin", C.c_int64), ("window_len", C.c_int64)]
 
 
 class Config(C.Structure):
@@ -99,6 +105,12 @@ def _load():
     L.kvm_merge_gate.argtypes = [vp, vp, C.c_int32, C.c_int64, C.c_int32, C.c_int32, vp, vp]
     L.kvm_head_layernorm.restype = C.c_int
     L.kvm_head_layernorm.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, C.c_int64, C.c_int32, C.c_float, vp]
+    L.kvm_state_snapshot_info.restype = C.c_int
+    L.kvm_state_snapshot_info.argtypes = [vp, C.POINTER(SnapshotInfo)]
+    L.kvm_state_export_window.restype = C.c_int
+    L.kvm_state_export_window.argtypes = [vp, vp, vp, vp, vp]
+    L.kvm_state_import.restype = C.c_int
+    L.kvm_state_import.argtypes = [vp, C.POINTER(SnapshotInfo)] + [vp] * 9
     L.kvm_status_string.restype = C.c_char_p
     L.kvm_status_string.argtypes = [C.c_int]
     return L
@@ -335,6 +347,34 @@ class KVMState:
         if rc != KVM_OK:
             raise KVMError(rc, "kvm_state_export")
         return dict(sum_k=sk, sum_v=sv, radius=rho, weight=w, count=cnt, k_read=kr, v_read=vr)
+
+    def snapshot(self, stream=None):
+        """kvm_state_snapshot_info + kvm_state_export + kvm_state_export_window: everything kvm_state_import needs."""
+        info = SnapshotInfo()
+        rc = lib.kvm_state_snapshot_info(self._h, C.byref(info))
+        if rc != KVM_OK:
+            raise KVMError(rc, "kvm_state_snapshot_info")
+        snap = self.export(readout=False, stream=stream)
+        n, d = info.window_len, self.cfg.head_dim
+        wk = torch.zeros((self.U, n, d), dtype=torch.float16); wv = torch.zeros((self.U, n, d), dtype=torch.float16)
+        wg = np.zeros((self.U, n), np.float32)
+        if info.block > 0:
+            rc = lib.kvm_state_export_window(self._h, C.c_void_p(wk.data_ptr()), C.c_void_p(wv.data_ptr()),
+                                             C.c_void_p(wg.ctypes.data), _stream_ptr(stream))
+            if rc != KVM_OK:
+                raise KVMError(rc, "kvm_state_export_window")
+        snap.update(info=info, win_k=wk, win_v=wv, win_gate=wg)
+        return snap
+
+    def restore(self, snap, stream=None):
+        """kvm_state_import of a snapshot() (possibly taken from another state of the same shape)."""
+        p = lambda a: C.c_void_p(a.ctypes.data) if a is not None and a.size else None
+        t = lambda a: C.c_void_p(a.data_ptr()) if a is not None and a.numel() else None
+        rc = lib.kvm_state_import(self._h, C.byref(snap["info"]), p(snap["sum_k"]), p(snap["sum_v"]), p(snap["radius"]),
+                                  p(snap["weight"]), p(snap["count"]), t(snap["win_k"]), t(snap["win_v"]),
+                                  p(snap.get("win_gate")), _stream_ptr(stream))
+        if rc != KVM_OK:
+            raise KVMError(rc, "kvm_state_import")
 
     def assignments(self, n=None, stream=None):
         n = self.info()["position"] if n is None else n

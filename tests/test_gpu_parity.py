@@ -275,5 +275,28 @@ def test_api_errors_leave_state_usable():
     st.prefill(q[:, :, 64:], k[:, :, 64:], v[:, :, 64:], 64, g, 0)
     assert st.info()["position"] == 128 and st.check() == 0
     st.free()
+    # a failed first call binds nothing: the state takes another block / growth afterwards
+    wl2 = wl.scaled(T=256)
+    st, g = pu.gpu_layer(wl2, params)                      # rows for fixed 64 (rounded up to 128), calls of 256 tokens
+    t2 = synth.make_inputs(wl2)
+    q, k, v = (t2[n].cuda() for n in "qkv")
+    with pytest.raises(kvm.KVMError) as e:
+        st.prefill(q, k, v, 8, kvm.growth("unbounded"), 0)   # 256 tokens in blocks of 8, never merging: 248 rows
+    assert e.value.code == 6
+    assert st.info() == dict(n_slots=0, position=0, n_folds=0)
+    # the host-buffer entry point validates the whole call before it copies anything
+    hq, hk, hv = (t2[n].contiguous() for n in "qkv")
+    ho = torch.zeros_like(hq)
+    for bad_block in (0, -64, 60):
+        with pytest.raises(kvm.KVMError) as e:
+            st.prefill_host(hq, hk, hv, bad_block, g, 0, ho)
+        assert e.value.code == 1
+    with pytest.raises(kvm.KVMError) as e:
+        st.prefill_host(hq, hk, hv, 8, kvm.growth("unbounded"), 0, ho)   # a later segment would exceed the capacity
+    assert e.value.code == 6
+    assert st.info() == dict(n_slots=0, position=0, n_folds=0) and float(ho.abs().sum()) == 0.0
+    y = st.prefill(q, k, v, 64, g, 0)                        # and the state is still unbound and usable
+    assert st.info()["position"] == 256 and st.check() == 0 and torch.isfinite(y.float()).all()
+    st.free()
     with pytest.raises(kvm.KVMError):
         kvm.KVMState(kvm.LayerConfig(1, 1, 1, 96, 64, 64, 64))   # head_dim 96 unsupported

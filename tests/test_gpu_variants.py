@@ -1,0 +1,79 @@
+"""GPU parity for the kernel variants that only large launches select, each at the smallest shape that
+still selects it, against the fp64 oracle on sampled (batch, head) units (units are independent end to
+end, so the oracle run on a unit alone is that unit's exact reference):
+
+  * the fold-decision kernel built for grids of more than 148 CTAs (two CTAs per SM, 64 registers);
+  * the decode kernel's direct-output branch (one row split per head) at head_dim 128, with and without
+    grouped queries;
+  * config 5's structure at a batch wide enough to select the kernels that the full batch selects;
+  * the minimum of two memory-key slots (one block of look-ahead), which very large batches run with.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2605_09877_b200 import synth
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def _sampled(wl, units, params=None, gate=False, decode_from=None, flags=0):
+    params = params or synth.make_layer_params(wl)
+    tensors = synth.make_inputs(wl)
+    if gate:
+        tensors["gate"] = synth.make_gate(wl)
+    y_gpu, st = pu.run_gpu(wl, tensors, params, decode_from=decode_from, flags=flags)
+    y_ref, o = pu.run_oracle(wl, tensors, params, units=units)
+    stats = pu.compare(wl, y_gpu, st, y_ref, o, units=units)
+    stats["counters"] = st.debug_counters()
+    st.free()
+    return stats
+
+
+def test_fold_decide_two_ctas_per_sm_variant_head_dim_128():
+    """160 units x block 256 at head_dim 128: one decision CTA per unit, 160 > 148 CTAs, so the 64-register
+    build runs (the one every many-unit shape uses); gates and affine LayerNorm included."""
+    wl = synth.Workload("t", 1, 160, 160, 128, 4 * 256 + 70, 256, "sqrt", sqrt_coeff=14, r=32, seed=31, kind="mixture")
+    params = synth.make_layer_params(wl, trivial=False)
+    print(_sampled(wl, [(0, 0), (0, 37), (0, 101), (0, 148), (0, 159)], params=params, gate=True))
+
+
+def test_decode_direct_output_branch_head_dim_128():
+    """640 query heads need no row split (nsplit == 1): the decode kernel writes its output directly.
+    40 steps from position 1004 cross the block boundary at 1024, so one of them folds."""
+    wl = synth.Workload("t", 20, 32, 32, 128, 1004 + 40, 256, "sqrt", r=0, seed=32)
+    print(_sampled(wl, [(0, 0), (7, 13), (19, 31)], decode_from=1004))
+
+
+def test_decode_grouped_queries_direct_and_split():
+    """Four query heads per kv head: 640 query heads (direct output) and 8 query heads (row splits)."""
+    wl = synth.Workload("t", 5, 128, 32, 128, 500 + 30, 128, "sqrt", r=32, seed=33)
+    params = synth.make_layer_params(wl, trivial=False)
+    print(_sampled(wl, [(0, 0), (2, 17), (4, 31)], params=params, decode_from=500))
+    wl = synth.Workload("t", 1, 8, 2, 128, 700 + 30, 128, "sqrt", r=32, seed=34)
+    print(_sampled(wl, [(0, 0), (0, 1)], decode_from=700))
+
+
+def test_config5_structure_at_a_batch_that_selects_the_full_batch_kernels():
+    """B8 x H32 = 256 units, block 256, sqrt growth, N(0,1) tokens, two prefill segments and a few decode
+    steps: every kernel selection that depends on the number of units (decision kernel build, rows-per-warp
+    apply, attention tail split, routing filter splits, decode without row splits) is the full batch's."""
+    wl = synth.CONFIGS["cfg5"].scaled(B=8, T=3072 + 20)
+    units = [(0, 0), (3, 9), (7, 31)]
+    params = synth.make_layer_params(wl)
+    tensors = synth.make_inputs(wl)
+    y_gpu, st = pu.run_gpu(wl, tensors, params, cuts=[0, 2048, 3072], decode_from=3072)
+    y_ref, o = pu.run_oracle(wl, tensors, params, units=units)
+    print(pu.compare(wl, y_gpu, st, y_ref, o, units=units))
+    st.free()
+
+
+def test_two_memory_key_slots_one_block_of_look_ahead():
+    """With only two memory-key slots every fold's keys are computed while the fold before it runs, and a
+    slot is rewritten as soon as its fold is done: routing must still see its own block's keys."""
+    from paper_2605_09877_b200 import kvm
+    wl = synth.CONFIGS["cfg3"].scaled(Hq=3, Hkv=3, T=256 * 12 + 31)
+    print(_sampled(wl, None, flags=kvm.FLAG_MIN_KEY_SLOTS))
+    wl = synth.CONFIGS["cfg2"].scaled(B=2, Hq=2, Hkv=2, T=128 * 14)
+    print(_sampled(wl, None, flags=kvm.FLAG_MIN_KEY_SLOTS, gate=True))

@@ -625,3 +625,24 @@ def test_append_score_counts_the_sink_row():
     assert np.array_equal(np.nonzero(app[0, C:2 * C])[0], [j_half])
     # the copy of the sink cannot merge into the sink; it goes to another row
     assert slot[0, C + 0] >= 1 and app[0, C + 0] == 0
+
+
+def test_attend_rows_definition_closed_forms_and_library_routine():
+    """oracle/attend_rows.py (single-query attention over given rows): equal keys give the plain mean of the
+    values, a dominant key gives its value, and torch's scaled_dot_product_attention (a library routine,
+    fp64) gives the same numbers; `scale` multiplies the logits (a transposed or unscaled product fails)."""
+    import torch
+    from oracle.attend_rows import attend_rows
+    rng = np.random.default_rng(5)
+    H, n, d = 3, 17, 8
+    q = rng.standard_normal((H, d)); k = rng.standard_normal((H, n, d)); v = rng.standard_normal((H, n, d))
+    same = np.repeat(k[:, :1], n, axis=1)
+    assert np.allclose(attend_rows(q, same, v, 0.7), v.mean(axis=1), atol=1e-13)
+    big = k.copy(); big[:, 5] = 50.0 * q
+    assert np.allclose(attend_rows(q, big, v, 1.0), v[:, 5], atol=1e-9)
+    ref = torch.nn.functional.scaled_dot_product_attention(torch.from_numpy(q)[:, None], torch.from_numpy(k), torch.from_numpy(v),
+                                                           scale=0.37)[:, 0].numpy()
+    assert np.allclose(attend_rows(q, k, v, 0.37), ref, atol=1e-13)
+    # two rows, by hand: logits (scale * q.k) = (ln 3, 0) -> weights (3/4, 1/4)
+    q1 = np.array([[1.0, 0.0]]); k1 = np.array([[[np.log(3.0) / 2.0, 9.0], [0.0, -4.0]]]); v1 = np.array([[[4.0, 0.0], [0.0, 8.0]]])
+    assert np.allclose(attend_rows(q1, k1, v1, 2.0), [[3.0, 2.0]], atol=1e-13)

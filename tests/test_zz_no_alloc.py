@@ -56,6 +56,37 @@ def test_noalloc_attention_matches_decode_step_twice():
     st.free()
 
 
+@pytest.mark.parametrize("d,heads,rows", [(128, 6, 1500), (64, 3, 8193), (64, 700, 300), (128, 40, 5000)])
+def test_noalloc_attention_matches_the_fp64_definition_and_allocates_nothing(d, heads, rows):
+    """The entry point against softmax(scale q K^T) V written out in fp64 on the same fp16 rows (so only the
+    kernel's fp32 arithmetic and the bf16 rounding of the output separate the two), at both head sizes, with
+    32 row splits of which the last ones are empty (8193 rows at head_dim 64), with one split per head
+    (700 heads) and with two calls in a row; free device memory as the driver reports it is the same before
+    and after the calls."""
+    from oracle.attend_rows import attend_rows
+    from paper_2605_09877_b200 import kvm
+    g = torch.Generator().manual_seed(1000 + d + heads)
+    q = torch.randn((heads, d), generator=g).to(torch.float16)
+    keys = torch.randn((heads, rows, d), generator=g).to(torch.float16)
+    vals = torch.randn((heads, rows, d), generator=g).to(torch.float16)
+    keys[:, rows // 3] *= 3.0                      # one peaked row per head
+    scale = 1.3 / math.sqrt(d)
+    ref = attend_rows(q.numpy(), keys.numpy(), vals.numpy(), scale)
+    qd, kd, vd = q.cuda(), keys.cuda(), vals.cuda()
+    out = torch.empty((heads, d), dtype=torch.bfloat16, device="cuda")
+    kvm.attend_rows_noalloc(qd, kd, vd, scale, out=out)      # (the first call on the device looks the array up)
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    for _ in range(2):
+        out.zero_()
+        kvm.attend_rows_noalloc(qd, kd, vd, scale, out=out)
+        torch.cuda.synchronize()
+        err = np.abs(out.double().cpu().numpy() - ref)
+        # half a bf16 ulp of the output plus fp32 accumulation
+        assert np.all(err <= 2.0 ** -8 * np.abs(ref) + 1e-4), float(err.max())
+    assert torch.cuda.mem_get_info()[0] == free0
+
+
 def test_noalloc_rejects_what_the_fixed_scratch_cannot_hold():
     from paper_2605_09877_b200 import kvm
     d = 128
