@@ -1,14 +1,19 @@
 #!/usr/bin/env python
 """Benchmark of the KVM layer hot path on B200 (one JSON line on stdout).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5] [--impl reference]
 
 A "step" is one pass of the whole hot path over one batch of synthetic input:
-  prefill workloads (cfg1..cfg4, paper-speed): kvm_prefill of the full sequence on an empty
-      state (ingest/RoPE, per-chunk attention over [state ; window], every fold);
+  cfg5 (default; the largest configuration: B64 H32 d128, 65536 tokens, block 256, 16 sqrt(N) budget):
+      kvm_prefill of the whole sequence on an empty state, fed as 16 segments of 4096 tokens that are all
+      resident in HBM (ingest, per-block attention over [state ; window], every fold); metric = prefill
+      tokens/s.  The same JSON line carries a "decode" record: the 256 single-token decode steps that
+      follow on that very state (us per step, HBM GB/s).
+  prefill workloads (cfg1..cfg4, paper-speed): kvm_prefill of the full sequence in one call;
       metric = prefill tokens/s (batch * sequence tokens per second).
   decode workload (cfg5-decode): one kvm_decode_step for the whole batch on a state of
-      m = 4096 rows plus a 256..511-token window; metric = decode us per step.
+      m = 4096 rows plus a 256..511-token window built by a short fixed-budget prefill (a quick way to
+      time the decode kernel alone); metric = decode us per step.
 `value` is measured with inputs resident in HBM; `e2e` goes through the *_host entry points
 with pinned host buffers (H2D and D2H inside the timed region).  With N > 1 every rank runs
 the same per-GPU workload on its own units (weak scaling, no data-path collective).
@@ -37,7 +42,9 @@ from paper_2605_09877_b200 import synth  # noqa: E402
 
 def workload(name):
     c = synth.CONFIGS
-    if name in c and name != "cfg5":
+    if name == "cfg5":
+        return c[name], "prefill+decode"
+    if name in c:
         return c[name], "prefill"
     if name == "paper-speed":   # the paper's speed-benchmark shape: B8 H32 d128 C256, KVM-sqrt, T=32768
         return synth.Workload("paper-speed", 8, 32, 32, 128, 32768, 256, "sqrt", r=0, seed=7), "prefill"
@@ -86,6 +93,13 @@ NCU_TRAFFIC = {
     ("cfg5", "decode"): 4.574e9,    # profiles/ncu_full_attn_route_decide_decode_small_cases.md (4.570 GB read + 4 MB written)
     ("cfg2", "attention"): 13.72e6,  # same file: 13.72 MB read, 0 written per launch (algorithmic: 14.6 MB)
 }
+
+
+def decode_bytes(wl, m, pos):
+    """Algorithmic bytes of the decode step at position `pos`: fp16 readout rows K^, V^ of the m state rows plus
+    the window tokens [b, pos] (keys and values), for every (batch, kv head)."""
+    b = max(0, (pos // wl.C + 1) * wl.C - wl.w * wl.C)
+    return wl.B * wl.Hkv * (m + pos - b + 1) * wl.d * 2 * 2
 
 
 def peaks():
@@ -149,7 +163,7 @@ def oracle_sample(wl, mode, budget_s=20.0):
     from oracle import kvm_oracle as ko
     from tests.parity_util import oracle_config
     cores = ko.threads()
-    if mode == "prefill":
+    if mode.startswith("prefill"):
         # sample: `n_units` (batch, head) units over a prefix of T_s tokens sized for ~budget_s
         n_units = min(cores, wl.B * wl.Hkv)
         T_s = wl.T
@@ -230,7 +244,7 @@ def aggregate(mode, local_ms_per_step, units_per_step, world, device="cuda"):
     """Whole-job value from per-rank step times: every rank processes `units_per_step` units per step
     (weak scaling), the job's step time is the slowest rank's.  Returns (value, ms_per_step)."""
     ms = max_over_ranks(local_ms_per_step, world, device)
-    if mode == "prefill":
+    if mode.startswith("prefill"):
         return world * units_per_step / (ms * 1e-3), ms     # tokens/s over all replicas
     return ms * 1e3, ms                                     # decode: us per step (each replica steps its batch)
 
@@ -248,10 +262,11 @@ def run_reference(args):
         last = res
     v = sum(vals) / len(vals)
     unit = last["unit"]
-    ms = (wl.B * wl.T / v * 1e3) if mode == "prefill" else v / 1e3
-    line = dict(metric="kvm_prefill_tokens_per_s" if mode == "prefill" else "kvm_decode_us_per_step", value=v, unit=unit,
+    pre = mode.startswith("prefill")
+    ms = (wl.B * wl.T / v * 1e3) if pre else v / 1e3
+    line = dict(metric="kvm_prefill_tokens_per_s" if pre else "kvm_decode_us_per_step", value=v, unit=unit,
                 n_gpus=args.gpus, steps=args.steps, warmup=args.warmup, ms_per_step=ms,
-                higher_is_better=(mode == "prefill"), scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                higher_is_better=pre, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
                 config=dict(workload=wl.name, mode=mode), impl="reference",
                 cpu_baseline=dict(value=v, unit=unit, cores=last["cores"], kind="oracle", sample=last["sample"]),
                 e2e=dict(value=v, unit=unit, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
@@ -420,18 +435,67 @@ def run_headln(args):
     return 0
 
 
+def decode_record(st, wl, dev, stream, pk, world):
+    """The decode half of the metric on the state the timed prefill left (position T, m rows, one block in the
+    window): wl.decode_steps single-token steps with fresh inputs, every step between two CUDA events; the last
+    one completes a block and folds.  The first half is timed as the user sees it (whole steps), the second
+    half also with the library's per-kernel brackets (attention incl. its ingest, without the fold)."""
+    n = wl.decode_steps
+    info0 = st.info()
+    dq = [synth.make_decode_inputs(wl.scaled(seed=wl.seed), i, device=dev) for i in range(n)]
+    out = torch.empty_like(dq[0]["q"])
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+    half = n // 2
+    torch.cuda.synchronize()
+    for i in range(n):
+        if i == half:
+            torch.cuda.synchronize()
+            st.profile_enable(True)
+            st.profile_read()
+        d = dq[i]
+        ev[i][0].record(stream)
+        st.decode_step(d["q"], d["k"], d["v"], out=out)
+        ev[i][1].record(stream)
+    torch.cuda.synchronize()
+    prof = st.profile_read()
+    st.profile_enable(False)
+    info1 = st.info()
+    us = [1e3 * a.elapsed_time(b) for a, b in ev]
+    plain = us[3:half]                                   # whole steps, user's view (the first three warm up)
+    nbytes = [decode_bytes(wl, info0["n_slots"], info0["position"] + i) for i in range(n)]
+    us_plain = sum(plain) / len(plain)
+    gbs_plain = sum(nbytes[3:half]) / 1e9 / (sum(plain) * 1e-6)
+    kern_ms, kern_n = prof["decode"]
+    nfold = info1["n_folds"] - info0["n_folds"]
+    kern_bytes = sum(nbytes[half:])
+    gbs_kern = kern_bytes / 1e9 / (kern_ms * 1e-3) if kern_ms > 0 else None
+    us_all = max_over_ranks(us_plain, world)
+    return dict(metric="kvm_decode_us_per_step", value=us_all, unit="us/step", us_per_sequence_token=us_all / wl.B,
+                steps=n, state_rows=info0["n_slots"], position0=info0["position"], folds_in_these_steps=nfold,
+                fold_step_us=us[-1] if nfold else None, median_us=sorted(plain)[len(plain) // 2],
+                min_us=min(plain), max_us=max(plain),
+                roofline=dict(bound="hbm", kernel="decode", achieved=gbs_plain, peak=pk["hbm"], unit="GB/s",
+                              frac=gbs_plain / pk["hbm"], frac_of_nominal_8TBs=gbs_plain / 8000.0,
+                              traffic=NCU_TRAFFIC.get(("cfg5", "decode")),
+                              peak_source=f"{pk['src']} copy bandwidth", bytes_per_step=sum(nbytes[3:half]) / len(plain),
+                              what="whole decode steps (ingest + attention kernels), CUDA events around each step",
+                              kernels_only_gbs=gbs_kern, kernels_only_us=1e3 * kern_ms / max(kern_n, 1)))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="cfg2")
+    ap.add_argument("--workload", default="cfg5")
     ap.add_argument("--impl", default="kvm")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--simt", action="store_true", help="time the scalar-core cross-check kernels")
     ap.add_argument("--tokens", type=int, default=0,
-                    help="prefill workloads: shorten the sequence to this many tokens (small cases for ncu captures)")
+                    help="prefill workloads: shorten the sequence to this many tokens (small cases for ncu captures; "
+                         "cfg5: a multiple of 4096)")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch size (small cases for ncu captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -445,6 +509,8 @@ def main():
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     wl, mode = workload(args.workload)
+    if args.batch:
+        wl = wl.scaled(B=args.batch, name=f"{wl.name}-B{args.batch}")
     if args.tokens and mode == "prefill":
         wl = wl.scaled(T=args.tokens, name=f"{wl.name}-T{args.tokens}")
     pk = peaks()
@@ -454,7 +520,27 @@ def main():
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
 
-    if mode == "prefill":
+    segs = None
+    if mode == "prefill+decode":
+        # the largest configuration: the sequence is fed in segments (q, k, v of all 65536 tokens are 103 GB,
+        # all resident before the timed region starts); the outputs of a segment overwrite the previous one's
+        T, seg = (args.tokens or wl.T), 4096
+        assert T % seg == 0
+        cap = kvm.kvm_plan_capacity(wl.C, wl.w, g, T + wl.decode_steps)
+        st = kvm.KVMState(kvm.LayerConfig(wl.B, wl.Hq, wl.Hkv, wl.d, wl.C, max(cap, wl.C), seg, n_bswa_chunks=wl.w,
+                                          sink_len=wl.S, device=local, flags=flags))
+        segs = [synth.make_segment(wl.scaled(seed=wl.seed + 1000 * rank), i, seg, device=dev) for i in range(T // seg)]
+        out = torch.empty_like(segs[0]["q"])
+        if T != wl.T:
+            wl = wl.scaled(T=T, name=f"{wl.name}-T{T}")
+
+        def step():
+            st.reset()
+            for t in segs:
+                st.prefill(t["q"], t["k"], t["v"], wl.C, g, wl.r, out=out)
+
+        units_per_step = wl.B * T   # tokens
+    elif mode == "prefill":
         T = wl.T
         cap = kvm.kvm_plan_capacity(wl.C, wl.w, g, T)
         st = kvm.KVMState(kvm.LayerConfig(wl.B, wl.Hq, wl.Hkv, wl.d, wl.C, max(cap, wl.C), T, n_bswa_chunks=wl.w,
@@ -509,17 +595,21 @@ def main():
     times = [a.elapsed_time(b) for a, b in ev]
     value, ms_step = aggregate(mode, sum(times) / K, units_per_step, world)
 
+    decode_rec = None
+    if mode == "prefill+decode":
+        decode_rec = decode_record(st, wl, dev, stream, pk, world)
+
     # per-phase device time (separate pass with event brackets) -> roofline of the dominant phase
     st.profile_enable(True)
     st.profile_read()
-    for i in range(min(K, 3)):
+    nprof = 1 if mode == "prefill+decode" else min(K, 3)
+    for i in range(nprof):
         flush.fill_(i)
         step()
     prof = st.profile_read()
     st.profile_enable(False)
-    nprof = min(K, 3)
 
-    if mode == "prefill":
+    if mode.startswith("prefill"):
         att_f, rt_f = prefill_flops(wl, wl.T)
         per_kernel = {k_: v_[0] / nprof for k_, v_ in prof.items()}
         # the dominant kernel by device time; the two tensor-core kernels have an algorithmic flop count
@@ -557,7 +647,20 @@ def main():
     # end to end through the host-buffer entry points (pinned memory)
     e2e = None
     if not args.no_e2e:
-        if mode == "prefill":
+        if mode == "prefill+decode":
+            # host buffers of two segments (pinned), sent alternately: a step copies every segment's q, k, v in
+            # and its outputs out (the host buffers of all 16 segments would be 137 GB of pinned memory)
+            hseg = [{n: segs[i][n].cpu().pin_memory() for n in "qkv"} for i in range(2)]
+            hout = torch.empty_like(hseg[0]["q"]).pin_memory()
+            nseg_ = len(segs)
+            def estep():
+                st.reset()
+                for i in range(nseg_):
+                    h = hseg[i & 1]
+                    st.prefill_host(h["q"], h["k"], h["v"], wl.C, g, wl.r, hout)
+            bi = nseg_ * sum(hseg[0][n].numel() for n in "qkv") * 2
+            bo = nseg_ * hout.numel() * 2
+        elif mode == "prefill":
             hq, hk, hv = (cpu[n].contiguous().pin_memory() for n in "qkv")
             hout = torch.empty_like(hq).pin_memory()
             def estep():
@@ -572,8 +675,8 @@ def main():
                 st.decode_step_host(hd["q"], hd["k"], hd["v"], hout)
             bi = sum(hd[n].numel() for n in "qkv") * 2
             bo = hout.numel() * 2
-        ne = min(K, 5)
-        for _ in range(2):
+        ne = 2 if mode == "prefill+decode" else min(K, 5)
+        for _ in range(1 if mode == "prefill+decode" else 2):
             estep()
         barrier(world)
         t0 = time.perf_counter()
@@ -581,7 +684,7 @@ def main():
             estep()
         torch.cuda.synchronize()
         dt = max_over_ranks((time.perf_counter() - t0) / ne, world)
-        ev_ = world * units_per_step / dt if mode == "prefill" else dt * 1e6
+        ev_ = world * units_per_step / dt if mode.startswith("prefill") else dt * 1e6
         e2e = dict(value=ev_, unit=unit, h2d_bytes_per_step=bi, d2h_bytes_per_step=bo)
 
     cpu_base = None
@@ -596,6 +699,10 @@ def main():
                                 growth=wl.growth, rope_dims=wl.r, l2="256 MiB flush between timed steps",
                                 kernels="simt" if args.simt else "default"),
                     clocks=clocks, e2e=e2e, gpu_launches=launches, roofline=roof, cpu_baseline=cpu_base)
+        if segs is not None:
+            line["config"]["segments"] = f"{len(segs)} kvm_prefill calls of 4096 tokens per step, all inputs resident in HBM"
+        if decode_rec is not None:
+            line["decode"] = decode_rec
         print(json.dumps(line))
     st.free()
     if world > 1:
