@@ -168,7 +168,7 @@ def oracle_sample(wl, mode, budget_s=20.0):
         n_units = min(cores, wl.B * wl.Hkv)
         T_s = wl.T
         att, rt = prefill_flops(wl.scaled(B=1, Hq=n_units * (wl.Hq // wl.Hkv), Hkv=n_units), T_s)
-        rate = 0.6e9 * cores   # rough fp64 flop/s of the plain loops; only used to size the sample
+        rate = 2.5e9 * cores   # rough fp64 flop/s of the plain loops; only used to size the sample
         while (att + rt) / rate > budget_s and T_s > 4 * wl.C:
             T_s //= 2
             att, rt = prefill_flops(wl.scaled(B=1, Hq=n_units * (wl.Hq // wl.Hkv), Hkv=n_units), T_s)
@@ -492,6 +492,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle leg")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--simt", action="store_true", help="time the scalar-core cross-check kernels")
+    ap.add_argument("--serial", action="store_true", help="force one readout copy and folds on the caller's stream")
     ap.add_argument("--tokens", type=int, default=0,
                     help="prefill workloads: shorten the sequence to this many tokens (small cases for ncu captures; "
                          "cfg5: a multiple of 4096)")
@@ -517,6 +518,8 @@ def main():
     W, K = max(args.warmup, 3), args.steps
     g = kvm.growth(wl.growth, wl.fixed_slots, wl.sqrt_coeff)
     flags = (kvm.FLAG_SIMT_ATTENTION | kvm.FLAG_SIMT_ROUTING) if args.simt else 0
+    if args.serial:
+        flags |= kvm.FLAG_SERIAL_FOLDS
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
 

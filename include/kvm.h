@@ -86,8 +86,10 @@ enum {
   KVM_FLAG_RECORD_ASSIGN = 1u << 1,  /* keep per-token slot ids / append flags for kvm_debug_assignments */
   KVM_FLAG_SIMT_ATTENTION = 1u << 2, /* use the scalar-core attention kernel (cross-check path) */
   KVM_FLAG_SIMT_ROUTING = 1u << 3,   /* use the scalar-core routing filter (cross-check path)   */
-  KVM_FLAG_MIN_KEY_SLOTS = 1u << 4   /* debug: keep only the minimum of two memory-key slots (the look-ahead
+  KVM_FLAG_MIN_KEY_SLOTS = 1u << 4,  /* debug: keep only the minimum of two memory-key slots (the look-ahead
                                         of one block that very large batches run with), whatever the size */
+  KVM_FLAG_SERIAL_FOLDS = 1u << 5    /* one readout copy and folds on the caller's stream between the attention
+                                        launches (what states of 256 or more units do by themselves) */
 };
 
 typedef struct {

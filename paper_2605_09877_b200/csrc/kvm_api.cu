@@ -325,7 +325,12 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   A(s.inv_freq_all, (size_t)(d / 2) * (d / 2 + 1) / 2);
   A(s.sumK, U * M * d); A(s.sumV, U * M * d); A(s.rho, U * M); A(s.wsum, U * M); A(s.cnt, U * M);
   A(s.kmu, U * M); A(s.krstd, U * M);
-  for (int i = 0; i < 2; ++i) { A(s.KhatBuf[i], U * M * d); A(s.VhatBuf[i], U * M * d); }
+  // with enough units every kernel of a fold fills the GPU by itself and nothing is gained by running the
+  // folds beside the attention: such a state keeps ONE readout copy (both names refer to it)
+  s.serial = s.U >= kSerialUnits || (cfg->flags & KVM_FLAG_SERIAL_FOLDS);
+  A(s.KhatBuf[0], U * M * d); A(s.VhatBuf[0], U * M * d);
+  if (s.serial) { s.KhatBuf[1] = s.KhatBuf[0]; s.VhatBuf[1] = s.VhatBuf[0]; }
+  else { A(s.KhatBuf[1], U * M * d); A(s.VhatBuf[1], U * M * d); }
   A(s.ringK, U * ringCap * d); A(s.ringV, U * ringCap * d); A(s.ringG, U * ringCap);
   A(s.stQ, (size_t)s.B * s.Hq * s.Tcall * d);
   A(s.stK, U * (size_t)s.stRows * d); A(s.stV, U * (size_t)s.stRows * d); A(s.stG, U * (size_t)s.stRows);
@@ -532,13 +537,15 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
   //   the caller's stream waits for the last fold before the call returns.
   // With the per-kernel timing hook on, everything stays on the caller's stream so that the
   // measured durations are those of kernels running alone.
-  const bool overlap = s.prof_hook == nullptr;
-  cudaStream_t fstream = overlap ? s.foldStream : stream;
+  // A state with so many units that every kernel fills the GPU by itself (State::serial) keeps one
+  // readout copy and runs its folds on the caller's stream between the attention launches; only the
+  // memory keys are still computed ahead on their own stream.
+  const bool ovk = s.prof_hook == nullptr;     // memory keys ahead of the folds on their own stream
+  const bool ovf = ovk && !s.serial;           // folds on their own stream beside the attention
+  cudaStream_t fstream = ovf ? s.foldStream : stream;
   bool ev_ok = true;
-  if (overlap) {
-    ev_ok = ev_ok && cudaEventRecord(s.evJoin, stream) == cudaSuccess;
-    ev_ok = ev_ok && cudaStreamWaitEvent(fstream, s.evJoin, 0) == cudaSuccess;
-  }
+  if (ovk) ev_ok = ev_ok && cudaEventRecord(s.evJoin, stream) == cudaSuccess;
+  if (ovf) ev_ok = ev_ok && cudaStreamWaitEvent(fstream, s.evJoin, 0) == cudaSuccess;
   int fold_pending = -1;               // evFold index the next attention must wait for
   // The folds of this call, planned ahead from the budget rule: fold i ends block cf0 + i, folds the
   // block that starts at bf0 + i*C and appends fold_na[i] rows.  Their memory keys (and new-row
@@ -561,8 +568,8 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
   const int n_call_folds = (int)fold_na.size();
   const int halves = 2;
   const int per_batch = s.kbSlots / 2;   // (kbSlots >= 2)
-  cudaStream_t kstream = overlap ? s.kbStream : stream;
-  if (overlap && n_call_folds > 0) ev_ok = ev_ok && cudaStreamWaitEvent(kstream, s.evJoin, 0) == cudaSuccess;
+  cudaStream_t kstream = ovk ? s.kbStream : stream;
+  if (ovk && n_call_folds > 0) ev_ok = ev_ok && cudaStreamWaitEvent(kstream, s.evJoin, 0) == cudaSuccess;
   bool batch_done_rec[2] = {false, false};
   auto launch_batch = [&](int k) {      // batch k = folds [k*per_batch, ...) into slot half k % halves
     const int f0 = k * per_batch;
@@ -575,10 +582,10 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
       // (m_sim restarts from the current rows: folds before f0 that are already launched moved s.m)
       if (i >= n_done_folds) { if (i >= f0 && fold_na[i] > 0 && fold_na[i] < C && m_sim > 0) want_gram = true; m_sim += fold_na[i]; }
     }
-    if (overlap && batch_done_rec[h]) ev_ok = ev_ok && cudaStreamWaitEvent(kstream, s.evBatchDone[h], 0) == cudaSuccess;
+    if (ovk && batch_done_rec[h]) ev_ok = ev_ok && cudaStreamWaitEvent(kstream, s.evBatchDone[h], 0) == cudaSuccess;
     const int64_t bf = (cf0 + f0 + 1) * C - L;   // first token of the first block of the batch
     s.launches += launch_kbar(&s, s.stK + (bf - ia.hist_start) * d, s.stRows * d, nf, h * per_batch, want_gram, kstream);
-    if (overlap) ev_ok = ev_ok && cudaEventRecord(s.evKb[h], kstream) == cudaSuccess;
+    if (ovk) ev_ok = ev_ok && cudaEventRecord(s.evKb[h], kstream) == cudaSuccess;
   };
   for (int64_t c = c0; c <= c_last; ++c) {
     const int64_t e = (c + 1) * C;
@@ -587,12 +594,12 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
     int64_t b = e - L; if (b < 0) b = 0;
     aa.q_row0 = qs - pos0; aa.nq = (int)(qe - qs); aa.t0 = qs; aa.m = s.m;
     aa.win_row0 = b - ia.hist_start; aa.b = b; aa.out = (__nv_bfloat16*)out; aa.out_t0 = qs - pos0;
-    if (overlap && fold_pending >= 0) {
+    if (ovf && fold_pending >= 0) {
       ev_ok = ev_ok && cudaStreamWaitEvent(stream, s.evFold[fold_pending], 0) == cudaSuccess;
       fold_pending = -1;
     }
     s.launches += launch_prev_copy(&s, stream);
-    if (overlap) ev_ok = ev_ok && cudaEventRecord(s.evPre[c & 1], stream) == cudaSuccess;
+    if (ovf) ev_ok = ev_ok && cudaEventRecord(s.evPre[c & 1], stream) == cudaSuccess;
     {
       KernelTimer pt(&s, 1, stream);
       if (s.flags & KVM_FLAG_SIMT_ATTENTION) s.launches += launch_attn_simt(&s, aa, stream);
@@ -601,8 +608,8 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
     if (qe == e && c >= s.w - 1) {
       const int fi = n_done_folds, bk = fi / per_batch;
       if (fi % per_batch == 0) {
-        if (!overlap || fi == 0) launch_batch(bk);        // (with one stream: just in time)
-        if (overlap) {
+        if (!ovk || fi == 0) launch_batch(bk);            // (with one stream: just in time)
+        if (ovk) {
           launch_batch(bk + 1);                            // one batch ahead
           ev_ok = ev_ok && cudaStreamWaitEvent(fstream, s.evKb[bk % halves], 0) == cudaSuccess;
         }
@@ -615,7 +622,7 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
       fa.slot = (bk % halves) * per_batch + fi % per_batch;
       // only the last kernel of the fold writes the readout copy: the routing filter and the
       // decisions run while the caller's stream still copies the previous fold's rows
-      fa.before_apply = overlap ? s.evPre[c & 1] : nullptr;
+      fa.before_apply = ovf ? s.evPre[c & 1] : nullptr;
       fa.early_start = true;
       {
         const int nl = launch_fold(&s, fa, fstream);
@@ -624,17 +631,17 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
       s.m += fa.n_append;
       s.nfolds += 1;
       n_done_folds += 1;
-      if (overlap && (n_done_folds % per_batch == 0 || n_done_folds == n_call_folds)) {
+      if (ovk && (n_done_folds % per_batch == 0 || n_done_folds == n_call_folds)) {
         ev_ok = ev_ok && cudaEventRecord(s.evBatchDone[bk % halves], fstream) == cudaSuccess;
         batch_done_rec[bk % halves] = true;
       }
-      if (overlap) {
+      if (ovf) {
         fold_pending = (int)(s.nfolds & 1);
         ev_ok = ev_ok && cudaEventRecord(s.evFold[fold_pending], fstream) == cudaSuccess;
       }
     }
   }
-  if (overlap && fold_pending >= 0) ev_ok = ev_ok && cudaStreamWaitEvent(stream, s.evFold[fold_pending], 0) == cudaSuccess;
+  if (ovf && fold_pending >= 0) ev_ok = ev_ok && cudaStreamWaitEvent(stream, s.evFold[fold_pending], 0) == cudaSuccess;
   s.pos = pos1;
   if (!ev_ok) { cudaGetLastError(); return KVM_ERR_CUDA; }
   return launch_ok() ? KVM_OK : KVM_ERR_CUDA;

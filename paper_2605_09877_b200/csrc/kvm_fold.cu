@@ -1270,6 +1270,7 @@ int launch_kbar(State* st, const __half* ok, int64_t unit_stride, int nblk, int 
 int launch_prev_copy(State* st, cudaStream_t s) {
   if (!st->prevValid) return 0;
   st->prevValid = false;
+  if (st->serial) return 0;   // one readout copy: nothing to bring over
   // the last fold (number nfolds) wrote copy nfolds & 1; the other copy lacks the rows it touched
   const int src = (int)(st->nfolds & 1), dst = src ^ 1;
   PrevFoldCopy pc;

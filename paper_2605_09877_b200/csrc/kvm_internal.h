@@ -15,6 +15,7 @@ constexpr int kMaxSplits = 32;      // routing filter / decode split count upper
 constexpr int kAttnSplitTiles = 37; // launches with at most this many (batch, head, query tile) CTAs - a quarter of the GPU - are split along the keys
 constexpr int kAttnMaxSplits = 8;
 constexpr int kRowAlign = 128;      // state capacity is rounded up to the attention key tile
+constexpr int kSerialUnits = 256;   // from this many (batch, kv head) units on, folds run on the caller's stream with one readout copy
 
 // State of one layer: host bookkeeping + device buffers.  U = batch * n_kv_heads "units";
 // unit u = b * Hkv + hk owns rows [u*Mcap, (u+1)*Mcap) of every per-row array.
@@ -53,6 +54,7 @@ struct State {
   // decode and the routing filter.  Two copies: the state after f folds is read from copy f & 1, so
   // fold f+1 can write copy (f+1) & 1 while the attention of the current block still reads copy f & 1.
   __half *KhatBuf[2], *VhatBuf[2];
+  bool serial;            // one readout copy (KhatBuf[1] == KhatBuf[0]), folds on the caller's stream
   // what the previous fold touched (host): its rows are copied into the other copy (launch_prev_copy)
   // before the next fold writes there; prevValid = such a copy is still owed
   bool prevValid, prevAllAppend;

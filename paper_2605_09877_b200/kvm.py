@@ -20,7 +20,7 @@ KVM_OK = 0
 STATUS = {0: "KVM_OK", 1: "KVM_ERR_INVALID_ARG", 2: "KVM_ERR_UNSUPPORTED", 3: "KVM_ERR_OOM",
           4: "KVM_ERR_CUDA", 5: "KVM_ERR_STATE_MISMATCH", 6: "KVM_ERR_CAPACITY", 7: "KVM_ERR_TIMEOUT"}
 GROWTH_FIXED, GROWTH_SQRT, GROWTH_UNBOUNDED, GROWTH_POWER, GROWTH_SATURATING = 0, 1, 2, 3, 4
-FLAG_NO_RADIUS, FLAG_RECORD_ASSIGN, FLAG_SIMT_ATTENTION, FLAG_SIMT_ROUTING, FLAG_MIN_KEY_SLOTS = 1, 2, 4, 8, 16
+FLAG_NO_RADIUS, FLAG_RECORD_ASSIGN, FLAG_SIMT_ATTENTION, FLAG_SIMT_ROUTING, FLAG_MIN_KEY_SLOTS, FLAG_SERIAL_FOLDS = 1, 2, 4, 8, 16, 32
 
 EXPORTS = ["kvm_plan_capacity", "kvm_state_create", "kvm_prefill", "kvm_decode_step", "kvm_prefill_host",
            "kvm_decode_step_host", "kvm_state_free", "kvm_state_info", "kvm_state_check", "kvm_state_export",

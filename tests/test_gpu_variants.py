@@ -77,3 +77,20 @@ def test_two_memory_key_slots_one_block_of_look_ahead():
     print(_sampled(wl, None, flags=kvm.FLAG_MIN_KEY_SLOTS))
     wl = synth.CONFIGS["cfg2"].scaled(B=2, Hq=2, Hkv=2, T=128 * 14)
     print(_sampled(wl, None, flags=kvm.FLAG_MIN_KEY_SLOTS, gate=True))
+
+
+def test_serial_folds_one_readout_copy():
+    """What states of 512 or more units do by themselves, forced on small shapes: folds on the caller's stream
+    between the attention launches, one readout copy written in place; segmented prefill, gates, decode with a
+    fold."""
+    from paper_2605_09877_b200 import kvm
+    wl = synth.CONFIGS["cfg3"].scaled(Hq=3, Hkv=3, T=256 * 9 + 31)
+    print(_sampled(wl, None, flags=kvm.FLAG_SERIAL_FOLDS))
+    wl = synth.Workload("t", 2, 4, 2, 128, 128 * 11 + 40, 128, "fixed", fixed_slots=400, r=32, seed=35)
+    params = synth.make_layer_params(wl, trivial=False)
+    tensors = synth.make_inputs(wl)
+    tensors["gate"] = synth.make_gate(wl)
+    y_gpu, st = pu.run_gpu(wl, tensors, params, cuts=[0, 300, 1000, 128 * 11], decode_from=128 * 11, flags=kvm.FLAG_SERIAL_FOLDS)
+    y_ref, o = pu.run_oracle(wl, tensors, params)
+    print(pu.compare(wl, y_gpu, st, y_ref, o))
+    st.free()
