@@ -3,10 +3,11 @@
 // the state's readout keys, reduced on the fly to the rows whose similarity lies within the
 // rounding bound of the row maximum (Section 3.2 "Append" score and "Merge" arg max; the exact
 // decision is taken later in fp64 on these candidates only).  The split is streamed twice:
-// pass 1 keeps the running maximum per token (one FMNMX per element), pass 2 repeats the
-// products and collects the few elements above (maximum - bound).  The tensor work doubles but
-// the epilogue, which is the bottleneck of a 128 x 128 x d tile, stays at ~2 instructions per
-// element instead of a sorted insertion.
+// pass 1 keeps the running maximum per token (three-input maxima: half an instruction per
+// element), pass 2 repeats the products, takes the maximum of every 32-column chunk the same way
+// and looks element by element only at the chunks in which some token of the warp has a value above
+// (maximum - bound).  The tensor work doubles but the epilogue, which is the bottleneck of a
+// 128 x 128 x d tile, stays near one instruction per element instead of a sorted insertion.
 //
 //   warp 0      TMA producer: the Kbar tiles once, then 128-row tiles of K_hat in a 3-stage ring
 //   warps 1, 10 MMA issuers, one thread per M tile: per key tile one 128x128x(d) product into a
@@ -171,7 +172,7 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
         const int buf = j & 1;
         const bool pass2 = j >= ntiles;
         const int jt = pass2 ? 2 * ntiles - 1 - j : j;
-        if (j == ntiles) cut = mx - thr;
+        if (j == ntiles) cut = (tok < p.C) ? mx - thr : INFINITY;   // (rows of the M tile past the block collect nothing)
         if (!tc::mbar_wait(&bars[RB_SFULL + buf], (j >> 1) & 1)) {
           atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; break;
         }
@@ -213,18 +214,31 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
             const int a = min(32, max(0, lo - c4 * 32)), b = min(32, max(0, nvalid - c4 * 32));
             vm = (b <= a) ? 0u : ((b == 32 ? 0xffffffffu : ((1u << b) - 1u)) & ~((1u << a) - 1u));
           }
-          if (!pass2) {
-            // four independent chains: one chain of 32 dependent maxima is latency-bound
-            float cm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-            if (plain) {
+          // maximum of the chunk's columns that count: four chains of three-input maxima (half an
+          // instruction per element)
+          float cmax;
+          if (plain) {
+            float t4[4] = {__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]), __uint_as_float(r[3])};
 #pragma unroll
-              for (int i = 0; i < 32; ++i) cm[i & 3] = fmaxf(cm[i & 3], __uint_as_float(r[i]));
-            } else {
+            for (int i = 4; i < 28; i += 8) {
 #pragma unroll
-              for (int i = 0; i < 32; ++i) cm[i & 3] = fmaxf(cm[i & 3], ((vm >> i) & 1u) ? __uint_as_float(r[i]) : -INFINITY);
+              for (int k = 0; k < 4; ++k) t4[k] = tc::fmax3(t4[k], __uint_as_float(r[i + k]), __uint_as_float(r[i + 4 + k]));
             }
-            mx = fmaxf(mx, fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3])));
+#pragma unroll
+            for (int k = 0; k < 4; ++k) t4[k] = fmaxf(t4[k], __uint_as_float(r[28 + k]));
+            cmax = fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3]));
           } else {
+            float cm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int i = 0; i < 32; ++i) cm[i & 3] = fmaxf(cm[i & 3], ((vm >> i) & 1u) ? __uint_as_float(r[i]) : -INFINITY);
+            cmax = fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3]));
+          }
+          if (!pass2) {
+            mx = fmaxf(mx, cmax);
+          } else {
+            // a chunk is looked at element by element only when some token of the warp has a candidate
+            // in it (about one chunk in four: a token has about one candidate among all rows of the split)
+            if (!__any_sync(0xffffffffu, cmax >= cut)) continue;
             uint32_t h4[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
             for (int i = 0; i < 32; ++i) h4[i & 3] |= (__uint_as_float(r[i]) >= cut) ? (1u << i) : 0u;
