@@ -576,11 +576,11 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
     if (f0 >= n_call_folds) return;
     const int nf = n_call_folds - f0 < per_batch ? n_call_folds - f0 : per_batch;
     const int h = k % halves;
-    bool want_gram = false;              // does a fold of the batch append some, not all, of its tokens?
+    bool want_gram = false;              // does a fold of the batch append more than a few, not all, of its tokens?
     int64_t m_sim = s.m;
     for (int i = 0; i < f0 + nf; ++i) {
       // (m_sim restarts from the current rows: folds before f0 that are already launched moved s.m)
-      if (i >= n_done_folds) { if (i >= f0 && fold_na[i] > 0 && fold_na[i] < C && m_sim > 0) want_gram = true; m_sim += fold_na[i]; }
+      if (i >= n_done_folds) { if (i >= f0 && fold_na[i] > kGramOnTheFly && fold_na[i] < C && m_sim > 0) want_gram = true; m_sim += fold_na[i]; }
     }
     if (ovk && batch_done_rec[h]) ev_ok = ev_ok && cudaStreamWaitEvent(kstream, s.evBatchDone[h], 0) == cudaSuccess;
     const int64_t bf = (cf0 + f0 + 1) * C - L;   // first token of the first block of the batch
@@ -680,7 +680,7 @@ KVM_API kvm_status_t kvm_decode_step(const void* q, const void* k, const void* v
     fa.b = b; fa.m = s.m; fa.first = (s.m == 0); fa.n_append = n_a; fa.slot = 0; fa.before_apply = nullptr;
     fa.early_start = false;   // the memory-key kernel runs right before the filter on this stream
     s.launches += launch_prev_copy(&s, stream);
-    s.launches += launch_kbar(&s, fa.ok, fa.unit_stride, 1, 0, n_a > 0 && n_a < C && s.m > 0, stream);
+    s.launches += launch_kbar(&s, fa.ok, fa.unit_stride, 1, 0, n_a > kGramOnTheFly && n_a < C && s.m > 0, stream);
     s.launches += launch_fold(&s, fa, stream);
     s.m += n_a;
     s.nfolds += 1;

@@ -68,7 +68,7 @@ __global__ void __launch_bounds__(256, 2) kbar_kernel(const __half* __restrict__
                                                       double* __restrict__ kbar64, __half* __restrict__ kbarH,
                                                       float* __restrict__ kbarNorm, double2* __restrict__ kbarHatStat,
                                                       __half* __restrict__ kbarHatH, int C, int Cmax, int CbarRows, int U, int Hkv, int r,
-                                                      double ln_eps) {
+                                                      double ln_eps, int write_hat) {
   constexpr int NI = D / 32;          // runs of four channels per lane
   constexpr int NC = 4 * NI;          // channels per lane
   constexpr double inv_d = 1.0 / D;   // D is a power of two: the multiplication is the division, exactly
@@ -140,7 +140,7 @@ __global__ void __launch_bounds__(256, 2) kbar_kernel(const __half* __restrict__
       const double hat = (double)wv[e] * ((kb[4 * i + e] - mu2) * rs2) + (double)bv[e];
       kh[e] = __float2half_rn((float)hat);
     }
-    if (live) *reinterpret_cast<uint2*>(kbarHatH + oh + x) = *reinterpret_cast<const uint2*>(kh);
+    if (live && write_hat) *reinterpret_cast<uint2*>(kbarHatH + oh + x) = *reinterpret_cast<const uint2*>(kh);
   }
   if (live && sub == 0) {
     kbarNorm[((int64_t)g * U + u) * Cmax + j] = (float)sqrt(n2) * 1.000001f;
@@ -283,7 +283,9 @@ struct FoldDecideParams {
   const float* kbarNorm;
   const double2* kbarHatStat;   // (mean, rstd) of kbar_j: LN_s(kbar_j), the key of the row token j would create,
                                 // is gam * ((kbar_j - mean) * rstd) + bet, the expression of the memory-key kernel
-  const float* gramT;        // [U, Cmax, Cmax] approximate kbarHat_a . kbar_j at [a][j] (fp16 operands)
+  const float* gramT;        // [U, Cmax, Cmax] approximate kbarHat_a . kbar_j at [a][j] (fp16 operands); folds that append more than kGramOnTheFly rows
+  const __half* kbarH;       // [U, CbarRows, D] memory keys in fp16 (operand of the products that small folds compute themselves)
+  int CbarRows;
   const float* candV;
   const int32_t* candI;
   const float *ln_w, *ln_b;
@@ -381,6 +383,7 @@ __global__ void __launch_bounds__(kDecideThreads, PER_SM) fold_decide_kernel(Fol
   __shared__ int s_wsum[kDecideWarps];
   __shared__ int s_gmaxi[kMaxBlock], s_fill[kMaxBlock];
   __shared__ float s_thr[kMaxBlock];
+  __shared__ __align__(16) __half s_hat[kGramOnTheFly][D];   // LN_s(kbar_a) of the rows a small fold appends
 
   // grid (R, U): CTA r of a unit refines the candidates of tokens [jlo, jhi); the CTA of the unit
   // that finishes last (a ticket, nobody waits) takes the decisions that need every token
@@ -644,29 +647,92 @@ __global__ void __launch_bounds__(kDecideThreads, PER_SM) fold_decide_kernel(Fol
   //      Those few pairs are recomputed in fp64; everything else is decided by the bound. ----
   if (tid == 0) { atomicAdd(&p.counters[1], min(s_np, kPairCap)); s_np = 0; }
   __syncthreads();
+  // A fold that appends only a few rows (n_a <= kGramOnTheFly, i.e. nearly every fold of a growing state)
+  // computes the approximate products itself, fp16 x fp16 -> fp32 on the scalar cores, against the new rows'
+  // keys LN_s(kbar_a) rounded to fp16 in shared memory: n_a x C products instead of the C x C that the
+  // batched tensor-core product of the block's token pairs holds.  The error bound is the same (fp16
+  // rounding of both operands; fp32 accumulation errs less than the tensor core's).
+  const bool otf = n_a <= kGramOnTheFly;
+  if (n_a > 0 && otf) {
+    for (int a = warp; a < n_a; a += kDecideWarps) {
+      const int jc = s_creator[a];
+      const double* ka = kbarU + (int64_t)jc * D;
+      const double2 hs = p.kbarHatStat[tokBase + jc];
+#pragma unroll
+      for (int c = 0; c < CH; ++c)
+        s_hat[a][lane + 32 * c] = __float2half_rn((float)(gam[c] * ((ka[lane + 32 * c] - hs.x) * hs.y) + bet[c]));
+    }
+    __syncthreads();
+  }
   if (n_a > 0 && tid < C) {
     const int j = tid;
     s_pcnt[j] = 0;
     s_exh[j] = 0;
     if (!s_app[j]) {
       const double eps = 0.5 * (double)(p.thr_coeff * p.kbarNorm[tokBase + j] + 1e-5f);
-      const float* gcol = p.gramT + (int64_t)u * p.Cmax * p.Cmax + j;
+      const double best_old = s_best[j];
+      // one pass over the products with the new rows, ascending a: contenders are kept while they reach the
+      // running bar (which only rises: a superset) and pruned against the final bar afterwards
       float gm = -INFINITY;
-#pragma unroll 8
-      for (int a = 0; a < n_a; ++a) gm = fmaxf(gm, gcol[(int64_t)s_creator[a] * p.Cmax]);
-      const double bar = fmax(s_best[j], (double)gm - eps) - eps;
-      // second and last pass over the row of products: the (few) contenders, kept in registers
       int cntc = 0, ca[4] = {0, 0, 0, 0};
-#pragma unroll 8
-      for (int a = 0; a < n_a; ++a) {
-        if ((double)gcol[(int64_t)s_creator[a] * p.Cmax] >= bar) {
+      float cp[4] = {0.f, 0.f, 0.f, 0.f};
+      auto consider = [&](int a, float pv) {
+        gm = fmaxf(gm, pv);
+        if ((double)pv >= fmax(best_old, (double)gm - eps) - eps) {
 #pragma unroll
           for (int k = 0; k < 4; ++k)
-            if (k == cntc) ca[k] = a;
+            if (k == cntc) { ca[k] = a; cp[k] = pv; }
           ++cntc;
         }
+      };
+      if (otf) {
+        const __half* kj = p.kbarH + ((int64_t)u * p.CbarRows + j) * D;
+        for (int a0 = 0; a0 < n_a; a0 += 4) {
+          float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 2
+          for (int ch = 0; ch < D / 8; ++ch) {
+            const uint4 kw = *reinterpret_cast<const uint4*>(kj + 8 * ch);
+            const __half2* kh = reinterpret_cast<const __half2*>(&kw);
+            float2 kf[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) kf[q] = __half22float2(kh[q]);
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+              const int a = min(a0 + t, n_a - 1);   // (a clamped duplicate is computed and dropped)
+              const uint4 hw = *reinterpret_cast<const uint4*>(&s_hat[a][8 * ch]);
+              const __half2* hh = reinterpret_cast<const __half2*>(&hw);
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const float2 hf = __half22float2(hh[q]);
+                acc[t] = fmaf(kf[q].x, hf.x, acc[t]);
+                acc[t] = fmaf(kf[q].y, hf.y, acc[t]);
+              }
+            }
+          }
+#pragma unroll
+          for (int t = 0; t < 4; ++t)
+            if (a0 + t < n_a) consider(a0 + t, acc[t]);
+        }
+      } else {
+        const float* gcol = p.gramT + (int64_t)u * p.Cmax * p.Cmax + j;
+#pragma unroll 8
+        for (int a = 0; a < n_a; ++a) consider(a, gcol[(int64_t)s_creator[a] * p.Cmax]);
       }
       bool exh = cntc > 4;   // more than four contenders: every new row exactly
+      if (!exh) {            // prune against the final bar (order kept: ascending new-row index)
+        const double bar = fmax(best_old, (double)gm - eps) - eps;
+        int kept = 0;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (k < cntc && (double)cp[k] >= bar) {
+#pragma unroll
+            for (int k2 = 0; k2 < 4; ++k2)
+              if (k2 == kept) ca[k2] = ca[k];
+            ++kept;
+          }
+        }
+        cntc = kept;
+      }
       int start = 0;
       if (!exh && cntc > 0) {
         start = atomicAdd(&s_np, cntc);
@@ -1257,10 +1323,10 @@ int launch_kbar(State* st, const __half* ok, int64_t unit_stride, int nblk, int 
   __half* khh = st->kbarHatH + (int64_t)slot0 * U * st->CbarRows * D;
   if (D == 128)
     kbar_kernel<128><<<grid, 256, 0, s>>>(ok, unit_stride, st->ln_w, st->ln_b, k64, kh, kn, khat, khh, C, st->Cmax,
-                                          st->CbarRows, st->U, st->Hkv, st->r, (double)st->ln_eps);
+                                          st->CbarRows, st->U, st->Hkv, st->r, (double)st->ln_eps, want_gram ? 1 : 0);
   else
     kbar_kernel<64><<<grid, 256, 0, s>>>(ok, unit_stride, st->ln_w, st->ln_b, k64, kh, kn, khat, khh, C, st->Cmax,
-                                         st->CbarRows, st->U, st->Hkv, st->r, (double)st->ln_eps);
+                                         st->CbarRows, st->U, st->Hkv, st->r, (double)st->ln_eps, want_gram ? 1 : 0);
   int launches = 1;
   // the new-row filter is only read by folds that append some but not all of their tokens
   if (want_gram) launches += launch_gram_tc(st, slot0, nblk, s);
@@ -1322,6 +1388,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
     FoldDecideParams p;
     p.kbar64 = kbar64; p.kbarNorm = kbarNorm; p.kbarHatStat = kbarHatStat;
     p.gramT = st->gramT + (int64_t)a.slot * U * st->Cmax * st->Cmax;
+    p.kbarH = kbarH; p.CbarRows = st->CbarRows;
     p.candV = st->candV; p.candI = st->candI; p.ln_w = st->ln_w; p.ln_b = st->ln_b;
     p.sumK = st->sumK; p.kmu = st->kmu; p.krstd = st->krstd;
     p.pi = st->foldPi[dst]; p.sorted = st->foldSorted[dst]; p.creator = st->foldCreator[dst];

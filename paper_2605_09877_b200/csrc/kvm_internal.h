@@ -15,6 +15,9 @@ constexpr int kMaxSplits = 32;      // routing filter / decode split count upper
 constexpr int kAttnSplitTiles = 37; // launches with at most this many (batch, head, query tile) CTAs - a quarter of the GPU - are split along the keys
 constexpr int kAttnMaxSplits = 8;
 constexpr int kRowAlign = 128;      // state capacity is rounded up to the attention key tile
+constexpr int kGramOnTheFly = 32;   // folds that append at most this many rows compute the products of the other tokens with the
+                                    // new rows inside the decision kernel; larger ones read them from the batched tensor-core
+                                    // product of all token pairs of the block (gramT), most of which such a fold would never read
 constexpr int kSerialUnits = 256;   // from this many (batch, kv head) units on, folds run on the caller's stream with one readout copy
 
 // State of one layer: host bookkeeping + device buffers.  U = batch * n_kv_heads "units";
