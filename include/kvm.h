@@ -177,8 +177,17 @@ kvm_status_t kvm_state_info(const kvm_state_t* state, int64_t* n_slots, int64_t*
                             int64_t* n_folds);
 
 /* Reads the device status word (set by bounded device-side waits or debug index checks)
- * after synchronising the stream: KVM_OK, KVM_ERR_TIMEOUT or KVM_ERR_CUDA. */
+ * after synchronising the stream and clears it: KVM_OK, KVM_ERR_TIMEOUT or KVM_ERR_CUDA.  A kernel
+ * whose wait ran out has torn down normally (its outputs are undefined); the state can be reset
+ * (kvm_state_reset) or restored (kvm_state_import) and used again. */
 kvm_status_t kvm_state_check(kvm_state_t* state, void* cuda_stream);
+
+/* Failure-detection self test (no counterpart in the paper): launches one thread that waits, with the
+ * library's bounded wait and a limit of `spins` iterations (1 .. 2^20), on a barrier that nothing ever
+ * arrives at, and reports the expiry exactly as the production kernels do: KVM_ERR_TIMEOUT in the
+ * state's status word, normal return.  kvm_state_check then returns KVM_ERR_TIMEOUT once.  Touches
+ * nothing else of the state. */
+kvm_status_t kvm_debug_expire_wait(kvm_state_t* state, int32_t spins, void* cuda_stream);
 
 /* Copies the state rows to HOST arrays (synchronises the stream).  Shapes, with
  * U = batch * n_kv_heads and m = n_slots:
@@ -257,9 +266,11 @@ kvm_status_t kvm_state_reset(kvm_state_t* state);
 kvm_status_t kvm_profile_enable(kvm_state_t* state, int32_t on);
 kvm_status_t kvm_profile_read(kvm_state_t* state, double* ms, int64_t* groups);
 
-/* Debug counters of the fold since the state was created (synchronises the stream):
+/* Debug counters since the state was created (synchronises the stream):
  * out[0] overflow tokens whose routing fell back to the exhaustive fp64 scan, out[1] candidate
- * (token, row) pairs refined in fp64, out[2] overflow tokens routed.  32-bit device counters. */
+ * (token, row) pairs refined in fp64, out[2] overflow tokens routed, out[3] input elements of q, k, v
+ * whose magnitude exceeded 65504 and was clamped on the way in (bf16 inputs are carried as fp16).
+ * `out` has room for four values.  32-bit device counters. */
 kvm_status_t kvm_debug_counters(kvm_state_t* state, int64_t* out, void* cuda_stream);
 
 /* Number of kernels the library has launched for this state so far (host counter). */
@@ -302,12 +313,15 @@ kvm_status_t kvm_attend_rows_noalloc(const void* q, const void* keys, const void
  *                                                    d_model a multiple of 8
  *   w_gate  device fp32 [n_kv_heads, d_model]
  *   gate    device fp32 [batch, n_kv_heads, n_tokens]   (out)
+ *   status  device int32 word or NULL: the tensor-core path waits on barriers with a bounded number of
+ *           spins; should such a wait ever run out, the gates of the affected tokens are NaN and
+ *           KVM_ERR_TIMEOUT is stored here (the word is never cleared by the library: zero it before)
  * Products and sums in fp32 (inputs bf16 -> fp32 exactly).  n_kv_heads <= 64 and batch <= 65535,
  * else KVM_ERR_UNSUPPORTED; bad pointers, alignment or sizes KVM_ERR_INVALID_ARG; nothing is
  * launched on an error.  The caller owns all three buffers; no allocation, no synchronisation;
  * the work is enqueued on cuda_stream on the current device. */
 kvm_status_t kvm_merge_gate(const void* x, const float* w_gate, int32_t batch, int64_t n_tokens, int32_t d_model,
-                            int32_t n_kv_heads, float* gate, void* cuda_stream);
+                            int32_t n_kv_heads, float* gate, int32_t* status, void* cuda_stream);
 
 /* Front end, LN_q / LN_k (Appendix, time mixer of the backbone: q_t <- RoPE_r(LN_q(q_t)),
  * k_t <- RoPE_r(LN_k(k_t))): LayerNorm over the head channels of every (batch, head, token) row, in

@@ -418,7 +418,7 @@ KVM_API kvm_status_t kvm_debug_counters(kvm_state_t* ks, int64_t* out, void* cud
   int32_t w[16];
   if (cudaMemcpyAsync(w, ks->s.status, sizeof(w), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return KVM_ERR_CUDA;
   if (cudaStreamSynchronize(stream) != cudaSuccess) return KVM_ERR_CUDA;
-  for (int i = 0; i < 3; ++i) out[i] = w[1 + i];
+  for (int i = 0; i < 4; ++i) out[i] = w[1 + i];
   return KVM_OK;
 }
 
@@ -470,7 +470,17 @@ KVM_API kvm_status_t kvm_state_check(kvm_state_t* ks, void* cuda_stream) {
   if (cudaMemcpyAsync(&w, ks->s.status, sizeof(w), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return KVM_ERR_CUDA;
   if (cudaStreamSynchronize(stream) != cudaSuccess) return KVM_ERR_CUDA;
   if (w == 0) return KVM_OK;
+  if (cudaMemsetAsync(ks->s.status, 0, sizeof(w), stream) != cudaSuccess) return KVM_ERR_CUDA;   // reported once
   return w == KVM_ERR_TIMEOUT ? KVM_ERR_TIMEOUT : KVM_ERR_CUDA;
+}
+
+KVM_API kvm_status_t kvm_debug_expire_wait(kvm_state_t* ks, int32_t spins, void* cuda_stream) {
+  if (!ks || spins < 1 || spins > (1 << 20)) return KVM_ERR_INVALID_ARG;
+  DeviceGuard guard(ks->s.device);
+  if (!guard.ok) return KVM_ERR_CUDA;
+  launch_expire_wait(&ks->s, spins, (cudaStream_t)cuda_stream);
+  ks->s.launches += 1;
+  return launch_ok() ? KVM_OK : KVM_ERR_CUDA;
 }
 
 KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kvm_state_t* ks, int32_t block,

@@ -586,6 +586,16 @@ int launch_attn_tc(State* st, const AttnArgs& a, cudaStream_t s) {
   return 1;
 }
 
+// Self test of the bounded waits (kvm_debug_expire_wait): the wait below can only run out.
+__global__ void expire_wait_kernel(int32_t* status, uint32_t spins) {
+  __shared__ uint64_t bar;
+  tc::mbar_init(&bar, 1);
+  tc::fence_barrier_init();
+  if (!tc::mbar_wait(&bar, 0, spins)) atomicExch(status, (int)KVM_ERR_TIMEOUT);
+}
+
+void launch_expire_wait(State* st, int spins, cudaStream_t s) { expire_wait_kernel<<<1, 1, 0, s>>>(st->status, (uint32_t)spins); }
+
 bool setup_attn_tc(State* st) {
   CUtensorMap* tm = reinterpret_cast<CUtensorMap*>(st->tmaps);
   bool ok = encode_tmap_rows(&tm[0], st->stQ, st->d, st->Tcall, (int64_t)st->B * st->Hq, 128);

@@ -15,7 +15,7 @@ __global__ void decode_ingest_kernel(const __nv_bfloat16* __restrict__ q, const 
                                      const double* __restrict__ inv_freq, __half* __restrict__ decQ,
                                      __half* __restrict__ ringK, __half* __restrict__ ringV,
                                      float* __restrict__ ringG, int nQ, int nKV, int d, int r, int64_t t,
-                                     int64_t ringCap, int64_t ringLen) {
+                                     int64_t ringCap, int64_t ringLen, int32_t* __restrict__ sat_counter) {
   // blocks [0, nQ): query heads; blocks [nQ, nQ + nKV): kv units
   const int x = threadIdx.x;
   if (x >= d) return;
@@ -34,6 +34,7 @@ __global__ void decode_ingest_kernel(const __nv_bfloat16* __restrict__ q, const 
     const float val = __bfloat162float(row[x]);
     const float oth = __bfloat162float(row[partner]);
     const float o = (x < r) ? (x < half ? val * cs - oth * sn : oth * sn + val * cs) : val;
+    if (!(fabsf(o) <= 65504.f)) atomicAdd(sat_counter, 1);   // (clamped: counted for the debug counter)
     decQ[(int64_t)blockIdx.x * d + x] = __float2half_rn(fminf(fmaxf(o, -65504.f), 65504.f));
   } else {
     const int u = blockIdx.x - nQ;
@@ -42,8 +43,11 @@ __global__ void decode_ingest_kernel(const __nv_bfloat16* __restrict__ q, const 
     const float oth = __bfloat162float(row[partner]);
     const float o = (x < r) ? (x < half ? val * cs - oth * sn : oth * sn + val * cs) : val;
     const int64_t rrow = (int64_t)u * ringCap + (t % ringLen);
+    const float vv = __bfloat162float(v[(int64_t)u * d + x]);
+    const int nsat = (!(fabsf(o) <= 65504.f) ? 1 : 0) + (!(fabsf(vv) <= 65504.f) ? 1 : 0);
+    if (nsat) atomicAdd(sat_counter, nsat);
     ringK[rrow * d + x] = __float2half_rn(fminf(fmaxf(o, -65504.f), 65504.f));
-    ringV[rrow * d + x] = __float2half_rn(fminf(fmaxf(__bfloat162float(v[(int64_t)u * d + x]), -65504.f), 65504.f));
+    ringV[rrow * d + x] = __float2half_rn(fminf(fmaxf(vv, -65504.f), 65504.f));
     if (x == 0) ringG[rrow] = gate ? gate[u] : 1.0f;
   }
 }
@@ -232,7 +236,7 @@ int launch_decode(State* st, const DecodeArgs& a, cudaStream_t s) {
   const int nQ = st->B * st->Hq, nKV = st->U;
   decode_ingest_kernel<<<nQ + nKV, D, 0, s>>>(a.q, a.k, a.v, a.gate, st->inv_freq, st->decQ, st->ringK, st->ringV,
                                               st->ringG, nQ, nKV, D, st->r, a.t, (int64_t)st->w * st->Cmax,
-                                              st->ringLen);
+                                              st->ringLen, st->status + 4);
   ++launches;
   DecodeParams p;
   p.decQ = st->decQ; p.Khat = st->KhatBuf[st->nfolds & 1]; p.Vhat = st->VhatBuf[st->nfolds & 1]; p.ringK = st->ringK; p.ringV = st->ringV;

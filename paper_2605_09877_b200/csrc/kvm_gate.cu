@@ -113,7 +113,7 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N) {   // as tc::id
 template <int NP>   // heads padded to a multiple of 16
 __global__ void __launch_bounds__(192, 1)
 merge_gate_tc_kernel(const __grid_constant__ CUtensorMap mapX, const float* __restrict__ w, float* __restrict__ gate,
-                     int64_t T, int dm, int H) {
+                     int64_t T, int dm, int H, int32_t* status) {
   constexpr int WBYTES = 2 * NP * 128;     // hi and lo tiles of one slice
   constexpr uint32_t TMEM_COLS = NP <= 32 ? 32 : 64;
   extern __shared__ uint8_t smem_raw[];
@@ -252,6 +252,9 @@ merge_gate_tc_kernel(const __grid_constant__ CUtensorMap mapX, const float* __re
       }
     }
   }
+  // a wait that ran out: the gates of this tile are NaN, and the caller's status word (if any) says why
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag && status) atomicExch(status, (int)KVM_ERR_TIMEOUT);
   tc::tc_fence_before();
   __syncthreads();
   if (warp == 1) {
@@ -261,7 +264,8 @@ merge_gate_tc_kernel(const __grid_constant__ CUtensorMap mapX, const float* __re
 }
 
 template <int NP>
-static bool launch_gate_tc(const CUtensorMap& map, const float* w, float* gate, int batch, int64_t T, int dm, int H, cudaStream_t s) {
+static bool launch_gate_tc(const CUtensorMap& map, const float* w, float* gate, int batch, int64_t T, int dm, int H, int32_t* status,
+                           cudaStream_t s) {
   const int smem = kGateTcStages * (kGateTcXBytes + 2 * NP * 128) + 256 + 1024;
   static bool attr_set = false;   // (per instantiation; setting it again is harmless)
   if (!attr_set) {
@@ -269,7 +273,7 @@ static bool launch_gate_tc(const CUtensorMap& map, const float* w, float* gate, 
     attr_set = true;
   }
   const dim3 grid((unsigned)((T + 127) / 128), (unsigned)batch);
-  merge_gate_tc_kernel<NP><<<grid, 192, smem, s>>>(map, w, gate, T, dm, H);
+  merge_gate_tc_kernel<NP><<<grid, 192, smem, s>>>(map, w, gate, T, dm, H, status);
   return true;
 }
 
@@ -279,9 +283,9 @@ using namespace kvm;
 
 extern "C" __attribute__((visibility("default")))
 kvm_status_t kvm_merge_gate(const void* x, const float* w_gate, int32_t batch, int64_t n_tokens, int32_t d_model,
-                                    int32_t n_kv_heads, float* gate, void* cuda_stream) {
+                                    int32_t n_kv_heads, float* gate, int32_t* status, void* cuda_stream) {
   if (!x || !w_gate || !gate || batch < 1 || n_tokens < 1 || d_model < 8 || n_kv_heads < 1) return KVM_ERR_INVALID_ARG;
-  if (d_model % 8 || ((uintptr_t)x & 15) || ((uintptr_t)w_gate & 3) || ((uintptr_t)gate & 3)) return KVM_ERR_INVALID_ARG;
+  if (d_model % 8 || ((uintptr_t)x & 15) || ((uintptr_t)w_gate & 3) || ((uintptr_t)gate & 3) || ((uintptr_t)status & 3)) return KVM_ERR_INVALID_ARG;
   if (n_kv_heads > 64) return KVM_ERR_UNSUPPORTED;
   if (batch > 65535) return KVM_ERR_UNSUPPORTED;
   cudaStream_t s = (cudaStream_t)cuda_stream;
@@ -292,10 +296,10 @@ kvm_status_t kvm_merge_gate(const void* x, const float* w_gate, int32_t batch, i
     CUtensorMap map;
     if (encode_tmap_rows(&map, x, d_model, n_tokens, batch, 128)) {
       bool ok;
-      if (n_kv_heads <= 16) ok = launch_gate_tc<16>(map, w_gate, gate, batch, n_tokens, d_model, n_kv_heads, s);
-      else if (n_kv_heads <= 32) ok = launch_gate_tc<32>(map, w_gate, gate, batch, n_tokens, d_model, n_kv_heads, s);
-      else if (n_kv_heads <= 48) ok = launch_gate_tc<48>(map, w_gate, gate, batch, n_tokens, d_model, n_kv_heads, s);
-      else ok = launch_gate_tc<64>(map, w_gate, gate, batch, n_tokens, d_model, n_kv_heads, s);
+      if (n_kv_heads <= 16) ok = launch_gate_tc<16>(map, w_gate, gate, batch, n_tokens, d_model, n_kv_heads, status, s);
+      else if (n_kv_heads <= 32) ok = launch_gate_tc<32>(map, w_gate, gate, batch, n_tokens, d_model, n_kv_heads, status, s);
+      else if (n_kv_heads <= 48) ok = launch_gate_tc<48>(map, w_gate, gate, batch, n_tokens, d_model, n_kv_heads, status, s);
+      else ok = launch_gate_tc<64>(map, w_gate, gate, batch, n_tokens, d_model, n_kv_heads, status, s);
       if (ok) return cudaGetLastError() == cudaSuccess ? KVM_OK : KVM_ERR_CUDA;
     }
     cudaGetLastError();   // fall through to the scalar path

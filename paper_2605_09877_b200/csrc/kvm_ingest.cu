@@ -47,7 +47,9 @@ __global__ void ingest_hist_kernel(__half* __restrict__ stK, __half* __restrict_
 // bits for the rotated values, the readout cache and the softmax weights).  Every bf16 value
 // with 2^-14 <= |x| <= 65504 converts exactly; larger magnitudes saturate, smaller ones round
 // with an absolute error below 2^-25.
-__device__ __forceinline__ __half2 to_half2_sat(float a, float b) {
+// (nsat counts the values that did not fit - magnitudes above 65504, infinities, NaNs - for the debug counter)
+__device__ __forceinline__ __half2 to_half2_sat(float a, float b, int& nsat) {
+  nsat += (!(fabsf(a) <= 65504.f) ? 1 : 0) + (!(fabsf(b) <= 65504.f) ? 1 : 0);
   a = fminf(fmaxf(a, -65504.f), 65504.f);
   b = fminf(fmaxf(b, -65504.f), 65504.f);
   return __floats2half2_rn(a, b);
@@ -77,10 +79,11 @@ __global__ void ingest_kv_kernel(__half* __restrict__ stK, __half* __restrict__ 
                                  int64_t sk0, int64_t sk1, int64_t sk2, int64_t sv0, int64_t sv1, int64_t sv2,
                                  int64_t sg0, int64_t sg1, int64_t sg2, int Hkv, int d, int r,
                                  int64_t stRows, int64_t ringCap, int64_t ringLen, int64_t pos0, int64_t n,
-                                 int64_t nhist, int64_t tail_start) {
+                                 int64_t nhist, int64_t tail_start, int32_t* __restrict__ sat_counter) {
   const int u = blockIdx.y;
   const int b = u / Hkv, hk = u % Hkv;
   const int hw = d / 2;
+  int nsat = 0;
   int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= n * hw) return;
   int64_t j = idx / hw;
@@ -88,8 +91,9 @@ __global__ void ingest_kv_kernel(__half* __restrict__ stK, __half* __restrict__ 
   const __nv_bfloat16* krow = k + b * sk0 + hk * sk1 + j * sk2;
   const __nv_bfloat16* vrow = v + b * sv0 + hk * sv1 + j * sv2;
   const float2* cs = ropeCS + j * (r >> 1);
-  const __half2 kk = to_half2_sat(rope_channel(krow, 2 * c2, r, cs), rope_channel(krow, 2 * c2 + 1, r, cs));
-  const __half2 vv = to_half2_sat(__bfloat162float(vrow[2 * c2]), __bfloat162float(vrow[2 * c2 + 1]));
+  const __half2 kk = to_half2_sat(rope_channel(krow, 2 * c2, r, cs), rope_channel(krow, 2 * c2 + 1, r, cs), nsat);
+  const __half2 vv = to_half2_sat(__bfloat162float(vrow[2 * c2]), __bfloat162float(vrow[2 * c2 + 1]), nsat);
+  if (nsat) atomicAdd(sat_counter, nsat);
   float g = gate ? gate[b * sg0 + hk * sg1 + j * sg2] : 1.0f;
   const int64_t row = (int64_t)u * stRows + nhist + j;
   reinterpret_cast<__half2*>(stK + row * d)[c2] = kk;
@@ -107,10 +111,11 @@ __global__ void ingest_kv_kernel(__half* __restrict__ stK, __half* __restrict__ 
 
 __global__ void ingest_q_kernel(__half* __restrict__ stQ, const __nv_bfloat16* __restrict__ q,
                                 const float2* __restrict__ ropeCS, int64_t sq0, int64_t sq1, int64_t sq2,
-                                int Hq, int d, int r, int64_t Tcall, int64_t n) {
+                                int Hq, int d, int r, int64_t Tcall, int64_t n, int32_t* __restrict__ sat_counter) {
   const int bh = blockIdx.y;
   const int b = bh / Hq, h = bh % Hq;
   const int hw = d / 2;
+  int nsat = 0;
   int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= n * hw) return;
   int64_t j = idx / hw;
@@ -118,7 +123,8 @@ __global__ void ingest_q_kernel(__half* __restrict__ stQ, const __nv_bfloat16* _
   const __nv_bfloat16* qrow = q + b * sq0 + h * sq1 + j * sq2;
   const float2* cs = ropeCS + j * (r >> 1);
   reinterpret_cast<__half2*>(stQ + ((int64_t)bh * Tcall + j) * d)[c2] =
-      to_half2_sat(rope_channel(qrow, 2 * c2, r, cs), rope_channel(qrow, 2 * c2 + 1, r, cs));
+      to_half2_sat(rope_channel(qrow, 2 * c2, r, cs), rope_channel(qrow, 2 * c2 + 1, r, cs), nsat);
+  if (nsat) atomicAdd(sat_counter, nsat);
 }
 
 // ---- 16-byte versions (rows 16-byte aligned, rotary half a multiple of 8 channels): a thread
@@ -155,9 +161,9 @@ __device__ __forceinline__ void rope8(const __nv_bfloat16* __restrict__ row, int
   }
 }
 
-__device__ __forceinline__ uint4 pack8_sat(const float (&x)[8]) {
+__device__ __forceinline__ uint4 pack8_sat(const float (&x)[8], int& nsat) {
   uint4 o;
-  __half2 h0 = to_half2_sat(x[0], x[1]), h1 = to_half2_sat(x[2], x[3]), h2 = to_half2_sat(x[4], x[5]), h3 = to_half2_sat(x[6], x[7]);
+  __half2 h0 = to_half2_sat(x[0], x[1], nsat), h1 = to_half2_sat(x[2], x[3], nsat), h2 = to_half2_sat(x[4], x[5], nsat), h3 = to_half2_sat(x[6], x[7], nsat);
   o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
   o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
   return o;
@@ -169,7 +175,7 @@ __global__ void __launch_bounds__(256) ingest_kv_vec_kernel(
     const __nv_bfloat16* __restrict__ v, const float* __restrict__ gate, const float2* __restrict__ ropeCS,
     int64_t sk0, int64_t sk1, int64_t sk2, int64_t sv0, int64_t sv1, int64_t sv2, int64_t sg0, int64_t sg1,
     int64_t sg2, int Hkv, int d, int r, int64_t stRows, int64_t ringCap, int64_t ringLen, int64_t pos0, int64_t n,
-    int64_t nhist, int64_t tail_start) {
+    int64_t nhist, int64_t tail_start, int32_t* __restrict__ sat_counter) {
   const int u = blockIdx.y;
   const int b = u / Hkv, hk = u % Hkv;
   const int w8 = d / 8;                       // 16-byte chunks per row
@@ -188,7 +194,9 @@ __global__ void __launch_bounds__(256) ingest_kv_vec_kernel(
       vx[2 * i] = f.x; vx[2 * i + 1] = f.y;
     }
   }
-  const uint4 kk = pack8_sat(kx), vv = pack8_sat(vx);
+  int nsat = 0;
+  const uint4 kk = pack8_sat(kx, nsat), vv = pack8_sat(vx, nsat);
+  if (nsat) atomicAdd(sat_counter, nsat);
   const float g = gate ? gate[b * sg0 + hk * sg1 + j * sg2] : 1.0f;
   const int64_t row = (int64_t)u * stRows + nhist + j;
   reinterpret_cast<uint4*>(stK + row * d)[c8] = kk;
@@ -205,7 +213,8 @@ __global__ void __launch_bounds__(256) ingest_kv_vec_kernel(
 
 __global__ void __launch_bounds__(256) ingest_q_vec_kernel(__half* __restrict__ stQ, const __nv_bfloat16* __restrict__ q,
                                                            const float2* __restrict__ ropeCS, int64_t sq0, int64_t sq1,
-                                                           int64_t sq2, int Hq, int d, int r, int64_t Tcall, int64_t n) {
+                                                           int64_t sq2, int Hq, int d, int r, int64_t Tcall, int64_t n,
+                                                           int32_t* __restrict__ sat_counter) {
   const int bh = blockIdx.y;
   const int b = bh / Hq, h = bh % Hq;
   const int w8 = d / 8, tpb = 256 / w8;
@@ -214,7 +223,9 @@ __global__ void __launch_bounds__(256) ingest_q_vec_kernel(__half* __restrict__ 
   if (j >= n) return;
   float qx[8];
   rope8(q + b * sq0 + h * sq1 + j * sq2, c8, r, ropeCS + j * (r >> 1), qx);
-  reinterpret_cast<uint4*>(stQ + ((int64_t)bh * Tcall + j) * d)[c8] = pack8_sat(qx);
+  int nsat = 0;
+  reinterpret_cast<uint4*>(stQ + ((int64_t)bh * Tcall + j) * d)[c8] = pack8_sat(qx, nsat);
+  if (nsat) atomicAdd(sat_counter, nsat);
 }
 
 int launch_ingest(State* st, const IngestArgs& a, cudaStream_t s) {
@@ -246,7 +257,7 @@ int launch_ingest(State* st, const IngestArgs& a, cudaStream_t s) {
                                               a.v, a.gate, st->ropeCS, a.sk[0], a.sk[1], a.sk[2], a.sv[0],
                                               a.sv[1], a.sv[2], a.sg[0], a.sg[1], a.sg[2], st->Hkv, d, st->r,
                                               st->stRows, (int64_t)st->w * st->Cmax, st->ringLen, a.pos0, a.n,
-                                              a.nhist, a.tail_start);
+                                              a.nhist, a.tail_start, st->status + 4);
     ++launches;
   } else {
     dim3 grid((unsigned)((a.n * hw + threads - 1) / threads), st->U);
@@ -254,18 +265,18 @@ int launch_ingest(State* st, const IngestArgs& a, cudaStream_t s) {
                                               a.v, a.gate, st->ropeCS, a.sk[0], a.sk[1], a.sk[2], a.sv[0],
                                               a.sv[1], a.sv[2], a.sg[0], a.sg[1], a.sg[2], st->Hkv, d, st->r,
                                               st->stRows, (int64_t)st->w * st->Cmax, st->ringLen, a.pos0, a.n,
-                                              a.nhist, a.tail_start);
+                                              a.nhist, a.tail_start, st->status + 4);
     ++launches;
   }
   if (rope_ok && al16(a.q, a.sq)) {
     dim3 grid((unsigned)((a.n + tpb - 1) / tpb), st->B * st->Hq);
     ingest_q_vec_kernel<<<grid, 256, 0, s>>>(st->stQ, a.q, st->ropeCS, a.sq[0], a.sq[1], a.sq[2], st->Hq, d,
-                                             st->r, st->Tcall, a.n);
+                                             st->r, st->Tcall, a.n, st->status + 4);
     ++launches;
   } else {
     dim3 grid((unsigned)((a.n * hw + threads - 1) / threads), st->B * st->Hq);
     ingest_q_kernel<<<grid, threads, 0, s>>>(st->stQ, a.q, st->ropeCS, a.sq[0], a.sq[1], a.sq[2], st->Hq, d,
-                                             st->r, st->Tcall, a.n);
+                                             st->r, st->Tcall, a.n, st->status + 4);
     ++launches;
   }
   return launches;

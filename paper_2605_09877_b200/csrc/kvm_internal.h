@@ -111,7 +111,7 @@ struct State {
   // ---- recording / status ----
   int32_t* slotTok;              // [U, Tassign]
   uint8_t* appTok;               // [U, Tassign]
-  int32_t* status;               // device status word
+  int32_t* status;               // device status word [0]; [1..3] fold debug counters; [4] inputs clamped to the fp16 range
   // ---- TMA tensor maps (host copies, passed to kernels by value):
   //      0 stQ, 1 Khat copy 0, 2 Vhat copy 0, 3 stK, 4 stV, 5 kbarH, 6 Khat copy 1, 7 Vhat copy 1,
   //      8 kbarHatH ----
@@ -189,6 +189,10 @@ struct DecodeArgs {
   int64_t m;
 };
 int launch_decode(State* st, const DecodeArgs& a, cudaStream_t s);
+
+// Self test of the bounded waits: one thread waits `spins` iterations on a barrier nobody arrives at and
+// records KVM_ERR_TIMEOUT in the status word.
+void launch_expire_wait(State* st, int spins, cudaStream_t s);
 
 // Brackets the launches issued during its lifetime with the state's timing hook (no-op when off).
 struct KernelTimer {

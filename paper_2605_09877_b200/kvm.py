@@ -26,7 +26,7 @@ EXPORTS = ["kvm_plan_capacity", "kvm_state_create", "kvm_prefill", "kvm_decode_s
            "kvm_decode_step_host", "kvm_state_free", "kvm_state_info", "kvm_state_check", "kvm_state_export",
            "kvm_debug_assignments", "kvm_launch_count", "kvm_status_string", "kvm_state_reset",
            "kvm_profile_enable", "kvm_profile_read", "kvm_debug_counters", "kvm_attend_rows_noalloc", "kvm_merge_gate", "kvm_head_layernorm",
-           "kvm_state_snapshot_info", "kvm_state_export_window", "kvm_state_import"]
+           "kvm_state_snapshot_info", "kvm_state_export_window", "kvm_state_import", "kvm_debug_expire_wait"]
 
 
 class KVMError(RuntimeError):
@@ -102,7 +102,9 @@ def _load():
     L.kvm_attend_rows_noalloc.restype = C.c_int
     L.kvm_attend_rows_noalloc.argtypes = [vp, vp, vp, C.c_int32, C.c_int64, C.c_int32, C.c_float, vp, vp]
     L.kvm_merge_gate.restype = C.c_int
-    L.kvm_merge_gate.argtypes = [vp, vp, C.c_int32, C.c_int64, C.c_int32, C.c_int32, vp, vp]
+    L.kvm_merge_gate.argtypes = [vp, vp, C.c_int32, C.c_int64, C.c_int32, C.c_int32, vp, vp, vp]
+    L.kvm_debug_expire_wait.restype = C.c_int
+    L.kvm_debug_expire_wait.argtypes = [vp, C.c_int32, vp]
     L.kvm_head_layernorm.restype = C.c_int
     L.kvm_head_layernorm.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, C.c_int64, C.c_int32, C.c_float, vp]
     L.kvm_state_snapshot_info.restype = C.c_int
@@ -128,9 +130,10 @@ def growth(kind: str, fixed_slots: int = 0, sqrt_coeff: int = 16, pow_num: int =
     return Growth(k, sqrt_coeff, fixed_slots, pow_num, pow_den, sat_half)
 
 
-def merge_gate(x: "torch.Tensor", w_gate: "torch.Tensor", out=None, stream=None) -> "torch.Tensor":
+def merge_gate(x: "torch.Tensor", w_gate: "torch.Tensor", out=None, stream=None, status=None) -> "torch.Tensor":
     """g = 1 + ELU(x W_g): x bf16 [B, T, d_model], w_gate fp32 [Hkv, d_model] -> fp32 [B, Hkv, T]
-    (argument marshalling only; the product runs in kvm_merge_gate)."""
+    (argument marshalling only; the product runs in kvm_merge_gate).  `status`: optional int32 CUDA tensor
+    of one element that receives KVM_ERR_TIMEOUT should a bounded device-side wait run out."""
     assert x.is_cuda and w_gate.is_cuda and x.dtype == torch.bfloat16 and w_gate.dtype == torch.float32
     assert x.is_contiguous() and w_gate.is_contiguous() and x.dim() == 3 and w_gate.dim() == 2
     B, T, dm = x.shape
@@ -139,7 +142,8 @@ def merge_gate(x: "torch.Tensor", w_gate: "torch.Tensor", out=None, stream=None)
     if out is None:
         out = torch.empty((B, H, T), dtype=torch.float32, device=x.device)
     rc = lib.kvm_merge_gate(C.c_void_p(x.data_ptr()), C.c_void_p(w_gate.data_ptr()), B, T, dm, H,
-                            C.c_void_p(out.data_ptr()), _stream_ptr(stream))
+                            C.c_void_p(out.data_ptr()), C.c_void_p(status.data_ptr()) if status is not None else None,
+                            _stream_ptr(stream))
     if rc != 0:
         raise KVMError(rc, "kvm_merge_gate")
     return out
@@ -325,11 +329,16 @@ class KVMState:
         return {names[i]: (ms[i], n[i]) for i in range(7)}
 
     def debug_counters(self, stream=None):
-        out = (C.c_int64 * 3)()
+        out = (C.c_int64 * 4)()
         rc = lib.kvm_debug_counters(self._h, out, _stream_ptr(stream))
         if rc != KVM_OK:
             raise KVMError(rc, "kvm_debug_counters")
-        return dict(exhaustive_tokens=out[0], candidate_pairs=out[1], tokens=out[2])
+        return dict(exhaustive_tokens=out[0], candidate_pairs=out[1], tokens=out[2], clamped_inputs=out[3])
+
+    def debug_expire_wait(self, spins: int = 10000, stream=None):
+        rc = lib.kvm_debug_expire_wait(self._h, spins, _stream_ptr(stream))
+        if rc != KVM_OK:
+            raise KVMError(rc, "kvm_debug_expire_wait")
 
     def launch_count(self):
         return lib.kvm_launch_count(self._h)
