@@ -88,8 +88,11 @@ enum {
   KVM_FLAG_SIMT_ROUTING = 1u << 3,   /* use the scalar-core routing filter (cross-check path)   */
   KVM_FLAG_MIN_KEY_SLOTS = 1u << 4,  /* debug: keep only the minimum of two memory-key slots (the look-ahead
                                         of one block that very large batches run with), whatever the size */
-  KVM_FLAG_SERIAL_FOLDS = 1u << 5    /* one readout copy and folds on the caller's stream between the attention
+  KVM_FLAG_SERIAL_FOLDS = 1u << 5,   /* one readout copy and folds on the caller's stream between the attention
                                         launches (what states of 256 or more units do by themselves) */
+  KVM_FLAG_FUSED_QK_LN = 1u << 6     /* fused front end: kvm_prefill / kvm_decode_step apply LN_q to q and LN_k to k
+                                        (ln_q_* / ln_k_* below) before the RoPE, exactly as kvm_head_layernorm
+                                        would have on the bf16 tensors, without its pass over q and k */
 };
 
 typedef struct {
@@ -109,6 +112,15 @@ typedef struct {
   int64_t max_seq_len;                             /* only used with KVM_FLAG_RECORD_ASSIGN               */
   int32_t device;                                  /* CUDA device ordinal                                 */
   uint32_t flags;
+  /* Fused front end (only read with KVM_FLAG_FUSED_QK_LN; Appendix, time mixer: q <- RoPE_r(LN_q(q)),
+   * k <- RoPE_r(LN_k(k))): host arrays, copied; NULL weight = 1, NULL bias = 0.  With the flag, q / k / v
+   * rows must be 16-byte aligned (pointers and strides) and rope_dims / 2 a multiple of 8, else
+   * kvm_prefill returns KVM_ERR_INVALID_ARG. */
+  float qk_ln_eps;                                 /* epsilon of LN_q and LN_k                            */
+  const float* ln_q_weight;                        /* host [n_q_heads, head_dim]                          */
+  const float* ln_q_bias;
+  const float* ln_k_weight;                        /* host [n_kv_heads, head_dim]                         */
+  const float* ln_k_bias;
 } kvm_config_t;
 
 /* Rows a state needs after `seq_len` tokens under (block, growth): the closed form of

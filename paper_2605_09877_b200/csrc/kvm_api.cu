@@ -315,7 +315,12 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   s.nsplitRoute = (int)((2 * 148 + U - 1) / U);
   if (s.nsplitRoute > kMaxSplits) s.nsplitRoute = kMaxSplits;
   if (s.nsplitRoute < 1) s.nsplitRoute = 1;
-  s.nsplitDec = (int)((4 * 148 + (size_t)s.B * s.Hq - 1) / ((size_t)s.B * s.Hq));
+  {
+    // decode CTAs serve up to eight query heads of a kv group; the row splits fill the GPU about four times
+    const int gq = (s.G % 8 == 0) ? 8 : (s.G % 4 == 0) ? 4 : (s.G % 2 == 0) ? 2 : 1;
+    const size_t ncta = (size_t)s.B * s.Hq / gq;
+    s.nsplitDec = (int)((4 * 148 + ncta - 1) / ncta);
+  }
   if (s.nsplitDec > kMaxSplits) s.nsplitDec = kMaxSplits;
   if (s.nsplitDec < 1) s.nsplitDec = 1;
 
@@ -323,6 +328,19 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
 #define A(ptr, count) if (rc == KVM_OK) rc = dev_alloc(ks, &(ptr), (count))
   A(s.ln_w, (size_t)s.Hkv * d); A(s.ln_b, (size_t)s.Hkv * d); A(s.tau_s, (size_t)s.Hq); A(s.tau_b, (size_t)s.Hq);
   A(s.inv_freq_all, (size_t)(d / 2) * (d / 2 + 1) / 2);
+  s.fusedLn = (cfg->flags & KVM_FLAG_FUSED_QK_LN) != 0;
+  s.qk_ln_eps = cfg->qk_ln_eps;
+  if (s.fusedLn) {
+    if (!(cfg->qk_ln_eps >= 0.f)) rc = KVM_ERR_INVALID_ARG;
+    auto up = [&](float** dst, const float* src, size_t n) {   // optional host array -> device (NULL stays NULL)
+      *dst = nullptr;
+      if (!src || rc != KVM_OK) return;
+      rc = dev_alloc(ks, dst, n, false);
+      if (rc == KVM_OK && cudaMemcpy(*dst, src, n * sizeof(float), cudaMemcpyHostToDevice) != cudaSuccess) rc = KVM_ERR_CUDA;
+    };
+    up(&s.lnq_w, cfg->ln_q_weight, (size_t)s.Hq * d); up(&s.lnq_b, cfg->ln_q_bias, (size_t)s.Hq * d);
+    up(&s.lnk_w, cfg->ln_k_weight, (size_t)s.Hkv * d); up(&s.lnk_b, cfg->ln_k_bias, (size_t)s.Hkv * d);
+  }
   A(s.sumK, U * M * d); A(s.sumV, U * M * d); A(s.rho, U * M); A(s.wsum, U * M); A(s.cnt, U * M);
   A(s.kmu, U * M); A(s.krstd, U * M);
   // with enough units every kernel of a fold fills the GPU by itself and nothing is gained by running the
@@ -516,6 +534,9 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
     const kvm_status_t rc = validate_prefill(s, block, growth, rope_dims, n);
     if (rc != KVM_OK) return rc;
   }
+  ia.q = (const __nv_bfloat16*)q; ia.k = (const __nv_bfloat16*)k; ia.v = (const __nv_bfloat16*)v;
+  // the fused front end works on whole 16-byte chunks of every row
+  if (s.fusedLn && !ingest_rows_aligned(rope_dims, ia)) return KVM_ERR_INVALID_ARG;
   if (!s.bound) bind_state(s, block, growth, rope_dims);
   const int C = s.C;
   const int64_t L = (int64_t)s.w * C;
@@ -663,6 +684,7 @@ KVM_API kvm_status_t kvm_decode_step(const void* q, const void* k, const void* v
   State& s = ks->s;
   if (!s.bound) return KVM_ERR_STATE_MISMATCH;
   if (((uintptr_t)q & 1) || ((uintptr_t)k & 1) || ((uintptr_t)v & 1) || ((uintptr_t)out & 1)) return KVM_ERR_INVALID_ARG;
+  if (s.fusedLn && ((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v) & 15) != 0)) return KVM_ERR_INVALID_ARG;
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   DeviceGuard guard(s.device);
   if (!guard.ok) return KVM_ERR_CUDA;

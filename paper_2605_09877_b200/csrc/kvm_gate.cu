@@ -317,6 +317,8 @@ kvm_status_t kvm_merge_gate(const void* x, const float* w_gate, int32_t batch, i
 // in place on the bf16 tensor that kvm_prefill / kvm_decode_step then take (they apply the RoPE).
 // HBM-bound: every element is read and written once.  d / 8 lanes share a row, 16 bytes each;
 // statistics in fp32 through shuffles inside the lane group (biased variance, as LN_s).
+#include "ln_rows.cuh"
+
 namespace kvm {
 
 constexpr int kLnRowsPerGroup = 4;   // rows per lane group, loaded up front: enough bytes in flight per SM for the HBM latency
@@ -354,34 +356,15 @@ __global__ void __launch_bounds__(256) head_layernorm_kernel(__nv_bfloat16* __re
       const float2 f = __bfloat1622float2(p2[i]);
       v[2 * i] = f.x; v[2 * i + 1] = f.y;
     }
-    float s = 0.f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) s += v[i];
-#pragma unroll
-    for (int o = LPR / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    const float mean = s * (1.f / D);
-    float q = 0.f;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) q += (v[i] - mean) * (v[i] - mean);
-#pragma unroll
-    for (int o = LPR / 2; o > 0; o >>= 1) q += __shfl_xor_sync(0xffffffffu, q, o);
-    const float rstd = rsqrtf(q * (1.f / D) + eps);
     if (h != h_cur) {   // consecutive rows nearly always belong to one head: its weights stay in registers
       h_cur = h;
-      if (weight) {
-        const float4 a = *reinterpret_cast<const float4*>(weight + (int64_t)h * D + sub * 8), b = *reinterpret_cast<const float4*>(weight + (int64_t)h * D + sub * 8 + 4);
-        wv[0] = a.x; wv[1] = a.y; wv[2] = a.z; wv[3] = a.w; wv[4] = b.x; wv[5] = b.y; wv[6] = b.z; wv[7] = b.w;
-      }
-      if (bias) {
-        const float4 a = *reinterpret_cast<const float4*>(bias + (int64_t)h * D + sub * 8), b = *reinterpret_cast<const float4*>(bias + (int64_t)h * D + sub * 8 + 4);
-        bv[0] = a.x; bv[1] = a.y; bv[2] = a.z; bv[3] = a.w; bv[4] = b.x; bv[5] = b.y; bv[6] = b.z; bv[7] = b.w;
-      }
+      ln_load_affine<D>(weight, bias, h, sub, wv, bv);
     }
+    ln_chunk8<D>(v, wv, bv, eps);
     uint32_t out[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const __nv_bfloat162 o2 = __floats2bfloat162_rn(fmaf((v[2 * i] - mean) * rstd, wv[2 * i], bv[2 * i]),
-                                                      fmaf((v[2 * i + 1] - mean) * rstd, wv[2 * i + 1], bv[2 * i + 1]));
+      const __nv_bfloat162 o2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);   // (already bf16 values: exact)
       out[i] = *reinterpret_cast<const uint32_t*>(&o2);
     }
     if (live) *reinterpret_cast<uint4*>(x + rr * D + sub * 8) = make_uint4(out[0], out[1], out[2], out[3]);

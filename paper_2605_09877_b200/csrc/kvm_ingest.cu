@@ -4,6 +4,7 @@
 // Staging layout per unit u (rows of d bf16):  [ history tokens hist_start .. pos0-1 | new tokens ]
 // so that the attention kernels address every window key of the call by (t - hist_start).
 #include "kvm_internal.h"
+#include "ln_rows.cuh"
 
 namespace kvm {
 
@@ -130,6 +131,22 @@ __global__ void ingest_q_kernel(__half* __restrict__ stQ, const __nv_bfloat16* _
 // ---- 16-byte versions (rows 16-byte aligned, rotary half a multiple of 8 channels): a thread
 //      converts eight consecutive channels of one token; same arithmetic as the scalar kernels ----
 
+// Rotation of eight consecutive rotary channels `out` with their partners `oth` (the same channels of the
+// other rotary half); c4 = the (cos, sin) pairs of these channels, two per float4.
+__device__ __forceinline__ void rope_rotate8(float (&out)[8], const float (&oth)[8], const float4* __restrict__ c4, bool lower) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float4 cc = c4[i];   // cos0 sin0 cos1 sin1
+    if (lower) {
+      out[2 * i] = out[2 * i] * cc.x - oth[2 * i] * cc.y;
+      out[2 * i + 1] = out[2 * i + 1] * cc.z - oth[2 * i + 1] * cc.w;
+    } else {
+      out[2 * i] = oth[2 * i] * cc.y + out[2 * i] * cc.x;
+      out[2 * i + 1] = oth[2 * i + 1] * cc.w + out[2 * i + 1] * cc.z;
+    }
+  }
+}
+
 // Eight bf16 channels starting at channel c8*8 of `row`, rotated when they lie in the rotary range.
 __device__ __forceinline__ void rope8(const __nv_bfloat16* __restrict__ row, int c8, int r,
                                       const float2* __restrict__ cs, float (&out)[8]) {
@@ -146,19 +163,13 @@ __device__ __forceinline__ void rope8(const __nv_bfloat16* __restrict__ row, int
   const bool lower = ch0 < half;
   const uint4 rawo = *reinterpret_cast<const uint4*>(row + (lower ? ch0 + half : ch0 - half));
   const __nv_bfloat162* po = reinterpret_cast<const __nv_bfloat162*>(&rawo);
-  const float4* c4 = reinterpret_cast<const float4*>(cs + (lower ? ch0 : ch0 - half));   // (cos, sin) pairs
+  float oth[8];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const float2 o = __bfloat1622float2(po[i]);
-    const float4 cc = c4[i];   // cos0 sin0 cos1 sin1
-    if (lower) {
-      out[2 * i] = out[2 * i] * cc.x - o.x * cc.y;
-      out[2 * i + 1] = out[2 * i + 1] * cc.z - o.y * cc.w;
-    } else {
-      out[2 * i] = o.x * cc.y + out[2 * i] * cc.x;
-      out[2 * i + 1] = o.y * cc.w + out[2 * i + 1] * cc.z;
-    }
+    oth[2 * i] = o.x; oth[2 * i + 1] = o.y;
   }
+  rope_rotate8(out, oth, reinterpret_cast<const float4*>(cs + (lower ? ch0 : ch0 - half)), lower);
 }
 
 __device__ __forceinline__ uint4 pack8_sat(const float (&x)[8], int& nsat) {
@@ -228,6 +239,113 @@ __global__ void __launch_bounds__(256) ingest_q_vec_kernel(__half* __restrict__ 
   if (nsat) atomicAdd(sat_counter, nsat);
 }
 
+// ---- LN_q / LN_k applied on the way in (fused front end): the d / 8 threads that convert a token's row
+//      first take its LayerNorm (ln_chunk8: the arithmetic of kvm_head_layernorm, result rounded to bf16
+//      as that kernel stores it), fetch the rotary partner chunk from the lane that holds it, rotate and
+//      stage.  Saves the read-modify-write pass of the stand-alone kernel over q and k. ----
+
+// this lane's eight channels of `row` after LN and partial RoPE (every lane of the warp must call)
+template <int D>
+__device__ __forceinline__ void ln_rope8(const __nv_bfloat16* __restrict__ row, int c8, int r, const float2* __restrict__ cs,
+                                         const float* __restrict__ lnw, const float* __restrict__ lnb, int h, float eps,
+                                         float (&out)[8]) {
+  constexpr int W8 = D / 8;
+  const uint4 raw = *reinterpret_cast<const uint4*>(row + c8 * 8);
+  const __nv_bfloat162* pv = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 f = __bfloat1622float2(pv[i]);
+    out[2 * i] = f.x; out[2 * i + 1] = f.y;
+  }
+  float w8[8], b8[8];
+  ln_load_affine<D>(lnw, lnb, h, c8, w8, b8);
+  ln_chunk8<D>(out, w8, b8, eps);
+  if (r == 0) return;   // (uniform)
+  const int half = r >> 1, ch0 = c8 * 8;
+  const bool inr = ch0 < r, lower = ch0 < half;
+  const int lane = threadIdx.x & 31;
+  const int src = (lane & ~(W8 - 1)) + (inr ? (lower ? c8 + half / 8 : c8 - half / 8) : c8);
+  float oth[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) oth[i] = __shfl_sync(0xffffffffu, out[i], src);
+  if (inr) rope_rotate8(out, oth, reinterpret_cast<const float4*>(cs + (lower ? ch0 : ch0 - half)), lower);
+}
+
+template <int D>
+__global__ void __launch_bounds__(256) ingest_kv_ln_kernel(
+    __half* __restrict__ stK, __half* __restrict__ stV, float* __restrict__ stG, __half* __restrict__ ringK,
+    __half* __restrict__ ringV, float* __restrict__ ringG, const __nv_bfloat16* __restrict__ k,
+    const __nv_bfloat16* __restrict__ v, const float* __restrict__ gate, const float2* __restrict__ ropeCS,
+    int64_t sk0, int64_t sk1, int64_t sk2, int64_t sv0, int64_t sv1, int64_t sv2, int64_t sg0, int64_t sg1,
+    int64_t sg2, int Hkv, int r, int64_t stRows, int64_t ringCap, int64_t ringLen, int64_t pos0, int64_t n,
+    int64_t nhist, int64_t tail_start, int32_t* __restrict__ sat_counter, const float* __restrict__ lnw,
+    const float* __restrict__ lnb, float eps) {
+  constexpr int d = D, w8 = D / 8, tpb = 256 / w8;
+  const int u = blockIdx.y;
+  const int b = u / Hkv, hk = u % Hkv;
+  const int64_t j0 = (int64_t)blockIdx.x * tpb + threadIdx.x / w8;
+  const int c8 = threadIdx.x % w8;
+  const bool live = j0 < n;                 // (rows past the end compute a copy of the last row: the shuffles need every lane)
+  const int64_t j = live ? j0 : n - 1;
+  float kx[8], vx[8];
+  ln_rope8<D>(k + b * sk0 + hk * sk1 + j * sk2, c8, r, ropeCS + j * (r >> 1), lnw, lnb, hk, eps, kx);
+  if (!live) return;
+  {
+    const uint4 raw = *reinterpret_cast<const uint4*>(v + b * sv0 + hk * sv1 + j * sv2 + c8 * 8);
+    const __nv_bfloat162* pv = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __bfloat1622float2(pv[i]);
+      vx[2 * i] = f.x; vx[2 * i + 1] = f.y;
+    }
+  }
+  int nsat = 0;
+  const uint4 kk = pack8_sat(kx, nsat), vv = pack8_sat(vx, nsat);
+  if (nsat) atomicAdd(sat_counter, nsat);
+  const float g = gate ? gate[b * sg0 + hk * sg1 + j * sg2] : 1.0f;
+  const int64_t row = (int64_t)u * stRows + nhist + j;
+  reinterpret_cast<uint4*>(stK + row * d)[c8] = kk;
+  reinterpret_cast<uint4*>(stV + row * d)[c8] = vv;
+  if (c8 == 0) stG[row] = g;
+  const int64_t t = pos0 + j;
+  if (t >= tail_start) {
+    const int64_t rrow = (int64_t)u * ringCap + t % ringLen;
+    reinterpret_cast<uint4*>(ringK + rrow * d)[c8] = kk;
+    reinterpret_cast<uint4*>(ringV + rrow * d)[c8] = vv;
+    if (c8 == 0) ringG[rrow] = g;
+  }
+}
+
+template <int D>
+__global__ void __launch_bounds__(256) ingest_q_ln_kernel(__half* __restrict__ stQ, const __nv_bfloat16* __restrict__ q,
+                                                          const float2* __restrict__ ropeCS, int64_t sq0, int64_t sq1,
+                                                          int64_t sq2, int Hq, int r, int64_t Tcall, int64_t n,
+                                                          int32_t* __restrict__ sat_counter, const float* __restrict__ lnw,
+                                                          const float* __restrict__ lnb, float eps) {
+  constexpr int w8 = D / 8, tpb = 256 / w8;
+  const int bh = blockIdx.y;
+  const int b = bh / Hq, h = bh % Hq;
+  const int64_t j0 = (int64_t)blockIdx.x * tpb + threadIdx.x / w8;
+  const int c8 = threadIdx.x % w8;
+  const bool live = j0 < n;
+  const int64_t j = live ? j0 : n - 1;
+  float qx[8];
+  ln_rope8<D>(q + b * sq0 + h * sq1 + j * sq2, c8, r, ropeCS + j * (r >> 1), lnw, lnb, h, eps, qx);
+  if (!live) return;
+  int nsat = 0;
+  reinterpret_cast<uint4*>(stQ + ((int64_t)bh * Tcall + j) * D)[c8] = pack8_sat(qx, nsat);
+  if (nsat) atomicAdd(sat_counter, nsat);
+}
+
+// Can this call take the 16-byte ingest kernels (which the fused front end requires)?
+bool ingest_rows_aligned(int r, const IngestArgs& a) {
+  auto al16 = [](const void* ptr, const int64_t* st3) {
+    return ((uintptr_t)ptr & 15) == 0 && (st3[0] & 7) == 0 && (st3[1] & 7) == 0 && (st3[2] & 7) == 0;
+  };
+  const bool rope_ok = r == 0 || ((r / 2) % 8) == 0;
+  return rope_ok && al16(a.k, a.sk) && al16(a.v, a.sv) && al16(a.q, a.sq);
+}
+
 int launch_ingest(State* st, const IngestArgs& a, cudaStream_t s) {
   int launches = 0;
   const int d = st->d, hw = d / 2;
@@ -251,6 +369,20 @@ int launch_ingest(State* st, const IngestArgs& a, cudaStream_t s) {
   };
   const bool rope_ok = st->r == 0 || ((st->r / 2) % 8) == 0;
   const int tpb = 256 / (d / 8);
+  if (st->fusedLn) {   // (the caller has checked ingest_rows_aligned)
+    dim3 gk((unsigned)((a.n + tpb - 1) / tpb), st->U), gq((unsigned)((a.n + tpb - 1) / tpb), st->B * st->Hq);
+#define KVM_LN_INGEST(DD)                                                                                                   \
+    ingest_kv_ln_kernel<DD><<<gk, 256, 0, s>>>(st->stK, st->stV, st->stG, st->ringK, st->ringV, st->ringG, a.k, a.v, a.gate, \
+                                               st->ropeCS, a.sk[0], a.sk[1], a.sk[2], a.sv[0], a.sv[1], a.sv[2], a.sg[0],   \
+                                               a.sg[1], a.sg[2], st->Hkv, st->r, st->stRows, (int64_t)st->w * st->Cmax,     \
+                                               st->ringLen, a.pos0, a.n, a.nhist, a.tail_start, st->status + 4, st->lnk_w,  \
+                                               st->lnk_b, st->qk_ln_eps);                                                   \
+    ingest_q_ln_kernel<DD><<<gq, 256, 0, s>>>(st->stQ, a.q, st->ropeCS, a.sq[0], a.sq[1], a.sq[2], st->Hq, st->r, st->Tcall, \
+                                              a.n, st->status + 4, st->lnq_w, st->lnq_b, st->qk_ln_eps)
+    if (d == 128) { KVM_LN_INGEST(128); } else { KVM_LN_INGEST(64); }
+#undef KVM_LN_INGEST
+    return launches + 2;
+  }
   if (rope_ok && al16(a.k, a.sk) && al16(a.v, a.sv)) {
     dim3 grid((unsigned)((a.n + tpb - 1) / tpb), st->U);
     ingest_kv_vec_kernel<<<grid, 256, 0, s>>>(st->stK, st->stV, st->stG, st->ringK, st->ringV, st->ringG, a.k,

@@ -43,6 +43,10 @@ struct State {
   // ---- parameters (device) ----
   float *ln_w, *ln_b;     // [Hkv, d]
   float *tau_s, *tau_b;   // [Hq]
+  // fused front end (KVM_FLAG_FUSED_QK_LN): LN_q / LN_k weights and biases, [Hq, d] / [Hkv, d] (NULL = 1 / 0)
+  bool fusedLn;
+  float qk_ln_eps;
+  float *lnq_w, *lnq_b, *lnk_w, *lnk_b;
   double* inv_freq;       // [r/2]: the bound rope_dims' slice of inv_freq_all
   double* inv_freq_all;   // base^(-2i/r), i < r/2, for every even r <= d, r's slice at offset (r/2)(r/2 - 1)/2
   bool assignDirty;       // recorded assignments of an earlier sequence are still in slotTok (cleared by the next prefill)
@@ -133,6 +137,7 @@ struct IngestArgs {
   int64_t pos0, n, hist_start, nhist, tail_start;
 };
 int launch_ingest(State* st, const IngestArgs& a, cudaStream_t s);
+bool ingest_rows_aligned(int r, const IngestArgs& a);   // rows 16-byte aligned, rotary half whole 8-channel chunks
 
 struct AttnArgs {
   int64_t q_row0;      // first query row in stQ (local token index)

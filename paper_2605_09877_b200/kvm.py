@@ -20,7 +20,7 @@ KVM_OK = 0
 STATUS = {0: "KVM_OK", 1: "KVM_ERR_INVALID_ARG", 2: "KVM_ERR_UNSUPPORTED", 3: "KVM_ERR_OOM",
           4: "KVM_ERR_CUDA", 5: "KVM_ERR_STATE_MISMATCH", 6: "KVM_ERR_CAPACITY", 7: "KVM_ERR_TIMEOUT"}
 GROWTH_FIXED, GROWTH_SQRT, GROWTH_UNBOUNDED, GROWTH_POWER, GROWTH_SATURATING = 0, 1, 2, 3, 4
-FLAG_NO_RADIUS, FLAG_RECORD_ASSIGN, FLAG_SIMT_ATTENTION, FLAG_SIMT_ROUTING, FLAG_MIN_KEY_SLOTS, FLAG_SERIAL_FOLDS = 1, 2, 4, 8, 16, 32
+FLAG_NO_RADIUS, FLAG_RECORD_ASSIGN, FLAG_SIMT_ATTENTION, FLAG_SIMT_ROUTING, FLAG_MIN_KEY_SLOTS, FLAG_SERIAL_FOLDS, FLAG_FUSED_QK_LN = 1, 2, 4, 8, 16, 32, 64
 
 EXPORTS = ["kvm_plan_capacity", "kvm_state_create", "kvm_prefill", "kvm_decode_step", "kvm_prefill_host",
            "kvm_decode_step_host", "kvm_state_free", "kvm_state_info", "kvm_state_check", "kvm_state_export",
@@ -58,6 +58,9 @@ class Config(C.Structure):
         ("tau_state", C.POINTER(C.c_float)), ("tau_bswa", C.POINTER(C.c_float)),
         ("max_block", C.c_int32), ("max_state_slots", C.c_int64), ("max_call_tokens", C.c_int64),
         ("max_seq_len", C.c_int64), ("device", C.c_int32), ("flags", C.c_uint32),
+        ("qk_ln_eps", C.c_float),
+        ("ln_q_weight", C.POINTER(C.c_float)), ("ln_q_bias", C.POINTER(C.c_float)),
+        ("ln_k_weight", C.POINTER(C.c_float)), ("ln_k_bias", C.POINTER(C.c_float)),
     ]
 
 
@@ -218,12 +221,20 @@ class LayerConfig:
 class KVMState:
     """Owns one kvm_state_t.  Methods map 1:1 to the C entry points of the same name."""
 
-    def __init__(self, cfg: LayerConfig, ln_weight=None, ln_bias=None, tau_state=None, tau_bswa=None):
+    def __init__(self, cfg: LayerConfig, ln_weight=None, ln_bias=None, tau_state=None, tau_bswa=None, qk_ln=None):
+        """qk_ln: dict(eps, q_weight, q_bias, k_weight, k_bias) turns the fused front end on (KVM_FLAG_FUSED_QK_LN)."""
         self.cfg = cfg
         keep = [_fp(ln_weight), _fp(ln_bias), _fp(tau_state), _fp(tau_bswa)]
+        flags, eps = cfg.flags, 0.0
+        ln4 = [(None, None)] * 4
+        if qk_ln is not None:
+            flags |= FLAG_FUSED_QK_LN
+            eps = float(qk_ln.get("eps", 1e-5))
+            ln4 = [_fp(qk_ln.get(n)) for n in ("q_weight", "q_bias", "k_weight", "k_bias")]
         c = Config(cfg.batch, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.n_bswa_chunks, cfg.sink_len,
                    cfg.rope_base, cfg.ln_eps, cfg.norm_eps, keep[0][1], keep[1][1], keep[2][1], keep[3][1],
-                   cfg.max_block, cfg.max_state_slots, cfg.max_call_tokens, cfg.max_seq_len, cfg.device, cfg.flags)
+                   cfg.max_block, cfg.max_state_slots, cfg.max_call_tokens, cfg.max_seq_len, cfg.device, flags,
+                   eps, ln4[0][1], ln4[1][1], ln4[2][1], ln4[3][1])
         h = C.c_void_p()
         rc = lib.kvm_state_create(C.byref(c), C.byref(h))
         if rc != KVM_OK:
