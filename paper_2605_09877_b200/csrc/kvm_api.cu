@@ -378,7 +378,9 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   }
   A(s.xScore, U * Cm); A(s.xBest, U * Cm); A(s.xArg, U * Cm); A(s.xCount, U);
   if (rc == KVM_OK && cudaMemset(s.xCount, 0, U * sizeof(int32_t)) != cudaSuccess) rc = KVM_ERR_CUDA;
-  A(s.candV, U * (size_t)(2 * s.nsplitRoute) * Cm * kTopK); A(s.candI, U * (size_t)(2 * s.nsplitRoute) * Cm * kTopK);
+  A(s.candV, U * (size_t)s.nsplitRoute * Cm * kTopK); A(s.candI, U * (size_t)s.nsplitRoute * Cm * kTopK);
+  A(s.chunkMeta, U * (size_t)s.nsplitRoute * Cm * kChunkCap); A(s.chunkMax, U * (size_t)s.nsplitRoute * Cm * kChunkCap);
+  if (rc == KVM_OK) rc = dev_alloc(ks, &s.chunkVal, U * (size_t)s.nsplitRoute * Cm * kChunkCap * 32, false);
   A(s.decPart, (size_t)s.B * s.Hq * s.nsplitDec * (d + 2)); A(s.decQ, (size_t)s.B * s.Hq * d);
   // (tiles x splits: up to kAttnSplitTiles x kAttnMaxSplits, or 2 kAttnSplitTiles tiles of two splits)
   A(s.attnPart, (size_t)kAttnSplitTiles * kAttnMaxSplits * (d + 2) * 128); A(s.attnCnt, (size_t)2 * kAttnSplitTiles);

@@ -172,11 +172,25 @@ __device__ __forceinline__ void rope8(const __nv_bfloat16* __restrict__ row, int
   rope_rotate8(out, oth, reinterpret_cast<const float4*>(cs + (lower ? ch0 : ch0 - half)), lower);
 }
 
+// Eight values -> eight fp16, clamped; nsat counts the values that did not fit.  A clamped value reads
+// +-65504 afterwards, which no bf16 input converts to exactly (its neighbours are 65280 and 65536), so the
+// packed result is tested first - one SIMD compare per pair - and the values are only looked at one by one
+// when it shows a hit.
 __device__ __forceinline__ uint4 pack8_sat(const float (&x)[8], int& nsat) {
   uint4 o;
-  __half2 h0 = to_half2_sat(x[0], x[1], nsat), h1 = to_half2_sat(x[2], x[3], nsat), h2 = to_half2_sat(x[4], x[5], nsat), h3 = to_half2_sat(x[6], x[7], nsat);
-  o.x = *reinterpret_cast<uint32_t*>(&h0); o.y = *reinterpret_cast<uint32_t*>(&h1);
-  o.z = *reinterpret_cast<uint32_t*>(&h2); o.w = *reinterpret_cast<uint32_t*>(&h3);
+  uint32_t w[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const __half2 h = __floats2half2_rn(fminf(fmaxf(x[2 * i], -65504.f), 65504.f), fminf(fmaxf(x[2 * i + 1], -65504.f), 65504.f));
+    w[i] = *reinterpret_cast<const uint32_t*>(&h);
+  }
+  const uint32_t any = (__vcmpeq2(w[0] & 0x7fff7fffu, 0x7bff7bffu) | __vcmpeq2(w[1] & 0x7fff7fffu, 0x7bff7bffu)) |
+                       (__vcmpeq2(w[2] & 0x7fff7fffu, 0x7bff7bffu) | __vcmpeq2(w[3] & 0x7fff7fffu, 0x7bff7bffu));
+  if (any) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) nsat += !(fabsf(x[i]) <= 65504.f) ? 1 : 0;
+  }
+  o.x = w[0]; o.y = w[1]; o.z = w[2]; o.w = w[3];
   return o;
 }
 

@@ -10,7 +10,8 @@
 namespace kvm {
 
 constexpr int kMaxBlock = 256;      // largest block C (one thread per overflow token in the fold)
-constexpr int kTopK = 8;            // routing filter keeps the K best approximate similarities per split
+constexpr int kTopK = 8;            // routing filter keeps at most K candidate rows per (token, row split)
+constexpr int kChunkCap = 16;       // 32-row chunks of approximate similarities the routing filter can record per (token, row split)
 constexpr int kMaxSplits = 32;      // routing filter / decode split count upper bound
 constexpr int kAttnSplitTiles = 37; // launches with at most this many (batch, head, query tile) CTAs - a quarter of the GPU - are split along the keys
 constexpr int kAttnMaxSplits = 8;
@@ -99,8 +100,13 @@ struct State {
   double *xScore, *xBest;        // [U, Cmax] hand-over between the CTAs of the decide kernel
   int32_t *xArg, *xCount;        // [U, Cmax]; [U]
   int nsplitRoute;               // splits the routing filter may use
-  float* candV;                  // [U, nsplitRoute, Cmax, kTopK]
-  int32_t* candI;
+  float* candV;                  // [U, nsplitRoute, Cmax, kTopK]  routing filter output: (split maximum, candidate count, ...)
+  int32_t* candI;                // [U, nsplitRoute, Cmax, kTopK]  candidate rows
+  // scratch of the routing filter's threads: the 32-row chunks of products a token recorded on its way through
+  // the split (maximum, first row and mask of valid rows, the 32 products)
+  float* chunkMax;               // [U, nsplitRoute, Cmax, kChunkCap]
+  int2* chunkMeta;               // [U, nsplitRoute, Cmax, kChunkCap]
+  float* chunkVal;               // [U, nsplitRoute, Cmax, kChunkCap, 32]
   // ---- split-KV attention scratch (device) ----
   float* attnPart;               // [kAttnSplitTiles][kAttnMaxSplits][d + 2][128]
   int32_t* attnCnt;              // [2 kAttnSplitTiles] tickets

@@ -2,22 +2,27 @@
 // the overflow block's memory keys (fp16, up to 256 tokens = two 128-row M tiles) and a split of
 // the state's readout keys, reduced on the fly to the rows whose similarity lies within the
 // rounding bound of the row maximum (Section 3.2 "Append" score and "Merge" arg max; the exact
-// decision is taken later in fp64 on these candidates only).  The split is streamed twice:
-// pass 1 keeps the running maximum per token (three-input maxima: half an instruction per
-// element), pass 2 repeats the products, takes the maximum of every 32-column chunk the same way
-// and looks element by element only at the chunks in which some token of the warp has a value above
-// (maximum - bound).  The tensor work doubles but the epilogue, which is the bottleneck of a
-// 128 x 128 x d tile, stays near one instruction per element instead of a sorted insertion.
+// decision is taken later in fp64 on these candidates only).  The split is streamed ONCE: per
+// 128-row tile a thread (one token) takes the maxima of its four 32-column chunks (three-input
+// maxima: half an instruction per element), raises its running maximum, and records every chunk
+// whose maximum reaches (running maximum - bound): the chunk's 32 products go to the token's list in
+// global memory as they are.  The running maximum only grows, so the recorded chunks are a superset
+// of the chunks that hold a row within the bound of the final maximum; after its last tile the thread
+// goes back over its own few records (their maxima first: usually one chunk survives) and lists the
+// rows above (final maximum - bound).  A token meets a new running maximum about ln(tiles) times,
+// and a new maximum nearly always makes the earlier records obsolete, so the list is restarted in
+// place and stays a record or two (128 bytes each) long, while the state is read, and multiplied,
+// once.
 //
 //   warp 0      TMA producer: the Kbar tiles once, then 128-row tiles of K_hat in a 3-stage ring
 //   warps 1, 10 MMA issuers, one thread per M tile: per key tile one 128x128x(d) product into a
 //               double-buffered TMEM accumulator (tcgen05.mma kind::f16)
-//   warps 2-9   epilogue: one thread per token row; tcgen05.ld of its 128 similarities, running
-//               maximum (pass 1) / list of at most kTopK candidate rows (pass 2) in registers.
-//               Pass 2 walks the tiles in the opposite direction.
+//   warps 2-9   epilogue: one thread per token row; tcgen05.ld of its 128 similarities, chunk maxima,
+//               running maximum, recorded chunks straight to global memory
 // Output per (unit, split, token): candI[0..kTopK) candidate rows in the order found (-1 = none),
 // candV[0] = the split's maximum over rows >= S, candV[1] = number of candidates found (more than
-// kTopK = the list overflowed and the decision kernel scans all rows for that token).
+// kTopK = the list overflowed - or more chunks were met than could be recorded - and the decision
+// kernel scans all rows for that token).  chunkMax / chunkMeta / chunkVal are the threads' scratch.
 // All waits are bounded (error word + normal teardown on expiry).
 #include "kvm_internal.h"
 #include "tc_common.cuh"
@@ -27,6 +32,9 @@ namespace kvm {
 struct RouteTcParams {
   float* candV;
   int32_t* candI;
+  float* chunkMax;
+  int2* chunkMeta;
+  float* chunkVal;
   int32_t* status;
   const float* kbarNorm;   // [U, Cmax] upper bound of ||kbar_j||
   int a_unit0;             // first unit of this block's slot in the memory-key tensor map
@@ -78,7 +86,7 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
   const int64_t i0 = gram ? 0 : (int64_t)split * per;
   const int64_t i1 = gram ? (int64_t)p.C : min(p.m, i0 + per);
   const int ntiles = i1 > i0 ? (int)((i1 - i0 + 127) / 128) : 0;
-  const int nsteps = gram ? ntiles : 2 * ntiles;   // a split's tiles are visited in pass 1 and again in pass 2
+  const int nsteps = ntiles;
 
   if (tid == 0) {
     tc::mbar_init(&bars[RB_AFULL], 1);
@@ -117,7 +125,7 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
       asm volatile("griddepcontrol.wait;" ::: "memory");
       for (int j = 0; j < nsteps; ++j) {
         const int s = j % Cfg::NS;
-        const int jt = j >= ntiles ? 2 * ntiles - 1 - j : j;   // pass 2 walks back: its first tiles are the ones pass 1 read last (L2)
+        const int jt = j;
         if (*abort_flag) break;
         if (j >= Cfg::NS && !tc::mbar_wait(&bars[RB_BFREE + s], ((j / Cfg::NS) - 1) & 1)) {
           atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; break;
@@ -161,27 +169,23 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
       const int quarter = warp & 3;
       const int tok = mt * 128 + quarter * 32 + lane;
       const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
-      int ci[kTopK];
-#pragma unroll
-      for (int k = 0; k < kTopK; ++k) ci[k] = -1;
-      int ncand = 0;
-      float mx = -INFINITY;        // pass 1: running maximum over rows >= S of this split
-      float cut = INFINITY;        // pass 2: collect rows whose similarity is >= cut
-      const float thr = (tok < p.C) ? p.thr_coeff * p.kbarNorm[(int64_t)u * p.Cmax + tok] + 1e-5f : 0.f;
+      int nrec = 0;
+      int sink_rec = 0;            // 1 once the record of the chunk that holds the sink rows sits in slot 0
+      float mx = -INFINITY;        // running maximum over rows >= S of this split
+      const bool live = tok < p.C;   // (rows of the M tile past the block record nothing)
+      const float thr = live ? p.thr_coeff * p.kbarNorm[(int64_t)u * p.Cmax + tok] + 1e-5f : 0.f;
+      const int64_t o = (((int64_t)u * p.nsplit + split) * p.Cmax + (live ? tok : 0)) * kChunkCap;
       for (int j = 0; j < nsteps; ++j) {
         const int buf = j & 1;
-        const bool pass2 = j >= ntiles;
-        const int jt = pass2 ? 2 * ntiles - 1 - j : j;
-        if (j == ntiles) cut = (tok < p.C) ? mx - thr : INFINITY;   // (rows of the M tile past the block collect nothing)
         if (!tc::mbar_wait(&bars[RB_SFULL + buf], (j >> 1) & 1)) {
           atomicExch(p.status, (int)KVM_ERR_TIMEOUT); *abort_flag = 1; break;
         }
         tc::tc_fence_after();
         const uint32_t ts = tmem + lane_base + buf * 256 + mt * 128;
-        const int row0 = (int)(i0 + (int64_t)jt * 128);
+        const int row0 = (int)(i0 + (int64_t)j * 128);
         const int nvalid = (int)min((int64_t)128, i1 - row0);
-        // pass 1 ignores the sink rows (< S) and the rows past the end of the split; pass 2 only the latter
-        const int lo = pass2 ? 0 : max(0, p.S - row0);
+        // the maximum ignores the sink rows (< S) and the rows past the end of the split; recorded chunks only the latter
+        const int lo = max(0, p.S - row0);
         const bool plain = nvalid == 128 && lo == 0;
         // all 128 columns of the row go to registers in one round trip; the accumulator is handed
         // back before they are looked at
@@ -192,10 +196,10 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
         tc::tc_fence_before();
         __syncwarp();
         if (lane == 0) tc::mbar_arrive(&bars[RB_ACCFREE + buf]);
+        if (gram) {   // row `tok` of gramT: 32 consecutive tokens j = row0 + c4*32 .. (rows past C are never read)
 #pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4) {
-          uint32_t (&r)[32] = rr[c4];
-          if (gram) {   // row `tok` of gramT: 32 consecutive tokens j = row0 + c4*32 .. (rows past C are never read)
+          for (int c4 = 0; c4 < 4; ++c4) {
+            uint32_t (&r)[32] = rr[c4];
             if (tok < p.C) {
               float* dst = p.gramT + ((int64_t)a_unit * p.Cmax + tok) * p.Cmax + row0 + c4 * 32;
               if (row0 + c4 * 32 + 32 <= p.Cmax) {
@@ -207,16 +211,15 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
                   if (row0 + c4 * 32 + i < p.Cmax) dst[i] = __uint_as_float(r[i]);
               }
             }
-            continue;
           }
-          uint32_t vm = 0xffffffffu;   // columns of this chunk that count
-          if (!plain) {
-            const int a = min(32, max(0, lo - c4 * 32)), b = min(32, max(0, nvalid - c4 * 32));
-            vm = (b <= a) ? 0u : ((b == 32 ? 0xffffffffu : ((1u << b) - 1u)) & ~((1u << a) - 1u));
-          }
-          // maximum of the chunk's columns that count: four chains of three-input maxima (half an
-          // instruction per element)
-          float cmax;
+          continue;
+        }
+        // chunk maxima: cm over the rows that count for the maximum, ca over all valid rows
+        float cm[4], ca[4];
+        uint32_t va[4];   // valid rows of each chunk (bit i = row i of the chunk)
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) {
+          uint32_t (&r)[32] = rr[c4];
           if (plain) {
             float t4[4] = {__uint_as_float(r[0]), __uint_as_float(r[1]), __uint_as_float(r[2]), __uint_as_float(r[3])};
 #pragma unroll
@@ -226,45 +229,91 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
             }
 #pragma unroll
             for (int k = 0; k < 4; ++k) t4[k] = fmaxf(t4[k], __uint_as_float(r[28 + k]));
-            cmax = fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3]));
+            cm[c4] = fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3]));
+            ca[c4] = cm[c4];
+            va[c4] = 0xffffffffu;
           } else {
-            float cm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            const int a = min(32, max(0, lo - c4 * 32)), b = min(32, max(0, nvalid - c4 * 32));
+            const uint32_t vall = b == 32 ? 0xffffffffu : ((1u << b) - 1u);
+            const uint32_t vns = (b <= a) ? 0u : (vall & ~((1u << a) - 1u));
+            float m1 = -INFINITY, m2 = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) cm[i & 3] = fmaxf(cm[i & 3], ((vm >> i) & 1u) ? __uint_as_float(r[i]) : -INFINITY);
-            cmax = fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3]));
-          }
-          if (!pass2) {
-            mx = fmaxf(mx, cmax);
-          } else {
-            // a chunk is looked at element by element only when some token of the warp has a candidate
-            // in it (about one chunk in four: a token has about one candidate among all rows of the split)
-            if (!__any_sync(0xffffffffu, cmax >= cut)) continue;
-            uint32_t h4[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-            for (int i = 0; i < 32; ++i) h4[i & 3] |= (__uint_as_float(r[i]) >= cut) ? (1u << i) : 0u;
-            uint32_t hit = (h4[0] | h4[1]) | (h4[2] | h4[3]);
-            hit &= vm;
-            while (hit) {   // rare per lane: about one candidate per token and split
-              const int bit = __ffs(hit) - 1;
-              hit &= hit - 1;
-              const int idx = row0 + c4 * 32 + bit;
-              if (ncand < kTopK) {
-#pragma unroll
-                for (int k = 0; k < kTopK; ++k)
-                  if (k == ncand) ci[k] = idx;
-              }
-              ++ncand;
+            for (int i = 0; i < 32; ++i) {
+              const float v = __uint_as_float(r[i]);
+              m1 = fmaxf(m1, ((vns >> i) & 1u) ? v : -INFINITY);
+              m2 = fmaxf(m2, ((vall >> i) & 1u) ? v : -INFINITY);
             }
+            cm[c4] = m1; ca[c4] = m2; va[c4] = vall;
+          }
+        }
+        const float tmax = fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3]));
+        // a maximum that beats the old one by more than the bound makes every earlier record obsolete (all
+        // their rows lie below the new line), except the one that may hold sink rows, which the maximum
+        // ignores: the list starts over, in place - it stays a record or two long and warm in L2
+        if (tmax > mx + thr) nrec = min(nrec, sink_rec);
+        mx = fmaxf(mx, tmax);
+        const float cut = mx - thr;
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) {
+          if (live && ca[c4] >= cut) {   // record the chunk: 128 bytes of products, as they are
+            if (nrec < kChunkCap) {
+              uint32_t (&r)[32] = rr[c4];
+              uint4* dst = reinterpret_cast<uint4*>(p.chunkVal + (o + nrec) * 32);
+#pragma unroll
+              for (int i = 0; i < 8; ++i) dst[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+              p.chunkMeta[o + nrec] = make_int2(row0 + c4 * 32, (int)va[c4]);
+              p.chunkMax[o + nrec] = ca[c4];
+            }
+            if (row0 + c4 * 32 < p.S) sink_rec = (nrec == 0) ? 1 : sink_rec;   // (the first chunk of the state; met first)
+            ++nrec;
           }
         }
       }
-      if (tok < p.C && !gram) {
-        const int64_t o = (((int64_t)u * p.nsplit + split) * p.Cmax + tok) * kTopK;
+      if (live && !gram) {
+        // back over this thread's own records (written above, read here by the same thread): the chunks
+        // whose maximum reaches the final line, and in them the valid rows that do
+        static_assert(kChunkCap == 16, "chunk maxima are read as four float4");
+        int ci[kTopK];
 #pragma unroll
-        for (int k = 0; k < kTopK; ++k) p.candI[o + k] = ci[k];
+        for (int k = 0; k < kTopK; ++k) ci[k] = -1;
+        int ncand = 0;
+        const float cut = mx - thr;
+        const float4* cm4 = reinterpret_cast<const float4*>(p.chunkMax + o);
+        const float4 c0 = cm4[0], c1 = cm4[1], c2 = cm4[2], c3 = cm4[3];
+        const float cmv[16] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w, c2.x, c2.y, c2.z, c2.w, c3.x, c3.y, c3.z, c3.w};
+        uint32_t kept = 0;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) kept |= (k < nrec && cmv[k] >= cut) ? (1u << k) : 0u;
+        while (kept) {
+          const int k = __ffs(kept) - 1;
+          kept &= kept - 1;
+          const int2 mt = p.chunkMeta[o + k];
+          const float4* v4 = reinterpret_cast<const float4*>(p.chunkVal + (o + k) * 32);
+          uint32_t hit = 0;
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const float4 v = v4[q];
+            hit |= ((v.x >= cut ? 1u : 0u) | (v.y >= cut ? 2u : 0u) | (v.z >= cut ? 4u : 0u) | (v.w >= cut ? 8u : 0u)) << (4 * q);
+          }
+          hit &= (uint32_t)mt.y;
+          while (hit) {
+            const int bit = __ffs(hit) - 1;
+            hit &= hit - 1;
+            if (ncand < kTopK) {
+#pragma unroll
+              for (int kk = 0; kk < kTopK; ++kk)
+                if (kk == ncand) ci[kk] = mt.x + bit;
+            }
+            ++ncand;
+          }
+        }
+        if (nrec > kChunkCap) ncand = kTopK + 1;   // records were lost: let the decision kernel scan every row
+        const int64_t oc = (((int64_t)u * p.nsplit + split) * p.Cmax + tok) * kTopK;
+#pragma unroll
+        for (int k = 0; k < kTopK; ++k) p.candI[oc + k] = ci[k];
         // values are not kept: the decision kernel needs the split's maximum and the candidate count
-        p.candV[o] = mx;
-        p.candV[o + 1] = (float)ncand;
+        p.candV[oc] = mx;
+        p.candV[oc + 1] = (float)ncand;
       }
     }
   }
@@ -278,7 +327,7 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
 
 int launch_route_filter_tc(State* st, int64_t m, int nsplit, int slot, bool early_start, cudaStream_t s) {
   RouteTcParams p;
-  p.candV = st->candV; p.candI = st->candI; p.status = st->status; p.m = m;
+  p.candV = st->candV; p.candI = st->candI; p.chunkMax = st->chunkMax; p.chunkMeta = st->chunkMeta; p.chunkVal = st->chunkVal; p.status = st->status; p.m = m;
   p.C = st->C; p.Cmax = st->Cmax; p.nsplit = nsplit; p.S = st->S;
   p.kbarNorm = st->kbarNorm + (int64_t)slot * st->U * st->Cmax; p.thr_coeff = route_thr_coeff(st);
   p.a_unit0 = slot * st->U; p.gramT = st->gramT; p.gram_mode = 0; p.U = st->U;
@@ -302,7 +351,7 @@ int launch_route_filter_tc(State* st, int64_t m, int nsplit, int slot, bool earl
 // New-row filter of nblk blocks whose memory keys sit in slots slot0 .. slot0 + nblk - 1.
 int launch_gram_tc(State* st, int slot0, int nblk, cudaStream_t s) {
   RouteTcParams p;
-  p.candV = st->candV; p.candI = st->candI; p.status = st->status; p.m = 0;
+  p.candV = st->candV; p.candI = st->candI; p.chunkMax = st->chunkMax; p.chunkMeta = st->chunkMeta; p.chunkVal = st->chunkVal; p.status = st->status; p.m = 0;
   p.C = st->C; p.Cmax = st->Cmax; p.nsplit = 1; p.S = st->S;
   p.kbarNorm = st->kbarNorm; p.thr_coeff = 0.f;
   p.a_unit0 = slot0 * st->U; p.gramT = st->gramT; p.gram_mode = 1; p.U = st->U;
