@@ -181,6 +181,7 @@ void bind_state(State& s, int32_t block, const kvm_growth_t& growth, int32_t r) 
   s.C = block; s.r = r; s.growth = growth; s.ringLen = (int64_t)s.w * block;
   const int k = r / 2;
   s.inv_freq = s.inv_freq_all + (int64_t)k * (k - 1) / 2;
+  s.recomputeK = s.serial && (int64_t)block * s.U >= 8192;   // (the threshold of the four-rows-per-warp apply kernel)
   s.bound = true;
 }
 
@@ -368,7 +369,7 @@ KVM_API kvm_status_t kvm_state_create(const kvm_config_t* cfg, kvm_state_t** out
   }
   {
     const size_t G = (size_t)s.kbSlots;
-    A(s.kbar64, G * U * Cm * d); A(s.kbarH, G * U * (size_t)s.CbarRows * d); A(s.kbarNorm, G * U * Cm);
+    A(s.kbarStat, G * U * Cm); A(s.kbar64, G * U * Cm * d); A(s.kbarH, G * U * (size_t)s.CbarRows * d); A(s.kbarNorm, G * U * Cm);
     A(s.kbarHatStat, G * U * Cm); A(s.kbarHatH, G * U * (size_t)s.CbarRows * d);
     A(s.gramT, G * U * Cm * Cm);
   }
@@ -613,7 +614,7 @@ KVM_API kvm_status_t kvm_prefill(const void* q, const void* k, const void* v, kv
     int64_t m_sim = s.m;
     for (int i = 0; i < f0 + nf; ++i) {
       // (m_sim restarts from the current rows: folds before f0 that are already launched moved s.m)
-      if (i >= n_done_folds) { if (i >= f0 && fold_na[i] > kGramOnTheFly && fold_na[i] < C && m_sim > 0) want_gram = true; m_sim += fold_na[i]; }
+      if (i >= n_done_folds) { if (i >= f0 && fold_na[i] > gram_from(&s) && fold_na[i] < C && m_sim > 0) want_gram = true; m_sim += fold_na[i]; }
     }
     if (ovk && batch_done_rec[h]) ev_ok = ev_ok && cudaStreamWaitEvent(kstream, s.evBatchDone[h], 0) == cudaSuccess;
     const int64_t bf = (cf0 + f0 + 1) * C - L;   // first token of the first block of the batch
@@ -714,7 +715,7 @@ KVM_API kvm_status_t kvm_decode_step(const void* q, const void* k, const void* v
     fa.b = b; fa.m = s.m; fa.first = (s.m == 0); fa.n_append = n_a; fa.slot = 0; fa.before_apply = nullptr;
     fa.early_start = false;   // the memory-key kernel runs right before the filter on this stream
     s.launches += launch_prev_copy(&s, stream);
-    s.launches += launch_kbar(&s, fa.ok, fa.unit_stride, 1, 0, n_a > kGramOnTheFly && n_a < C && s.m > 0, stream);
+    s.launches += launch_kbar(&s, fa.ok, fa.unit_stride, 1, 0, n_a > gram_from(&s) && n_a < C && s.m > 0, stream);
     s.launches += launch_fold(&s, fa, stream);
     s.m += n_a;
     s.nfolds += 1;

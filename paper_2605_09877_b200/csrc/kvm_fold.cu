@@ -45,6 +45,49 @@ __device__ __forceinline__ void row_stats(const double (&x)[CH], int D, double e
   rstd = 1.0 / sqrt(warp_sum_d(q) / D + eps);
 }
 
+// The memory key kbar_j = LN_s(zero_r(k_j)) (Eq. 1) in fp64 is two thirds of everything the memory-key kernel
+// writes, and the decision and application kernels read it back row by row.  States with enough units to
+// fill the GPU - where the folds are bound by memory traffic, not by their chain of dependent launches - do
+// not keep it (RK = true): every kernel that needs kbar_j recomputes it from the fp16 key and the token's
+// (mean, rstd), with the roundings pinned so that all of them get the same bits.
+__device__ __forceinline__ double ln_affine(double v, double mean, double rstd, double w, double b) {
+  return __dadd_rn(__dmul_rn(w, __dmul_rn(__dsub_rn(v, mean), rstd)), b);
+}
+template <int D, bool RK>
+struct KbarRows {            // the memory keys of one unit's folded block
+  const double* k64;         // !RK: [C][D] fp64
+  const __half* k16;         // RK: the block's keys [C][D] fp16 ...
+  const double2* stat;       //     ... and (mean, rstd) of zero_r(k_j) per token
+  int r;                     //     leading channels that zero_r clears
+  // channel x of kbar_j; g, b = LN_s weight and bias of that channel
+  __device__ __forceinline__ double at(int j, int x, double g, double b) const {
+    if (!RK) return k64[(int64_t)j * D + x];
+    const double2 st = stat[j];
+    const double v = x < r ? 0.0 : (double)__half2float(k16[(int64_t)j * D + x]);
+    return ln_affine(v, st.x, st.y, g, b);
+  }
+};
+
+// channels x .. x + 3 of kbar_j (x a multiple of 4) for the kernels that hold rows as runs of four channels
+template <int D, bool RK>
+__device__ __forceinline__ void kbar_run4(const KbarRows<D, RK>& kr, int j, int x, const float* __restrict__ ln_w_h,
+                                          const float* __restrict__ ln_b_h, double (&out)[4]) {
+  if (!RK) {
+    const double* kb = kr.k64 + (int64_t)j * D + x;
+    const double2 k01 = *reinterpret_cast<const double2*>(kb), k23 = *reinterpret_cast<const double2*>(kb + 2);
+    out[0] = k01.x; out[1] = k01.y; out[2] = k23.x; out[3] = k23.y;
+  } else {
+    alignas(8) __half hv[4];
+    *reinterpret_cast<uint2*>(hv) = *reinterpret_cast<const uint2*>(kr.k16 + (int64_t)j * D + x);
+    const float4 w4 = *reinterpret_cast<const float4*>(ln_w_h + x), b4 = *reinterpret_cast<const float4*>(ln_b_h + x);
+    const float wv[4] = {w4.x, w4.y, w4.z, w4.w}, bv[4] = {b4.x, b4.y, b4.z, b4.w};
+    const double2 st = kr.stat[j];
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      out[e] = ln_affine(x + e < kr.r ? 0.0 : (double)__half2float(hv[e]), st.x, st.y, (double)wv[e], (double)bv[e]);
+  }
+}
+
 // ------------------------------------------------------------------------------------------
 // 1. memory keys (one warp per overflow token)
 
@@ -62,13 +105,13 @@ __device__ __forceinline__ double group8_sum_d(double v) {
   return v;
 }
 
-template <int D>
+template <int D, bool RK>
 __global__ void __launch_bounds__(256, 2) kbar_kernel(const __half* __restrict__ ok, int64_t unit_stride,
                                                       const float* __restrict__ ln_w, const float* __restrict__ ln_b,
                                                       double* __restrict__ kbar64, __half* __restrict__ kbarH,
                                                       float* __restrict__ kbarNorm, double2* __restrict__ kbarHatStat,
                                                       __half* __restrict__ kbarHatH, int C, int Cmax, int CbarRows, int U, int Hkv, int r,
-                                                      double ln_eps, int write_hat) {
+                                                      double ln_eps, int write_hat, double2* __restrict__ kbarStat) {
   constexpr int NI = D / 32;          // runs of four channels per lane
   constexpr int NC = 4 * NI;          // channels per lane
   constexpr double inv_d = 1.0 / D;   // D is a power of two: the multiplication is the division, exactly
@@ -108,14 +151,17 @@ __global__ void __launch_bounds__(256, 2) kbar_kernel(const __half* __restrict__
     alignas(8) __half kh[4];
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
-      const double t = (double)wv[e] * ((val[4 * i + e] - mean) * rstd) + (double)bv[e];
+      const double t = RK ? ln_affine(val[4 * i + e], mean, rstd, (double)wv[e], (double)bv[e])
+                          : (double)wv[e] * ((val[4 * i + e] - mean) * rstd) + (double)bv[e];
       kb[4 * i + e] = t;
       kh[e] = __float2half_rn((float)t);
       n2 += t * t;
     }
     if (live) {
-      reinterpret_cast<double2*>(kbar64 + o + x)[0] = make_double2(kb[4 * i], kb[4 * i + 1]);
-      reinterpret_cast<double2*>(kbar64 + o + x)[1] = make_double2(kb[4 * i + 2], kb[4 * i + 3]);
+      if (!RK) {
+        reinterpret_cast<double2*>(kbar64 + o + x)[0] = make_double2(kb[4 * i], kb[4 * i + 1]);
+        reinterpret_cast<double2*>(kbar64 + o + x)[1] = make_double2(kb[4 * i + 2], kb[4 * i + 3]);
+      }
       *reinterpret_cast<uint2*>(kbarH + oh + x) = *reinterpret_cast<const uint2*>(kh);
     }
   }
@@ -145,6 +191,7 @@ __global__ void __launch_bounds__(256, 2) kbar_kernel(const __half* __restrict__
   if (live && sub == 0) {
     kbarNorm[((int64_t)g * U + u) * Cmax + j] = (float)sqrt(n2) * 1.000001f;
     kbarHatStat[((int64_t)g * U + u) * Cmax + j] = make_double2(mu2, rs2);
+    if (RK) kbarStat[((int64_t)g * U + u) * Cmax + j] = make_double2(mean, rstd);
   }
 }
 
@@ -280,12 +327,17 @@ __global__ void __launch_bounds__(256) route_filter_simt_kernel(const __half* __
 
 struct FoldDecideParams {
   const double* kbar64;
+  const __half* ok;          // (RK) keys of the folded block: unit u at ok + u * unit_stride, [C][D]
+  int64_t unit_stride;
+  const double2* kbarStat;   // (RK) [U, Cmax] (mean, rstd) of zero_r(k_j)
+  int r;
   const float* kbarNorm;
   const double2* kbarHatStat;   // (mean, rstd) of kbar_j: LN_s(kbar_j), the key of the row token j would create,
                                 // is gam * ((kbar_j - mean) * rstd) + bet, the expression of the memory-key kernel
   const float* gramT;        // [U, Cmax, Cmax] approximate kbarHat_a . kbar_j at [a][j] (fp16 operands); folds that append more than kGramOnTheFly rows
   const __half* kbarH;       // [U, CbarRows, D] memory keys in fp16 (operand of the products that small folds compute themselves)
   int CbarRows;
+  int otf_max;               // folds that append at most this many rows compute those products themselves (0: never)
   const float* candV;
   const int32_t* candI;
   const float *ln_w, *ln_b;
@@ -369,7 +421,7 @@ __device__ __forceinline__ void sort_n(K& key, int& val, K* sk, int* sv, int t) 
 
 // PER_SM = 2 for grids that fill the GPU twice over (64 registers, a few spills), 1 for the small grids
 // of chain-bound shapes, where a CTA has an SM to itself anyway and keeps everything in registers.
-template <int D, int PER_SM>
+template <int D, int PER_SM, bool RK>
 __global__ void __launch_bounds__(kDecideThreads, PER_SM) fold_decide_kernel(FoldDecideParams p) {
   constexpr int CH = D / 32;
   __shared__ double s_score[kMaxBlock], s_best[kMaxBlock];
@@ -395,9 +447,11 @@ __global__ void __launch_bounds__(kDecideThreads, PER_SM) fold_decide_kernel(Fol
   const int jlo = (int)blockIdx.x * ((C + R - 1) / R), jhi = min(C, jlo + (C + R - 1) / R);
   const int64_t m = p.m;
   const int n_a = p.n_append;
-  const double* kbarU = p.kbar64 + (int64_t)u * p.Cmax * D;
   const int64_t rowBase = (int64_t)u * p.Mcap;
   const int64_t tokBase = (int64_t)u * p.Cmax;
+  KbarRows<D, RK> kbarU;
+  kbarU.k64 = p.kbar64 + (int64_t)u * p.Cmax * D; kbarU.k16 = p.ok + (int64_t)u * p.unit_stride;
+  kbarU.stat = p.kbarStat + tokBase; kbarU.r = p.r;
 
   double gam[CH], bet[CH];
 #pragma unroll
@@ -533,12 +587,12 @@ __global__ void __launch_bounds__(kDecideThreads, PER_SM) fold_decide_kernel(Fol
     for (int k = 0; k < 8; ++k) {
       const int q = min(q0 + k * kDecideWarps, np - 1);   // clamped duplicates are computed and dropped
       const int j = s_ptok[q], i = s_prow[q];
-      const double* kb = kbarU + (int64_t)j * D;
       const double* sk = p.sumK + (rowBase + i) * D;
       const double mu = p.kmu[rowBase + i], rs = p.krstd[rowBase + i];
       double acc = 0.0;
 #pragma unroll
-      for (int c = 0; c < CH; ++c) acc += kb[lane + 32 * c] * (gam[c] * ((sk[lane + 32 * c] - mu) * rs) + bet[c]);
+      for (int c = 0; c < CH; ++c)
+        acc += kbarU.at(j, lane + 32 * c, gam[c], bet[c]) * (gam[c] * ((sk[lane + 32 * c] - mu) * rs) + bet[c]);
       part[k] = acc;
     }
     const double z0 = warp_reduce4(part[0], part[1], part[2], part[3], lane);
@@ -571,7 +625,7 @@ __global__ void __launch_bounds__(kDecideThreads, PER_SM) fold_decide_kernel(Fol
     if (!s_exh[j]) continue;
     double kb[CH];
 #pragma unroll
-    for (int i = 0; i < CH; ++i) kb[i] = kbarU[(int64_t)j * D + lane + 32 * i];
+    for (int i = 0; i < CH; ++i) kb[i] = kbarU.at(j, lane + 32 * i, gam[i], bet[i]);
     double score = -INFINITY, best = -INFINITY;
     int barg = -1;
     for (int64_t i = 0; i < m; ++i) {
@@ -652,15 +706,15 @@ __global__ void __launch_bounds__(kDecideThreads, PER_SM) fold_decide_kernel(Fol
   // keys LN_s(kbar_a) rounded to fp16 in shared memory: n_a x C products instead of the C x C that the
   // batched tensor-core product of the block's token pairs holds.  The error bound is the same (fp16
   // rounding of both operands; fp32 accumulation errs less than the tensor core's).
-  const bool otf = n_a <= kGramOnTheFly;
+  const bool otf = n_a <= p.otf_max;
   if (n_a > 0 && otf) {
     for (int a = warp; a < n_a; a += kDecideWarps) {
       const int jc = s_creator[a];
-      const double* ka = kbarU + (int64_t)jc * D;
       const double2 hs = p.kbarHatStat[tokBase + jc];
 #pragma unroll
       for (int c = 0; c < CH; ++c)
-        s_hat[a][lane + 32 * c] = __float2half_rn((float)(gam[c] * ((ka[lane + 32 * c] - hs.x) * hs.y) + bet[c]));
+        s_hat[a][lane + 32 * c] =
+            __float2half_rn((float)(gam[c] * ((kbarU.at(jc, lane + 32 * c, gam[c], bet[c]) - hs.x) * hs.y) + bet[c]));
     }
     __syncthreads();
   }
@@ -761,15 +815,14 @@ __global__ void __launch_bounds__(kDecideThreads, PER_SM) fold_decide_kernel(Fol
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
         const int q = min(q0 + k * kDecideWarps, np2 - 1);
-        const double* kb = kbarU + (int64_t)s_ptok[q] * D;
+        const int jt = s_ptok[q];
         const int jc = s_creator[s_prow[q]];
-        const double* ka = kbarU + (int64_t)jc * D;
         const double2 hs = p.kbarHatStat[tokBase + jc];
         double acc = 0.0;
 #pragma unroll
         for (int c = 0; c < CH; ++c) {
-          const double hat = gam[c] * ((ka[lane + 32 * c] - hs.x) * hs.y) + bet[c];
-          acc += kb[lane + 32 * c] * hat;
+          const double hat = gam[c] * ((kbarU.at(jc, lane + 32 * c, gam[c], bet[c]) - hs.x) * hs.y) + bet[c];
+          acc += kbarU.at(jt, lane + 32 * c, gam[c], bet[c]) * hat;
         }
         part[k] = acc;
       }
@@ -786,16 +839,16 @@ __global__ void __launch_bounds__(kDecideThreads, PER_SM) fold_decide_kernel(Fol
       if (!s_exh[j]) continue;
       double kb[CH];
 #pragma unroll
-      for (int c = 0; c < CH; ++c) kb[c] = kbarU[(int64_t)j * D + lane + 32 * c];
+      for (int c = 0; c < CH; ++c) kb[c] = kbarU.at(j, lane + 32 * c, gam[c], bet[c]);
       double best = s_best[j];
       int arg = s_barg[j];
       for (int a = 0; a < n_a; ++a) {
-        const double* ka = kbarU + (int64_t)s_creator[a] * D;
-        const double2 hs = p.kbarHatStat[tokBase + s_creator[a]];
+        const int jc = s_creator[a];
+        const double2 hs = p.kbarHatStat[tokBase + jc];
         double acc = 0.0;
 #pragma unroll
         for (int c = 0; c < CH; ++c) {
-          const double hat = gam[c] * ((ka[lane + 32 * c] - hs.x) * hs.y) + bet[c];
+          const double hat = gam[c] * ((kbarU.at(jc, lane + 32 * c, gam[c], bet[c]) - hs.x) * hs.y) + bet[c];
           acc += kb[c] * hat;
         }
         acc = warp_sum_d(acc);
@@ -857,6 +910,9 @@ __global__ void __launch_bounds__(kDecideThreads, PER_SM) fold_decide_kernel(Fol
 // 4. application: one warp per touched row
 
 struct FoldApplyParams {
+  const __half* ok;          // (RK) keys of the folded block, laid out like ov
+  const double2* kbarStat;   // (RK) [U, Cmax] (mean, rstd) of zero_r(k_j)
+  int r;
   const __half* ov;
   const float* og;
   int64_t unit_stride, gate_stride;
@@ -1010,7 +1066,7 @@ __global__ void __launch_bounds__(256, 4) fold_apply_kernel(FoldApplyParams p) {
 constexpr int kApplyRowsPerWarp = 4;
 constexpr int kApplyRowsPerCta = 8 * kApplyRowsPerWarp;
 
-template <int D>
+template <int D, bool RK>
 __global__ void __launch_bounds__(256, 2) fold_apply_rows4_kernel(FoldApplyParams p) {
   constexpr int NI = D / 32;          // runs of four channels per lane
   constexpr int NC = 4 * NI;          // channels per lane
@@ -1034,7 +1090,11 @@ __global__ void __launch_bounds__(256, 2) fold_apply_rows4_kernel(FoldApplyParam
   }
   if ((blockIdx.x * 8 + warp) * kApplyRowsPerWarp >= p.C) return;   // (whole warp)
   const int64_t rowBase = (int64_t)u * p.Mcap;
-  const double* kbarU = p.kbar64 + tokBase * D;
+  KbarRows<D, RK> kbarU;
+  kbarU.k64 = p.kbar64 + tokBase * D; kbarU.k16 = p.ok + (int64_t)u * p.unit_stride;
+  kbarU.stat = p.kbarStat + tokBase; kbarU.r = p.r;
+  const float* lnwH = p.ln_w + hk * D;
+  const float* lnbH = p.ln_b + hk * D;
   const __half* ovU = p.ov + (int64_t)u * p.unit_stride;
   const float* ogU = p.og + (int64_t)u * p.gate_stride;
   const int nmerge = p.all_append ? 0 : p.nmerge[u];
@@ -1073,13 +1133,13 @@ __global__ void __launch_bounds__(256, 2) fold_apply_rows4_kernel(FoldApplyParam
     for (int c = 0; c < NC; ++c) { kx[c] = 0.0; vx[c] = 0.f; }
     if (act) {
       if (task == 0) {
-        const double* kb = kbarU + (int64_t)jc * D;
         const __half* vr = ovU + (int64_t)jc * D;
 #pragma unroll
         for (int i = 0; i < NI; ++i) {
           const int x = 32 * i + 4 * sub;
-          const double2 k01 = *reinterpret_cast<const double2*>(kb + x), k23 = *reinterpret_cast<const double2*>(kb + x + 2);
-          kx[4 * i] = k01.x; kx[4 * i + 1] = k01.y; kx[4 * i + 2] = k23.x; kx[4 * i + 3] = k23.y;
+          double k4[4];
+          kbar_run4<D, RK>(kbarU, jc, x, lnwH, lnbH, k4);
+          kx[4 * i] = k4[0]; kx[4 * i + 1] = k4[1]; kx[4 * i + 2] = k4[2]; kx[4 * i + 3] = k4[3];
           alignas(8) __half hv[4];
           *reinterpret_cast<uint2*>(hv) = *reinterpret_cast<const uint2*>(vr + x);
 #pragma unroll
@@ -1114,14 +1174,14 @@ __global__ void __launch_bounds__(256, 2) fold_apply_rows4_kernel(FoldApplyParam
         const int j = s_sorted[qq];
         if (s_pi[j] != rowi) break;
         const float g = ogU[j];
-        const double* kb = kbarU + (int64_t)j * D;
         const __half* vr = ovU + (int64_t)j * D;
 #pragma unroll
         for (int i = 0; i < NI; ++i) {
           const int x = 32 * i + 4 * sub;
-          const double2 k01 = *reinterpret_cast<const double2*>(kb + x), k23 = *reinterpret_cast<const double2*>(kb + x + 2);
-          kx[4 * i] += (double)g * k01.x; kx[4 * i + 1] += (double)g * k01.y;
-          kx[4 * i + 2] += (double)g * k23.x; kx[4 * i + 3] += (double)g * k23.y;
+          double k4[4];
+          kbar_run4<D, RK>(kbarU, j, x, lnwH, lnbH, k4);
+          kx[4 * i] += (double)g * k4[0]; kx[4 * i + 1] += (double)g * k4[1];
+          kx[4 * i + 2] += (double)g * k4[2]; kx[4 * i + 3] += (double)g * k4[3];
           alignas(8) __half hv[4];
           *reinterpret_cast<uint2*>(hv) = *reinterpret_cast<const uint2*>(vr + x);
 #pragma unroll
@@ -1321,12 +1381,13 @@ int launch_kbar(State* st, const __half* ok, int64_t unit_stride, int nblk, int 
   float* kn = st->kbarNorm + (int64_t)slot0 * U * st->Cmax;
   double2* khat = st->kbarHatStat + (int64_t)slot0 * U * st->Cmax;
   __half* khh = st->kbarHatH + (int64_t)slot0 * U * st->CbarRows * D;
-  if (D == 128)
-    kbar_kernel<128><<<grid, 256, 0, s>>>(ok, unit_stride, st->ln_w, st->ln_b, k64, kh, kn, khat, khh, C, st->Cmax,
-                                          st->CbarRows, st->U, st->Hkv, st->r, (double)st->ln_eps, want_gram ? 1 : 0);
-  else
-    kbar_kernel<64><<<grid, 256, 0, s>>>(ok, unit_stride, st->ln_w, st->ln_b, k64, kh, kn, khat, khh, C, st->Cmax,
-                                         st->CbarRows, st->U, st->Hkv, st->r, (double)st->ln_eps, want_gram ? 1 : 0);
+  double2* kst = st->kbarStat + (int64_t)slot0 * U * st->Cmax;
+#define KVM_KBAR(DD, RR)                                                                                                   \
+  kbar_kernel<DD, RR><<<grid, 256, 0, s>>>(ok, unit_stride, st->ln_w, st->ln_b, k64, kh, kn, khat, khh, C, st->Cmax,        \
+                                           st->CbarRows, st->U, st->Hkv, st->r, (double)st->ln_eps, want_gram ? 1 : 0, kst)
+  if (D == 128) { if (st->recomputeK) KVM_KBAR(128, true); else KVM_KBAR(128, false); }
+  else { if (st->recomputeK) KVM_KBAR(64, true); else KVM_KBAR(64, false); }
+#undef KVM_KBAR
   int launches = 1;
   // the new-row filter is only read by folds that append some but not all of their tokens
   if (want_gram) launches += launch_gram_tc(st, slot0, nblk, s);
@@ -1387,8 +1448,9 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
     }
     FoldDecideParams p;
     p.kbar64 = kbar64; p.kbarNorm = kbarNorm; p.kbarHatStat = kbarHatStat;
+    p.ok = a.ok; p.unit_stride = a.unit_stride; p.kbarStat = st->kbarStat + (int64_t)a.slot * U * st->Cmax; p.r = st->r;
     p.gramT = st->gramT + (int64_t)a.slot * U * st->Cmax * st->Cmax;
-    p.kbarH = kbarH; p.CbarRows = st->CbarRows;
+    p.kbarH = kbarH; p.CbarRows = st->CbarRows; p.otf_max = gram_from(st);
     p.candV = st->candV; p.candI = st->candI; p.ln_w = st->ln_w; p.ln_b = st->ln_b;
     p.sumK = st->sumK; p.kmu = st->kmu; p.krstd = st->krstd;
     p.pi = st->foldPi[dst]; p.sorted = st->foldSorted[dst]; p.creator = st->foldCreator[dst];
@@ -1424,13 +1486,22 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
                      (sms_wanted <= 148 || st->U >= 148);
     lc.attrs = at; lc.numAttrs = pdl ? 1 : 0;
     const bool roomy = R * st->U <= 148;
-    if (D == 128) { if (roomy) cudaLaunchKernelEx(&lc, fold_decide_kernel<128, 1>, p); else cudaLaunchKernelEx(&lc, fold_decide_kernel<128, 2>, p); }
-    else { if (roomy) cudaLaunchKernelEx(&lc, fold_decide_kernel<64, 1>, p); else cudaLaunchKernelEx(&lc, fold_decide_kernel<64, 2>, p); }
+#define KVM_DECIDE(DD, PP, RR) cudaLaunchKernelEx(&lc, fold_decide_kernel<DD, PP, RR>, p)
+    const bool rk = st->recomputeK;
+    if (D == 128) {
+      if (roomy) { if (rk) KVM_DECIDE(128, 1, true); else KVM_DECIDE(128, 1, false); }
+      else { if (rk) KVM_DECIDE(128, 2, true); else KVM_DECIDE(128, 2, false); }
+    } else {
+      if (roomy) { if (rk) KVM_DECIDE(64, 1, true); else KVM_DECIDE(64, 1, false); }
+      else { if (rk) KVM_DECIDE(64, 2, true); else KVM_DECIDE(64, 2, false); }
+    }
+#undef KVM_DECIDE
     ++launches;
   }
   FoldApplyParams q;
   q.ov = a.ov; q.og = a.og; q.unit_stride = a.unit_stride; q.gate_stride = a.gate_stride;
   q.kbar64 = kbar64; q.ln_w = st->ln_w; q.ln_b = st->ln_b;
+  q.ok = a.ok; q.kbarStat = st->kbarStat + (int64_t)a.slot * U * st->Cmax; q.r = st->r;
   q.pi = st->foldPi[dst]; q.sorted = st->foldSorted[dst]; q.creator = st->foldCreator[dst];
   q.segnew = st->foldSegNew[dst]; q.nmerge = st->foldNMerge[dst];
   q.sumK = st->sumK; q.sumV = st->sumV; q.rho = st->rho; q.wsum = st->wsum; q.cnt = st->cnt;
@@ -1444,8 +1515,8 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
   KernelTimer kt(st, 5, s);
   if (apply_uses_rows4(st)) {
     dim3 grid((C + kApplyRowsPerCta - 1) / kApplyRowsPerCta, st->U);
-    if (D == 128) fold_apply_rows4_kernel<128><<<grid, 256, 0, s>>>(q);
-    else fold_apply_rows4_kernel<64><<<grid, 256, 0, s>>>(q);
+    if (D == 128) { if (st->recomputeK) fold_apply_rows4_kernel<128, true><<<grid, 256, 0, s>>>(q); else fold_apply_rows4_kernel<128, false><<<grid, 256, 0, s>>>(q); }
+    else { if (st->recomputeK) fold_apply_rows4_kernel<64, true><<<grid, 256, 0, s>>>(q); else fold_apply_rows4_kernel<64, false><<<grid, 256, 0, s>>>(q); }
   } else {
     dim3 grid((C + 7) / 8, st->U);
     if (D == 128) fold_apply_kernel<128><<<grid, 256, 0, s>>>(q);

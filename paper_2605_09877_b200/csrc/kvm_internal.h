@@ -16,9 +16,10 @@ constexpr int kMaxSplits = 32;      // routing filter / decode split count upper
 constexpr int kAttnSplitTiles = 37; // launches with at most this many (batch, head, query tile) CTAs - a quarter of the GPU - are split along the keys
 constexpr int kAttnMaxSplits = 8;
 constexpr int kRowAlign = 128;      // state capacity is rounded up to the attention key tile
-constexpr int kGramOnTheFly = 32;   // folds that append at most this many rows compute the products of the other tokens with the
-                                    // new rows inside the decision kernel; larger ones read them from the batched tensor-core
-                                    // product of all token pairs of the block (gramT), most of which such a fold would never read
+constexpr int kGramOnTheFly = 32;   // in a state with enough units to fill the GPU (State::serial), folds that append at most this
+                                    // many rows compute the products of the other tokens with the new rows inside the decision
+                                    // kernel; all other folds read them from the batched tensor-core product of all token pairs of
+                                    // the block (gramT), computed off the folds' critical path - most of it never read
 constexpr int kSerialUnits = 256;   // from this many (batch, kv head) units on, folds run on the caller's stream with one readout copy
 
 // State of one layer: host bookkeeping + device buffers.  U = batch * n_kv_heads "units";
@@ -87,6 +88,9 @@ struct State {
   //      call computes them for up to kbSlots consecutive overflow blocks in one launch; slot g holds
   //      one block's arrays in the layouts below ----
   int kbSlots;
+  bool recomputeK;               // (bound with the block) serial && the four-rows-per-warp apply kernel: kbar64 is not kept,
+                                 // the fold kernels recompute kbar_j from the fp16 key and kbarStat
+  double2* kbarStat;             // [kbSlots][U, Cmax]  (mean, rstd) of zero_r(k_j)
   double* kbar64;                // [kbSlots][U, Cmax, d]
   __half* kbarH;                 // [kbSlots][U, CbarRows, d]
   float* kbarNorm;               // [kbSlots][U, Cmax]
@@ -132,6 +136,8 @@ struct State {
 };
 
 inline int64_t budget_of(const kvm_growth_t& g, int64_t e);
+// folds that append more rows than this (and not the whole block) take the batched product of the block's token pairs
+inline int gram_from(const State* st) { return st->serial ? kGramOnTheFly : 0; }
 
 // ---------------- launchers (each returns the number of kernels it launched) ----------------
 
