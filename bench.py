@@ -87,12 +87,32 @@ def prefill_flops(wl, T):
     return 4 * wl.d * att_pairs * units_q, 2 * wl.d * route_pairs * units_kv
 
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the kernels that carry a
-# roofline, from the ncu captures summarised under profiles/ (null until captured for the workload).
-NCU_TRAFFIC = {
-    ("cfg5", "decode"): 4.574e9,    # profiles/ncu_full_attn_route_decide_decode_small_cases.md (4.570 GB read + 4 MB written)
-    ("cfg2", "attention"): 13.72e6,  # same file: 13.72 MB read, 0 written per launch (algorithmic: 14.6 MB)
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the kernels that carry a roofline, from the ncu
+# captures summarised under profiles/ncu_full_cfg5_small_case_prefill_and_decode_kernels.md.  The captures run a
+# small case of the same kernels (256 units instead of 2048; 640 decode heads instead of 2048); both kernels read
+# every key / value row of a (batch, head) unit once per launch, so the traffic of a launch grows in proportion to
+# units x rows: the figure reported for a full-size launch is the algorithmic bytes of that launch times the
+# measured ratio (traffic / algorithmic bytes) of the captured launches.
+NCU_TRAFFIC_RATIO = {
+    "attention": (268.54e6 + 13.6e6) / 278.2e6,   # captured: 268.5 MB read + 13.6 MB written; algorithmic 278.2 MB per launch
+    "decode": 1.4320e9 / 1.4293e9,                # captured: 1.428 GB read + 4 MB written; algorithmic 1.4293 GB per launch
 }
+
+
+def attention_bytes_per_launch(wl, T):
+    """Algorithmic bytes of an average attention launch of a prefill: per (batch, kv head) unit the fp16 readout rows
+    K^, V^ of the state and the fp16 window keys and values the block can see, once; per (batch, q head) the block's
+    fp16 queries read and its bf16 outputs written."""
+    folds = {e: (m0, na) for e, m0, na in fold_schedule(wl, T)}
+    m, tot, n = 0, 0, 0
+    for c in range(T // wl.C):
+        e = (c + 1) * wl.C
+        win = min(c, wl.w - 1) * wl.C + wl.C
+        tot += wl.B * wl.Hkv * (m + win) * wl.d * 2 * 2 + wl.B * wl.Hq * wl.C * wl.d * 2 * 2
+        n += 1
+        if e in folds:
+            m = folds[e][0] + folds[e][1]
+    return tot / max(n, 1)
 
 
 def decode_bytes(wl, m, pos):
@@ -476,7 +496,7 @@ def decode_record(st, wl, dev, stream, pk, world):
                 min_us=min(plain), max_us=max(plain),
                 roofline=dict(bound="hbm", kernel="decode", achieved=gbs_plain, peak=pk["hbm"], unit="GB/s",
                               frac=gbs_plain / pk["hbm"], frac_of_nominal_8TBs=gbs_plain / 8000.0,
-                              traffic=NCU_TRAFFIC.get(("cfg5", "decode")),
+                              traffic=sum(nbytes[3:half]) / len(plain) * NCU_TRAFFIC_RATIO["decode"],
                               peak_source=f"{pk['src']} copy bandwidth", bytes_per_step=sum(nbytes[3:half]) / len(plain),
                               what="whole decode steps (ingest + attention kernels), CUDA events around each step",
                               kernels_only_gbs=gbs_kern, kernels_only_us=1e3 * kern_ms / max(kern_n, 1)))
@@ -624,8 +644,11 @@ def main():
         ach = ((att_f if dom == "attention" else rt_f) / 1e12) / (dom_ms * 1e-3)
         peak = pk["tf_sust"]
         roof = dict(bound="tensor", kernel=dom, achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak,
-                    traffic=NCU_TRAFFIC.get((wl.name, dom)),
+                    traffic=(attention_bytes_per_launch(wl, wl.T) * NCU_TRAFFIC_RATIO["attention"]) if dom == "attention" else None,
+                    traffic_source="algorithmic bytes of an average launch x (DRAM traffic / algorithmic bytes) of the ncu small-case capture (profiles/)",
+                    algorithmic_bytes_per_launch=attention_bytes_per_launch(wl, wl.T) if dom == "attention" else None,
                     peak_source=f"{pk['src']} bf16 sustained (fp16 operands run at the bf16 rate)",
+                    frac_of_burst=ach / pk["tf_burst"], frac_of_nominal_2250=ach / 2250.0,
                     launches_per_step=n_dom, avg_launch_us=1e3 * dom_ms / max(n_dom, 1),
                     share_of_device_time=dom_ms / max(sum(per_kernel.values()), 1e-9),
                     whole_step_tflops=(att_f + rt_f) / 1e12 / (ms_step * 1e-3),
@@ -642,7 +665,7 @@ def main():
         dec_ms = prof["decode"][0] / max(prof["decode"][1], 1)
         ach = bytes_step / 1e9 / (dec_ms * 1e-3)
         roof = dict(bound="hbm", kernel="decode", achieved=ach, peak=pk["hbm"], unit="GB/s", frac=ach / pk["hbm"],
-                    traffic=NCU_TRAFFIC.get((wl.name, "decode")), peak_source=f"{pk['src']} copy bandwidth",
+                    traffic=bytes_step * NCU_TRAFFIC_RATIO["decode"], peak_source=f"{pk['src']} copy bandwidth",
                     bytes_per_step=bytes_step,
                     frac_of_nominal_8TBs=ach / 8000.0, phase_ms={k_: v_[0] / max(v_[1], 1) for k_, v_ in prof.items()})
         metric, unit, hib = "kvm_decode_us_per_step", "us/step", False
