@@ -188,7 +188,7 @@ def oracle_sample(wl, mode, budget_s=20.0):
         n_units = min(cores, wl.B * wl.Hkv)
         T_s = wl.T
         att, rt = prefill_flops(wl.scaled(B=1, Hq=n_units * (wl.Hq // wl.Hkv), Hkv=n_units), T_s)
-        rate = 2.5e9 * cores   # rough fp64 flop/s of the plain loops; only used to size the sample
+        rate = 3.0e9 * cores   # measured fp64 flop/s of the plain loops on this kind of host; only sizes the sample
         while (att + rt) / rate > budget_s and T_s > 4 * wl.C:
             T_s //= 2
             att, rt = prefill_flops(wl.scaled(B=1, Hq=n_units * (wl.Hq // wl.Hkv), Hkv=n_units), T_s)

@@ -24,13 +24,20 @@ def _continue(st, g, wl, q, k, v, gate, a, b, dec_from):
     return y.cpu()
 
 
-@pytest.mark.parametrize("wl,cut,params_trivial,use_gate", [
-    (synth.Workload("snapA", 2, 4, 2, 128, 256 * 6 + 90, 256, "sqrt", sqrt_coeff=10, r=32, seed=41), 256 * 3 + 77, False, True),
-    (synth.Workload("snapB", 1, 3, 3, 64, 64 * 20 + 5, 64, "fixed", fixed_slots=200, r=0, seed=42, kind="mixture"), 64 * 9, True, False),
-    (synth.Workload("snapC", 1, 2, 2, 64, 300, 32, "sqrt", sqrt_coeff=6, r=16, seed=43, w=3), 17, True, False),   # cut before any fold
-    (synth.Workload("snapD", 1, 40, 40, 128, 256 * 5 + 33, 256, "sqrt", r=0, seed=44), 256 * 4 + 1, True, False),  # four-rows-per-warp apply
+SERIAL = 1 << 5   # KVM_FLAG_SERIAL_FOLDS
+
+
+@pytest.mark.parametrize("wl,cut,params_trivial,use_gate,flags", [
+    (synth.Workload("snapA", 2, 4, 2, 128, 256 * 6 + 90, 256, "sqrt", sqrt_coeff=10, r=32, seed=41), 256 * 3 + 77, False, True, 0),
+    (synth.Workload("snapB", 1, 3, 3, 64, 64 * 20 + 5, 64, "fixed", fixed_slots=200, r=0, seed=42, kind="mixture"), 64 * 9, True, False, 0),
+    (synth.Workload("snapC", 1, 2, 2, 64, 300, 32, "sqrt", sqrt_coeff=6, r=16, seed=43, w=3), 17, True, False, 0),   # cut before any fold
+    (synth.Workload("snapD", 1, 40, 40, 128, 256 * 5 + 33, 256, "sqrt", r=0, seed=44), 256 * 4 + 1, True, False, 0),  # four-rows-per-warp apply
+    # one readout copy, folds on the caller's stream
+    (synth.Workload("snapF", 1, 4, 2, 128, 128 * 9 + 60, 128, "sqrt", sqrt_coeff=5, r=32, seed=46), 128 * 4 + 9, False, True, SERIAL),
+    # the same with 64 units x block 128: no fp64 memory keys are kept, the import rebuilds the per-row statistics
+    (synth.Workload("snapG", 2, 32, 32, 128, 128 * 8 + 50, 128, "sqrt", sqrt_coeff=5, r=32, seed=47), 128 * 5 + 3, False, False, SERIAL),
 ])
-def test_snapshot_restore_continue_equals_uninterrupted_run(wl, cut, params_trivial, use_gate):
+def test_snapshot_restore_continue_equals_uninterrupted_run(wl, cut, params_trivial, use_gate, flags):
     params = synth.make_layer_params(wl, trivial=params_trivial)
     tensors = synth.make_inputs(wl)
     gate_cpu = synth.make_gate(wl) if use_gate else None
@@ -38,20 +45,20 @@ def test_snapshot_restore_continue_equals_uninterrupted_run(wl, cut, params_triv
     gate = None if gate_cpu is None else gate_cpu.cuda()
     dec_from = wl.T - 40
     # uninterrupted: prefill [0, cut), prefill [cut, dec_from), decode the rest (same call boundaries as the resumed run)
-    ref, g = pu.gpu_layer(wl, params)
+    ref, g = pu.gpu_layer(wl, params, flags=flags)
     y0 = _continue(ref, g, wl, q, k, v, gate, 0, cut, cut)
     y_ref = _continue(ref, g, wl, q, k, v, gate, cut, wl.T, dec_from)
     e_ref = ref.export()
     slot_ref, app_ref = ref.assignments()
     ref.free()
     # interrupted: prefill [0, cut) -> snapshot -> free -> create -> import -> continue
-    a, g = pu.gpu_layer(wl, params)
+    a, g = pu.gpu_layer(wl, params, flags=flags)
     y0b = _continue(a, g, wl, q, k, v, gate, 0, cut, cut)
     assert torch.equal(y0, y0b)
     snap = a.snapshot()
     info_a = a.info()
     a.free()
-    b, g = pu.gpu_layer(wl, params)
+    b, g = pu.gpu_layer(wl, params, flags=flags)
     b.restore(snap)
     assert b.info() == info_a
     y_b = _continue(b, g, wl, q, k, v, gate, cut, wl.T, dec_from)

@@ -6,7 +6,9 @@ end, so the oracle run on a unit alone is that unit's exact reference):
   * the decode kernel's direct-output branch (one row split per head) at head_dim 128, with and without
     grouped queries;
   * config 5's structure at a batch wide enough to select the kernels that the full batch selects;
-  * the minimum of two memory-key slots (one block of look-ahead), which very large batches run with.
+  * the minimum of two memory-key slots (one block of look-ahead), which very large batches run with;
+  * what states that fill the GPU do: folds on the caller's stream with one readout copy, new-row products
+    inside the decision kernel for folds that append few rows, memory keys recomputed from their fp16 copy.
 """
 import numpy as np
 import pytest
@@ -80,7 +82,7 @@ def test_two_memory_key_slots_one_block_of_look_ahead():
 
 
 def test_serial_folds_one_readout_copy():
-    """What states of 512 or more units do by themselves, forced on small shapes: folds on the caller's stream
+    """What states of 256 or more units do by themselves, forced on small shapes: folds on the caller's stream
     between the attention launches, one readout copy written in place; segmented prefill, gates, decode with a
     fold."""
     from paper_2605_09877_b200 import kvm
@@ -94,3 +96,21 @@ def test_serial_folds_one_readout_copy():
     y_ref, o = pu.run_oracle(wl, tensors, params)
     print(pu.compare(wl, y_gpu, st, y_ref, o))
     st.free()
+
+
+def test_small_appends_compute_their_products_in_the_decision_kernel_and_keys_are_recomputed():
+    """Serial states: a fold that appends at most 32 rows computes the products of its new rows with the block's
+    keys itself (here every fold after the first: 4 sqrt(N) slots), larger ones use the batched launch (the
+    second case, 16 sqrt(N): both kinds in one run).  64 units x block 128 is also the size from which no fp64
+    memory keys are kept: every fp64 key the fold kernels use is recomputed from the fp16 key and the token's
+    LayerNorm statistics.  Exact slots against the oracle say that the recomputed keys equal the stored ones."""
+    from paper_2605_09877_b200 import kvm
+    wl = synth.Workload("t", 2, 32, 32, 128, 128 * 12 + 31, 128, "sqrt", sqrt_coeff=4, r=32, seed=36)
+    params = synth.make_layer_params(wl, trivial=False)
+    stats = _sampled(wl, [(0, 0), (0, 19), (1, 7), (1, 31)], params=params, gate=True, flags=kvm.FLAG_SERIAL_FOLDS)
+    print(stats)
+    wl = synth.Workload("t", 2, 32, 32, 128, 128 * 40 + 77, 128, "sqrt", sqrt_coeff=16, r=32, seed=37, kind="mixture")
+    print(_sampled(wl, [(0, 3), (1, 30)], flags=kvm.FLAG_SERIAL_FOLDS, decode_from=128 * 40 + 40))
+    # the same small-append shape below the size threshold keeps its fp64 keys: products inside the kernel only
+    wl = synth.Workload("t", 1, 3, 3, 64, 64 * 14 + 9, 64, "sqrt", sqrt_coeff=3, r=16, seed=38)
+    print(_sampled(wl, None, flags=kvm.FLAG_SERIAL_FOLDS))
