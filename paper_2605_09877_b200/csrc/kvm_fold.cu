@@ -907,6 +907,568 @@ __global__ void __launch_bounds__(kDecideThreads, PER_SM) fold_decide_kernel(Fol
 }
 
 // ------------------------------------------------------------------------------------------
+// 3b. decisions for states with more units than SMs (one CTA per unit, four CTAs per SM), folds that append rows
+//
+// With thousands of units the exact similarities are what the decision costs: every pair reads a 1 KB row of
+// fp64 key sums from HBM, and a fold that appends rows asked for the exact score (best similarity over all
+// rows) of every token just to rank them.  Here the routing filter's maxima rank them first: the exact score
+// of token j lies in [gmax_j - eps_j, gmax_j + eps_j] (eps_j = the bound on the fp16 rounding of its
+// products, half the filter's window), so a token is appended for certain when fewer than n_a others can
+// rank before it, merged for certain when n_a others rank before it for certain, and only the tokens in
+// between are scored exactly (round 1).  A token that is merged for certain with a single candidate row and
+// no new row in reach needs no exact similarity at all; the others get their old candidates and the new rows
+// in reach compared exactly in round 2.  The decisions are those of the kernel above bit for bit: the bounds
+// only remove work whose outcome they fix.
+// The products with the rows a small fold appends (n_a <= kGramOnTheFly) run on the tensor cores
+// (mma.sync m16n8k16, fp16 x fp16 -> fp32): tokens x new rows, the new rows' keys in shared memory.
+
+constexpr int kPrunedThreads = 256;
+constexpr int kPrunedWarps = kPrunedThreads / 32;
+constexpr int kPairCap2 = 1024;
+static_assert(kPrunedThreads == kMaxBlock, "one thread per token of the block");
+
+__device__ __forceinline__ void mma_m16n8k16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+template <int D, bool RK>
+__global__ void __launch_bounds__(kPrunedThreads, 4) fold_decide_pruned_kernel(FoldDecideParams p) {
+  constexpr int CH = D / 32;
+  constexpr int HS = D + 32;   // row stride of the new rows' keys in halves: consecutive rows start 16 banks apart
+  __shared__ double s_lo[kMaxBlock], s_hi[kMaxBlock];   // bounds of the score; then exact score / exact best of scored tokens
+  __shared__ int s_barg[kMaxBlock], s_pi[kMaxBlock], s_creator[kMaxBlock];
+  __shared__ int s_pstart[kMaxBlock], s_pcnt[kMaxBlock], s_nold[kMaxBlock];
+  __shared__ int s_gmaxi[kMaxBlock], s_fill[kMaxBlock], s_ulist[kMaxBlock];
+  __shared__ float s_thr[kMaxBlock];
+  __shared__ unsigned char s_app[kMaxBlock], s_exh[kMaxBlock], s_cls[kMaxBlock], s_sink[kMaxBlock], s_ccnt[kMaxBlock];
+  __shared__ unsigned char s_cont[4 * kMaxBlock];
+  __shared__ int s_prow[kPairCap2];
+  __shared__ unsigned short s_ptok[kPairCap2];
+  __shared__ double s_pval[kPairCap2];
+  __shared__ int s_np, s_nexh, s_nunc, s_npairs;
+  __shared__ int s_wsum[kPrunedWarps];
+  __shared__ __align__(16) __half s_hat[kGramOnTheFly * HS];
+
+  const int u = blockIdx.y, hk = u % p.Hkv;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int C = p.C;
+  const int nsort = C <= 128 ? 128 : 256;
+  const int64_t m = p.m;
+  const int n_a = p.n_append;
+  const int64_t rowBase = (int64_t)u * p.Mcap;
+  const int64_t tokBase = (int64_t)u * p.Cmax;
+  KbarRows<D, RK> kbarU;
+  kbarU.k64 = p.kbar64 + (int64_t)u * p.Cmax * D; kbarU.k16 = p.ok + (int64_t)u * p.unit_stride;
+  kbarU.stat = p.kbarStat + tokBase; kbarU.r = p.r;
+  const float* lnwH = p.ln_w + hk * D;
+  const float* lnbH = p.ln_b + hk * D;
+  enum { UNSURE = 0, SURE_APPEND = 1, SURE_MERGE = 2 };
+
+  if (tid == 0) { s_np = 0; s_nexh = 0; s_nunc = 0; s_npairs = 0; }
+  s_app[tid] = 0; s_exh[tid] = 0; s_cls[tid] = UNSURE; s_sink[tid] = 0; s_ccnt[tid] = 0;
+  s_pcnt[tid] = 0; s_nold[tid] = 0; s_pstart[tid] = 0; s_pi[tid] = -1; s_barg[tid] = -1; s_creator[tid] = -1;
+  s_gmaxi[tid] = (int)0x80000000; s_fill[tid] = 0; s_thr[tid] = 0.f;
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (tid < p.Cmax) p.segnew[tokBase + tid] = -1;
+  __syncthreads();
+
+  // exact fp64 value of the pairs [0, np) of the list: rows < m are rows of the state, kbar_j . LN_s(s^K_i);
+  // rows >= m are rows this fold appends, kbar_j . LN_s(kbar_c) with c the creator of row (i - m).  One warp
+  // per pair, eight pairs in flight per warp.
+  auto exact_pairs = [&](int np) {
+    double gam[CH], bet[CH];
+#pragma unroll
+    for (int c = 0; c < CH; ++c) { gam[c] = (double)lnwH[lane + 32 * c]; bet[c] = (double)lnbH[lane + 32 * c]; }
+    for (int q0 = warp; q0 < np; q0 += 8 * kPrunedWarps) {
+      double part[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int q = min(q0 + k * kPrunedWarps, np - 1);   // clamped duplicates are computed and dropped
+        const int j = s_ptok[q], i = s_prow[q];
+        double acc = 0.0;
+        if (i < m) {
+          const double* sk = p.sumK + (rowBase + i) * D;
+          const double mu = p.kmu[rowBase + i], rs = p.krstd[rowBase + i];
+#pragma unroll
+          for (int c = 0; c < CH; ++c)
+            acc += kbarU.at(j, lane + 32 * c, gam[c], bet[c]) * (gam[c] * ((sk[lane + 32 * c] - mu) * rs) + bet[c]);
+        } else {
+          const int jc = s_creator[i - (int)m];
+          const double2 hs = p.kbarHatStat[tokBase + jc];
+#pragma unroll
+          for (int c = 0; c < CH; ++c) {
+            const double hat = gam[c] * ((kbarU.at(jc, lane + 32 * c, gam[c], bet[c]) - hs.x) * hs.y) + bet[c];
+            acc += kbarU.at(j, lane + 32 * c, gam[c], bet[c]) * hat;
+          }
+        }
+        part[k] = acc;
+      }
+      const double z0 = warp_reduce4(part[0], part[1], part[2], part[3], lane);
+      const double z1 = warp_reduce4(part[4], part[5], part[6], part[7], lane);
+      if ((lane & 7) == 0) {
+        const int qa = q0 + (lane >> 3) * kPrunedWarps, qb = qa + 4 * kPrunedWarps;
+        if (qa < np) s_pval[qa] = z0;
+        if (qb < np) s_pval[qb] = z1;
+      }
+    }
+  };
+  // exclusive prefix sum of c over the threads of the CTA (all threads call)
+  auto block_scan = [&](int c) {
+    int incl = c;
+#pragma unroll
+    for (int o2 = 1; o2 < 32; o2 <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o2);
+      if (lane >= o2) incl += v;
+    }
+    __syncthreads();   // (s_wsum may still be read from an earlier call)
+    if (lane == 31) s_wsum[warp] = incl;
+    __syncthreads();
+    int start = incl - c;
+    for (int w = 0; w < warp; ++w) start += s_wsum[w];
+    return start;
+  };
+
+  // ---- 1: per token, the filter's maximum over the splits (rows >= S), the window, the number of candidates ----
+  const int nitems = C * p.nsplit;
+  const int64_t ostep = (int64_t)p.Cmax * kTopK;
+  const int64_t obase = (int64_t)u * p.nsplit * p.Cmax * kTopK;
+  for (int it = tid; it < nitems; it += kPrunedThreads) {
+    const int sp = it / C, j = it % C;
+    const int vi = __float_as_int(p.candV[obase + sp * ostep + (int64_t)j * kTopK]);
+    atomicMax(&s_gmaxi[j], vi >= 0 ? vi : vi ^ 0x7fffffff);
+    if (sp == 0) s_thr[j] = p.thr_coeff * p.kbarNorm[tokBase + j] + 1e-5f;
+  }
+  __syncthreads();
+  for (int it = tid; it < nitems; it += kPrunedThreads) {
+    const int sp = it / C, j = it % C;
+    const int gi = s_gmaxi[j];
+    const float gmax = __int_as_float(gi >= 0 ? gi : gi ^ 0x7fffffff);
+    if (!(gmax > -INFINITY)) { s_exh[j] = 1; continue; }
+    const int64_t o = obase + sp * ostep + (int64_t)j * kTopK;
+    const float2 hd = *reinterpret_cast<const float2*>(p.candV + o);
+    int i[kTopK];
+    load_cand_rows(p.candI, o, i);
+    const bool keep = hd.x >= gmax - s_thr[j];
+    if (hd.y > (float)kTopK && (keep || sp == 0)) s_exh[j] = 1;   // list overflowed
+    int call = 0, cold = 0;
+#pragma unroll
+    for (int k = 0; k < kTopK; ++k) {
+      if (i[k] >= 0 && (i[k] < p.S || keep)) ++call;
+      if (i[k] >= p.S && keep) ++cold;
+      if (i[k] >= 0 && i[k] < p.S) s_sink[j] = 1;   // a sink row in reach: its product is not among the maxima
+    }
+    if (call > 0) atomicAdd(&s_pcnt[j], call);
+    if (cold > 0) atomicAdd(&s_nold[j], cold);
+  }
+  __syncthreads();
+  // ---- 2: which tokens are appended or merged whatever their exact scores turn out to be ----
+  {
+    const bool have = tid < C;
+    const bool open = have && (s_exh[tid] || s_sink[tid]);   // no usable bounds: scored exactly
+    double lo = INFINITY, hi = INFINITY;                      // (threads past the block rank after everything)
+    if (have) {
+      const int gi = s_gmaxi[tid];
+      const double g = (double)__int_as_float(gi >= 0 ? gi : gi ^ 0x7fffffff);
+      const double eps = 0.5 * (double)s_thr[tid];
+      lo = open ? -INFINITY : g - eps;
+      hi = open ? INFINITY : g + eps;
+    }
+    s_lo[tid] = lo; s_hi[tid] = hi;
+    __syncthreads();
+    int may = 0, must = 0;   // tokens that may / must rank before this one (ties may)
+    for (int i = 0; i < C; ++i) {
+      may += s_lo[i] <= hi ? 1 : 0;
+      must += s_hi[i] < lo ? 1 : 0;
+    }
+    may -= 1;   // (itself)
+    if (have && !open) s_cls[tid] = may <= n_a - 1 ? SURE_APPEND : (must >= n_a ? SURE_MERGE : UNSURE);
+    __syncthreads();
+  }
+  // ---- 3: round 1: exact score, best old row of the unsure tokens ----
+  {
+    const bool unsure = tid < C && s_cls[tid] == UNSURE;
+    bool exh = unsure && s_exh[tid];
+    int c = (unsure && !exh) ? s_pcnt[tid] : 0;
+    if (c > kPairPerTok) { exh = true; c = 0; }
+    const int start = block_scan(c);
+    if (start + c > kPairCap2) { exh = unsure; c = 0; }
+    s_pstart[tid] = start; s_pcnt[tid] = c; s_fill[tid] = 0; s_exh[tid] = exh ? 1 : 0;
+    const unsigned wend = __reduce_max_sync(0xffffffffu, (unsigned)(c > 0 ? start + c : 0));
+    if (lane == 0 && wend > 0) atomicMax(&s_np, (int)wend);
+    const int ne = __syncthreads_count(exh);
+    if (tid == 0) s_nexh += ne;
+  }
+  __syncthreads();
+  for (int it = tid; it < nitems; it += kPrunedThreads) {
+    const int sp = it / C, j = it % C;
+    if (s_cls[j] != UNSURE || s_exh[j] || s_pcnt[j] == 0) continue;
+    const int gi = s_gmaxi[j];
+    const float gmax = __int_as_float(gi >= 0 ? gi : gi ^ 0x7fffffff);
+    const int64_t o = obase + sp * ostep + (int64_t)j * kTopK;
+    const bool keep = p.candV[o] >= gmax - s_thr[j];
+    int i[kTopK];
+    load_cand_rows(p.candI, o, i);
+    int c = 0;
+#pragma unroll
+    for (int k = 0; k < kTopK; ++k)
+      if (i[k] >= 0 && (i[k] < p.S || keep)) ++c;
+    if (c == 0) continue;
+    int w = s_pstart[j] + atomicAdd(&s_fill[j], c);
+#pragma unroll
+    for (int k = 0; k < kTopK; ++k) {
+      if (i[k] >= 0 && (i[k] < p.S || keep)) {
+        s_prow[w] = i[k];
+        s_ptok[w] = (unsigned short)j;
+        ++w;
+      }
+    }
+  }
+  __syncthreads();
+  {
+    const int np = min(s_np, kPairCap2);
+    exact_pairs(np);
+    if (tid == 0) s_npairs += np;
+  }
+  __syncthreads();
+  if (tid < C && s_cls[tid] == UNSURE && !s_exh[tid]) {
+    double score = -INFINITY, best = -INFINITY;
+    int barg = -1;
+    const int st0 = s_pstart[tid];
+    for (int q = st0; q < st0 + s_pcnt[tid]; ++q) {
+      const double v = s_pval[q];
+      const int i = s_prow[q];
+      if (v > score) score = v;
+      if (i >= p.S && (v > best || (v == best && i < barg))) { best = v; barg = i; }
+    }
+    s_lo[tid] = score; s_hi[tid] = best; s_barg[tid] = barg;
+  }
+  for (int j = warp; j < C; j += kPrunedWarps) {   // no usable list: every row exactly, one warp per token
+    if (!s_exh[j]) continue;
+    double gam[CH], bet[CH], kb[CH];
+#pragma unroll
+    for (int c = 0; c < CH; ++c) {
+      gam[c] = (double)lnwH[lane + 32 * c]; bet[c] = (double)lnbH[lane + 32 * c];
+      kb[c] = kbarU.at(j, lane + 32 * c, gam[c], bet[c]);
+    }
+    double score = -INFINITY, best = -INFINITY;
+    int barg = -1;
+    for (int64_t i = 0; i < m; ++i) {
+      const double acc = warp_sim<CH>(kb, p.sumK + (rowBase + i) * D, p.kmu[rowBase + i], p.krstd[rowBase + i], gam, bet, lane);
+      if (acc > score) score = acc;
+      if (i >= p.S && acc > best) { best = acc; barg = (int)i; }
+    }
+    if (lane == 0) { s_lo[j] = score; s_hi[j] = best; s_barg[j] = barg; }
+  }
+  __syncthreads();
+  // ---- 4: append selection: the certain ones, then the unsure ones by exact score (ties: smaller token) ----
+  {
+    const bool have = tid < C;
+    const int cls = have ? s_cls[tid] : SURE_MERGE;
+    const int n_sure = __syncthreads_count(have && cls == SURE_APPEND);
+    if (have && cls == UNSURE) s_ulist[atomicAdd(&s_nunc, 1)] = tid;
+    __syncthreads();
+    bool ap = have && cls == SURE_APPEND;
+    if (have && cls == UNSURE) {
+      const double sj = s_lo[tid];
+      int rank = 0;
+      const int nu = s_nunc;
+      for (int k = 0; k < nu; ++k) {
+        const int i = s_ulist[k];
+        const double si = s_lo[i];
+        rank += (si < sj || (si == sj && i < tid)) ? 1 : 0;
+      }
+      ap = rank < n_a - n_sure;
+    }
+    s_app[tid] = ap ? 1 : 0;
+    // rows are laid down in ascending token order: position of an appended token = appended tokens before it
+    const unsigned bal = __ballot_sync(0xffffffffu, ap);
+    const int before_w = __popc(bal & ((1u << lane) - 1u));
+    __syncthreads();
+    if (lane == 0) s_wsum[warp] = __popc(bal);
+    __syncthreads();
+    if (ap) {
+      int before = before_w;
+      for (int wq = 0; wq < warp; ++wq) before += s_wsum[wq];
+      s_creator[before] = tid;
+    }
+    __syncthreads();
+  }
+  // ---- 5: the new rows in reach of every merged token.  best_old below is the exact best old similarity of a
+  //      scored token, a lower bound of it for the others; products are within eps_j of the exact values, so a
+  //      new row can only win when its product reaches max(best_old, best product - eps_j) - eps_j. ----
+  const bool otf = n_a <= p.otf_max;
+  if (otf) {
+    for (int e = tid; e < kGramOnTheFly * HS / 8; e += kPrunedThreads) reinterpret_cast<uint4*>(s_hat)[e] = make_uint4(0u, 0u, 0u, 0u);
+    __syncthreads();
+    double gam[CH], bet[CH];
+#pragma unroll
+    for (int c = 0; c < CH; ++c) { gam[c] = (double)lnwH[lane + 32 * c]; bet[c] = (double)lnbH[lane + 32 * c]; }
+    for (int a = warp; a < n_a; a += kPrunedWarps) {
+      const int jc = s_creator[a];
+      const double2 hs = p.kbarHatStat[tokBase + jc];
+#pragma unroll
+      for (int c = 0; c < CH; ++c)
+        s_hat[a * HS + lane + 32 * c] =
+            __float2half_rn((float)(gam[c] * ((kbarU.at(jc, lane + 32 * c, gam[c], bet[c]) - hs.x) * hs.y) + bet[c]));
+    }
+    __syncthreads();
+    // 16 tokens x 8 new rows per instruction; lane (g, t) = (lane / 4, lane % 4) holds tokens g and g + 8 of the
+    // tile and new rows 8 nt + 2 t, + 1.  The channels are dealt to the instruction's k index in runs of eight per
+    // lane (the same permutation on both operands leaves the sums unchanged), so that both operands are read
+    // 16 bytes at a time.
+    const int g = lane >> 2, t = lane & 3;
+    const int NT = (n_a + 7) / 8;
+    const __half* kU = p.kbarH + (int64_t)u * p.CbarRows * D;
+    for (int mt = warp; mt * 16 < C; mt += kPrunedWarps) {
+      const int j0 = mt * 16 + g, j1 = j0 + 8;
+      const __half* r0 = kU + (int64_t)min(j0, C - 1) * D + 8 * t;
+      const __half* r1 = kU + (int64_t)min(j1, C - 1) * D + 8 * t;
+      float acc[4][4];
+#pragma unroll
+      for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
+#pragma unroll
+      for (int ks = 0; ks < D / 32; ++ks) {
+        const uint4 a0 = *reinterpret_cast<const uint4*>(r0 + 32 * ks), a1 = *reinterpret_cast<const uint4*>(r1 + 32 * ks);
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+          if (nt < NT) {
+            const uint4 b = *reinterpret_cast<const uint4*>(&s_hat[(nt * 8 + g) * HS + 32 * ks + 8 * t]);
+            mma_m16n8k16(acc[nt], a0.x, a1.x, a0.y, a1.y, b.x, b.y);
+            mma_m16n8k16(acc[nt], a0.z, a1.z, a0.w, a1.w, b.z, b.w);
+          }
+        }
+      }
+      // per token: best product over the new rows, then the rows in reach as a bit mask
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int j = h ? j1 : j0;
+        float gm = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+          for (int e = 0; e < 2; ++e)
+            if (nt * 8 + 2 * t + e < n_a) gm = fmaxf(gm, acc[nt][2 * h + e]);
+        gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, 1));
+        gm = fmaxf(gm, __shfl_xor_sync(0xffffffffu, gm, 2));
+        unsigned mask = 0;
+        if (j < C && !s_app[j]) {
+          const double eps = 0.5 * (double)s_thr[j];
+          const double best_old = s_cls[j] == UNSURE ? s_hi[j] : s_lo[j];
+          const double bar = fmax(best_old, (double)gm - eps) - eps;
+#pragma unroll
+          for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+            for (int e = 0; e < 2; ++e)
+              if (nt * 8 + 2 * t + e < n_a && (double)acc[nt][2 * h + e] >= bar) mask |= 1u << (nt * 8 + 2 * t + e);
+        }
+        mask |= __shfl_xor_sync(0xffffffffu, mask, 1);
+        mask |= __shfl_xor_sync(0xffffffffu, mask, 2);
+        if (t == 0 && j < C) s_fill[j] = (int)mask;
+      }
+    }
+    __syncthreads();
+    if (tid < C && !s_app[tid]) {
+      unsigned mask = (unsigned)s_fill[tid];
+      const int n = __popc(mask);
+      s_ccnt[tid] = (unsigned char)min(n, 5);
+      if (n <= 4) {
+        for (int k = 0; k < n; ++k) {   // ascending new-row index
+          const int a = __ffs(mask) - 1;
+          mask &= mask - 1;
+          s_cont[4 * tid + k] = (unsigned char)a;
+        }
+      }
+    }
+  } else if (tid < C && !s_app[tid]) {
+    const int j = tid;
+    const double eps = 0.5 * (double)s_thr[j];
+    const double best_old = s_cls[j] == UNSURE ? s_hi[j] : s_lo[j];
+    // one pass over the batched products with the new rows, ascending a: rows are kept while they reach the
+    // running bar (which only rises: a superset) and pruned against the final bar afterwards
+    float gm = -INFINITY;
+    int cntc = 0, ca[4] = {0, 0, 0, 0};
+    float cp[4] = {0.f, 0.f, 0.f, 0.f};
+    const float* gcol = p.gramT + (int64_t)u * p.Cmax * p.Cmax + j;
+#pragma unroll 8
+    for (int a = 0; a < n_a; ++a) {
+      const float pv = gcol[(int64_t)s_creator[a] * p.Cmax];
+      gm = fmaxf(gm, pv);
+      if ((double)pv >= fmax(best_old, (double)gm - eps) - eps) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (k == cntc) { ca[k] = a; cp[k] = pv; }
+        ++cntc;
+      }
+    }
+    int kept = cntc;
+    if (cntc <= 4) {
+      const double bar = fmax(best_old, (double)gm - eps) - eps;
+      kept = 0;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (k < cntc && (double)cp[k] >= bar) {
+          s_cont[4 * j + kept] = (unsigned char)ca[k];
+          ++kept;
+        }
+      }
+    }
+    s_ccnt[j] = (unsigned char)min(kept, 5);
+  }
+  __syncthreads();
+  // ---- 6: round 2: merged tokens whose target is still open: the old candidates of a token without an exact best
+  //      (unless it has one candidate and no new row in reach), and the new rows in reach ----
+  if (tid == 0) s_np = 0;
+  {
+    const bool mg = tid < C && !s_app[tid];
+    const bool scored = mg && s_cls[tid] == UNSURE;
+    const int nnew = mg ? s_ccnt[tid] : 0;
+    const int nold = (mg && !scored) ? s_nold[tid] : 0;
+    bool exh = mg && (nnew > 4 || (!scored && nold == 0));   // (no old candidate cannot happen; scanned if it does)
+    int c = 0;
+    bool single = false;
+    if (mg && !exh) {
+      if (!scored && nold == 1 && nnew == 0) single = true;
+      else c = nold + nnew;
+      if (c > kPairPerTok) { exh = true; c = 0; }
+    }
+    const int start = block_scan(c);
+    if (start + c > kPairCap2) { exh = mg; c = 0; single = false; }
+    s_pstart[tid] = start; s_pcnt[tid] = c;
+    s_fill[tid] = single ? -1 : ((mg && !scored && !exh && c > 0) ? 0 : -2);   // -1: take the only candidate; 0: list the old candidates; -2: none
+    s_exh[tid] = exh ? 1 : 0;
+    if (mg && !exh && c > 0) {   // the new rows go behind the old candidates
+      for (int k = 0; k < nnew; ++k) {
+        s_prow[start + nold + k] = (int)m + s_cont[4 * tid + k];
+        s_ptok[start + nold + k] = (unsigned short)tid;
+      }
+    }
+    const unsigned wend = __reduce_max_sync(0xffffffffu, (unsigned)(c > 0 ? start + c : 0));
+    if (lane == 0 && wend > 0) atomicMax(&s_np, (int)wend);
+    const int ne = __syncthreads_count(exh);
+    if (tid == 0) s_nexh += ne;
+  }
+  __syncthreads();
+  for (int it = tid; it < nitems; it += kPrunedThreads) {
+    const int sp = it / C, j = it % C;
+    const int mode = s_fill[j];
+    if (mode == -2) continue;
+    const int gi = s_gmaxi[j];
+    const float gmax = __int_as_float(gi >= 0 ? gi : gi ^ 0x7fffffff);
+    const int64_t o = obase + sp * ostep + (int64_t)j * kTopK;
+    if (!(p.candV[o] >= gmax - s_thr[j])) continue;
+    int i[kTopK];
+    load_cand_rows(p.candI, o, i);
+    if (mode == -1) {
+#pragma unroll
+      for (int k = 0; k < kTopK; ++k)
+        if (i[k] >= p.S) s_barg[j] = i[k];
+      continue;
+    }
+    int c = 0;
+#pragma unroll
+    for (int k = 0; k < kTopK; ++k)
+      if (i[k] >= p.S) ++c;
+    if (c == 0) continue;
+    int w = s_pstart[j] + atomicAdd(&s_fill[j], c);   // (stays >= 0: a list mode)
+#pragma unroll
+    for (int k = 0; k < kTopK; ++k) {
+      if (i[k] >= p.S) {
+        s_prow[w] = i[k];
+        s_ptok[w] = (unsigned short)j;
+        ++w;
+      }
+    }
+  }
+  __syncthreads();
+  {
+    const int np2 = min(s_np, kPairCap2);
+    exact_pairs(np2);
+    if (tid == 0) s_npairs += np2;
+  }
+  for (int j = warp; j < C; j += kPrunedWarps) {   // lists that did not fit: every row in question exactly
+    if (!s_exh[j] || s_app[j]) continue;
+    double gam[CH], bet[CH], kb[CH];
+#pragma unroll
+    for (int c = 0; c < CH; ++c) {
+      gam[c] = (double)lnwH[lane + 32 * c]; bet[c] = (double)lnbH[lane + 32 * c];
+      kb[c] = kbarU.at(j, lane + 32 * c, gam[c], bet[c]);
+    }
+    double best = -INFINITY;
+    int arg = -1;
+    if (s_cls[j] == UNSURE) { best = s_hi[j]; arg = s_barg[j]; }
+    else {
+      for (int64_t i = p.S; i < m; ++i) {
+        const double acc = warp_sim<CH>(kb, p.sumK + (rowBase + i) * D, p.kmu[rowBase + i], p.krstd[rowBase + i], gam, bet, lane);
+        if (acc > best) { best = acc; arg = (int)i; }
+      }
+    }
+    for (int a = 0; a < n_a; ++a) {
+      const int jc = s_creator[a];
+      const double2 hs = p.kbarHatStat[tokBase + jc];
+      double acc = 0.0;
+#pragma unroll
+      for (int c = 0; c < CH; ++c) {
+        const double hat = gam[c] * ((kbarU.at(jc, lane + 32 * c, gam[c], bet[c]) - hs.x) * hs.y) + bet[c];
+        acc += kb[c] * hat;
+      }
+      acc = warp_sum_d(acc);
+      if (acc > best) { best = acc; arg = (int)m + a; }
+    }
+    if (lane == 0) { s_hi[j] = best; s_barg[j] = arg; }
+  }
+  __syncthreads();
+  const bool merged = tid < C && !s_app[tid];
+  if (merged) {
+    double best = -INFINITY;
+    int arg = s_barg[tid];   // (a token with one candidate and no new row in reach: that candidate)
+    if (s_cls[tid] == UNSURE || s_exh[tid]) best = s_hi[tid];
+    if (!s_exh[tid]) {
+      const int st0 = s_pstart[tid];
+      for (int q = st0; q < st0 + s_pcnt[tid]; ++q) {   // ties: the lowest row (old rows before new ones)
+        const double v = s_pval[q];
+        const int i = s_prow[q];
+        if (v > best || (v == best && i < arg)) { best = v; arg = i; }
+      }
+    }
+    s_pi[tid] = arg;
+  }
+  const int nm = __syncthreads_count(merged);
+  // ---- 7: order merged tokens by (row, token); publish ----
+  {
+    unsigned* ekey = reinterpret_cast<unsigned*>(s_prow);   // (the pair list is idle here)
+    if (tid < nsort) {
+      const int pj = tid < C ? s_pi[tid] : -1;
+      unsigned kq = pj >= 0 ? (((unsigned)pj << 9) | (unsigned)tid) : 0xffffffffu;   // rows < 2^23, tokens < 2^9
+      if (tid < C) {
+        p.pi[tokBase + tid] = pj;
+        p.creator[tokBase + tid] = s_creator[tid];
+      }
+      int zero = 0;
+      if (nsort == 128) sort_n<unsigned, 128>(kq, zero, ekey + 256, reinterpret_cast<int*>(s_pval), tid);
+      else sort_n<unsigned, 256>(kq, zero, ekey + 256, reinterpret_cast<int*>(s_pval), tid);
+      ekey[tid] = kq;
+      asm volatile("bar.sync 2, %0;" ::"r"(nsort) : "memory");
+      if (kq != 0xffffffffu) {
+        const int rowq = (int)(kq >> 9);
+        p.sorted[tokBase + tid] = (int)(kq & 511u);
+        const bool head = tid == 0 || (int)(ekey[tid - 1] >> 9) != rowq;
+        if (head && rowq >= m) p.segnew[tokBase + (rowq - (int)m)] = tid;
+      }
+    }
+  }
+  if (tid == 0) {
+    p.nmerge[u] = nm;
+    atomicAdd(&p.counters[0], s_nexh);
+    atomicAdd(&p.counters[1], s_npairs);
+    atomicAdd(&p.counters[2], C);
+  }
+}
+
+// ------------------------------------------------------------------------------------------
 // 4. application: one warp per touched row
 
 struct FoldApplyParams {
@@ -1488,7 +2050,11 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
     const bool roomy = R * st->U <= 148;
 #define KVM_DECIDE(DD, PP, RR) cudaLaunchKernelEx(&lc, fold_decide_kernel<DD, PP, RR>, p)
     const bool rk = st->recomputeK;
-    if (D == 128) {
+    if (st->U > 148 && a.n_append > 0) {   // (R == 1 here) more units than SMs: bounds first, few exact pairs
+      lc.blockDim = dim3(kPrunedThreads);
+      if (D == 128) { if (rk) cudaLaunchKernelEx(&lc, fold_decide_pruned_kernel<128, true>, p); else cudaLaunchKernelEx(&lc, fold_decide_pruned_kernel<128, false>, p); }
+      else { if (rk) cudaLaunchKernelEx(&lc, fold_decide_pruned_kernel<64, true>, p); else cudaLaunchKernelEx(&lc, fold_decide_pruned_kernel<64, false>, p); }
+    } else if (D == 128) {
       if (roomy) { if (rk) KVM_DECIDE(128, 1, true); else KVM_DECIDE(128, 1, false); }
       else { if (rk) KVM_DECIDE(128, 2, true); else KVM_DECIDE(128, 2, false); }
     } else {

@@ -114,3 +114,18 @@ def test_small_appends_compute_their_products_in_the_decision_kernel_and_keys_ar
     # the same small-append shape below the size threshold keeps its fp64 keys: products inside the kernel only
     wl = synth.Workload("t", 1, 3, 3, 64, 64 * 14 + 9, 64, "sqrt", sqrt_coeff=3, r=16, seed=38)
     print(_sampled(wl, None, flags=kvm.FLAG_SERIAL_FOLDS))
+
+
+def test_bounds_first_decisions_head_dim_64_three_sink_rows_duplicated_keys():
+    """More units than SMs: the decision kernel that ranks the tokens by the filter's bounds first and scores
+    only the ones in doubt.  Head dimension 64, three sink rows (a sink row in reach takes a token's bounds
+    away), mixture keys (near-duplicates inside a block: new rows in reach of many tokens), with the batched
+    new-row products and with the products computed inside the kernel."""
+    from paper_2605_09877_b200 import kvm
+    wl = synth.Workload("t", 1, 160, 160, 64, 64 * 11 + 20, 64, "sqrt", sqrt_coeff=5, r=16, seed=39, kind="mixture", S=3)
+    params = synth.make_layer_params(wl, trivial=False)
+    units = [(0, 0), (0, 77), (0, 159)]
+    print(_sampled(wl, units, params=params, gate=True))
+    print(_sampled(wl, units, params=params, gate=True, flags=kvm.FLAG_SERIAL_FOLDS))
+    wl = synth.Workload("t", 5, 32, 32, 128, 128 * 9 + 3, 128, "fixed", fixed_slots=300, r=32, seed=40, S=2)
+    print(_sampled(wl, [(0, 0), (3, 11), (4, 31)], flags=kvm.FLAG_SERIAL_FOLDS))
