@@ -147,10 +147,10 @@ __device__ __forceinline__ void rope_rotate8(float (&out)[8], const float (&oth)
   }
 }
 
-// Eight bf16 channels starting at channel c8*8 of `row`, rotated when they lie in the rotary range.
-__device__ __forceinline__ void rope8(const __nv_bfloat16* __restrict__ row, int c8, int r,
-                                      const float2* __restrict__ cs, float (&out)[8]) {
-  const uint4 raw = *reinterpret_cast<const uint4*>(row + c8 * 8);
+// Eight bf16 channels starting at channel c8*8 of a row: `raw` holds them, `rawo` their partners of the other
+// rotary half (only read when the channels lie in the rotary range); rotated when they do.
+__device__ __forceinline__ void rope8_from(const uint4& raw, const uint4& rawo, int c8, int r,
+                                           const float2* __restrict__ cs, float (&out)[8]) {
   const __nv_bfloat162* pv = reinterpret_cast<const __nv_bfloat162*>(&raw);
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -161,7 +161,6 @@ __device__ __forceinline__ void rope8(const __nv_bfloat16* __restrict__ row, int
   if (ch0 >= r) return;
   const int half = r >> 1;
   const bool lower = ch0 < half;
-  const uint4 rawo = *reinterpret_cast<const uint4*>(row + (lower ? ch0 + half : ch0 - half));
   const __nv_bfloat162* po = reinterpret_cast<const __nv_bfloat162*>(&rawo);
   float oth[8];
 #pragma unroll
@@ -170,6 +169,11 @@ __device__ __forceinline__ void rope8(const __nv_bfloat16* __restrict__ row, int
     oth[2 * i] = o.x; oth[2 * i + 1] = o.y;
   }
   rope_rotate8(out, oth, reinterpret_cast<const float4*>(cs + (lower ? ch0 : ch0 - half)), lower);
+}
+// where the partners of chunk c8 start (any chunk outside the rotary range: itself, never used)
+__device__ __forceinline__ int rope_partner8(int c8, int r) {
+  const int ch0 = c8 * 8, half = r >> 1;
+  return ch0 >= r ? ch0 : (ch0 < half ? ch0 + half : ch0 - half);
 }
 
 // Eight values -> eight fp16, clamped; nsat counts the values that did not fit.  A clamped value reads
@@ -194,6 +198,10 @@ __device__ __forceinline__ uint4 pack8_sat(const float (&x)[8], int& nsat) {
   return o;
 }
 
+// Tokens per thread of the 16-byte kernels: all loads of a thread's tokens are issued before the first value
+// is looked at (a thread with one token had 32 bytes in flight, and a CTA lived for 16 tokens).
+constexpr int kIngestTok = 4;
+
 __global__ void __launch_bounds__(256) ingest_kv_vec_kernel(
     __half* __restrict__ stK, __half* __restrict__ stV, float* __restrict__ stG, __half* __restrict__ ringK,
     __half* __restrict__ ringV, float* __restrict__ ringG, const __nv_bfloat16* __restrict__ k,
@@ -204,36 +212,53 @@ __global__ void __launch_bounds__(256) ingest_kv_vec_kernel(
   const int u = blockIdx.y;
   const int b = u / Hkv, hk = u % Hkv;
   const int w8 = d / 8;                       // 16-byte chunks per row
-  const int tpb = 256 / w8;                   // tokens per block
-  const int64_t j = (int64_t)blockIdx.x * tpb + threadIdx.x / w8;
+  const int tpb = 256 / w8;                   // tokens per pass of the block
+  const int64_t j0 = (int64_t)blockIdx.x * tpb * kIngestTok + threadIdx.x / w8;
   const int c8 = threadIdx.x % w8;
-  if (j >= n) return;
-  float kx[8], vx[8];
-  rope8(k + b * sk0 + hk * sk1 + j * sk2, c8, r, ropeCS + j * (r >> 1), kx);
-  {
-    const uint4 raw = *reinterpret_cast<const uint4*>(v + b * sv0 + hk * sv1 + j * sv2 + c8 * 8);
-    const __nv_bfloat162* pv = reinterpret_cast<const __nv_bfloat162*>(&raw);
+  const int po = rope_partner8(c8, r);
+  const bool rot = c8 * 8 < r;
+  uint4 kr[kIngestTok], ko[kIngestTok], vr[kIngestTok];
+  float g[kIngestTok];
+#pragma unroll
+  for (int it = 0; it < kIngestTok; ++it) {
+    const int64_t j = j0 + (int64_t)it * tpb;
+    kr[it] = ko[it] = vr[it] = make_uint4(0u, 0u, 0u, 0u);
+    g[it] = 1.0f;
+    if (j < n) {
+      const __nv_bfloat16* krow = k + b * sk0 + hk * sk1 + j * sk2;
+      kr[it] = *reinterpret_cast<const uint4*>(krow + c8 * 8);
+      if (rot) ko[it] = *reinterpret_cast<const uint4*>(krow + po);
+      vr[it] = *reinterpret_cast<const uint4*>(v + b * sv0 + hk * sv1 + j * sv2 + c8 * 8);
+      if (gate) g[it] = gate[b * sg0 + hk * sg1 + j * sg2];
+    }
+  }
+  int nsat = 0;
+#pragma unroll
+  for (int it = 0; it < kIngestTok; ++it) {
+    const int64_t j = j0 + (int64_t)it * tpb;
+    if (j >= n) continue;
+    float kx[8], vx[8];
+    rope8_from(kr[it], ko[it], c8, r, ropeCS + j * (r >> 1), kx);
+    const __nv_bfloat162* pv = reinterpret_cast<const __nv_bfloat162*>(&vr[it]);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const float2 f = __bfloat1622float2(pv[i]);
       vx[2 * i] = f.x; vx[2 * i + 1] = f.y;
     }
+    const uint4 kk = pack8_sat(kx, nsat), vv = pack8_sat(vx, nsat);
+    const int64_t row = (int64_t)u * stRows + nhist + j;
+    reinterpret_cast<uint4*>(stK + row * d)[c8] = kk;
+    reinterpret_cast<uint4*>(stV + row * d)[c8] = vv;
+    if (c8 == 0) stG[row] = g[it];
+    const int64_t t = pos0 + j;
+    if (t >= tail_start) {
+      const int64_t rrow = (int64_t)u * ringCap + t % ringLen;
+      reinterpret_cast<uint4*>(ringK + rrow * d)[c8] = kk;
+      reinterpret_cast<uint4*>(ringV + rrow * d)[c8] = vv;
+      if (c8 == 0) ringG[rrow] = g[it];
+    }
   }
-  int nsat = 0;
-  const uint4 kk = pack8_sat(kx, nsat), vv = pack8_sat(vx, nsat);
   if (nsat) atomicAdd(sat_counter, nsat);
-  const float g = gate ? gate[b * sg0 + hk * sg1 + j * sg2] : 1.0f;
-  const int64_t row = (int64_t)u * stRows + nhist + j;
-  reinterpret_cast<uint4*>(stK + row * d)[c8] = kk;
-  reinterpret_cast<uint4*>(stV + row * d)[c8] = vv;
-  if (c8 == 0) stG[row] = g;
-  const int64_t t = pos0 + j;
-  if (t >= tail_start) {
-    const int64_t rrow = (int64_t)u * ringCap + t % ringLen;
-    reinterpret_cast<uint4*>(ringK + rrow * d)[c8] = kk;
-    reinterpret_cast<uint4*>(ringV + rrow * d)[c8] = vv;
-    if (c8 == 0) ringG[rrow] = g;
-  }
 }
 
 __global__ void __launch_bounds__(256) ingest_q_vec_kernel(__half* __restrict__ stQ, const __nv_bfloat16* __restrict__ q,
@@ -243,13 +268,30 @@ __global__ void __launch_bounds__(256) ingest_q_vec_kernel(__half* __restrict__ 
   const int bh = blockIdx.y;
   const int b = bh / Hq, h = bh % Hq;
   const int w8 = d / 8, tpb = 256 / w8;
-  const int64_t j = (int64_t)blockIdx.x * tpb + threadIdx.x / w8;
+  const int64_t j0 = (int64_t)blockIdx.x * tpb * kIngestTok + threadIdx.x / w8;
   const int c8 = threadIdx.x % w8;
-  if (j >= n) return;
-  float qx[8];
-  rope8(q + b * sq0 + h * sq1 + j * sq2, c8, r, ropeCS + j * (r >> 1), qx);
+  const int po = rope_partner8(c8, r);
+  const bool rot = c8 * 8 < r;
+  uint4 qr[kIngestTok], qo[kIngestTok];
+#pragma unroll
+  for (int it = 0; it < kIngestTok; ++it) {
+    const int64_t j = j0 + (int64_t)it * tpb;
+    qr[it] = qo[it] = make_uint4(0u, 0u, 0u, 0u);
+    if (j < n) {
+      const __nv_bfloat16* qrow = q + b * sq0 + h * sq1 + j * sq2;
+      qr[it] = *reinterpret_cast<const uint4*>(qrow + c8 * 8);
+      if (rot) qo[it] = *reinterpret_cast<const uint4*>(qrow + po);
+    }
+  }
   int nsat = 0;
-  reinterpret_cast<uint4*>(stQ + ((int64_t)bh * Tcall + j) * d)[c8] = pack8_sat(qx, nsat);
+#pragma unroll
+  for (int it = 0; it < kIngestTok; ++it) {
+    const int64_t j = j0 + (int64_t)it * tpb;
+    if (j >= n) continue;
+    float qx[8];
+    rope8_from(qr[it], qo[it], c8, r, ropeCS + j * (r >> 1), qx);
+    reinterpret_cast<uint4*>(stQ + ((int64_t)bh * Tcall + j) * d)[c8] = pack8_sat(qx, nsat);
+  }
   if (nsat) atomicAdd(sat_counter, nsat);
 }
 
@@ -398,7 +440,7 @@ int launch_ingest(State* st, const IngestArgs& a, cudaStream_t s) {
     return launches + 2;
   }
   if (rope_ok && al16(a.k, a.sk) && al16(a.v, a.sv)) {
-    dim3 grid((unsigned)((a.n + tpb - 1) / tpb), st->U);
+    dim3 grid((unsigned)((a.n + tpb * kIngestTok - 1) / (tpb * kIngestTok)), st->U);
     ingest_kv_vec_kernel<<<grid, 256, 0, s>>>(st->stK, st->stV, st->stG, st->ringK, st->ringV, st->ringG, a.k,
                                               a.v, a.gate, st->ropeCS, a.sk[0], a.sk[1], a.sk[2], a.sv[0],
                                               a.sv[1], a.sv[2], a.sg[0], a.sg[1], a.sg[2], st->Hkv, d, st->r,
@@ -415,7 +457,7 @@ int launch_ingest(State* st, const IngestArgs& a, cudaStream_t s) {
     ++launches;
   }
   if (rope_ok && al16(a.q, a.sq)) {
-    dim3 grid((unsigned)((a.n + tpb - 1) / tpb), st->B * st->Hq);
+    dim3 grid((unsigned)((a.n + tpb * kIngestTok - 1) / (tpb * kIngestTok)), st->B * st->Hq);
     ingest_q_vec_kernel<<<grid, 256, 0, s>>>(st->stQ, a.q, st->ropeCS, a.sq[0], a.sq[1], a.sq[2], st->Hq, d,
                                              st->r, st->Tcall, a.n, st->status + 4);
     ++launches;
