@@ -1634,14 +1634,15 @@ __global__ void __launch_bounds__(256, 2) fold_apply_rows4_kernel(FoldApplyParam
   constexpr int NC = 4 * NI;          // channels per lane
   constexpr double inv_d = 1.0 / D;   // D is a power of two: multiplying is dividing, exactly
   __shared__ int s_pi[kMaxBlock], s_sorted[kMaxBlock], s_creator[kMaxBlock], s_segnew[kMaxBlock];
+  __shared__ int s_nmerge;
   // the routing filter of the next fold may start its set-up now; it waits for this grid to finish
   // before it reads the readout keys written here
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int u = blockIdx.y, hk = u % p.Hkv;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, sub = lane & 7;
-  const int q = (blockIdx.x * 8 + warp) * kApplyRowsPerWarp + (lane >> 3);
   const int64_t tokBase = (int64_t)u * p.Cmax;
   if (!p.all_append) {   // the decisions of this unit, read once per CTA instead of chased per warp
+    if (threadIdx.x == 0) s_nmerge = p.nmerge[u];
     for (int i = threadIdx.x; i < p.C; i += 256) {
       s_pi[i] = p.pi[tokBase + i];
       s_sorted[i] = p.sorted[tokBase + i];
@@ -1650,7 +1651,6 @@ __global__ void __launch_bounds__(256, 2) fold_apply_rows4_kernel(FoldApplyParam
     }
     __syncthreads();
   }
-  if ((blockIdx.x * 8 + warp) * kApplyRowsPerWarp >= p.C) return;   // (whole warp)
   const int64_t rowBase = (int64_t)u * p.Mcap;
   KbarRows<D, RK> kbarU;
   kbarU.k64 = p.kbar64 + tokBase * D; kbarU.k16 = p.ok + (int64_t)u * p.unit_stride;
@@ -1659,11 +1659,15 @@ __global__ void __launch_bounds__(256, 2) fold_apply_rows4_kernel(FoldApplyParam
   const float* lnbH = p.ln_b + hk * D;
   const __half* ovU = p.ov + (int64_t)u * p.unit_stride;
   const float* ogU = p.og + (int64_t)u * p.gate_stride;
-  const int nmerge = p.all_append ? 0 : p.nmerge[u];
+  const int nmerge = p.all_append ? 0 : s_nmerge;
   const int m = (int)p.m;
 
+  // A warp takes groups of four row slots in turn (with few CTAs per unit the stores of one group drain
+  // while the next group's rows are fetched, and the decisions are read once for more work).
   // task 0: the q-th appended row; task 1: the segment of an old row whose head sits at sorted[q]
+  for (int qg = blockIdx.x * 8 + warp; qg * kApplyRowsPerWarp < p.C; qg += gridDim.x * 8)
   for (int task = 0; task < 2; ++task) {
+    const int q = qg * kApplyRowsPerWarp + (lane >> 3);
     bool act = q < p.C;
     int rowi = 0, seg = -1, jc = -1;
     if (act) {
@@ -2080,7 +2084,10 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
   if (a.before_apply && cudaStreamWaitEvent(s, a.before_apply, 0) != cudaSuccess) return -1000000;
   KernelTimer kt(st, 5, s);
   if (apply_uses_rows4(st)) {
-    dim3 grid((C + kApplyRowsPerCta - 1) / kApplyRowsPerCta, st->U);
+    // CTAs per unit: one when the units alone fill the GPU's CTA slots (measured at 256 and 2048 units: 1 beats
+    // 2, 4 and 8), else enough to fill them, at most one per 32 row slots
+    const int R = std::max(1, std::min(2 * 148 / st->U, (C + kApplyRowsPerCta - 1) / kApplyRowsPerCta));
+    dim3 grid(R, st->U);
     if (D == 128) { if (st->recomputeK) fold_apply_rows4_kernel<128, true><<<grid, 256, 0, s>>>(q); else fold_apply_rows4_kernel<128, false><<<grid, 256, 0, s>>>(q); }
     else { if (st->recomputeK) fold_apply_rows4_kernel<64, true><<<grid, 256, 0, s>>>(q); else fold_apply_rows4_kernel<64, false><<<grid, 256, 0, s>>>(q); }
   } else {
