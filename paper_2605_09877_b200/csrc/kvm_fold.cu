@@ -166,6 +166,12 @@ __global__ void __launch_bounds__(256, 2) kbar_kernel(const __half* __restrict__
     }
   }
   n2 = group8_sum_d(n2);
+  if (live && sub == 0) {
+    kbarNorm[((int64_t)g * U + u) * Cmax + j] = (float)sqrt(n2) * 1.000001f;
+    if (RK) kbarStat[((int64_t)g * U + u) * Cmax + j] = make_double2(mean, rstd);
+  }
+  // (write_hat < 0: the decision kernel takes these statistics itself, for the few tokens that create rows)
+  if (write_hat < 0) return;
   // LN_s applied to kbar itself: the readout key of the row that this token would create
   sum = 0.0;
 #pragma unroll
@@ -188,11 +194,7 @@ __global__ void __launch_bounds__(256, 2) kbar_kernel(const __half* __restrict__
     }
     if (live && write_hat) *reinterpret_cast<uint2*>(kbarHatH + oh + x) = *reinterpret_cast<const uint2*>(kh);
   }
-  if (live && sub == 0) {
-    kbarNorm[((int64_t)g * U + u) * Cmax + j] = (float)sqrt(n2) * 1.000001f;
-    kbarHatStat[((int64_t)g * U + u) * Cmax + j] = make_double2(mu2, rs2);
-    if (RK) kbarStat[((int64_t)g * U + u) * Cmax + j] = make_double2(mean, rstd);
-  }
+  if (live && sub == 0) kbarHatStat[((int64_t)g * U + u) * Cmax + j] = make_double2(mu2, rs2);
 }
 
 // Rows that the last fold touched are current in one readout copy only: bring them over to the
@@ -350,6 +352,7 @@ struct FoldDecideParams {
   int64_t Mcap, m;
   int C, Cmax, Hkv, S, n_append, nsplit;
   float thr_coeff;
+  double ln_eps;
 };
 
 constexpr int kPairCap = 1536;
@@ -950,6 +953,7 @@ __global__ void __launch_bounds__(kPrunedThreads, 4) fold_decide_pruned_kernel(F
   __shared__ int s_np, s_nexh, s_nunc, s_npairs;
   __shared__ int s_wsum[kPrunedWarps];
   __shared__ __align__(16) __half s_hat[kGramOnTheFly * HS];
+  __shared__ double2 s_hs[kGramOnTheFly];   // (mean, rstd) of LN_s(kbar_c) for the creators of a small fold
 
   const int u = blockIdx.y, hk = u % p.Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -974,6 +978,10 @@ __global__ void __launch_bounds__(kPrunedThreads, 4) fold_decide_pruned_kernel(F
   if (tid < p.Cmax) p.segnew[tokBase + tid] = -1;
   __syncthreads();
 
+  // a fold that appends few rows computes the products with them itself, and the statistics of their keys
+  const bool otf = n_a <= p.otf_max;
+  // (mean, rstd) of LN_s(kbar_c) of new row a, created by token jc
+  auto hat_stat = [&](int a, int jc) { return otf ? s_hs[a] : p.kbarHatStat[tokBase + jc]; };
   // exact fp64 value of the pairs [0, np) of the list: rows < m are rows of the state, kbar_j . LN_s(s^K_i);
   // rows >= m are rows this fold appends, kbar_j . LN_s(kbar_c) with c the creator of row (i - m).  One warp
   // per pair, eight pairs in flight per warp.
@@ -996,7 +1004,7 @@ __global__ void __launch_bounds__(kPrunedThreads, 4) fold_decide_pruned_kernel(F
             acc += kbarU.at(j, lane + 32 * c, gam[c], bet[c]) * (gam[c] * ((sk[lane + 32 * c] - mu) * rs) + bet[c]);
         } else {
           const int jc = s_creator[i - (int)m];
-          const double2 hs = p.kbarHatStat[tokBase + jc];
+          const double2 hs = hat_stat(i - (int)m, jc);
 #pragma unroll
           for (int c = 0; c < CH; ++c) {
             const double hat = gam[c] * ((kbarU.at(jc, lane + 32 * c, gam[c], bet[c]) - hs.x) * hs.y) + bet[c];
@@ -1198,16 +1206,37 @@ __global__ void __launch_bounds__(kPrunedThreads, 4) fold_decide_pruned_kernel(F
   // ---- 5: the new rows in reach of every merged token.  best_old below is the exact best old similarity of a
   //      scored token, a lower bound of it for the others; products are within eps_j of the exact values, so a
   //      new row can only win when its product reaches max(best_old, best product - eps_j) - eps_j. ----
-  const bool otf = n_a <= p.otf_max;
   if (otf) {
     for (int e = tid; e < kGramOnTheFly * HS / 8; e += kPrunedThreads) reinterpret_cast<uint4*>(s_hat)[e] = make_uint4(0u, 0u, 0u, 0u);
+    {   // the memory-key kernel skipped these for such folds: eight lanes per creator, its arithmetic and order
+      constexpr int NI = D / 32, NC = 4 * NI;
+      constexpr double inv_d = 1.0 / D;
+      const int a = warp * 4 + (lane >> 3), sub = lane & 7;
+      const int jc = s_creator[min(a, n_a - 1)];   // (groups past the last creator compute a copy and store nothing)
+      double kb[NC];
+#pragma unroll
+      for (int i = 0; i < NI; ++i) {
+        double k4[4];
+        kbar_run4<D, RK>(kbarU, jc, 32 * i + 4 * sub, lnwH, lnbH, k4);
+        kb[4 * i] = k4[0]; kb[4 * i + 1] = k4[1]; kb[4 * i + 2] = k4[2]; kb[4 * i + 3] = k4[3];
+      }
+      double sum = 0.0;
+#pragma unroll
+      for (int c = 0; c < NC; ++c) sum += kb[c];
+      const double mu2 = group8_sum_d(sum) * inv_d;
+      double dev = 0.0;
+#pragma unroll
+      for (int c = 0; c < NC; ++c) dev += (kb[c] - mu2) * (kb[c] - mu2);
+      const double rs2 = 1.0 / sqrt(group8_sum_d(dev) * inv_d + p.ln_eps);
+      if (sub == 0 && a < n_a) s_hs[a] = make_double2(mu2, rs2);
+    }
     __syncthreads();
     double gam[CH], bet[CH];
 #pragma unroll
     for (int c = 0; c < CH; ++c) { gam[c] = (double)lnwH[lane + 32 * c]; bet[c] = (double)lnbH[lane + 32 * c]; }
     for (int a = warp; a < n_a; a += kPrunedWarps) {
       const int jc = s_creator[a];
-      const double2 hs = p.kbarHatStat[tokBase + jc];
+      const double2 hs = s_hs[a];
 #pragma unroll
       for (int c = 0; c < CH; ++c)
         s_hat[a * HS + lane + 32 * c] =
@@ -1408,7 +1437,7 @@ __global__ void __launch_bounds__(kPrunedThreads, 4) fold_decide_pruned_kernel(F
     }
     for (int a = 0; a < n_a; ++a) {
       const int jc = s_creator[a];
-      const double2 hs = p.kbarHatStat[tokBase + jc];
+      const double2 hs = hat_stat(a, jc);
       double acc = 0.0;
 #pragma unroll
       for (int c = 0; c < CH; ++c) {
@@ -1937,6 +1966,10 @@ int launch_refresh_rows(State* st, int64_t m, cudaStream_t s) {
 int launch_route_filter_tc(State* st, int64_t m, int nsplit, int slot, bool early_start, cudaStream_t s);
 int launch_gram_tc(State* st, int slot0, int nblk, cudaStream_t s);
 
+// Folds that compute their new-row products themselves (no batched product: want_gram false) and run the
+// decision kernel for many units take the statistics of LN_s(kbar_c) there, for the creators only.
+static bool hat_stats_in_decide(const State* st) { return st->U > 148 && gram_from(st) > 0; }
+
 int launch_kbar(State* st, const __half* ok, int64_t unit_stride, int nblk, int slot0, bool want_gram, cudaStream_t s) {
   KernelTimer kt(st, 2, s);
   const int C = st->C, D = st->d;
@@ -1950,7 +1983,8 @@ int launch_kbar(State* st, const __half* ok, int64_t unit_stride, int nblk, int 
   double2* kst = st->kbarStat + (int64_t)slot0 * U * st->Cmax;
 #define KVM_KBAR(DD, RR)                                                                                                   \
   kbar_kernel<DD, RR><<<grid, 256, 0, s>>>(ok, unit_stride, st->ln_w, st->ln_b, k64, kh, kn, khat, khh, C, st->Cmax,        \
-                                           st->CbarRows, st->U, st->Hkv, st->r, (double)st->ln_eps, want_gram ? 1 : 0, kst)
+                                           st->CbarRows, st->U, st->Hkv, st->r, (double)st->ln_eps,                         \
+                                           want_gram ? 1 : (hat_stats_in_decide(st) ? -1 : 0), kst)
   if (D == 128) { if (st->recomputeK) KVM_KBAR(128, true); else KVM_KBAR(128, false); }
   else { if (st->recomputeK) KVM_KBAR(64, true); else KVM_KBAR(64, false); }
 #undef KVM_KBAR
@@ -2026,6 +2060,7 @@ int launch_fold(State* st, const FoldArgs& a, cudaStream_t s) {
     p.Mcap = st->Mcap; p.m = a.m;
     p.C = C; p.Cmax = st->Cmax; p.Hkv = st->Hkv; p.S = st->S; p.n_append = a.n_append; p.nsplit = nsplit;
     p.thr_coeff = route_thr_coeff(st);
+    p.ln_eps = (double)st->ln_eps;
     KernelTimer kt(st, 4, s);
     // CTAs per unit (measured on U = 1, 8, 32, 256): about 64 CTAs in all, at least two per unit while
     // 2U CTAs fit the GPU in one wave, at most eight, at least 16 tokens each - beyond that the
