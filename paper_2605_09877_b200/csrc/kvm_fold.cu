@@ -106,7 +106,7 @@ __device__ __forceinline__ double group8_sum_d(double v) {
 }
 
 template <int D, bool RK>
-__global__ void __launch_bounds__(256, 2) kbar_kernel(const __half* __restrict__ ok, int64_t unit_stride,
+__global__ void __launch_bounds__(256, RK ? 4 : 2) kbar_kernel(const __half* __restrict__ ok, int64_t unit_stride,
                                                       const float* __restrict__ ln_w, const float* __restrict__ ln_b,
                                                       double* __restrict__ kbar64, __half* __restrict__ kbarH,
                                                       float* __restrict__ kbarNorm, double2* __restrict__ kbarHatStat,
@@ -141,6 +141,36 @@ __global__ void __launch_bounds__(256, 2) kbar_kernel(const __half* __restrict__
   const double rstd = 1.0 / sqrt(group8_sum_d(dev) * inv_d + ln_eps);
   const int64_t o = (((int64_t)g * U + u) * Cmax + jj) * D;
   const int64_t oh = (((int64_t)g * U + u) * CbarRows + jj) * D;
+  if (RK && write_hat < 0) {
+    // Nothing below is kept in fp64 for such a launch: the fp64 memory key is recomputed where it is needed from
+    // (mean, rstd), which stay exact as above; what is written here - the fp16 key for the routing filter and its
+    // norm for the filter's window - only has to be as good as an fp16 operand, so the affine map runs in fp32.
+    // (|fp16(fp32 result) - kbar| exceeds half an fp16 ulp by < 2^-22 of the operands' magnitudes, inside the
+    // 2^-13 |a| |b| that the window keeps in reserve; the norm is rounded up by more than its fp32 summation error.)
+    const float mean_f = (float)mean, rstd_f = (float)rstd;
+    float n2f = 0.f;
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+      const int x = 32 * i + 4 * sub;
+      const float4 w4 = *reinterpret_cast<const float4*>(ln_w + hk * D + x), b4 = *reinterpret_cast<const float4*>(ln_b + hk * D + x);
+      const float wv[4] = {w4.x, w4.y, w4.z, w4.w}, bv[4] = {b4.x, b4.y, b4.z, b4.w};
+      alignas(8) __half kh[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float tf = fmaf(wv[e], ((float)val[4 * i + e] - mean_f) * rstd_f, bv[e]);
+        kh[e] = __float2half_rn(tf);
+        n2f = fmaf(tf, tf, n2f);
+      }
+      if (live) *reinterpret_cast<uint2*>(kbarH + oh + x) = *reinterpret_cast<const uint2*>(kh);
+    }
+#pragma unroll
+    for (int o2 = 4; o2 > 0; o2 >>= 1) n2f += __shfl_xor_sync(0xffffffffu, n2f, o2);
+    if (live && sub == 0) {
+      kbarNorm[((int64_t)g * U + u) * Cmax + j] = sqrtf(n2f) * 1.00002f;
+      kbarStat[((int64_t)g * U + u) * Cmax + j] = make_double2(mean, rstd);
+    }
+    return;
+  }
   double kb[NC];
   double n2 = 0.0;
 #pragma unroll
