@@ -53,7 +53,12 @@ struct RouteTcCfg {
   static constexpr int TILE_BYTES = NKB * BOX_BYTES;
   static constexpr int OFF_A = 0;
   static constexpr int OFF_B = OFF_A + MT * TILE_BYTES;
-  static constexpr int OFF_BAR = OFF_B + NS * TILE_BYTES;
+  // the first two records of every token (32 products each), [record][16-byte piece][token]: with the list
+  // restarted at nearly every new maximum a token rarely has more, and a record costs eight 16-byte stores
+  // that every lane of a warp waits for whenever one of its 32 tokens records
+  static constexpr int OFF_REC = OFF_B + NS * TILE_BYTES;
+  static constexpr int REC_SLOTS = 2;
+  static constexpr int OFF_BAR = OFF_REC + REC_SLOTS * 8 * 256 * 16;
   static constexpr int SMEM_BYTES = (OFF_BAR + 256 + 1024) > 120 * 1024 ? (OFF_BAR + 256 + 1024) : 120 * 1024;
   static constexpr uint32_t TMEM_COLS = 512;   // [buffer][M tile] x 128 columns
 };
@@ -171,6 +176,11 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
       const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
       int nrec = 0;
       int sink_rec = 0;            // 1 once the record of the chunk that holds the sink rows sits in slot 0
+      // records 0 and 1: products in shared memory, first row / valid rows / maximum in registers
+      uint4* srec = reinterpret_cast<uint4*>(base + Cfg::OFF_REC) + tok;
+      int rrow[2] = {0, 0};
+      uint32_t rval[2] = {0u, 0u};
+      float rmax[2] = {-INFINITY, -INFINITY};
       float mx = -INFINITY;        // running maximum over rows >= S of this split
       const bool live = tok < p.C;   // (rows of the M tile past the block record nothing)
       const float thr = live ? p.thr_coeff * p.kbarNorm[(int64_t)u * p.Cmax + tok] + 1e-5f : 0.f;
@@ -256,8 +266,13 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
 #pragma unroll
         for (int c4 = 0; c4 < 4; ++c4) {
           if (live && ca[c4] >= cut) {   // record the chunk: 128 bytes of products, as they are
-            if (nrec < kChunkCap) {
-              uint32_t (&r)[32] = rr[c4];
+            uint32_t (&r)[32] = rr[c4];
+            if (nrec < Cfg::REC_SLOTS) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) srec[(nrec * 8 + i) * 256] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+              if (nrec == 0) { rrow[0] = row0 + c4 * 32; rval[0] = va[c4]; rmax[0] = ca[c4]; }
+              else { rrow[1] = row0 + c4 * 32; rval[1] = va[c4]; rmax[1] = ca[c4]; }
+            } else if (nrec < kChunkCap) {
               uint4* dst = reinterpret_cast<uint4*>(p.chunkVal + (o + nrec) * 32);
 #pragma unroll
               for (int i = 0; i < 8; ++i) dst[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
@@ -278,22 +293,37 @@ route_filter_tc_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_co
         for (int k = 0; k < kTopK; ++k) ci[k] = -1;
         int ncand = 0;
         const float cut = mx - thr;
-        const float4* cm4 = reinterpret_cast<const float4*>(p.chunkMax + o);
-        const float4 c0 = cm4[0], c1 = cm4[1], c2 = cm4[2], c3 = cm4[3];
-        const float cmv[16] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w, c2.x, c2.y, c2.z, c2.w, c3.x, c3.y, c3.z, c3.w};
         uint32_t kept = 0;
+        if (nrec > Cfg::REC_SLOTS) {   // (rare) records past the ones in shared memory
+          const float4* cm4 = reinterpret_cast<const float4*>(p.chunkMax + o);
+          const float4 c0 = cm4[0], c1 = cm4[1], c2 = cm4[2], c3 = cm4[3];
+          const float cmv[16] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w, c2.x, c2.y, c2.z, c2.w, c3.x, c3.y, c3.z, c3.w};
 #pragma unroll
-        for (int k = 0; k < 16; ++k) kept |= (k < nrec && cmv[k] >= cut) ? (1u << k) : 0u;
+          for (int k = Cfg::REC_SLOTS; k < 16; ++k) kept |= (k < nrec && cmv[k] >= cut) ? (1u << k) : 0u;
+        }
+        if (nrec > 0 && rmax[0] >= cut) kept |= 1u;
+        if (nrec > 1 && rmax[1] >= cut) kept |= 2u;
         while (kept) {
           const int k = __ffs(kept) - 1;
           kept &= kept - 1;
-          const int2 mt = p.chunkMeta[o + k];
-          const float4* v4 = reinterpret_cast<const float4*>(p.chunkVal + (o + k) * 32);
+          int2 mt;
           uint32_t hit = 0;
+          if (k < Cfg::REC_SLOTS) {
+            mt = k == 0 ? make_int2(rrow[0], (int)rval[0]) : make_int2(rrow[1], (int)rval[1]);
 #pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            const float4 v = v4[q];
-            hit |= ((v.x >= cut ? 1u : 0u) | (v.y >= cut ? 2u : 0u) | (v.z >= cut ? 4u : 0u) | (v.w >= cut ? 8u : 0u)) << (4 * q);
+            for (int q = 0; q < 8; ++q) {
+              const uint4 w = srec[(k * 8 + q) * 256];
+              const float4 v = make_float4(__uint_as_float(w.x), __uint_as_float(w.y), __uint_as_float(w.z), __uint_as_float(w.w));
+              hit |= ((v.x >= cut ? 1u : 0u) | (v.y >= cut ? 2u : 0u) | (v.z >= cut ? 4u : 0u) | (v.w >= cut ? 8u : 0u)) << (4 * q);
+            }
+          } else {
+            mt = p.chunkMeta[o + k];
+            const float4* v4 = reinterpret_cast<const float4*>(p.chunkVal + (o + k) * 32);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+              const float4 v = v4[q];
+              hit |= ((v.x >= cut ? 1u : 0u) | (v.y >= cut ? 2u : 0u) | (v.z >= cut ? 4u : 0u) | (v.w >= cut ? 8u : 0u)) << (4 * q);
+            }
           }
           hit &= (uint32_t)mt.y;
           while (hit) {
