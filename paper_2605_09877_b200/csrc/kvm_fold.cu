@@ -390,7 +390,7 @@ constexpr int kPairPerTok = 24;
 
 constexpr int kDecideThreads = 512;
 constexpr int kDecideWarps = kDecideThreads / 32;
-static_assert(kDecideThreads >= 2 * kMaxBlock, "the ranking loops give every token at least two threads");
+static_assert(kDecideThreads == 2 * kMaxBlock, "the ranking loops give every token two threads");
 
 // The candidate rows (kTopK entries, -1 = none) of one token in one split: two 16-byte loads.
 __device__ __forceinline__ void load_cand_rows(const int32_t* candI, int64_t o, int (&i)[kTopK]) {
@@ -475,7 +475,6 @@ __global__ void __launch_bounds__(kDecideThreads, PER_SM) fold_decide_kernel(Fol
   const int u = blockIdx.y, hk = u % p.Hkv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int C = p.C;
-  const int nsort = C <= 128 ? 128 : 256;   // threads that take part in the block-wide sorts
   const int R = gridDim.x;
   const int jlo = (int)blockIdx.x * ((C + R - 1) / R), jhi = min(C, jlo + (C + R - 1) / R);
   const int64_t m = p.m;
@@ -697,18 +696,35 @@ __global__ void __launch_bounds__(kDecideThreads, PER_SM) fold_decide_kernel(Fol
   }
   // ---- B: append selection: the n_a smallest scores, ties to the smaller token index ----
   if (n_a > 0) {
-    // sort (score, token) ascending; the first n_a entries are appended
-    if (tid < nsort) {
-      unsigned long long kbits = ~0ull;
-      if (tid < C) {   // order-preserving integer image of the double
-        const long long bits = __double_as_longlong(s_score[tid]);
-        kbits = (unsigned long long)bits ^ (bits < 0 ? ~0ull : 0x8000000000000000ull);
+    // rank of every token in the order (score, token): the n_a lowest are appended.  Counted, not sorted: two
+    // threads per token, each over half of the other tokens (a 256-entry bitonic sort is 36 dependent stages,
+    // six of them through shared memory and barriers; this is 128 independent compare-and-adds per thread).
+    {
+      unsigned long long* skey = reinterpret_cast<unsigned long long*>(s_pval);   // (the pair list is idle here)
+      if (tid < kMaxBlock) {
+        unsigned long long kbits = ~0ull;
+        if (tid < C) {   // order-preserving integer image of the double
+          const long long bits = __double_as_longlong(s_score[tid]);
+          kbits = (unsigned long long)bits ^ (bits < 0 ? ~0ull : 0x8000000000000000ull);
+        }
+        skey[tid] = kbits;
+        s_fill[tid] = 0;   // (idle here: the rank)
       }
-      int tok = tid;
-      // (the pair list is idle here)
-      if (nsort == 128) sort_n<unsigned long long, 128>(kbits, tok, reinterpret_cast<unsigned long long*>(s_pval), s_prow, tid);
-      else sort_n<unsigned long long, 256>(kbits, tok, reinterpret_cast<unsigned long long*>(s_pval), s_prow, tid);
-      if (tok < C) s_app[tok] = tid < n_a ? 1 : 0;
+      __syncthreads();
+      const int j = tid & (kMaxBlock - 1), h = tid / kMaxBlock;   // kDecideThreads == 2 kMaxBlock
+      if (j < C) {
+        const unsigned long long kj = skey[j];
+        const int half_n = (C + 1) / 2, i0 = h * half_n, i1 = min(C, i0 + half_n);
+        int cnt = 0;
+#pragma unroll 4
+        for (int i = i0; i < i1; ++i) {
+          const unsigned long long ki = skey[i];
+          cnt += (ki < kj || (ki == kj && i < j)) ? 1 : 0;
+        }
+        atomicAdd(&s_fill[j], cnt);
+      }
+      __syncthreads();
+      if (tid < C) s_app[tid] = s_fill[tid] < n_a ? 1 : 0;
     }
     __syncthreads();
     // rows are laid down in ascending token order: position of an appended token = appended tokens before it
@@ -801,9 +817,16 @@ __global__ void __launch_bounds__(kDecideThreads, PER_SM) fold_decide_kernel(Fol
             if (a0 + t < n_a) consider(a0 + t, acc[t]);
         }
       } else {
+        // (all loads of a batch in flight before the first product is looked at)
         const float* gcol = p.gramT + (int64_t)u * p.Cmax * p.Cmax + j;
-#pragma unroll 8
-        for (int a = 0; a < n_a; ++a) consider(a, gcol[(int64_t)s_creator[a] * p.Cmax]);
+        for (int a0 = 0; a0 < n_a; a0 += 16) {
+          float pv[16];
+#pragma unroll
+          for (int t = 0; t < 16; ++t) pv[t] = a0 + t < n_a ? gcol[(int64_t)s_creator[a0 + t] * p.Cmax] : 0.f;
+#pragma unroll
+          for (int t = 0; t < 16; ++t)
+            if (a0 + t < n_a) consider(a0 + t, pv[t]);
+        }
       }
       bool exh = cntc > 4;   // more than four contenders: every new row exactly
       if (!exh) {            // prune against the final bar (order kept: ascending new-row index)
@@ -909,26 +932,38 @@ __global__ void __launch_bounds__(kDecideThreads, PER_SM) fold_decide_kernel(Fol
     if (tid == 0) s_nmerge = nm;
   }
   // ---- E: order merged tokens by (row, token); publish ----
-  {
+  {   // (ranks counted as in the append selection; keys of merged tokens are distinct, the others go last)
     unsigned* ekey = reinterpret_cast<unsigned*>(s_prow);   // (the pair list is idle here)
-    if (tid < nsort) {
+    unsigned* ukey = ekey + 256;                             // unsorted keys
+    if (tid < kMaxBlock) {
       const int pj = tid < C ? s_pi[tid] : -1;
-      unsigned kq = pj >= 0 ? (((unsigned)pj << 9) | (unsigned)tid) : 0xffffffffu;   // rows < 2^23, tokens < 2^9
+      ukey[tid] = pj >= 0 ? (((unsigned)pj << 9) | (unsigned)tid) : 0xffffffffu;   // rows < 2^23, tokens < 2^9
+      ekey[tid] = 0xffffffffu;
+      s_fill[tid] = 0;
       if (tid < C) {
         p.pi[tokBase + tid] = pj;
         p.creator[tokBase + tid] = s_creator[tid];
       }
-      int zero = 0;
-      if (nsort == 128) sort_n<unsigned, 128>(kq, zero, ekey + 256, reinterpret_cast<int*>(s_pval), tid);
-      else sort_n<unsigned, 256>(kq, zero, ekey + 256, reinterpret_cast<int*>(s_pval), tid);
-      ekey[tid] = kq;
-      asm volatile("bar.sync 2, %0;" ::"r"(nsort) : "memory");
-      if (kq != 0xffffffffu) {
-        const int rowq = (int)(kq >> 9);
-        p.sorted[tokBase + tid] = (int)(kq & 511u);
-        const bool head = tid == 0 || (int)(ekey[tid - 1] >> 9) != rowq;
-        if (head && rowq >= m) p.segnew[tokBase + (rowq - (int)m)] = tid;
-      }
+    }
+    __syncthreads();
+    const int j = tid & (kMaxBlock - 1), h = tid / kMaxBlock;
+    const unsigned kj = ukey[j];
+    if (j < C && kj != 0xffffffffu) {
+      const int half_n = (C + 1) / 2, i0 = h * half_n, i1 = min(C, i0 + half_n);
+      int cnt = 0;
+#pragma unroll 4
+      for (int i = i0; i < i1; ++i) cnt += ukey[i] < kj ? 1 : 0;
+      atomicAdd(&s_fill[j], cnt);
+    }
+    __syncthreads();
+    if (tid < C && ukey[tid] != 0xffffffffu) ekey[s_fill[tid]] = ukey[tid];   // ranks 0 .. nmerge-1
+    __syncthreads();
+    const unsigned kq = tid < kMaxBlock ? ekey[tid] : 0xffffffffu;
+    if (kq != 0xffffffffu) {
+      const int rowq = (int)(kq >> 9);
+      p.sorted[tokBase + tid] = (int)(kq & 511u);
+      const bool head = tid == 0 || (int)(ekey[tid - 1] >> 9) != rowq;
+      if (head && rowq >= m) p.segnew[tokBase + (rowq - (int)m)] = tid;
     }
   }
   if (tid == 0) {
