@@ -200,7 +200,7 @@ __device__ __forceinline__ uint4 pack8_sat(const float (&x)[8], int& nsat) {
 
 // Tokens per thread of the 16-byte kernels: all loads of a thread's tokens are issued before the first value
 // is looked at (a thread with one token had 32 bytes in flight, and a CTA lived for 16 tokens).
-constexpr int kIngestTok = 4;
+constexpr int kIngestTok = 2;
 
 __global__ void __launch_bounds__(256) ingest_kv_vec_kernel(
     __half* __restrict__ stK, __half* __restrict__ stV, float* __restrict__ stG, __half* __restrict__ ringK,
