@@ -129,3 +129,26 @@ def test_bounds_first_decisions_head_dim_64_three_sink_rows_duplicated_keys():
     print(_sampled(wl, units, params=params, gate=True, flags=kvm.FLAG_SERIAL_FOLDS))
     wl = synth.Workload("t", 5, 32, 32, 128, 128 * 9 + 3, 128, "fixed", fixed_slots=300, r=32, seed=40, S=2)
     print(_sampled(wl, [(0, 0), (3, 11), (4, 31)], flags=kvm.FLAG_SERIAL_FOLDS))
+
+
+def test_bounds_first_decisions_with_exactly_tied_scores():
+    """More units than SMs, every key of a sequence equal (all similarities tie exactly) or every key repeated in
+    the next block half (ties in pairs): the bounds decide nothing, every token is scored, and appended tokens,
+    rows and merge targets must follow the tie rules (smaller token, lowest row) as in the oracle."""
+    wl = synth.Workload("t", 1, 160, 160, 64, 32 * 9 + 5, 32, "sqrt", sqrt_coeff=3, r=0, seed=41)
+    params = synth.make_layer_params(wl)
+    units = [(0, 0), (0, 80), (0, 159)]
+    tensors = synth.make_inputs(wl)
+    tensors["k"] = torch.full_like(tensors["k"], 0.5)
+    y_gpu, st = pu.run_gpu(wl, tensors, params)
+    y_ref, o = pu.run_oracle(wl, tensors, params, units=units)
+    print(pu.compare(wl, y_gpu, st, y_ref, o, units=units))
+    st.free()
+    tensors = synth.make_inputs(wl)
+    k = tensors["k"]
+    for b0 in range(0, wl.T - 31, 32):   # second half of every block repeats the first half
+        k[:, :, b0 + 16:b0 + 32] = k[:, :, b0:b0 + 16]
+    y_gpu, st = pu.run_gpu(wl, tensors, params)
+    y_ref, o = pu.run_oracle(wl, tensors, params, units=units)
+    print(pu.compare(wl, y_gpu, st, y_ref, o, units=units))
+    st.free()
