@@ -740,12 +740,12 @@ KVM_API kvm_status_t kvm_prefill_host(const void* q_host, const void* k_host, co
   if (!guard.ok) return KVM_ERR_CUDA;
   rc = ensure_host_staging(ks);
   if (rc != KVM_OK) return rc;
-  // The call is cut into up to eight segments of whole blocks; segment i+1 is copied in, and segment
+  // The call is cut into up to eight segments of at least two whole blocks; segment i+1 is copied in, and segment
   // i-1 copied out, while segment i is computed (three streams, the copies as strided 2-D copies into /
   // out of staging buffers that have the host layout [batch, head, token, channel]).
   const int64_t n = n_tokens;
   const int64_t d = s.d;
-  int nseg = (int)(n / (4 * (int64_t)block));
+  int nseg = (int)(n / (2 * (int64_t)block));   // (the last segment's compute and copy-out are not overlapped: keep it short)
   if (nseg > 8) nseg = 8;
   if (nseg < 1) nseg = 1;
   const int64_t seg_len = ((n + nseg - 1) / nseg + block - 1) / block * block;
