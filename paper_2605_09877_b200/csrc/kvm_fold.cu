@@ -1816,9 +1816,9 @@ __global__ void __launch_bounds__(256, 2) fold_apply_rows4_kernel(FoldApplyParam
 #pragma unroll
         for (int i = 0; i < NI; ++i) {
           const int x = 32 * i + 4 * sub;
-          const double2 k01 = *reinterpret_cast<const double2*>(p.sumK + row * D + x), k23 = *reinterpret_cast<const double2*>(p.sumK + row * D + x + 2);
+          const double2 k01 = __ldcs(reinterpret_cast<const double2*>(p.sumK + row * D + x)), k23 = __ldcs(reinterpret_cast<const double2*>(p.sumK + row * D + x + 2));
           kx[4 * i] = k01.x; kx[4 * i + 1] = k01.y; kx[4 * i + 2] = k23.x; kx[4 * i + 3] = k23.y;
-          const float4 v4 = *reinterpret_cast<const float4*>(p.sumV + row * D + x);
+          const float4 v4 = __ldcs(reinterpret_cast<const float4*>(p.sumV + row * D + x));
           vx[4 * i] = v4.x; vx[4 * i + 1] = v4.y; vx[4 * i + 2] = v4.z; vx[4 * i + 3] = v4.w;
         }
         wacc = p.wsum[row];
@@ -1884,11 +1884,11 @@ __global__ void __launch_bounds__(256, 2) fold_apply_rows4_kernel(FoldApplyParam
         kh[e] = __float2half_rn((float)hat);
         vh[e] = __float2half_rn((float)((double)vx[4 * i + e] * vscale));
       }
-      reinterpret_cast<double2*>(p.sumK + row * D + x)[0] = make_double2(kx[4 * i], kx[4 * i + 1]);
-      reinterpret_cast<double2*>(p.sumK + row * D + x)[1] = make_double2(kx[4 * i + 2], kx[4 * i + 3]);
-      *reinterpret_cast<float4*>(p.sumV + row * D + x) = make_float4(vx[4 * i], vx[4 * i + 1], vx[4 * i + 2], vx[4 * i + 3]);
-      *reinterpret_cast<uint2*>(p.Khat + row * D + x) = *reinterpret_cast<const uint2*>(kh);
-      *reinterpret_cast<uint2*>(p.Vhat + row * D + x) = *reinterpret_cast<const uint2*>(vh);
+      __stcs(reinterpret_cast<double2*>(p.sumK + row * D + x), make_double2(kx[4 * i], kx[4 * i + 1]));
+      __stcs(reinterpret_cast<double2*>(p.sumK + row * D + x) + 1, make_double2(kx[4 * i + 2], kx[4 * i + 3]));
+      __stcs(reinterpret_cast<float4*>(p.sumV + row * D + x), make_float4(vx[4 * i], vx[4 * i + 1], vx[4 * i + 2], vx[4 * i + 3]));
+      __stcs(reinterpret_cast<uint2*>(p.Khat + row * D + x), *reinterpret_cast<const uint2*>(kh));
+      __stcs(reinterpret_cast<uint2*>(p.Vhat + row * D + x), *reinterpret_cast<const uint2*>(vh));
     }
     if (sub == 0) {
       p.rho[row] = (float)rad;
