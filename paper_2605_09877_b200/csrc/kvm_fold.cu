@@ -983,9 +983,9 @@ __global__ void __launch_bounds__(kDecideThreads, PER_SM) fold_decide_kernel(Fol
 // of token j lies in [gmax_j - eps_j, gmax_j + eps_j] (eps_j = the bound on the fp16 rounding of its
 // products, half the filter's window), so a token is appended for certain when fewer than n_a others can
 // rank before it, merged for certain when n_a others rank before it for certain, and only the tokens in
-// between are scored exactly (round 1).  A token that is merged for certain with a single candidate row and
+// between are scored exactly (first exact pass).  A token that is merged for certain with a single candidate row and
 // no new row in reach needs no exact similarity at all; the others get their old candidates and the new rows
-// in reach compared exactly in round 2.  The decisions are those of the kernel above bit for bit: the bounds
+// in reach compared exactly in a second exact pass.  The decisions are those of the kernel above bit for bit: the bounds
 // only remove work whose outcome they fix.
 // The products with the rows a small fold appends (n_a <= kGramOnTheFly) run on the tensor cores
 // (mma.sync m16n8k16, fp16 x fp16 -> fp32): tokens x new rows, the new rows' keys in shared memory.
@@ -1159,7 +1159,7 @@ __global__ void __launch_bounds__(kPrunedThreads, 4) fold_decide_pruned_kernel(F
     if (have && !open) s_cls[tid] = may <= n_a - 1 ? SURE_APPEND : (must >= n_a ? SURE_MERGE : UNSURE);
     __syncthreads();
   }
-  // ---- 3: round 1: exact score, best old row of the unsure tokens ----
+  // ---- 3: first exact pass: score and best old row of the unsure tokens ----
   {
     const bool unsure = tid < C && s_cls[tid] == UNSURE;
     bool exh = unsure && s_exh[tid];
@@ -1413,7 +1413,7 @@ __global__ void __launch_bounds__(kPrunedThreads, 4) fold_decide_pruned_kernel(F
     s_ccnt[j] = (unsigned char)min(kept, 5);
   }
   __syncthreads();
-  // ---- 6: round 2: merged tokens whose target is still open: the old candidates of a token without an exact best
+  // ---- 6: second exact pass: merged tokens whose target is still open: the old candidates of a token without an exact best
   //      (unless it has one candidate and no new row in reach), and the new rows in reach ----
   if (tid == 0) s_np = 0;
   {
