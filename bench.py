@@ -188,9 +188,9 @@ def oracle_sample(wl, mode, budget_s=20.0):
         n_units = min(cores, wl.B * wl.Hkv)
         T_s = wl.T
         att, rt = prefill_flops(wl.scaled(B=1, Hq=n_units * (wl.Hq // wl.Hkv), Hkv=n_units), T_s)
-        rate = 3.0e9 * cores   # measured fp64 flop/s of the plain loops on this kind of host; only sizes the sample
+        rate = 1.6e9 * cores   # fp64 flop/s of the plain loops at the long end (3.2e9 on short prefixes); only sizes the sample
         while (att + rt) / rate > budget_s and T_s > 4 * wl.C:
-            T_s //= 2
+            T_s = max(4 * wl.C, int(T_s * 0.75) // (4 * wl.C) * (4 * wl.C))
             att, rt = prefill_flops(wl.scaled(B=1, Hq=n_units * (wl.Hq // wl.Hkv), Hkv=n_units), T_s)
         small = wl.scaled(B=1, Hq=n_units * (wl.Hq // wl.Hkv), Hkv=n_units, T=T_s)
         t = synth.make_inputs(small)
