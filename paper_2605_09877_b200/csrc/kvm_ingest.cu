@@ -176,23 +176,27 @@ __device__ __forceinline__ int rope_partner8(int c8, int r) {
   return ch0 >= r ? ch0 : (ch0 < half ? ch0 + half : ch0 - half);
 }
 
-// Eight values -> eight fp16, clamped; nsat counts the values that did not fit.  A clamped value reads
-// +-65504 afterwards, which no bf16 input converts to exactly (its neighbours are 65280 and 65536), so the
-// packed result is tested first - one SIMD compare per pair - and the values are only looked at one by one
-// when it shows a hit.
+// Eight values -> eight fp16, clamped; nsat counts the values that did not fit.  The conversion itself saturates
+// (cvt.rn.satfinite: a value beyond the fp16 range becomes +-65504, which no bf16 input converts to exactly -
+// its neighbours are 65280 and 65536), so the packed result is tested first - one SIMD compare per pair, which
+// also catches a NaN - and the values are only looked at one by one, and a NaN replaced by -65504 as a plain
+// fmin/fmax clamp would, when it shows a hit.
 __device__ __forceinline__ uint4 pack8_sat(const float (&x)[8], int& nsat) {
   uint4 o;
   uint32_t w[4];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const __half2 h = __floats2half2_rn(fminf(fmaxf(x[2 * i], -65504.f), 65504.f), fminf(fmaxf(x[2 * i + 1], -65504.f), 65504.f));
-    w[i] = *reinterpret_cast<const uint32_t*>(&h);
-  }
-  const uint32_t any = (__vcmpeq2(w[0] & 0x7fff7fffu, 0x7bff7bffu) | __vcmpeq2(w[1] & 0x7fff7fffu, 0x7bff7bffu)) |
-                       (__vcmpeq2(w[2] & 0x7fff7fffu, 0x7bff7bffu) | __vcmpeq2(w[3] & 0x7fff7fffu, 0x7bff7bffu));
+  for (int i = 0; i < 4; ++i)
+    asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(x[2 * i + 1]), "f"(x[2 * i]));   // (first source: upper half)
+  const uint32_t any = (__vcmpgeu2(w[0] & 0x7fff7fffu, 0x7bff7bffu) | __vcmpgeu2(w[1] & 0x7fff7fffu, 0x7bff7bffu)) |
+                       (__vcmpgeu2(w[2] & 0x7fff7fffu, 0x7bff7bffu) | __vcmpgeu2(w[3] & 0x7fff7fffu, 0x7bff7bffu));
   if (any) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) nsat += !(fabsf(x[i]) <= 65504.f) ? 1 : 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __half2 h = __floats2half2_rn(fminf(fmaxf(x[2 * i], -65504.f), 65504.f), fminf(fmaxf(x[2 * i + 1], -65504.f), 65504.f));
+      w[i] = *reinterpret_cast<const uint32_t*>(&h);
+    }
   }
   o.x = w[0]; o.y = w[1]; o.z = w[2]; o.w = w[3];
   return o;
