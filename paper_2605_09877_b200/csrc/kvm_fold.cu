@@ -124,12 +124,16 @@ __global__ void __launch_bounds__(256, RK ? 4 : 2) kbar_kernel(const __half* __r
   const int jj = live ? j : C - 1;    //  the shuffles below need every lane)
   const __half* row = ok + (int64_t)u * unit_stride + ((int64_t)g * C + jj) * D;
   double val[NC];
+  float valf[NC];   // (the same values in fp32, for the launches that need nothing else in fp64)
 #pragma unroll
   for (int i = 0; i < NI; ++i) {
     alignas(8) __half hv[4];
     *reinterpret_cast<uint2*>(hv) = *reinterpret_cast<const uint2*>(row + 32 * i + 4 * sub);
 #pragma unroll
-    for (int e = 0; e < 4; ++e) val[4 * i + e] = (32 * i + 4 * sub + e < r) ? 0.0 : (double)__half2float(hv[e]);
+    for (int e = 0; e < 4; ++e) {
+      valf[4 * i + e] = (32 * i + 4 * sub + e < r) ? 0.f : __half2float(hv[e]);
+      val[4 * i + e] = (double)valf[4 * i + e];
+    }
   }
   double sum = 0.0;
 #pragma unroll
@@ -157,7 +161,7 @@ __global__ void __launch_bounds__(256, RK ? 4 : 2) kbar_kernel(const __half* __r
       alignas(8) __half kh[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
-        const float tf = fmaf(wv[e], ((float)val[4 * i + e] - mean_f) * rstd_f, bv[e]);
+        const float tf = fmaf(wv[e], (valf[4 * i + e] - mean_f) * rstd_f, bv[e]);
         kh[e] = __float2half_rn(tf);
         n2f = fmaf(tf, tf, n2f);
       }
