@@ -183,3 +183,31 @@ def test_many_units_run_to_run_and_across_variants_identical_bits():
         assert np.array_equal(e["sum_k"], outs[0][1][U0:U1]) and np.array_equal(e["sum_v"], outs[0][2][U0:U1])
         assert np.array_equal(e["count"], outs[0][3][U0:U1])
         st.free()
+
+
+_SWEEP = [
+    # (B, Hq, Hkv, d, C, blocks, extra, growth kwargs, r, S, w, kind, flags_serial, gate, decode)
+    (5, 32, 32, 64, 16, 14, 3, dict(growth="sqrt", sqrt_coeff=2), 0, 0, 2, "normal", False, False, 0),
+    (3, 64, 64, 64, 32, 10, 9, dict(growth="fixed", fixed_slots=96), 16, 2, 3, "mixture", True, True, 12),
+    (10, 32, 16, 128, 64, 8, 1, dict(growth="power", sqrt_coeff=6, pow_num=2, pow_den=3), 32, 1, 2, "scaled_keys", False, True, 0),
+    (6, 32, 32, 128, 128, 7, 50, dict(growth="saturating", fixed_slots=400, sat_half=600), 0, 4, 2, "needles", True, False, 20),
+    (20, 8, 8, 64, 64, 9, 0, dict(growth="sqrt", sqrt_coeff=9), 16, 1, 4, "mixture", True, False, 0),
+    (1, 150, 150, 128, 256, 4, 17, dict(growth="sqrt", sqrt_coeff=16), 32, 1, 2, "normal", True, True, 0),
+]
+
+
+@pytest.mark.parametrize("case", range(len(_SWEEP)))
+def test_shape_sweep_with_more_units_than_sms(case):
+    """Seeded sweep over the shapes the many-unit kernels meet: head dimension, block length from 16 to 256, every
+    budget rule, sink rows from 0 to 4, window lengths, grouped queries, gates, rotary dimensions, with and without
+    the serial-fold flag, prefill followed by decode steps; sampled units against the oracle."""
+    from paper_2605_09877_b200 import kvm
+    B, Hq, Hkv, d, C, nb, extra, gk, r, S, w, kind, serial, gate, dec = _SWEEP[case]
+    T = C * nb + extra + dec
+    wl = synth.Workload("sweep", B, Hq, Hkv, d, T, C, r=r, S=S, w=w, seed=100 + case, kind=kind, **gk)
+    assert B * Hkv > 148
+    params = synth.make_layer_params(wl, trivial=(case % 2 == 0))
+    units = [(0, 0), (B // 2, Hkv // 2), (B - 1, Hkv - 1)]
+    stats = _sampled(wl, units, params=params, gate=gate, decode_from=(T - dec) if dec else None,
+                     flags=kvm.FLAG_SERIAL_FOLDS if serial else 0)
+    print(case, stats)
